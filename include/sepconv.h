@@ -1,0 +1,205 @@
+/*
+ * sepconv.h -- C ABI of the B200 (sm_100a) time-channel separable convolution library.
+ *
+ * The library computes the forward and backward pass of the block that makes up a
+ * Jasper/QuartzNet-style convolutional acoustic encoder, the `JasperEncoder` neural module of
+ * the NeMo paper (arXiv 1909.09577, section 4.1.1), whose ports are
+ *     (audio_signal [B, C, T], length [B])  ->  (encoded [B, C', T'], encoded_len [B]).
+ * Tensors are described the way the paper's neural types describe them (section 3.2, Table 1):
+ * every axis carries a semantic tag (batch / channel / time) and a size, and a mismatch is
+ * reported with the same vocabulary (dimension-incompatible, transposed, incompatible).
+ * Precision follows section 3.3: 16-bit (or fp32) activations and convolution weights, fp32
+ * accumulation, statistics, affine parameters and parameter gradients.
+ *
+ * One layer ("block") computes, for x [B, C_in, T_in] and lengths len[b] (in input frames):
+ *     xm = x where t <  len[b], else 0                                   (padding mask)
+ *     u[b,c,t]  = sum_k wd[c,k] * xm[b,c,t*stride + k - (K-1)/2]          (depthwise, zero "same" padding)
+ *     v[b,o,t]  = sum_c wp[o,c] * u[b,c,t]  (+ bias[o])                   (pointwise 1x1)
+ *     len'[b]   = ceil(len[b]/stride);  N = sum_b len'[b]
+ *     mean, var = per-channel moments of v over the N valid frames (biased variance)
+ *     bn        = gamma * (v - mean) / sqrt(var + eps) + beta            (training-mode batch norm)
+ *     r         = 0 | xr (identity) | BN_r(wr * xr)  (projection), xr = residual source masked by len'
+ *     y         = relu(bn + r)           (res_before_relu = 1, the default)
+ *               = relu(bn) + r           (res_before_relu = 0)
+ *     y = 0 for t >= len'[b]
+ * and the exact gradient of that map.  T' = floor((T_in + 2P - K)/stride) + 1 with P = (K-1)/2.
+ *
+ * Conventions common to all calls
+ *   - Every pointer named *_dev or held in an sc_tensor / sc_block_params / sc_block_saved /
+ *     sc_block_grads is a DEVICE pointer owned by the caller; descriptors are HOST structs.
+ *   - Tensors are dense [B, C, T] with time contiguous; base pointers 16-byte aligned.
+ *   - Activations and conv weights (wd, wp, wr) use desc->io_dtype; gamma, beta, bias, the saved
+ *     statistics, running statistics and every parameter gradient are float32.
+ *   - Calls enqueue work on `cuda_stream` and return without synchronising.  The library never
+ *     allocates or frees device memory inside these calls and keeps no pointer past the call.
+ *   - Return value: SC_OK or a negative sc_status.  Nothing throws across the boundary.  Errors
+ *     that only the device can see (a length outside [1, T], a bounded wait that ran out) are
+ *     written to a status word that sepconv_last_status() returns.
+ *   - Results are deterministic: reductions use a fixed order, no floating-point atomics.
+ */
+#ifndef SEPCONV_H_
+#define SEPCONV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sc_ctx sc_ctx;
+
+typedef enum { SC_F32 = 0, SC_F16 = 1, SC_BF16 = 2 } sc_dtype;
+/* semantic axis tags (section 3.2) */
+typedef enum { SC_AX_BATCH = 0, SC_AX_CHANNEL = 1, SC_AX_TIME = 2 } sc_axis;
+typedef enum { SC_RES_NONE = 0, SC_RES_IDENTITY = 1, SC_RES_PROJ = 2 } sc_residual;
+
+typedef enum {
+    SC_OK = 0,
+    SC_ERR_NULL = -1,              /* a required pointer is null                                   */
+    SC_ERR_INCOMPATIBLE = -2,      /* wrong dtype or rank                                          */
+    SC_ERR_DIM_INCOMPATIBLE = -3,  /* an axis size disagrees with the descriptor                   */
+    SC_ERR_TRANSPOSED = -4,        /* right sizes, wrong axis order (e.g. [B,T,C]) or not dense    */
+    SC_ERR_ALIGNMENT = -5,         /* base pointer not 16-byte aligned                             */
+    SC_ERR_UNSUPPORTED = -6,       /* even K, stride not 1|2, illegal residual, ...                */
+    SC_ERR_WORKSPACE = -7,         /* workspace too small or null                                  */
+    SC_ERR_LENGTHS = -8,           /* (device) some length is outside [1, T_in]                    */
+    SC_ERR_DEVICE_TIMEOUT = -9,    /* (device) a bounded wait inside a kernel ran out              */
+    SC_ERR_ARCH = -10,             /* the device is not compute capability 10.x                    */
+    SC_ERR_CUDA = -11              /* a CUDA runtime/driver call failed                            */
+} sc_status;
+
+/* A typed tensor argument: size/stride in elements, tag[i] names axis i. */
+typedef struct {
+    void*   ptr;
+    int32_t dtype;      /* sc_dtype */
+    int32_t rank;       /* must be 3 */
+    int64_t size[3];
+    int64_t stride[3];
+    int32_t tag[3];     /* sc_axis; the library expects {BATCH, CHANNEL, TIME} */
+} sc_tensor;
+
+typedef struct {
+    int32_t B, C_in, C_out, T_in;
+    int32_t K, stride;          /* K odd; stride 1 or 2 (ignored when has_dw = 0)                  */
+    int32_t io_dtype;           /* sc_dtype of activations and conv weights                        */
+    int32_t residual;           /* sc_residual                                                     */
+    int32_t C_res;              /* channels of the residual source (0: same as C_in)               */
+    int32_t has_dw, has_bn, has_relu, has_bias;
+    int32_t res_before_relu;    /* 1: y = relu(bn + r);  0: y = relu(bn) + r                       */
+    float   bn_eps, bn_momentum;
+} sc_block_desc;
+
+typedef struct {          /* device pointers; absent parts may be null                             */
+    const void  *wd;      /* [C_in, K]      io_dtype                                               */
+    const void  *wp;      /* [C_out, C_in]  io_dtype                                               */
+    const float *gamma, *beta;       /* [C_out]                                                    */
+    const float *bias;               /* [C_out]                                                    */
+    const void  *wr;      /* [C_out, C_res] io_dtype                                               */
+    const float *gamma_r, *beta_r;   /* [C_out]                                                    */
+} sc_block_params;
+
+typedef struct {          /* written by sepconv_fwd, read by sepconv_bwd; caller-owned             */
+    void  *u;             /* [B, C_in, T']  io_dtype (has_dw only)                                 */
+    void  *v;             /* [B, C_out, T'] io_dtype (has_bn only)                                 */
+    float *mean, *invstd; /* [C_out]                                                               */
+    void  *vr;            /* [B, C_out, T'] io_dtype (projection residual only)                    */
+    float *mean_r, *invstd_r;
+} sc_block_saved;
+
+typedef struct {          /* float32 parameter gradients, same shapes as the parameters            */
+    float *dwd, *dwp, *dgamma, *dbeta, *dbias, *dwr, *dgamma_r, *dbeta_r;
+} sc_block_grads;
+
+/* Encoder = a fixed list of layers.  res_from[i] = index of the layer whose INPUT feeds layer i's
+ * residual branch (-1: layer i's own input).  B and T_in of layers[0] are the encoder's; the
+ * B/T_in fields of later layers are ignored and derived.  param_offsets / grad_offsets are HOST
+ * arrays of n_layers*8 byte offsets (order: wd, wp, gamma, beta, bias, wr, gamma_r, beta_r; -1 for
+ * an absent parameter) into the caller's flat device blobs. */
+typedef struct {
+    int32_t              n_layers;
+    const sc_block_desc* layers;
+    const int32_t*       res_from;
+} sc_encoder_desc;
+
+/* ---- context ------------------------------------------------------------------------------ */
+
+/* Creates a context on CUDA device `device` (which must be compute capability 10.x) and allocates
+ * the 64-byte device status word -- the only device allocation the library ever makes.
+ * Returns SC_ERR_ARCH on any other architecture. */
+int  sepconv_ctx_create(sc_ctx** out, int device);
+void sepconv_ctx_destroy(sc_ctx* ctx);
+
+/* Synchronises `cuda_stream`, returns the device status word (SC_OK, SC_ERR_LENGTHS or
+ * SC_ERR_DEVICE_TIMEOUT) and clears it. */
+int  sepconv_last_status(sc_ctx* ctx, void* cuda_stream);
+const char* sepconv_strerror(int status);
+
+/* ---- one block ---------------------------------------------------------------------------- */
+
+/* Bytes of scratch the two block calls need for this descriptor (host-only computation). */
+int  sepconv_workspace_bytes(const sc_block_desc* desc, size_t* fwd_bytes, size_t* bwd_bytes);
+
+/* Forward of one block (definition at the top of this file).
+ *   x              [B, C_in, T_in]
+ *   x_res          residual source [B, C_res, T']; null = x (requires stride 1)
+ *   lengths_dev    int32 [B], valid input frames, each in [1, T_in]
+ *   y              [B, C_out, T'] (written, zero in padded frames)
+ *   out_lengths_dev int32 [B] <- len' (nullable)
+ *   saved          intermediates for the backward pass (see sc_block_saved)
+ *   running_mean/var  float32 [C_out], updated in place with bn_momentum (nullable)
+ */
+int  sepconv_fwd(sc_ctx* ctx, const sc_block_desc* desc,
+                 const sc_tensor* x, const sc_tensor* x_res, const int32_t* lengths_dev,
+                 const sc_block_params* params, sc_tensor* y, int32_t* out_lengths_dev,
+                 sc_block_saved* saved, float* running_mean, float* running_var,
+                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Backward of one block: the exact adjoint of sepconv_fwd.
+ *   dy       upstream gradient [B, C_out, T'] (values in padded frames are ignored)
+ *   x, x_res, y, lengths_dev, params, saved: as given to / produced by sepconv_fwd
+ *   dx       [B, C_in, T_in]  <- gradient w.r.t. x (zero in padded frames)
+ *   dx_res   [B, C_res, T']   <- gradient w.r.t. x_res; null = the residual path's gradient is
+ *            added into dx (only legal when the residual source is x)
+ *   dx_add   optional [B, C_in, T_in] tensor added into dx before rounding (a gradient that
+ *            reaches the same input along another path)
+ *   grads    parameter gradients, float32; accumulate != 0 adds into them instead of overwriting
+ *            (gradient accumulation, section 3.3)
+ */
+int  sepconv_bwd(sc_ctx* ctx, const sc_block_desc* desc,
+                 const sc_tensor* dy, const sc_tensor* x, const sc_tensor* x_res, const sc_tensor* y,
+                 const int32_t* lengths_dev, const sc_block_params* params,
+                 const sc_block_saved* saved,
+                 sc_tensor* dx, sc_tensor* dx_res, const sc_tensor* dx_add,
+                 sc_block_grads* grads, int accumulate,
+                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ---- whole encoder -------------------------------------------------------------------------- */
+
+int  encoder_workspace_bytes(const sc_encoder_desc* desc, size_t* bytes);
+
+/* Forward through every layer, then backward from `dlogits`, in one call.
+ *   x [B, C_0, T_in], lengths_dev int32 [B]
+ *   params_blob / grads_blob: flat device blobs addressed by param_offsets / grad_offsets
+ *   dlogits [B, C_last, T_last] upstream gradient; logits [B, C_last, T_last] (written)
+ *   out_lengths_dev int32 [B] <- encoded lengths;  dx (nullable) <- gradient w.r.t. x
+ * All per-layer intermediates live in `workspace`.
+ */
+int  encoder_fwd_bwd(sc_ctx* ctx, const sc_encoder_desc* desc,
+                     const sc_tensor* x, const int32_t* lengths_dev,
+                     const void* params_blob, const int64_t* param_offsets,
+                     const sc_tensor* dlogits, sc_tensor* logits, int32_t* out_lengths_dev,
+                     void* grads_blob, const int64_t* grad_offsets, sc_tensor* dx,
+                     int accumulate, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Selects the kernel family for the pointwise contractions: 0 = automatic (tensor cores where
+ * the shape allows), 1 = force the plain fp32-accumulate SIMT kernels.  Used by tests. */
+int  sepconv_set_gemm_mode(sc_ctx* ctx, int mode);
+
+/* Number of kernel launches this context has enqueued so far (for reporting). */
+int64_t sepconv_launch_count(sc_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SEPCONV_H_ */

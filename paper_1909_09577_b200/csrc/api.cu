@@ -1,0 +1,612 @@
+// C-ABI layer: argument validation, workspace planning and the launch sequence of one block and of
+// the whole encoder.  All arithmetic lives in the kernel files; this file only orders launches.
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/sepconv.h"
+#include "common.cuh"
+#include "kernels.h"
+#include "tc_gemm.h"
+
+using namespace sc;
+
+struct sc_ctx {
+    int device = 0;
+    int sm_count = 0;
+    int* status_dev = nullptr;
+    int64_t launches = 0;
+    int gemm_mode = 0;
+    TcState tc;
+};
+
+namespace {
+
+size_t esize(int dtype) { return dtype == SC_F32 ? 4 : 2; }
+
+// Bump allocator over the caller's workspace; with base == nullptr it only measures.
+struct Bump {
+    char* base; size_t off = 0, cap;
+    Bump(void* b, size_t c) : base((char*)b), cap(c) {}
+    void* take(size_t bytes) {
+        size_t o = (off + 255) & ~(size_t)255;
+        off = o + bytes;
+        return base ? base + o : nullptr;
+    }
+    bool ok() const { return base == nullptr || off <= cap; }
+};
+
+struct Dims { int B, Cin, Cout, Cres, T, Tp, K, s; };
+
+int desc_dims(const sc_block_desc* d, Dims* o) {
+    if (!d) return SC_ERR_NULL;
+    if (d->io_dtype < 0 || d->io_dtype > 2) return SC_ERR_INCOMPATIBLE;
+    if (d->B < 1 || d->C_in < 1 || d->C_out < 1 || d->T_in < 1) return SC_ERR_DIM_INCOMPATIBLE;
+    o->B = d->B; o->Cin = d->C_in; o->Cout = d->C_out; o->T = d->T_in;
+    o->K = d->has_dw ? d->K : 1; o->s = d->has_dw ? d->stride : 1;
+    if (o->K < 1 || (o->K & 1) == 0) return SC_ERR_UNSUPPORTED;
+    if (o->s != 1 && o->s != 2) return SC_ERR_UNSUPPORTED;
+    const int P = (o->K - 1) / 2;
+    o->Tp = (o->T + 2 * P - o->K) / o->s + 1;
+    o->Cres = d->C_res > 0 ? d->C_res : d->C_in;
+    if (d->residual < 0 || d->residual > 2) return SC_ERR_UNSUPPORTED;
+    if (d->residual == SC_RES_IDENTITY && o->Cres != o->Cout) return SC_ERR_UNSUPPORTED;
+    if (d->residual != SC_RES_NONE && !d->has_bn) return SC_ERR_UNSUPPORTED;
+    if (!d->has_bn && d->has_relu) return SC_ERR_UNSUPPORTED;
+    if (d->has_bn && d->has_bias) return SC_ERR_UNSUPPORTED;   // a bias before batch norm cancels
+    return SC_OK;
+}
+
+int check_tensor(const sc_tensor* t, int dtype, int64_t B, int64_t C, int64_t T) {
+    if (!t || !t->ptr) return SC_ERR_NULL;
+    if (t->dtype != dtype || t->rank != 3) return SC_ERR_INCOMPATIBLE;
+    const int64_t want[3] = {B, C, T};
+    const int wtag[3] = {SC_AX_BATCH, SC_AX_CHANNEL, SC_AX_TIME};
+    bool tags_ok = true, sizes_ok = true;
+    for (int i = 0; i < 3; ++i) { tags_ok &= (t->tag[i] == wtag[i]); sizes_ok &= (t->size[i] == want[i]); }
+    if (!tags_ok) {
+        // same axes in another order -> transposed; otherwise not a [batch, channel, time] tensor
+        int seen = 0;
+        for (int i = 0; i < 3; ++i) if (t->tag[i] >= 0 && t->tag[i] <= 2) seen |= 1 << t->tag[i];
+        return seen == 7 ? SC_ERR_TRANSPOSED : SC_ERR_INCOMPATIBLE;
+    }
+    if (!sizes_ok) return SC_ERR_DIM_INCOMPATIBLE;
+    if (t->stride[2] != 1 || t->stride[1] != T || t->stride[0] != C * T) return SC_ERR_TRANSPOSED;
+    if (((uintptr_t)t->ptr & 15) != 0) return SC_ERR_ALIGNMENT;
+    return SC_OK;
+}
+
+struct BlockIO {                 // raw pointers after validation
+    const void* x; const void* xres; void* y;
+    const int* len_in; int* len_out; int* nvalid;
+    bool x_clean, res_clean;     // inputs known to be zero in padded frames
+    bool lengths_ready;          // len_out / nvalid already computed
+};
+
+// ---- forward scratch ---------------------------------------------------------------------------
+struct FwdScratch { float2 *partials, *ss, *ss_r; void* xr; int* len_out; int* nvalid; };
+
+void plan_fwd(const sc_block_desc* d, const Dims& m, Bump& ws, FwdScratch* f, const TcState* tc) {
+    const size_t parts = (size_t)m.B * tc_max_parts_per_sample(m.Tp) * m.Cout;
+    f->len_out = (int*)ws.take(sizeof(int) * m.B);
+    f->nvalid = (int*)ws.take(sizeof(int));
+    f->partials = (float2*)ws.take(sizeof(float2) * parts);
+    f->ss = (float2*)ws.take(sizeof(float2) * m.Cout);
+    f->ss_r = (float2*)ws.take(sizeof(float2) * m.Cout);
+    f->xr = (d->residual == SC_RES_PROJ) ? ws.take(esize(d->io_dtype) * m.B * m.Cres * m.Tp) : nullptr;
+}
+
+// v = w * u for every sample, plus masked batch statistics -> mean/invstd/scale-shift.
+void pointwise_bn(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const Dims& m, int Cin,
+                  const void* w, const void* u, void* v, const int* len_out, const int* nvalid,
+                  const float* gamma, const float* beta, float* mean, float* invstd, float2* ss,
+                  float2* partials, float* rmean, float* rvar) {
+    int parts = 1, tile_w = m.Tp;
+    bool fused = false;
+    if (ctx->gemm_mode == 0 && tc_fwd_supported(&ctx->tc, d->io_dtype, Cin, m.Cout, m.Tp)) {
+        fused = tc_gemm_fwd(&ctx->tc, L, d->io_dtype, w, u, nullptr, v, len_out, m.B, Cin, m.Cout, m.Tp,
+                            partials, &parts, &tile_w);
+    } else {
+        gemm_fwd_simt(L, d->io_dtype, w, u, nullptr, v, len_out, m.B, Cin, m.Cout, m.Tp);
+    }
+    if (!fused) { bn_stats(L, d->io_dtype, v, len_out, m.B, m.Cout, m.Tp, partials); parts = 1; tile_w = m.Tp; }
+    bn_finalize(L, partials, parts, tile_w, len_out, nvalid, m.B, m.Cout, gamma, beta, d->bn_eps,
+                d->bn_momentum, mean, invstd, ss, rmean, rvar);
+}
+
+int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const Dims& m, BlockIO io,
+                   const sc_block_params* p, sc_block_saved* sv, float* rmean, float* rvar,
+                   const FwdScratch& f) {
+    const int dt = d->io_dtype;
+    if (!io.lengths_ready) lengths(L, io.len_in, m.B, m.T, m.s, io.len_out, io.nvalid);
+    const void* u;
+    if (d->has_dw) {
+        dw_fwd(L, dt, io.x, p->wd, sv->u, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s);
+        u = sv->u;
+    } else if (io.x_clean) {
+        u = io.x;
+    } else {
+        mask_copy(L, dt, sv->u, io.x, io.len_in, m.B, m.Cin, m.T);
+        u = sv->u;
+    }
+    if (!d->has_bn) {   // linear layer: y = mask * (w u + bias)
+        if (ctx->gemm_mode == 0 && tc_fwd_supported(&ctx->tc, dt, m.Cin, m.Cout, m.Tp)) {
+            int parts, tw;
+            tc_gemm_fwd(&ctx->tc, L, dt, p->wp, u, d->has_bias ? p->bias : nullptr, io.y, io.len_out, m.B, m.Cin,
+                        m.Cout, m.Tp, nullptr, &parts, &tw);
+        } else {
+            gemm_fwd_simt(L, dt, p->wp, u, d->has_bias ? p->bias : nullptr, io.y, io.len_out, m.B, m.Cin, m.Cout, m.Tp);
+        }
+        return SC_OK;
+    }
+    pointwise_bn(ctx, L, d, m, m.Cin, p->wp, u, sv->v, io.len_out, io.nvalid, p->gamma, p->beta, sv->mean,
+                 sv->invstd, f.ss, f.partials, rmean, rvar);
+    ApplyArgs a{};
+    a.v = sv->v; a.ss = f.ss; a.residual = d->residual; a.y = io.y; a.len_out = io.len_out;
+    a.B = m.B; a.C = m.Cout; a.Tp = m.Tp; a.has_relu = d->has_relu; a.res_before_relu = d->res_before_relu;
+    if (d->residual == SC_RES_IDENTITY) a.xres = io.xres;
+    if (d->residual == SC_RES_PROJ) {
+        const void* xr = io.xres;
+        if (!io.res_clean) { mask_copy(L, dt, f.xr, io.xres, io.len_out, m.B, m.Cres, m.Tp); xr = f.xr; }
+        pointwise_bn(ctx, L, d, m, m.Cres, p->wr, xr, sv->vr, io.len_out, io.nvalid, p->gamma_r, p->beta_r,
+                     sv->mean_r, sv->invstd_r, f.ss_r, f.partials, nullptr, nullptr);
+        a.vr = sv->vr; a.ss_r = f.ss_r;
+    }
+    bn_apply(L, dt, a);
+    return SC_OK;
+}
+
+// ---- backward scratch --------------------------------------------------------------------------
+struct BwdScratch {
+    int* len_out; int* nvalid;
+    float4 *partials, *coef, *coef_r; float2* ss;
+    void *gv, *gvr, *gres, *gu, *gxr, *xr;
+    float* wpart; size_t wpart_bytes;
+};
+
+void plan_bwd(const sc_block_desc* d, const Dims& m, Bump& ws, BwdScratch* s, const TcState* tc) {
+    const size_t e = esize(d->io_dtype);
+    const size_t act_out = e * m.B * m.Cout * m.Tp, act_in = e * m.B * m.Cin * m.Tp;
+    s->len_out = (int*)ws.take(sizeof(int) * m.B);
+    s->nvalid = (int*)ws.take(sizeof(int));
+    s->partials = (float4*)ws.take(sizeof(float4) * m.B * m.Cout);
+    s->coef = (float4*)ws.take(sizeof(float4) * m.Cout);
+    s->coef_r = (float4*)ws.take(sizeof(float4) * m.Cout);
+    s->ss = (float2*)ws.take(sizeof(float2) * m.Cout);
+    s->gv = ws.take(act_out);
+    s->gvr = d->residual == SC_RES_PROJ ? ws.take(act_out) : nullptr;
+    s->gres = d->residual == SC_RES_IDENTITY ? ws.take(act_out) : nullptr;
+    s->gu = ws.take(act_in);
+    s->gxr = d->residual == SC_RES_PROJ ? ws.take(e * m.B * m.Cres * m.Tp) : nullptr;
+    s->xr = d->residual == SC_RES_PROJ ? ws.take(e * m.B * m.Cres * m.Tp) : nullptr;
+    size_t wb = gemm_wgrad_simt_scratch_bytes(m.B, std::max(m.Cin, m.Cres), m.Cout);
+    wb = std::max(wb, tc_wgrad_scratch_bytes(tc, std::max(m.Cin, m.Cres), m.Cout));
+    wb = std::max(wb, dw_wgrad_scratch_bytes(m.B, m.Cin, m.K));
+    s->wpart = (float*)ws.take(wb);
+    s->wpart_bytes = wb;
+}
+
+void pointwise_wgrad(sc_ctx* ctx, const Launch& L, int dt, const void* gv, const void* u, float* dw,
+                     float* part, int acc, int B, int Cin, int Cout, int Tp, const int* len_out) {
+    if (ctx->gemm_mode == 0 && tc_wgrad_supported(&ctx->tc, dt, Cin, Cout, Tp))
+        tc_gemm_wgrad(&ctx->tc, L, dt, gv, u, dw, part, acc, B, Cin, Cout, Tp, len_out);
+    else
+        gemm_wgrad_simt(L, dt, gv, u, dw, part, acc, B, Cin, Cout, Tp);
+}
+void pointwise_dgrad(sc_ctx* ctx, const Launch& L, int dt, const void* w, const void* gv, void* gu, int B,
+                     int Cin, int Cout, int Tp, const int* len_out) {
+    if (ctx->gemm_mode == 0 && tc_dgrad_supported(&ctx->tc, dt, Cin, Cout, Tp))
+        tc_gemm_dgrad(&ctx->tc, L, dt, w, gv, gu, B, Cin, Cout, Tp, len_out);
+    else
+        gemm_dgrad_simt(L, dt, w, gv, gu, B, Cin, Cout, Tp);
+}
+
+struct BwdIO {
+    const void *dy, *x, *xres, *y;
+    void *dx, *dx_res; const void* dx_add;
+    const int* len_in; const int* len_out; const int* nvalid;
+    bool x_clean, res_clean;
+};
+
+int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const Dims& m, BwdIO io,
+                   const sc_block_params* p, const sc_block_saved* sv, sc_block_grads* g, int acc,
+                   const BwdScratch& s) {
+    const int dt = d->io_dtype;
+    BnBwdArgs a{};
+    a.g = io.dy; a.y = io.y; a.v = sv->v; a.vr = sv->vr;
+    a.mean = sv->mean; a.invstd = sv->invstd; a.mean_r = sv->mean_r; a.invstd_r = sv->invstd_r;
+    a.ss = s.ss; a.len_out = io.len_out; a.nvalid = io.nvalid;
+    a.B = m.B; a.C = m.Cout; a.Tp = m.Tp; a.has_bn = d->has_bn; a.has_relu = d->has_relu;
+    a.res_before_relu = d->res_before_relu; a.residual = d->residual;
+    a.partials = s.partials; a.coef = s.coef; a.coef_r = s.coef_r;
+    a.gv = s.gv; a.gvr = s.gvr;
+    // identity residual: its gradient is the gated upstream gradient itself
+    a.gres = (d->residual == SC_RES_IDENTITY) ? (io.dx_res ? io.dx_res : s.gres) : nullptr;
+    if (d->has_bn && d->has_relu && !d->res_before_relu)
+        bn_scale_shift(L, sv->mean, sv->invstd, p->gamma, p->beta, s.ss, m.Cout);
+    bn_bwd_reduce(L, dt, a);
+    bn_bwd_finalize(L, a, p->gamma, p->gamma_r, g->dgamma, g->dbeta, g->dgamma_r, g->dbeta_r,
+                    d->has_bias ? g->dbias : nullptr, acc);
+    bn_bwd_apply(L, dt, a);
+
+    const void* u = d->has_dw ? sv->u : (io.x_clean ? io.x : sv->u);
+    pointwise_wgrad(ctx, L, dt, s.gv, u, g->dwp, s.wpart, acc, m.B, m.Cin, m.Cout, m.Tp, io.len_out);
+
+    const void* extra = nullptr;    // residual-path gradient to fold into dx
+    if (d->residual == SC_RES_PROJ) {
+        const void* xr = io.xres;
+        if (!io.res_clean) { mask_copy(L, dt, s.xr, io.xres, io.len_out, m.B, m.Cres, m.Tp); xr = s.xr; }
+        pointwise_wgrad(ctx, L, dt, s.gvr, xr, g->dwr, s.wpart, acc, m.B, m.Cres, m.Cout, m.Tp, io.len_out);
+        void* tgt = io.dx_res ? io.dx_res : s.gxr;
+        if (io.dx_res || io.dx) pointwise_dgrad(ctx, L, dt, p->wr, s.gvr, tgt, m.B, m.Cres, m.Cout, m.Tp, io.len_out);
+        if (!io.dx_res) extra = s.gxr;
+    } else if (d->residual == SC_RES_IDENTITY && !io.dx_res) {
+        extra = s.gres;
+    }
+
+    if (d->has_dw) {
+        pointwise_dgrad(ctx, L, dt, p->wp, s.gv, s.gu, m.B, m.Cin, m.Cout, m.Tp, io.len_out);
+        dw_wgrad(L, dt, s.gu, io.x, g->dwd, s.wpart, acc, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s);
+        if (io.dx)
+            dw_dgrad(L, dt, s.gu, p->wd, io.dx, io.dx_add, extra, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s);
+    } else if (io.dx) {
+        if (!io.dx_add && !extra) {
+            pointwise_dgrad(ctx, L, dt, p->wp, s.gv, io.dx, m.B, m.Cin, m.Cout, m.Tp, io.len_out);
+        } else {
+            pointwise_dgrad(ctx, L, dt, p->wp, s.gv, s.gu, m.B, m.Cin, m.Cout, m.Tp, io.len_out);
+            ew_add_masked(L, dt, io.dx, s.gu, io.dx_add, extra, io.len_in, m.B, m.Cin, m.T);
+        }
+    }
+    return SC_OK;
+}
+
+int check_params(const sc_block_desc* d, const sc_block_params* p) {
+    if (!p || !p->wp) return SC_ERR_NULL;
+    if (d->has_dw && !p->wd) return SC_ERR_NULL;
+    if (d->has_bn && (!p->gamma || !p->beta)) return SC_ERR_NULL;
+    if (d->has_bias && !p->bias) return SC_ERR_NULL;
+    if (d->residual == SC_RES_PROJ && (!p->wr || !p->gamma_r || !p->beta_r)) return SC_ERR_NULL;
+    return SC_OK;
+}
+int check_saved(const sc_block_desc* d, const sc_block_saved* s, bool x_clean) {
+    if (!s) return SC_ERR_NULL;
+    if ((d->has_dw || !x_clean) && !s->u) return SC_ERR_NULL;
+    if (d->has_bn && (!s->v || !s->mean || !s->invstd)) return SC_ERR_NULL;
+    if (d->residual == SC_RES_PROJ && (!s->vr || !s->mean_r || !s->invstd_r)) return SC_ERR_NULL;
+    return SC_OK;
+}
+int check_grads(const sc_block_desc* d, const sc_block_grads* g) {
+    if (!g || !g->dwp) return SC_ERR_NULL;
+    if (d->has_dw && !g->dwd) return SC_ERR_NULL;
+    if (d->has_bn && (!g->dgamma || !g->dbeta)) return SC_ERR_NULL;
+    if (d->has_bias && !g->dbias) return SC_ERR_NULL;
+    if (d->residual == SC_RES_PROJ && (!g->dwr || !g->dgamma_r || !g->dbeta_r)) return SC_ERR_NULL;
+    return SC_OK;
+}
+
+int finish(sc_ctx* ctx) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { fprintf(stderr, "sepconv: CUDA error: %s\n", cudaGetErrorString(e)); return SC_ERR_CUDA; }
+    (void)ctx;
+    return SC_OK;
+}
+
+#define SC_TRY(expr) do { int _r = (expr); if (_r != SC_OK) return _r; } while (0)
+
+}  // namespace
+
+// =================================================================================================
+extern "C" {
+
+int sepconv_ctx_create(sc_ctx** out, int device) {
+    if (!out) return SC_ERR_NULL;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return SC_ERR_CUDA;
+    if (prop.major != 10) return SC_ERR_ARCH;
+    if (cudaSetDevice(device) != cudaSuccess) return SC_ERR_CUDA;
+    sc_ctx* c = new (std::nothrow) sc_ctx();
+    if (!c) return SC_ERR_CUDA;
+    c->device = device;
+    c->sm_count = prop.multiProcessorCount;
+    if (cudaMalloc(&c->status_dev, 64) != cudaSuccess) { delete c; return SC_ERR_CUDA; }
+    cudaMemset(c->status_dev, 0, 64);
+    int r = tc_init(&c->tc, device, c->sm_count);
+    if (r != SC_OK) { cudaFree(c->status_dev); delete c; return r; }
+    *out = c;
+    return SC_OK;
+}
+
+void sepconv_ctx_destroy(sc_ctx* ctx) {
+    if (!ctx) return;
+    cudaFree(ctx->status_dev);
+    delete ctx;
+}
+
+int sepconv_last_status(sc_ctx* ctx, void* stream) {
+    if (!ctx) return SC_ERR_NULL;
+    int h = 0;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(&h, ctx->status_dev, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return SC_ERR_CUDA;
+    if (cudaMemsetAsync(ctx->status_dev, 0, sizeof(int), st) != cudaSuccess) return SC_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SC_ERR_CUDA;
+    return h;
+}
+
+const char* sepconv_strerror(int s) {
+    switch (s) {
+        case SC_OK: return "ok";
+        case SC_ERR_NULL: return "a required pointer is null";
+        case SC_ERR_INCOMPATIBLE: return "incompatible tensor type (dtype, rank or axis tags)";
+        case SC_ERR_DIM_INCOMPATIBLE: return "an axis size disagrees with the descriptor";
+        case SC_ERR_TRANSPOSED: return "axes are transposed or the tensor is not dense [batch, channel, time]";
+        case SC_ERR_ALIGNMENT: return "pointer is not 16-byte aligned";
+        case SC_ERR_UNSUPPORTED: return "unsupported block configuration";
+        case SC_ERR_WORKSPACE: return "workspace is null or too small";
+        case SC_ERR_LENGTHS: return "a length lies outside [1, T]";
+        case SC_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+        case SC_ERR_ARCH: return "device is not compute capability 10.x";
+        case SC_ERR_CUDA: return "a CUDA call failed";
+        default: return "unknown status";
+    }
+}
+
+int sepconv_set_gemm_mode(sc_ctx* ctx, int mode) {
+    if (!ctx) return SC_ERR_NULL;
+    if (mode != 0 && mode != 1) return SC_ERR_UNSUPPORTED;
+    ctx->gemm_mode = mode;
+    return SC_OK;
+}
+
+int64_t sepconv_launch_count(sc_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int sepconv_workspace_bytes(const sc_block_desc* desc, size_t* fwd, size_t* bwd) {
+    Dims m;
+    SC_TRY(desc_dims(desc, &m));
+    if (fwd) { Bump b(nullptr, 0); FwdScratch f; plan_fwd(desc, m, b, &f, nullptr); *fwd = b.off + 256; }
+    if (bwd) { Bump b(nullptr, 0); BwdScratch s; plan_bwd(desc, m, b, &s, nullptr); *bwd = b.off + 256; }
+    return SC_OK;
+}
+
+int sepconv_fwd(sc_ctx* ctx, const sc_block_desc* desc, const sc_tensor* x, const sc_tensor* x_res,
+                const int32_t* lengths_dev, const sc_block_params* params, sc_tensor* y,
+                int32_t* out_lengths_dev, sc_block_saved* saved, float* running_mean, float* running_var,
+                void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!ctx || !lengths_dev) return SC_ERR_NULL;
+    Dims m;
+    SC_TRY(desc_dims(desc, &m));
+    const int dt = desc->io_dtype;
+    SC_TRY(check_tensor(x, dt, m.B, m.Cin, m.T));
+    SC_TRY(check_tensor(y, dt, m.B, m.Cout, m.Tp));
+    if (desc->residual != SC_RES_NONE) {
+        if (x_res) SC_TRY(check_tensor(x_res, dt, m.B, m.Cres, m.Tp));
+        else if (m.s != 1 || m.Cres != m.Cin) return SC_ERR_UNSUPPORTED;
+    }
+    SC_TRY(check_params(desc, params));
+    SC_TRY(check_saved(desc, saved, false));
+    if (!workspace) return SC_ERR_WORKSPACE;
+    Bump ws(workspace, workspace_bytes);
+    FwdScratch f;
+    plan_fwd(desc, m, ws, &f, &ctx->tc);
+    if (!ws.ok()) return SC_ERR_WORKSPACE;
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches};
+    BlockIO io{};
+    io.x = x->ptr; io.xres = desc->residual != SC_RES_NONE ? (x_res ? x_res->ptr : x->ptr) : nullptr;
+    io.y = y->ptr; io.len_in = lengths_dev; io.len_out = f.len_out; io.nvalid = f.nvalid;
+    io.x_clean = false; io.res_clean = false; io.lengths_ready = false;
+    SC_TRY(block_fwd_impl(ctx, L, desc, m, io, params, saved, running_mean, running_var, f));
+    if (out_lengths_dev)
+        cudaMemcpyAsync(out_lengths_dev, f.len_out, sizeof(int) * m.B, cudaMemcpyDeviceToDevice, L.stream);
+    return finish(ctx);
+}
+
+int sepconv_bwd(sc_ctx* ctx, const sc_block_desc* desc, const sc_tensor* dy, const sc_tensor* x,
+                const sc_tensor* x_res, const sc_tensor* y, const int32_t* lengths_dev,
+                const sc_block_params* params, const sc_block_saved* saved, sc_tensor* dx,
+                sc_tensor* dx_res, const sc_tensor* dx_add, sc_block_grads* grads, int accumulate,
+                void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!ctx || !lengths_dev) return SC_ERR_NULL;
+    Dims m;
+    SC_TRY(desc_dims(desc, &m));
+    const int dt = desc->io_dtype;
+    SC_TRY(check_tensor(dy, dt, m.B, m.Cout, m.Tp));
+    SC_TRY(check_tensor(x, dt, m.B, m.Cin, m.T));
+    SC_TRY(check_tensor(y, dt, m.B, m.Cout, m.Tp));
+    SC_TRY(check_tensor(dx, dt, m.B, m.Cin, m.T));
+    if (dx_add) SC_TRY(check_tensor(dx_add, dt, m.B, m.Cin, m.T));
+    if (desc->residual != SC_RES_NONE) {
+        if (x_res) SC_TRY(check_tensor(x_res, dt, m.B, m.Cres, m.Tp));
+        else if (m.s != 1 || m.Cres != m.Cin) return SC_ERR_UNSUPPORTED;
+        if (dx_res) SC_TRY(check_tensor(dx_res, dt, m.B, m.Cres, m.Tp));
+        else if (m.s != 1 || m.Cres != m.Cin) return SC_ERR_UNSUPPORTED;
+    }
+    SC_TRY(check_params(desc, params));
+    SC_TRY(check_saved(desc, saved, false));
+    SC_TRY(check_grads(desc, grads));
+    if (!workspace) return SC_ERR_WORKSPACE;
+    Bump ws(workspace, workspace_bytes);
+    BwdScratch s;
+    plan_bwd(desc, m, ws, &s, &ctx->tc);
+    if (!ws.ok()) return SC_ERR_WORKSPACE;
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches};
+    lengths(L, lengths_dev, m.B, m.T, m.s, s.len_out, s.nvalid);
+    BwdIO io{};
+    io.dy = dy->ptr; io.x = x->ptr; io.y = y->ptr;
+    io.xres = desc->residual != SC_RES_NONE ? (x_res ? x_res->ptr : x->ptr) : nullptr;
+    io.dx = dx->ptr; io.dx_res = (desc->residual != SC_RES_NONE && dx_res) ? dx_res->ptr : nullptr;
+    io.dx_add = dx_add ? dx_add->ptr : nullptr;
+    io.len_in = lengths_dev; io.len_out = s.len_out; io.nvalid = s.nvalid;
+    io.x_clean = false; io.res_clean = false;
+    SC_TRY(block_bwd_impl(ctx, L, desc, m, io, params, saved, grads, accumulate, s));
+    return finish(ctx);
+}
+
+// ---- encoder ---------------------------------------------------------------------------------
+namespace {
+struct LayerPlan {
+    sc_block_desc d; Dims m;
+    sc_block_saved sv; void* y; int* len_out; int* nvalid;
+    bool own_lengths;
+};
+struct EncPlan {
+    std::vector<LayerPlan> L;
+    void* gbuf[2]; void* pending;
+    size_t bytes;
+    size_t scratch_mark;           // offset where the shared per-layer scratch starts
+};
+
+int plan_encoder(const sc_encoder_desc* e, void* base, size_t cap, EncPlan* P, const TcState* tc) {
+    if (!e || !e->layers || e->n_layers < 1) return SC_ERR_NULL;
+    Bump ws(base, cap);
+    P->L.resize(e->n_layers);
+    int B = e->layers[0].B, T = e->layers[0].T_in, C = e->layers[0].C_in;
+    size_t max_act = 0, max_res = 0;
+    for (int i = 0; i < e->n_layers; ++i) {
+        LayerPlan& lp = P->L[i];
+        lp.d = e->layers[i];
+        lp.d.B = B; lp.d.T_in = T;
+        if (lp.d.C_in != C) return SC_ERR_DIM_INCOMPATIBLE;
+        if (lp.d.io_dtype != e->layers[0].io_dtype) return SC_ERR_INCOMPATIBLE;
+        if (lp.d.residual != SC_RES_NONE) {
+            int j = e->res_from ? e->res_from[i] : -1;
+            if (j < 0) j = i;
+            if (j > i) return SC_ERR_UNSUPPORTED;
+            lp.d.C_res = e->layers[j].C_in;
+        }
+        SC_TRY(desc_dims(&lp.d, &lp.m));
+        const Dims& m = lp.m;
+        const size_t es = esize(lp.d.io_dtype);
+        if (lp.d.residual != SC_RES_NONE) {
+            int j = (e->res_from && e->res_from[i] >= 0) ? e->res_from[i] : i;
+            if (P->L[j].m.T != m.Tp) return SC_ERR_UNSUPPORTED;
+            max_res = std::max(max_res, es * m.B * m.Cres * m.Tp);
+        }
+        lp.own_lengths = (i == 0) || (m.s != 1);
+        if (lp.own_lengths) { lp.len_out = (int*)ws.take(sizeof(int) * B); lp.nvalid = (int*)ws.take(sizeof(int)); }
+        else { lp.len_out = P->L[i - 1].len_out; lp.nvalid = P->L[i - 1].nvalid; }
+        memset(&lp.sv, 0, sizeof(lp.sv));
+        if (lp.d.has_dw) lp.sv.u = ws.take(es * B * m.Cin * m.Tp);
+        else if (i == 0) lp.sv.u = ws.take(es * B * m.Cin * m.Tp);
+        if (lp.d.has_bn) {
+            lp.sv.v = ws.take(es * B * m.Cout * m.Tp);
+            lp.sv.mean = (float*)ws.take(4 * m.Cout); lp.sv.invstd = (float*)ws.take(4 * m.Cout);
+        }
+        if (lp.d.residual == SC_RES_PROJ) {
+            lp.sv.vr = ws.take(es * B * m.Cout * m.Tp);
+            lp.sv.mean_r = (float*)ws.take(4 * m.Cout); lp.sv.invstd_r = (float*)ws.take(4 * m.Cout);
+        }
+        lp.y = (i + 1 < e->n_layers) ? ws.take(es * B * m.Cout * m.Tp) : nullptr;
+        max_act = std::max(max_act, es * B * (size_t)m.Cin * m.T);
+        max_act = std::max(max_act, es * B * (size_t)m.Cout * m.Tp);
+        C = m.Cout; T = m.Tp;
+    }
+    // shared scratch: plan every layer from the same offset and keep the maximum
+    const size_t mark = ws.off;
+    size_t hi = mark;
+    for (int i = 0; i < e->n_layers; ++i) {
+        Bump b(base, cap); b.off = mark; FwdScratch f; plan_fwd(&P->L[i].d, P->L[i].m, b, &f, tc); hi = std::max(hi, b.off);
+        Bump c(base, cap); c.off = mark; BwdScratch s; plan_bwd(&P->L[i].d, P->L[i].m, c, &s, tc); hi = std::max(hi, c.off);
+    }
+    ws.off = hi;
+    P->gbuf[0] = ws.take(max_act); P->gbuf[1] = ws.take(max_act);
+    P->pending = max_res ? ws.take(max_res) : nullptr;
+    P->bytes = ws.off + 256;
+    if (!ws.ok()) return SC_ERR_WORKSPACE;
+    P->scratch_mark = mark;
+    return SC_OK;
+}
+
+sc_block_params layer_params(const void* blob, const int64_t* off) {
+    auto at = [&](int j) -> const void* { return off[j] < 0 ? nullptr : (const char*)blob + off[j]; };
+    sc_block_params p;
+    p.wd = at(0); p.wp = at(1); p.gamma = (const float*)at(2); p.beta = (const float*)at(3);
+    p.bias = (const float*)at(4); p.wr = at(5); p.gamma_r = (const float*)at(6); p.beta_r = (const float*)at(7);
+    return p;
+}
+sc_block_grads layer_grads(void* blob, const int64_t* off) {
+    auto at = [&](int j) -> float* { return off[j] < 0 ? nullptr : (float*)((char*)blob + off[j]); };
+    sc_block_grads g;
+    g.dwd = at(0); g.dwp = at(1); g.dgamma = at(2); g.dbeta = at(3); g.dbias = at(4);
+    g.dwr = at(5); g.dgamma_r = at(6); g.dbeta_r = at(7);
+    return g;
+}
+}  // namespace
+
+int encoder_workspace_bytes(const sc_encoder_desc* desc, size_t* bytes) {
+    if (!bytes) return SC_ERR_NULL;
+    EncPlan P;
+    SC_TRY(plan_encoder(desc, nullptr, 0, &P, nullptr));
+    *bytes = P.bytes;
+    return SC_OK;
+}
+
+int encoder_fwd_bwd(sc_ctx* ctx, const sc_encoder_desc* e, const sc_tensor* x, const int32_t* lengths_dev,
+                    const void* params_blob, const int64_t* param_offsets, const sc_tensor* dlogits,
+                    sc_tensor* logits, int32_t* out_lengths_dev, void* grads_blob,
+                    const int64_t* grad_offsets, sc_tensor* dx, int accumulate, void* workspace,
+                    size_t workspace_bytes, void* cuda_stream) {
+    if (!ctx || !lengths_dev || !params_blob || !param_offsets || !grads_blob || !grad_offsets) return SC_ERR_NULL;
+    if (!workspace) return SC_ERR_WORKSPACE;
+    EncPlan P;
+    SC_TRY(plan_encoder(e, workspace, workspace_bytes, &P, &ctx->tc));
+    const int n = e->n_layers;
+    const size_t mark = P.scratch_mark;
+    const Dims& m0 = P.L[0].m; const Dims& ml = P.L[n - 1].m;
+    const int dt = P.L[0].d.io_dtype;
+    SC_TRY(check_tensor(x, dt, m0.B, m0.Cin, m0.T));
+    SC_TRY(check_tensor(logits, dt, ml.B, ml.Cout, ml.Tp));
+    SC_TRY(check_tensor(dlogits, dt, ml.B, ml.Cout, ml.Tp));
+    if (dx) SC_TRY(check_tensor(dx, dt, m0.B, m0.Cin, m0.T));
+    std::vector<sc_block_params> prm(n);
+    std::vector<sc_block_grads> grd(n);
+    for (int i = 0; i < n; ++i) {
+        prm[i] = layer_params(params_blob, param_offsets + 8 * i);
+        grd[i] = layer_grads(grads_blob, grad_offsets + 8 * i);
+        SC_TRY(check_params(&P.L[i].d, &prm[i]));
+        SC_TRY(check_grads(&P.L[i].d, &grd[i]));
+    }
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches};
+    auto input_of = [&](int i) -> const void* { return i == 0 ? x->ptr : P.L[i - 1].y; };
+    auto len_in_of = [&](int i) -> const int* { return i == 0 ? lengths_dev : P.L[i - 1].len_out; };
+    auto res_src = [&](int i) -> int { return (e->res_from && e->res_from[i] >= 0) ? e->res_from[i] : i; };
+
+    // forward
+    for (int i = 0; i < n; ++i) {
+        LayerPlan& lp = P.L[i];
+        Bump b(workspace, workspace_bytes); b.off = mark;
+        FwdScratch f; plan_fwd(&lp.d, lp.m, b, &f, &ctx->tc);
+        BlockIO io{};
+        io.x = input_of(i);
+        io.xres = lp.d.residual != SC_RES_NONE ? input_of(res_src(i)) : nullptr;
+        io.y = (i + 1 < n) ? lp.y : logits->ptr;
+        io.len_in = len_in_of(i); io.len_out = lp.len_out; io.nvalid = lp.nvalid;
+        io.x_clean = i > 0; io.res_clean = lp.d.residual != SC_RES_NONE && res_src(i) > 0;
+        io.lengths_ready = !lp.own_lengths;
+        SC_TRY(block_fwd_impl(ctx, L, &lp.d, lp.m, io, &prm[i], &lp.sv, nullptr, nullptr, f));
+    }
+    if (out_lengths_dev)
+        cudaMemcpyAsync(out_lengths_dev, P.L[n - 1].len_out, sizeof(int) * m0.B, cudaMemcpyDeviceToDevice, L.stream);
+
+    // backward
+    const void* g = dlogits->ptr;
+    std::vector<char> has_pending(n, 0);
+    for (int i = n - 1; i >= 0; --i) {
+        LayerPlan& lp = P.L[i];
+        Bump b(workspace, workspace_bytes); b.off = mark;
+        BwdScratch s; plan_bwd(&lp.d, lp.m, b, &s, &ctx->tc);
+        BwdIO io{};
+        io.dy = g; io.x = input_of(i); io.y = (i + 1 < n) ? lp.y : logits->ptr;
+        io.xres = lp.d.residual != SC_RES_NONE ? input_of(res_src(i)) : nullptr;
+        io.dx = (i == 0) ? (dx ? dx->ptr : nullptr) : P.gbuf[i & 1];
+        io.dx_res = nullptr;
+        if (lp.d.residual != SC_RES_NONE && res_src(i) != i) { io.dx_res = P.pending; has_pending[res_src(i)] = 1; }
+        io.dx_add = has_pending[i] ? P.pending : nullptr;
+        io.len_in = len_in_of(i); io.len_out = lp.len_out; io.nvalid = lp.nvalid;
+        io.x_clean = i > 0; io.res_clean = lp.d.residual != SC_RES_NONE && res_src(i) > 0;
+        SC_TRY(block_bwd_impl(ctx, L, &lp.d, lp.m, io, &prm[i], &lp.sv, &grd[i], accumulate, s));
+        g = io.dx;
+    }
+    return finish(ctx);
+}
+
+}  // extern "C"

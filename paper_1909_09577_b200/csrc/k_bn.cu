@@ -1,0 +1,395 @@
+// Lengths, masked batch-norm statistics / apply / backward, and small elementwise kernels.
+// All of these stream [B,C,T] tensors once; one CTA handles one (sample, channel) row so that the
+// per-channel coefficients are loaded once and reductions stay inside the CTA (warp shuffles +
+// one shared-memory step).  Cross-CTA reductions go through per-row partials that a finalize
+// kernel sums in a fixed order, so results are bit-repeatable.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace sc {
+namespace {
+
+constexpr int kRowThreads = 128;
+
+template <typename T>
+__device__ __forceinline__ void load_chunk(const T* row, int t0, int Tp, bool vec, float (&f)[8]) {
+    if (vec && t0 + 8 <= Tp) { ld8<T>(row + t0, f); return; }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) f[i] = (t0 + i < Tp) ? ldf(row + t0 + i) : 0.f;
+}
+template <typename T>
+__device__ __forceinline__ void store_chunk(T* row, int t0, int Tp, bool vec, const float (&f)[8]) {
+    if (vec && t0 + 8 <= Tp) { st8<T>(row + t0, f); return; }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) if (t0 + i < Tp) stf(row + t0 + i, f[i]);
+}
+
+// Sum of `v` over the CTA (kRowThreads threads); result valid in every thread.
+template <int N>
+__device__ __forceinline__ void block_sum(float (&v)[N]) {
+    __shared__ float sh[N][kRowThreads / 32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int i = 0; i < N; ++i) v[i] = warp_sum(v[i]);
+    __syncthreads();   // protect sh against a previous use
+    if (lane == 0) {
+#pragma unroll
+        for (int i = 0; i < N; ++i) sh[i][warp] = v[i];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < kRowThreads / 32; ++w) s += sh[i][w];
+        v[i] = s;
+    }
+}
+
+__global__ void lengths_kernel(const int* __restrict__ len_in, int B, int T_in, int stride,
+                               int* __restrict__ len_out, int* __restrict__ nvalid, int* status) {
+    // single CTA; B is small (<= a few thousand)
+    __shared__ int total;
+    if (threadIdx.x == 0) total = 0;
+    __syncthreads();
+    int local = 0;
+    for (int b = threadIdx.x; b < B; b += blockDim.x) {
+        int l = len_in[b];
+        if (l < 1 || l > T_in) { raise_status(status, kErrLengths); l = min(max(l, 0), T_in); }
+        int lo = (l + stride - 1) / stride;
+        len_out[b] = lo;
+        local += lo;
+    }
+    atomicAdd(&total, local);   // integer: order-independent
+    __syncthreads();
+    if (threadIdx.x == 0) *nvalid = total;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kRowThreads)
+bn_stats_kernel(const T* __restrict__ v, const int* __restrict__ len_out, int C, int Tp,
+                float2* __restrict__ partials) {
+    const int row = blockIdx.x, b = row / C;
+    const int len = min(len_out[b], Tp);
+    const T* p = v + (size_t)row * Tp;
+    const bool vec = (Tp % 8 == 0);
+    float s[1] = {0.f};
+    for (int t0 = threadIdx.x * 8; t0 < len; t0 += kRowThreads * 8) {
+        float f[8];
+        load_chunk(p, t0, Tp, vec, f);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) if (t0 + i < len) s[0] += f[i];
+    }
+    block_sum(s);
+    const float mean = len > 0 ? s[0] / (float)len : 0.f;
+    float q[1] = {0.f};
+    for (int t0 = threadIdx.x * 8; t0 < len; t0 += kRowThreads * 8) {
+        float f[8];
+        load_chunk(p, t0, Tp, vec, f);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) if (t0 + i < len) { float d = f[i] - mean; q[0] += d * d; }
+    }
+    block_sum(q);
+    if (threadIdx.x == 0) partials[row] = make_float2(s[0], q[0]);
+}
+
+__global__ void bn_finalize_kernel(const float2* __restrict__ partials, int parts_per_b, int tile_w,
+                                   const int* __restrict__ len_out, const int* __restrict__ nvalid, int B,
+                                   int C, const float* __restrict__ gamma, const float* __restrict__ beta,
+                                   float eps, float momentum, float* __restrict__ mean_out,
+                                   float* __restrict__ invstd_out, float2* __restrict__ scale_shift,
+                                   float* running_mean, float* running_var) {
+    const int o = blockIdx.x * blockDim.x + threadIdx.x;
+    if (o >= C) return;
+    double n = 0.0, mean = 0.0, m2 = 0.0;
+    for (int b = 0; b < B; ++b) {
+        const int len = len_out[b];
+        for (int j = 0; j < parts_per_b; ++j) {
+            int cnt = min(max(len - j * tile_w, 0), tile_w);
+            if (cnt <= 0) break;
+            float2 p = partials[((size_t)b * parts_per_b + j) * C + o];
+            double nb = cnt, mb = (double)p.x / nb, nt = n + nb, d = mb - mean;
+            mean += d * (nb / nt);
+            m2 += (double)p.y + d * d * (n * nb / nt);
+            n = nt;
+        }
+    }
+    const double N = (double)(*nvalid);
+    const double var = N > 0 ? m2 / N : 0.0;
+    const float invstd = (float)(1.0 / sqrt(var + (double)eps));
+    const float mu = (float)mean;
+    mean_out[o] = mu;
+    invstd_out[o] = invstd;
+    const float sc_ = gamma[o] * invstd;
+    scale_shift[o] = make_float2(sc_, beta[o] - mu * sc_);
+    if (running_mean) running_mean[o] = (1.f - momentum) * running_mean[o] + momentum * mu;
+    if (running_var) {
+        double unb = N > 1 ? var * (N / (N - 1.0)) : var;
+        running_var[o] = (1.f - momentum) * running_var[o] + momentum * (float)unb;
+    }
+}
+
+__global__ void bn_scale_shift_kernel(const float* mean, const float* invstd, const float* gamma,
+                                      const float* beta, float2* ss, int C) {
+    const int o = blockIdx.x * blockDim.x + threadIdx.x;
+    if (o >= C) return;
+    const float sc_ = gamma[o] * invstd[o];
+    ss[o] = make_float2(sc_, beta[o] - mean[o] * sc_);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kRowThreads) bn_apply_kernel(ApplyArgs a) {
+    const int row = blockIdx.x, b = row / a.C, o = row % a.C;
+    const int Tp = a.Tp, len = min(a.len_out[b], Tp);
+    const bool vec = (Tp % 8 == 0);
+    const T* v = (const T*)a.v + (size_t)row * Tp;
+    const T* xr = a.residual == 1 ? (const T*)a.xres + (size_t)row * Tp : nullptr;
+    const T* vr = a.residual == 2 ? (const T*)a.vr + (size_t)row * Tp : nullptr;
+    T* y = (T*)a.y + (size_t)row * Tp;
+    const float2 ss = a.ss[o];
+    const float2 sr = a.residual == 2 ? a.ss_r[o] : make_float2(0.f, 0.f);
+    for (int t0 = threadIdx.x * 8; t0 < Tp; t0 += kRowThreads * 8) {
+        float out[8];
+        if (t0 < len) {
+            float f[8], r[8];
+            load_chunk(v, t0, Tp, vec, f);
+            if (a.residual == 1) load_chunk(xr, t0, Tp, vec, r);
+            else if (a.residual == 2) {
+                load_chunk(vr, t0, Tp, vec, r);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) r[i] = fmaf(sr.x, r[i], sr.y);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) r[i] = 0.f;
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float bn = fmaf(ss.x, f[i], ss.y);
+                float q;
+                if (a.res_before_relu) { q = bn + r[i]; if (a.has_relu) q = fmaxf(q, 0.f); }
+                else { q = (a.has_relu ? fmaxf(bn, 0.f) : bn) + r[i]; }
+                out[i] = (t0 + i < len) ? q : 0.f;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) out[i] = 0.f;
+        }
+        store_chunk(y, t0, Tp, vec, out);
+    }
+}
+
+// Shared by the reduce and apply steps of the backward pass: per element gate and normalised value.
+template <typename T>
+struct BwdRow {
+    const T *g, *y, *v, *vr;
+    float mean, invstd, mean_r, invstd_r;
+    float2 ss;
+    int len, Tp;
+    bool vec;
+    __device__ BwdRow(const BnBwdArgs& a, int row, int b, int o) {
+        Tp = a.Tp; len = min(a.len_out[b], Tp); vec = (Tp % 8 == 0);
+        g = (const T*)a.g + (size_t)row * Tp;
+        y = a.y ? (const T*)a.y + (size_t)row * Tp : nullptr;
+        v = a.v ? (const T*)a.v + (size_t)row * Tp : nullptr;
+        vr = (a.residual == 2) ? (const T*)a.vr + (size_t)row * Tp : nullptr;
+        mean = a.has_bn ? a.mean[o] : 0.f; invstd = a.has_bn ? a.invstd[o] : 1.f;
+        mean_r = (a.residual == 2) ? a.mean_r[o] : 0.f; invstd_r = (a.residual == 2) ? a.invstd_r[o] : 1.f;
+        ss = (a.has_relu && !a.res_before_relu && a.has_bn) ? a.ss[o] : make_float2(1.f, 0.f);
+    }
+    // ga: gated upstream gradient; gr: gradient reaching the residual sum; vh/vhr: normalised values
+    __device__ __forceinline__ void chunk(const BnBwdArgs& a, int t0, float (&ga)[8], float (&gr)[8],
+                                          float (&vh)[8], float (&vhr)[8]) const {
+        float fg[8], fy[8], fv[8], fr[8];
+        load_chunk(g, t0, Tp, vec, fg);
+        const bool need_y = a.has_relu && a.res_before_relu;
+        if (need_y) load_chunk(y, t0, Tp, vec, fy);
+        const bool need_v = a.has_bn;
+        if (need_v) load_chunk(v, t0, Tp, vec, fv);
+        if (a.residual == 2) load_chunk(vr, t0, Tp, vec, fr);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const bool in = (t0 + i < len);
+            const float gm = in ? fg[i] : 0.f;
+            bool gate = true;
+            if (a.has_relu) gate = a.res_before_relu ? (fy[i] > 0.f) : (fmaf(ss.x, fv[i], ss.y) > 0.f);
+            ga[i] = gate ? gm : 0.f;
+            gr[i] = a.res_before_relu ? ga[i] : gm;
+            vh[i] = (need_v && in) ? (fv[i] - mean) * invstd : 0.f;
+            vhr[i] = (a.residual == 2 && in) ? (fr[i] - mean_r) * invstd_r : 0.f;
+        }
+    }
+};
+
+template <typename T>
+__global__ void __launch_bounds__(kRowThreads) bn_bwd_reduce_kernel(BnBwdArgs a) {
+    const int row = blockIdx.x, b = row / a.C, o = row % a.C;
+    BwdRow<T> R(a, row, b, o);
+    float s[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int t0 = threadIdx.x * 8; t0 < R.len; t0 += kRowThreads * 8) {
+        float ga[8], gr[8], vh[8], vhr[8];
+        R.chunk(a, t0, ga, gr, vh, vhr);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            s[0] += ga[i]; s[1] += ga[i] * vh[i]; s[2] += gr[i]; s[3] += gr[i] * vhr[i];
+        }
+    }
+    block_sum(s);
+    if (threadIdx.x == 0) a.partials[row] = make_float4(s[0], s[1], s[2], s[3]);
+}
+
+__global__ void bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const float* gamma_r,
+                                       float* dgamma, float* dbeta, float* dgamma_r, float* dbeta_r,
+                                       float* dbias, int accumulate) {
+    const int o = blockIdx.x * blockDim.x + threadIdx.x;
+    if (o >= a.C) return;
+    double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+    for (int b = 0; b < a.B; ++b) {
+        float4 p = a.partials[(size_t)b * a.C + o];
+        s0 += p.x; s1 += p.y; s2 += p.z; s3 += p.w;
+    }
+    const float N = (float)(*a.nvalid);
+    auto put = [&](float* dst, double val) {
+        if (dst) dst[o] = accumulate ? dst[o] + (float)val : (float)val;
+    };
+    if (a.has_bn) {
+        put(dbeta, s0); put(dgamma, s1);
+        a.coef[o] = make_float4(gamma[o] * a.invstd[o], (float)s0 / N, (float)s1 / N, 0.f);
+    } else {
+        put(dbias, s0);
+        a.coef[o] = make_float4(1.f, 0.f, 0.f, 0.f);
+    }
+    if (a.residual == 2) {
+        put(dbeta_r, s2); put(dgamma_r, s3);
+        a.coef_r[o] = make_float4(gamma_r[o] * a.invstd_r[o], (float)s2 / N, (float)s3 / N, 0.f);
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kRowThreads) bn_bwd_apply_kernel(BnBwdArgs a) {
+    const int row = blockIdx.x, b = row / a.C, o = row % a.C;
+    BwdRow<T> R(a, row, b, o);
+    const float4 cf = a.coef[o];
+    const float4 cr = (a.residual == 2) ? a.coef_r[o] : make_float4(0.f, 0.f, 0.f, 0.f);
+    T* gv = (T*)a.gv + (size_t)row * R.Tp;
+    T* gvr = (a.residual == 2) ? (T*)a.gvr + (size_t)row * R.Tp : nullptr;
+    T* gres = (a.residual == 1) ? (T*)a.gres + (size_t)row * R.Tp : nullptr;
+    for (int t0 = threadIdx.x * 8; t0 < R.Tp; t0 += kRowThreads * 8) {
+        float o1[8], o2[8];
+        if (t0 < R.len) {
+            float ga[8], gr[8], vh[8], vhr[8];
+            R.chunk(a, t0, ga, gr, vh, vhr);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const bool in = (t0 + i < R.len);
+                o1[i] = in ? cf.x * (ga[i] - cf.y - vh[i] * cf.z) : 0.f;
+                if (a.residual == 2) o2[i] = in ? cr.x * (gr[i] - cr.y - vhr[i] * cr.z) : 0.f;
+                else o2[i] = gr[i];
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { o1[i] = 0.f; o2[i] = 0.f; }
+        }
+        store_chunk(gv, t0, R.Tp, R.vec, o1);
+        if (gvr) store_chunk(gvr, t0, R.Tp, R.vec, o2);
+        if (gres) store_chunk(gres, t0, R.Tp, R.vec, o2);
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kRowThreads)
+ew_add_masked_kernel(T* out, const T* a, const T* b, const T* c, const int* len, int C, int Tt) {
+    const int row = blockIdx.x, bb = row / C;
+    const int l = min(len[bb], Tt);
+    const bool vec = (Tt % 8 == 0);
+    const size_t off = (size_t)row * Tt;
+    for (int t0 = threadIdx.x * 8; t0 < Tt; t0 += kRowThreads * 8) {
+        float f[8];
+        if (t0 < l) {
+            load_chunk(a + off, t0, Tt, vec, f);
+            if (b) { float q[8]; load_chunk(b + off, t0, Tt, vec, q);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) f[i] += q[i]; }
+            if (c) { float q[8]; load_chunk(c + off, t0, Tt, vec, q);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) f[i] += q[i]; }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) if (t0 + i >= l) f[i] = 0.f;
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) f[i] = 0.f;
+        }
+        store_chunk(out + off, t0, Tt, vec, f);
+    }
+}
+
+}  // namespace
+
+#define SC_DISPATCH(dtype, ...)                                             \
+    switch (dtype) {                                                        \
+        case F32: { using T = float; __VA_ARGS__; break; }                  \
+        case F16: { using T = __half; __VA_ARGS__; break; }                 \
+        default:  { using T = __nv_bfloat16; __VA_ARGS__; break; }          \
+    }
+
+void lengths(const Launch& L, const int* len_in, int B, int T_in, int stride, int* len_out, int* nvalid) {
+    lengths_kernel<<<1, 256, 0, L.stream>>>(len_in, B, T_in, stride, len_out, nvalid, L.status);
+    L.count();
+}
+
+void bn_stats(const Launch& L, int dtype, const void* v, const int* len_out, int B, int C, int Tp,
+              float2* partials) {
+    SC_DISPATCH(dtype, (bn_stats_kernel<T><<<B * C, kRowThreads, 0, L.stream>>>((const T*)v, len_out, C, Tp, partials)));
+    L.count();
+}
+
+void bn_finalize(const Launch& L, const float2* partials, int parts_per_b, int tile_w, const int* len_out,
+                 const int* nvalid, int B, int C, const float* gamma, const float* beta, float eps,
+                 float momentum, float* mean, float* invstd, float2* scale_shift, float* running_mean,
+                 float* running_var) {
+    bn_finalize_kernel<<<(C + 63) / 64, 64, 0, L.stream>>>(partials, parts_per_b, tile_w, len_out, nvalid, B, C,
+                                                            gamma, beta, eps, momentum, mean, invstd,
+                                                            scale_shift, running_mean, running_var);
+    L.count();
+}
+
+void bn_scale_shift(const Launch& L, const float* mean, const float* invstd, const float* gamma,
+                    const float* beta, float2* ss, int C) {
+    bn_scale_shift_kernel<<<(C + 127) / 128, 128, 0, L.stream>>>(mean, invstd, gamma, beta, ss, C);
+    L.count();
+}
+
+void bn_apply(const Launch& L, int dtype, const ApplyArgs& a) {
+    SC_DISPATCH(dtype, (bn_apply_kernel<T><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a)));
+    L.count();
+}
+
+void bn_bwd_reduce(const Launch& L, int dtype, const BnBwdArgs& a) {
+    SC_DISPATCH(dtype, (bn_bwd_reduce_kernel<T><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a)));
+    L.count();
+}
+
+void bn_bwd_finalize(const Launch& L, const BnBwdArgs& a, const float* gamma, const float* gamma_r,
+                     float* dgamma, float* dbeta, float* dgamma_r, float* dbeta_r, float* dbias,
+                     int accumulate) {
+    bn_bwd_finalize_kernel<<<(a.C + 63) / 64, 64, 0, L.stream>>>(a, gamma, gamma_r, dgamma, dbeta, dgamma_r,
+                                                                  dbeta_r, dbias, accumulate);
+    L.count();
+}
+
+void bn_bwd_apply(const Launch& L, int dtype, const BnBwdArgs& a) {
+    SC_DISPATCH(dtype, (bn_bwd_apply_kernel<T><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a)));
+    L.count();
+}
+
+void ew_add_masked(const Launch& L, int dtype, void* out, const void* a, const void* b, const void* c,
+                   const int* len, int B, int C, int Tt) {
+    SC_DISPATCH(dtype, (ew_add_masked_kernel<T><<<B * C, kRowThreads, 0, L.stream>>>((T*)out, (const T*)a, (const T*)b,
+                                                                                      (const T*)c, len, C, Tt)));
+    L.count();
+}
+
+void mask_copy(const Launch& L, int dtype, void* out, const void* in, const int* len, int B, int C, int Tt) {
+    ew_add_masked(L, dtype, out, in, nullptr, nullptr, len, B, C, Tt);
+}
+
+}  // namespace sc

@@ -1,0 +1,369 @@
+// Depthwise (per-channel) correlation over time: forward, input gradient, tap gradient.
+//
+// Stride-1 layers (all but the first layer of the encoder) use register-blocked kernels: a thread
+// owns R consecutive outputs, keeps a 2R-wide sliding window of the shared-memory tile and R taps
+// in registers and performs R*R FMAs per 2R shared loads.  The input gradient of a stride-1
+// correlation is the same correlation with flipped taps, so one kernel serves both.  Any other
+// stride goes through plain tiled kernels.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace sc {
+namespace {
+
+constexpr int R = 8;          // outputs (or taps) per thread
+constexpr int CH = 8;         // channels per CTA in the stride-1 kernel (one warp each)
+constexpr int TT = 32 * R;    // outputs per channel per CTA
+
+// Conflict-free placement for 16-byte shared loads at an 8-float lane pitch.
+__device__ __forceinline__ int phys(int i) { return i + ((i >> 5) << 2); }
+
+template <typename T>
+__global__ void __launch_bounds__(32 * CH)
+dw_corr_s1_kernel(const T* __restrict__ in, const T* __restrict__ w, T* __restrict__ out,
+                  const T* __restrict__ add1, const T* __restrict__ add2,
+                  const int* __restrict__ len_src, const int* __restrict__ len_dst,
+                  int C, int Tt, int K, int Kpad, int flip) {
+    extern __shared__ float smem[];
+    const int lane = threadIdx.x, wrp = threadIdx.y;
+    const int b = blockIdx.z, c = blockIdx.y * CH + wrp, t0 = blockIdx.x * TT;
+    if (c >= C) return;                       // warps are independent: no CTA-wide barrier below
+    const int P = (K - 1) / 2;
+    const int XW = TT + Kpad;                 // logical tile width
+    float* xs = smem + (size_t)wrp * (phys(XW) + 4 + Kpad);
+    float* ws = xs + phys(XW) + 4;
+    const int ls = min(len_src[b], Tt), ld = min(len_dst[b], Tt);
+    const size_t row = ((size_t)b * C + c) * Tt;
+    T* orow = out + row;
+    const bool vec = (Tt % 8 == 0);
+
+    if (t0 >= ld) {                           // tile lies wholly in padding: zeros
+        float z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        const int t = t0 + lane * R;
+        if (vec) { if (t < Tt) st8<T>(orow + t, z); }
+        else { for (int r = 0; r < R; ++r) if (t + r < Tt) stf(orow + t + r, 0.f); }
+        return;
+    }
+    // taps (zero padded to Kpad)
+    for (int k = lane; k < Kpad; k += 32)
+        ws[k] = (k < K) ? ldf(w + (size_t)c * K + (flip ? K - 1 - k : k)) : 0.f;
+    // input tile: logical index i <-> frame tau = t0 - P + i, zero outside [0, ls)
+    const T* irow = in + row;
+    const int tau0 = t0 - P;
+    if (vec) {
+        const int a0 = (tau0 >= 0) ? (tau0 & ~7) : -(((-tau0) + 7) & ~7);   // floor to a multiple of 8
+        const int nchunk = (tau0 + XW - a0 + 7) / 8;
+        for (int j = lane; j < nchunk; j += 32) {
+            const int ta = a0 + 8 * j;
+            float f[8];
+            if (ta >= 0 && ta < ls) ld8<T>(irow + ta, f);
+            else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) f[e] = 0.f;
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int i = ta + e - tau0;
+                if (i >= 0 && i < XW) xs[phys(i)] = (ta + e < ls) ? f[e] : 0.f;
+            }
+        }
+    } else {
+        for (int i = lane; i < XW; i += 32) {
+            const int tau = tau0 + i;
+            xs[phys(i)] = (tau >= 0 && tau < ls) ? ldf(irow + tau) : 0.f;
+        }
+    }
+    __syncwarp();
+
+    float acc[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) acc[r] = 0.f;
+    float win[2 * R];
+    const int base = lane * R;
+    {
+        const float4 a = *reinterpret_cast<const float4*>(xs + phys(base));
+        const float4 bq = *reinterpret_cast<const float4*>(xs + phys(base + 4));
+        win[0] = a.x; win[1] = a.y; win[2] = a.z; win[3] = a.w;
+        win[4] = bq.x; win[5] = bq.y; win[6] = bq.z; win[7] = bq.w;
+    }
+    for (int kk = 0; kk < Kpad; kk += R) {
+        const float4 a = *reinterpret_cast<const float4*>(xs + phys(base + kk + R));
+        const float4 bq = *reinterpret_cast<const float4*>(xs + phys(base + kk + R + 4));
+        win[8] = a.x; win[9] = a.y; win[10] = a.z; win[11] = a.w;
+        win[12] = bq.x; win[13] = bq.y; win[14] = bq.z; win[15] = bq.w;
+        const float4 w0 = *reinterpret_cast<const float4*>(ws + kk);
+        const float4 w1 = *reinterpret_cast<const float4*>(ws + kk + 4);
+        const float wv[R] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+        for (int q = 0; q < R; ++q)
+#pragma unroll
+            for (int r = 0; r < R; ++r) acc[r] = fmaf(wv[q], win[r + q], acc[r]);
+#pragma unroll
+        for (int r = 0; r < R; ++r) win[r] = win[r + R];
+    }
+
+    const int t = t0 + base;
+    if (t >= Tt) return;
+    if (vec) {
+        if (add1) { float f[8]; ld8<T>(add1 + row + t, f);
+#pragma unroll
+            for (int r = 0; r < R; ++r) acc[r] += f[r]; }
+        if (add2) { float f[8]; ld8<T>(add2 + row + t, f);
+#pragma unroll
+            for (int r = 0; r < R; ++r) acc[r] += f[r]; }
+#pragma unroll
+        for (int r = 0; r < R; ++r) if (t + r >= ld) acc[r] = 0.f;
+        st8<T>(orow + t, acc);
+    } else {
+        for (int r = 0; r < R; ++r) {
+            if (t + r >= Tt) break;
+            float q = acc[r];
+            if (add1) q += ldf(add1 + row + t + r);
+            if (add2) q += ldf(add2 + row + t + r);
+            stf(orow + t + r, (t + r < ld) ? q : 0.f);
+        }
+    }
+}
+
+// ---- any stride: plain tiled kernels (used by the stride-2 first layer) ---------------------
+constexpr int GT = 256;   // outputs per CTA
+
+template <typename T>
+__global__ void __launch_bounds__(GT)
+dw_fwd_generic_kernel(const T* __restrict__ x, const T* __restrict__ w, T* __restrict__ u,
+                      const int* __restrict__ len_in, const int* __restrict__ len_out,
+                      int C, int Tt, int Tp, int K, int s) {
+    extern __shared__ float smem[];
+    const int b = blockIdx.z, c = blockIdx.y, t0 = blockIdx.x * GT;
+    const int P = (K - 1) / 2, XW = (GT - 1) * s + K;
+    float* xs = smem;
+    float* ws = smem + XW;
+    const int li = min(len_in[b], Tt), lo = min(len_out[b], Tp);
+    const T* xrow = x + ((size_t)b * C + c) * Tt;
+    for (int k = threadIdx.x; k < K; k += GT) ws[k] = ldf(w + (size_t)c * K + k);
+    const int tau0 = t0 * s - P;
+    for (int i = threadIdx.x; i < XW; i += GT) {
+        const int tau = tau0 + i;
+        xs[i] = (tau >= 0 && tau < li) ? ldf(xrow + tau) : 0.f;
+    }
+    __syncthreads();
+    const int t = t0 + threadIdx.x;
+    if (t >= Tp) return;
+    float acc = 0.f;
+    for (int k = 0; k < K; ++k) acc = fmaf(ws[k], xs[threadIdx.x * s + k], acc);
+    stf(u + ((size_t)b * C + c) * Tp + t, (t < lo) ? acc : 0.f);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(GT)
+dw_dgrad_generic_kernel(const T* __restrict__ gu, const T* __restrict__ w, T* __restrict__ dx,
+                        const T* __restrict__ add1, const T* __restrict__ add2,
+                        const int* __restrict__ len_in, const int* __restrict__ len_out,
+                        int C, int Tt, int Tp, int K, int s) {
+    extern __shared__ float smem[];
+    const int b = blockIdx.z, c = blockIdx.y, tau0 = blockIdx.x * GT;
+    const int P = (K - 1) / 2;
+    // outputs tau0..tau0+GT-1 read gu[t] for t in [tlo, thi]
+    const int num = tau0 + P - (K - 1);
+    const int tlo = (num >= 0) ? (num + s - 1) / s : -((-num) / s);
+    const int thi = (tau0 + GT - 1 + P) / s;
+    const int GW = thi - tlo + 1;
+    float* gs = smem;
+    float* ws = smem + GW;
+    const int li = min(len_in[b], Tt), lo = min(len_out[b], Tp);
+    const T* grow = gu + ((size_t)b * C + c) * Tp;
+    for (int k = threadIdx.x; k < K; k += GT) ws[k] = ldf(w + (size_t)c * K + k);
+    for (int i = threadIdx.x; i < GW; i += GT) {
+        const int t = tlo + i;
+        gs[i] = (t >= 0 && t < lo) ? ldf(grow + t) : 0.f;
+    }
+    __syncthreads();
+    const int tau = tau0 + threadIdx.x;
+    if (tau >= Tt) return;
+    float acc = 0.f;
+    for (int k = 0; k < K; ++k) {
+        const int q = tau + P - k;
+        if (q >= 0 && q % s == 0) { const int t = q / s; if (t >= tlo && t <= thi) acc = fmaf(ws[k], gs[t - tlo], acc); }
+    }
+    const size_t o = ((size_t)b * C + c) * Tt + tau;
+    if (add1) acc += ldf(add1 + o);
+    if (add2) acc += ldf(add2 + o);
+    stf(dx + o, (tau < li) ? acc : 0.f);
+}
+
+// One warp per (b,c) row; lane k-strided taps; plain but correct for any stride.
+template <typename T>
+__global__ void __launch_bounds__(128)
+dw_wgrad_generic_kernel(const T* __restrict__ gu, const T* __restrict__ x, float* __restrict__ partials,
+                        const int* __restrict__ len_in, const int* __restrict__ len_out,
+                        int B, int C, int Tt, int Tp, int K, int s) {
+    const int c = blockIdx.x, lane = threadIdx.x & 31, wrp = threadIdx.x >> 5;
+    const int P = (K - 1) / 2;
+    // partials[b][c][k]; warps stride over samples
+    for (int b = wrp; b < B; b += 4) {
+        const int li = min(len_in[b], Tt), lo = min(len_out[b], Tp);
+        const T* grow = gu + ((size_t)b * C + c) * Tp;
+        const T* xrow = x + ((size_t)b * C + c) * Tt;
+        for (int k = 0; k < K; ++k) {
+            float acc = 0.f;
+            for (int t = lane; t < lo; t += 32) {
+                const int tau = t * s + k - P;
+                if (tau >= 0 && tau < li) acc = fmaf(ldf(grow + t), ldf(xrow + tau), acc);
+            }
+            acc = warp_sum(acc);
+            if (lane == 0) partials[((size_t)b * C + c) * K + k] = acc;
+        }
+    }
+}
+
+// ---- stride-1 tap gradient: register-blocked --------------------------------------------------
+// CTA = one channel, a group of BG samples.  Thread (kg, seg): tap group kg (R taps) x time segment.
+constexpr int WG_THREADS = 128;
+constexpr int WG_TT = 1024;     // frames per shared-memory tile
+constexpr int WG_BG = 8;        // samples per CTA
+
+template <typename T>
+__global__ void __launch_bounds__(WG_THREADS)
+dw_wgrad_s1_kernel(const T* __restrict__ gu, const T* __restrict__ x, float* __restrict__ partials,
+                   const int* __restrict__ len_in, const int* __restrict__ len_out,
+                   int B, int C, int Tt, int K, int Kpad) {
+    extern __shared__ float smem[];
+    const int c = blockIdx.x, bg = blockIdx.y;
+    const int P = (K - 1) / 2;
+    const int NG = Kpad / R;                       // tap groups
+    const int nseg = WG_THREADS / NG;              // time segments
+    const int seglen = ((WG_TT + nseg - 1) / nseg + R - 1) / R * R;
+    const int GW = nseg * seglen;                  // >= WG_TT, zero filled beyond
+    const int XW = GW + Kpad;
+    float* gs = smem;                              // [GW]
+    float* xs = smem + GW;                         // [XW]: index i <-> frame t0 - P + i
+    float* red = xs + XW;                          // [nseg][Kpad]
+    const int tid = threadIdx.x;
+    const bool active = tid < NG * nseg;
+    const int kg = tid % NG, seg = tid / NG;
+    float acc[R];
+#pragma unroll
+    for (int q = 0; q < R; ++q) acc[q] = 0.f;
+
+    const int b_end = min(B, (bg + 1) * WG_BG);
+    for (int b = bg * WG_BG; b < b_end; ++b) {
+        const int li = min(len_in[b], Tt), lo = min(len_out[b], Tt);
+        const T* grow = gu + ((size_t)b * C + c) * Tt;
+        const T* xrow = x + ((size_t)b * C + c) * Tt;
+        for (int t0 = 0; t0 < lo; t0 += WG_TT) {
+            __syncthreads();
+            for (int i = tid; i < GW; i += WG_THREADS) {
+                const int t = t0 + i;
+                gs[i] = (i < WG_TT && t < lo) ? ldf(grow + t) : 0.f;
+            }
+            for (int i = tid; i < XW; i += WG_THREADS) {
+                const int tau = t0 - P + i;
+                xs[i] = (tau >= 0 && tau < li) ? ldf(xrow + tau) : 0.f;
+            }
+            __syncthreads();
+            if (active) {
+                const int ts = seg * seglen;
+                const float* xp = xs + ts + kg * R;
+                float win[2 * R];
+#pragma unroll
+                for (int r = 0; r < R; ++r) win[r] = xp[r];
+                for (int tt = 0; tt < seglen; tt += R) {
+#pragma unroll
+                    for (int r = 0; r < R; ++r) win[R + r] = xp[tt + R + r];
+                    float g[R];
+#pragma unroll
+                    for (int r = 0; r < R; ++r) g[r] = gs[ts + tt + r];
+#pragma unroll
+                    for (int r = 0; r < R; ++r)
+#pragma unroll
+                        for (int q = 0; q < R; ++q) acc[q] = fmaf(g[r], win[r + q], acc[q]);
+#pragma unroll
+                    for (int r = 0; r < R; ++r) win[r] = win[R + r];
+                }
+            }
+        }
+    }
+    __syncthreads();
+    if (active) {
+#pragma unroll
+        for (int q = 0; q < R; ++q) red[seg * Kpad + kg * R + q] = acc[q];
+    }
+    __syncthreads();
+    for (int k = tid; k < K; k += WG_THREADS) {
+        float sum = 0.f;
+        for (int sgi = 0; sgi < nseg; ++sgi) sum += red[sgi * Kpad + k];
+        partials[((size_t)bg * C + c) * K + k] = sum;
+    }
+}
+
+inline int kpad(int K) { return (K + R - 1) / R * R; }
+inline int host_phys(int i) { return i + ((i >> 5) << 2); }
+
+}  // namespace
+
+#define SC_DISPATCH(dtype, ...)                                             \
+    switch (dtype) {                                                        \
+        case F32: { using T = float; __VA_ARGS__; break; }                  \
+        case F16: { using T = __half; __VA_ARGS__; break; }                 \
+        default:  { using T = __nv_bfloat16; __VA_ARGS__; break; }          \
+    }
+
+static void corr_s1(const Launch& L, int dtype, const void* in, const void* w, void* out, const void* add1,
+                    const void* add2, const int* len_src, const int* len_dst, int B, int C, int Tt, int K,
+                    int flip) {
+    const int Kp = kpad(K);
+    const size_t smem = (size_t)CH * (host_phys(TT + Kp) + 4 + Kp) * sizeof(float);
+    dim3 grid((Tt + TT - 1) / TT, (C + CH - 1) / CH, B), block(32, CH);
+    SC_DISPATCH(dtype, (dw_corr_s1_kernel<T><<<grid, block, smem, L.stream>>>(
+                           (const T*)in, (const T*)w, (T*)out, (const T*)add1, (const T*)add2, len_src, len_dst,
+                           C, Tt, K, Kp, flip)));
+    L.count();
+}
+
+void dw_fwd(const Launch& L, int dtype, const void* x, const void* wd, void* u, const int* len_in,
+            const int* len_out, int B, int C, int Tt, int Tp, int K, int s) {
+    if (s == 1) { corr_s1(L, dtype, x, wd, u, nullptr, nullptr, len_in, len_out, B, C, Tt, K, 0); return; }
+    const size_t smem = (size_t)((GT - 1) * s + K + K) * sizeof(float);
+    dim3 grid((Tp + GT - 1) / GT, C, B);
+    SC_DISPATCH(dtype, (dw_fwd_generic_kernel<T><<<grid, GT, smem, L.stream>>>((const T*)x, (const T*)wd, (T*)u, len_in,
+                                                                               len_out, C, Tt, Tp, K, s)));
+    L.count();
+}
+
+void dw_dgrad(const Launch& L, int dtype, const void* gu, const void* wd, void* dx, const void* add1,
+              const void* add2, const int* len_in, const int* len_out, int B, int C, int Tt, int Tp,
+              int K, int s) {
+    if (s == 1) { corr_s1(L, dtype, gu, wd, dx, add1, add2, len_out, len_in, B, C, Tt, K, 1); return; }
+    const size_t smem = (size_t)((GT + K) / s + 4 + K) * sizeof(float);
+    dim3 grid((Tt + GT - 1) / GT, C, B);
+    SC_DISPATCH(dtype, (dw_dgrad_generic_kernel<T><<<grid, GT, smem, L.stream>>>(
+                           (const T*)gu, (const T*)wd, (T*)dx, (const T*)add1, (const T*)add2, len_in, len_out, C,
+                           Tt, Tp, K, s)));
+    L.count();
+}
+
+size_t dw_wgrad_scratch_bytes(int B, int C, int K) { return (size_t)B * C * K * sizeof(float); }
+
+void dw_wgrad(const Launch& L, int dtype, const void* gu, const void* x, float* dwd, float* partials,
+              int accumulate, const int* len_in, const int* len_out, int B, int C, int Tt, int Tp,
+              int K, int s) {
+    int nsplit;
+    if (s == 1) {
+        const int Kp = kpad(K), NG = Kp / R, nseg = WG_THREADS / NG;
+        const int seglen = ((WG_TT + nseg - 1) / nseg + R - 1) / R * R;
+        const int GW = nseg * seglen;
+        const size_t smem = (size_t)(GW + GW + Kp + nseg * Kp) * sizeof(float);
+        nsplit = (B + WG_BG - 1) / WG_BG;
+        dim3 grid(C, nsplit);
+        SC_DISPATCH(dtype, (dw_wgrad_s1_kernel<T><<<grid, WG_THREADS, smem, L.stream>>>(
+                               (const T*)gu, (const T*)x, partials, len_in, len_out, B, C, Tt, K, Kp)));
+    } else {
+        nsplit = B;
+        SC_DISPATCH(dtype, (dw_wgrad_generic_kernel<T><<<C, 128, 0, L.stream>>>((const T*)gu, (const T*)x, partials,
+                                                                                 len_in, len_out, B, C, Tt, Tp, K, s)));
+    }
+    L.count();
+    reduce_partials(L, partials, nsplit, (int64_t)C * K, dwd, accumulate);
+}
+
+}  // namespace sc

@@ -1,0 +1,95 @@
+// Internal launcher interface between the C-ABI layer (api.cu) and the kernel files.
+// Every function enqueues on L.stream and returns; all pointers are device pointers.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace sc {
+
+struct Launch {
+    cudaStream_t stream;
+    int* status;          // device status word
+    int64_t* counter;     // host launch counter
+    void count(int n = 1) const { if (counter) *counter += n; }
+};
+
+// ---- lengths -------------------------------------------------------------------------------
+// len_out[b] = ceil(len_in[b]/stride); *nvalid = sum_b len_out[b]; flags lengths outside [1,T_in].
+void lengths(const Launch& L, const int* len_in, int B, int T_in, int stride, int* len_out, int* nvalid);
+
+// ---- depthwise ------------------------------------------------------------------------------
+// u[b,c,t] = sum_k wd[c,k] * x[b,c,t*s+k-P] (x masked by len_in), written as 0 for t >= len_out[b].
+void dw_fwd(const Launch& L, int dtype, const void* x, const void* wd, void* u, const int* len_in,
+            const int* len_out, int B, int C, int T, int Tp, int K, int s);
+// dx[b,c,tau] = [tau < len_in[b]] * (sum_{k,t: t*s+k-P=tau} wd[c,k]*gu[b,c,t] + add1 + add2)
+void dw_dgrad(const Launch& L, int dtype, const void* gu, const void* wd, void* dx, const void* add1,
+              const void* add2, const int* len_in, const int* len_out, int B, int C, int T, int Tp,
+              int K, int s);
+// dwd[c,k] (+)= sum_{b,t<len_out} gu[b,c,t] * x[b,c,t*s+k-P] (x masked by len_in).
+// partials: float [B*C*K] scratch.
+void dw_wgrad(const Launch& L, int dtype, const void* gu, const void* x, float* dwd, float* partials,
+              int accumulate, const int* len_in, const int* len_out, int B, int C, int T, int Tp,
+              int K, int s);
+size_t dw_wgrad_scratch_bytes(int B, int C, int K);
+// out = [t < len[b]] * (a + b + c)   (b, c nullable)
+void ew_add_masked(const Launch& L, int dtype, void* out, const void* a, const void* b, const void* c,
+                   const int* len, int B, int C, int T);
+
+// ---- pointwise, SIMT (any shape, fp32 accumulate) ------------------------------------------
+// v[b,o,t] = [t<len_out[b]] * (sum_c w[o,c]*u[b,c,t] + bias[o])
+void gemm_fwd_simt(const Launch& L, int dtype, const void* w, const void* u, const float* bias, void* v,
+                   const int* len_out, int B, int Cin, int Cout, int Tp);
+// gu[b,c,t] = sum_o w[o,c]*gv[b,o,t]
+void gemm_dgrad_simt(const Launch& L, int dtype, const void* w, const void* gv, void* gu, int B, int Cin,
+                     int Cout, int Tp);
+// dw[o,c] (+)= sum_{b,t} gv[b,o,t]*u[b,c,t];  partials: float [nsplit*Cout*Cin]
+void gemm_wgrad_simt(const Launch& L, int dtype, const void* gv, const void* u, float* dw, float* partials,
+                     int accumulate, int B, int Cin, int Cout, int Tp);
+size_t gemm_wgrad_simt_scratch_bytes(int B, int Cin, int Cout);
+// out[i] (+)= sum_s partials[s*n + i], fixed order
+void reduce_partials(const Launch& L, const float* partials, int nsplit, int64_t n, float* out, int accumulate);
+
+// ---- batch norm -----------------------------------------------------------------------------
+// Per-(b,channel) row moments over t < len_out[b]: partials[(b*C+o)] = (sum, M2 about the row mean).
+void bn_stats(const Launch& L, int dtype, const void* v, const int* len_out, int B, int C, int Tp,
+              float2* partials);
+// Merge partials in a fixed order. parts_per_b tiles of tile_w frames per sample.
+// mean/invstd [C]; scale_shift[o] = (gamma*invstd, beta - mean*gamma*invstd); running stats optional.
+void bn_finalize(const Launch& L, const float2* partials, int parts_per_b, int tile_w, const int* len_out,
+                 const int* nvalid, int B, int C, const float* gamma, const float* beta, float eps,
+                 float momentum, float* mean, float* invstd, float2* scale_shift, float* running_mean,
+                 float* running_var);
+// scale_shift from saved statistics (backward needs it for the gate of the relu-then-add variant).
+void bn_scale_shift(const Launch& L, const float* mean, const float* invstd, const float* gamma,
+                    const float* beta, float2* scale_shift, int C);
+
+struct ApplyArgs {
+    const void* v;  const float2* ss;            // main branch
+    int residual;                                  // 0 none, 1 identity, 2 projection
+    const void* xres;                              // identity source [B,C,Tp]
+    const void* vr; const float2* ss_r;          // projection branch
+    void* y; const int* len_out;
+    int B, C, Tp, has_relu, res_before_relu;
+};
+void bn_apply(const Launch& L, int dtype, const ApplyArgs& a);
+
+struct BnBwdArgs {
+    const void* g; const void* y; const void* v; const void* vr;
+    const float* mean; const float* invstd; const float* mean_r; const float* invstd_r;
+    const float2* ss;                              // for the relu-then-add gate
+    const int* len_out; const int* nvalid;
+    int B, C, Tp, has_bn, has_relu, res_before_relu, residual;
+    float4* partials;                              // [B*C]
+    float4* coef; float4* coef_r;                  // [C]: (k, c1, c2, unused)
+    void* gv; void* gvr; void* gres;               // outputs of the apply step (gvr: proj, gres: identity)
+};
+void bn_bwd_reduce(const Launch& L, int dtype, const BnBwdArgs& a);
+void bn_bwd_finalize(const Launch& L, const BnBwdArgs& a, const float* gamma, const float* gamma_r,
+                     float* dgamma, float* dbeta, float* dgamma_r, float* dbeta_r, float* dbias,
+                     int accumulate);
+void bn_bwd_apply(const Launch& L, int dtype, const BnBwdArgs& a);
+
+// masked copy: out = [t<len[b]] ? in : 0
+void mask_copy(const Launch& L, int dtype, void* out, const void* in, const int* len, int B, int C, int T);
+
+}  // namespace sc

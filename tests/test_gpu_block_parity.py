@@ -1,0 +1,141 @@
+"""GPU parity of sepconv_fwd / sepconv_bwd (through the C ABI) against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import synth_inputs as si
+from tests import parity_util as U
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def api():
+    import paper_1909_09577_b200 as api
+    return api
+
+
+@pytest.fixture(scope="module")
+def ctx(api):
+    c = api.Context(0)
+    yield c
+    c.close()
+
+
+def _draw_block(L, B, T, dtype, seed, ragged, affine="random", lo_frac=0.25):
+    w = si.Workload("t", dtype, B, T, [L], seed, len_lo=max(1, int(T * lo_frac)) if ragged else None,
+                    len_hi=T if ragged else None, affine=affine)
+    return si.draw(w)
+
+
+SMALL = [
+    # (layer kwargs, B, T, ragged)
+    (dict(C_in=8, C_out=8, K=5, residual="identity"), 3, 40, True),
+    (dict(C_in=24, C_out=40, K=9, residual="proj"), 3, 77, True),          # T not a multiple of 8
+    (dict(C_in=16, C_out=32, K=33, stride=2, residual="none"), 2, 130, True),
+    (dict(C_in=16, C_out=32, K=7, stride=2, residual="none"), 2, 131, True),   # odd T with stride 2
+    (dict(C_in=16, C_out=16, K=11, residual="identity", res_before_relu=False), 2, 64, True),
+    (dict(C_in=16, C_out=24, K=3, residual="proj", res_before_relu=False), 2, 64, True),
+    (dict(C_in=64, C_out=29, K=1, has_dw=False, has_bn=False, has_relu=False, has_bias=True), 3, 50, True),
+    (dict(C_in=32, C_out=64, K=1, has_dw=False), 3, 48, True),
+    (dict(C_in=8, C_out=8, K=87, residual="none"), 2, 300, True),          # halo wider than some samples
+    (dict(C_in=130, C_out=70, K=15, residual="proj"), 2, 520, False),      # several tiles + ragged channel tail
+    (dict(C_in=8, C_out=8, K=3, has_relu=False), 2, 33, True),
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
+@pytest.mark.parametrize("case", range(len(SMALL)))
+def test_small_blocks(api, ctx, dtype, case):
+    kw, B, T, ragged = SMALL[case]
+    L = si.LayerCfg(**kw)
+    d = _draw_block(L, B, T, dtype, seed=100 + case, ragged=ragged)
+    rep = U.run_block(ctx, api, L, dtype, d.x, d.lengths, d.params[0], d.g)
+    rep.check()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_len_one_and_full(api, ctx, dtype):
+    L = si.LayerCfg(16, 16, K=9, residual="identity")
+    d = _draw_block(L, 4, 64, dtype, seed=7, ragged=False)
+    d.lengths[:] = [1, 64, 2, 63]
+    U.run_block(ctx, api, L, dtype, d.x, d.lengths, d.params[0], d.g).check()
+
+
+def test_external_residual_and_dx_add(api, ctx):
+    """Residual taken from another tensor (as the encoder's blocks do), its gradient returned
+    separately, and an extra gradient folded into dx."""
+    rng = np.random.default_rng(3)
+    L = si.LayerCfg(32, 48, K=7, residual="proj", C_res_override=16)
+    d = _draw_block(L, 3, 96, "bf16", seed=8, ragged=True)
+    x_res = si.quantise(rng.standard_normal((3, 16, 96)).astype(np.float32), "bf16")
+    dx_add = si.quantise(rng.standard_normal((3, 32, 96)).astype(np.float32), "bf16")
+    U.run_block(ctx, api, L, "bf16", d.x, d.lengths, d.params[0], d.g, x_res=x_res, want_dx_res=True,
+                dx_add=dx_add).check()
+
+
+@pytest.mark.parametrize("i", [1, 2, 3])
+@pytest.mark.parametrize("affine", ["unit", "random"])
+def test_benchmark_block_configs(api, ctx, i, affine):
+    """Configs 1-3 at full size, seeds as specified; reports error/allowed per tensor."""
+    w = si.config(i, affine=affine)
+    d = si.draw(w)
+    rep = U.run_block(ctx, api, w.layers[0], w.dtype, d.x, d.lengths, d.params[0], d.g)
+    print(f"\nconfig {i} ({affine}) error/allowed: {rep}; adopted gates {rep.adopted}")
+    rep.check()
+
+
+def test_gradient_accumulation(api, ctx):
+    L = si.LayerCfg(16, 24, K=5, residual="proj")
+    d = _draw_block(L, 2, 48, "f32", seed=5, ragged=True)
+    desc = api.block_desc(L, 2, 48, "f32")
+    xd, pd = U.dev(d.x, "f32"), U.params_dev(d.params[0], "f32")
+    ld = torch.from_numpy(d.lengths).cuda()
+    y, _, saved = api.sepconv_fwd(ctx, desc, xd, ld, pd)
+    gd = U.dev(d.g, "f32")
+    _, _, g1 = api.sepconv_bwd(ctx, desc, gd, xd, y, ld, pd, saved)
+    g2 = {k: v.clone() for k, v in g1.items()}
+    api.sepconv_bwd(ctx, desc, gd, xd, y, ld, pd, saved, grads=g2, accumulate=True)
+    for k in g1:
+        torch.testing.assert_close(g2[k], 2 * g1[k], rtol=1e-6, atol=1e-7)
+
+
+def test_bitwise_repeatable(api, ctx):
+    w = si.config(3)
+    d = si.draw(w)
+    L = w.layers[0]
+    desc = api.block_desc(L, w.B, w.T, w.dtype)
+    xd, pd = U.dev(d.x, w.dtype), U.params_dev(d.params[0], w.dtype)
+    ld = torch.from_numpy(d.lengths).cuda()
+    gd = U.dev(d.g, w.dtype)
+    outs = []
+    for _ in range(2):
+        y, _, saved = api.sepconv_fwd(ctx, desc, xd, ld, pd)
+        dx, _, grads = api.sepconv_bwd(ctx, desc, gd, xd, y, ld, pd, saved)
+        outs.append([y, dx] + [grads[k] for k in sorted(grads)])
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+
+
+def test_running_stats(api, ctx):
+    from oracle import sepconv_oracle as O
+    L = si.LayerCfg(8, 12, K=5)
+    d = _draw_block(L, 3, 40, "f32", seed=2, ragged=True)
+    desc = api.block_desc(L, 3, 40, "f32")
+    rm = torch.zeros(12, device="cuda"); rv = torch.ones(12, device="cuda")
+    api.sepconv_fwd(ctx, desc, U.dev(d.x, "f32"), torch.from_numpy(d.lengths).cuda(), U.params_dev(d.params[0], "f32"),
+                    running_mean=rm, running_var=rv)
+    S = O.block_fwd(L, d.x, d.lengths, d.params[0])
+    erm, erv = O.running_stats_update(np.zeros(12), np.ones(12), S["mean"], S["var"], S["N"])
+    np.testing.assert_allclose(rm.cpu().numpy(), erm, rtol=1e-4, atol=1e-6)
+    np.testing.assert_allclose(rv.cpu().numpy(), erv, rtol=1e-4, atol=1e-6)
+
+
+def test_invalid_length_sets_status(api, ctx):
+    L = si.LayerCfg(8, 8, K=3)
+    d = _draw_block(L, 2, 32, "f32", seed=1, ragged=False)
+    desc = api.block_desc(L, 2, 32, "f32")
+    bad = torch.tensor([0, 40], dtype=torch.int32, device="cuda")
+    api.sepconv_fwd(ctx, desc, U.dev(d.x, "f32"), bad, U.params_dev(d.params[0], "f32"))
+    assert ctx.last_status() == -8
+    assert ctx.last_status() == 0      # cleared by the read
