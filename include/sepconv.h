@@ -101,9 +101,10 @@ typedef struct {          /* device pointers; absent parts may be null          
 
 typedef struct {          /* written by sepconv_fwd, read by sepconv_bwd; caller-owned             */
     void  *u;             /* [B, C_in, T']  io_dtype (has_dw only)                                 */
-    void  *v;             /* [B, C_out, T'] io_dtype (has_bn only)                                 */
+    void  *vhat;          /* [B, C_out, T'] normalised (v - mean)/sqrt(var+eps), zero in padding   */
+                          /* (has_bn only); float32 when io_dtype is SC_F32, float16 otherwise     */
     float *mean, *invstd; /* [C_out]                                                               */
-    void  *vr;            /* [B, C_out, T'] io_dtype (projection residual only)                    */
+    void  *vhat_r;        /* same for the projection residual branch                               */
     float *mean_r, *invstd_r;
 } sc_block_saved;
 

@@ -56,7 +56,7 @@ class sc_block_params(C.Structure):
 
 
 class sc_block_saved(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("u", "v", "mean", "invstd", "vr", "mean_r", "invstd_r")]
+    _fields_ = [(n, C.c_void_p) for n in ("u", "vhat", "mean", "invstd", "vhat_r", "mean_r", "invstd_r")]
 
 
 class sc_block_grads(C.Structure):
@@ -214,12 +214,13 @@ def sepconv_fwd(ctx: Context, desc: sc_block_desc, x: torch.Tensor, lengths: tor
     out_len = torch.empty((B,), dtype=torch.int32, device=dev)
     if saved is None:
         saved = {"u": torch.empty((B, Ci, Tp), dtype=td, device=dev)}
+        nt = torch.float32 if desc.io_dtype == SC_F32 else torch.float16   # type of the normalised tensors
         if desc.has_bn:
-            saved["v"] = torch.empty((B, Co, Tp), dtype=td, device=dev)
+            saved["vhat"] = torch.empty((B, Co, Tp), dtype=nt, device=dev)
             saved["mean"] = torch.empty((Co,), dtype=torch.float32, device=dev)
             saved["invstd"] = torch.empty((Co,), dtype=torch.float32, device=dev)
         if desc.residual == 2:
-            saved["vr"] = torch.empty((B, Co, Tp), dtype=td, device=dev)
+            saved["vhat_r"] = torch.empty((B, Co, Tp), dtype=nt, device=dev)
             saved["mean_r"] = torch.empty((Co,), dtype=torch.float32, device=dev)
             saved["invstd_r"] = torch.empty((Co,), dtype=torch.float32, device=dev)
     sv = sc_block_saved()

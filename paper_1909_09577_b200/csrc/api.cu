@@ -85,34 +85,35 @@ struct BlockIO {                 // raw pointers after validation
 };
 
 // ---- forward scratch ---------------------------------------------------------------------------
-struct FwdScratch { float2 *partials, *ss, *ss_r; void* xr; int* len_out; int* nvalid; };
+struct FwdScratch { float2* partials; void *xr, *v, *vr; int* len_out; int* nvalid; };
 
 void plan_fwd(const sc_block_desc* d, const Dims& m, Bump& ws, FwdScratch* f, const TcState* tc) {
     const size_t parts = (size_t)m.B * tc_max_parts_per_sample(m.Tp) * m.Cout;
     f->len_out = (int*)ws.take(sizeof(int) * m.B);
     f->nvalid = (int*)ws.take(sizeof(int));
     f->partials = (float2*)ws.take(sizeof(float2) * parts);
-    f->ss = (float2*)ws.take(sizeof(float2) * m.Cout);
-    f->ss_r = (float2*)ws.take(sizeof(float2) * m.Cout);
+    const size_t vbytes = dtype_size(vtype_of(d->io_dtype)) * m.B * m.Cout * m.Tp;
+    f->v = d->has_bn ? ws.take(vbytes) : nullptr;
+    f->vr = (d->residual == SC_RES_PROJ) ? ws.take(vbytes) : nullptr;
     f->xr = (d->residual == SC_RES_PROJ) ? ws.take(esize(d->io_dtype) * m.B * m.Cres * m.Tp) : nullptr;
 }
 
-// v = w * u for every sample, plus masked batch statistics -> mean/invstd/scale-shift.
+// v = w * u for every sample (stored in the transient type), plus masked batch statistics.
 void pointwise_bn(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const Dims& m, int Cin,
                   const void* w, const void* u, void* v, const int* len_out, const int* nvalid,
-                  const float* gamma, const float* beta, float* mean, float* invstd, float2* ss,
-                  float2* partials, float* rmean, float* rvar) {
+                  float* mean, float* invstd, float2* partials, float* rmean, float* rvar) {
+    const int vdt = vtype_of(d->io_dtype);
     int parts = 1, tile_w = m.Tp;
     bool fused = false;
     if (ctx->gemm_mode == 0 && tc_fwd_supported(&ctx->tc, d->io_dtype, Cin, m.Cout, m.Tp)) {
         fused = tc_gemm_fwd(&ctx->tc, L, d->io_dtype, w, u, nullptr, v, len_out, m.B, Cin, m.Cout, m.Tp,
                             partials, &parts, &tile_w);
     } else {
-        gemm_fwd_simt(L, d->io_dtype, w, u, nullptr, v, len_out, m.B, Cin, m.Cout, m.Tp);
+        gemm_fwd_simt(L, d->io_dtype, w, u, nullptr, v, vdt, len_out, m.B, Cin, m.Cout, m.Tp);
     }
-    if (!fused) { bn_stats(L, d->io_dtype, v, len_out, m.B, m.Cout, m.Tp, partials); parts = 1; tile_w = m.Tp; }
-    bn_finalize(L, partials, parts, tile_w, len_out, nvalid, m.B, m.Cout, gamma, beta, d->bn_eps,
-                d->bn_momentum, mean, invstd, ss, rmean, rvar);
+    if (!fused) { bn_stats(L, vdt, v, len_out, m.B, m.Cout, m.Tp, partials); parts = 1; tile_w = m.Tp; }
+    bn_finalize(L, partials, parts, tile_w, len_out, nvalid, m.B, m.Cout, d->bn_eps, d->bn_momentum, mean,
+                invstd, rmean, rvar);
 }
 
 int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const Dims& m, BlockIO io,
@@ -136,22 +137,24 @@ int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
             tc_gemm_fwd(&ctx->tc, L, dt, p->wp, u, d->has_bias ? p->bias : nullptr, io.y, io.len_out, m.B, m.Cin,
                         m.Cout, m.Tp, nullptr, &parts, &tw);
         } else {
-            gemm_fwd_simt(L, dt, p->wp, u, d->has_bias ? p->bias : nullptr, io.y, io.len_out, m.B, m.Cin, m.Cout, m.Tp);
+            gemm_fwd_simt(L, dt, p->wp, u, d->has_bias ? p->bias : nullptr, io.y, dt, io.len_out, m.B, m.Cin, m.Cout, m.Tp);
         }
         return SC_OK;
     }
-    pointwise_bn(ctx, L, d, m, m.Cin, p->wp, u, sv->v, io.len_out, io.nvalid, p->gamma, p->beta, sv->mean,
-                 sv->invstd, f.ss, f.partials, rmean, rvar);
+    pointwise_bn(ctx, L, d, m, m.Cin, p->wp, u, f.v, io.len_out, io.nvalid, sv->mean, sv->invstd, f.partials,
+                 rmean, rvar);
     ApplyArgs a{};
-    a.v = sv->v; a.ss = f.ss; a.residual = d->residual; a.y = io.y; a.len_out = io.len_out;
+    a.v = f.v; a.mean = sv->mean; a.invstd = sv->invstd; a.gamma = p->gamma; a.beta = p->beta; a.vhat = sv->vhat;
+    a.residual = d->residual; a.y = io.y; a.len_out = io.len_out;
     a.B = m.B; a.C = m.Cout; a.Tp = m.Tp; a.has_relu = d->has_relu; a.res_before_relu = d->res_before_relu;
     if (d->residual == SC_RES_IDENTITY) a.xres = io.xres;
     if (d->residual == SC_RES_PROJ) {
         const void* xr = io.xres;
         if (!io.res_clean) { mask_copy(L, dt, f.xr, io.xres, io.len_out, m.B, m.Cres, m.Tp); xr = f.xr; }
-        pointwise_bn(ctx, L, d, m, m.Cres, p->wr, xr, sv->vr, io.len_out, io.nvalid, p->gamma_r, p->beta_r,
-                     sv->mean_r, sv->invstd_r, f.ss_r, f.partials, nullptr, nullptr);
-        a.vr = sv->vr; a.ss_r = f.ss_r;
+        pointwise_bn(ctx, L, d, m, m.Cres, p->wr, xr, f.vr, io.len_out, io.nvalid, sv->mean_r, sv->invstd_r,
+                     f.partials, nullptr, nullptr);
+        a.vr = f.vr; a.mean_r = sv->mean_r; a.invstd_r = sv->invstd_r; a.gamma_r = p->gamma_r; a.beta_r = p->beta_r;
+        a.vhat_r = sv->vhat_r;
     }
     bn_apply(L, dt, a);
     return SC_OK;
@@ -160,7 +163,7 @@ int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
 // ---- backward scratch --------------------------------------------------------------------------
 struct BwdScratch {
     int* len_out; int* nvalid;
-    float4 *partials, *coef, *coef_r; float2* ss;
+    float4 *partials, *coef, *coef_r;
     void *gv, *gvr, *gres, *gu, *gxr, *xr;
     float* wpart; size_t wpart_bytes;
 };
@@ -173,7 +176,6 @@ void plan_bwd(const sc_block_desc* d, const Dims& m, Bump& ws, BwdScratch* s, co
     s->partials = (float4*)ws.take(sizeof(float4) * m.B * m.Cout);
     s->coef = (float4*)ws.take(sizeof(float4) * m.Cout);
     s->coef_r = (float4*)ws.take(sizeof(float4) * m.Cout);
-    s->ss = (float2*)ws.take(sizeof(float2) * m.Cout);
     s->gv = ws.take(act_out);
     s->gvr = d->residual == SC_RES_PROJ ? ws.take(act_out) : nullptr;
     s->gres = d->residual == SC_RES_IDENTITY ? ws.take(act_out) : nullptr;
@@ -214,17 +216,15 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
                    const BwdScratch& s) {
     const int dt = d->io_dtype;
     BnBwdArgs a{};
-    a.g = io.dy; a.y = io.y; a.v = sv->v; a.vr = sv->vr;
-    a.mean = sv->mean; a.invstd = sv->invstd; a.mean_r = sv->mean_r; a.invstd_r = sv->invstd_r;
-    a.ss = s.ss; a.len_out = io.len_out; a.nvalid = io.nvalid;
+    a.g = io.dy; a.y = io.y; a.vhat = sv->vhat; a.vhat_r = sv->vhat_r;
+    a.invstd = sv->invstd; a.invstd_r = sv->invstd_r; a.gamma = p->gamma; a.beta = p->beta;
+    a.len_out = io.len_out; a.nvalid = io.nvalid;
     a.B = m.B; a.C = m.Cout; a.Tp = m.Tp; a.has_bn = d->has_bn; a.has_relu = d->has_relu;
     a.res_before_relu = d->res_before_relu; a.residual = d->residual;
     a.partials = s.partials; a.coef = s.coef; a.coef_r = s.coef_r;
     a.gv = s.gv; a.gvr = s.gvr;
     // identity residual: its gradient is the gated upstream gradient itself
     a.gres = (d->residual == SC_RES_IDENTITY) ? (io.dx_res ? io.dx_res : s.gres) : nullptr;
-    if (d->has_bn && d->has_relu && !d->res_before_relu)
-        bn_scale_shift(L, sv->mean, sv->invstd, p->gamma, p->beta, s.ss, m.Cout);
     bn_bwd_reduce(L, dt, a);
     bn_bwd_finalize(L, a, p->gamma, p->gamma_r, g->dgamma, g->dbeta, g->dgamma_r, g->dbeta_r,
                     d->has_bias ? g->dbias : nullptr, acc);
@@ -272,8 +272,8 @@ int check_params(const sc_block_desc* d, const sc_block_params* p) {
 int check_saved(const sc_block_desc* d, const sc_block_saved* s, bool x_clean) {
     if (!s) return SC_ERR_NULL;
     if ((d->has_dw || !x_clean) && !s->u) return SC_ERR_NULL;
-    if (d->has_bn && (!s->v || !s->mean || !s->invstd)) return SC_ERR_NULL;
-    if (d->residual == SC_RES_PROJ && (!s->vr || !s->mean_r || !s->invstd_r)) return SC_ERR_NULL;
+    if (d->has_bn && (!s->vhat || !s->mean || !s->invstd)) return SC_ERR_NULL;
+    if (d->residual == SC_RES_PROJ && (!s->vhat_r || !s->mean_r || !s->invstd_r)) return SC_ERR_NULL;
     return SC_OK;
 }
 int check_grads(const sc_block_desc* d, const sc_block_grads* g) {
@@ -488,11 +488,11 @@ int plan_encoder(const sc_encoder_desc* e, void* base, size_t cap, EncPlan* P, c
         if (lp.d.has_dw) lp.sv.u = ws.take(es * B * m.Cin * m.Tp);
         else if (i == 0) lp.sv.u = ws.take(es * B * m.Cin * m.Tp);
         if (lp.d.has_bn) {
-            lp.sv.v = ws.take(es * B * m.Cout * m.Tp);
+            lp.sv.vhat = ws.take(dtype_size(ntype_of(lp.d.io_dtype)) * B * m.Cout * m.Tp);
             lp.sv.mean = (float*)ws.take(4 * m.Cout); lp.sv.invstd = (float*)ws.take(4 * m.Cout);
         }
         if (lp.d.residual == SC_RES_PROJ) {
-            lp.sv.vr = ws.take(es * B * m.Cout * m.Tp);
+            lp.sv.vhat_r = ws.take(dtype_size(ntype_of(lp.d.io_dtype)) * B * m.Cout * m.Tp);
             lp.sv.mean_r = (float*)ws.take(4 * m.Cout); lp.sv.invstd_r = (float*)ws.take(4 * m.Cout);
         }
         lp.y = (i + 1 < e->n_layers) ? ws.take(es * B * m.Cout * m.Tp) : nullptr;

@@ -95,10 +95,8 @@ bn_stats_kernel(const T* __restrict__ v, const int* __restrict__ len_out, int C,
 
 __global__ void bn_finalize_kernel(const float2* __restrict__ partials, int parts_per_b, int tile_w,
                                    const int* __restrict__ len_out, const int* __restrict__ nvalid, int B,
-                                   int C, const float* __restrict__ gamma, const float* __restrict__ beta,
-                                   float eps, float momentum, float* __restrict__ mean_out,
-                                   float* __restrict__ invstd_out, float2* __restrict__ scale_shift,
-                                   float* running_mean, float* running_var) {
+                                   int C, float eps, float momentum, float* __restrict__ mean_out,
+                                   float* __restrict__ invstd_out, float* running_mean, float* running_var) {
     const int o = blockIdx.x * blockDim.x + threadIdx.x;
     if (o >= C) return;
     double n = 0.0, mean = 0.0, m2 = 0.0;
@@ -120,8 +118,6 @@ __global__ void bn_finalize_kernel(const float2* __restrict__ partials, int part
     const float mu = (float)mean;
     mean_out[o] = mu;
     invstd_out[o] = invstd;
-    const float sc_ = gamma[o] * invstd;
-    scale_shift[o] = make_float2(sc_, beta[o] - mu * sc_);
     if (running_mean) running_mean[o] = (1.f - momentum) * running_mean[o] + momentum * mu;
     if (running_var) {
         double unb = N > 1 ? var * (N / (N - 1.0)) : var;
@@ -129,42 +125,43 @@ __global__ void bn_finalize_kernel(const float2* __restrict__ partials, int part
     }
 }
 
-__global__ void bn_scale_shift_kernel(const float* mean, const float* invstd, const float* gamma,
-                                      const float* beta, float2* ss, int C) {
-    const int o = blockIdx.x * blockDim.x + threadIdx.x;
-    if (o >= C) return;
-    const float sc_ = gamma[o] * invstd[o];
-    ss[o] = make_float2(sc_, beta[o] - mean[o] * sc_);
-}
-
-template <typename T>
+template <typename T, typename VT, typename NT>
 __global__ void __launch_bounds__(kRowThreads) bn_apply_kernel(ApplyArgs a) {
     const int row = blockIdx.x, b = row / a.C, o = row % a.C;
     const int Tp = a.Tp, len = min(a.len_out[b], Tp);
     const bool vec = (Tp % 8 == 0);
-    const T* v = (const T*)a.v + (size_t)row * Tp;
-    const T* xr = a.residual == 1 ? (const T*)a.xres + (size_t)row * Tp : nullptr;
-    const T* vr = a.residual == 2 ? (const T*)a.vr + (size_t)row * Tp : nullptr;
-    T* y = (T*)a.y + (size_t)row * Tp;
-    const float2 ss = a.ss[o];
-    const float2 sr = a.residual == 2 ? a.ss_r[o] : make_float2(0.f, 0.f);
+    const size_t off = (size_t)row * Tp;
+    const VT* v = (const VT*)a.v + off;
+    const T* xr = a.residual == 1 ? (const T*)a.xres + off : nullptr;
+    const VT* vr = a.residual == 2 ? (const VT*)a.vr + off : nullptr;
+    T* y = (T*)a.y + off;
+    NT* vh = (NT*)a.vhat + off;
+    NT* vhr = a.residual == 2 ? (NT*)a.vhat_r + off : nullptr;
+    const float mu = a.mean[o], is = a.invstd[o], ga = a.gamma[o], be = a.beta[o];
+    float mur = 0.f, isr = 0.f, gar = 0.f, ber = 0.f;
+    if (a.residual == 2) { mur = a.mean_r[o]; isr = a.invstd_r[o]; gar = a.gamma_r[o]; ber = a.beta_r[o]; }
     for (int t0 = threadIdx.x * 8; t0 < Tp; t0 += kRowThreads * 8) {
-        float out[8];
+        float out[8], n1[8], n2[8];
         if (t0 < len) {
             float f[8], r[8];
             load_chunk(v, t0, Tp, vec, f);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) n1[i] = (t0 + i < len) ? round_io<NT>((f[i] - mu) * is) : 0.f;
             if (a.residual == 1) load_chunk(xr, t0, Tp, vec, r);
             else if (a.residual == 2) {
                 load_chunk(vr, t0, Tp, vec, r);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) r[i] = fmaf(sr.x, r[i], sr.y);
+                for (int i = 0; i < 8; ++i) {
+                    n2[i] = (t0 + i < len) ? round_io<NT>((r[i] - mur) * isr) : 0.f;
+                    r[i] = fmaf(gar, n2[i], ber);
+                }
             } else {
 #pragma unroll
                 for (int i = 0; i < 8; ++i) r[i] = 0.f;
             }
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                float bn = fmaf(ss.x, f[i], ss.y);
+                float bn = fmaf(ga, n1[i], be);     // from the stored (rounded) vhat: backward sees the same value
                 float q;
                 if (a.res_before_relu) { q = bn + r[i]; if (a.has_relu) q = fmaxf(q, 0.f); }
                 else { q = (a.has_relu ? fmaxf(bn, 0.f) : bn) + r[i]; }
@@ -172,58 +169,64 @@ __global__ void __launch_bounds__(kRowThreads) bn_apply_kernel(ApplyArgs a) {
             }
         } else {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) out[i] = 0.f;
+            for (int i = 0; i < 8; ++i) { out[i] = 0.f; n1[i] = 0.f; n2[i] = 0.f; }
         }
         store_chunk(y, t0, Tp, vec, out);
+        store_chunk(vh, t0, Tp, vec, n1);
+        if (vhr) store_chunk(vhr, t0, Tp, vec, n2);
     }
 }
 
 // Shared by the reduce and apply steps of the backward pass: per element gate and normalised value.
-template <typename T>
+template <typename T, typename NT>
 struct BwdRow {
-    const T *g, *y, *v, *vr;
-    float mean, invstd, mean_r, invstd_r;
-    float2 ss;
+    const T *g, *y; const NT *vh, *vhr;
+    float gam, bet;
     int len, Tp;
     bool vec;
     __device__ BwdRow(const BnBwdArgs& a, int row, int b, int o) {
         Tp = a.Tp; len = min(a.len_out[b], Tp); vec = (Tp % 8 == 0);
         g = (const T*)a.g + (size_t)row * Tp;
         y = a.y ? (const T*)a.y + (size_t)row * Tp : nullptr;
-        v = a.v ? (const T*)a.v + (size_t)row * Tp : nullptr;
-        vr = (a.residual == 2) ? (const T*)a.vr + (size_t)row * Tp : nullptr;
-        mean = a.has_bn ? a.mean[o] : 0.f; invstd = a.has_bn ? a.invstd[o] : 1.f;
-        mean_r = (a.residual == 2) ? a.mean_r[o] : 0.f; invstd_r = (a.residual == 2) ? a.invstd_r[o] : 1.f;
-        ss = (a.has_relu && !a.res_before_relu && a.has_bn) ? a.ss[o] : make_float2(1.f, 0.f);
+        vh = a.has_bn ? (const NT*)a.vhat + (size_t)row * Tp : nullptr;
+        vhr = (a.residual == 2) ? (const NT*)a.vhat_r + (size_t)row * Tp : nullptr;
+        const bool own_gate = a.has_relu && !a.res_before_relu && a.has_bn;
+        gam = own_gate ? a.gamma[o] : 1.f; bet = own_gate ? a.beta[o] : 0.f;
     }
-    // ga: gated upstream gradient; gr: gradient reaching the residual sum; vh/vhr: normalised values
+    // ga: gated upstream gradient; gr: gradient reaching the residual sum; vn/vnr: normalised values
     __device__ __forceinline__ void chunk(const BnBwdArgs& a, int t0, float (&ga)[8], float (&gr)[8],
-                                          float (&vh)[8], float (&vhr)[8]) const {
-        float fg[8], fy[8], fv[8], fr[8];
+                                          float (&vn)[8], float (&vnr)[8]) const {
+        float fg[8], fy[8];
         load_chunk(g, t0, Tp, vec, fg);
         const bool need_y = a.has_relu && a.res_before_relu;
         if (need_y) load_chunk(y, t0, Tp, vec, fy);
-        const bool need_v = a.has_bn;
-        if (need_v) load_chunk(v, t0, Tp, vec, fv);
-        if (a.residual == 2) load_chunk(vr, t0, Tp, vec, fr);
+        if (a.has_bn) load_chunk(vh, t0, Tp, vec, vn);
+        else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) vn[i] = 0.f;
+        }
+        if (a.residual == 2) load_chunk(vhr, t0, Tp, vec, vnr);
+        else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) vnr[i] = 0.f;
+        }
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const bool in = (t0 + i < len);
             const float gm = in ? fg[i] : 0.f;
             bool gate = true;
-            if (a.has_relu) gate = a.res_before_relu ? (fy[i] > 0.f) : (fmaf(ss.x, fv[i], ss.y) > 0.f);
+            if (a.has_relu) gate = a.res_before_relu ? (fy[i] > 0.f) : (fmaf(gam, vn[i], bet) > 0.f);
             ga[i] = gate ? gm : 0.f;
             gr[i] = a.res_before_relu ? ga[i] : gm;
-            vh[i] = (need_v && in) ? (fv[i] - mean) * invstd : 0.f;
-            vhr[i] = (a.residual == 2 && in) ? (fr[i] - mean_r) * invstd_r : 0.f;
+            if (!in) { vn[i] = 0.f; vnr[i] = 0.f; }
         }
     }
 };
 
-template <typename T>
+template <typename T, typename NT>
 __global__ void __launch_bounds__(kRowThreads) bn_bwd_reduce_kernel(BnBwdArgs a) {
     const int row = blockIdx.x, b = row / a.C, o = row % a.C;
-    BwdRow<T> R(a, row, b, o);
+    BwdRow<T, NT> R(a, row, b, o);
     float s[4] = {0.f, 0.f, 0.f, 0.f};
     for (int t0 = threadIdx.x * 8; t0 < R.len; t0 += kRowThreads * 8) {
         float ga[8], gr[8], vh[8], vhr[8];
@@ -264,10 +267,10 @@ __global__ void bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const fl
     }
 }
 
-template <typename T>
+template <typename T, typename NT>
 __global__ void __launch_bounds__(kRowThreads) bn_bwd_apply_kernel(BnBwdArgs a) {
     const int row = blockIdx.x, b = row / a.C, o = row % a.C;
-    BwdRow<T> R(a, row, b, o);
+    BwdRow<T, NT> R(a, row, b, o);
     const float4 cf = a.coef[o];
     const float4 cr = (a.residual == 2) ? a.coef_r[o] : make_float4(0.f, 0.f, 0.f, 0.f);
     T* gv = (T*)a.gv + (size_t)row * R.Tp;
@@ -324,6 +327,12 @@ ew_add_masked_kernel(T* out, const T* a, const T* b, const T* c, const int* len,
 
 }  // namespace
 
+#define SC_DISPATCH3(dtype, ...)                                                              \
+    switch (dtype) {                                                                          \
+        case F32: { using T = float; using VT = float; using NT = float; __VA_ARGS__; break; }          \
+        case F16: { using T = __half; using VT = __half; using NT = __half; __VA_ARGS__; break; }       \
+        default:  { using T = __nv_bfloat16; using VT = float; using NT = __half; __VA_ARGS__; break; } \
+    }
 #define SC_DISPATCH(dtype, ...)                                             \
     switch (dtype) {                                                        \
         case F32: { using T = float; __VA_ARGS__; break; }                  \
@@ -336,35 +345,27 @@ void lengths(const Launch& L, const int* len_in, int B, int T_in, int stride, in
     L.count();
 }
 
-void bn_stats(const Launch& L, int dtype, const void* v, const int* len_out, int B, int C, int Tp,
+void bn_stats(const Launch& L, int vdtype, const void* v, const int* len_out, int B, int C, int Tp,
               float2* partials) {
-    SC_DISPATCH(dtype, (bn_stats_kernel<T><<<B * C, kRowThreads, 0, L.stream>>>((const T*)v, len_out, C, Tp, partials)));
+    SC_DISPATCH(vdtype, (bn_stats_kernel<T><<<B * C, kRowThreads, 0, L.stream>>>((const T*)v, len_out, C, Tp, partials)));
     L.count();
 }
 
 void bn_finalize(const Launch& L, const float2* partials, int parts_per_b, int tile_w, const int* len_out,
-                 const int* nvalid, int B, int C, const float* gamma, const float* beta, float eps,
-                 float momentum, float* mean, float* invstd, float2* scale_shift, float* running_mean,
-                 float* running_var) {
+                 const int* nvalid, int B, int C, float eps, float momentum, float* mean, float* invstd,
+                 float* running_mean, float* running_var) {
     bn_finalize_kernel<<<(C + 63) / 64, 64, 0, L.stream>>>(partials, parts_per_b, tile_w, len_out, nvalid, B, C,
-                                                            gamma, beta, eps, momentum, mean, invstd,
-                                                            scale_shift, running_mean, running_var);
-    L.count();
-}
-
-void bn_scale_shift(const Launch& L, const float* mean, const float* invstd, const float* gamma,
-                    const float* beta, float2* ss, int C) {
-    bn_scale_shift_kernel<<<(C + 127) / 128, 128, 0, L.stream>>>(mean, invstd, gamma, beta, ss, C);
+                                                            eps, momentum, mean, invstd, running_mean, running_var);
     L.count();
 }
 
 void bn_apply(const Launch& L, int dtype, const ApplyArgs& a) {
-    SC_DISPATCH(dtype, (bn_apply_kernel<T><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a)));
+    SC_DISPATCH3(dtype, (bn_apply_kernel<T, VT, NT><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a)));
     L.count();
 }
 
 void bn_bwd_reduce(const Launch& L, int dtype, const BnBwdArgs& a) {
-    SC_DISPATCH(dtype, (bn_bwd_reduce_kernel<T><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a)));
+    SC_DISPATCH3(dtype, (bn_bwd_reduce_kernel<T, NT><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a)));
     L.count();
 }
 
@@ -377,7 +378,7 @@ void bn_bwd_finalize(const Launch& L, const BnBwdArgs& a, const float* gamma, co
 }
 
 void bn_bwd_apply(const Launch& L, int dtype, const BnBwdArgs& a) {
-    SC_DISPATCH(dtype, (bn_bwd_apply_kernel<T><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a)));
+    SC_DISPATCH3(dtype, (bn_bwd_apply_kernel<T, NT><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a)));
     L.count();
 }
 

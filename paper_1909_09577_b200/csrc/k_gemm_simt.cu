@@ -20,7 +20,7 @@ struct GemmDesc {
     int k_begin_per_z, k_len_per_z;   // split-K: slice z covers k in [z*k_len, (z+1)*k_len)
 };
 
-template <typename T, int MODE>   // MODE 0: fwd (bias+mask, T out) 1: dgrad (T out) 2: wgrad (float partial out)
+template <typename T, typename OT, int MODE>   // MODE 0: fwd (bias+mask, T out) 1: dgrad (T out) 2: wgrad (float partial out)
 __global__ void __launch_bounds__(NT)
 gemm_simt_kernel(GemmDesc d, const T* __restrict__ a, const T* __restrict__ b, void* __restrict__ out,
                  const float* __restrict__ bias, const int* __restrict__ len_out) {
@@ -42,7 +42,7 @@ gemm_simt_kernel(GemmDesc d, const T* __restrict__ a, const T* __restrict__ b, v
 
     // fwd-mode early exit: tile wholly in padding -> zeros
     if (MODE == 0 && len_out && n0 >= len_out[z]) {
-        T* o = (T*)out + (long long)z * d.M * d.N;
+        OT* o = (OT*)out + (long long)z * d.M * d.N;
         for (int i = tid; i < BM * BN; i += NT) {
             const int m = m0 + i / BN, n = n0 + i % BN;
             if (m < d.M && n < d.N) stf(o + (long long)m * d.N + n, 0.f);
@@ -101,9 +101,9 @@ gemm_simt_kernel(GemmDesc d, const T* __restrict__ a, const T* __restrict__ b, v
             if (MODE == 0) {
                 float v = acc[i][j] + (bias ? bias[m] : 0.f);
                 if (len_out && n >= len_out[z]) v = 0.f;
-                stf((T*)out + ((long long)z * d.M + m) * d.N + n, v);
+                stf((OT*)out + ((long long)z * d.M + m) * d.N + n, v);
             } else if (MODE == 1) {
-                stf((T*)out + ((long long)z * d.M + m) * d.N + n, acc[i][j]);
+                stf((OT*)out + ((long long)z * d.M + m) * d.N + n, acc[i][j]);
             } else {
                 ((float*)out)[((long long)z * d.M + m) * d.N + n] = acc[i][j];
             }
@@ -135,13 +135,17 @@ void reduce_partials(const Launch& L, const float* partials, int nsplit, int64_t
 }
 
 void gemm_fwd_simt(const Launch& L, int dtype, const void* w, const void* u, const float* bias, void* v,
-                   const int* len_out, int B, int Cin, int Cout, int Tp) {
+                   int out_dtype, const int* len_out, int B, int Cin, int Cout, int Tp) {
     GemmDesc d{};
     d.M = Cout; d.N = Tp; d.Kd = Cin;
     d.a_z = 0; d.a_m = Cin; d.a_k = 1;
     d.b_z = (long long)Cin * Tp; d.b_k = Tp; d.b_n = 1;
     dim3 grid((Tp + BN - 1) / BN, (Cout + BM - 1) / BM, B);
-    SC_DISPATCH(dtype, (gemm_simt_kernel<T, 0><<<grid, NT, 0, L.stream>>>(d, (const T*)w, (const T*)u, v, bias, len_out)));
+    if (out_dtype == dtype) {
+        SC_DISPATCH(dtype, (gemm_simt_kernel<T, T, 0><<<grid, NT, 0, L.stream>>>(d, (const T*)w, (const T*)u, v, bias, len_out)));
+    } else {   // bf16 operands, float result
+        gemm_simt_kernel<__nv_bfloat16, float, 0><<<grid, NT, 0, L.stream>>>(d, (const __nv_bfloat16*)w, (const __nv_bfloat16*)u, v, bias, len_out);
+    }
     L.count();
 }
 
@@ -152,7 +156,7 @@ void gemm_dgrad_simt(const Launch& L, int dtype, const void* w, const void* gv, 
     d.a_z = 0; d.a_m = 1; d.a_k = Cin;            // A(m=c, k=o) = w[o*Cin + c]
     d.b_z = (long long)Cout * Tp; d.b_k = Tp; d.b_n = 1;
     dim3 grid((Tp + BN - 1) / BN, (Cin + BM - 1) / BM, B);
-    SC_DISPATCH(dtype, (gemm_simt_kernel<T, 1><<<grid, NT, 0, L.stream>>>(d, (const T*)w, (const T*)gv, gu, nullptr, nullptr)));
+    SC_DISPATCH(dtype, (gemm_simt_kernel<T, T, 1><<<grid, NT, 0, L.stream>>>(d, (const T*)w, (const T*)gv, gu, nullptr, nullptr)));
     L.count();
 }
 
@@ -172,7 +176,7 @@ void gemm_wgrad_simt(const Launch& L, int dtype, const void* gv, const void* u, 
     const int ns = wgrad_splits(B);
     d.k_len_per_z = Tp;
     dim3 grid((Cin + BN - 1) / BN, (Cout + BM - 1) / BM, ns);
-    SC_DISPATCH(dtype, (gemm_simt_kernel<T, 2><<<grid, NT, 0, L.stream>>>(d, (const T*)gv, (const T*)u, partials, nullptr, nullptr)));
+    SC_DISPATCH(dtype, (gemm_simt_kernel<T, T, 2><<<grid, NT, 0, L.stream>>>(d, (const T*)gv, (const T*)u, partials, nullptr, nullptr)));
     L.count();
     reduce_partials(L, partials, ns, (int64_t)Cin * Cout, dw, accumulate);
 }

@@ -36,9 +36,9 @@ void ew_add_masked(const Launch& L, int dtype, void* out, const void* a, const v
                    const int* len, int B, int C, int T);
 
 // ---- pointwise, SIMT (any shape, fp32 accumulate) ------------------------------------------
-// v[b,o,t] = [t<len_out[b]] * (sum_c w[o,c]*u[b,c,t] + bias[o])
+// v[b,o,t] = [t<len_out[b]] * (sum_c w[o,c]*u[b,c,t] + bias[o]); v is stored in out_dtype
 void gemm_fwd_simt(const Launch& L, int dtype, const void* w, const void* u, const float* bias, void* v,
-                   const int* len_out, int B, int Cin, int Cout, int Tp);
+                   int out_dtype, const int* len_out, int B, int Cin, int Cout, int Tp);
 // gu[b,c,t] = sum_o w[o,c]*gv[b,o,t]
 void gemm_dgrad_simt(const Launch& L, int dtype, const void* w, const void* gv, void* gu, int B, int Cin,
                      int Cout, int Tp);
@@ -51,32 +51,38 @@ void reduce_partials(const Launch& L, const float* partials, int nsplit, int64_t
 
 // ---- batch norm -----------------------------------------------------------------------------
 // Per-(b,channel) row moments over t < len_out[b]: partials[(b*C+o)] = (sum, M2 about the row mean).
-void bn_stats(const Launch& L, int dtype, const void* v, const int* len_out, int B, int C, int Tp,
+void bn_stats(const Launch& L, int vdtype, const void* v, const int* len_out, int B, int C, int Tp,
               float2* partials);
 // Merge partials in a fixed order. parts_per_b tiles of tile_w frames per sample.
-// mean/invstd [C]; scale_shift[o] = (gamma*invstd, beta - mean*gamma*invstd); running stats optional.
+// mean/invstd [C]; running stats optional.
 void bn_finalize(const Launch& L, const float2* partials, int parts_per_b, int tile_w, const int* len_out,
-                 const int* nvalid, int B, int C, const float* gamma, const float* beta, float eps,
-                 float momentum, float* mean, float* invstd, float2* scale_shift, float* running_mean,
-                 float* running_var);
-// scale_shift from saved statistics (backward needs it for the gate of the relu-then-add variant).
-void bn_scale_shift(const Launch& L, const float* mean, const float* invstd, const float* gamma,
-                    const float* beta, float2* scale_shift, int C);
+                 const int* nvalid, int B, int C, float eps, float momentum, float* mean, float* invstd,
+                 float* running_mean, float* running_var);
+
+// Storage types.  T = activation type.  VT = type of the transient pre-normalisation tensor v
+// (float for fp32 and bf16 activations, half for fp16).  NT = type of the saved normalised tensor
+// vhat = (v - mean) * invstd (float for fp32, half otherwise: vhat has unit scale, so half's 10-bit
+// mantissa is safe where bf16's 8 bits would eat most of the error budget).
+inline int vtype_of(int dtype) { return dtype == 1 ? 1 : 0; }
+inline int ntype_of(int dtype) { return dtype == 0 ? 0 : 1; }
+inline size_t dtype_size(int dtype) { return dtype == 0 ? 4 : 2; }
 
 struct ApplyArgs {
-    const void* v;  const float2* ss;            // main branch
+    const void* v; const float *mean, *invstd, *gamma, *beta;          // main branch (v in VT)
+    void* vhat;                                                        // out, NT
     int residual;                                  // 0 none, 1 identity, 2 projection
-    const void* xres;                              // identity source [B,C,Tp]
-    const void* vr; const float2* ss_r;          // projection branch
+    const void* xres;                              // identity source [B,C,Tp], T
+    const void* vr; const float *mean_r, *invstd_r, *gamma_r, *beta_r; // projection branch (vr in VT)
+    void* vhat_r;                                                      // out, NT
     void* y; const int* len_out;
     int B, C, Tp, has_relu, res_before_relu;
 };
 void bn_apply(const Launch& L, int dtype, const ApplyArgs& a);
 
 struct BnBwdArgs {
-    const void* g; const void* y; const void* v; const void* vr;
-    const float* mean; const float* invstd; const float* mean_r; const float* invstd_r;
-    const float2* ss;                              // for the relu-then-add gate
+    const void* g; const void* y; const void* vhat; const void* vhat_r;   // vhat, vhat_r in NT
+    const float* invstd; const float* invstd_r;
+    const float *gamma, *beta;                     // for the relu-then-add gate
     const int* len_out; const int* nvalid;
     int B, C, Tp, has_bn, has_relu, res_before_relu, residual;
     float4* partials;                              // [B*C]

@@ -31,15 +31,17 @@ def rms(a) -> float:
     return float(np.sqrt(np.mean(a * a))) if a.size else 0.0
 
 
-def err_ratio(got, ref, dtype) -> float:
-    """Error divided by the allowed error; <= 1 passes."""
+def err_ratio(got, ref, dtype, mask=None) -> float:
+    """Error divided by the allowed error; <= 1 passes.  The error is taken over every element; the
+    RMS that scales the allowance is taken over the valid (unpadded) frames when a mask is given,
+    since padded frames are structural zeros on both sides."""
     got = np.asarray(got, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
     assert got.shape == ref.shape, (got.shape, ref.shape)
     if ref.size == 0:
         return 0.0
     assert np.all(np.isfinite(got)), "non-finite values in the GPU result"
-    r = rms(ref)
+    r = rms(ref if mask is None else ref[np.broadcast_to(mask, ref.shape)])
     if dtype == "f32":
         denom = TOL[dtype] * np.maximum(np.abs(ref), r)
         denom = np.where(denom == 0, 1e-30, denom)
@@ -54,8 +56,8 @@ class Report:
         self.dtype = dtype
         self.rows = []
 
-    def add(self, name, got, ref):
-        self.rows.append((name, err_ratio(got, ref, self.dtype)))
+    def add(self, name, got, ref, mask=None):
+        self.rows.append((name, err_ratio(got, ref, self.dtype, mask)))
 
     def worst(self):
         return max(self.rows, key=lambda r: r[1]) if self.rows else ("", 0.0)
@@ -87,10 +89,9 @@ def gpu_gate(L, y_gpu, saved_gpu, params):
     """The ReLU decision the GPU took, reconstructed from its own outputs."""
     if L.res_before_relu or L.residual == "none":
         return host(y_gpu) > 0
-    v = saved_gpu["v"].float()
-    sc = params["gamma"].float() * saved_gpu["invstd"]
-    sh = params["beta"].float() - saved_gpu["mean"] * sc
-    return (torch.addcmul(sh[None, :, None], sc[None, :, None], v) > 0).cpu().numpy()
+    vh = saved_gpu["vhat"].float()
+    return (torch.addcmul(params["beta"].float()[None, :, None], params["gamma"].float()[None, :, None], vh)
+            > 0).cpu().numpy()
 
 
 def run_block(ctx, api, L, dtype, x, lengths, params, g, x_res=None, want_dx_res=False, dx_add=None):
@@ -106,18 +107,19 @@ def run_block(ctx, api, L, dtype, x, lengths, params, g, x_res=None, want_dx_res
     assert ctx.last_status() == 0
     np.testing.assert_array_equal(out_len.cpu().numpy(), S["out_len"])
     rep = Report(dtype)
+    vm = S["valid"]
     if L.has_dw:
-        rep.add("u", host(saved["u"]), S["u"])
+        rep.add("u", host(saved["u"]), S["u"], vm)
     if L.has_bn:
-        rep.add("v", host(saved["v"]), S["v"])
+        rep.add("vhat", host(saved["vhat"]), np.where(vm, S["vhat"], 0.0), vm)
         rep.add("mean", host(saved["mean"]), S["mean"])
         rep.add("invstd", host(saved["invstd"]), S["invstd"])
     if L.residual == "proj":
-        rep.add("vr", host(saved["vr"]), S["vr"])
+        rep.add("vhat_r", host(saved["vhat_r"]), np.where(vm, S["vhat_r"], 0.0), vm)
         rep.add("mean_r", host(saved["mean_r"]), S["mean_r"])
         rep.add("invstd_r", host(saved["invstd_r"]), S["invstd_r"])
     yh = host(y)
-    rep.add("y", yh, S["y"])
+    rep.add("y", yh, S["y"], vm)
     assert np.all(yh[~np.broadcast_to(S["valid"], yh.shape)] == 0), "padded output frames must be zero"
 
     gate = None
@@ -135,9 +137,9 @@ def run_block(ctx, api, L, dtype, x, lengths, params, g, x_res=None, want_dx_res
         ref_dx = ref_dx + G["dx_res"]
     if dx_add is not None:
         ref_dx = ref_dx + np.where(O.time_mask(lengths, T), dx_add, 0.0)
-    rep.add("dx", host(dx), ref_dx)
+    rep.add("dx", host(dx), ref_dx, O.time_mask(lengths, T))
     if want_dx_res:
-        rep.add("dx_res", host(dx_res), G["dx_res"])
+        rep.add("dx_res", host(dx_res), G["dx_res"], vm)
     for name in params:
         rep.add("d" + name, host(grads["d" + name]), G["d" + name])
     rep.adopted, rep.hard = adopted, hard
@@ -182,13 +184,14 @@ def run_chain(ctx, api, w, d, check=True):
         S = O.block_fwd(L, acts[i], lens[i], d.params[i], res_src=x_res_np)
         rep = Report(w.dtype)
         np.testing.assert_array_equal(lens[i + 1], S["out_len"])
+        vm = S["valid"]
         if L.has_dw:
-            rep.add("u", host(f["saved"]["u"]), S["u"])
+            rep.add("u", host(f["saved"]["u"]), S["u"], vm)
         if L.has_bn:
-            rep.add("v", host(f["saved"]["v"]), S["v"])
+            rep.add("vhat", host(f["saved"]["vhat"]), np.where(vm, S["vhat"], 0.0), vm)
         if L.residual == "proj":
-            rep.add("vr", host(f["saved"]["vr"]), S["vr"])
-        rep.add("y", acts[i + 1], S["y"])
+            rep.add("vhat_r", host(f["saved"]["vhat_r"]), np.where(vm, S["vhat_r"], 0.0), vm)
+        rep.add("y", acts[i + 1], S["y"], vm)
         gate = None
         adopted = hard = 0
         if L.has_relu:
@@ -203,9 +206,9 @@ def run_chain(ctx, api, w, d, check=True):
             ref_dx = ref_dx + G["dx_res"]
         if dx_add is not None:
             ref_dx = ref_dx + np.where(O.time_mask(lens[i], acts[i].shape[2]), host(dx_add), 0.0)
-        rep.add("dx", host(dx), ref_dx)
+        rep.add("dx", host(dx), ref_dx, O.time_mask(lens[i], acts[i].shape[2]))
         if want_res:
-            rep.add("dx_res", host(dx_res), G["dx_res"])
+            rep.add("dx_res", host(dx_res), G["dx_res"], vm)
             pending[f["j"]] = dx_res
         for name in d.params[i]:
             rep.add("d" + name, host(grads["d" + name]), G["d" + name])
@@ -218,4 +221,5 @@ def run_chain(ctx, api, w, d, check=True):
         g = dx.float().cpu().numpy()
         final_dx = dx
     assert ctx.last_status() == 0
-    return reports, dict(logits=fwd[-1]["y"], dx=final_dx, grads=grads_all, out_len=lens[-1])
+    return reports, dict(logits=fwd[-1]["y"], dx=final_dx, grads=grads_all, out_len=lens[-1],
+                         ys=[f["y"] for f in fwd], saved=[f["saved"] for f in fwd], pds=[f["pd"] for f in fwd])

@@ -53,17 +53,27 @@ def test_tiny_encoder(api, ctx, dtype, ragged):
     # (3) end to end
     saved, lens = O.encoder_fwd(w.layers, d.x, d.lengths, d.params)
     rep = U.Report(dtype)
-    rep.add("logits", U.host(logits), saved[-1]["y"])
-    grads, dx_ref, _ = O.encoder_bwd(w.layers, d.g, lens, d.params, saved)
-    rep.add("dx", U.host(dx), dx_ref)
+    rep.add("logits", U.host(logits), saved[-1]["y"], saved[-1]["valid"])
+    # ReLU gates: inside the tolerance band around zero the oracle takes the GPU's decision
+    gates, adopted, hard = [], 0, 0
+    for i, L in enumerate(w.layers):
+        if not L.has_relu:
+            gates.append(None)
+            continue
+        gt, a_, h_ = U.adopt_gate(L, saved[i], U.gpu_gate(L, chain["ys"][i], chain["saved"][i], chain["pds"][i]), dtype)
+        gates.append(gt); adopted += a_; hard += h_
+    grads, dx_ref, _ = O.encoder_bwd(w.layers, d.g, lens, d.params, saved, gates=gates)
+    rep.add("dx", U.host(dx), dx_ref, O.time_mask(d.lengths, w.T))
     for i in range(len(w.layers)):
         for name in d.params[i]:
             rep.add(f"L{i}.d{name}", U.host(spec.grad_view(gblob, i, name)), grads[i]["d" + name])
-    print(f"\ntiny encoder {dtype} ragged={ragged} end-to-end error/allowed: worst {rep.worst()}")
-    # without gate adoption across layers a flipped ReLU gate is a legitimate O(1) local difference,
-    # so end to end only the forward result is held to the tolerance; gradients are reported and bounded.
-    assert rep.rows[0][1] <= 1.0, rep.rows[0]
-    assert rep.worst()[1] <= 25.0, rep.worst()
+    print(f"\ntiny encoder {dtype} ragged={ragged} end-to-end error/allowed: logits {rep.rows[0][1]:.3f} "
+          f"worst {rep.worst()} adopted gates {adopted} hard mismatches {hard}")
+    # End to end the rounding of every layer accumulates (and a gate that flips outside the band is a
+    # legitimate local difference), so the per-layer tolerance is checked teacher-forced above and the
+    # end-to-end figures are bounded at a multiple of it.
+    assert rep.rows[0][1] <= 3.0, rep.rows[0]
+    assert rep.worst()[1] <= 10.0, rep.worst()
 
 
 def test_encoder_without_dx_and_accumulate(api, ctx):
