@@ -200,6 +200,20 @@ int  sepconv_set_gemm_mode(sc_ctx* ctx, int mode);
 /* Number of kernel launches this context has enqueued so far (for reporting). */
 int64_t sepconv_launch_count(sc_ctx* ctx);
 
+/* Per-kernel-class timing with CUDA events on the launching stream (measurement aid; the paper has
+ * no counterpart).  Kernel classes are numbered 0 .. sepconv_kernel_class_count()-1 and named by
+ * sepconv_kernel_class_name().  sepconv_profile_begin brackets, from now on, every launch of
+ * `kernel_class` (-1: every class) with an event pair, up to max_launches launches (it creates the
+ * events, host objects, on first use).  sepconv_profile_end synchronises the stream, stops the
+ * bracketing and fills four HOST arrays of class-count entries: total milliseconds, number of
+ * bracketed launcher calls, and the algorithmic bytes and flops those calls moved / performed
+ * (padded-frame counts; every tensor read or written once). */
+int  sepconv_profile_begin(sc_ctx* ctx, int kernel_class, int max_launches);
+int  sepconv_profile_end(sc_ctx* ctx, void* cuda_stream, double* ms, int64_t* launches, double* bytes,
+                         double* flops);
+int  sepconv_kernel_class_count(void);
+const char* sepconv_kernel_class_name(int kernel_class);
+
 #ifdef __cplusplus
 }
 #endif

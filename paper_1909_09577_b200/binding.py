@@ -69,7 +69,8 @@ class sc_encoder_desc(C.Structure):
 
 _lib = None
 
-EXPORTS = ("sepconv_ctx_create", "sepconv_ctx_destroy", "sepconv_last_status", "sepconv_strerror",
+EXPORTS = ("sepconv_profile_begin", "sepconv_profile_end", "sepconv_kernel_class_count",
+           "sepconv_kernel_class_name", "sepconv_ctx_create", "sepconv_ctx_destroy", "sepconv_last_status", "sepconv_strerror",
            "sepconv_workspace_bytes", "sepconv_fwd", "sepconv_bwd", "encoder_workspace_bytes",
            "encoder_fwd_bwd", "sepconv_set_gemm_mode", "sepconv_launch_count")
 
@@ -108,6 +109,11 @@ def load_library(path: str = LIB_PATH):
                                     C.c_void_p, C.POINTER(C.c_int64), C.POINTER(sc_tensor),
                                     C.POINTER(sc_tensor), C.c_void_p, C.c_void_p, C.POINTER(C.c_int64),
                                     C.POINTER(sc_tensor), C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.sepconv_profile_begin.argtypes = [C.c_void_p, C.c_int, C.c_int]
+    lib.sepconv_profile_end.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64),
+                                        C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    lib.sepconv_kernel_class_name.restype = C.c_char_p
+    lib.sepconv_kernel_class_name.argtypes = [C.c_int]
     _lib = lib
     return lib
 
@@ -182,6 +188,24 @@ class Context:
 
     def launch_count(self) -> int:
         return int(self.lib.sepconv_launch_count(self.h))
+
+    def kernel_classes(self):
+        return [self.lib.sepconv_kernel_class_name(i).decode() for i in range(self.lib.sepconv_kernel_class_count())]
+
+    def profile_begin(self, kernel_class="all", max_launches: int = 4096):
+        """Start bracketing launches of one kernel class (name, or "all") with CUDA events."""
+        cls = -1 if kernel_class == "all" else self.kernel_classes().index(kernel_class)
+        _check(self.lib.sepconv_profile_begin(self.h, cls, max_launches), "sepconv_profile_begin")
+
+    def profile_end(self, stream=None):
+        """Synchronise and return {class name: dict(ms, launches, bytes, flops)} for bracketed classes."""
+        n = self.lib.sepconv_kernel_class_count()
+        ms, cnt = (C.c_double * n)(), (C.c_int64 * n)()
+        by, fl = (C.c_double * n)(), (C.c_double * n)()
+        _check(self.lib.sepconv_profile_end(self.h, _stream_ptr(stream), ms, cnt, by, fl), "sepconv_profile_end")
+        names = self.kernel_classes()
+        return {names[i]: dict(ms=ms[i], launches=int(cnt[i]), bytes=by[i], flops=fl[i])
+                for i in range(n) if cnt[i] > 0}
 
 
 def sepconv_workspace_bytes(desc: sc_block_desc):

@@ -19,7 +19,17 @@ struct sc_ctx {
     int64_t launches = 0;
     int gemm_mode = 0;
     TcState tc;
+    Prof prof;
 };
+
+namespace sc {
+const char* kclass_name(int c) {
+    static const char* n[KC_COUNT] = {"lengths", "dw_fwd", "dw_dgrad", "dw_wgrad", "pw_fwd", "pw_dgrad", "pw_wgrad",
+                                      "bn_stats", "bn_finalize", "bn_apply", "bn_bwd_reduce", "bn_bwd_finalize",
+                                      "bn_bwd_apply", "elementwise", "reduce_partials"};
+    return (c >= 0 && c < KC_COUNT) ? n[c] : "?";
+}
+}  // namespace sc
 
 namespace {
 
@@ -319,6 +329,7 @@ int sepconv_ctx_create(sc_ctx** out, int device) {
 
 void sepconv_ctx_destroy(sc_ctx* ctx) {
     if (!ctx) return;
+    for (cudaEvent_t e : ctx->prof.events) cudaEventDestroy(e);
     cudaFree(ctx->status_dev);
     delete ctx;
 }
@@ -360,6 +371,38 @@ int sepconv_set_gemm_mode(sc_ctx* ctx, int mode) {
 
 int64_t sepconv_launch_count(sc_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+int sepconv_profile_begin(sc_ctx* ctx, int kernel_class, int max_launches) {
+    if (!ctx) return SC_ERR_NULL;
+    if (kernel_class < -1 || kernel_class >= KC_COUNT || max_launches < 1) return SC_ERR_UNSUPPORTED;
+    Prof& p = ctx->prof;
+    while (p.events.size() < (size_t)2 * max_launches) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) return SC_ERR_CUDA;
+        p.events.push_back(e);
+    }
+    p.recs.clear(); p.used = 0; p.filter = kernel_class;
+    return SC_OK;
+}
+
+int sepconv_profile_end(sc_ctx* ctx, void* cuda_stream, double* ms, int64_t* launches, double* bytes,
+                        double* flops) {
+    if (!ctx || !ms || !launches || !bytes || !flops) return SC_ERR_NULL;
+    Prof& p = ctx->prof;
+    p.filter = -2;
+    if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return SC_ERR_CUDA;
+    for (int c = 0; c < KC_COUNT; ++c) { ms[c] = 0; launches[c] = 0; bytes[c] = 0; flops[c] = 0; }
+    for (const Prof::Rec& r : p.recs) {
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, p.events[r.e0], p.events[r.e0 + 1]) != cudaSuccess) return SC_ERR_CUDA;
+        ms[r.cls] += t; launches[r.cls] += 1; bytes[r.cls] += r.bytes; flops[r.cls] += r.flops;
+    }
+    p.recs.clear(); p.used = 0;
+    return SC_OK;
+}
+
+int sepconv_kernel_class_count(void) { return KC_COUNT; }
+const char* sepconv_kernel_class_name(int c) { return kclass_name(c); }
+
 int sepconv_workspace_bytes(const sc_block_desc* desc, size_t* fwd, size_t* bwd) {
     Dims m;
     SC_TRY(desc_dims(desc, &m));
@@ -389,7 +432,7 @@ int sepconv_fwd(sc_ctx* ctx, const sc_block_desc* desc, const sc_tensor* x, cons
     FwdScratch f;
     plan_fwd(desc, m, ws, &f, &ctx->tc);
     if (!ws.ok()) return SC_ERR_WORKSPACE;
-    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches};
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof};
     BlockIO io{};
     io.x = x->ptr; io.xres = desc->residual != SC_RES_NONE ? (x_res ? x_res->ptr : x->ptr) : nullptr;
     io.y = y->ptr; io.len_in = lengths_dev; io.len_out = f.len_out; io.nvalid = f.nvalid;
@@ -428,7 +471,7 @@ int sepconv_bwd(sc_ctx* ctx, const sc_block_desc* desc, const sc_tensor* dy, con
     BwdScratch s;
     plan_bwd(desc, m, ws, &s, &ctx->tc);
     if (!ws.ok()) return SC_ERR_WORKSPACE;
-    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches};
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof};
     lengths(L, lengths_dev, m.B, m.T, m.s, s.len_out, s.nvalid);
     BwdIO io{};
     io.dy = dy->ptr; io.x = x->ptr; io.y = y->ptr;
@@ -565,7 +608,7 @@ int encoder_fwd_bwd(sc_ctx* ctx, const sc_encoder_desc* e, const sc_tensor* x, c
         SC_TRY(check_params(&P.L[i].d, &prm[i]));
         SC_TRY(check_grads(&P.L[i].d, &grd[i]));
     }
-    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches};
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof};
     auto input_of = [&](int i) -> const void* { return i == 0 ? x->ptr : P.L[i - 1].y; };
     auto len_in_of = [&](int i) -> const int* { return i == 0 ? lengths_dev : P.L[i - 1].len_out; };
     auto res_src = [&](int i) -> int { return (e->res_from && e->res_from[i] >= 0) ? e->res_from[i] : i; };

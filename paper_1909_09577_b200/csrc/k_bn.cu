@@ -341,12 +341,14 @@ ew_add_masked_kernel(T* out, const T* a, const T* b, const T* c, const int* len,
     }
 
 void lengths(const Launch& L, const int* len_in, int B, int T_in, int stride, int* len_out, int* nvalid) {
+    KScope ks_(L, KC_LENGTHS, 8.0 * B, 0.0);
     lengths_kernel<<<1, 256, 0, L.stream>>>(len_in, B, T_in, stride, len_out, nvalid, L.status);
     L.count();
 }
 
 void bn_stats(const Launch& L, int vdtype, const void* v, const int* len_out, int B, int C, int Tp,
               float2* partials) {
+    KScope ks_(L, KC_BN_STATS, (double)dtype_size(vdtype) * B * C * Tp, 0.0);
     SC_DISPATCH(vdtype, (bn_stats_kernel<T><<<B * C, kRowThreads, 0, L.stream>>>((const T*)v, len_out, C, Tp, partials)));
     L.count();
 }
@@ -354,17 +356,20 @@ void bn_stats(const Launch& L, int vdtype, const void* v, const int* len_out, in
 void bn_finalize(const Launch& L, const float2* partials, int parts_per_b, int tile_w, const int* len_out,
                  const int* nvalid, int B, int C, float eps, float momentum, float* mean, float* invstd,
                  float* running_mean, float* running_var) {
+    KScope ks_(L, KC_BN_FINALIZE, 8.0 * B * parts_per_b * C, 0.0);
     bn_finalize_kernel<<<(C + 63) / 64, 64, 0, L.stream>>>(partials, parts_per_b, tile_w, len_out, nvalid, B, C,
                                                             eps, momentum, mean, invstd, running_mean, running_var);
     L.count();
 }
 
 void bn_apply(const Launch& L, int dtype, const ApplyArgs& a) {
+    KScope ks_(L, KC_BN_APPLY, (double)a.B * a.C * a.Tp * (dtype_size(vtype_of(dtype)) + dtype_size(dtype) + dtype_size(ntype_of(dtype)) + (a.residual == 1 ? dtype_size(dtype) : 0) + (a.residual == 2 ? dtype_size(vtype_of(dtype)) + dtype_size(ntype_of(dtype)) : 0)), 0.0);
     SC_DISPATCH3(dtype, (bn_apply_kernel<T, VT, NT><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a)));
     L.count();
 }
 
 void bn_bwd_reduce(const Launch& L, int dtype, const BnBwdArgs& a) {
+    KScope ks_(L, KC_BN_BWD_REDUCE, (double)a.B * a.C * a.Tp * (dtype_size(dtype) * (a.has_relu && a.res_before_relu ? 2 : 1) + (a.has_bn ? dtype_size(ntype_of(dtype)) : 0) + (a.residual == 2 ? dtype_size(ntype_of(dtype)) : 0)), 0.0);
     SC_DISPATCH3(dtype, (bn_bwd_reduce_kernel<T, NT><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a)));
     L.count();
 }
@@ -372,18 +377,21 @@ void bn_bwd_reduce(const Launch& L, int dtype, const BnBwdArgs& a) {
 void bn_bwd_finalize(const Launch& L, const BnBwdArgs& a, const float* gamma, const float* gamma_r,
                      float* dgamma, float* dbeta, float* dgamma_r, float* dbeta_r, float* dbias,
                      int accumulate) {
+    KScope ks_(L, KC_BN_BWD_FINALIZE, 16.0 * a.B * a.C, 0.0);
     bn_bwd_finalize_kernel<<<(a.C + 63) / 64, 64, 0, L.stream>>>(a, gamma, gamma_r, dgamma, dbeta, dgamma_r,
                                                                   dbeta_r, dbias, accumulate);
     L.count();
 }
 
 void bn_bwd_apply(const Launch& L, int dtype, const BnBwdArgs& a) {
+    KScope ks_(L, KC_BN_BWD_APPLY, (double)a.B * a.C * a.Tp * (dtype_size(dtype) * (a.has_relu && a.res_before_relu ? 2 : 1) + (a.has_bn ? dtype_size(ntype_of(dtype)) : 0) + (a.residual == 2 ? dtype_size(ntype_of(dtype)) : 0) + dtype_size(dtype) * (1 + (a.residual != 0 ? 1 : 0))), 0.0);
     SC_DISPATCH3(dtype, (bn_bwd_apply_kernel<T, NT><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a)));
     L.count();
 }
 
 void ew_add_masked(const Launch& L, int dtype, void* out, const void* a, const void* b, const void* c,
                    const int* len, int B, int C, int Tt) {
+    KScope ks_(L, KC_EW, (double)dtype_size(dtype) * B * C * Tt * (2 + (b ? 1 : 0) + (c ? 1 : 0)), 0.0);
     SC_DISPATCH(dtype, (ew_add_masked_kernel<T><<<B * C, kRowThreads, 0, L.stream>>>((T*)out, (const T*)a, (const T*)b,
                                                                                       (const T*)c, len, C, Tt)));
     L.count();

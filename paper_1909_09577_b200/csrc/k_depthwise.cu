@@ -311,6 +311,8 @@ inline int host_phys(int i) { return i + ((i >> 5) << 2); }
 static void corr_s1(const Launch& L, int dtype, const void* in, const void* w, void* out, const void* add1,
                     const void* add2, const int* len_src, const int* len_dst, int B, int C, int Tt, int K,
                     int flip) {
+    KScope ks_(L, flip ? KC_DW_DGRAD : KC_DW_FWD,
+               (double)dtype_size(dtype) * B * C * Tt * (2 + (add1 ? 1 : 0) + (add2 ? 1 : 0)), 2.0 * B * C * Tt * K);
     const int Kp = kpad(K);
     const size_t smem = (size_t)CH * (host_phys(TT + Kp) + 4 + Kp) * sizeof(float);
     dim3 grid((Tt + TT - 1) / TT, (C + CH - 1) / CH, B), block(32, CH);
@@ -323,6 +325,7 @@ static void corr_s1(const Launch& L, int dtype, const void* in, const void* w, v
 void dw_fwd(const Launch& L, int dtype, const void* x, const void* wd, void* u, const int* len_in,
             const int* len_out, int B, int C, int Tt, int Tp, int K, int s) {
     if (s == 1) { corr_s1(L, dtype, x, wd, u, nullptr, nullptr, len_in, len_out, B, C, Tt, K, 0); return; }
+    KScope ks_(L, KC_DW_FWD, (double)dtype_size(dtype) * B * C * (Tt + Tp), 2.0 * B * C * Tp * K);
     const size_t smem = (size_t)((GT - 1) * s + K + K) * sizeof(float);
     dim3 grid((Tp + GT - 1) / GT, C, B);
     SC_DISPATCH(dtype, (dw_fwd_generic_kernel<T><<<grid, GT, smem, L.stream>>>((const T*)x, (const T*)wd, (T*)u, len_in,
@@ -334,6 +337,7 @@ void dw_dgrad(const Launch& L, int dtype, const void* gu, const void* wd, void* 
               const void* add2, const int* len_in, const int* len_out, int B, int C, int Tt, int Tp,
               int K, int s) {
     if (s == 1) { corr_s1(L, dtype, gu, wd, dx, add1, add2, len_out, len_in, B, C, Tt, K, 1); return; }
+    KScope ks_(L, KC_DW_DGRAD, (double)dtype_size(dtype) * B * C * (Tt * (1 + (add1 ? 1 : 0) + (add2 ? 1 : 0)) + Tp), 2.0 * B * C * Tp * K);
     const size_t smem = (size_t)((GT + K) / s + 4 + K) * sizeof(float);
     dim3 grid((Tt + GT - 1) / GT, C, B);
     SC_DISPATCH(dtype, (dw_dgrad_generic_kernel<T><<<grid, GT, smem, L.stream>>>(
@@ -348,6 +352,8 @@ void dw_wgrad(const Launch& L, int dtype, const void* gu, const void* x, float* 
               int accumulate, const int* len_in, const int* len_out, int B, int C, int Tt, int Tp,
               int K, int s) {
     int nsplit;
+    {
+    KScope ks_(L, KC_DW_WGRAD, (double)dtype_size(dtype) * B * C * (Tt + Tp), 2.0 * B * C * Tp * K);
     if (s == 1) {
         const int Kp = kpad(K), NG = Kp / R, nseg = WG_THREADS / NG;
         const int seglen = ((WG_TT + nseg - 1) / nseg + R - 1) / R * R;
@@ -363,6 +369,7 @@ void dw_wgrad(const Launch& L, int dtype, const void* gu, const void* x, float* 
                                                                                  len_in, len_out, B, C, Tt, Tp, K, s)));
     }
     L.count();
+    }
     reduce_partials(L, partials, nsplit, (int64_t)C * K, dwd, accumulate);
 }
 

@@ -130,12 +130,14 @@ __global__ void reduce_partials_kernel(const float* __restrict__ p, int nsplit, 
     }
 
 void reduce_partials(const Launch& L, const float* partials, int nsplit, int64_t n, float* out, int accumulate) {
+    KScope ks_(L, KC_REDUCE, 4.0 * (nsplit + 1) * n, 0.0);
     reduce_partials_kernel<<<(unsigned)((n + 255) / 256), 256, 0, L.stream>>>(partials, nsplit, n, out, accumulate);
     L.count();
 }
 
 void gemm_fwd_simt(const Launch& L, int dtype, const void* w, const void* u, const float* bias, void* v,
                    int out_dtype, const int* len_out, int B, int Cin, int Cout, int Tp) {
+    KScope ks_(L, KC_PW_FWD, (double)B * Tp * (dtype_size(dtype) * Cin + dtype_size(out_dtype) * Cout), 2.0 * B * Tp * Cin * Cout);
     GemmDesc d{};
     d.M = Cout; d.N = Tp; d.Kd = Cin;
     d.a_z = 0; d.a_m = Cin; d.a_k = 1;
@@ -151,6 +153,7 @@ void gemm_fwd_simt(const Launch& L, int dtype, const void* w, const void* u, con
 
 void gemm_dgrad_simt(const Launch& L, int dtype, const void* w, const void* gv, void* gu, int B, int Cin,
                      int Cout, int Tp) {
+    KScope ks_(L, KC_PW_DGRAD, (double)dtype_size(dtype) * B * Tp * (Cin + Cout), 2.0 * B * Tp * Cin * Cout);
     GemmDesc d{};
     d.M = Cin; d.N = Tp; d.Kd = Cout;
     d.a_z = 0; d.a_m = 1; d.a_k = Cin;            // A(m=c, k=o) = w[o*Cin + c]
@@ -168,16 +171,19 @@ size_t gemm_wgrad_simt_scratch_bytes(int B, int Cin, int Cout) {
 
 void gemm_wgrad_simt(const Launch& L, int dtype, const void* gv, const void* u, float* dw, float* partials,
                      int accumulate, int B, int Cin, int Cout, int Tp) {
+    const int ns = wgrad_splits(B);
+    {
+    KScope ks_(L, KC_PW_WGRAD, (double)dtype_size(dtype) * B * Tp * (Cin + Cout), 2.0 * B * Tp * Cin * Cout);
     GemmDesc d{};
     d.M = Cout; d.N = Cin; d.Kd = B * Tp;
     d.kt = Tp;
     d.a_m = Tp; d.a_kz = (long long)Cout * Tp;    // A(m=o, k=(b,t)) = gv[b,o,t]
     d.b_n = Tp; d.b_kz = (long long)Cin * Tp;     // B(k=(b,t), n=c) = u[b,c,t]
-    const int ns = wgrad_splits(B);
     d.k_len_per_z = Tp;
     dim3 grid((Cin + BN - 1) / BN, (Cout + BM - 1) / BM, ns);
     SC_DISPATCH(dtype, (gemm_simt_kernel<T, T, 2><<<grid, NT, 0, L.stream>>>(d, (const T*)gv, (const T*)u, partials, nullptr, nullptr)));
     L.count();
+    }
     reduce_partials(L, partials, ns, (int64_t)Cin * Cout, dw, accumulate);
 }
 

@@ -3,14 +3,48 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <vector>
 
 namespace sc {
+
+// Kernel classes, for launch counting and per-class event timing.
+enum KClass : int {
+    KC_LENGTHS = 0, KC_DW_FWD, KC_DW_DGRAD, KC_DW_WGRAD, KC_PW_FWD, KC_PW_DGRAD, KC_PW_WGRAD,
+    KC_BN_STATS, KC_BN_FINALIZE, KC_BN_APPLY, KC_BN_BWD_REDUCE, KC_BN_BWD_FINALIZE, KC_BN_BWD_APPLY,
+    KC_EW, KC_REDUCE, KC_COUNT
+};
+const char* kclass_name(int c);
+
+// Optional event timing of one kernel class (or all): a start/stop event pair brackets each launch
+// of the selected class on the launching stream; totals are read back after a synchronise.
+struct Prof {
+    int filter = -2;                       // -2 off, -1 every class, >= 0 one class
+    std::vector<cudaEvent_t> events;       // pool, pairs
+    struct Rec { int cls; int e0; double bytes, flops; };
+    std::vector<Rec> recs;
+    size_t used = 0;
+};
 
 struct Launch {
     cudaStream_t stream;
     int* status;          // device status word
     int64_t* counter;     // host launch counter
+    Prof* prof = nullptr;
     void count(int n = 1) const { if (counter) *counter += n; }
+};
+
+// Brackets the launches of one launcher call.  bytes/flops are the algorithmic figures of the call.
+struct KScope {
+    const Launch& L; int slot = -1;
+    KScope(const Launch& l, int cls, double bytes, double flops) : L(l) {
+        Prof* p = L.prof;
+        if (!p || p->filter == -2 || (p->filter >= 0 && p->filter != cls)) return;
+        if (p->used + 2 > p->events.size()) return;
+        slot = (int)p->used; p->used += 2;
+        p->recs.push_back({cls, slot, bytes, flops});
+        cudaEventRecord(p->events[slot], L.stream);
+    }
+    ~KScope() { if (slot >= 0) cudaEventRecord(L.prof->events[slot + 1], L.stream); }
 };
 
 // ---- lengths -------------------------------------------------------------------------------
