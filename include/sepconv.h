@@ -175,6 +175,33 @@ int  sepconv_bwd(sc_ctx* ctx, const sc_block_desc* desc,
                  sc_block_grads* grads, int accumulate,
                  void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Forward of one block without a workspace argument and without any allocation (the paper has no
+ * counterpart; this exists for integration reasons only).
+ *
+ * Who needs it: code that runs where device allocation is forbidden or impossible -- inside a
+ * real-time audio pipeline whose memory is fixed at start-up, under a framework that owns the whole
+ * device heap and hands out no raw buffers, or in a plugin loaded after the host application has
+ * already committed all device memory.  Such a caller can still pass its own inputs and outputs but
+ * has nowhere to get the scratch that sepconv_fwd asks for.
+ *
+ * The scratch is a fixed array of SEPCONV_STATIC_SCRATCH_BYTES inside the library image: every GPU on
+ * which the library is loaded sets that much memory aside until the process exits.  A block whose
+ * forward scratch (sepconv_workspace_bytes) exceeds it is refused with SC_ERR_WORKSPACE and a message
+ * on stderr; nothing is enqueued.  Arguments and results are exactly those of sepconv_fwd (running
+ * statistics are not updated).  The call itself uses no cudaMalloc/cudaFree or other allocating
+ * routine.
+ *
+ * The first call on each device looks up the array's device address (with the context's device
+ * current, as for every other call); make that first call outside any stream capture.
+ * All calls on a device share the one array and it keeps the previous call's contents: two calls
+ * whose GPU work overlaps (different streams, no dependency between them) race on it -- keep such
+ * calls on one stream or order them with events. */
+#define SEPCONV_STATIC_SCRATCH_BYTES (8u << 20)
+int  sepconv_fwd_static(sc_ctx* ctx, const sc_block_desc* desc,
+                        const sc_tensor* x, const sc_tensor* x_res, const int32_t* lengths_dev,
+                        const sc_block_params* params, sc_tensor* y, int32_t* out_lengths_dev,
+                        sc_block_saved* saved, void* cuda_stream);
+
 /* ---- whole encoder -------------------------------------------------------------------------- */
 
 int  encoder_workspace_bytes(const sc_encoder_desc* desc, size_t* bytes);

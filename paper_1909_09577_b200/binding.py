@@ -69,7 +69,7 @@ class sc_encoder_desc(C.Structure):
 
 _lib = None
 
-EXPORTS = ("sepconv_profile_begin", "sepconv_profile_end", "sepconv_kernel_class_count",
+EXPORTS = ("sepconv_fwd_static", "sepconv_profile_begin", "sepconv_profile_end", "sepconv_kernel_class_count",
            "sepconv_kernel_class_name", "sepconv_ctx_create", "sepconv_ctx_destroy", "sepconv_last_status", "sepconv_strerror",
            "sepconv_workspace_bytes", "sepconv_fwd", "sepconv_bwd", "encoder_workspace_bytes",
            "encoder_fwd_bwd", "sepconv_set_gemm_mode", "sepconv_launch_count")
@@ -99,6 +99,9 @@ def load_library(path: str = LIB_PATH):
                                 C.c_void_p, C.POINTER(sc_block_params), C.POINTER(sc_tensor), C.c_void_p,
                                 C.POINTER(sc_block_saved), C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
                                 C.c_void_p]
+    lib.sepconv_fwd_static.argtypes = [C.c_void_p, C.POINTER(sc_block_desc), C.POINTER(sc_tensor),
+                                       C.POINTER(sc_tensor), C.c_void_p, C.POINTER(sc_block_params),
+                                       C.POINTER(sc_tensor), C.c_void_p, C.POINTER(sc_block_saved), C.c_void_p]
     lib.sepconv_bwd.argtypes = [C.c_void_p, C.POINTER(sc_block_desc), C.POINTER(sc_tensor), C.POINTER(sc_tensor),
                                 C.POINTER(sc_tensor), C.POINTER(sc_tensor), C.c_void_p,
                                 C.POINTER(sc_block_params), C.POINTER(sc_block_saved), C.POINTER(sc_tensor),
@@ -260,6 +263,24 @@ def sepconv_fwd(ctx: Context, desc: sc_block_desc, x: torch.Tensor, lengths: tor
                              workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
     _check(rc, "sepconv_fwd")
     return y, out_len, saved
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def sepconv_fwd_static(ctx: Context, desc: sc_block_desc, x: torch.Tensor, lengths: torch.Tensor,
+                       params: Dict[str, torch.Tensor], y: torch.Tensor, out_lengths: torch.Tensor,
+                       saved: Dict[str, torch.Tensor], x_res: Optional[torch.Tensor] = None, stream=None):
+    """sepconv_fwd for callers that cannot allocate: every buffer (y, out_lengths, saved) is passed in
+    and the scratch is the library's built-in fixed array.  This wrapper allocates nothing either."""
+    sv = sc_block_saved()
+    for n, _ in sc_block_saved._fields_:
+        setattr(sv, n, saved[n].data_ptr() if n in saved else None)
+    p = _params_struct(params)
+    rc = ctx.lib.sepconv_fwd_static(ctx.h, C.byref(desc), tensor_arg(x), tensor_arg(x_res), lengths.data_ptr(),
+                                    C.byref(p), tensor_arg(y), out_lengths.data_ptr(), C.byref(sv),
+                                    _stream_ptr(stream))
+    _check(rc, "sepconv_fwd_static")
 
 
 def sepconv_bwd(ctx: Context, desc: sc_block_desc, dy: torch.Tensor, x: torch.Tensor, y: torch.Tensor,
