@@ -116,7 +116,7 @@ void pointwise_bn(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const Di
     int parts = 1, tile_w = m.Tp;
     bool fused = false;
     if (ctx->gemm_mode == 0 && tc_fwd_supported(&ctx->tc, d->io_dtype, Cin, m.Cout, m.Tp)) {
-        fused = tc_gemm_fwd(&ctx->tc, L, d->io_dtype, w, u, nullptr, v, len_out, m.B, Cin, m.Cout, m.Tp,
+        fused = tc_gemm_fwd(&ctx->tc, L, d->io_dtype, w, u, nullptr, v, vdt, len_out, m.B, Cin, m.Cout, m.Tp,
                             partials, &parts, &tile_w);
     } else {
         gemm_fwd_simt(L, d->io_dtype, w, u, nullptr, v, vdt, len_out, m.B, Cin, m.Cout, m.Tp);
@@ -144,7 +144,7 @@ int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
     if (!d->has_bn) {   // linear layer: y = mask * (w u + bias)
         if (ctx->gemm_mode == 0 && tc_fwd_supported(&ctx->tc, dt, m.Cin, m.Cout, m.Tp)) {
             int parts, tw;
-            tc_gemm_fwd(&ctx->tc, L, dt, p->wp, u, d->has_bias ? p->bias : nullptr, io.y, io.len_out, m.B, m.Cin,
+            tc_gemm_fwd(&ctx->tc, L, dt, p->wp, u, d->has_bias ? p->bias : nullptr, io.y, dt, io.len_out, m.B, m.Cin,
                         m.Cout, m.Tp, nullptr, &parts, &tw);
         } else {
             gemm_fwd_simt(L, dt, p->wp, u, d->has_bias ? p->bias : nullptr, io.y, dt, io.len_out, m.B, m.Cin, m.Cout, m.Tp);

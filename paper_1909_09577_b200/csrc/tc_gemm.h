@@ -22,11 +22,11 @@ bool tc_dgrad_supported(const TcState* st, int dtype, int Cin, int Cout, int Tp)
 bool tc_wgrad_supported(const TcState* st, int dtype, int Cin, int Cout, int Tp);
 size_t tc_wgrad_scratch_bytes(const TcState* st, int Cin, int Cout);
 
-// v[b,o,t] = [t < len_out[b]] * (sum_c w[o,c] u[b,c,t] + bias[o]).  When `partials` is non-null the
+// v[b,o,t] = [t < len_out[b]] * (sum_c w[o,c] u[b,c,t] + bias[o]), stored in out_dtype.  When `partials` is non-null the
 // epilogue also writes per-(sample, time-tile, channel) (sum, M2) over valid frames, computed from the
 // fp32 accumulators, and reports the tiling through parts_per_b / tile_w; returns true if it did.
 bool tc_gemm_fwd(const TcState* st, const Launch& L, int dtype, const void* w, const void* u, const float* bias,
-                 void* v, const int* len_out, int B, int Cin, int Cout, int Tp, float2* partials,
+                 void* v, int out_dtype, const int* len_out, int B, int Cin, int Cout, int Tp, float2* partials,
                  int* parts_per_b, int* tile_w);
 // gu[b,c,t] = sum_o w[o,c] gv[b,o,t]
 void tc_gemm_dgrad(const TcState* st, const Launch& L, int dtype, const void* w, const void* gv, void* gu, int B,

@@ -44,13 +44,45 @@ SMALL = [
 ]
 
 
+@pytest.fixture(params=[0, 1], ids=["tensorcore", "simt"])
+def gemm_mode(request, ctx):
+    """0: tensor-core contractions where the shape allows; 1: plain SIMT contractions everywhere."""
+    ctx.set_gemm_mode(request.param)
+    yield request.param
+    ctx.set_gemm_mode(0)
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
 @pytest.mark.parametrize("case", range(len(SMALL)))
-def test_small_blocks(api, ctx, dtype, case):
+def test_small_blocks(api, ctx, dtype, case, gemm_mode):
+    if dtype == "f32" and gemm_mode == 1:
+        pytest.skip("fp32 always uses the SIMT contractions")
     kw, B, T, ragged = SMALL[case]
     L = si.LayerCfg(**kw)
     d = _draw_block(L, B, T, dtype, seed=100 + case, ragged=ragged)
     rep = U.run_block(ctx, api, L, dtype, d.x, d.lengths, d.params[0], d.g)
+    rep.check()
+
+
+TC_SHAPES = [
+    # shapes that exercise the tensor-core tiling: channel tails, several k-blocks, T' tails, tiny C_out
+    (dict(C_in=64, C_out=256, K=33, stride=2, residual="none"), 4, 400, True),
+    (dict(C_in=256, C_out=256, K=5, residual="identity"), 3, 328, True),
+    (dict(C_in=320, C_out=200, K=5, residual="proj"), 2, 136, True),
+    (dict(C_in=1024, C_out=29, K=1, has_dw=False, has_bn=False, has_relu=False, has_bias=True), 3, 200, True),
+    (dict(C_in=512, C_out=1024, K=1, has_dw=False), 2, 264, True),
+    (dict(C_in=72, C_out=136, K=3, residual="proj"), 5, 64, False),
+]
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f16"])
+@pytest.mark.parametrize("case", range(len(TC_SHAPES)))
+def test_tensorcore_shapes(api, ctx, dtype, case):
+    kw, B, T, ragged = TC_SHAPES[case]
+    L = si.LayerCfg(**kw)
+    d = _draw_block(L, B, T, dtype, seed=200 + case, ragged=ragged, lo_frac=0.1)
+    rep = U.run_block(ctx, api, L, dtype, d.x, d.lengths, d.params[0], d.g)
+    print(f"\ntc shape {case} {dtype}: {rep}")
     rep.check()
 
 
@@ -76,12 +108,12 @@ def test_external_residual_and_dx_add(api, ctx):
 
 @pytest.mark.parametrize("i", [1, 2, 3])
 @pytest.mark.parametrize("affine", ["unit", "random"])
-def test_benchmark_block_configs(api, ctx, i, affine):
+def test_benchmark_block_configs(api, ctx, i, affine, gemm_mode):
     """Configs 1-3 at full size, seeds as specified; reports error/allowed per tensor."""
     w = si.config(i, affine=affine)
     d = si.draw(w)
     rep = U.run_block(ctx, api, w.layers[0], w.dtype, d.x, d.lengths, d.params[0], d.g)
-    print(f"\nconfig {i} ({affine}) error/allowed: {rep}; adopted gates {rep.adopted}")
+    print(f"\nconfig {i} ({affine}, gemm_mode {gemm_mode}) error/allowed: {rep}; adopted gates {rep.adopted}")
     rep.check()
 
 
