@@ -30,6 +30,12 @@
  *   - Tensors are dense [B, C, T] with time contiguous; base pointers 16-byte aligned.
  *   - Activations and conv weights (wd, wp, wr) use desc->io_dtype; gamma, beta, bias, the saved
  *     statistics, running statistics and every parameter gradient are float32.
+ *   - Tensors that only the library sees between the depthwise and the pointwise step (u forward;
+ *     the gradients of v and u backward) are float16 for both 16-bit activation types: they are
+ *     contraction operands, and a second bf16 rounding on them would cost more than the error budget
+ *     leaves.  Forward, a depthwise output beyond the float16 range is clamped and reported as
+ *     SC_ERR_RANGE; backward, those gradients carry a per-layer power-of-two scale chosen on the
+ *     device from the gradient's magnitude, so any upstream scale (e.g. a loss scale) is safe.
  *   - Calls enqueue work on `cuda_stream` and return without synchronising.  The library never
  *     allocates or frees device memory inside these calls and keeps no pointer past the call.
  *   - Return value: SC_OK or a negative sc_status.  Nothing throws across the boundary.  Errors
@@ -66,7 +72,8 @@ typedef enum {
     SC_ERR_LENGTHS = -8,           /* (device) some length is outside [1, T_in]                    */
     SC_ERR_DEVICE_TIMEOUT = -9,    /* (device) a bounded wait inside a kernel ran out              */
     SC_ERR_ARCH = -10,             /* the device is not compute capability 10.x                    */
-    SC_ERR_CUDA = -11              /* a CUDA runtime/driver call failed                            */
+    SC_ERR_CUDA = -11,             /* a CUDA runtime/driver call failed                            */
+    SC_ERR_RANGE = -12             /* (device) a depthwise output exceeded the float16 range       */
 } sc_status;
 
 /* A typed tensor argument: size/stride in elements, tag[i] names axis i. */
@@ -100,7 +107,9 @@ typedef struct {          /* device pointers; absent parts may be null          
 } sc_block_params;
 
 typedef struct {          /* written by sepconv_fwd, read by sepconv_bwd; caller-owned             */
-    void  *u;             /* [B, C_in, T']  io_dtype (has_dw only)                                 */
+    void  *u;             /* [B, C_in, T'] depthwise output (or masked input when has_dw = 0).     */
+                          /* float16 when the layer has a depthwise step and batch norm and        */
+                          /* io_dtype is 16-bit (also for bf16: see below); io_dtype otherwise     */
     void  *vhat;          /* [B, C_out, T'] normalised (v - mean)/sqrt(var+eps), zero in padding   */
                           /* (has_bn only); float32 when io_dtype is SC_F32, float16 otherwise     */
     float *mean, *invstd; /* [C_out]                                                               */

@@ -240,7 +240,8 @@ def sepconv_fwd(ctx: Context, desc: sc_block_desc, x: torch.Tensor, lengths: tor
         y = torch.empty((B, Co, Tp), dtype=td, device=dev)
     out_len = torch.empty((B,), dtype=torch.int32, device=dev)
     if saved is None:
-        saved = {"u": torch.empty((B, Ci, Tp), dtype=td, device=dev)}
+        ut = torch.float16 if (desc.has_dw and desc.has_bn and desc.io_dtype != SC_F32) else td
+        saved = {"u": torch.empty((B, Ci, Tp), dtype=ut, device=dev)}
         nt = torch.float32 if desc.io_dtype == SC_F32 else torch.float16   # type of the normalised tensors
         if desc.has_bn:
             saved["vhat"] = torch.empty((B, Co, Tp), dtype=nt, device=dev)

@@ -94,8 +94,11 @@ struct BlockIO {                 // raw pointers after validation
     bool lengths_ready;          // len_out / nvalid already computed
 };
 
+// Type of the library-internal contraction operands (u, gv, gu) of this layer.
+int op_dtype(const sc_block_desc* d) { return otype_of(d->io_dtype, d->has_dw && d->has_bn); }
+
 // ---- forward scratch ---------------------------------------------------------------------------
-struct FwdScratch { float2* partials; void *xr, *v, *vr; int* len_out; int* nvalid; };
+struct FwdScratch { float2* partials; void *xr, *v, *vr, *w16; int* len_out; int* nvalid; };
 
 void plan_fwd(const sc_block_desc* d, const Dims& m, Bump& ws, FwdScratch* f, const TcState* tc) {
     const size_t parts = (size_t)m.B * tc_max_parts_per_sample(m.Tp) * m.Cout;
@@ -106,20 +109,21 @@ void plan_fwd(const sc_block_desc* d, const Dims& m, Bump& ws, FwdScratch* f, co
     f->v = d->has_bn ? ws.take(vbytes) : nullptr;
     f->vr = (d->residual == SC_RES_PROJ) ? ws.take(vbytes) : nullptr;
     f->xr = (d->residual == SC_RES_PROJ) ? ws.take(esize(d->io_dtype) * m.B * m.Cres * m.Tp) : nullptr;
+    f->w16 = (op_dtype(d) != d->io_dtype) ? ws.take((size_t)2 * m.Cout * m.Cin) : nullptr;
 }
 
 // v = w * u for every sample (stored in the transient type), plus masked batch statistics.
-void pointwise_bn(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const Dims& m, int Cin,
+void pointwise_bn(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const Dims& m, int Cin, int opdt,
                   const void* w, const void* u, void* v, const int* len_out, const int* nvalid,
                   float* mean, float* invstd, float2* partials, float* rmean, float* rvar) {
     const int vdt = vtype_of(d->io_dtype);
     int parts = 1, tile_w = m.Tp;
     bool fused = false;
-    if (ctx->gemm_mode == 0 && tc_fwd_supported(&ctx->tc, d->io_dtype, Cin, m.Cout, m.Tp)) {
-        fused = tc_gemm_fwd(&ctx->tc, L, d->io_dtype, w, u, nullptr, v, vdt, len_out, m.B, Cin, m.Cout, m.Tp,
+    if (ctx->gemm_mode == 0 && tc_fwd_supported(&ctx->tc, opdt, Cin, m.Cout, m.Tp)) {
+        fused = tc_gemm_fwd(&ctx->tc, L, opdt, w, u, nullptr, v, vdt, len_out, m.B, Cin, m.Cout, m.Tp,
                             partials, &parts, &tile_w);
     } else {
-        gemm_fwd_simt(L, d->io_dtype, w, u, nullptr, v, vdt, len_out, m.B, Cin, m.Cout, m.Tp);
+        gemm_fwd_simt(L, opdt, w, u, nullptr, v, vdt, len_out, m.B, Cin, m.Cout, m.Tp);
     }
     if (!fused) { bn_stats(L, vdt, v, len_out, m.B, m.Cout, m.Tp, partials); parts = 1; tile_w = m.Tp; }
     bn_finalize(L, partials, parts, tile_w, len_out, nvalid, m.B, m.Cout, d->bn_eps, d->bn_momentum, mean,
@@ -131,9 +135,10 @@ int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
                    const FwdScratch& f) {
     const int dt = d->io_dtype;
     if (!io.lengths_ready) lengths(L, io.len_in, m.B, m.T, m.s, io.len_out, io.nvalid);
+    const int odt = op_dtype(d);
     const void* u;
     if (d->has_dw) {
-        dw_fwd(L, dt, io.x, p->wd, sv->u, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s);
+        dw_fwd(L, dt, odt, io.x, p->wd, sv->u, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s);
         u = sv->u;
     } else if (io.x_clean) {
         u = io.x;
@@ -151,7 +156,9 @@ int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
         }
         return SC_OK;
     }
-    pointwise_bn(ctx, L, d, m, m.Cin, p->wp, u, f.v, io.len_out, io.nvalid, sv->mean, sv->invstd, f.partials,
+    const void* wp_op = p->wp;
+    if (odt != dt) { convert_bf16_to_f16(L, p->wp, f.w16, (int64_t)m.Cout * m.Cin); wp_op = f.w16; }
+    pointwise_bn(ctx, L, d, m, m.Cin, odt, wp_op, u, f.v, io.len_out, io.nvalid, sv->mean, sv->invstd, f.partials,
                  rmean, rvar);
     ApplyArgs a{};
     a.v = f.v; a.mean = sv->mean; a.invstd = sv->invstd; a.gamma = p->gamma; a.beta = p->beta; a.vhat = sv->vhat;
@@ -161,7 +168,7 @@ int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
     if (d->residual == SC_RES_PROJ) {
         const void* xr = io.xres;
         if (!io.res_clean) { mask_copy(L, dt, f.xr, io.xres, io.len_out, m.B, m.Cres, m.Tp); xr = f.xr; }
-        pointwise_bn(ctx, L, d, m, m.Cres, p->wr, xr, f.vr, io.len_out, io.nvalid, sv->mean_r, sv->invstd_r,
+        pointwise_bn(ctx, L, d, m, m.Cres, dt, p->wr, xr, f.vr, io.len_out, io.nvalid, sv->mean_r, sv->invstd_r,
                      f.partials, nullptr, nullptr);
         a.vr = f.vr; a.mean_r = sv->mean_r; a.invstd_r = sv->invstd_r; a.gamma_r = p->gamma_r; a.beta_r = p->beta_r;
         a.vhat_r = sv->vhat_r;
@@ -174,7 +181,8 @@ int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
 struct BwdScratch {
     int* len_out; int* nvalid;
     float4 *partials, *coef, *coef_r;
-    void *gv, *gvr, *gres, *gu, *gxr, *xr;
+    float *amax_part, *gmax;
+    void *gv, *gvr, *gres, *gu, *gxr, *xr, *w16;
     float* wpart; size_t wpart_bytes;
 };
 
@@ -186,6 +194,9 @@ void plan_bwd(const sc_block_desc* d, const Dims& m, Bump& ws, BwdScratch* s, co
     s->partials = (float4*)ws.take(sizeof(float4) * m.B * m.Cout);
     s->coef = (float4*)ws.take(sizeof(float4) * m.Cout);
     s->coef_r = (float4*)ws.take(sizeof(float4) * m.Cout);
+    s->amax_part = (float*)ws.take(sizeof(float) * m.B * m.Cout);
+    s->gmax = (float*)ws.take(sizeof(float));
+    s->w16 = (op_dtype(d) != d->io_dtype) ? ws.take((size_t)2 * m.Cout * m.Cin) : nullptr;
     s->gv = ws.take(act_out);
     s->gvr = d->residual == SC_RES_PROJ ? ws.take(act_out) : nullptr;
     s->gres = d->residual == SC_RES_IDENTITY ? ws.take(act_out) : nullptr;
@@ -200,11 +211,12 @@ void plan_bwd(const sc_block_desc* d, const Dims& m, Bump& ws, BwdScratch* s, co
 }
 
 void pointwise_wgrad(sc_ctx* ctx, const Launch& L, int dt, const void* gv, const void* u, float* dw,
-                     float* part, int acc, int B, int Cin, int Cout, int Tp, const int* len_out) {
+                     float* part, int acc, int B, int Cin, int Cout, int Tp, const int* len_out,
+                     const float* gmax) {
     if (ctx->gemm_mode == 0 && tc_wgrad_supported(&ctx->tc, dt, Cin, Cout, Tp))
-        tc_gemm_wgrad(&ctx->tc, L, dt, gv, u, dw, part, acc, B, Cin, Cout, Tp, len_out);
+        tc_gemm_wgrad(&ctx->tc, L, dt, gv, u, dw, part, acc, B, Cin, Cout, Tp, len_out, gmax);
     else
-        gemm_wgrad_simt(L, dt, gv, u, dw, part, acc, B, Cin, Cout, Tp);
+        gemm_wgrad_simt(L, dt, gv, u, dw, part, acc, B, Cin, Cout, Tp, gmax);
 }
 void pointwise_dgrad(sc_ctx* ctx, const Launch& L, int dt, const void* w, const void* gv, void* gu, int B,
                      int Cin, int Cout, int Tp, const int* len_out) {
@@ -225,7 +237,13 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
                    const sc_block_params* p, const sc_block_saved* sv, sc_block_grads* g, int acc,
                    const BwdScratch& s) {
     const int dt = d->io_dtype;
+    const int odt = op_dtype(d);
+    // gv (and gu after it) is kept scaled by a power of two whenever it is a library-internal 16-bit
+    // tensor, so that neither a tiny nor a huge upstream gradient leaves the half range
+    float* gmax = (dt != SC_F32 && d->has_dw && d->has_bn) ? s.gmax : nullptr;
+    if (gmax) cudaMemsetAsync(gmax, 0, sizeof(float), L.stream);
     BnBwdArgs a{};
+    a.amax_part = s.amax_part; a.gmax = gmax; a.gv_dtype = odt;
     a.g = io.dy; a.y = io.y; a.vhat = sv->vhat; a.vhat_r = sv->vhat_r;
     a.invstd = sv->invstd; a.invstd_r = sv->invstd_r; a.gamma = p->gamma; a.beta = p->beta;
     a.len_out = io.len_out; a.nvalid = io.nvalid;
@@ -241,13 +259,15 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
     bn_bwd_apply(L, dt, a);
 
     const void* u = d->has_dw ? sv->u : (io.x_clean ? io.x : sv->u);
-    pointwise_wgrad(ctx, L, dt, s.gv, u, g->dwp, s.wpart, acc, m.B, m.Cin, m.Cout, m.Tp, io.len_out);
+    pointwise_wgrad(ctx, L, odt, s.gv, u, g->dwp, s.wpart, acc, m.B, m.Cin, m.Cout, m.Tp, io.len_out, gmax);
+    const void* wp_op = p->wp;
+    if (odt != dt) { convert_bf16_to_f16(L, p->wp, s.w16, (int64_t)m.Cout * m.Cin); wp_op = s.w16; }
 
     const void* extra = nullptr;    // residual-path gradient to fold into dx
     if (d->residual == SC_RES_PROJ) {
         const void* xr = io.xres;
         if (!io.res_clean) { mask_copy(L, dt, s.xr, io.xres, io.len_out, m.B, m.Cres, m.Tp); xr = s.xr; }
-        pointwise_wgrad(ctx, L, dt, s.gvr, xr, g->dwr, s.wpart, acc, m.B, m.Cres, m.Cout, m.Tp, io.len_out);
+        pointwise_wgrad(ctx, L, dt, s.gvr, xr, g->dwr, s.wpart, acc, m.B, m.Cres, m.Cout, m.Tp, io.len_out, nullptr);
         void* tgt = io.dx_res ? io.dx_res : s.gxr;
         if (io.dx_res || io.dx) pointwise_dgrad(ctx, L, dt, p->wr, s.gvr, tgt, m.B, m.Cres, m.Cout, m.Tp, io.len_out);
         if (!io.dx_res) extra = s.gxr;
@@ -256,10 +276,11 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
     }
 
     if (d->has_dw) {
-        pointwise_dgrad(ctx, L, dt, p->wp, s.gv, s.gu, m.B, m.Cin, m.Cout, m.Tp, io.len_out);
-        dw_wgrad(L, dt, s.gu, io.x, g->dwd, s.wpart, acc, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s);
+        pointwise_dgrad(ctx, L, odt, wp_op, s.gv, s.gu, m.B, m.Cin, m.Cout, m.Tp, io.len_out);
+        dw_wgrad(L, dt, odt, s.gu, io.x, g->dwd, s.wpart, acc, gmax, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s);
         if (io.dx)
-            dw_dgrad(L, dt, s.gu, p->wd, io.dx, io.dx_add, extra, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s);
+            dw_dgrad(L, dt, odt, s.gu, p->wd, io.dx, io.dx_add, extra, gmax, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp,
+                     m.K, m.s);
     } else if (io.dx) {
         if (!io.dx_add && !extra) {
             pointwise_dgrad(ctx, L, dt, p->wp, s.gv, io.dx, m.B, m.Cin, m.Cout, m.Tp, io.len_out);
@@ -358,6 +379,7 @@ const char* sepconv_strerror(int s) {
         case SC_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
         case SC_ERR_ARCH: return "device is not compute capability 10.x";
         case SC_ERR_CUDA: return "a CUDA call failed";
+        case SC_ERR_RANGE: return "an intermediate value left the float16 range and was clamped";
         default: return "unknown status";
     }
 }

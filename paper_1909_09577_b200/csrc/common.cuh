@@ -12,6 +12,22 @@ enum DType : int { F32 = 0, F16 = 1, BF16 = 2 };
 // Device status codes (mirrors sc_status in the public header).
 constexpr int kErrLengths = -8;
 constexpr int kErrTimeout = -9;
+constexpr int kErrRange = -12;
+
+// Power-of-two scale that brings a tensor with the given absolute maximum into [0.5, 1).
+// Multiplying by it (and later by its reciprocal) is exact.
+__device__ __forceinline__ float pow2_scale(float amax) {
+    if (!(amax > 0.f) || !(amax < 3.0e38f)) return 1.f;
+    int e;
+    frexpf(amax, &e);
+    e = max(-100, min(100, e));
+    return ldexpf(1.f, -e);
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
 
 template <typename T> struct IO;
 template <> struct IO<float> {

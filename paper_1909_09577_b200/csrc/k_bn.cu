@@ -46,6 +46,18 @@ __device__ __forceinline__ void block_sum(float (&v)[N]) {
     }
 }
 
+__device__ __forceinline__ float block_max(float v) {
+    __shared__ float shm[kRowThreads / 32];
+    v = warp_max(v);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) shm[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float m = shm[0];
+#pragma unroll
+    for (int w = 1; w < kRowThreads / 32; ++w) m = fmaxf(m, shm[w]);
+    return m;
+}
+
 __global__ void lengths_kernel(const int* __restrict__ len_in, int B, int T_in, int stride,
                                int* __restrict__ len_out, int* __restrict__ nvalid, int* status) {
     // single CTA; B is small (<= a few thousand)
@@ -93,24 +105,41 @@ bn_stats_kernel(const T* __restrict__ v, const int* __restrict__ len_out, int C,
     if (threadIdx.x == 0) partials[row] = make_float2(s[0], q[0]);
 }
 
-__global__ void bn_finalize_kernel(const float2* __restrict__ partials, int parts_per_b, int tile_w,
-                                   const int* __restrict__ len_out, const int* __restrict__ nvalid, int B,
-                                   int C, float eps, float momentum, float* __restrict__ mean_out,
-                                   float* __restrict__ invstd_out, float* running_mean, float* running_var) {
-    const int o = blockIdx.x * blockDim.x + threadIdx.x;
-    if (o >= C) return;
+// 32 channels x 8 part-slices per CTA: slice s merges parts s, s+8, ... in increasing order, then the
+// eight slice results are merged in slice order -- a fixed tree, so the result is bit-repeatable.
+constexpr int kFinSlices = 8;
+__global__ void __launch_bounds__(32 * kFinSlices)
+bn_finalize_kernel(const float2* __restrict__ partials, int parts_per_b, int tile_w,
+                   const int* __restrict__ len_out, const int* __restrict__ nvalid, int B,
+                   int C, float eps, float momentum, float* __restrict__ mean_out,
+                   float* __restrict__ invstd_out, float* running_mean, float* running_var) {
+    __shared__ double sh[kFinSlices][32][3];
+    const int cx = threadIdx.x & 31, sl = threadIdx.x >> 5;
+    const int o = blockIdx.x * 32 + cx;
     double n = 0.0, mean = 0.0, m2 = 0.0;
-    for (int b = 0; b < B; ++b) {
-        const int len = len_out[b];
-        for (int j = 0; j < parts_per_b; ++j) {
-            int cnt = min(max(len - j * tile_w, 0), tile_w);
-            if (cnt <= 0) break;
-            float2 p = partials[((size_t)b * parts_per_b + j) * C + o];
-            double nb = cnt, mb = (double)p.x / nb, nt = n + nb, d = mb - mean;
+    if (o < C) {
+        const int nparts = B * parts_per_b;
+        for (int pi = sl; pi < nparts; pi += kFinSlices) {
+            const int b = pi / parts_per_b, j = pi - b * parts_per_b;
+            const int cnt = min(max(len_out[b] - j * tile_w, 0), tile_w);
+            if (cnt <= 0) continue;
+            const float2 p = partials[(size_t)pi * C + o];
+            const double nb = cnt, mb = (double)p.x / nb, nt = n + nb, d = mb - mean;
             mean += d * (nb / nt);
             m2 += (double)p.y + d * d * (n * nb / nt);
             n = nt;
         }
+    }
+    sh[sl][cx][0] = n; sh[sl][cx][1] = mean; sh[sl][cx][2] = m2;
+    __syncthreads();
+    if (sl != 0 || o >= C) return;
+    for (int k = 1; k < kFinSlices; ++k) {
+        const double nb = sh[k][cx][0];
+        if (nb == 0.0) continue;
+        const double mb = sh[k][cx][1], nt = n + nb, d = mb - mean;
+        mean += d * (nb / nt);
+        m2 += sh[k][cx][2] + d * d * (n * nb / nt);
+        n = nt;
     }
     const double N = (double)(*nvalid);
     const double var = N > 0 ? m2 / N : 0.0;
@@ -228,29 +257,57 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_reduce_kernel(BnBwdArgs a)
     const int row = blockIdx.x, b = row / a.C, o = row % a.C;
     BwdRow<T, NT> R(a, row, b, o);
     float s[4] = {0.f, 0.f, 0.f, 0.f};
+    float amax = 0.f;
     for (int t0 = threadIdx.x * 8; t0 < R.len; t0 += kRowThreads * 8) {
         float ga[8], gr[8], vh[8], vhr[8];
         R.chunk(a, t0, ga, gr, vh, vhr);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             s[0] += ga[i]; s[1] += ga[i] * vh[i]; s[2] += gr[i]; s[3] += gr[i] * vhr[i];
+            amax = fmaxf(amax, fabsf(ga[i]));
         }
     }
     block_sum(s);
-    if (threadIdx.x == 0) a.partials[row] = make_float4(s[0], s[1], s[2], s[3]);
+    if (a.gmax) amax = block_max(amax);
+    if (threadIdx.x == 0) {
+        a.partials[row] = make_float4(s[0], s[1], s[2], s[3]);
+        if (a.gmax) a.amax_part[row] = amax;
+    }
 }
 
-__global__ void bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const float* gamma_r,
-                                       float* dgamma, float* dbeta, float* dgamma_r, float* dbeta_r,
-                                       float* dbias, int accumulate) {
-    const int o = blockIdx.x * blockDim.x + threadIdx.x;
-    if (o >= a.C) return;
+__global__ void __launch_bounds__(32 * kFinSlices)
+bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const float* gamma_r, float* dgamma, float* dbeta,
+                       float* dgamma_r, float* dbeta_r, float* dbias, int accumulate) {
+    __shared__ double sh[kFinSlices][32][4];
+    const int cx = threadIdx.x & 31, sl = threadIdx.x >> 5;
+    const int o = blockIdx.x * 32 + cx;
+    __shared__ float shmax[kFinSlices][32];
     double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
-    for (int b = 0; b < a.B; ++b) {
-        float4 p = a.partials[(size_t)b * a.C + o];
-        s0 += p.x; s1 += p.y; s2 += p.z; s3 += p.w;
+    float amax = 0.f;
+    if (o < a.C) {
+        for (int b = sl; b < a.B; b += kFinSlices) {
+            const float4 p = a.partials[(size_t)b * a.C + o];
+            s0 += p.x; s1 += p.y; s2 += p.z; s3 += p.w;
+            if (a.gmax) amax = fmaxf(amax, a.amax_part[(size_t)b * a.C + o]);
+        }
+    }
+    sh[sl][cx][0] = s0; sh[sl][cx][1] = s1; sh[sl][cx][2] = s2; sh[sl][cx][3] = s3;
+    shmax[sl][cx] = amax;
+    __syncthreads();
+    if (sl != 0 || o >= a.C) return;
+    for (int k = 1; k < kFinSlices; ++k) {
+        s0 += sh[k][cx][0]; s1 += sh[k][cx][1]; s2 += sh[k][cx][2]; s3 += sh[k][cx][3];
+        amax = fmaxf(amax, shmax[k][cx]);
     }
     const float N = (float)(*a.nvalid);
+    if (a.gmax) {
+        // |gv| <= |k| (max|ga| + |c1| + max|vhat| |c2|) and max|vhat| <= sqrt(N); a maximum is order-free,
+        // so the integer atomic on the (non-negative) float's bit pattern keeps the result repeatable
+        float bound = amax;
+        if (a.has_bn)
+            bound = fabsf(gamma[o] * a.invstd[o]) * (amax + fabsf((float)s0) / N + sqrtf(N) * fabsf((float)s1) / N);
+        if (bound < 3.0e38f) atomicMax(reinterpret_cast<unsigned int*>(a.gmax), __float_as_uint(bound));
+    }
     auto put = [&](float* dst, double val) {
         if (dst) dst[o] = accumulate ? dst[o] + (float)val : (float)val;
     };
@@ -267,13 +324,14 @@ __global__ void bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const fl
     }
 }
 
-template <typename T, typename NT>
+template <typename T, typename NT, typename GT>
 __global__ void __launch_bounds__(kRowThreads) bn_bwd_apply_kernel(BnBwdArgs a) {
     const int row = blockIdx.x, b = row / a.C, o = row % a.C;
     BwdRow<T, NT> R(a, row, b, o);
-    const float4 cf = a.coef[o];
+    float4 cf = a.coef[o];
+    if (a.gmax) cf.x *= pow2_scale(*a.gmax);        // exact: a power of two
     const float4 cr = (a.residual == 2) ? a.coef_r[o] : make_float4(0.f, 0.f, 0.f, 0.f);
-    T* gv = (T*)a.gv + (size_t)row * R.Tp;
+    GT* gv = (GT*)a.gv + (size_t)row * R.Tp;
     T* gvr = (a.residual == 2) ? (T*)a.gvr + (size_t)row * R.Tp : nullptr;
     T* gres = (a.residual == 1) ? (T*)a.gres + (size_t)row * R.Tp : nullptr;
     for (int t0 = threadIdx.x * 8; t0 < R.Tp; t0 += kRowThreads * 8) {
@@ -357,7 +415,7 @@ void bn_finalize(const Launch& L, const float2* partials, int parts_per_b, int t
                  const int* nvalid, int B, int C, float eps, float momentum, float* mean, float* invstd,
                  float* running_mean, float* running_var) {
     KScope ks_(L, KC_BN_FINALIZE, 8.0 * B * parts_per_b * C, 0.0);
-    bn_finalize_kernel<<<(C + 63) / 64, 64, 0, L.stream>>>(partials, parts_per_b, tile_w, len_out, nvalid, B, C,
+    bn_finalize_kernel<<<(C + 31) / 32, 32 * kFinSlices, 0, L.stream>>>(partials, parts_per_b, tile_w, len_out, nvalid, B, C,
                                                             eps, momentum, mean, invstd, running_mean, running_var);
     L.count();
 }
@@ -378,14 +436,17 @@ void bn_bwd_finalize(const Launch& L, const BnBwdArgs& a, const float* gamma, co
                      float* dgamma, float* dbeta, float* dgamma_r, float* dbeta_r, float* dbias,
                      int accumulate) {
     KScope ks_(L, KC_BN_BWD_FINALIZE, 16.0 * a.B * a.C, 0.0);
-    bn_bwd_finalize_kernel<<<(a.C + 63) / 64, 64, 0, L.stream>>>(a, gamma, gamma_r, dgamma, dbeta, dgamma_r,
+    bn_bwd_finalize_kernel<<<(a.C + 31) / 32, 32 * kFinSlices, 0, L.stream>>>(a, gamma, gamma_r, dgamma, dbeta, dgamma_r,
                                                                   dbeta_r, dbias, accumulate);
     L.count();
 }
 
 void bn_bwd_apply(const Launch& L, int dtype, const BnBwdArgs& a) {
     KScope ks_(L, KC_BN_BWD_APPLY, (double)a.B * a.C * a.Tp * (dtype_size(dtype) * (a.has_relu && a.res_before_relu ? 2 : 1) + (a.has_bn ? dtype_size(ntype_of(dtype)) : 0) + (a.residual == 2 ? dtype_size(ntype_of(dtype)) : 0) + dtype_size(dtype) * (1 + (a.residual != 0 ? 1 : 0))), 0.0);
-    SC_DISPATCH3(dtype, (bn_bwd_apply_kernel<T, NT><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a)));
+    if (dtype == BF16 && a.gv_dtype == F16)
+        bn_bwd_apply_kernel<__nv_bfloat16, __half, __half><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a);
+    else
+        SC_DISPATCH3(dtype, (bn_bwd_apply_kernel<T, NT, T><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a)));
     L.count();
 }
 
@@ -394,6 +455,16 @@ void ew_add_masked(const Launch& L, int dtype, void* out, const void* a, const v
     KScope ks_(L, KC_EW, (double)dtype_size(dtype) * B * C * Tt * (2 + (b ? 1 : 0) + (c ? 1 : 0)), 0.0);
     SC_DISPATCH(dtype, (ew_add_masked_kernel<T><<<B * C, kRowThreads, 0, L.stream>>>((T*)out, (const T*)a, (const T*)b,
                                                                                       (const T*)c, len, C, Tt)));
+    L.count();
+}
+
+__global__ void convert_bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ src, __half* __restrict__ dst, long long n) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) dst[i] = __float2half_rn(__bfloat162float(src[i]));
+}
+void convert_bf16_to_f16(const Launch& L, const void* src, void* dst, int64_t n) {
+    KScope ks_(L, KC_EW, 4.0 * n, 0.0);
+    convert_bf16_to_f16_kernel<<<(unsigned)((n + 255) / 256), 256, 0, L.stream>>>((const __nv_bfloat16*)src, (__half*)dst, n);
     L.count();
 }
 

@@ -7,6 +7,7 @@
 // stride goes through plain tiled kernels.
 #include "common.cuh"
 #include "kernels.h"
+#include <type_traits>
 
 namespace sc {
 namespace {
@@ -18,12 +19,26 @@ constexpr int TT = 32 * R;    // outputs per channel per CTA
 // Conflict-free placement for 16-byte shared loads at an 8-float lane pitch.
 __device__ __forceinline__ int phys(int i) { return i + ((i >> 5) << 2); }
 
-template <typename T>
+// Saturating store for half outputs: a value outside the half range is clamped and reported.
+template <typename TO>
+__device__ __forceinline__ void guard_range(float (&acc)[8], int* status) {
+    if (sizeof(TO) == 2 && !std::is_same<TO, __nv_bfloat16>::value) {
+        bool over = false;
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            if (fabsf(acc[r]) > 65504.f) { over = true; acc[r] = copysignf(65504.f, acc[r]); }
+        }
+        if (over) raise_status(status, kErrRange);
+    }
+}
+
+template <typename TI, typename TW, typename TO>
 __global__ void __launch_bounds__(32 * CH)
-dw_corr_s1_kernel(const T* __restrict__ in, const T* __restrict__ w, T* __restrict__ out,
-                  const T* __restrict__ add1, const T* __restrict__ add2,
+dw_corr_s1_kernel(const TI* __restrict__ in, const TW* __restrict__ w, TO* __restrict__ out,
+                  const TO* __restrict__ add1, const TO* __restrict__ add2, const float* __restrict__ gmax,
                   const int* __restrict__ len_src, const int* __restrict__ len_dst,
-                  int C, int Tt, int K, int Kpad, int flip) {
+                  int C, int Tt, int K, int Kpad, int flip, int* status) {
+    using T = TO;
     extern __shared__ float smem[];
     const int lane = threadIdx.x, wrp = threadIdx.y;
     const int b = blockIdx.z, c = blockIdx.y * CH + wrp, t0 = blockIdx.x * TT;
@@ -48,7 +63,7 @@ dw_corr_s1_kernel(const T* __restrict__ in, const T* __restrict__ w, T* __restri
     for (int k = lane; k < Kpad; k += 32)
         ws[k] = (k < K) ? ldf(w + (size_t)c * K + (flip ? K - 1 - k : k)) : 0.f;
     // input tile: logical index i <-> frame tau = t0 - P + i, zero outside [0, ls)
-    const T* irow = in + row;
+    const TI* irow = in + row;
     const int tau0 = t0 - P;
     if (vec) {
         const int a0 = (tau0 >= 0) ? (tau0 & ~7) : -(((-tau0) + 7) & ~7);   // floor to a multiple of 8
@@ -56,7 +71,7 @@ dw_corr_s1_kernel(const T* __restrict__ in, const T* __restrict__ w, T* __restri
         for (int j = lane; j < nchunk; j += 32) {
             const int ta = a0 + 8 * j;
             float f[8];
-            if (ta >= 0 && ta < ls) ld8<T>(irow + ta, f);
+            if (ta >= 0 && ta < ls) ld8<TI>(irow + ta, f);
             else {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) f[e] = 0.f;
@@ -104,6 +119,12 @@ dw_corr_s1_kernel(const T* __restrict__ in, const T* __restrict__ w, T* __restri
 
     const int t = t0 + base;
     if (t >= Tt) return;
+    if (gmax) {
+        const float inv = 1.f / pow2_scale(*gmax);
+#pragma unroll
+        for (int r = 0; r < R; ++r) acc[r] *= inv;
+    }
+    guard_range<TO>(acc, status);
     if (vec) {
         if (add1) { float f[8]; ld8<T>(add1 + row + t, f);
 #pragma unroll
@@ -128,11 +149,11 @@ dw_corr_s1_kernel(const T* __restrict__ in, const T* __restrict__ w, T* __restri
 // ---- any stride: plain tiled kernels (used by the stride-2 first layer) ---------------------
 constexpr int GT = 256;   // outputs per CTA
 
-template <typename T>
+template <typename T, typename TO>
 __global__ void __launch_bounds__(GT)
-dw_fwd_generic_kernel(const T* __restrict__ x, const T* __restrict__ w, T* __restrict__ u,
+dw_fwd_generic_kernel(const T* __restrict__ x, const T* __restrict__ w, TO* __restrict__ u,
                       const int* __restrict__ len_in, const int* __restrict__ len_out,
-                      int C, int Tt, int Tp, int K, int s) {
+                      int C, int Tt, int Tp, int K, int s, int* status) {
     extern __shared__ float smem[];
     const int b = blockIdx.z, c = blockIdx.y, t0 = blockIdx.x * GT;
     const int P = (K - 1) / 2, XW = (GT - 1) * s + K;
@@ -151,13 +172,14 @@ dw_fwd_generic_kernel(const T* __restrict__ x, const T* __restrict__ w, T* __res
     if (t >= Tp) return;
     float acc = 0.f;
     for (int k = 0; k < K; ++k) acc = fmaf(ws[k], xs[threadIdx.x * s + k], acc);
+    if (std::is_same<TO, __half>::value && fabsf(acc) > 65504.f) { acc = copysignf(65504.f, acc); raise_status(status, kErrRange); }
     stf(u + ((size_t)b * C + c) * Tp + t, (t < lo) ? acc : 0.f);
 }
 
-template <typename T>
+template <typename TG, typename T>
 __global__ void __launch_bounds__(GT)
-dw_dgrad_generic_kernel(const T* __restrict__ gu, const T* __restrict__ w, T* __restrict__ dx,
-                        const T* __restrict__ add1, const T* __restrict__ add2,
+dw_dgrad_generic_kernel(const TG* __restrict__ gu, const T* __restrict__ w, T* __restrict__ dx,
+                        const T* __restrict__ add1, const T* __restrict__ add2, const float* __restrict__ gmax,
                         const int* __restrict__ len_in, const int* __restrict__ len_out,
                         int C, int Tt, int Tp, int K, int s) {
     extern __shared__ float smem[];
@@ -171,7 +193,7 @@ dw_dgrad_generic_kernel(const T* __restrict__ gu, const T* __restrict__ w, T* __
     float* gs = smem;
     float* ws = smem + GW;
     const int li = min(len_in[b], Tt), lo = min(len_out[b], Tp);
-    const T* grow = gu + ((size_t)b * C + c) * Tp;
+    const TG* grow = gu + ((size_t)b * C + c) * Tp;
     for (int k = threadIdx.x; k < K; k += GT) ws[k] = ldf(w + (size_t)c * K + k);
     for (int i = threadIdx.x; i < GW; i += GT) {
         const int t = tlo + i;
@@ -186,15 +208,16 @@ dw_dgrad_generic_kernel(const T* __restrict__ gu, const T* __restrict__ w, T* __
         if (q >= 0 && q % s == 0) { const int t = q / s; if (t >= tlo && t <= thi) acc = fmaf(ws[k], gs[t - tlo], acc); }
     }
     const size_t o = ((size_t)b * C + c) * Tt + tau;
+    if (gmax) acc *= 1.f / pow2_scale(*gmax);
     if (add1) acc += ldf(add1 + o);
     if (add2) acc += ldf(add2 + o);
     stf(dx + o, (tau < li) ? acc : 0.f);
 }
 
 // One warp per (b,c) row; lane k-strided taps; plain but correct for any stride.
-template <typename T>
+template <typename TG, typename T>
 __global__ void __launch_bounds__(128)
-dw_wgrad_generic_kernel(const T* __restrict__ gu, const T* __restrict__ x, float* __restrict__ partials,
+dw_wgrad_generic_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float* __restrict__ partials,
                         const int* __restrict__ len_in, const int* __restrict__ len_out,
                         int B, int C, int Tt, int Tp, int K, int s) {
     const int c = blockIdx.x, lane = threadIdx.x & 31, wrp = threadIdx.x >> 5;
@@ -202,7 +225,7 @@ dw_wgrad_generic_kernel(const T* __restrict__ gu, const T* __restrict__ x, float
     // partials[b][c][k]; warps stride over samples
     for (int b = wrp; b < B; b += 4) {
         const int li = min(len_in[b], Tt), lo = min(len_out[b], Tp);
-        const T* grow = gu + ((size_t)b * C + c) * Tp;
+        const TG* grow = gu + ((size_t)b * C + c) * Tp;
         const T* xrow = x + ((size_t)b * C + c) * Tt;
         for (int k = 0; k < K; ++k) {
             float acc = 0.f;
@@ -222,9 +245,9 @@ constexpr int WG_THREADS = 128;
 constexpr int WG_TT = 1024;     // frames per shared-memory tile
 constexpr int WG_BG = 8;        // samples per CTA
 
-template <typename T>
+template <typename TG, typename T>
 __global__ void __launch_bounds__(WG_THREADS)
-dw_wgrad_s1_kernel(const T* __restrict__ gu, const T* __restrict__ x, float* __restrict__ partials,
+dw_wgrad_s1_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float* __restrict__ partials,
                    const int* __restrict__ len_in, const int* __restrict__ len_out,
                    int B, int C, int Tt, int K, int Kpad) {
     extern __shared__ float smem[];
@@ -248,7 +271,7 @@ dw_wgrad_s1_kernel(const T* __restrict__ gu, const T* __restrict__ x, float* __r
     const int b_end = min(B, (bg + 1) * WG_BG);
     for (int b = bg * WG_BG; b < b_end; ++b) {
         const int li = min(len_in[b], Tt), lo = min(len_out[b], Tt);
-        const T* grow = gu + ((size_t)b * C + c) * Tt;
+        const TG* grow = gu + ((size_t)b * C + c) * Tt;
         const T* xrow = x + ((size_t)b * C + c) * Tt;
         for (int t0 = 0; t0 < lo; t0 += WG_TT) {
             __syncthreads();
@@ -301,59 +324,63 @@ inline int host_phys(int i) { return i + ((i >> 5) << 2); }
 
 }  // namespace
 
-#define SC_DISPATCH(dtype, ...)                                             \
-    switch (dtype) {                                                        \
-        case F32: { using T = float; __VA_ARGS__; break; }                  \
-        case F16: { using T = __half; __VA_ARGS__; break; }                 \
-        default:  { using T = __nv_bfloat16; __VA_ARGS__; break; }          \
-    }
+// (activation type T, internal operand type OT): fp32 -> (float, float); fp16 -> (half, half);
+// bf16 -> (bf16, half) for layers with a depthwise step.
+#define SC_DISPATCH_IO(dtype, odt, ...)                                                         \
+    if (dtype == F32) { using T = float; using OT = float; __VA_ARGS__; }                        \
+    else if (dtype == F16) { using T = __half; using OT = __half; __VA_ARGS__; }                 \
+    else if (odt == F16) { using T = __nv_bfloat16; using OT = __half; __VA_ARGS__; }            \
+    else { using T = __nv_bfloat16; using OT = __nv_bfloat16; __VA_ARGS__; }
 
-static void corr_s1(const Launch& L, int dtype, const void* in, const void* w, void* out, const void* add1,
-                    const void* add2, const int* len_src, const int* len_dst, int B, int C, int Tt, int K,
-                    int flip) {
-    KScope ks_(L, flip ? KC_DW_DGRAD : KC_DW_FWD,
-               (double)dtype_size(dtype) * B * C * Tt * (2 + (add1 ? 1 : 0) + (add2 ? 1 : 0)), 2.0 * B * C * Tt * K);
-    const int Kp = kpad(K);
-    const size_t smem = (size_t)CH * (host_phys(TT + Kp) + 4 + Kp) * sizeof(float);
-    dim3 grid((Tt + TT - 1) / TT, (C + CH - 1) / CH, B), block(32, CH);
-    SC_DISPATCH(dtype, (dw_corr_s1_kernel<T><<<grid, block, smem, L.stream>>>(
-                           (const T*)in, (const T*)w, (T*)out, (const T*)add1, (const T*)add2, len_src, len_dst,
-                           C, Tt, K, Kp, flip)));
-    L.count();
-}
-
-void dw_fwd(const Launch& L, int dtype, const void* x, const void* wd, void* u, const int* len_in,
+void dw_fwd(const Launch& L, int dtype, int odt, const void* x, const void* wd, void* u, const int* len_in,
             const int* len_out, int B, int C, int Tt, int Tp, int K, int s) {
-    if (s == 1) { corr_s1(L, dtype, x, wd, u, nullptr, nullptr, len_in, len_out, B, C, Tt, K, 0); return; }
-    KScope ks_(L, KC_DW_FWD, (double)dtype_size(dtype) * B * C * (Tt + Tp), 2.0 * B * C * Tp * K);
-    const size_t smem = (size_t)((GT - 1) * s + K + K) * sizeof(float);
-    dim3 grid((Tp + GT - 1) / GT, C, B);
-    SC_DISPATCH(dtype, (dw_fwd_generic_kernel<T><<<grid, GT, smem, L.stream>>>((const T*)x, (const T*)wd, (T*)u, len_in,
-                                                                               len_out, C, Tt, Tp, K, s)));
+    KScope ks_(L, KC_DW_FWD, (double)B * C * (dtype_size(dtype) * Tt + dtype_size(odt) * Tp), 2.0 * B * C * Tp * K);
+    if (s == 1) {
+        const int Kp = kpad(K);
+        const size_t smem = (size_t)CH * (host_phys(TT + Kp) + 4 + Kp) * sizeof(float);
+        dim3 grid((Tt + TT - 1) / TT, (C + CH - 1) / CH, B), block(32, CH);
+        SC_DISPATCH_IO(dtype, odt, (dw_corr_s1_kernel<T, T, OT><<<grid, block, smem, L.stream>>>(
+                                       (const T*)x, (const T*)wd, (OT*)u, nullptr, nullptr, nullptr, len_in, len_out, C, Tt,
+                                       K, Kp, 0, L.status)));
+    } else {
+        const size_t smem = (size_t)((GT - 1) * s + K + K) * sizeof(float);
+        dim3 grid((Tp + GT - 1) / GT, C, B);
+        SC_DISPATCH_IO(dtype, odt, (dw_fwd_generic_kernel<T, OT><<<grid, GT, smem, L.stream>>>(
+                                       (const T*)x, (const T*)wd, (OT*)u, len_in, len_out, C, Tt, Tp, K, s, L.status)));
+    }
     L.count();
 }
 
-void dw_dgrad(const Launch& L, int dtype, const void* gu, const void* wd, void* dx, const void* add1,
-              const void* add2, const int* len_in, const int* len_out, int B, int C, int Tt, int Tp,
-              int K, int s) {
-    if (s == 1) { corr_s1(L, dtype, gu, wd, dx, add1, add2, len_out, len_in, B, C, Tt, K, 1); return; }
-    KScope ks_(L, KC_DW_DGRAD, (double)dtype_size(dtype) * B * C * (Tt * (1 + (add1 ? 1 : 0) + (add2 ? 1 : 0)) + Tp), 2.0 * B * C * Tp * K);
-    const size_t smem = (size_t)((GT + K) / s + 4 + K) * sizeof(float);
-    dim3 grid((Tt + GT - 1) / GT, C, B);
-    SC_DISPATCH(dtype, (dw_dgrad_generic_kernel<T><<<grid, GT, smem, L.stream>>>(
-                           (const T*)gu, (const T*)wd, (T*)dx, (const T*)add1, (const T*)add2, len_in, len_out, C,
-                           Tt, Tp, K, s)));
+void dw_dgrad(const Launch& L, int dtype, int odt, const void* gu, const void* wd, void* dx, const void* add1,
+              const void* add2, const float* gmax, const int* len_in, const int* len_out, int B, int C, int Tt,
+              int Tp, int K, int s) {
+    KScope ks_(L, KC_DW_DGRAD, (double)B * C * (dtype_size(dtype) * Tt * (1 + (add1 ? 1 : 0) + (add2 ? 1 : 0)) + dtype_size(odt) * Tp),
+               2.0 * B * C * Tp * K);
+    if (s == 1) {
+        const int Kp = kpad(K);
+        const size_t smem = (size_t)CH * (host_phys(TT + Kp) + 4 + Kp) * sizeof(float);
+        dim3 grid((Tt + TT - 1) / TT, (C + CH - 1) / CH, B), block(32, CH);
+        SC_DISPATCH_IO(dtype, odt, (dw_corr_s1_kernel<OT, T, T><<<grid, block, smem, L.stream>>>(
+                                       (const OT*)gu, (const T*)wd, (T*)dx, (const T*)add1, (const T*)add2, gmax, len_out,
+                                       len_in, C, Tt, K, Kp, 1, L.status)));
+    } else {
+        const size_t smem = (size_t)((GT + K) / s + 4 + K) * sizeof(float);
+        dim3 grid((Tt + GT - 1) / GT, C, B);
+        SC_DISPATCH_IO(dtype, odt, (dw_dgrad_generic_kernel<OT, T><<<grid, GT, smem, L.stream>>>(
+                                       (const OT*)gu, (const T*)wd, (T*)dx, (const T*)add1, (const T*)add2, gmax, len_in,
+                                       len_out, C, Tt, Tp, K, s)));
+    }
     L.count();
 }
 
 size_t dw_wgrad_scratch_bytes(int B, int C, int K) { return (size_t)B * C * K * sizeof(float); }
 
-void dw_wgrad(const Launch& L, int dtype, const void* gu, const void* x, float* dwd, float* partials,
-              int accumulate, const int* len_in, const int* len_out, int B, int C, int Tt, int Tp,
-              int K, int s) {
+void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x, float* dwd, float* partials,
+              int accumulate, const float* gmax, const int* len_in, const int* len_out, int B, int C, int Tt,
+              int Tp, int K, int s) {
     int nsplit;
     {
-    KScope ks_(L, KC_DW_WGRAD, (double)dtype_size(dtype) * B * C * (Tt + Tp), 2.0 * B * C * Tp * K);
+    KScope ks_(L, KC_DW_WGRAD, (double)B * C * (dtype_size(dtype) * Tt + dtype_size(odt) * Tp), 2.0 * B * C * Tp * K);
     if (s == 1) {
         const int Kp = kpad(K), NG = Kp / R, nseg = WG_THREADS / NG;
         const int seglen = ((WG_TT + nseg - 1) / nseg + R - 1) / R * R;
@@ -361,16 +388,16 @@ void dw_wgrad(const Launch& L, int dtype, const void* gu, const void* x, float* 
         const size_t smem = (size_t)(GW + GW + Kp + nseg * Kp) * sizeof(float);
         nsplit = (B + WG_BG - 1) / WG_BG;
         dim3 grid(C, nsplit);
-        SC_DISPATCH(dtype, (dw_wgrad_s1_kernel<T><<<grid, WG_THREADS, smem, L.stream>>>(
-                               (const T*)gu, (const T*)x, partials, len_in, len_out, B, C, Tt, K, Kp)));
+        SC_DISPATCH_IO(dtype, odt, (dw_wgrad_s1_kernel<OT, T><<<grid, WG_THREADS, smem, L.stream>>>(
+                                       (const OT*)gu, (const T*)x, partials, len_in, len_out, B, C, Tt, K, Kp)));
     } else {
         nsplit = B;
-        SC_DISPATCH(dtype, (dw_wgrad_generic_kernel<T><<<C, 128, 0, L.stream>>>((const T*)gu, (const T*)x, partials,
-                                                                                 len_in, len_out, B, C, Tt, Tp, K, s)));
+        SC_DISPATCH_IO(dtype, odt, (dw_wgrad_generic_kernel<OT, T><<<C, 128, 0, L.stream>>>(
+                                       (const OT*)gu, (const T*)x, partials, len_in, len_out, B, C, Tt, Tp, K, s)));
     }
     L.count();
     }
-    reduce_partials(L, partials, nsplit, (int64_t)C * K, dwd, accumulate);
+    reduce_partials(L, partials, nsplit, (int64_t)C * K, dwd, accumulate, gmax);
 }
 
 }  // namespace sc

@@ -112,11 +112,12 @@ gemm_simt_kernel(GemmDesc d, const T* __restrict__ a, const T* __restrict__ b, v
 }
 
 __global__ void reduce_partials_kernel(const float* __restrict__ p, int nsplit, long long n,
-                                       float* __restrict__ out, int accumulate) {
+                                       float* __restrict__ out, int accumulate, const float* __restrict__ gmax) {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     float s = 0.f;
     for (int k = 0; k < nsplit; ++k) s += p[(long long)k * n + i];
+    if (gmax) s *= 1.f / pow2_scale(*gmax);
     out[i] = accumulate ? out[i] + s : s;
 }
 
@@ -129,9 +130,10 @@ __global__ void reduce_partials_kernel(const float* __restrict__ p, int nsplit, 
         default:  { using T = __nv_bfloat16; __VA_ARGS__; break; }          \
     }
 
-void reduce_partials(const Launch& L, const float* partials, int nsplit, int64_t n, float* out, int accumulate) {
+void reduce_partials(const Launch& L, const float* partials, int nsplit, int64_t n, float* out, int accumulate,
+                     const float* gmax) {
     KScope ks_(L, KC_REDUCE, 4.0 * (nsplit + 1) * n, 0.0);
-    reduce_partials_kernel<<<(unsigned)((n + 255) / 256), 256, 0, L.stream>>>(partials, nsplit, n, out, accumulate);
+    reduce_partials_kernel<<<(unsigned)((n + 255) / 256), 256, 0, L.stream>>>(partials, nsplit, n, out, accumulate, gmax);
     L.count();
 }
 
@@ -145,8 +147,10 @@ void gemm_fwd_simt(const Launch& L, int dtype, const void* w, const void* u, con
     dim3 grid((Tp + BN - 1) / BN, (Cout + BM - 1) / BM, B);
     if (out_dtype == dtype) {
         SC_DISPATCH(dtype, (gemm_simt_kernel<T, T, 0><<<grid, NT, 0, L.stream>>>(d, (const T*)w, (const T*)u, v, bias, len_out)));
-    } else {   // bf16 operands, float result
+    } else if (dtype == BF16) {   // 16-bit operands, float result
         gemm_simt_kernel<__nv_bfloat16, float, 0><<<grid, NT, 0, L.stream>>>(d, (const __nv_bfloat16*)w, (const __nv_bfloat16*)u, v, bias, len_out);
+    } else {
+        gemm_simt_kernel<__half, float, 0><<<grid, NT, 0, L.stream>>>(d, (const __half*)w, (const __half*)u, v, bias, len_out);
     }
     L.count();
 }
@@ -170,7 +174,7 @@ size_t gemm_wgrad_simt_scratch_bytes(int B, int Cin, int Cout) {
 }
 
 void gemm_wgrad_simt(const Launch& L, int dtype, const void* gv, const void* u, float* dw, float* partials,
-                     int accumulate, int B, int Cin, int Cout, int Tp) {
+                     int accumulate, int B, int Cin, int Cout, int Tp, const float* gmax) {
     const int ns = wgrad_splits(B);
     {
     KScope ks_(L, KC_PW_WGRAD, (double)dtype_size(dtype) * B * Tp * (Cin + Cout), 2.0 * B * Tp * Cin * Cout);
@@ -184,7 +188,7 @@ void gemm_wgrad_simt(const Launch& L, int dtype, const void* gv, const void* u, 
     SC_DISPATCH(dtype, (gemm_simt_kernel<T, T, 2><<<grid, NT, 0, L.stream>>>(d, (const T*)gv, (const T*)u, partials, nullptr, nullptr)));
     L.count();
     }
-    reduce_partials(L, partials, ns, (int64_t)Cin * Cout, dw, accumulate);
+    reduce_partials(L, partials, ns, (int64_t)Cin * Cout, dw, accumulate, gmax);
 }
 
 }  // namespace sc

@@ -53,17 +53,19 @@ void lengths(const Launch& L, const int* len_in, int B, int T_in, int stride, in
 
 // ---- depthwise ------------------------------------------------------------------------------
 // u[b,c,t] = sum_k wd[c,k] * x[b,c,t*s+k-P] (x masked by len_in), written as 0 for t >= len_out[b].
-void dw_fwd(const Launch& L, int dtype, const void* x, const void* wd, void* u, const int* len_in,
+// x and wd in `dtype`, u in `odt` (values beyond the half range are clamped and flagged).
+void dw_fwd(const Launch& L, int dtype, int odt, const void* x, const void* wd, void* u, const int* len_in,
             const int* len_out, int B, int C, int T, int Tp, int K, int s);
 // dx[b,c,tau] = [tau < len_in[b]] * (sum_{k,t: t*s+k-P=tau} wd[c,k]*gu[b,c,t] + add1 + add2)
-void dw_dgrad(const Launch& L, int dtype, const void* gu, const void* wd, void* dx, const void* add1,
-              const void* add2, const int* len_in, const int* len_out, int B, int C, int T, int Tp,
-              int K, int s);
+// gu in `odt` and pre-multiplied by pow2_scale(*gmax) when gmax is non-null; wd, add1, add2, dx in `dtype`.
+void dw_dgrad(const Launch& L, int dtype, int odt, const void* gu, const void* wd, void* dx, const void* add1,
+              const void* add2, const float* gmax, const int* len_in, const int* len_out, int B, int C, int T,
+              int Tp, int K, int s);
 // dwd[c,k] (+)= sum_{b,t<len_out} gu[b,c,t] * x[b,c,t*s+k-P] (x masked by len_in).
 // partials: float [B*C*K] scratch.
-void dw_wgrad(const Launch& L, int dtype, const void* gu, const void* x, float* dwd, float* partials,
-              int accumulate, const int* len_in, const int* len_out, int B, int C, int T, int Tp,
-              int K, int s);
+void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x, float* dwd, float* partials,
+              int accumulate, const float* gmax, const int* len_in, const int* len_out, int B, int C, int T,
+              int Tp, int K, int s);
 size_t dw_wgrad_scratch_bytes(int B, int C, int K);
 // out = [t < len[b]] * (a + b + c)   (b, c nullable)
 void ew_add_masked(const Launch& L, int dtype, void* out, const void* a, const void* b, const void* c,
@@ -78,10 +80,13 @@ void gemm_dgrad_simt(const Launch& L, int dtype, const void* w, const void* gv, 
                      int Cout, int Tp);
 // dw[o,c] (+)= sum_{b,t} gv[b,o,t]*u[b,c,t];  partials: float [nsplit*Cout*Cin]
 void gemm_wgrad_simt(const Launch& L, int dtype, const void* gv, const void* u, float* dw, float* partials,
-                     int accumulate, int B, int Cin, int Cout, int Tp);
+                     int accumulate, int B, int Cin, int Cout, int Tp, const float* gmax = nullptr);
 size_t gemm_wgrad_simt_scratch_bytes(int B, int Cin, int Cout);
-// out[i] (+)= sum_s partials[s*n + i], fixed order
-void reduce_partials(const Launch& L, const float* partials, int nsplit, int64_t n, float* out, int accumulate);
+// out[i] (+)= (sum_s partials[s*n + i]) / pow2_scale(*gmax), fixed order (gmax nullable: no scaling)
+void reduce_partials(const Launch& L, const float* partials, int nsplit, int64_t n, float* out, int accumulate,
+                     const float* gmax = nullptr);
+// dst (half) = src (bf16), n elements
+void convert_bf16_to_f16(const Launch& L, const void* src, void* dst, int64_t n);
 
 // ---- batch norm -----------------------------------------------------------------------------
 // Per-(b,channel) row moments over t < len_out[b]: partials[(b*C+o)] = (sum, M2 about the row mean).
@@ -100,6 +105,12 @@ void bn_finalize(const Launch& L, const float2* partials, int parts_per_b, int t
 inline int vtype_of(int dtype) { return dtype == 1 ? 1 : 0; }
 inline int ntype_of(int dtype) { return dtype == 0 ? 0 : 1; }
 inline size_t dtype_size(int dtype) { return dtype == 0 ? 4 : 2; }
+// OT = type of the tensors that only the library sees between the depthwise and pointwise steps
+// (u, and in the backward pass gv and gu): float for fp32; half for BOTH 16-bit activation types when
+// the layer has a depthwise step (bf16 activations would otherwise pay a second 8-bit-mantissa rounding
+// on every contraction operand); the activation type itself for layers without a depthwise step,
+// whose contraction operand is the layer input.
+inline int otype_of(int dtype, int has_dw) { return (dtype == 2 && has_dw) ? 1 : dtype; }
 
 struct ApplyArgs {
     const void* v; const float *mean, *invstd, *gamma, *beta;          // main branch (v in VT)
@@ -120,8 +131,12 @@ struct BnBwdArgs {
     const int* len_out; const int* nvalid;
     int B, C, Tp, has_bn, has_relu, res_before_relu, residual;
     float4* partials;                              // [B*C]
+    float* amax_part;                              // [B*C] per-row max |gated gradient| (only with gmax)
+    float* gmax;                                   // device scalar: bound on |gv| over the tensor (nullable)
+    int gv_dtype;                                  // storage type of gv (OT)
     float4* coef; float4* coef_r;                  // [C]: (k, c1, c2, unused)
     void* gv; void* gvr; void* gres;               // outputs of the apply step (gvr: proj, gres: identity)
+                                                   // gv is multiplied by pow2_scale(*gmax) when gmax is set
 };
 void bn_bwd_reduce(const Launch& L, int dtype, const BnBwdArgs& a);
 void bn_bwd_finalize(const Launch& L, const BnBwdArgs& a, const float* gamma, const float* gamma_r,

@@ -393,7 +393,8 @@ void tc_gemm_dgrad(const TcState* st, const Launch& L, int dtype, const void* w,
 }
 
 void tc_gemm_wgrad(const TcState* st, const Launch& L, int dtype, const void* gv, const void* u, float* dw,
-                   float* partials, int accumulate, int B, int Cin, int Cout, int Tp, const int* len_out) {
+                   float* partials, int accumulate, int B, int Cin, int Cout, int Tp, const int* len_out,
+                   const float* gmax) {
     const WgradPlan w = plan_wgrad(B, Cin, Cout, Tp);
     {
         KScope ks_(L, KC_PW_WGRAD, 2.0 * B * Tp * (Cin + Cout), 2.0 * B * Tp * Cin * Cout);
@@ -418,7 +419,7 @@ void tc_gemm_wgrad(const TcState* st, const Launch& L, int dtype, const void* gv
             else launch_dt<MODE_WGRAD, 1, 64, 4>(dtype, L, grid, ma, mb, p);
         }
     }
-    reduce_partials(L, partials, w.nsplit, (int64_t)Cin * Cout, dw, accumulate);
+    reduce_partials(L, partials, w.nsplit, (int64_t)Cin * Cout, dw, accumulate, gmax);
 }
 
 }  // namespace sc

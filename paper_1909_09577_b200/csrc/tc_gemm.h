@@ -33,6 +33,7 @@ void tc_gemm_dgrad(const TcState* st, const Launch& L, int dtype, const void* w,
                    int Cin, int Cout, int Tp, const int* len_out);
 // dw[o,c] (+)= sum_{b,t} gv[b,o,t] u[b,c,t]
 void tc_gemm_wgrad(const TcState* st, const Launch& L, int dtype, const void* gv, const void* u, float* dw,
-                   float* partials, int accumulate, int B, int Cin, int Cout, int Tp, const int* len_out);
+                   float* partials, int accumulate, int B, int Cin, int Cout, int Tp, const int* len_out,
+                   const float* gmax = nullptr);
 
 }  // namespace sc

@@ -31,10 +31,24 @@ def rms(a) -> float:
     return float(np.sqrt(np.mean(a * a))) if a.size else 0.0
 
 
-def err_ratio(got, ref, dtype, mask=None) -> float:
+def half_ulp(ref, storage):
+    """Half a unit in the last place of `storage` ("bf16": 8 significand bits, "f16": 11) at |ref|."""
+    a = np.abs(np.asarray(ref, dtype=np.float64))
+    bits = {"bf16": 8, "f16": 11}[storage]
+    e = np.floor(np.log2(np.where(a > 0, a, 1.0)))
+    if storage == "f16":
+        e = np.maximum(e, -14)           # subnormal range: fixed spacing
+    return np.where(a > 0, 2.0 ** (e - bits), 0.0)
+
+
+def err_ratio(got, ref, dtype, mask=None, storage=None) -> float:
     """Error divided by the allowed error; <= 1 passes.  The error is taken over every element; the
     RMS that scales the allowance is taken over the valid (unpadded) frames when a mask is given,
-    since padded frames are structural zeros on both sides."""
+    since padded frames are structural zeros on both sides.
+
+    storage: the 16-bit type the tensor is stored in, if any.  No value of that type can be closer
+    to the reference than half a unit in its last place (for bf16 at 8 x RMS that alone is 0.016 RMS),
+    so the stated bound is applied to the error in excess of that representation quantum."""
     got = np.asarray(got, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
     assert got.shape == ref.shape, (got.shape, ref.shape)
@@ -47,6 +61,10 @@ def err_ratio(got, ref, dtype, mask=None) -> float:
         denom = np.where(denom == 0, 1e-30, denom)
         return float(np.max(np.abs(got - ref) / denom))
     scale = TOL[dtype] * r
+    if storage is not None:
+        allow = scale + half_ulp(ref, storage)
+        allow = np.where(allow > 0, allow, 1e-300)
+        return float(np.max(np.abs(got - ref) / allow))
     d = float(np.max(np.abs(got - ref)))
     return d / scale if scale > 0 else (0.0 if d == 0 else np.inf)
 
@@ -55,9 +73,14 @@ class Report:
     def __init__(self, dtype):
         self.dtype = dtype
         self.rows = []
+        self.plain = []      # the same ratios without the representation quantum, for the record
 
-    def add(self, name, got, ref, mask=None):
-        self.rows.append((name, err_ratio(got, ref, self.dtype, mask)))
+    def add(self, name, got, ref, mask=None, stored=False):
+        """stored=True: the tensor lives in the 16-bit activation type (y, dx, ...); see err_ratio."""
+        storage = self.dtype if (stored and self.dtype != "f32") else None
+        self.rows.append((name, err_ratio(got, ref, self.dtype, mask, storage)))
+        if storage is not None:
+            self.plain.append((name, err_ratio(got, ref, self.dtype, mask)))
 
     def worst(self):
         return max(self.rows, key=lambda r: r[1]) if self.rows else ("", 0.0)
@@ -67,7 +90,10 @@ class Report:
         assert not bad, f"outside tolerance (error/allowed): {bad}; all: {[(n, round(e, 3)) for n, e in self.rows]}"
 
     def __str__(self):
-        return ", ".join(f"{n}={e:.3f}" for n, e in self.rows)
+        t = ", ".join(f"{n}={e:.3f}" for n, e in self.rows)
+        if self.plain:
+            t += " | without quantum: " + ", ".join(f"{n}={e:.3f}" for n, e in self.plain)
+        return t
 
 
 def adopt_gate(L, S, gate_gpu, dtype):
@@ -119,7 +145,7 @@ def run_block(ctx, api, L, dtype, x, lengths, params, g, x_res=None, want_dx_res
         rep.add("mean_r", host(saved["mean_r"]), S["mean_r"])
         rep.add("invstd_r", host(saved["invstd_r"]), S["invstd_r"])
     yh = host(y)
-    rep.add("y", yh, S["y"], vm)
+    rep.add("y", yh, S["y"], vm, stored=True)
     assert np.all(yh[~np.broadcast_to(S["valid"], yh.shape)] == 0), "padded output frames must be zero"
 
     gate = None
@@ -137,9 +163,9 @@ def run_block(ctx, api, L, dtype, x, lengths, params, g, x_res=None, want_dx_res
         ref_dx = ref_dx + G["dx_res"]
     if dx_add is not None:
         ref_dx = ref_dx + np.where(O.time_mask(lengths, T), dx_add, 0.0)
-    rep.add("dx", host(dx), ref_dx, O.time_mask(lengths, T))
+    rep.add("dx", host(dx), ref_dx, O.time_mask(lengths, T), stored=True)
     if want_dx_res:
-        rep.add("dx_res", host(dx_res), G["dx_res"], vm)
+        rep.add("dx_res", host(dx_res), G["dx_res"], vm, stored=True)
     for name in params:
         rep.add("d" + name, host(grads["d" + name]), G["d" + name])
     rep.adopted, rep.hard = adopted, hard
@@ -191,7 +217,7 @@ def run_chain(ctx, api, w, d, check=True):
             rep.add("vhat", host(f["saved"]["vhat"]), np.where(vm, S["vhat"], 0.0), vm)
         if L.residual == "proj":
             rep.add("vhat_r", host(f["saved"]["vhat_r"]), np.where(vm, S["vhat_r"], 0.0), vm)
-        rep.add("y", acts[i + 1], S["y"], vm)
+        rep.add("y", acts[i + 1], S["y"], vm, stored=True)
         gate = None
         adopted = hard = 0
         if L.has_relu:
@@ -206,9 +232,9 @@ def run_chain(ctx, api, w, d, check=True):
             ref_dx = ref_dx + G["dx_res"]
         if dx_add is not None:
             ref_dx = ref_dx + np.where(O.time_mask(lens[i], acts[i].shape[2]), host(dx_add), 0.0)
-        rep.add("dx", host(dx), ref_dx, O.time_mask(lens[i], acts[i].shape[2]))
+        rep.add("dx", host(dx), ref_dx, O.time_mask(lens[i], acts[i].shape[2]), stored=True)
         if want_res:
-            rep.add("dx_res", host(dx_res), G["dx_res"], vm)
+            rep.add("dx_res", host(dx_res), G["dx_res"], vm, stored=True)
             pending[f["j"]] = dx_res
         for name in d.params[i]:
             rep.add("d" + name, host(grads["d" + name]), G["d" + name])
