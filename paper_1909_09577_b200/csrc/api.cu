@@ -454,7 +454,7 @@ int sepconv_fwd(sc_ctx* ctx, const sc_block_desc* desc, const sc_tensor* x, cons
     FwdScratch f;
     plan_fwd(desc, m, ws, &f, &ctx->tc);
     if (!ws.ok()) return SC_ERR_WORKSPACE;
-    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof};
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode};
     BlockIO io{};
     io.x = x->ptr; io.xres = desc->residual != SC_RES_NONE ? (x_res ? x_res->ptr : x->ptr) : nullptr;
     io.y = y->ptr; io.len_in = lengths_dev; io.len_out = f.len_out; io.nvalid = f.nvalid;
@@ -493,7 +493,7 @@ int sepconv_bwd(sc_ctx* ctx, const sc_block_desc* desc, const sc_tensor* dy, con
     BwdScratch s;
     plan_bwd(desc, m, ws, &s, &ctx->tc);
     if (!ws.ok()) return SC_ERR_WORKSPACE;
-    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof};
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode};
     lengths(L, lengths_dev, m.B, m.T, m.s, s.len_out, s.nvalid);
     BwdIO io{};
     io.dy = dy->ptr; io.x = x->ptr; io.y = y->ptr;
@@ -630,7 +630,7 @@ int encoder_fwd_bwd(sc_ctx* ctx, const sc_encoder_desc* e, const sc_tensor* x, c
         SC_TRY(check_params(&P.L[i].d, &prm[i]));
         SC_TRY(check_grads(&P.L[i].d, &grd[i]));
     }
-    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof};
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode};
     auto input_of = [&](int i) -> const void* { return i == 0 ? x->ptr : P.L[i - 1].y; };
     auto len_in_of = [&](int i) -> const int* { return i == 0 ? lengths_dev : P.L[i - 1].len_out; };
     auto res_src = [&](int i) -> int { return (e->res_from && e->res_from[i] >= 0) ? e->res_from[i] : i; };

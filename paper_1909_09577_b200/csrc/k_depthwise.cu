@@ -335,6 +335,10 @@ inline int host_phys(int i) { return i + ((i >> 5) << 2); }
 void dw_fwd(const Launch& L, int dtype, int odt, const void* x, const void* wd, void* u, const int* len_in,
             const int* len_out, int B, int C, int Tt, int Tp, int K, int s) {
     KScope ks_(L, KC_DW_FWD, (double)B * C * (dtype_size(dtype) * Tt + dtype_size(odt) * Tp), 2.0 * B * C * Tp * K);
+    if (!L.simt_only && dw_tc_supported(dtype, Tt, K, s)) {
+        dw_tc_fwd(L, dtype, odt, x, wd, u, len_in, len_out, B, C, Tt, K);
+        return;
+    }
     if (s == 1) {
         const int Kp = kpad(K);
         const size_t smem = (size_t)CH * (host_phys(TT + Kp) + 4 + Kp) * sizeof(float);
@@ -356,6 +360,10 @@ void dw_dgrad(const Launch& L, int dtype, int odt, const void* gu, const void* w
               int Tp, int K, int s) {
     KScope ks_(L, KC_DW_DGRAD, (double)B * C * (dtype_size(dtype) * Tt * (1 + (add1 ? 1 : 0) + (add2 ? 1 : 0)) + dtype_size(odt) * Tp),
                2.0 * B * C * Tp * K);
+    if (!L.simt_only && dw_tc_supported(dtype, Tt, K, s)) {
+        dw_tc_dgrad(L, dtype, odt, gu, wd, dx, add1, add2, gmax, len_in, len_out, B, C, Tt, K);
+        return;
+    }
     if (s == 1) {
         const int Kp = kpad(K);
         const size_t smem = (size_t)CH * (host_phys(TT + Kp) + 4 + Kp) * sizeof(float);

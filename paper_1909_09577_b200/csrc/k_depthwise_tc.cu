@@ -1,0 +1,212 @@
+// Stride-1 depthwise correlation on the tensor cores (forward and input gradient).
+//
+// For one channel the K-tap correlation over time is a banded Toeplitz product.  Time is cut into
+// blocks of 64 frames; output block i only needs input blocks i-1, i, i+1 (K <= 129):
+//     U_i[j] = sum_{d in {-1,0,1}} sum_{j'} X_{i+d}[j'] * T_d[j', j],   T_d[j', j] = w[j' + 64 d - j + P].
+// The MMA runs with the 64-frame blocks of many samples as its M rows, the 64 positions inside a
+// block as N, and the position inside the input block as the contraction:  D = sum_d A_d * T_d with
+// fp32 accumulation in tensor memory.  A is staged by the CTA's threads (coalesced 16-byte loads)
+// into a no-swizzle layout whose rows sit 16 bytes apart inside each 8-element column chunk, so the
+// shifted operand A_d is the same buffer with its start address moved by d rows -- the input is read
+// from HBM once and staged once.  Every sample's row run carries one zero block in front and behind
+// (the "same" padding and the separation between samples); their output rows are discarded.
+// Frames at or beyond a sample's length are zeroed while staging (the padding mask).  After
+// tcgen05.ld a thread owns one whole 64-frame output block: 128 contiguous bytes per lane, lanes
+// contiguous, so stores coalesce.  The input gradient is the same product with the taps flipped.
+#include <type_traits>
+
+#include "common.cuh"
+#include "kernels.h"
+#include "sm100.cuh"
+
+namespace sc {
+namespace {
+
+constexpr int NB = 64;              // frames per block
+constexpr int MAXROWS = 256;        // block rows (incl. separators) per CTA: two MMA M-tiles
+constexpr int ROWS_ALLOC = 264;     // + one slack row in front, a few behind
+constexpr int kThreads = 128;
+
+__device__ __forceinline__ uint64_t desc_noswz(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46);
+}
+
+template <typename T> struct Fmt16;
+template <> struct Fmt16<__half> { static constexpr uint32_t v = 0; };
+template <> struct Fmt16<__nv_bfloat16> { static constexpr uint32_t v = 1; };
+
+template <typename T> __device__ __forceinline__ unsigned short bits16(float v);
+template <> __device__ __forceinline__ unsigned short bits16<__half>(float v) { return __half_as_ushort(__float2half_rn(v)); }
+template <> __device__ __forceinline__ unsigned short bits16<__nv_bfloat16>(float v) { return __bfloat16_as_ushort(__float2bfloat16_rn(v)); }
+
+// TI: type of the input tensor and of both MMA operands; TW: tap type; TO: output (and add1/add2) type.
+template <typename TI, typename TW, typename TO, bool FLIP>
+__global__ void __launch_bounds__(kThreads)
+dw_tc_kernel(const TI* __restrict__ in, const TW* __restrict__ w, TO* __restrict__ out,
+             const TO* __restrict__ add1, const TO* __restrict__ add2, const float* __restrict__ gmax,
+             const int* __restrict__ len_src, const int* __restrict__ len_dst,
+             int B, int C, int Tt, int K, int nb, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
+    uint4* A16 = reinterpret_cast<uint4*>(smem);                        // [8 chunks][ROWS_ALLOC] 16-byte units
+    uint4* B16 = A16 + 8 * ROWS_ALLOC;                                  // [3 shifts][8 chunks][64 rows]
+    float* taps = reinterpret_cast<float*>(B16 + 3 * 8 * 64);           // [K], K <= 129
+    uint64_t* bar = reinterpret_cast<uint64_t*>(taps + 132);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int c = blockIdx.x, b0 = blockIdx.y * nb;
+    const int nbh = min(nb, B - b0);                 // samples in this CTA
+    const int nblk = (Tt + NB - 1) / NB, S = nblk + 2;
+    const int rows = nbh * S;
+    const int nmt = (rows + 127) / 128;
+    const int P = (K - 1) / 2;
+    const int vpr = Tt / 8;                          // 16-byte vectors per row (Tt is a multiple of 8)
+
+    if (tid == 0) { ptx::mbar_init(bar, 1); ptx::fence_barrier_init(); }
+    if (warp == 0) { ptx::tmem_alloc(tmem_slot, 128); ptx::tmem_relinquish(); }
+    for (int i = tid; i < 8 * ROWS_ALLOC; i += kThreads) A16[i] = make_uint4(0, 0, 0, 0);
+    for (int k = tid; k < K; k += kThreads) taps[k] = ldf(w + (size_t)c * K + k);
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    // ---- stage the input rows: frame t = 64 i + 8 q + e  ->  A16[q][1 + seg*S + 1 + i] ----
+    for (int idx = tid; idx < nbh * vpr; idx += kThreads) {
+        const int seg = idx / vpr, vq = idx - seg * vpr, t = vq * 8;
+        const int ls = min(len_src[b0 + seg], Tt);
+        if (t >= ls) continue;
+        uint4 v = *reinterpret_cast<const uint4*>(in + ((size_t)(b0 + seg) * C + c) * Tt + t);
+        if (t + 8 > ls) {                            // the length falls inside this vector
+            unsigned short* h = reinterpret_cast<unsigned short*>(&v);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) if (t + e >= ls) h[e] = 0;
+        }
+        A16[(vq & 7) * ROWS_ALLOC + 1 + seg * S + 1 + (vq >> 3)] = v;
+    }
+    // ---- Toeplitz blocks: B16[d][q][n] holds T_d[j' = 8q..8q+7, j = n] ----
+    for (int idx = tid; idx < 3 * 8 * 64; idx += kThreads) {
+        const int d = idx / 512, q = (idx >> 6) & 7, n = idx & 63;
+        uint4 v;
+        unsigned short* h = reinterpret_cast<unsigned short*>(&v);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int delta = 8 * q + e + NB * (d - 1) - n;      // input position minus output position
+            const int kk = FLIP ? P - delta : delta + P;
+            h[e] = (kk >= 0 && kk < K) ? bits16<TI>(taps[kk]) : (unsigned short)0;
+        }
+        B16[idx] = v;
+    }
+    ptx::fence_proxy_async();                        // generic-proxy writes -> visible to the tensor core
+    __syncthreads();
+
+    if (tid == 0) {
+        constexpr uint32_t IDESC = ptx::instr_desc(Fmt16<TI>::v, 0, 0, 128, NB);
+        const uint32_t aA = ptx::smem_u32(A16), aB = ptx::smem_u32(B16);
+        for (int mt = 0; mt < nmt; ++mt) {
+#pragma unroll
+            for (int d = 0; d < 3; ++d) {
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    const uint64_t adesc = desc_noswz(aA + ((2 * ks) * ROWS_ALLOC + 1 + mt * 128 + (d - 1)) * 16,
+                                                      ROWS_ALLOC * 16, 128);
+                    const uint64_t bdesc = desc_noswz(aB + (d * 8 + 2 * ks) * 1024, 1024, 128);
+                    ptx::mma_f16(tmem + mt * NB, adesc, bdesc, IDESC, (d > 0 || ks > 0) ? 1u : 0u);
+                }
+            }
+        }
+        ptx::mma_commit(bar);
+    }
+    __syncwarp();
+
+    bool ok = ptx::mbar_wait(bar, 0);
+    ok = __all_sync(0xffffffffu, ok);
+    ptx::tc_fence_after();
+    if (ok) {
+        const float inv = gmax ? 1.f / pow2_scale(*gmax) : 1.f;
+        for (int mt = 0; mt < nmt; ++mt) {
+            const int Rw = mt * 128 + warp * 32 + lane;
+            const int seg = Rw / S, sr = Rw - seg * S;
+            const bool live = (Rw < rows) && sr >= 1 && sr <= nblk;
+            const int b = b0 + seg;
+            const int ld = live ? min(len_dst[b], Tt) : 0;
+            const size_t rbase = ((size_t)b * C + c) * Tt;
+#pragma unroll 1
+            for (int h = 0; h < 2; ++h) {
+                uint32_t r[32];
+                ptx::tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + mt * NB + 32 * h, r);
+                ptx::tmem_ld_wait();
+                if (!live) continue;
+#pragma unroll
+                for (int g8 = 0; g8 < 4; ++g8) {
+                    const int t = (sr - 1) * NB + 32 * h + 8 * g8;
+                    if (t >= Tt) break;
+                    float f[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(r[8 * g8 + e]) * inv;
+                    if (t < ld) {
+                        if (add1) { float a[8]; ld8<TO>(add1 + rbase + t, a);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) f[e] += a[e]; }
+                        if (add2) { float a[8]; ld8<TO>(add2 + rbase + t, a);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) f[e] += a[e]; }
+                    }
+                    bool over = false;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        if (t + e >= ld) f[e] = 0.f;
+                        if (std::is_same<TO, __half>::value && fabsf(f[e]) > 65504.f) { f[e] = copysignf(65504.f, f[e]); over = true; }
+                    }
+                    if (over) raise_status(status, kErrRange);
+                    st8<TO>(out + rbase + t, f);
+                }
+            }
+        }
+    } else if (tid == 0) {
+        raise_status(status, kErrTimeout);
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 0) ptx::tmem_dealloc(tmem, 128);
+}
+
+constexpr size_t kSmemBytes = (size_t)(8 * ROWS_ALLOC + 3 * 8 * 64) * 16 + 132 * 4 + 64 + 128;
+
+template <typename TI, typename TW, typename TO, bool FLIP>
+void launch_tc(const Launch& L, const void* in, const void* w, void* out, const void* add1, const void* add2,
+               const float* gmax, const int* len_src, const int* len_dst, int B, int C, int Tt, int K) {
+    auto kern = dw_tc_kernel<TI, TW, TO, FLIP>;
+    static bool configured = false;
+    if (!configured) { cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes); configured = true; }
+    const int S = (Tt + NB - 1) / NB + 2;
+    const int nb = std::max(1, std::min(B, MAXROWS / S));
+    dim3 grid(C, (B + nb - 1) / nb);
+    kern<<<grid, kThreads, kSmemBytes, L.stream>>>((const TI*)in, (const TW*)w, (TO*)out, (const TO*)add1, (const TO*)add2,
+                                                   gmax, len_src, len_dst, B, C, Tt, K, nb, L.status);
+    L.count();
+}
+
+}  // namespace
+
+bool dw_tc_supported(int dtype, int Tt, int K, int s) {
+    return dtype != F32 && s == 1 && Tt % 8 == 0 && K <= 129 && (Tt + NB - 1) / NB + 2 <= MAXROWS;
+}
+
+void dw_tc_fwd(const Launch& L, int dtype, int odt, const void* x, const void* wd, void* u, const int* len_in,
+               const int* len_out, int B, int C, int Tt, int K) {
+    if (dtype == F16) launch_tc<__half, __half, __half, false>(L, x, wd, u, nullptr, nullptr, nullptr, len_in, len_out, B, C, Tt, K);
+    else if (odt == F16) launch_tc<__nv_bfloat16, __nv_bfloat16, __half, false>(L, x, wd, u, nullptr, nullptr, nullptr, len_in, len_out, B, C, Tt, K);
+    else launch_tc<__nv_bfloat16, __nv_bfloat16, __nv_bfloat16, false>(L, x, wd, u, nullptr, nullptr, nullptr, len_in, len_out, B, C, Tt, K);
+}
+
+void dw_tc_dgrad(const Launch& L, int dtype, int odt, const void* gu, const void* wd, void* dx, const void* add1,
+                 const void* add2, const float* gmax, const int* len_in, const int* len_out, int B, int C, int Tt,
+                 int K) {
+    if (dtype == F16) launch_tc<__half, __half, __half, true>(L, gu, wd, dx, add1, add2, gmax, len_out, len_in, B, C, Tt, K);
+    else if (odt == F16) launch_tc<__half, __nv_bfloat16, __nv_bfloat16, true>(L, gu, wd, dx, add1, add2, gmax, len_out, len_in, B, C, Tt, K);
+    else launch_tc<__nv_bfloat16, __nv_bfloat16, __nv_bfloat16, true>(L, gu, wd, dx, add1, add2, gmax, len_out, len_in, B, C, Tt, K);
+}
+
+}  // namespace sc

@@ -30,6 +30,7 @@ struct Launch {
     int* status;          // device status word
     int64_t* counter;     // host launch counter
     Prof* prof = nullptr;
+    int simt_only = 0;    // 1: never take a tensor-core kernel (used by tests)
     void count(int n = 1) const { if (counter) *counter += n; }
 };
 
@@ -67,6 +68,13 @@ void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x
               int accumulate, const float* gmax, const int* len_in, const int* len_out, int B, int C, int T,
               int Tp, int K, int s);
 size_t dw_wgrad_scratch_bytes(int B, int C, int K);
+// Tensor-core forms of the stride-1 depthwise forward / input gradient (16-bit types, K <= 129).
+bool dw_tc_supported(int dtype, int T, int K, int s);
+void dw_tc_fwd(const Launch& L, int dtype, int odt, const void* x, const void* wd, void* u, const int* len_in,
+               const int* len_out, int B, int C, int T, int K);
+void dw_tc_dgrad(const Launch& L, int dtype, int odt, const void* gu, const void* wd, void* dx, const void* add1,
+                 const void* add2, const float* gmax, const int* len_in, const int* len_out, int B, int C, int T,
+                 int K);
 // out = [t < len[b]] * (a + b + c)   (b, c nullable)
 void ew_add_masked(const Launch& L, int dtype, void* out, const void* a, const void* b, const void* c,
                    const int* len, int B, int C, int T);
