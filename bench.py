@@ -144,6 +144,10 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=4, choices=[4, 5])
+    ap.add_argument("--block", default=None,
+                    help="profile aid: time one sepconv block instead of the encoder, as C_in,C_out,K,B,T "
+                         "(e.g. 512,512,63,32,800); residual projection from the block input")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end (host buffers) leg")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--profile-class", default=DOMINANT_CLASS)
     ap.add_argument("--breakdown", default=None, help="write a per-kernel-class event-time table to this file")
@@ -168,6 +172,10 @@ def main():
     dev = torch.device("cuda", local)
 
     w = si.config(args.config)
+    if args.block:
+        ci, co, k, bb, tt = [int(q) for q in args.block.split(",")]
+        w = si.Workload(f"block_{ci}_{co}_k{k}_B{bb}_T{tt}", "bf16", bb, tt,
+                        [si.LayerCfg(ci, co, K=k, residual="proj")], seed=5)
     d = si.draw(w)
     ctx = api.Context(local)
     ctx.set_gemm_mode(args.gemm_mode)
@@ -233,9 +241,12 @@ def main():
     clocks = sampler.stop(t0, t1) if sampler else None
 
     # ---- end to end: pinned host inputs in, logits + gradients out, every step --------------------
-    for _ in range(2):
-        step_e2e()
-    ms_e2e, _, _ = timed(step_e2e, args.steps)
+    if args.no_e2e:
+        ms_e2e = float("nan")
+    else:
+        for _ in range(2):
+            step_e2e()
+        ms_e2e, _, _ = timed(step_e2e, args.steps)
     h2d = x_h.numel() * x_h.element_size() + g_h.numel() * g_h.element_size() + len_h.numel() * 4
     d2h = logits_h.numel() * logits_h.element_size() + grads_h.numel()
 

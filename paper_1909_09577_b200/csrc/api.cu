@@ -92,6 +92,7 @@ struct BlockIO {                 // raw pointers after validation
     const int* len_in; int* len_out; int* nvalid;
     bool x_clean, res_clean;     // inputs known to be zero in padded frames
     bool lengths_ready;          // len_out / nvalid already computed
+    void* w16_keep;              // optional: where to leave the float16 copy of wp for the backward pass
 };
 
 // Type of the library-internal contraction operands (u, gv, gu) of this layer.
@@ -157,7 +158,11 @@ int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
         return SC_OK;
     }
     const void* wp_op = p->wp;
-    if (odt != dt) { convert_bf16_to_f16(L, p->wp, f.w16, (int64_t)m.Cout * m.Cin); wp_op = f.w16; }
+    if (odt != dt) {
+        void* dst = io.w16_keep ? io.w16_keep : f.w16;
+        convert_bf16_to_f16(L, p->wp, dst, (int64_t)m.Cout * m.Cin);
+        wp_op = dst;
+    }
     pointwise_bn(ctx, L, d, m, m.Cin, odt, wp_op, u, f.v, io.len_out, io.nvalid, sv->mean, sv->invstd, f.partials,
                  rmean, rvar);
     ApplyArgs a{};
@@ -231,6 +236,7 @@ struct BwdIO {
     void *dx, *dx_res; const void* dx_add;
     const int* len_in; const int* len_out; const int* nvalid;
     bool x_clean, res_clean;
+    const void* w16_kept;        // float16 copy of wp left by the forward pass (optional)
 };
 
 int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const Dims& m, BwdIO io,
@@ -261,7 +267,10 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
     const void* u = d->has_dw ? sv->u : (io.x_clean ? io.x : sv->u);
     pointwise_wgrad(ctx, L, odt, s.gv, u, g->dwp, s.wpart, acc, m.B, m.Cin, m.Cout, m.Tp, io.len_out, gmax);
     const void* wp_op = p->wp;
-    if (odt != dt) { convert_bf16_to_f16(L, p->wp, s.w16, (int64_t)m.Cout * m.Cin); wp_op = s.w16; }
+    if (odt != dt) {
+        if (io.w16_kept) wp_op = io.w16_kept;
+        else { convert_bf16_to_f16(L, p->wp, s.w16, (int64_t)m.Cout * m.Cin); wp_op = s.w16; }
+    }
 
     const void* extra = nullptr;    // residual-path gradient to fold into dx
     if (d->residual == SC_RES_PROJ) {
@@ -510,7 +519,7 @@ int sepconv_bwd(sc_ctx* ctx, const sc_block_desc* desc, const sc_tensor* dy, con
 namespace {
 struct LayerPlan {
     sc_block_desc d; Dims m;
-    sc_block_saved sv; void* y; int* len_out; int* nvalid;
+    sc_block_saved sv; void* y; int* len_out; int* nvalid; void* w16;
     bool own_lengths;
 };
 struct EncPlan {
@@ -561,6 +570,7 @@ int plan_encoder(const sc_encoder_desc* e, void* base, size_t cap, EncPlan* P, c
             lp.sv.mean_r = (float*)ws.take(4 * m.Cout); lp.sv.invstd_r = (float*)ws.take(4 * m.Cout);
         }
         lp.y = (i + 1 < e->n_layers) ? ws.take(es * B * m.Cout * m.Tp) : nullptr;
+        lp.w16 = (op_dtype(&lp.d) != lp.d.io_dtype) ? ws.take((size_t)2 * m.Cout * m.Cin) : nullptr;
         max_act = std::max(max_act, es * B * (size_t)m.Cin * m.T);
         max_act = std::max(max_act, es * B * (size_t)m.Cout * m.Tp);
         C = m.Cout; T = m.Tp;
@@ -647,6 +657,7 @@ int encoder_fwd_bwd(sc_ctx* ctx, const sc_encoder_desc* e, const sc_tensor* x, c
         io.len_in = len_in_of(i); io.len_out = lp.len_out; io.nvalid = lp.nvalid;
         io.x_clean = i > 0; io.res_clean = lp.d.residual != SC_RES_NONE && res_src(i) > 0;
         io.lengths_ready = !lp.own_lengths;
+        io.w16_keep = lp.w16;
         SC_TRY(block_fwd_impl(ctx, L, &lp.d, lp.m, io, &prm[i], &lp.sv, nullptr, nullptr, f));
     }
     if (out_lengths_dev)
@@ -668,6 +679,7 @@ int encoder_fwd_bwd(sc_ctx* ctx, const sc_encoder_desc* e, const sc_tensor* x, c
         io.dx_add = has_pending[i] ? P.pending : nullptr;
         io.len_in = len_in_of(i); io.len_out = lp.len_out; io.nvalid = lp.nvalid;
         io.x_clean = i > 0; io.res_clean = lp.d.residual != SC_RES_NONE && res_src(i) > 0;
+        io.w16_kept = lp.w16;
         SC_TRY(block_bwd_impl(ctx, L, &lp.d, lp.m, io, &prm[i], &lp.sv, &grd[i], accumulate, s));
         g = io.dx;
     }

@@ -9,7 +9,12 @@
 namespace sc {
 namespace {
 
-constexpr int kRowThreads = 128;
+constexpr int kRowThreads = 256;          // 8 warps per CTA, one (sample, channel) row per warp
+constexpr int kRowsPerCta = kRowThreads / 32;
+#define SC_ROW_SETUP(nrows)                                                  \
+    const int row = blockIdx.x * kRowsPerCta + (threadIdx.x >> 5);          \
+    if (row >= (nrows)) return;                                              \
+    const int lane = threadIdx.x & 31;
 
 template <typename T>
 __device__ __forceinline__ void load_chunk(const T* row, int t0, int Tp, bool vec, float (&f)[8]) {
@@ -24,39 +29,14 @@ __device__ __forceinline__ void store_chunk(T* row, int t0, int Tp, bool vec, co
     for (int i = 0; i < 8; ++i) if (t0 + i < Tp) stf(row + t0 + i, f[i]);
 }
 
-// Sum of `v` over the CTA (kRowThreads threads); result valid in every thread.
+// Sum of `v` over the warp that owns the row; result valid in every lane.
 template <int N>
 __device__ __forceinline__ void block_sum(float (&v)[N]) {
-    __shared__ float sh[N][kRowThreads / 32];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
     for (int i = 0; i < N; ++i) v[i] = warp_sum(v[i]);
-    __syncthreads();   // protect sh against a previous use
-    if (lane == 0) {
-#pragma unroll
-        for (int i = 0; i < N; ++i) sh[i][warp] = v[i];
-    }
-    __syncthreads();
-#pragma unroll
-    for (int i = 0; i < N; ++i) {
-        float s = 0.f;
-#pragma unroll
-        for (int w = 0; w < kRowThreads / 32; ++w) s += sh[i][w];
-        v[i] = s;
-    }
 }
 
-__device__ __forceinline__ float block_max(float v) {
-    __shared__ float shm[kRowThreads / 32];
-    v = warp_max(v);
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) shm[threadIdx.x >> 5] = v;
-    __syncthreads();
-    float m = shm[0];
-#pragma unroll
-    for (int w = 1; w < kRowThreads / 32; ++w) m = fmaxf(m, shm[w]);
-    return m;
-}
+__device__ __forceinline__ float block_max(float v) { return warp_max(v); }
 
 __global__ void lengths_kernel(const int* __restrict__ len_in, int B, int T_in, int stride,
                                int* __restrict__ len_out, int* __restrict__ nvalid, int* status) {
@@ -79,14 +59,15 @@ __global__ void lengths_kernel(const int* __restrict__ len_in, int B, int T_in, 
 
 template <typename T>
 __global__ void __launch_bounds__(kRowThreads)
-bn_stats_kernel(const T* __restrict__ v, const int* __restrict__ len_out, int C, int Tp,
+bn_stats_kernel(const T* __restrict__ v, const int* __restrict__ len_out, int nrows, int C, int Tp,
                 float2* __restrict__ partials) {
-    const int row = blockIdx.x, b = row / C;
+    SC_ROW_SETUP(nrows)
+    const int b = row / C;
     const int len = min(len_out[b], Tp);
     const T* p = v + (size_t)row * Tp;
     const bool vec = (Tp % 8 == 0);
     float s[1] = {0.f};
-    for (int t0 = threadIdx.x * 8; t0 < len; t0 += kRowThreads * 8) {
+    for (int t0 = lane * 8; t0 < len; t0 += 256) {
         float f[8];
         load_chunk(p, t0, Tp, vec, f);
 #pragma unroll
@@ -95,53 +76,62 @@ bn_stats_kernel(const T* __restrict__ v, const int* __restrict__ len_out, int C,
     block_sum(s);
     const float mean = len > 0 ? s[0] / (float)len : 0.f;
     float q[1] = {0.f};
-    for (int t0 = threadIdx.x * 8; t0 < len; t0 += kRowThreads * 8) {
+    for (int t0 = lane * 8; t0 < len; t0 += 256) {
         float f[8];
         load_chunk(p, t0, Tp, vec, f);
 #pragma unroll
         for (int i = 0; i < 8; ++i) if (t0 + i < len) { float d = f[i] - mean; q[0] += d * d; }
     }
     block_sum(q);
-    if (threadIdx.x == 0) partials[row] = make_float2(s[0], q[0]);
+    if (lane == 0) partials[row] = make_float2(s[0], q[0]);
 }
 
-// 32 channels x 8 part-slices per CTA: slice s merges parts s, s+8, ... in increasing order, then the
-// eight slice results are merged in slice order -- a fixed tree, so the result is bit-repeatable.
-constexpr int kFinSlices = 8;
+// 32 channels x 32 part-slices per CTA.  Pass 1 sums the partial sums (slice s takes parts s, s+32, ...
+// in increasing order; the slice results are then added in slice order), which gives the mean; pass 2
+// sums M2_p + n_p (mean_p - mean)^2 the same way.  The order is fixed, so the result is bit-repeatable,
+// and no term depends on the previous one, so the loads and divisions pipeline.
+constexpr int kFinSlices = 32;
 __global__ void __launch_bounds__(32 * kFinSlices)
 bn_finalize_kernel(const float2* __restrict__ partials, int parts_per_b, int tile_w,
                    const int* __restrict__ len_out, const int* __restrict__ nvalid, int B,
                    int C, float eps, float momentum, float* __restrict__ mean_out,
                    float* __restrict__ invstd_out, float* running_mean, float* running_var) {
-    __shared__ double sh[kFinSlices][32][3];
+    __shared__ double sh[kFinSlices][33];
+    __shared__ double sh_mean[32];
     const int cx = threadIdx.x & 31, sl = threadIdx.x >> 5;
     const int o = blockIdx.x * 32 + cx;
-    double n = 0.0, mean = 0.0, m2 = 0.0;
-    if (o < C) {
-        const int nparts = B * parts_per_b;
+    const int nparts = B * parts_per_b;
+    const double N = (double)(*nvalid);
+    double s1 = 0.0;
+    if (o < C)
         for (int pi = sl; pi < nparts; pi += kFinSlices) {
             const int b = pi / parts_per_b, j = pi - b * parts_per_b;
-            const int cnt = min(max(len_out[b] - j * tile_w, 0), tile_w);
+            if (len_out[b] - j * tile_w > 0) s1 += (double)partials[(size_t)pi * C + o].x;
+        }
+    sh[sl][cx] = s1;
+    __syncthreads();
+    if (sl == 0) {
+        double t = 0.0;
+        for (int k = 0; k < kFinSlices; ++k) t += sh[k][cx];
+        sh_mean[cx] = N > 0 ? t / N : 0.0;
+    }
+    __syncthreads();
+    const double mean = sh_mean[cx];
+    double q = 0.0;
+    if (o < C)
+        for (int pi = sl; pi < nparts; pi += kFinSlices) {
+            const int b = pi / parts_per_b, j = pi - b * parts_per_b;
+            const int cnt = min(len_out[b] - j * tile_w, tile_w);
             if (cnt <= 0) continue;
             const float2 p = partials[(size_t)pi * C + o];
-            const double nb = cnt, mb = (double)p.x / nb, nt = n + nb, d = mb - mean;
-            mean += d * (nb / nt);
-            m2 += (double)p.y + d * d * (n * nb / nt);
-            n = nt;
+            const double d = (double)p.x / (double)cnt - mean;
+            q += (double)p.y + (double)cnt * d * d;
         }
-    }
-    sh[sl][cx][0] = n; sh[sl][cx][1] = mean; sh[sl][cx][2] = m2;
+    sh[sl][cx] = q;
     __syncthreads();
     if (sl != 0 || o >= C) return;
-    for (int k = 1; k < kFinSlices; ++k) {
-        const double nb = sh[k][cx][0];
-        if (nb == 0.0) continue;
-        const double mb = sh[k][cx][1], nt = n + nb, d = mb - mean;
-        mean += d * (nb / nt);
-        m2 += sh[k][cx][2] + d * d * (n * nb / nt);
-        n = nt;
-    }
-    const double N = (double)(*nvalid);
+    double m2 = 0.0;
+    for (int k = 0; k < kFinSlices; ++k) m2 += sh[k][cx];
     const double var = N > 0 ? m2 / N : 0.0;
     const float invstd = (float)(1.0 / sqrt(var + (double)eps));
     const float mu = (float)mean;
@@ -156,7 +146,8 @@ bn_finalize_kernel(const float2* __restrict__ partials, int parts_per_b, int til
 
 template <typename T, typename VT, typename NT>
 __global__ void __launch_bounds__(kRowThreads) bn_apply_kernel(ApplyArgs a) {
-    const int row = blockIdx.x, b = row / a.C, o = row % a.C;
+    SC_ROW_SETUP(a.B * a.C)
+    const int b = row / a.C, o = row % a.C;
     const int Tp = a.Tp, len = min(a.len_out[b], Tp);
     const bool vec = (Tp % 8 == 0);
     const size_t off = (size_t)row * Tp;
@@ -169,7 +160,7 @@ __global__ void __launch_bounds__(kRowThreads) bn_apply_kernel(ApplyArgs a) {
     const float mu = a.mean[o], is = a.invstd[o], ga = a.gamma[o], be = a.beta[o];
     float mur = 0.f, isr = 0.f, gar = 0.f, ber = 0.f;
     if (a.residual == 2) { mur = a.mean_r[o]; isr = a.invstd_r[o]; gar = a.gamma_r[o]; ber = a.beta_r[o]; }
-    for (int t0 = threadIdx.x * 8; t0 < Tp; t0 += kRowThreads * 8) {
+    for (int t0 = lane * 8; t0 < Tp; t0 += 256) {
         float out[8], n1[8], n2[8];
         if (t0 < len) {
             float f[8], r[8];
@@ -254,11 +245,12 @@ struct BwdRow {
 
 template <typename T, typename NT>
 __global__ void __launch_bounds__(kRowThreads) bn_bwd_reduce_kernel(BnBwdArgs a) {
-    const int row = blockIdx.x, b = row / a.C, o = row % a.C;
+    SC_ROW_SETUP(a.B * a.C)
+    const int b = row / a.C, o = row % a.C;
     BwdRow<T, NT> R(a, row, b, o);
     float s[4] = {0.f, 0.f, 0.f, 0.f};
     float amax = 0.f;
-    for (int t0 = threadIdx.x * 8; t0 < R.len; t0 += kRowThreads * 8) {
+    for (int t0 = lane * 8; t0 < R.len; t0 += 256) {
         float ga[8], gr[8], vh[8], vhr[8];
         R.chunk(a, t0, ga, gr, vh, vhr);
 #pragma unroll
@@ -269,7 +261,7 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_reduce_kernel(BnBwdArgs a)
     }
     block_sum(s);
     if (a.gmax) amax = block_max(amax);
-    if (threadIdx.x == 0) {
+    if (lane == 0) {
         a.partials[row] = make_float4(s[0], s[1], s[2], s[3]);
         if (a.gmax) a.amax_part[row] = amax;
     }
@@ -278,7 +270,7 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_reduce_kernel(BnBwdArgs a)
 __global__ void __launch_bounds__(32 * kFinSlices)
 bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const float* gamma_r, float* dgamma, float* dbeta,
                        float* dgamma_r, float* dbeta_r, float* dbias, int accumulate) {
-    __shared__ double sh[kFinSlices][32][4];
+    __shared__ float4 shs[kFinSlices][32];
     const int cx = threadIdx.x & 31, sl = threadIdx.x >> 5;
     const int o = blockIdx.x * 32 + cx;
     __shared__ float shmax[kFinSlices][32];
@@ -291,12 +283,13 @@ bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const float* gamma_r, fl
             if (a.gmax) amax = fmaxf(amax, a.amax_part[(size_t)b * a.C + o]);
         }
     }
-    sh[sl][cx][0] = s0; sh[sl][cx][1] = s1; sh[sl][cx][2] = s2; sh[sl][cx][3] = s3;
+    shs[sl][cx] = make_float4((float)s0, (float)s1, (float)s2, (float)s3);
     shmax[sl][cx] = amax;
     __syncthreads();
     if (sl != 0 || o >= a.C) return;
     for (int k = 1; k < kFinSlices; ++k) {
-        s0 += sh[k][cx][0]; s1 += sh[k][cx][1]; s2 += sh[k][cx][2]; s3 += sh[k][cx][3];
+        const float4 t = shs[k][cx];
+        s0 += t.x; s1 += t.y; s2 += t.z; s3 += t.w;
         amax = fmaxf(amax, shmax[k][cx]);
     }
     const float N = (float)(*a.nvalid);
@@ -326,7 +319,8 @@ bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const float* gamma_r, fl
 
 template <typename T, typename NT, typename GT>
 __global__ void __launch_bounds__(kRowThreads) bn_bwd_apply_kernel(BnBwdArgs a) {
-    const int row = blockIdx.x, b = row / a.C, o = row % a.C;
+    SC_ROW_SETUP(a.B * a.C)
+    const int b = row / a.C, o = row % a.C;
     BwdRow<T, NT> R(a, row, b, o);
     float4 cf = a.coef[o];
     if (a.gmax) cf.x *= pow2_scale(*a.gmax);        // exact: a power of two
@@ -334,7 +328,7 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_apply_kernel(BnBwdArgs a) 
     GT* gv = (GT*)a.gv + (size_t)row * R.Tp;
     T* gvr = (a.residual == 2) ? (T*)a.gvr + (size_t)row * R.Tp : nullptr;
     T* gres = (a.residual == 1) ? (T*)a.gres + (size_t)row * R.Tp : nullptr;
-    for (int t0 = threadIdx.x * 8; t0 < R.Tp; t0 += kRowThreads * 8) {
+    for (int t0 = lane * 8; t0 < R.Tp; t0 += 256) {
         float o1[8], o2[8];
         if (t0 < R.len) {
             float ga[8], gr[8], vh[8], vhr[8];
@@ -358,12 +352,13 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_apply_kernel(BnBwdArgs a) 
 
 template <typename T>
 __global__ void __launch_bounds__(kRowThreads)
-ew_add_masked_kernel(T* out, const T* a, const T* b, const T* c, const int* len, int C, int Tt) {
-    const int row = blockIdx.x, bb = row / C;
+ew_add_masked_kernel(T* out, const T* a, const T* b, const T* c, const int* len, int nrows, int C, int Tt) {
+    SC_ROW_SETUP(nrows)
+    const int bb = row / C;
     const int l = min(len[bb], Tt);
     const bool vec = (Tt % 8 == 0);
     const size_t off = (size_t)row * Tt;
-    for (int t0 = threadIdx.x * 8; t0 < Tt; t0 += kRowThreads * 8) {
+    for (int t0 = lane * 8; t0 < Tt; t0 += 256) {
         float f[8];
         if (t0 < l) {
             load_chunk(a + off, t0, Tt, vec, f);
@@ -407,7 +402,7 @@ void lengths(const Launch& L, const int* len_in, int B, int T_in, int stride, in
 void bn_stats(const Launch& L, int vdtype, const void* v, const int* len_out, int B, int C, int Tp,
               float2* partials) {
     KScope ks_(L, KC_BN_STATS, (double)dtype_size(vdtype) * B * C * Tp, 0.0);
-    SC_DISPATCH(vdtype, (bn_stats_kernel<T><<<B * C, kRowThreads, 0, L.stream>>>((const T*)v, len_out, C, Tp, partials)));
+    SC_DISPATCH(vdtype, (bn_stats_kernel<T><<<(B * C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>((const T*)v, len_out, B * C, C, Tp, partials)));
     L.count();
 }
 
@@ -422,13 +417,13 @@ void bn_finalize(const Launch& L, const float2* partials, int parts_per_b, int t
 
 void bn_apply(const Launch& L, int dtype, const ApplyArgs& a) {
     KScope ks_(L, KC_BN_APPLY, (double)a.B * a.C * a.Tp * (dtype_size(vtype_of(dtype)) + dtype_size(dtype) + dtype_size(ntype_of(dtype)) + (a.residual == 1 ? dtype_size(dtype) : 0) + (a.residual == 2 ? dtype_size(vtype_of(dtype)) + dtype_size(ntype_of(dtype)) : 0)), 0.0);
-    SC_DISPATCH3(dtype, (bn_apply_kernel<T, VT, NT><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a)));
+    SC_DISPATCH3(dtype, (bn_apply_kernel<T, VT, NT><<<(a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>(a)));
     L.count();
 }
 
 void bn_bwd_reduce(const Launch& L, int dtype, const BnBwdArgs& a) {
     KScope ks_(L, KC_BN_BWD_REDUCE, (double)a.B * a.C * a.Tp * (dtype_size(dtype) * (a.has_relu && a.res_before_relu ? 2 : 1) + (a.has_bn ? dtype_size(ntype_of(dtype)) : 0) + (a.residual == 2 ? dtype_size(ntype_of(dtype)) : 0)), 0.0);
-    SC_DISPATCH3(dtype, (bn_bwd_reduce_kernel<T, NT><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a)));
+    SC_DISPATCH3(dtype, (bn_bwd_reduce_kernel<T, NT><<<(a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>(a)));
     L.count();
 }
 
@@ -444,17 +439,17 @@ void bn_bwd_finalize(const Launch& L, const BnBwdArgs& a, const float* gamma, co
 void bn_bwd_apply(const Launch& L, int dtype, const BnBwdArgs& a) {
     KScope ks_(L, KC_BN_BWD_APPLY, (double)a.B * a.C * a.Tp * (dtype_size(dtype) * (a.has_relu && a.res_before_relu ? 2 : 1) + (a.has_bn ? dtype_size(ntype_of(dtype)) : 0) + (a.residual == 2 ? dtype_size(ntype_of(dtype)) : 0) + dtype_size(dtype) * (1 + (a.residual != 0 ? 1 : 0))), 0.0);
     if (dtype == BF16 && a.gv_dtype == F16)
-        bn_bwd_apply_kernel<__nv_bfloat16, __half, __half><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a);
+        bn_bwd_apply_kernel<__nv_bfloat16, __half, __half><<<(a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>(a);
     else
-        SC_DISPATCH3(dtype, (bn_bwd_apply_kernel<T, NT, T><<<a.B * a.C, kRowThreads, 0, L.stream>>>(a)));
+        SC_DISPATCH3(dtype, (bn_bwd_apply_kernel<T, NT, T><<<(a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>(a)));
     L.count();
 }
 
 void ew_add_masked(const Launch& L, int dtype, void* out, const void* a, const void* b, const void* c,
                    const int* len, int B, int C, int Tt) {
     KScope ks_(L, KC_EW, (double)dtype_size(dtype) * B * C * Tt * (2 + (b ? 1 : 0) + (c ? 1 : 0)), 0.0);
-    SC_DISPATCH(dtype, (ew_add_masked_kernel<T><<<B * C, kRowThreads, 0, L.stream>>>((T*)out, (const T*)a, (const T*)b,
-                                                                                      (const T*)c, len, C, Tt)));
+    SC_DISPATCH(dtype, (ew_add_masked_kernel<T><<<(B * C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>((T*)out, (const T*)a, (const T*)b,
+                                                                                      (const T*)c, len, B * C, C, Tt)));
     L.count();
 }
 

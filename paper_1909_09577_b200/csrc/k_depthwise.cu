@@ -8,6 +8,7 @@
 #include "common.cuh"
 #include "kernels.h"
 #include <type_traits>
+#include <algorithm>
 
 namespace sc {
 namespace {
@@ -319,6 +320,109 @@ dw_wgrad_s1_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float* __
     }
 }
 
+// ---- stride-1 tap gradient, register accumulators ------------------------------------------------
+// dwd[c,k] = sum_{b,t} gu[b,c,t] * x[b,c,t+k-P].  A thread owns 8 consecutive frames of gu (registers)
+// and ALL taps: 8*NCH accumulators in registers, a 16-wide sliding window of x from shared memory, so
+// the inner loop is 64 FMAs per two 16-byte shared loads.  Threads sweep the (row, 8-frame chunk)
+// pairs of NR staged rows; the per-thread accumulators are summed over the warp with shuffles and over
+// the CTA's warps in a fixed order (the "warp-level time reduction"), one partial per CTA.
+constexpr int WR_THREADS = 128;
+
+template <typename TG, typename T, int NCH>
+__global__ void __launch_bounds__(WR_THREADS, 3)
+dw_wgrad_reg_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float* __restrict__ partials,
+                    const int* __restrict__ len_in, const int* __restrict__ len_out,
+                    int B, int C, int Tt, int K, int Ppad, int NR, int NST, int RSP) {
+    extern __shared__ float smem[];
+    const int tid = threadIdx.x, lane = tid & 31, wrp = tid >> 5;
+    const int c = blockIdx.x;
+    const int P = (K - 1) / 2, shift = Ppad - P;
+    const int cpr = Tt / 8;                        // 8-frame chunks per row (Tt % 8 == 0)
+    const int XW = Tt + 8 * NCH + 8;               // x row: Ppad zeros, Tt frames, zeros up to XW
+    float* gs = smem;                              // [NR][RSP]
+    float* xs = smem + (size_t)NR * RSP;           // [NR][RSP]
+    float acc[8 * NCH];
+#pragma unroll
+    for (int i = 0; i < 8 * NCH; ++i) acc[i] = 0.f;
+
+    for (int st = 0; st < NST; ++st) {
+        const int b0 = (blockIdx.y * NST + st) * NR;
+        if (b0 >= B) break;
+        const int nr = min(NR, B - b0);
+        __syncthreads();
+        // zero the halos of x (frames before 0 and after Tt) -- everything else is overwritten
+        for (int i = tid; i < nr * (XW - Tt); i += WR_THREADS) {
+            const int r = i / (XW - Tt), j = i - r * (XW - Tt);
+            const int col = j < Ppad ? j : Tt + j;
+            xs[r * RSP + phys(col)] = 0.f;
+        }
+        for (int i = tid; i < nr * cpr; i += WR_THREADS) {
+            const int r = i / cpr, t = (i - r * cpr) * 8;
+            const int b = b0 + r;
+            const int li = min(len_in[b], Tt), lo = min(len_out[b], Tt);
+            const size_t off = ((size_t)b * C + c) * Tt + t;
+            float fg[8], fx[8];
+            if (t < lo) ld8<TG>(gu + off, fg);
+            if (t < li) ld8<T>(x + off, fx);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { if (t + e >= lo) fg[e] = 0.f; if (t + e >= li) fx[e] = 0.f; }
+            float* gd = gs + r * RSP + phys(t);
+            // Ppad is a multiple of 4 only, so the two halves may straddle a 32-float padding boundary
+            float* xd0 = xs + r * RSP + phys(t + Ppad);
+            float* xd1 = xs + r * RSP + phys(t + Ppad + 4);
+            *reinterpret_cast<float4*>(gd) = make_float4(fg[0], fg[1], fg[2], fg[3]);
+            *reinterpret_cast<float4*>(gd + 4) = make_float4(fg[4], fg[5], fg[6], fg[7]);
+            *reinterpret_cast<float4*>(xd0) = make_float4(fx[0], fx[1], fx[2], fx[3]);
+            *reinterpret_cast<float4*>(xd1) = make_float4(fx[4], fx[5], fx[6], fx[7]);
+        }
+        __syncthreads();
+        for (int i = tid; i < nr * cpr; i += WR_THREADS) {
+            const int r = i / cpr, t = (i - r * cpr) * 8;
+            const float* gp = gs + r * RSP;
+            const float* xp = xs + r * RSP;
+            float g[8], win[16];
+            {
+                const float4 a = *reinterpret_cast<const float4*>(gp + phys(t));
+                const float4 bq = *reinterpret_cast<const float4*>(gp + phys(t + 4));
+                g[0] = a.x; g[1] = a.y; g[2] = a.z; g[3] = a.w; g[4] = bq.x; g[5] = bq.y; g[6] = bq.z; g[7] = bq.w;
+                const float4 c0 = *reinterpret_cast<const float4*>(xp + phys(t));
+                const float4 c1 = *reinterpret_cast<const float4*>(xp + phys(t + 4));
+                win[0] = c0.x; win[1] = c0.y; win[2] = c0.z; win[3] = c0.w;
+                win[4] = c1.x; win[5] = c1.y; win[6] = c1.z; win[7] = c1.w;
+            }
+#pragma unroll
+            for (int ch = 0; ch < NCH; ++ch) {
+                const float4 c0 = *reinterpret_cast<const float4*>(xp + phys(t + 8 * ch + 8));
+                const float4 c1 = *reinterpret_cast<const float4*>(xp + phys(t + 8 * ch + 12));
+                win[8] = c0.x; win[9] = c0.y; win[10] = c0.z; win[11] = c0.w;
+                win[12] = c1.x; win[13] = c1.y; win[14] = c1.z; win[15] = c1.w;
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+#pragma unroll
+                    for (int rr = 0; rr < 8; ++rr) acc[8 * ch + q] = fmaf(g[rr], win[rr + q], acc[8 * ch + q]);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) win[q] = win[q + 8];
+            }
+        }
+    }
+    // warp tree, then the four warps in order
+    __syncthreads();
+    float* red = smem;                             // [4][8*NCH]
+#pragma unroll
+    for (int i = 0; i < 8 * NCH; ++i) {
+        float v = warp_sum(acc[i]);
+        if (lane == 0) red[wrp * 8 * NCH + i] = v;
+    }
+    __syncthreads();
+    for (int k = tid; k < K; k += WR_THREADS) {
+        const int kk = k + shift;
+        float sum = 0.f;
+#pragma unroll
+        for (int w = 0; w < WR_THREADS / 32; ++w) sum += red[w * 8 * NCH + kk];
+        partials[((size_t)blockIdx.y * C + c) * K + k] = sum;
+    }
+}
+
 inline int kpad(int K) { return (K + R - 1) / R * R; }
 inline int host_phys(int i) { return i + ((i >> 5) << 2); }
 
@@ -389,7 +493,38 @@ void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x
     int nsplit;
     {
     KScope ks_(L, KC_DW_WGRAD, (double)B * C * (dtype_size(dtype) * Tt + dtype_size(odt) * Tp), 2.0 * B * C * Tp * K);
-    if (s == 1) {
+    const int P = (K - 1) / 2, Ppad = (P + 3) / 4 * 4;
+    const int nch = (K + (Ppad - P) + 7) / 8;
+    if (s == 1 && Tt % 8 == 0 && nch >= 2 && nch <= 12) {
+        // rows staged per pass: the count whose (rows x chunks) best fills the 128 threads, within 64 KiB
+        const int cpr = Tt / 8;
+        const int rs = host_phys(Tt + 8 * nch + 8) + 4, rsp = (rs + 3) / 4 * 4;
+        int NR = 1; double best = 0.0;
+        for (int nr = 1; nr <= 8 && nr <= B; ++nr) {
+            if ((size_t)2 * nr * rsp * sizeof(float) > 64 * 1024) break;
+            const int work = nr * cpr, iters = (work + WR_THREADS - 1) / WR_THREADS;
+            const double eff = (double)work / (iters * WR_THREADS);
+            if (eff > best + 1e-9) { best = eff; NR = nr; }
+        }
+        const int NST = 2;
+        nsplit = (B + NR * NST - 1) / (NR * NST);
+        const size_t smem = std::max((size_t)2 * NR * rsp, (size_t)4 * 8 * nch) * sizeof(float);
+        dim3 grid(C, nsplit);
+#define SC_WR_CASE(N)                                                                                          \
+        case N: {                                                                                              \
+            SC_DISPATCH_IO(dtype, odt, {                                                                       \
+                auto kern = dw_wgrad_reg_kernel<OT, T, N>;                                                     \
+                static bool cfg_done = false;                                                                  \
+                if (!cfg_done) { cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024); cfg_done = true; } \
+                kern<<<grid, WR_THREADS, smem, L.stream>>>((const OT*)gu, (const T*)x, partials, len_in, len_out, \
+                                                           B, C, Tt, K, Ppad, NR, NST, rsp); });               \
+        } break;
+        switch (nch) {
+            SC_WR_CASE(2) SC_WR_CASE(3) SC_WR_CASE(4) SC_WR_CASE(5) SC_WR_CASE(6) SC_WR_CASE(7) SC_WR_CASE(8)
+            SC_WR_CASE(9) SC_WR_CASE(10) SC_WR_CASE(11) SC_WR_CASE(12)
+        }
+#undef SC_WR_CASE
+    } else if (s == 1) {
         const int Kp = kpad(K), NG = Kp / R, nseg = WG_THREADS / NG;
         const int seglen = ((WG_TT + nseg - 1) / nseg + R - 1) / R * R;
         const int GW = nseg * seglen;

@@ -24,7 +24,8 @@ namespace {
 
 constexpr int NB = 64;              // frames per block
 constexpr int MAXROWS = 256;        // block rows (incl. separators) per CTA: two MMA M-tiles
-constexpr int ROWS_ALLOC = 264;     // + one slack row in front, a few behind
+constexpr int ROWS_ALLOC = 265;     // + one slack row in front, a few behind; 8m+1 so that the eight
+                                    // chunk columns start in different 16-byte bank groups
 constexpr int kThreads = 128;
 
 __device__ __forceinline__ uint64_t desc_noswz(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
@@ -50,9 +51,12 @@ dw_tc_kernel(const TI* __restrict__ in, const TW* __restrict__ w, TO* __restrict
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
     uint4* A16 = reinterpret_cast<uint4*>(smem);                        // [8 chunks][ROWS_ALLOC] 16-byte units
     uint4* B16 = A16 + 8 * ROWS_ALLOC;                                  // [3 shifts][8 chunks][64 rows]
-    float* taps = reinterpret_cast<float*>(B16 + 3 * 8 * 64);           // [K], K <= 129
-    uint64_t* bar = reinterpret_cast<uint64_t*>(taps + 132);
+    // coef[128 + delta] = coefficient that input position (output position + delta) contributes, as
+    // 16-bit operand bits; zero outside the taps.  |delta| <= 127, plus slack for the 5-word reads.
+    uint32_t* coefw = reinterpret_cast<uint32_t*>(B16 + 3 * 8 * 64);    // 132 words = 264 halfwords
+    uint64_t* bar = reinterpret_cast<uint64_t*>(coefw + 132);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar + 1);
+    int* lens = reinterpret_cast<int*>(tmem_slot + 2);                  // [nb <= 128] source lengths
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int c = blockIdx.x, b0 = blockIdx.y * nb;
@@ -66,37 +70,61 @@ dw_tc_kernel(const TI* __restrict__ in, const TW* __restrict__ w, TO* __restrict
     if (tid == 0) { ptx::mbar_init(bar, 1); ptx::fence_barrier_init(); }
     if (warp == 0) { ptx::tmem_alloc(tmem_slot, 128); ptx::tmem_relinquish(); }
     for (int i = tid; i < 8 * ROWS_ALLOC; i += kThreads) A16[i] = make_uint4(0, 0, 0, 0);
-    for (int k = tid; k < K; k += kThreads) taps[k] = ldf(w + (size_t)c * K + k);
+    for (int i = tid; i < nbh; i += kThreads) lens[i] = len_src[b0 + i];
+    for (int i = tid; i < 264; i += kThreads) {
+        const int delta = i - 128;
+        const int kk = FLIP ? P - delta : delta + P;
+        reinterpret_cast<unsigned short*>(coefw)[i] =
+            (delta >= -127 && delta <= 127 && kk >= 0 && kk < K) ? bits16<TI>(ldf(w + (size_t)c * K + kk)) : (unsigned short)0;
+    }
     ptx::tc_fence_before();
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
     // ---- stage the input rows: frame t = 64 i + 8 q + e  ->  A16[q][1 + seg*S + 1 + i] ----
-    for (int idx = tid; idx < nbh * vpr; idx += kThreads) {
-        const int seg = idx / vpr, vq = idx - seg * vpr, t = vq * 8;
-        const int ls = min(len_src[b0 + seg], Tt);
-        if (t >= ls) continue;
-        uint4 v = *reinterpret_cast<const uint4*>(in + ((size_t)(b0 + seg) * C + c) * Tt + t);
-        if (t + 8 > ls) {                            // the length falls inside this vector
-            unsigned short* h = reinterpret_cast<unsigned short*>(&v);
+    // All of a thread's loads are issued before the first store so that they overlap (a CTA stages at
+    // most nb * nblk * 8 <= 2048 vectors, i.e. 16 per thread).
+    {
+        const int nvec = nbh * vpr;
+        uint4 v[16];
+        int dst[16];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) if (t + e >= ls) h[e] = 0;
+        for (int it = 0; it < 16; ++it) {
+            const int idx = tid + it * kThreads;
+            dst[it] = -1;
+            if (idx < nvec) {
+                const int seg = idx / vpr, vq = idx - seg * vpr, t = vq * 8;
+                const int ls = min(lens[seg], Tt);
+                if (t < ls) {
+                    v[it] = *reinterpret_cast<const uint4*>(in + ((size_t)(b0 + seg) * C + c) * Tt + t);
+                    dst[it] = (vq & 7) * ROWS_ALLOC + 1 + seg * S + 1 + (vq >> 3);
+                    if (t + 8 > ls) dst[it] |= (ls - t) << 20;      // the length falls inside this vector
+                }
+            }
         }
-        A16[(vq & 7) * ROWS_ALLOC + 1 + seg * S + 1 + (vq >> 3)] = v;
+#pragma unroll
+        for (int it = 0; it < 16; ++it) {
+            if (dst[it] < 0) continue;
+            const int keep = dst[it] >> 20;
+            if (keep) {
+                unsigned short* h = reinterpret_cast<unsigned short*>(&v[it]);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) if (e >= keep) h[e] = 0;
+            }
+            A16[dst[it] & 0xFFFFF] = v[it];
+        }
     }
     // ---- Toeplitz blocks: B16[d][q][n] holds T_d[j' = 8q..8q+7, j = n] ----
     for (int idx = tid; idx < 3 * 8 * 64; idx += kThreads) {
         const int d = idx / 512, q = (idx >> 6) & 7, n = idx & 63;
-        uint4 v;
-        unsigned short* h = reinterpret_cast<unsigned short*>(&v);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int delta = 8 * q + e + NB * (d - 1) - n;      // input position minus output position
-            const int kk = FLIP ? P - delta : delta + P;
-            h[e] = (kk >= 0 && kk < K) ? bits16<TI>(taps[kk]) : (unsigned short)0;
-        }
-        B16[idx] = v;
+        // eight consecutive deltas starting at 8q + 64(d-1) - n: an unaligned 16-byte window of coef
+        const int s0 = 8 * q + NB * (d - 1) - n + 128;           // in [1, 247]
+        const uint32_t* cw = coefw + (s0 >> 1);
+        const uint32_t sh = (s0 & 1) * 16;
+        const uint32_t w0 = cw[0], w1 = cw[1], w2 = cw[2], w3 = cw[3], w4 = cw[4];
+        B16[idx] = make_uint4(__funnelshift_r(w0, w1, sh), __funnelshift_r(w1, w2, sh), __funnelshift_r(w2, w3, sh),
+                              __funnelshift_r(w3, w4, sh));
     }
     ptx::fence_proxy_async();                        // generic-proxy writes -> visible to the tensor core
     __syncthreads();
@@ -172,7 +200,7 @@ dw_tc_kernel(const TI* __restrict__ in, const TW* __restrict__ w, TO* __restrict
     if (warp == 0) ptx::tmem_dealloc(tmem, 128);
 }
 
-constexpr size_t kSmemBytes = (size_t)(8 * ROWS_ALLOC + 3 * 8 * 64) * 16 + 132 * 4 + 64 + 128;
+constexpr size_t kSmemBytes = (size_t)(8 * ROWS_ALLOC + 3 * 8 * 64) * 16 + 132 * 4 + 64 + 128 * 4 + 128;   // A, B, coef, barrier, alignment
 
 template <typename TI, typename TW, typename TO, bool FLIP>
 void launch_tc(const Launch& L, const void* in, const void* w, void* out, const void* add1, const void* add2,

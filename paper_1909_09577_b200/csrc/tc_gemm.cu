@@ -313,12 +313,12 @@ constexpr int FWD_BN = 128;
 struct WgradPlan { int mt, bn, tiles, nsplit, kb_per_split, nkb_total, nkb_t; };
 WgradPlan plan_wgrad(int B, int Cin, int Cout, int Tp) {
     WgradPlan w;
-    w.mt = Cout > 128 ? 2 : 1;
-    w.bn = Cin >= 256 ? 256 : (Cin > 64 ? 128 : 64);
+    w.mt = Cout >= 512 ? 2 : 1;
+    w.bn = Cin >= 512 ? 256 : (Cin > 64 ? 128 : 64);
     w.tiles = ((Cout + 128 * w.mt - 1) / (128 * w.mt)) * ((Cin + w.bn - 1) / w.bn);
     w.nkb_t = (Tp + BK - 1) / BK;
     w.nkb_total = B * w.nkb_t;
-    int ns = std::max(1, std::min(64, 296 / w.tiles));
+    int ns = std::max(1, 148 / w.tiles);        // one CTA per SM, one wave
     ns = std::min(ns, w.nkb_total);
     w.kb_per_split = (w.nkb_total + ns - 1) / ns;
     w.nsplit = (w.nkb_total + w.kb_per_split - 1) / w.kb_per_split;
@@ -346,7 +346,7 @@ bool tc_dgrad_supported(const TcState* st, int dtype, int Cin, int Cout, int Tp)
 bool tc_wgrad_supported(const TcState* st, int dtype, int Cin, int Cout, int Tp) { return shape_ok(st, dtype, Cin, Cout, Tp); }
 
 size_t tc_wgrad_scratch_bytes(const TcState*, int Cin, int Cout) {
-    // upper bound over every batch size: at most min(64, 296 / tiles) splits
+    // upper bound over every batch size: at most 148 / tiles splits
     WgradPlan w = plan_wgrad(1 << 20, Cin, Cout, 64);
     return (size_t)w.nsplit * Cin * Cout * sizeof(float);
 }
