@@ -196,10 +196,10 @@ void plan_bwd(const sc_block_desc* d, const Dims& m, Bump& ws, BwdScratch* s, co
     const size_t act_out = e * m.B * m.Cout * m.Tp, act_in = e * m.B * m.Cin * m.Tp;
     s->len_out = (int*)ws.take(sizeof(int) * m.B);
     s->nvalid = (int*)ws.take(sizeof(int));
-    s->partials = (float4*)ws.take(sizeof(float4) * m.B * m.Cout);
+    s->partials = (float4*)ws.take(sizeof(float4) * m.B * m.Cout * bn_bwd_max_slots(m.Tp));
     s->coef = (float4*)ws.take(sizeof(float4) * m.Cout);
     s->coef_r = (float4*)ws.take(sizeof(float4) * m.Cout);
-    s->amax_part = (float*)ws.take(sizeof(float) * m.B * m.Cout);
+    s->amax_part = (float*)ws.take(sizeof(float) * m.B * m.Cout * bn_bwd_max_slots(m.Tp));
     s->gmax = (float*)ws.take(sizeof(float));
     s->w16 = (op_dtype(d) != d->io_dtype) ? ws.take((size_t)2 * m.Cout * m.Cin) : nullptr;
     s->gv = ws.take(act_out);

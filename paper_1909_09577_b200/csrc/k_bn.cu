@@ -151,12 +151,12 @@ __global__ void __launch_bounds__(kRowThreads) bn_apply_kernel(ApplyArgs a) {
     const int Tp = a.Tp, len = min(a.len_out[b], Tp);
     const bool vec = (Tp % 8 == 0);
     const size_t off = (size_t)row * Tp;
-    const VT* v = (const VT*)a.v + off;
-    const T* xr = a.residual == 1 ? (const T*)a.xres + off : nullptr;
-    const VT* vr = a.residual == 2 ? (const VT*)a.vr + off : nullptr;
-    T* y = (T*)a.y + off;
-    NT* vh = (NT*)a.vhat + off;
-    NT* vhr = a.residual == 2 ? (NT*)a.vhat_r + off : nullptr;
+    const VT* __restrict__ v = (const VT*)a.v + off;
+    const T* __restrict__ xr = a.residual == 1 ? (const T*)a.xres + off : nullptr;
+    const VT* __restrict__ vr = a.residual == 2 ? (const VT*)a.vr + off : nullptr;
+    T* __restrict__ y = (T*)a.y + off;
+    NT* __restrict__ vh = (NT*)a.vhat + off;
+    NT* __restrict__ vhr = a.residual == 2 ? (NT*)a.vhat_r + off : nullptr;
     const float mu = a.mean[o], is = a.invstd[o], ga = a.gamma[o], be = a.beta[o];
     float mur = 0.f, isr = 0.f, gar = 0.f, ber = 0.f;
     if (a.residual == 2) { mur = a.mean_r[o]; isr = a.invstd_r[o]; gar = a.gamma_r[o]; ber = a.beta_r[o]; }
@@ -200,7 +200,7 @@ __global__ void __launch_bounds__(kRowThreads) bn_apply_kernel(ApplyArgs a) {
 // Shared by the reduce and apply steps of the backward pass: per element gate and normalised value.
 template <typename T, typename NT>
 struct BwdRow {
-    const T *g, *y; const NT *vh, *vhr;
+    const T* __restrict__ g; const T* __restrict__ y; const NT* __restrict__ vh; const NT* __restrict__ vhr;
     float gam, bet;
     int len, Tp;
     bool vec;
@@ -262,8 +262,8 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_reduce_kernel(BnBwdArgs a)
     block_sum(s);
     if (a.gmax) amax = block_max(amax);
     if (lane == 0) {
-        a.partials[row] = make_float4(s[0], s[1], s[2], s[3]);
-        if (a.gmax) a.amax_part[row] = amax;
+        a.partials[(size_t)row * a.nslots] = make_float4(s[0], s[1], s[2], s[3]);
+        if (a.gmax) a.amax_part[(size_t)row * a.nslots] = amax;
     }
 }
 
@@ -277,10 +277,17 @@ bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const float* gamma_r, fl
     double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
     float amax = 0.f;
     if (o < a.C) {
-        for (int b = sl; b < a.B; b += kFinSlices) {
-            const float4 p = a.partials[(size_t)b * a.C + o];
+        const int vpr = a.Tp / 8;
+        for (int pi = sl; pi < a.B * a.nslots; pi += kFinSlices) {
+            const int b = pi / a.nslots, slot = pi - b * a.nslots;
+            const long long r = (long long)b * a.C + o;
+            if (a.nslots > 1) {      // slots in use for this row (see bn_bwd_reduce_fast_kernel)
+                const int used = (int)((((r + 1) * vpr - 1) >> 5) - ((r * vpr) >> 5)) + 1;
+                if (slot >= used) continue;
+            }
+            const float4 p = a.partials[(size_t)r * a.nslots + slot];
             s0 += p.x; s1 += p.y; s2 += p.z; s3 += p.w;
-            if (a.gmax) amax = fmaxf(amax, a.amax_part[(size_t)b * a.C + o]);
+            if (a.gmax) amax = fmaxf(amax, a.amax_part[(size_t)r * a.nslots + slot]);
         }
     }
     shs[sl][cx] = make_float4((float)s0, (float)s1, (float)s2, (float)s3);
@@ -325,9 +332,9 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_apply_kernel(BnBwdArgs a) 
     float4 cf = a.coef[o];
     if (a.gmax) cf.x *= pow2_scale(*a.gmax);        // exact: a power of two
     const float4 cr = (a.residual == 2) ? a.coef_r[o] : make_float4(0.f, 0.f, 0.f, 0.f);
-    GT* gv = (GT*)a.gv + (size_t)row * R.Tp;
-    T* gvr = (a.residual == 2) ? (T*)a.gvr + (size_t)row * R.Tp : nullptr;
-    T* gres = (a.residual == 1) ? (T*)a.gres + (size_t)row * R.Tp : nullptr;
+    GT* __restrict__ gv = (GT*)a.gv + (size_t)row * R.Tp;
+    T* __restrict__ gvr = (a.residual == 2) ? (T*)a.gvr + (size_t)row * R.Tp : nullptr;
+    T* __restrict__ gres = (a.residual == 1) ? (T*)a.gres + (size_t)row * R.Tp : nullptr;
     for (int t0 = lane * 8; t0 < R.Tp; t0 += 256) {
         float o1[8], o2[8];
         if (t0 < R.len) {
@@ -347,6 +354,130 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_apply_kernel(BnBwdArgs a) 
         store_chunk(gv, t0, R.Tp, R.vec, o1);
         if (gvr) store_chunk(gvr, t0, R.Tp, R.vec, o2);
         if (gres) store_chunk(gres, t0, R.Tp, R.vec, o2);
+    }
+}
+
+// ---- flattened fast paths (the encoder's configuration: BN + ReLU, residual joined before the ReLU,
+// rows a multiple of 8 frames).  One 8-frame vector per thread: no row tails, few registers, so many
+// warps and many 16-byte loads in flight per SM.
+template <typename T, typename VT, typename NT, int RES>
+__global__ void __launch_bounds__(256) bn_apply_fast_kernel(ApplyArgs a, int vpr, long long total) {
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (idx >= total) return;
+    const int row = (int)(idx / vpr), t0 = (int)(idx - (long long)row * vpr) * 8;
+    const int b = row / a.C, o = row - b * a.C;
+    const int len = min(a.len_out[b], a.Tp);
+    const size_t off = (size_t)row * a.Tp + t0;
+    float out[8], n1[8], n2[8];
+    if (t0 < len) {
+        float f[8], r[8];
+        ld8<VT>((const VT*)a.v + off, f);
+        if (RES == 1) ld8<T>((const T*)a.xres + off, r);
+        if (RES == 2) ld8<VT>((const VT*)a.vr + off, r);
+        const float mu = a.mean[o], is = a.invstd[o], ga = a.gamma[o], be = a.beta[o];
+        float mur = 0.f, isr = 0.f, gar = 0.f, ber = 0.f;
+        if (RES == 2) { mur = a.mean_r[o]; isr = a.invstd_r[o]; gar = a.gamma_r[o]; ber = a.beta_r[o]; }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const bool in = t0 + i < len;
+            n1[i] = in ? round_io<NT>((f[i] - mu) * is) : 0.f;
+            float rr = 0.f;
+            if (RES == 1) rr = r[i];
+            if (RES == 2) { n2[i] = in ? round_io<NT>((r[i] - mur) * isr) : 0.f; rr = fmaf(gar, n2[i], ber); }
+            out[i] = in ? fmaxf(fmaf(ga, n1[i], be) + rr, 0.f) : 0.f;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { out[i] = 0.f; n1[i] = 0.f; n2[i] = 0.f; }
+    }
+    st8<T>((T*)a.y + off, out);
+    st8<NT>((NT*)a.vhat + off, n1);
+    if (RES == 2) st8<NT>((NT*)a.vhat_r + off, n2);
+}
+
+template <typename T, typename NT, typename GT, int RES>
+__global__ void __launch_bounds__(256) bn_bwd_apply_fast_kernel(BnBwdArgs a, int vpr, long long total) {
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (idx >= total) return;
+    const int row = (int)(idx / vpr), t0 = (int)(idx - (long long)row * vpr) * 8;
+    const int b = row / a.C, o = row - b * a.C;
+    const int len = min(a.len_out[b], a.Tp);
+    const size_t off = (size_t)row * a.Tp + t0;
+    float o1[8], o2[8];
+    if (t0 < len) {
+        float g[8], y[8], vn[8], vnr[8];
+        ld8<T>((const T*)a.g + off, g);
+        ld8<T>((const T*)a.y + off, y);
+        ld8<NT>((const NT*)a.vhat + off, vn);
+        if (RES == 2) ld8<NT>((const NT*)a.vhat_r + off, vnr);
+        float4 cf = a.coef[o];
+        if (a.gmax) cf.x *= pow2_scale(*a.gmax);
+        float4 cr = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (RES == 2) cr = a.coef_r[o];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const bool in = t0 + i < len;
+            const float ga = (in && y[i] > 0.f) ? g[i] : 0.f;
+            o1[i] = in ? cf.x * (ga - cf.y - vn[i] * cf.z) : 0.f;
+            if (RES == 2) o2[i] = in ? cr.x * (ga - cr.y - vnr[i] * cr.z) : 0.f;
+            if (RES == 1) o2[i] = ga;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { o1[i] = 0.f; o2[i] = 0.f; }
+    }
+    st8<GT>((GT*)a.gv + off, o1);
+    if (RES == 2) st8<T>((T*)a.gvr + off, o2);
+    if (RES == 1) st8<T>((T*)a.gres + off, o2);
+}
+
+// Flattened reduce: one 8-frame vector per thread; a warp's 32 consecutive vectors belong to at most two
+// rows (vpr >= 32), so two masked warp reductions give one partial per (row, warp) pair.  Row r's
+// partials sit in slots [0, last_warp(r) - first_warp(r)] with first_warp(r) = (r * vpr) >> 5: a static
+// assignment, summed later in slot order.
+template <typename T, typename NT, int RES>
+__global__ void __launch_bounds__(256) bn_bwd_reduce_fast_kernel(BnBwdArgs a, int vpr, long long total) {
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    const int lane = threadIdx.x & 31;
+    const long long warp_first = idx - lane;
+    if (warp_first >= total) return;
+    const bool valid = idx < total;
+    const long long cidx = valid ? idx : total - 1;
+    const int row = (int)(cidx / vpr), t0 = (int)(cidx - (long long)row * vpr) * 8;
+    const int b = row / a.C;
+    const int len = min(a.len_out[b], a.Tp);
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f, amax = 0.f;
+    if (valid && t0 < len) {
+        const size_t off = (size_t)row * a.Tp + t0;
+        float g[8], y[8], vn[8], vnr[8];
+        ld8<T>((const T*)a.g + off, g);
+        ld8<T>((const T*)a.y + off, y);
+        ld8<NT>((const NT*)a.vhat + off, vn);
+        if (RES == 2) ld8<NT>((const NT*)a.vhat_r + off, vnr);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float ga = (t0 + i < len && y[i] > 0.f) ? g[i] : 0.f;
+            s0 += ga; s1 += ga * vn[i];
+            if (RES == 2) { s2 += ga; s3 += ga * vnr[i]; }
+            amax = fmaxf(amax, fabsf(ga));
+        }
+    }
+    const int row0 = (int)(warp_first / vpr);
+    const long long wg = warp_first >> 5;                    // global warp index
+#pragma unroll
+    for (int seg = 0; seg < 2; ++seg) {
+        const int r = row0 + seg;
+        if (seg == 1 && (long long)r * vpr >= warp_first + 32) break;     // warp lies inside one row (uniform)
+        const bool mine = valid && row == r;
+        float v[4] = {mine ? s0 : 0.f, mine ? s1 : 0.f, mine ? s2 : 0.f, mine ? s3 : 0.f};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v[i] = warp_sum(v[i]);
+        const float m = a.gmax ? warp_max(mine ? amax : 0.f) : 0.f;
+        if (lane == 0 && (long long)r * vpr < total) {
+            const int slot = (int)(wg - (((long long)r * vpr) >> 5));
+            a.partials[(size_t)r * a.nslots + slot] = make_float4(v[0], v[1], v[2], v[3]);
+            if (a.gmax) a.amax_part[(size_t)r * a.nslots + slot] = m;
+        }
     }
 }
 
@@ -417,11 +548,33 @@ void bn_finalize(const Launch& L, const float2* partials, int parts_per_b, int t
 
 void bn_apply(const Launch& L, int dtype, const ApplyArgs& a) {
     KScope ks_(L, KC_BN_APPLY, (double)a.B * a.C * a.Tp * (dtype_size(vtype_of(dtype)) + dtype_size(dtype) + dtype_size(ntype_of(dtype)) + (a.residual == 1 ? dtype_size(dtype) : 0) + (a.residual == 2 ? dtype_size(vtype_of(dtype)) + dtype_size(ntype_of(dtype)) : 0)), 0.0);
+    if (a.Tp % 8 == 0 && a.has_relu && a.res_before_relu) {
+        const int vpr = a.Tp / 8;
+        const long long total = (long long)a.B * a.C * vpr;
+        const unsigned grid = (unsigned)((total + 255) / 256);
+#define SC_APPLY_FAST(RES) SC_DISPATCH3(dtype, (bn_apply_fast_kernel<T, VT, NT, RES><<<grid, 256, 0, L.stream>>>(a, vpr, total)))
+        if (a.residual == 0) { SC_APPLY_FAST(0); } else if (a.residual == 1) { SC_APPLY_FAST(1); } else { SC_APPLY_FAST(2); }
+#undef SC_APPLY_FAST
+        L.count();
+        return;
+    }
     SC_DISPATCH3(dtype, (bn_apply_kernel<T, VT, NT><<<(a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>(a)));
     L.count();
 }
 
-void bn_bwd_reduce(const Launch& L, int dtype, const BnBwdArgs& a) {
+void bn_bwd_reduce(const Launch& L, int dtype, BnBwdArgs& a) {
+    a.nslots = 1;
+    if (a.Tp % 8 == 0 && a.Tp >= 256 && a.has_bn && a.has_relu && a.res_before_relu) {
+        KScope ks2_(L, KC_BN_BWD_REDUCE, (double)a.B * a.C * a.Tp * (dtype_size(dtype) * 2 + dtype_size(ntype_of(dtype)) * (a.residual == 2 ? 2 : 1)), 0.0);
+        const int vpr = a.Tp / 8;
+        a.nslots = bn_bwd_max_slots(a.Tp);
+        const long long total = (long long)a.B * a.C * vpr;
+        const unsigned grid = (unsigned)((total + 255) / 256);
+        if (a.residual == 2) { SC_DISPATCH3(dtype, (bn_bwd_reduce_fast_kernel<T, NT, 2><<<grid, 256, 0, L.stream>>>(a, vpr, total))); }
+        else { SC_DISPATCH3(dtype, (bn_bwd_reduce_fast_kernel<T, NT, 0><<<grid, 256, 0, L.stream>>>(a, vpr, total))); }
+        L.count();
+        return;
+    }
     KScope ks_(L, KC_BN_BWD_REDUCE, (double)a.B * a.C * a.Tp * (dtype_size(dtype) * (a.has_relu && a.res_before_relu ? 2 : 1) + (a.has_bn ? dtype_size(ntype_of(dtype)) : 0) + (a.residual == 2 ? dtype_size(ntype_of(dtype)) : 0)), 0.0);
     SC_DISPATCH3(dtype, (bn_bwd_reduce_kernel<T, NT><<<(a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>(a)));
     L.count();
@@ -438,6 +591,20 @@ void bn_bwd_finalize(const Launch& L, const BnBwdArgs& a, const float* gamma, co
 
 void bn_bwd_apply(const Launch& L, int dtype, const BnBwdArgs& a) {
     KScope ks_(L, KC_BN_BWD_APPLY, (double)a.B * a.C * a.Tp * (dtype_size(dtype) * (a.has_relu && a.res_before_relu ? 2 : 1) + (a.has_bn ? dtype_size(ntype_of(dtype)) : 0) + (a.residual == 2 ? dtype_size(ntype_of(dtype)) : 0) + dtype_size(dtype) * (1 + (a.residual != 0 ? 1 : 0))), 0.0);
+    if (a.Tp % 8 == 0 && a.has_bn && a.has_relu && a.res_before_relu) {
+        const int vpr = a.Tp / 8;
+        const long long total = (long long)a.B * a.C * vpr;
+        const unsigned grid = (unsigned)((total + 255) / 256);
+#define SC_BWD_FAST(RES)                                                                                          \
+        if (dtype == BF16 && a.gv_dtype == F16)                                                                   \
+            bn_bwd_apply_fast_kernel<__nv_bfloat16, __half, __half, RES><<<grid, 256, 0, L.stream>>>(a, vpr, total); \
+        else                                                                                                      \
+            SC_DISPATCH3(dtype, (bn_bwd_apply_fast_kernel<T, NT, T, RES><<<grid, 256, 0, L.stream>>>(a, vpr, total)))
+        if (a.residual == 0) { SC_BWD_FAST(0); } else if (a.residual == 1) { SC_BWD_FAST(1); } else { SC_BWD_FAST(2); }
+#undef SC_BWD_FAST
+        L.count();
+        return;
+    }
     if (dtype == BF16 && a.gv_dtype == F16)
         bn_bwd_apply_kernel<__nv_bfloat16, __half, __half><<<(a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>(a);
     else

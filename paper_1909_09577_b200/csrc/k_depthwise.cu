@@ -240,6 +240,49 @@ dw_wgrad_generic_kernel(const TG* __restrict__ gu, const T* __restrict__ x, floa
     }
 }
 
+// Any stride, K <= 128: CTA = (channel, sample); thread (k, group) accumulates tap k over the frames
+// t = group (mod ngroups) of a shared-memory tile; groups are then summed in order.
+constexpr int WS_TT = 512;
+template <typename TG, typename T>
+__global__ void __launch_bounds__(128)
+dw_wgrad_strided_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float* __restrict__ partials,
+                        const int* __restrict__ len_in, const int* __restrict__ len_out,
+                        int C, int Tt, int Tp, int K, int s) {
+    extern __shared__ float smem[];
+    const int c = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+    const int P = (K - 1) / 2, XW = (WS_TT - 1) * s + K;
+    float* gs = smem;                 // [WS_TT]
+    float* xs = smem + WS_TT;         // [XW]
+    float* red = xs + XW;             // [128]
+    const int ngrp = 128 / K, k = tid % K, grp = tid / K;
+    const bool active = grp < ngrp;
+    const int li = min(len_in[b], Tt), lo = min(len_out[b], Tp);
+    const TG* grow = gu + ((size_t)b * C + c) * Tp;
+    const T* xrow = x + ((size_t)b * C + c) * Tt;
+    float acc = 0.f;
+    for (int t0 = 0; t0 < lo; t0 += WS_TT) {
+        __syncthreads();
+        for (int i = tid; i < WS_TT; i += 128) gs[i] = (t0 + i < lo) ? ldf(grow + t0 + i) : 0.f;
+        for (int i = tid; i < XW; i += 128) {
+            const int tau = t0 * s - P + i;
+            xs[i] = (tau >= 0 && tau < li) ? ldf(xrow + tau) : 0.f;
+        }
+        __syncthreads();
+        if (active) {
+            const int n = min(WS_TT, lo - t0);
+            for (int t = grp; t < n; t += ngrp) acc = fmaf(gs[t], xs[t * s + k], acc);
+        }
+    }
+    __syncthreads();
+    red[tid] = active ? acc : 0.f;
+    __syncthreads();
+    if (tid < K) {
+        float sum = 0.f;
+        for (int g = 0; g < ngrp; ++g) sum += red[g * K + tid];
+        partials[((size_t)b * C + c) * K + tid] = sum;
+    }
+}
+
 // ---- stride-1 tap gradient: register-blocked --------------------------------------------------
 // CTA = one channel, a group of BG samples.  Thread (kg, seg): tap group kg (R taps) x time segment.
 constexpr int WG_THREADS = 128;
@@ -423,6 +466,138 @@ dw_wgrad_reg_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float* _
     }
 }
 
+// ---- the same for 16-bit tensors: rows stay 16-bit in shared memory, filled by cp.async ----------
+// Shared rows hold the raw 16-bit values (half the footprint, and 16-byte lane pitch is conflict-free
+// without padding); conversion to fp32 happens in registers.  Two buffers: the next pass's rows are in
+// flight (cp.async) while the current pass computes.
+__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async8(void* dst, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+template <typename T> __device__ __forceinline__ void cvt8(const uint4& r, float (&f)[8]);
+template <> __device__ __forceinline__ void cvt8<__half>(const uint4& r, float (&f)[8]) {
+    const __half2* h = reinterpret_cast<const __half2*>(&r);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { const float2 q = __half22float2(h[i]); f[2 * i] = q.x; f[2 * i + 1] = q.y; }
+}
+template <> __device__ __forceinline__ void cvt8<__nv_bfloat16>(const uint4& r, float (&f)[8]) {
+    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(w[i] << 16); f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u); }
+}
+
+template <typename TG, typename T, int NCH>
+__global__ void __launch_bounds__(WR_THREADS, 3)
+dw_wgrad_reg16_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float* __restrict__ partials,
+                      const int* __restrict__ len_in, const int* __restrict__ len_out,
+                      int B, int C, int Tt, int K, int Ppad, int NR, int NST, int RS) {
+    static_assert(sizeof(TG) == 2 && sizeof(T) == 2, "16-bit tensors only");
+    extern __shared__ __align__(16) unsigned short smem16[];
+    const int tid = threadIdx.x, lane = tid & 31, wrp = tid >> 5;
+    const int c = blockIdx.x;
+    const int P = (K - 1) / 2, shift = Ppad - P;
+    const int cpr = Tt / 8;
+    const int XW = Tt + 8 * NCH + 8;
+    const int halo = XW - Tt;
+    const size_t bufsz = (size_t)2 * NR * RS;               // elements per buffer: g rows then x rows
+    float acc[8 * NCH];
+#pragma unroll
+    for (int i = 0; i < 8 * NCH; ++i) acc[i] = 0.f;
+
+    auto issue = [&](int st) {
+        const int b0 = (blockIdx.y * NST + st) * NR;
+        const int nr = min(NR, B - b0);
+        unsigned short* gs = smem16 + (st & 1) * bufsz;
+        unsigned short* xs = gs + (size_t)NR * RS;
+        for (int i = tid; i < nr * halo; i += WR_THREADS) {
+            const int r = i / halo, j = i - r * halo;
+            xs[r * RS + (j < Ppad ? j : Tt + j)] = 0;
+        }
+        for (int i = tid; i < nr * cpr; i += WR_THREADS) {
+            const int r = i / cpr, t = (i - r * cpr) * 8;
+            const int b = b0 + r;
+            const int li = min(len_in[b], Tt), lo = min(len_out[b], Tt);
+            const size_t off = ((size_t)b * C + c) * Tt + t;
+            unsigned short* gd = gs + r * RS + t;
+            unsigned short* xd = xs + r * RS + t + Ppad;
+            if (t < lo) cp_async16(gd, gu + off); else *reinterpret_cast<uint4*>(gd) = make_uint4(0, 0, 0, 0);
+            if (t < li) cp_async8(xd, x + off); else *reinterpret_cast<uint2*>(xd) = make_uint2(0, 0);
+            if (t + 4 < li) cp_async8(xd + 4, x + off + 4); else *reinterpret_cast<uint2*>(xd + 4) = make_uint2(0, 0);
+        }
+        cp_async_commit();
+    };
+    // after this thread's copies have landed: zero the tail of the vector a length falls into
+    auto patch = [&](int st) {
+        const int b0 = (blockIdx.y * NST + st) * NR;
+        const int nr = min(NR, B - b0);
+        unsigned short* gs = smem16 + (st & 1) * bufsz;
+        unsigned short* xs = gs + (size_t)NR * RS;
+        for (int i = tid; i < nr * cpr; i += WR_THREADS) {
+            const int r = i / cpr, t = (i - r * cpr) * 8;
+            const int li = min(len_in[b0 + r], Tt), lo = min(len_out[b0 + r], Tt);
+            if (t < lo && t + 8 > lo) for (int e = lo - t; e < 8; ++e) gs[r * RS + t + e] = 0;
+            if (t < li && t + 8 > li) for (int e = li - t; e < 8; ++e) xs[r * RS + t + Ppad + e] = 0;
+        }
+    };
+
+    const int nst = min(NST, (B - (int)blockIdx.y * NST * NR + NR - 1) / NR);   // passes with at least one row
+    if (nst > 0) issue(0);
+    for (int st = 0; st < nst; ++st) {
+        if (st + 1 < nst) { issue(st + 1); cp_async_wait<1>(); } else { cp_async_wait<0>(); }
+        patch(st);
+        __syncthreads();
+        const int b0 = (blockIdx.y * NST + st) * NR;
+        const int nr = min(NR, B - b0);
+        const unsigned short* gs = smem16 + (st & 1) * bufsz;
+        const unsigned short* xs = gs + (size_t)NR * RS;
+        for (int i = tid; i < nr * cpr; i += WR_THREADS) {
+            const int r = i / cpr, t = (i - r * cpr) * 8;
+            const unsigned short* xp = xs + r * RS + t;
+            float g[8], win[16];
+            cvt8<TG>(*reinterpret_cast<const uint4*>(gs + r * RS + t), g);
+            {
+                float lo8[8];
+                cvt8<T>(*reinterpret_cast<const uint4*>(xp), lo8);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) win[q] = lo8[q];
+            }
+#pragma unroll
+            for (int ch = 0; ch < NCH; ++ch) {
+                float hi8[8];
+                cvt8<T>(*reinterpret_cast<const uint4*>(xp + 8 * ch + 8), hi8);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) win[8 + q] = hi8[q];
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+#pragma unroll
+                    for (int rr = 0; rr < 8; ++rr) acc[8 * ch + q] = fmaf(g[rr], win[rr + q], acc[8 * ch + q]);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) win[q] = win[q + 8];
+            }
+        }
+        __syncthreads();
+    }
+    float* red = reinterpret_cast<float*>(smem16);       // [4][8*NCH]
+#pragma unroll
+    for (int i = 0; i < 8 * NCH; ++i) {
+        const float v = warp_sum(acc[i]);
+        if (lane == 0) red[wrp * 8 * NCH + i] = v;
+    }
+    __syncthreads();
+    for (int k = tid; k < K; k += WR_THREADS) {
+        const int kk = k + shift;
+        float sum = 0.f;
+#pragma unroll
+        for (int w = 0; w < WR_THREADS / 32; ++w) sum += red[w * 8 * NCH + kk];
+        partials[((size_t)blockIdx.y * C + c) * K + k] = sum;
+    }
+}
+
 inline int kpad(int K) { return (K + R - 1) / R * R; }
 inline int host_phys(int i) { return i + ((i >> 5) << 2); }
 
@@ -496,34 +671,74 @@ void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x
     const int P = (K - 1) / 2, Ppad = (P + 3) / 4 * 4;
     const int nch = (K + (Ppad - P) + 7) / 8;
     if (s == 1 && Tt % 8 == 0 && nch >= 2 && nch <= 12) {
-        // rows staged per pass: the count whose (rows x chunks) best fills the 128 threads, within 64 KiB
+        // rows staged per pass: the count whose (rows x chunks) best fills the 128 threads
         const int cpr = Tt / 8;
-        const int rs = host_phys(Tt + 8 * nch + 8) + 4, rsp = (rs + 3) / 4 * 4;
-        int NR = 1; double best = 0.0;
-        for (int nr = 1; nr <= 8 && nr <= B; ++nr) {
-            if ((size_t)2 * nr * rsp * sizeof(float) > 64 * 1024) break;
-            const int work = nr * cpr, iters = (work + WR_THREADS - 1) / WR_THREADS;
-            const double eff = (double)work / (iters * WR_THREADS);
-            if (eff > best + 1e-9) { best = eff; NR = nr; }
-        }
         const int NST = 2;
-        nsplit = (B + NR * NST - 1) / (NR * NST);
-        const size_t smem = std::max((size_t)2 * NR * rsp, (size_t)4 * 8 * nch) * sizeof(float);
-        dim3 grid(C, nsplit);
+        if (dtype == F32) {
+            const int rs = host_phys(Tt + 8 * nch + 8) + 4, rsp = (rs + 3) / 4 * 4;
+            int NR = 1; double best = 0.0;
+            for (int nr = 1; nr <= 8 && nr <= B; ++nr) {
+                if ((size_t)2 * nr * rsp * sizeof(float) > 64 * 1024) break;
+                const int work = nr * cpr, iters = (work + WR_THREADS - 1) / WR_THREADS;
+                const double eff = (double)work / (iters * WR_THREADS);
+                if (eff > best + 1e-9) { best = eff; NR = nr; }
+            }
+            nsplit = (B + NR * NST - 1) / (NR * NST);
+            const size_t smem = std::max((size_t)2 * NR * rsp, (size_t)4 * 8 * nch) * sizeof(float);
+            dim3 grid(C, nsplit);
 #define SC_WR_CASE(N)                                                                                          \
-        case N: {                                                                                              \
-            SC_DISPATCH_IO(dtype, odt, {                                                                       \
-                auto kern = dw_wgrad_reg_kernel<OT, T, N>;                                                     \
+            case N: {                                                                                          \
+                auto kern = dw_wgrad_reg_kernel<float, float, N>;                                              \
                 static bool cfg_done = false;                                                                  \
                 if (!cfg_done) { cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024); cfg_done = true; } \
-                kern<<<grid, WR_THREADS, smem, L.stream>>>((const OT*)gu, (const T*)x, partials, len_in, len_out, \
-                                                           B, C, Tt, K, Ppad, NR, NST, rsp); });               \
-        } break;
-        switch (nch) {
-            SC_WR_CASE(2) SC_WR_CASE(3) SC_WR_CASE(4) SC_WR_CASE(5) SC_WR_CASE(6) SC_WR_CASE(7) SC_WR_CASE(8)
-            SC_WR_CASE(9) SC_WR_CASE(10) SC_WR_CASE(11) SC_WR_CASE(12)
-        }
+                kern<<<grid, WR_THREADS, smem, L.stream>>>((const float*)gu, (const float*)x, partials, len_in, len_out, \
+                                                           B, C, Tt, K, Ppad, NR, NST, rsp);                   \
+            } break;
+            switch (nch) {
+                SC_WR_CASE(2) SC_WR_CASE(3) SC_WR_CASE(4) SC_WR_CASE(5) SC_WR_CASE(6) SC_WR_CASE(7) SC_WR_CASE(8)
+                SC_WR_CASE(9) SC_WR_CASE(10) SC_WR_CASE(11) SC_WR_CASE(12)
+            }
 #undef SC_WR_CASE
+        } else {
+            const int RS = (Tt + 8 * nch + 8 + 7) / 8 * 8;
+            int NR = 1; double best = 0.0;
+            for (int nr = 1; nr <= 8 && nr <= B; ++nr) {
+                if ((size_t)2 * 2 * nr * RS * 2 > 96 * 1024) break;
+                const int work = nr * cpr, iters = (work + WR_THREADS - 1) / WR_THREADS;
+                const double eff = (double)work / (iters * WR_THREADS);
+                if (eff > best + 1e-9) { best = eff; NR = nr; }
+            }
+            nsplit = (B + NR * NST - 1) / (NR * NST);
+            const size_t smem = std::max((size_t)2 * 2 * NR * RS * 2, (size_t)4 * 8 * nch * sizeof(float));
+            dim3 grid(C, nsplit);
+#define SC_WR_CASE(N)                                                                                          \
+            case N: {                                                                                          \
+                if (dtype == F16) {                                                                            \
+                    auto kern = dw_wgrad_reg16_kernel<__half, __half, N>;                                      \
+                    static bool cfg_done = false;                                                              \
+                    if (!cfg_done) { cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024); cfg_done = true; } \
+                    kern<<<grid, WR_THREADS, smem, L.stream>>>((const __half*)gu, (const __half*)x, partials, len_in, len_out, \
+                                                               B, C, Tt, K, Ppad, NR, NST, RS);               \
+                } else if (odt == F16) {                                                                       \
+                    auto kern = dw_wgrad_reg16_kernel<__half, __nv_bfloat16, N>;                               \
+                    static bool cfg_done = false;                                                              \
+                    if (!cfg_done) { cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024); cfg_done = true; } \
+                    kern<<<grid, WR_THREADS, smem, L.stream>>>((const __half*)gu, (const __nv_bfloat16*)x, partials, len_in, len_out, \
+                                                               B, C, Tt, K, Ppad, NR, NST, RS);               \
+                } else {                                                                                       \
+                    auto kern = dw_wgrad_reg16_kernel<__nv_bfloat16, __nv_bfloat16, N>;                        \
+                    static bool cfg_done = false;                                                              \
+                    if (!cfg_done) { cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024); cfg_done = true; } \
+                    kern<<<grid, WR_THREADS, smem, L.stream>>>((const __nv_bfloat16*)gu, (const __nv_bfloat16*)x, partials, len_in, len_out, \
+                                                               B, C, Tt, K, Ppad, NR, NST, RS);               \
+                }                                                                                              \
+            } break;
+            switch (nch) {
+                SC_WR_CASE(2) SC_WR_CASE(3) SC_WR_CASE(4) SC_WR_CASE(5) SC_WR_CASE(6) SC_WR_CASE(7) SC_WR_CASE(8)
+                SC_WR_CASE(9) SC_WR_CASE(10) SC_WR_CASE(11) SC_WR_CASE(12)
+            }
+#undef SC_WR_CASE
+        }
     } else if (s == 1) {
         const int Kp = kpad(K), NG = Kp / R, nseg = WG_THREADS / NG;
         const int seglen = ((WG_TT + nseg - 1) / nseg + R - 1) / R * R;
@@ -533,6 +748,12 @@ void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x
         dim3 grid(C, nsplit);
         SC_DISPATCH_IO(dtype, odt, (dw_wgrad_s1_kernel<OT, T><<<grid, WG_THREADS, smem, L.stream>>>(
                                        (const OT*)gu, (const T*)x, partials, len_in, len_out, B, C, Tt, K, Kp)));
+    } else if (K <= 128) {
+        nsplit = B;
+        const size_t smem = (size_t)(WS_TT + (WS_TT - 1) * s + K + 128) * sizeof(float);
+        dim3 grid(C, B);
+        SC_DISPATCH_IO(dtype, odt, (dw_wgrad_strided_kernel<OT, T><<<grid, 128, smem, L.stream>>>(
+                                       (const OT*)gu, (const T*)x, partials, len_in, len_out, C, Tt, Tp, K, s)));
     } else {
         nsplit = B;
         SC_DISPATCH_IO(dtype, odt, (dw_wgrad_generic_kernel<OT, T><<<C, 128, 0, L.stream>>>(

@@ -138,15 +138,18 @@ struct BnBwdArgs {
     const float *gamma, *beta;                     // for the relu-then-add gate
     const int* len_out; const int* nvalid;
     int B, C, Tp, has_bn, has_relu, res_before_relu, residual;
-    float4* partials;                              // [B*C]
-    float* amax_part;                              // [B*C] per-row max |gated gradient| (only with gmax)
+    float4* partials;                              // [B*C*nslots]
+    float* amax_part;                              // [B*C*nslots] max |gated gradient| (only with gmax)
+    int nslots;                                    // partial slots per (sample, channel) row; set by bn_bwd_reduce
     float* gmax;                                   // device scalar: bound on |gv| over the tensor (nullable)
     int gv_dtype;                                  // storage type of gv (OT)
     float4* coef; float4* coef_r;                  // [C]: (k, c1, c2, unused)
     void* gv; void* gvr; void* gres;               // outputs of the apply step (gvr: proj, gres: identity)
                                                    // gv is multiplied by pow2_scale(*gmax) when gmax is set
 };
-void bn_bwd_reduce(const Launch& L, int dtype, const BnBwdArgs& a);
+void bn_bwd_reduce(const Launch& L, int dtype, BnBwdArgs& a);
+// partial slots per row that bn_bwd_reduce may use for rows of Tp frames (for scratch sizing)
+inline int bn_bwd_max_slots(int Tp) { return Tp / 256 + 2; }
 void bn_bwd_finalize(const Launch& L, const BnBwdArgs& a, const float* gamma, const float* gamma_r,
                      float* dgamma, float* dbeta, float* dgamma_r, float* dbeta_r, float* dbias,
                      int accumulate);
