@@ -18,6 +18,7 @@
 
 #include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 
 #include "common.cuh"
 #include "sm100.cuh"
@@ -68,6 +69,44 @@ __device__ __forceinline__ void store_row_chunk(OT* row, int col0, int ncols_tot
     for (int i = 0; i < 32; ++i) if (col0 + i < ncols_total) stf(row + col0 + i, f[i]);
 }
 
+// Coalesced store of a warp's 32 x 32 accumulator block.  After tcgen05.ld lane l holds 32 consecutive
+// columns of row l; storing that directly makes every store instruction touch 32 different rows with
+// 16 bytes each (half-filled sectors).  The block is transposed through a per-warp shared-memory
+// buffer (row pitch 36 floats) so that each instruction writes whole 128-byte (fp32) or 64-byte
+// (16-bit) row segments.  `rows_left` / `cols_left` bound the valid part; cols are a multiple of 8.
+constexpr int kStgPitch = 36;
+constexpr int kStgFloatsPerWarp = 32 * kStgPitch;
+template <typename OT>
+__device__ __forceinline__ void store_block_staged(float* stg, const float (&f)[32], OT* out, size_t ld,
+                                                   int rows_left, int cols_left, int lane) {
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+        *reinterpret_cast<float4*>(stg + lane * kStgPitch + 4 * i) = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
+    __syncwarp();
+    if (sizeof(OT) == 4) {
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int r = it * 4 + (lane >> 3), c = (lane & 7) * 4;
+            if (r < rows_left && c < cols_left) {
+                const float4 v = *reinterpret_cast<const float4*>(stg + r * kStgPitch + c);
+                *reinterpret_cast<float4*>(reinterpret_cast<float*>(out) + (size_t)r * ld + c) = v;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int r = it * 8 + (lane >> 2), c = (lane & 3) * 8;
+            if (r < rows_left && c < cols_left) {
+                const float4 a = *reinterpret_cast<const float4*>(stg + r * kStgPitch + c);
+                const float4 b = *reinterpret_cast<const float4*>(stg + r * kStgPitch + c + 4);
+                const float g[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+                st8<OT>(out + (size_t)r * ld + c, g);
+            }
+        }
+    }
+}
+
 template <typename T, int MODE, int MT, int BN, int STAGES>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, TcParams p) {
@@ -84,6 +123,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     uint64_t* empty = full + STAGES;
     uint64_t* accum = empty + STAGES;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
+    float* stg_all = reinterpret_cast<float*>(smem + STAGES * STAGE + 256);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n0 = blockIdx.x * BN;
@@ -242,11 +282,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
 #pragma unroll
                     for (int i = 0; i < 32; ++i) if (i >= nv) f[i] = 0.f;
                 }
-                if (row < p.M) {
-                    const size_t rbase = ((size_t)z * p.M + row) * p.Ncols;
-                    if (MODE == MODE_FWD && p.out_f32) store_row_chunk(reinterpret_cast<float*>(p.out) + rbase, n0 + c0, p.Ncols, f);
-                    else if (MODE == MODE_WGRAD) store_row_chunk(reinterpret_cast<float*>(p.out) + rbase, n0 + c0, p.Ncols, f);
-                    else store_row_chunk(reinterpret_cast<T*>(p.out) + rbase, n0 + c0, p.Ncols, f);
+                {
+                    const int row_w = m0 + mt * 128 + warp * 32;             // first row of this warp's block
+                    const size_t base = ((size_t)z * p.M + row_w) * p.Ncols + n0 + c0;
+                    float* stg = stg_all + warp * kStgFloatsPerWarp;
+                    const int rl = p.M - row_w, cl = p.Ncols - (n0 + c0);
+                    if ((MODE == MODE_FWD && p.out_f32) || MODE == MODE_WGRAD)
+                        store_block_staged<float>(stg, f, reinterpret_cast<float*>(p.out) + base, p.Ncols, rl, cl, lane);
+                    else
+                        store_block_staged<T>(stg, f, reinterpret_cast<T*>(p.out) + base, p.Ncols, rl, cl, lane);
                 }
             }
             if (MODE == MODE_FWD && p.stats && row < p.M)
@@ -258,6 +302,199 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);
     }
 
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 0) ptx::tmem_dealloc(tmem, TMEM_COLS);
+}
+
+// ---- persistent, warp-specialised form for the forward and input-gradient contractions -----------
+// One CTA per SM loops over output tiles (tile = blockIdx.x + i * gridDim.x).  Warps 0-3 are the
+// epilogue (warp w owns TMEM lanes 32w..32w+31), warp 4 is the TMA producer, warp 5 issues the MMAs.
+// The accumulator is double-buffered in tensor memory, so the epilogue of tile i (TMEM -> registers ->
+// statistics -> global stores) overlaps the loads and MMAs of tile i+1; the shared-memory ring keeps
+// running across tile boundaries.  Barrier set-up and the TMEM allocation are paid once per CTA.
+constexpr int kPThreads = 192;
+
+template <typename T, int MODE, int MT, int BN, int STAGES>
+__global__ void __launch_bounds__(kPThreads, 1)
+tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                          TcParams p, int tiles_n, int tiles_m, int tiles_total) {
+    static_assert(MODE == MODE_FWD || MODE == MODE_DGRAD, "forward / input gradient only");
+    constexpr int A_BYTES = MT * 128 * 128;
+    constexpr int B_BYTES = BN * 128;
+    constexpr int STAGE = A_BYTES + B_BYTES;
+    constexpr uint32_t ACC_COLS = MT * BN;
+    constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;
+    static_assert(TMEM_COLS == 128 || TMEM_COLS == 256 || TMEM_COLS == 512, "tmem columns");
+    constexpr uint32_t IDESC = ptx::instr_desc(Fmt<T>::v, MODE == MODE_DGRAD ? 1u : 0u, 1u, 128, BN);
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE);
+    uint64_t* empty = full + STAGES;
+    uint64_t* acc_full = empty + STAGES;       // [2]
+    uint64_t* acc_empty = acc_full + 2;        // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    float* stg_all = reinterpret_cast<float*>(smem + STAGES * STAGE + 256);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
+        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 128); }
+        ptx::fence_barrier_init();
+        ptx::prefetch_tensormap(&mapA);
+        ptx::prefetch_tensormap(&mapB);
+    }
+    if (warp == 0) { ptx::tmem_alloc(tmem_slot, TMEM_COLS); ptx::tmem_relinquish(); }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    const int nkb = (p.Kdim + BK - 1) / BK;
+
+    // tile -> (n0, m0, sample); returns false for a tile wholly in the sample's padding
+    auto tile_info = [&](int tile, int& n0, int& m0, int& z, int& len) -> bool {
+        const int tn = tile % tiles_n, r = tile / tiles_n;
+        n0 = tn * BN; m0 = (r % tiles_m) * (128 * MT); z = r / tiles_m;
+        len = p.len_out ? min(p.len_out[z], p.Tp) : p.Tp;
+        return n0 < len;
+    };
+
+    if (warp == 4) {
+        if (lane == 0) {                              // ---- TMA producer ----
+            int it = 0;
+            bool dead = false;
+            for (int tile = blockIdx.x; tile < tiles_total && !dead; tile += gridDim.x) {
+                int n0, m0, z, len;
+                if (!tile_info(tile, n0, m0, z, len)) continue;
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % STAGES, ph = (it / STAGES) & 1;
+                    if (!ptx::mbar_wait(&empty[s], ph ^ 1)) { raise_status(p.status, kErrTimeout); dead = true; break; }
+                    ptx::mbar_arrive_expect_tx(&full[s], STAGE);
+                    uint8_t* sA = smem + s * STAGE;
+                    uint8_t* sB = sA + A_BYTES;
+                    const int k0 = kb * BK;
+                    if (MODE == MODE_FWD) {
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt) ptx::tma_load_2d(sA + mt * 16384, &mapA, &full[s], k0, m0 + mt * 128);
+                    } else {
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                            for (int j = 0; j < 2; ++j)
+                                ptx::tma_load_2d(sA + mt * 16384 + j * 8192, &mapA, &full[s], m0 + mt * 128 + 64 * j, k0);
+                    }
+#pragma unroll
+                    for (int j = 0; j < BN / 64; ++j) ptx::tma_load_3d(sB + j * 8192, &mapB, &full[s], n0 + 64 * j, k0, z);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 5) {
+        if (lane == 0) {                              // ---- MMA issuer ----
+            int it = 0, j = 0;
+            bool dead = false;
+            for (int tile = blockIdx.x; tile < tiles_total && !dead; tile += gridDim.x) {
+                int n0, m0, z, len;
+                if (!tile_info(tile, n0, m0, z, len)) continue;
+                const int buf = j & 1;
+                if (!ptx::mbar_wait(&acc_empty[buf], ((j >> 1) & 1) ^ 1)) { raise_status(p.status, kErrTimeout); break; }
+                ptx::tc_fence_after();
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % STAGES, ph = (it / STAGES) & 1;
+                    if (!ptx::mbar_wait(&full[s], ph)) { raise_status(p.status, kErrTimeout); dead = true; break; }
+                    ptx::tc_fence_after();
+                    const uint32_t aA = ptx::smem_u32(smem + s * STAGE), aB = aA + A_BYTES;
+#pragma unroll
+                    for (int ks = 0; ks < BK / 16; ++ks) {
+                        const uint64_t bdesc = ptx::smem_desc(aB + ks * 2048, 8192, 1024);
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt) {
+                            const uint64_t adesc = (MODE == MODE_DGRAD) ? ptx::smem_desc(aA + mt * 16384 + ks * 2048, 8192, 1024)
+                                                                        : ptx::smem_desc(aA + mt * 16384 + ks * 32, 16, 1024);
+                            ptx::mma_f16(tmem + buf * ACC_COLS + mt * BN, adesc, bdesc, IDESC, (kb > 0 || ks > 0) ? 1u : 0u);
+                        }
+                    }
+                    ptx::mma_commit(&empty[s]);
+                }
+                if (!dead) ptx::mma_commit(&acc_full[buf]);
+                ++j;
+            }
+        }
+        __syncwarp();
+    } else {                                          // ---- epilogue warps 0..3 ----
+        int j = 0;
+        for (int tile = blockIdx.x; tile < tiles_total; tile += gridDim.x) {
+            int n0, m0, z, len;
+            if (!tile_info(tile, n0, m0, z, len)) {
+                if (p.zero_fill) {
+                    const int esz = (MODE == MODE_FWD && p.out_f32) ? 4 : (int)sizeof(T);
+                    const int vec_per_row = BN * esz / 16;
+                    for (int i = tid; i < 128 * MT * vec_per_row; i += 128) {
+                        const int r = m0 + i / vec_per_row, cb = (i % vec_per_row) * (16 / esz);
+                        if (r < p.M && n0 + cb < p.Ncols) {
+                            uint8_t* dst = reinterpret_cast<uint8_t*>(p.out) + (((size_t)z * p.M + r) * p.Ncols + n0 + cb) * esz;
+                            *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
+                        }
+                    }
+                }
+                continue;
+            }
+            const int buf = j & 1;
+            bool ok = ptx::mbar_wait(&acc_full[buf], (j >> 1) & 1);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) { if (lane == 0) raise_status(p.status, kErrTimeout); break; }
+            ptx::tc_fence_after();
+#pragma unroll 1
+            for (int mt = 0; mt < MT; ++mt) {
+                const int row = m0 + mt * 128 + warp * 32 + lane;
+                float sn = 0.f, smean = 0.f, sm2 = 0.f;
+                const float bias = (MODE == MODE_FWD && p.bias && row < p.M) ? p.bias[row] : 0.f;
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    if (n0 + c0 >= p.Ncols) break;
+                    float f[32];
+                    {
+                        uint32_t r[32];
+                        ptx::tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + buf * ACC_COLS + mt * BN + c0, r);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(r[i]) + bias;
+                    }
+                    if (MODE == MODE_FWD) {
+                        const int nv = max(0, min(32, len - (n0 + c0)));
+                        if (p.stats && nv > 0) {
+                            float s = 0.f;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) if (i < nv) s += f[i];
+                            const float cm = s / (float)nv;
+                            float q = 0.f;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) if (i < nv) { const float d = f[i] - cm; q = fmaf(d, d, q); }
+                            chan_merge(sn, smean, sm2, (float)nv, cm, q);
+                        }
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) if (i >= nv) f[i] = 0.f;
+                    }
+                    {
+                        const int row_w = m0 + mt * 128 + warp * 32;
+                        const size_t base = ((size_t)z * p.M + row_w) * p.Ncols + n0 + c0;
+                        float* stg = stg_all + warp * kStgFloatsPerWarp;
+                        const int rl = p.M - row_w, cl = p.Ncols - (n0 + c0);
+                        if (MODE == MODE_FWD && p.out_f32)
+                            store_block_staged<float>(stg, f, reinterpret_cast<float*>(p.out) + base, p.Ncols, rl, cl, lane);
+                        else
+                            store_block_staged<T>(stg, f, reinterpret_cast<T*>(p.out) + base, p.Ncols, rl, cl, lane);
+                    }
+                }
+                if (MODE == MODE_FWD && p.stats && row < p.M)
+                    p.stats[((size_t)z * tiles_n + (n0 / BN)) * p.M + row] = make_float2(smean * sn, sm2);
+            }
+            ptx::tc_fence_before();
+            ptx::mbar_arrive(&acc_empty[buf]);        // this thread is done reading the accumulator
+            ++j;
+        }
+    }
     ptx::tc_fence_before();
     __syncthreads();
     if (warp == 0) ptx::tmem_dealloc(tmem, TMEM_COLS);
@@ -287,7 +524,7 @@ bool make_map(const TcState* st, CUtensorMap* m, int dtype, const void* base, in
 
 template <typename T, int MODE, int MT, int BN, int STAGES>
 void launch(const Launch& L, dim3 grid, const CUtensorMap& a, const CUtensorMap& b, const TcParams& p) {
-    constexpr int smem = STAGES * (MT * 16384 + BN * 128) + 1024 + 256;
+    constexpr int smem = STAGES * (MT * 16384 + BN * 128) + 1024 + 256 + 4 * kStgFloatsPerWarp * 4;
     static bool configured = false;
     auto kern = tc_gemm_kernel<T, MODE, MT, BN, STAGES>;
     if (!configured) {
@@ -302,6 +539,27 @@ template <int MODE, int MT, int BN, int STAGES>
 void launch_dt(int dtype, const Launch& L, dim3 grid, const CUtensorMap& a, const CUtensorMap& b, const TcParams& p) {
     if (dtype == F16) launch<__half, MODE, MT, BN, STAGES>(L, grid, a, b, p);
     else launch<__nv_bfloat16, MODE, MT, BN, STAGES>(L, grid, a, b, p);
+}
+
+template <typename T, int MODE, int MT, int BN, int STAGES>
+void launch_persistent(const Launch& L, int sm_count, const CUtensorMap& a, const CUtensorMap& b, const TcParams& p,
+                       int tiles_n, int tiles_m, int batch) {
+    constexpr int smem = STAGES * (MT * 16384 + BN * 128) + 1024 + 256 + 4 * kStgFloatsPerWarp * 4;
+    static bool configured = false;
+    auto kern = tc_gemm_persistent_kernel<T, MODE, MT, BN, STAGES>;
+    if (!configured) {
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        configured = true;
+    }
+    const int total = tiles_n * tiles_m * batch;
+    kern<<<std::min(sm_count, total), kPThreads, smem, L.stream>>>(a, b, p, tiles_n, tiles_m, total);
+    L.count();
+}
+template <int MODE, int MT, int BN, int STAGES>
+void launch_persistent_dt(int dtype, const Launch& L, int sm_count, const CUtensorMap& a, const CUtensorMap& b,
+                          const TcParams& p, int tiles_n, int tiles_m, int batch) {
+    if (dtype == F16) launch_persistent<__half, MODE, MT, BN, STAGES>(L, sm_count, a, b, p, tiles_n, tiles_m, batch);
+    else launch_persistent<__nv_bfloat16, MODE, MT, BN, STAGES>(L, sm_count, a, b, p, tiles_n, tiles_m, batch);
 }
 
 bool shape_ok(const TcState* st, int dtype, int Cin, int Cout, int Tp) {
@@ -335,6 +593,8 @@ int tc_init(TcState* st, int device, int sm_count) {
     cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
     st->encode_fn = (e == cudaSuccess && q == cudaDriverEntryPointSuccess) ? fn : nullptr;
     st->ready = st->encode_fn != nullptr;
+    const char* e_p = getenv("SEPCONV_GEMM_PERSISTENT");
+    st->persistent = !(e_p && e_p[0] == '0');
     if (!st->ready) { fprintf(stderr, "sepconv: cuTensorMapEncodeTiled not available\n"); return -11; }
     return 0;
 }
@@ -368,7 +628,10 @@ bool tc_gemm_fwd(const TcState* st, const Launch& L, int dtype, const void* w, c
     p.out_f32 = (out_dtype == F32);
     const int mt = Cout > 128 ? 2 : 1;
     dim3 grid((Tp + FWD_BN - 1) / FWD_BN, (Cout + 128 * mt - 1) / (128 * mt), B);
-    if (mt == 2) launch_dt<MODE_FWD, 2, FWD_BN, 2>(dtype, L, grid, ma, mb, p);
+    if (st->persistent) {
+        if (mt == 2) launch_persistent_dt<MODE_FWD, 2, FWD_BN, 4>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
+        else launch_persistent_dt<MODE_FWD, 1, FWD_BN, 6>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
+    } else if (mt == 2) launch_dt<MODE_FWD, 2, FWD_BN, 2>(dtype, L, grid, ma, mb, p);
     else launch_dt<MODE_FWD, 1, FWD_BN, 3>(dtype, L, grid, ma, mb, p);
     *parts_per_b = grid.x; *tile_w = FWD_BN;
     return partials != nullptr;
@@ -388,7 +651,10 @@ void tc_gemm_dgrad(const TcState* st, const Launch& L, int dtype, const void* w,
     p.M = Cin; p.Ncols = Tp; p.Kdim = Cout; p.B = B; p.Tp = Tp; p.zero_fill = 1;
     const int mt = Cin > 128 ? 2 : 1;
     dim3 grid((Tp + FWD_BN - 1) / FWD_BN, (Cin + 128 * mt - 1) / (128 * mt), B);
-    if (mt == 2) launch_dt<MODE_DGRAD, 2, FWD_BN, 2>(dtype, L, grid, ma, mb, p);
+    if (st->persistent) {
+        if (mt == 2) launch_persistent_dt<MODE_DGRAD, 2, FWD_BN, 4>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
+        else launch_persistent_dt<MODE_DGRAD, 1, FWD_BN, 6>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
+    } else if (mt == 2) launch_dt<MODE_DGRAD, 2, FWD_BN, 2>(dtype, L, grid, ma, mb, p);
     else launch_dt<MODE_DGRAD, 1, FWD_BN, 3>(dtype, L, grid, ma, mb, p);
 }
 

@@ -10,6 +10,7 @@ struct TcState {
     void* encode_fn = nullptr;   // cuTensorMapEncodeTiled, resolved through the runtime
     int sm_count = 0;
     bool ready = false;
+    bool persistent = true;      // forward / input gradient: persistent warp-specialised kernel
 };
 
 int tc_init(TcState* st, int device, int sm_count);
