@@ -93,6 +93,7 @@ struct BlockIO {                 // raw pointers after validation
     bool x_clean, res_clean;     // inputs known to be zero in padded frames
     bool lengths_ready;          // len_out / nvalid already computed
     void* w16_keep;              // optional: where to leave the float16 copy of wp for the backward pass
+    bool w16_ready;              // w16_keep already holds the copy
 };
 
 // Type of the library-internal contraction operands (u, gv, gu) of this layer.
@@ -160,7 +161,7 @@ int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
     const void* wp_op = p->wp;
     if (odt != dt) {
         void* dst = io.w16_keep ? io.w16_keep : f.w16;
-        convert_bf16_to_f16(L, p->wp, dst, (int64_t)m.Cout * m.Cin);
+        if (!(io.w16_keep && io.w16_ready)) convert_bf16_to_f16(L, p->wp, dst, (int64_t)m.Cout * m.Cin);
         wp_op = dst;
     }
     pointwise_bn(ctx, L, d, m, m.Cin, odt, wp_op, u, f.v, io.len_out, io.nvalid, sv->mean, sv->invstd, f.partials,
@@ -645,6 +646,17 @@ int encoder_fwd_bwd(sc_ctx* ctx, const sc_encoder_desc* e, const sc_tensor* x, c
     auto len_in_of = [&](int i) -> const int* { return i == 0 ? lengths_dev : P.L[i - 1].len_out; };
     auto res_src = [&](int i) -> int { return (e->res_from && e->res_from[i] >= 0) ? e->res_from[i] : i; };
 
+    // float16 copies of the pointwise weights of every layer that needs one: one launch
+    {
+        ConvertList cl; cl.count = 0;
+        for (int i = 0; i < n; ++i) {
+            if (!P.L[i].w16) continue;
+            if (cl.count == 48) { convert_bf16_to_f16_many(L, cl); cl.count = 0; }
+            cl.src[cl.count] = prm[i].wp; cl.dst[cl.count] = P.L[i].w16; cl.n[cl.count] = P.L[i].m.Cout * P.L[i].m.Cin;
+            ++cl.count;
+        }
+        convert_bf16_to_f16_many(L, cl);
+    }
     // forward
     for (int i = 0; i < n; ++i) {
         LayerPlan& lp = P.L[i];
@@ -657,7 +669,7 @@ int encoder_fwd_bwd(sc_ctx* ctx, const sc_encoder_desc* e, const sc_tensor* x, c
         io.len_in = len_in_of(i); io.len_out = lp.len_out; io.nvalid = lp.nvalid;
         io.x_clean = i > 0; io.res_clean = lp.d.residual != SC_RES_NONE && res_src(i) > 0;
         io.lengths_ready = !lp.own_lengths;
-        io.w16_keep = lp.w16;
+        io.w16_keep = lp.w16; io.w16_ready = true;
         SC_TRY(block_fwd_impl(ctx, L, &lp.d, lp.m, io, &prm[i], &lp.sv, nullptr, nullptr, f));
     }
     if (out_lengths_dev)

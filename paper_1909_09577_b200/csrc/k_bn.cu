@@ -102,9 +102,26 @@ bn_finalize_kernel(const float2* __restrict__ partials, int parts_per_b, int til
     const int o = blockIdx.x * 32 + cx;
     const int nparts = B * parts_per_b;
     const double N = (double)(*nvalid);
+    // this thread's parts: sl, sl+32, ...; the first eight are kept in registers between the two passes
+    constexpr int kKeep = 8;
+    float2 keep[kKeep];
+    int cnts[kKeep];
+#pragma unroll
+    for (int i = 0; i < kKeep; ++i) {
+        const int pi = sl + i * kFinSlices;
+        cnts[i] = 0;
+        keep[i] = make_float2(0.f, 0.f);
+        if (o < C && pi < nparts) {
+            const int b = pi / parts_per_b, j = pi - b * parts_per_b;
+            cnts[i] = max(0, min(len_out[b] - j * tile_w, tile_w));
+            if (cnts[i] > 0) keep[i] = partials[(size_t)pi * C + o];
+        }
+    }
     double s1 = 0.0;
+#pragma unroll
+    for (int i = 0; i < kKeep; ++i) if (cnts[i] > 0) s1 += (double)keep[i].x;
     if (o < C)
-        for (int pi = sl; pi < nparts; pi += kFinSlices) {
+        for (int pi = sl + kKeep * kFinSlices; pi < nparts; pi += kFinSlices) {
             const int b = pi / parts_per_b, j = pi - b * parts_per_b;
             if (len_out[b] - j * tile_w > 0) s1 += (double)partials[(size_t)pi * C + o].x;
         }
@@ -118,8 +135,14 @@ bn_finalize_kernel(const float2* __restrict__ partials, int parts_per_b, int til
     __syncthreads();
     const double mean = sh_mean[cx];
     double q = 0.0;
+#pragma unroll
+    for (int i = 0; i < kKeep; ++i)
+        if (cnts[i] > 0) {
+            const double d = (double)keep[i].x / (double)cnts[i] - mean;
+            q += (double)keep[i].y + (double)cnts[i] * d * d;
+        }
     if (o < C)
-        for (int pi = sl; pi < nparts; pi += kFinSlices) {
+        for (int pi = sl + kKeep * kFinSlices; pi < nparts; pi += kFinSlices) {
             const int b = pi / parts_per_b, j = pi - b * parts_per_b;
             const int cnt = min(len_out[b] - j * tile_w, tile_w);
             if (cnt <= 0) continue;
@@ -278,16 +301,32 @@ bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const float* gamma_r, fl
     float amax = 0.f;
     if (o < a.C) {
         const int vpr = a.Tp / 8;
-        for (int pi = sl; pi < a.B * a.nslots; pi += kFinSlices) {
-            const int b = pi / a.nslots, slot = pi - b * a.nslots;
-            const long long r = (long long)b * a.C + o;
-            if (a.nslots > 1) {      // slots in use for this row (see bn_bwd_reduce_fast_kernel)
-                const int used = (int)((((r + 1) * vpr - 1) >> 5) - ((r * vpr) >> 5)) + 1;
-                if (slot >= used) continue;
+        const int np = a.B * a.nslots;
+        for (int base = sl; base < np; base += 8 * kFinSlices) {
+            float4 pv[8]; float am[8]; bool use[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {          // issue every load before the first add
+                const int pi = base + i * kFinSlices;
+                use[i] = pi < np;
+                pv[i] = make_float4(0.f, 0.f, 0.f, 0.f); am[i] = 0.f;
+                if (use[i]) {
+                    const int b = pi / a.nslots, slot = pi - b * a.nslots;
+                    const long long r = (long long)b * a.C + o;
+                    if (a.nslots > 1) {      // slots in use for this row (see bn_bwd_reduce_fast_kernel)
+                        const int used = (int)((((r + 1) * vpr - 1) >> 5) - ((r * vpr) >> 5)) + 1;
+                        use[i] = slot < used;
+                    }
+                    if (use[i]) {
+                        pv[i] = a.partials[(size_t)r * a.nslots + slot];
+                        if (a.gmax) am[i] = a.amax_part[(size_t)r * a.nslots + slot];
+                    }
+                }
             }
-            const float4 p = a.partials[(size_t)r * a.nslots + slot];
-            s0 += p.x; s1 += p.y; s2 += p.z; s3 += p.w;
-            if (a.gmax) amax = fmaxf(amax, a.amax_part[(size_t)r * a.nslots + slot]);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                s0 += pv[i].x; s1 += pv[i].y; s2 += pv[i].z; s3 += pv[i].w;
+                amax = fmaxf(amax, am[i]);
+            }
         }
     }
     shs[sl][cx] = make_float4((float)s0, (float)s1, (float)s2, (float)s3);
@@ -627,6 +666,23 @@ __global__ void convert_bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ src
 void convert_bf16_to_f16(const Launch& L, const void* src, void* dst, int64_t n) {
     KScope ks_(L, KC_EW, 4.0 * n, 0.0);
     convert_bf16_to_f16_kernel<<<(unsigned)((n + 255) / 256), 256, 0, L.stream>>>((const __nv_bfloat16*)src, (__half*)dst, n);
+    L.count();
+}
+
+__global__ void convert_many_kernel(ConvertList list) {
+    const int item = blockIdx.y;
+    const __nv_bfloat16* src = (const __nv_bfloat16*)list.src[item];
+    __half* dst = (__half*)list.dst[item];
+    const int n = list.n[item];
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
+        dst[i] = __float2half_rn(__bfloat162float(src[i]));
+}
+void convert_bf16_to_f16_many(const Launch& L, const ConvertList& list) {
+    if (list.count == 0) return;
+    double total = 0;
+    for (int i = 0; i < list.count; ++i) total += list.n[i];
+    KScope ks_(L, KC_EW, 4.0 * total, 0.0);
+    convert_many_kernel<<<dim3(64, list.count), 256, 0, L.stream>>>(list);
     L.count();
 }
 

@@ -95,6 +95,9 @@ void reduce_partials(const Launch& L, const float* partials, int nsplit, int64_t
                      const float* gmax = nullptr);
 // dst (half) = src (bf16), n elements
 void convert_bf16_to_f16(const Launch& L, const void* src, void* dst, int64_t n);
+// the same for up to 48 arrays in one launch
+struct ConvertList { const void* src[48]; void* dst[48]; int n[48]; int count; };
+void convert_bf16_to_f16_many(const Launch& L, const ConvertList& list);
 
 // ---- batch norm -----------------------------------------------------------------------------
 // Per-(b,channel) row moments over t < len_out[b]: partials[(b*C+o)] = (sum, M2 about the row mean).
