@@ -26,7 +26,7 @@ constexpr int NB = 64;              // frames per block
 constexpr int MAXROWS = 256;        // block rows (incl. separators) per CTA: two MMA M-tiles
 constexpr int ROWS_ALLOC = 265;     // + one slack row in front, a few behind; 8m+1 so that the eight
                                     // chunk columns start in different 16-byte bank groups
-constexpr int kThreads = 128;
+constexpr int kThreads = 256;       // warps 0-3 read back M-tile 0, warps 4-7 M-tile 1
 
 __device__ __forceinline__ uint64_t desc_noswz(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
     return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46);
@@ -84,13 +84,13 @@ dw_tc_kernel(const TI* __restrict__ in, const TW* __restrict__ w, TO* __restrict
 
     // ---- stage the input rows: frame t = 64 i + 8 q + e  ->  A16[q][1 + seg*S + 1 + i] ----
     // All of a thread's loads are issued before the first store so that they overlap (a CTA stages at
-    // most nb * nblk * 8 <= 2048 vectors, i.e. 16 per thread).
+    // most nb * nblk * 8 <= 2048 vectors, i.e. 8 per thread).
     {
         const int nvec = nbh * vpr;
-        uint4 v[16];
-        int dst[16];
+        uint4 v[8];
+        int dst[8];
 #pragma unroll
-        for (int it = 0; it < 16; ++it) {
+        for (int it = 0; it < 8; ++it) {
             const int idx = tid + it * kThreads;
             dst[it] = -1;
             if (idx < nvec) {
@@ -104,7 +104,7 @@ dw_tc_kernel(const TI* __restrict__ in, const TW* __restrict__ w, TO* __restrict
             }
         }
 #pragma unroll
-        for (int it = 0; it < 16; ++it) {
+        for (int it = 0; it < 8; ++it) {
             if (dst[it] < 0) continue;
             const int keep = dst[it] >> 20;
             if (keep) {
@@ -153,8 +153,9 @@ dw_tc_kernel(const TI* __restrict__ in, const TW* __restrict__ w, TO* __restrict
     ptx::tc_fence_after();
     if (ok) {
         const float inv = gmax ? 1.f / pow2_scale(*gmax) : 1.f;
-        for (int mt = 0; mt < nmt; ++mt) {
-            const int Rw = mt * 128 + warp * 32 + lane;
+        const int mt = warp >> 2, wq = warp & 3;          // this warp's M-tile and TMEM lane quarter
+        if (mt < nmt) {
+            const int Rw = mt * 128 + wq * 32 + lane;
             const int seg = Rw / S, sr = Rw - seg * S;
             const bool live = (Rw < rows) && sr >= 1 && sr <= nblk;
             const int b = b0 + seg;
@@ -163,7 +164,7 @@ dw_tc_kernel(const TI* __restrict__ in, const TW* __restrict__ w, TO* __restrict
 #pragma unroll 1
             for (int h = 0; h < 2; ++h) {
                 uint32_t r[32];
-                ptx::tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + mt * NB + 32 * h, r);
+                ptx::tmem_ld32(tmem + ((uint32_t)(wq * 32) << 16) + mt * NB + 32 * h, r);
                 ptx::tmem_ld_wait();
                 if (!live) continue;
 #pragma unroll
