@@ -47,28 +47,6 @@ template <typename T> struct Fmt;
 template <> struct Fmt<__half> { static constexpr uint32_t v = 0; };
 template <> struct Fmt<__nv_bfloat16> { static constexpr uint32_t v = 1; };
 
-__device__ __forceinline__ void store32(float* dst, const float (&f)[32]) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-        reinterpret_cast<float4*>(dst)[i] = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
-}
-template <typename T>
-__device__ __forceinline__ void store32(T* dst, const float (&f)[32]) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        float g[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) g[j] = f[8 * i + j];
-        st8<T>(dst + 8 * i, g);
-    }
-}
-
-template <typename OT>
-__device__ __forceinline__ void store_row_chunk(OT* row, int col0, int ncols_total, const float (&f)[32]) {
-    if (col0 + 32 <= ncols_total) { store32(row + col0, f); return; }
-    for (int i = 0; i < 32; ++i) if (col0 + i < ncols_total) stf(row + col0 + i, f[i]);
-}
-
 // Coalesced store of a warp's 32 x 32 accumulator block.  After tcgen05.ld lane l holds 32 consecutive
 // columns of row l; storing that directly makes every store instruction touch 32 different rows with
 // 16 bytes each (half-filled sectors).  The block is transposed through a per-warp shared-memory
@@ -308,15 +286,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
 }
 
 // ---- persistent, warp-specialised form for the forward and input-gradient contractions -----------
-// One CTA per SM loops over output tiles (tile = blockIdx.x + i * gridDim.x).  Warps 0-3 are the
-// epilogue (warp w owns TMEM lanes 32w..32w+31), warp 4 is the TMA producer, warp 5 issues the MMAs.
+// One CTA per SM loops over output tiles (tile = blockIdx.x + i * gridDim.x).  The first 4*MT warps are
+// the epilogue (warp e reads M-sub-tile e/4, TMEM lanes 32(e%4)..+31), the next warp is the TMA
+// producer, the last one issues the MMAs.
 // The accumulator is double-buffered in tensor memory, so the epilogue of tile i (TMEM -> registers ->
 // statistics -> global stores) overlaps the loads and MMAs of tile i+1; the shared-memory ring keeps
 // running across tile boundaries.  Barrier set-up and the TMEM allocation are paid once per CTA.
-constexpr int kPThreads = 192;
 
 template <typename T, int MODE, int MT, int BN, int STAGES>
-__global__ void __launch_bounds__(kPThreads, 1)
+__global__ void __launch_bounds__(32 * (4 * MT + 2), 1)
 tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                           TcParams p, int tiles_n, int tiles_m, int tiles_total) {
     static_assert(MODE == MODE_FWD || MODE == MODE_DGRAD, "forward / input gradient only");
@@ -340,7 +318,7 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap mapA, const __grid
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
-        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 128); }
+        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 128 * MT); }
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&mapA);
         ptx::prefetch_tensormap(&mapB);
@@ -360,7 +338,7 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap mapA, const __grid
         return n0 < len;
     };
 
-    if (warp == 4) {
+    if (warp == 4 * MT) {
         if (lane == 0) {                              // ---- TMA producer ----
             int it = 0;
             bool dead = false;
@@ -390,7 +368,7 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap mapA, const __grid
             }
         }
         __syncwarp();
-    } else if (warp == 5) {
+    } else if (warp == 4 * MT + 1) {
         if (lane == 0) {                              // ---- MMA issuer ----
             int it = 0, j = 0;
             bool dead = false;
@@ -422,7 +400,8 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap mapA, const __grid
             }
         }
         __syncwarp();
-    } else {                                          // ---- epilogue warps 0..3 ----
+    } else {                                          // ---- epilogue warps ----
+        const int mt = warp >> 2, wq = warp & 3;
         int j = 0;
         for (int tile = blockIdx.x; tile < tiles_total; tile += gridDim.x) {
             int n0, m0, z, len;
@@ -430,7 +409,7 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap mapA, const __grid
                 if (p.zero_fill) {
                     const int esz = (MODE == MODE_FWD && p.out_f32) ? 4 : (int)sizeof(T);
                     const int vec_per_row = BN * esz / 16;
-                    for (int i = tid; i < 128 * MT * vec_per_row; i += 128) {
+                    for (int i = tid; i < 128 * MT * vec_per_row; i += 128 * MT) {
                         const int r = m0 + i / vec_per_row, cb = (i % vec_per_row) * (16 / esz);
                         if (r < p.M && n0 + cb < p.Ncols) {
                             uint8_t* dst = reinterpret_cast<uint8_t*>(p.out) + (((size_t)z * p.M + r) * p.Ncols + n0 + cb) * esz;
@@ -445,9 +424,8 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap mapA, const __grid
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) { if (lane == 0) raise_status(p.status, kErrTimeout); break; }
             ptx::tc_fence_after();
-#pragma unroll 1
-            for (int mt = 0; mt < MT; ++mt) {
-                const int row = m0 + mt * 128 + warp * 32 + lane;
+            {
+                const int row = m0 + mt * 128 + wq * 32 + lane;
                 float sn = 0.f, smean = 0.f, sm2 = 0.f;
                 const float bias = (MODE == MODE_FWD && p.bias && row < p.M) ? p.bias[row] : 0.f;
 #pragma unroll 1
@@ -456,7 +434,7 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap mapA, const __grid
                     float f[32];
                     {
                         uint32_t r[32];
-                        ptx::tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + buf * ACC_COLS + mt * BN + c0, r);
+                        ptx::tmem_ld32(tmem + ((uint32_t)(wq * 32) << 16) + buf * ACC_COLS + mt * BN + c0, r);
                         ptx::tmem_ld_wait();
 #pragma unroll
                         for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(r[i]) + bias;
@@ -477,7 +455,7 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap mapA, const __grid
                         for (int i = 0; i < 32; ++i) if (i >= nv) f[i] = 0.f;
                     }
                     {
-                        const int row_w = m0 + mt * 128 + warp * 32;
+                        const int row_w = m0 + mt * 128 + wq * 32;
                         const size_t base = ((size_t)z * p.M + row_w) * p.Ncols + n0 + c0;
                         float* stg = stg_all + warp * kStgFloatsPerWarp;
                         const int rl = p.M - row_w, cl = p.Ncols - (n0 + c0);
@@ -544,7 +522,7 @@ void launch_dt(int dtype, const Launch& L, dim3 grid, const CUtensorMap& a, cons
 template <typename T, int MODE, int MT, int BN, int STAGES>
 void launch_persistent(const Launch& L, int sm_count, const CUtensorMap& a, const CUtensorMap& b, const TcParams& p,
                        int tiles_n, int tiles_m, int batch) {
-    constexpr int smem = STAGES * (MT * 16384 + BN * 128) + 1024 + 256 + 4 * kStgFloatsPerWarp * 4;
+    constexpr int smem = STAGES * (MT * 16384 + BN * 128) + 1024 + 256 + 4 * MT * kStgFloatsPerWarp * 4;
     static bool configured = false;
     auto kern = tc_gemm_persistent_kernel<T, MODE, MT, BN, STAGES>;
     if (!configured) {
@@ -552,7 +530,7 @@ void launch_persistent(const Launch& L, int sm_count, const CUtensorMap& a, cons
         configured = true;
     }
     const int total = tiles_n * tiles_m * batch;
-    kern<<<std::min(sm_count, total), kPThreads, smem, L.stream>>>(a, b, p, tiles_n, tiles_m, total);
+    kern<<<std::min(sm_count, total), 32 * (4 * MT + 2), smem, L.stream>>>(a, b, p, tiles_n, tiles_m, total);
     L.count();
 }
 template <int MODE, int MT, int BN, int STAGES>
@@ -629,7 +607,7 @@ bool tc_gemm_fwd(const TcState* st, const Launch& L, int dtype, const void* w, c
     const int mt = Cout > 128 ? 2 : 1;
     dim3 grid((Tp + FWD_BN - 1) / FWD_BN, (Cout + 128 * mt - 1) / (128 * mt), B);
     if (st->persistent) {
-        if (mt == 2) launch_persistent_dt<MODE_FWD, 2, FWD_BN, 4>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
+        if (mt == 2) launch_persistent_dt<MODE_FWD, 2, FWD_BN, 3>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
         else launch_persistent_dt<MODE_FWD, 1, FWD_BN, 6>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
     } else if (mt == 2) launch_dt<MODE_FWD, 2, FWD_BN, 2>(dtype, L, grid, ma, mb, p);
     else launch_dt<MODE_FWD, 1, FWD_BN, 3>(dtype, L, grid, ma, mb, p);
@@ -652,7 +630,7 @@ void tc_gemm_dgrad(const TcState* st, const Launch& L, int dtype, const void* w,
     const int mt = Cin > 128 ? 2 : 1;
     dim3 grid((Tp + FWD_BN - 1) / FWD_BN, (Cin + 128 * mt - 1) / (128 * mt), B);
     if (st->persistent) {
-        if (mt == 2) launch_persistent_dt<MODE_DGRAD, 2, FWD_BN, 4>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
+        if (mt == 2) launch_persistent_dt<MODE_DGRAD, 2, FWD_BN, 3>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
         else launch_persistent_dt<MODE_DGRAD, 1, FWD_BN, 6>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
     } else if (mt == 2) launch_dt<MODE_DGRAD, 2, FWD_BN, 2>(dtype, L, grid, ma, mb, p);
     else launch_dt<MODE_DGRAD, 1, FWD_BN, 3>(dtype, L, grid, ma, mb, p);
