@@ -442,14 +442,16 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap mapA, const __grid
                     if (MODE == MODE_FWD) {
                         const int nv = max(0, min(32, len - (n0 + c0)));
                         if (p.stats && nv > 0) {
-                            float s = 0.f;
+                            // sums about a pivot taken from the row itself (its first frame in this tile):
+                            // one pass, and no cancellation beyond the spread of the data
+                            if (c0 == 0) smean = f[0];
+                            if (nv == 32) {
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) if (i < nv) s += f[i];
-                            const float cm = s / (float)nv;
-                            float q = 0.f;
+                                for (int i = 0; i < 32; ++i) { const float d = f[i] - smean; sn += d; sm2 = fmaf(d, d, sm2); }
+                            } else {
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) if (i < nv) { const float d = f[i] - cm; q = fmaf(d, d, q); }
-                            chan_merge(sn, smean, sm2, (float)nv, cm, q);
+                                for (int i = 0; i < 32; ++i) if (i < nv) { const float d = f[i] - smean; sn += d; sm2 = fmaf(d, d, sm2); }
+                            }
                         }
 #pragma unroll
                         for (int i = 0; i < 32; ++i) if (i >= nv) f[i] = 0.f;
@@ -465,8 +467,12 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap mapA, const __grid
                             store_block_staged<T>(stg, f, reinterpret_cast<T*>(p.out) + base, p.Ncols, rl, cl, lane);
                     }
                 }
-                if (MODE == MODE_FWD && p.stats && row < p.M)
-                    p.stats[((size_t)z * tiles_n + (n0 / BN)) * p.M + row] = make_float2(smean * sn, sm2);
+                if (MODE == MODE_FWD && p.stats && row < p.M) {
+                    // (sum, M2 about the tile mean) from the pivot-shifted sums; cnt = valid frames of this tile
+                    const float cnt = (float)max(1, min(BN, len - n0));
+                    p.stats[((size_t)z * tiles_n + (n0 / BN)) * p.M + row] =
+                        make_float2(fmaf(smean, cnt, sn), sm2 - sn * sn / cnt);
+                }
             }
             ptx::tc_fence_before();
             ptx::mbar_arrive(&acc_empty[buf]);        // this thread is done reading the accumulator
