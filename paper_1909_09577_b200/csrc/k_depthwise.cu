@@ -508,6 +508,14 @@ dw_wgrad_reg16_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float*
     float acc[8 * NCH];
 #pragma unroll
     for (int i = 0; i < 8 * NCH; ++i) acc[i] = 0.f;
+    // lengths of this CTA's rows, read once (NR * NST <= 32 rows)
+    __shared__ int s_li[32], s_lo[32];
+    if (tid < NR * NST) {
+        const int b = blockIdx.y * NST * NR + tid;
+        s_li[tid] = b < B ? min(len_in[b], Tt) : 0;
+        s_lo[tid] = b < B ? min(len_out[b], Tt) : 0;
+    }
+    __syncthreads();
 
     auto issue = [&](int st) {
         const int b0 = (blockIdx.y * NST + st) * NR;
@@ -521,7 +529,7 @@ dw_wgrad_reg16_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float*
         for (int i = tid; i < nr * cpr; i += WR_THREADS) {
             const int r = i / cpr, t = (i - r * cpr) * 8;
             const int b = b0 + r;
-            const int li = min(len_in[b], Tt), lo = min(len_out[b], Tt);
+            const int li = s_li[st * NR + r], lo = s_lo[st * NR + r];
             const size_t off = ((size_t)b * C + c) * Tt + t;
             unsigned short* gd = gs + r * RS + t;
             unsigned short* xd = xs + r * RS + t + Ppad;
@@ -539,7 +547,7 @@ dw_wgrad_reg16_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float*
         unsigned short* xs = gs + (size_t)NR * RS;
         for (int i = tid; i < nr * cpr; i += WR_THREADS) {
             const int r = i / cpr, t = (i - r * cpr) * 8;
-            const int li = min(len_in[b0 + r], Tt), lo = min(len_out[b0 + r], Tt);
+            const int li = s_li[st * NR + r], lo = s_lo[st * NR + r];
             if (t < lo && t + 8 > lo) for (int e = lo - t; e < 8; ++e) gs[r * RS + t + e] = 0;
             if (t < li && t + 8 > li) for (int e = li - t; e < 8; ++e) xs[r * RS + t + Ppad + e] = 0;
         }
@@ -673,7 +681,7 @@ void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x
     if (s == 1 && Tt % 8 == 0 && nch >= 2 && nch <= 12) {
         // rows staged per pass: the count whose (rows x chunks) best fills the 128 threads
         const int cpr = Tt / 8;
-        const int NST = 2;
+        const int NST = (dtype == F32) ? 2 : 4;
         if (dtype == F32) {
             const int rs = host_phys(Tt + 8 * nch + 8) + 4, rsp = (rs + 3) / 4 * 4;
             int NR = 1; double best = 0.0;
