@@ -565,6 +565,7 @@ dw_wgrad_reg16_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float*
         const unsigned short* xs = gs + (size_t)NR * RS;
         for (int i = tid; i < nr * cpr; i += WR_THREADS) {
             const int r = i / cpr, t = (i - r * cpr) * 8;
+            if (t >= s_lo[st * NR + r]) continue;          // gradient is zero in padding: nothing to add
             const unsigned short* xp = xs + r * RS + t;
             float g[8], win[16];
             cvt8<TG>(*reinterpret_cast<const uint4*>(gs + r * RS + t), g);

@@ -176,7 +176,7 @@ def run_block(ctx, api, L, dtype, x, lengths, params, g, x_res=None, want_dx_res
     return rep
 
 
-def run_chain(ctx, api, w, d, check=True):
+def run_chain(ctx, api, w, d, check=True, oracle_layers=None):
     """Teacher-forced chain: every layer runs through sepconv_fwd / sepconv_bwd on the GPU's own
     previous output, and the oracle evaluates the same layer on the same (stored) input.  Returns
     (per-layer reports, dict of final GPU tensors)."""
@@ -207,6 +207,18 @@ def run_chain(ctx, api, w, d, check=True):
         L = layers[i]
         f = fwd[i]
         x_res_np = acts[f["j"]] if f["xr"] is not None else None
+        if oracle_layers is not None and i not in oracle_layers:
+            # GPU only: keeps the gradient flowing without the (slow) oracle evaluation of this layer
+            want_res = f["xr"] is not None
+            dx_add = pending.pop(i, None)
+            dx, dx_res, grads = api.sepconv_bwd(ctx, f["desc"], dev(g, w.dtype), f["xd"], f["y"], f["ld"], f["pd"],
+                                                f["saved"], x_res=f["xr"], dx_add=dx_add, want_dx_res=want_res)
+            if want_res:
+                pending[f["j"]] = dx_res
+            grads_all[i] = grads
+            g = dx.float().cpu().numpy()
+            final_dx = dx
+            continue
         S = O.block_fwd(L, acts[i], lens[i], d.params[i], res_src=x_res_np)
         rep = Report(w.dtype)
         np.testing.assert_array_equal(lens[i + 1], S["out_len"])

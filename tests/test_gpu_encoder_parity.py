@@ -119,3 +119,32 @@ def test_config4_encoder_layers_teacher_forced(api, ctx):
     assert sum(r.hard for r in reports) == 0
     for r in reports:
         r.check()
+
+
+def test_config5_ragged_encoder_full_size(api, ctx):
+    """Config 5 at full size (B=64, T=3200, ragged).  The oracle needs minutes per layer at this size, so
+    it checks a sample of layers teacher-forced (the stride-2 first layer, one 256-wide and one 512-wide
+    sub-block with a block residual, and the logits layer); every layer is covered by properties that
+    hold at any size: the one-call encoder equals the chain of block calls bit for bit, padded frames
+    are zero, and the returned lengths are ceil(len/2)."""
+    w = si.config(5)
+    d = si.draw(w)
+    sample = {0, 10, 20, 28}
+    reports, chain = U.run_chain(ctx, api, w, d, check=False, oracle_layers=sample)
+    _summarise([r for r in reports if r is not None], "gpurun_out/parity_cfg5_sampled_layers.txt",
+               f"config 5, layers {sorted(sample)}")
+    spec, logits, out_len, gblob, dx = run_encoder(ctx, api, w, d)
+    assert torch.equal(logits, chain["logits"]) and torch.equal(dx, chain["dx"])
+    for i in range(len(w.layers)):
+        for name in d.params[i]:
+            assert torch.equal(spec.grad_view(gblob, i, name), chain["grads"][i]["d" + name]), (i, name)
+    np.testing.assert_array_equal(out_len.cpu().numpy(), (d.lengths + 1) // 2)
+    t = torch.arange(logits.shape[2], device="cuda")[None, None, :]
+    pad = t >= out_len.cuda()[:, None, None]
+    assert torch.all(logits.masked_select(pad.expand_as(logits)) == 0)
+    tin = torch.arange(dx.shape[2], device="cuda")[None, None, :]
+    pad_in = tin >= torch.from_numpy(d.lengths).cuda()[:, None, None]
+    assert torch.all(dx.masked_select(pad_in.expand_as(dx)) == 0)
+    for i in sample:
+        assert reports[i].hard == 0
+        reports[i].check()
