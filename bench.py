@@ -93,6 +93,22 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def max_over_ranks(ms, device=None):
+    """Slowest rank's time (every rank gets it); a no-op outside a process group."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(frames_per_rank_step, steps, ms_max, world):
+    """Whole-job frames per second: every rank ran `steps` independent replicas' steps in ms_max."""
+    return world * frames_per_rank_step * steps / (ms_max * 1e-3)
+
+
 def oracle_sample(w, B_sample, repeats=1):
     """Times the fp64 oracle (as it stands) on a B_sample-sample slice of the workload.
     Returns (frames per second, threads used, description)."""
@@ -222,11 +238,7 @@ def main():
         e1.record(stream)
         barrier()
         t1 = time.time()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(e0.elapsed_time(e1), dev)
         return ms, t0, t1
 
     for _ in range(args.warmup):
@@ -301,8 +313,8 @@ def main():
         return
     frames = w.B * w.T
     peaks = measured_peaks()
-    value = world * frames * args.steps / (ms * 1e-3)
-    e2e = world * frames * args.steps / (ms_e2e * 1e-3)
+    value = job_throughput(frames, args.steps, ms, world)
+    e2e = job_throughput(frames, args.steps, ms_e2e, world)
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
