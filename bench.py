@@ -30,6 +30,9 @@ METRIC = "encoder fwd+bwd audio frames/sec"
 UNIT = "frames/s"
 # The kernel class that takes the largest share of the step (see profiles/); its roofline is reported.
 DOMINANT_CLASS = "dw_wgrad"
+# measured DRAM bytes / algorithmic bytes of that class's kernel (profiles/block512_dram_traffic.txt:
+# dw_wgrad_reg16_kernel read 52.5 MB for 52.4 MB of operands); scales with the elements processed
+TRAFFIC_RATIO = {"dw_wgrad": 52.5 / 52.4}
 
 
 def measured_peaks():
@@ -333,7 +336,9 @@ def main():
         alu_peak = 148 * 128 * 1.965e9 / 1e12     # T FMA/s: SMs x fp32 lanes x max clock
         if args.profile_class.startswith("dw_"):
             line["roofline"] = {"kernel": args.profile_class, "bound": "alu", "achieved": tfs / 2, "peak": alu_peak,
-                                "unit": "TFMA/s", "frac": tfs / 2 / alu_peak, "traffic": None,
+                                "unit": "TFMA/s", "frac": tfs / 2 / alu_peak,
+                                "traffic": (TRAFFIC_RATIO[args.profile_class] * pc["bytes"] / pc["launches"]
+                                            if args.profile_class in TRAFFIC_RATIO else None),
                                 "hbm_gbs": gbs, "hbm_frac": gbs / peaks["hbm_gbs"], "peak_source": "derived: 148 SMs x 128 lanes x 1.965 GHz",
                                 "launches": pc["launches"], "avg_ms": per_ms}
         elif args.profile_class.startswith("pw_") and args.gemm_mode == 0 and tfs > 0.2 * peaks["hbm_gbs"] * 1e-3 * 212:
