@@ -492,7 +492,7 @@ template <> __device__ __forceinline__ void cvt8<__nv_bfloat16>(const uint4& r, 
 }
 
 template <typename TG, typename T, int NCH>
-__global__ void __launch_bounds__(WR_THREADS, 3)
+__global__ void __launch_bounds__(WR_THREADS, (NCH <= 8 ? 4 : 3))
 dw_wgrad_reg16_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float* __restrict__ partials,
                       const int* __restrict__ len_in, const int* __restrict__ len_out,
                       int B, int C, int Tt, int K, int Ppad, int NR, int NST, int RS) {
@@ -563,8 +563,9 @@ dw_wgrad_reg16_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float*
         const int nr = min(NR, B - b0);
         const unsigned short* gs = smem16 + (st & 1) * bufsz;
         const unsigned short* xs = gs + (size_t)NR * RS;
-        for (int i = tid; i < nr * cpr; i += WR_THREADS) {
-            const int r = i / cpr, t = (i - r * cpr) * 8;
+        int r = tid / cpr, t = (tid - r * cpr) * 8;          // chunk index -> (row, frame), then stepped without divisions
+        for (int i = tid; i < nr * cpr; i += WR_THREADS, t += WR_THREADS * 8) {
+            while (t >= Tt) { t -= Tt; ++r; }
             if (t >= s_lo[st * NR + r]) continue;          // gradient is zero in padding: nothing to add
             const unsigned short* xp = xs + r * RS + t;
             float g[8], win[16];
@@ -592,10 +593,29 @@ dw_wgrad_reg16_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float*
         __syncthreads();
     }
     float* red = reinterpret_cast<float*>(smem16);       // [4][8*NCH]
+    {
+        // Warp reduction that halves the number of live values at every step: lane pairs (l, l^s) split the
+        // values between them, each keeps one half and adds the partner's copy of it.  VP/32 sums per lane
+        // remain after five steps (VP - VP/32 shuffles instead of 5 VP); the pairing is fixed, so is the order.
+        constexpr int VP = (8 * NCH + 31) / 32 * 32;
+        float v[VP];
 #pragma unroll
-    for (int i = 0; i < 8 * NCH; ++i) {
-        const float v = warp_sum(acc[i]);
-        if (lane == 0) red[wrp * 8 * NCH + i] = v;
+        for (int i = 0; i < VP; ++i) v[i] = i < 8 * NCH ? acc[i] : 0.f;
+        int base = 0;
+#pragma unroll
+        for (int sstep = 16, n = VP / 2; sstep >= 1; sstep >>= 1, n >>= 1) {
+            const bool up = (lane & sstep) != 0;
+#pragma unroll
+            for (int i = 0; i < n; ++i) {
+                const float lo = v[i], hi = v[i + n];
+                const float got = __shfl_xor_sync(0xffffffffu, up ? lo : hi, sstep);
+                v[i] = (up ? hi : lo) + got;
+            }
+            if (up) base += n;
+        }
+#pragma unroll
+        for (int i = 0; i < VP / 32; ++i)
+            if (base + i < 8 * NCH) red[wrp * 8 * NCH + base + i] = v[i];
     }
     __syncthreads();
     for (int k = tid; k < K; k += WR_THREADS) {
