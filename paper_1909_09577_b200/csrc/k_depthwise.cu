@@ -526,8 +526,9 @@ dw_wgrad_reg16_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float*
             const int r = i / halo, j = i - r * halo;
             xs[r * RS + (j < Ppad ? j : Tt + j)] = 0;
         }
-        for (int i = tid; i < nr * cpr; i += WR_THREADS) {
-            const int r = i / cpr, t = (i - r * cpr) * 8;
+        int r = tid / cpr, t = (tid - r * cpr) * 8;
+        for (int i = tid; i < nr * cpr; i += WR_THREADS, t += WR_THREADS * 8) {
+            while (t >= Tt) { t -= Tt; ++r; }
             const int b = b0 + r;
             const int li = s_li[st * NR + r], lo = s_lo[st * NR + r];
             const size_t off = ((size_t)b * C + c) * Tt + t;
@@ -545,11 +546,14 @@ dw_wgrad_reg16_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float*
         const int nr = min(NR, B - b0);
         unsigned short* gs = smem16 + (st & 1) * bufsz;
         unsigned short* xs = gs + (size_t)NR * RS;
-        for (int i = tid; i < nr * cpr; i += WR_THREADS) {
-            const int r = i / cpr, t = (i - r * cpr) * 8;
+        // the copies that can straddle a length were issued by thread (row*cpr + len/8) % 128: that thread waits
+        // for its own copies above, so it is the one that may overwrite the tail
+        for (int r = 0; r < nr; ++r) {
             const int li = s_li[st * NR + r], lo = s_lo[st * NR + r];
-            if (t < lo && t + 8 > lo) for (int e = lo - t; e < 8; ++e) gs[r * RS + t + e] = 0;
-            if (t < li && t + 8 > li) for (int e = li - t; e < 8; ++e) xs[r * RS + t + Ppad + e] = 0;
+            if ((lo & 7) && ((r * cpr + (lo >> 3)) % WR_THREADS) == tid)
+                for (int e = lo; e < ((lo + 7) & ~7); ++e) gs[r * RS + e] = 0;
+            if ((li & 7) && ((r * cpr + (li >> 3)) % WR_THREADS) == tid)
+                for (int e = li; e < ((li + 7) & ~7); ++e) xs[r * RS + Ppad + e] = 0;
         }
     };
 

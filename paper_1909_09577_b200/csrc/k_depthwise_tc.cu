@@ -89,12 +89,14 @@ dw_tc_kernel(const TI* __restrict__ in, const TW* __restrict__ w, TO* __restrict
         const int nvec = nbh * vpr;
         uint4 v[8];
         int dst[8];
+        int seg = tid / vpr, vq = tid - seg * vpr;          // vector index -> (sample, vector in row), stepped without divisions
 #pragma unroll
-        for (int it = 0; it < 8; ++it) {
+        for (int it = 0; it < 8; ++it, vq += kThreads) {
             const int idx = tid + it * kThreads;
+            while (vq >= vpr) { vq -= vpr; ++seg; }
             dst[it] = -1;
             if (idx < nvec) {
-                const int seg = idx / vpr, vq = idx - seg * vpr, t = vq * 8;
+                const int t = vq * 8;
                 const int ls = min(lens[seg], Tt);
                 if (t < ls) {
                     v[it] = *reinterpret_cast<const uint4*>(in + ((size_t)(b0 + seg) * C + c) * Tt + t);
