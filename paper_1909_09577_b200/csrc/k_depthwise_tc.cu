@@ -174,23 +174,37 @@ dw_tc_kernel(const TI* __restrict__ in, const TW* __restrict__ w, TO* __restrict
                     const int t = (sr - 1) * NB + 32 * h + 8 * g8;
                     if (t >= Tt) break;
                     float f[8];
+                    if (t >= ld) {                                   // whole vector in padding
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(r[8 * g8 + e]) * inv;
-                    if (t < ld) {
+                        for (int e = 0; e < 8; ++e) f[e] = 0.f;
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(r[8 * g8 + e]);
+                        if (gmax) {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) f[e] *= inv;
+                        }
                         if (add1) { float a[8]; ld8<TO>(add1 + rbase + t, a);
 #pragma unroll
                             for (int e = 0; e < 8; ++e) f[e] += a[e]; }
                         if (add2) { float a[8]; ld8<TO>(add2 + rbase + t, a);
 #pragma unroll
                             for (int e = 0; e < 8; ++e) f[e] += a[e]; }
-                    }
-                    bool over = false;
+                        if (t + 8 > ld) {                            // the length falls inside this vector
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        if (t + e >= ld) f[e] = 0.f;
-                        if (std::is_same<TO, __half>::value && fabsf(f[e]) > 65504.f) { f[e] = copysignf(65504.f, f[e]); over = true; }
+                            for (int e = 0; e < 8; ++e) if (t + e >= ld) f[e] = 0.f;
+                        }
+                        if (std::is_same<TO, __half>::value) {       // range guard: one max over the vector, clamp only if hit
+                            float m = 0.f;
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) m = fmaxf(m, fabsf(f[e]));
+                            if (m > 65504.f) {
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) f[e] = fminf(fmaxf(f[e], -65504.f), 65504.f);
+                                raise_status(status, kErrRange);
+                            }
+                        }
                     }
-                    if (over) raise_status(status, kErrRange);
                     st8<TO>(out + rbase + t, f);
                 }
             }
