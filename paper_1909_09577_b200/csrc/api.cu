@@ -287,7 +287,11 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
 
     if (d->has_dw) {
         pointwise_dgrad(ctx, L, odt, wp_op, s.gv, s.gu, m.B, m.Cin, m.Cout, m.Tp, io.len_out);
-        dw_wgrad(L, dt, odt, s.gu, io.x, g->dwd, s.wpart, acc, gmax, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s);
+        if (ctx->gemm_mode == 0 && dw_wgrad_tc_supported(&ctx->tc, dt, m.B, m.T, m.K, m.s))
+            dw_wgrad_tc(&ctx->tc, L, dt, odt, s.gu, io.x, g->dwd, s.wpart, acc, gmax, io.len_in, io.len_out, m.B, m.Cin,
+                        m.T, m.K, io.x_clean ? 1 : 0);
+        else
+            dw_wgrad(L, dt, odt, s.gu, io.x, g->dwd, s.wpart, acc, gmax, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s);
         if (io.dx)
             dw_dgrad(L, dt, odt, s.gu, p->wd, io.dx, io.dx_add, extra, gmax, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp,
                      m.K, m.s);

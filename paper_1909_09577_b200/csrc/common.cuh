@@ -52,6 +52,26 @@ template <> __device__ __forceinline__ float round_io<float>(float v) { return v
 template <> __device__ __forceinline__ float round_io<__half>(float v) { return __half2float(__float2half_rn(v)); }
 template <> __device__ __forceinline__ float round_io<__nv_bfloat16>(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 
+// Rounds the first n of 8 consecutive values to the storage type with error diffusion: the rounding
+// residual of one element is added to the next before it is rounded, so the residuals of a vector do
+// not add up.  Plain rounding is biased whenever the values sit on a lattice that the storage grid
+// resolves only up to a constant offset (a 16-bit gradient times a short binary fraction, minus a
+// per-channel constant); a bias of a fraction of a unit in the last place per element, summed over
+// every frame of a channel by the weight-gradient contraction, would dominate that gradient's error.
+template <typename ST> __device__ __forceinline__ void diffuse8(float (&v)[8], int n) {
+    if (sizeof(ST) == 4) return;
+    float r = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        if (i < n) {
+            const float t = v[i] + r;
+            const float q = round_io<ST>(t);
+            r = t - q;
+            v[i] = q;
+        }
+    }
+}
+
 // 8 consecutive elements <-> 8 floats.  Pointers must be aligned to 8 elements.
 template <typename T> __device__ __forceinline__ void ld8(const T* p, float (&f)[8]);
 template <> __device__ __forceinline__ void ld8<float>(const float* p, float (&f)[8]) {

@@ -386,6 +386,8 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_apply_kernel(BnBwdArgs a) 
                 if (a.residual == 2) o2[i] = in ? cr.x * (gr[i] - cr.y - vhr[i] * cr.z) : 0.f;
                 else o2[i] = gr[i];
             }
+            diffuse8<GT>(o1, R.len - t0);
+            if (a.residual == 2) diffuse8<T>(o2, R.len - t0);
         } else {
 #pragma unroll
             for (int i = 0; i < 8; ++i) { o1[i] = 0.f; o2[i] = 0.f; }
@@ -461,6 +463,8 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_fast_kernel(BnBwdArgs a, int
             if (RES == 2) o2[i] = in ? cr.x * (ga - cr.y - vnr[i] * cr.z) : 0.f;
             if (RES == 1) o2[i] = ga;
         }
+        diffuse8<GT>(o1, len - t0);
+        if (RES == 2) diffuse8<T>(o2, len - t0);
     } else {
 #pragma unroll
         for (int i = 0; i < 8; ++i) { o1[i] = 0.f; o2[i] = 0.f; }

@@ -68,6 +68,13 @@ void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x
               int accumulate, const float* gmax, const int* len_in, const int* len_out, int B, int C, int T,
               int Tp, int K, int s);
 size_t dw_wgrad_scratch_bytes(int B, int C, int K);
+// Tensor-core form of the stride-1 tap gradient (16-bit types, B >= 16, K <= 127): same result as dw_wgrad.
+// x_clean != 0 promises that x is already zero at and beyond len_in.  partials: float [8*C*K] at least.
+struct TcState;
+bool dw_wgrad_tc_supported(const TcState* st, int dtype, int B, int T, int K, int s);
+void dw_wgrad_tc(const TcState* st, const Launch& L, int dtype, int odt, const void* gu, const void* x, float* dwd,
+                 float* partials, int accumulate, const float* gmax, const int* len_in, const int* len_out, int B,
+                 int C, int T, int K, int x_clean);
 // Tensor-core forms of the stride-1 depthwise forward / input gradient (16-bit types, K <= 129).
 bool dw_tc_supported(int dtype, int T, int K, int s);
 void dw_tc_fwd(const Launch& L, int dtype, int odt, const void* x, const void* wd, void* u, const int* len_in,

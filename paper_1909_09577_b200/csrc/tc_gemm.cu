@@ -489,8 +489,11 @@ using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, voi
                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-bool make_map(const TcState* st, CUtensorMap* m, int dtype, const void* base, int rank, const uint64_t* dims,
-              const uint32_t* box) {
+}  // namespace
+
+bool tc_make_map(const TcState* st, void* map_out, int dtype, const void* base, int rank, const uint64_t* dims,
+                 const uint32_t* box) {
+    CUtensorMap* m = static_cast<CUtensorMap*>(map_out);
     cuuint64_t gdim[3]; cuuint64_t gstride[2]; cuuint32_t bdim[3]; cuuint32_t estr[3] = {1, 1, 1};
     uint64_t stride = 2;
     for (int i = 0; i < rank; ++i) {
@@ -504,6 +507,12 @@ bool make_map(const TcState* st, CUtensorMap* m, int dtype, const void* base, in
         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { fprintf(stderr, "sepconv: cuTensorMapEncodeTiled failed (%d)\n", (int)r); return false; }
     return true;
+}
+
+namespace {
+bool make_map(const TcState* st, CUtensorMap* m, int dtype, const void* base, int rank, const uint64_t* dims,
+              const uint32_t* box) {
+    return tc_make_map(st, m, dtype, base, rank, dims, box);
 }
 
 template <typename T, int MODE, int MT, int BN, int STAGES>

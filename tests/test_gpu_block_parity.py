@@ -72,6 +72,12 @@ TC_SHAPES = [
     (dict(C_in=1024, C_out=29, K=1, has_dw=False, has_bn=False, has_relu=False, has_bias=True), 3, 200, True),
     (dict(C_in=512, C_out=1024, K=1, has_dw=False), 2, 264, True),
     (dict(C_in=72, C_out=136, K=3, residual="proj"), 5, 64, False),
+    # tensor-core tap gradient: sample chunks with a ragged tail, T' that is no multiple of 128, wide halos,
+    # more (channel, split) units than SMs
+    (dict(C_in=24, C_out=16, K=87, residual="none"), 20, 328, True),
+    (dict(C_in=16, C_out=24, K=121, residual="proj"), 40, 136, True),
+    (dict(C_in=160, C_out=8, K=39, residual="none"), 33, 1000, True),
+    (dict(C_in=8, C_out=8, K=5, residual="identity"), 16, 128, False),
 ]
 
 
