@@ -12,9 +12,10 @@
 // frames outside [0,T) are zero-filled by the TMA unit (the "same" padding).  One elected thread issues
 // tcgen05.mma into a 128 x N fp32 accumulator in tensor memory; the accumulator is double-buffered so
 // that the diagonal sums of one (channel, split) unit overlap the loads and MMAs of the next.
-// Roles: warps 0-3 epilogue (TMEM -> shared memory -> diagonal sums), warps 4-7 operand preparation
-// (x is converted to the type of gu and masked by the sample length, in place), warp 8 TMA producer,
-// warp 9 MMA issuer.  Every wait is bounded; on expiry the CTA raises the status word and leaves.
+// Roles: warps 0-3 epilogue (TMEM -> shared memory -> diagonal sums), warps 4-11 operand preparation
+// (x is converted to the type of gu and masked by the sample length, in place; two groups of four warps
+// take alternate steps), warp 12 TMA producer (one box per lane: issuing a TMA copy costs a thread
+// about a hundred cycles, so the boxes of a step are issued side by side), warp 13 MMA issuer.  Every wait is bounded; on expiry the CTA raises the status word and leaves.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
@@ -32,10 +33,12 @@ namespace {
 
 constexpr int WT_STAGES = 6;
 constexpr int WT_STAGE_BYTES = 24576;      // 128 frames of gu + up to 256 frames of x, 32 samples, 16-bit
-constexpr int WT_THREADS = 320;
+constexpr int WT_THREADS = 448;
 constexpr int WT_ACC_COLS = 256;
 constexpr int WT_MAX_CHUNKS = 64;
-constexpr int WT_STG_PITCH = 33;
+constexpr int WT_STG_PITCH = 36;                     // floats per staging row
+constexpr int WT_STG_FLOATS = 63 * WT_STG_PITCH;     // per epilogue warp
+constexpr int WT_XW = 128;
 
 struct WtParams {
     float* partials; const int* len_in; const int* len_out; int* status;
@@ -54,42 +57,58 @@ template <typename T> struct FmtW;
 template <> struct FmtW<__half> { static constexpr uint32_t v = 0; };
 template <> struct FmtW<__nv_bfloat16> { static constexpr uint32_t v = 1; };
 
-// One 16-byte vector (8 frames) of x: convert TX -> TG, zero frames at or beyond `nvalid`.
+// One 16-byte vector (8 frames) of x: convert TX -> TG and zero the frames at or beyond `nvalid`.
+// amax collects the largest magnitude seen (a bf16 value of 2^16 or more has no half counterpart).
 template <typename TG, typename TX>
-__device__ __forceinline__ uint4 prep8(uint4 raw, int nvalid, bool& over) {
-    float f[8];
-    if (std::is_same<TX, __half>::value) {
-        const __half2* h = reinterpret_cast<const __half2*>(&raw);
+__device__ __forceinline__ uint4 prep8(uint4 raw, int nvalid, float& amax) {
+    uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+    if (!std::is_same<TG, TX>::value) {
+        // bf16 -> half through fp32: a bf16 is the upper half of the float with the same value
 #pragma unroll
-        for (int i = 0; i < 4; ++i) { float2 q = __half22float2(h[i]); f[2 * i] = q.x; f[2 * i + 1] = q.y; }
-    } else {
-        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { float2 q = __bfloat1622float2(h[i]); f[2 * i] = q.x; f[2 * i + 1] = q.y; }
-    }
-#pragma unroll
-    for (int i = 0; i < 8; ++i) if (i >= nvalid) f[i] = 0.f;
-    uint4 r;
-    if (std::is_same<TG, __half>::value) {
-        if (!std::is_same<TX, __half>::value) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                if (fabsf(f[i]) > 65504.f) { f[i] = copysignf(65504.f, f[i]); over = true; }
+        for (int i = 0; i < 4; ++i) {
+            const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+            amax = fmaxf(amax, fmaxf(fabsf(lo), fabsf(hi)));
+            const __half2 h = __floats2half2_rn(lo, hi);
+            w[i] = *reinterpret_cast<const uint32_t*>(&h);
         }
-        __half2* h = reinterpret_cast<__half2*>(&r);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) h[i] = __floats2half2_rn(f[2 * i], f[2 * i + 1]);
-    } else {
-        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&r);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
     }
-    return r;
+    if (nvalid < 8) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (2 * i >= nvalid) w[i] = 0u;
+            else if (2 * i + 1 >= nvalid) w[i] &= 0x0000FFFFu;
+        }
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
 __device__ __forceinline__ void bar_sync_named(int id, int nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
+
+// Walks the contraction steps of one unit: (chunk, tb) advance without divisions; a step is skipped when
+// its time block lies past every sample of its chunk (never the unit's first step, so that an
+// accumulator is always written).  Every role walks the same sequence.
+struct StepWalk {
+    int ks, ks0, ks1, chunk, tb, ntb, cl;
+    const int* chunk_len;
+    __device__ __forceinline__ void begin(int sp, int ks_per_split, int ks_total, int ntb_, const int* cl_) {
+        ks0 = sp * ks_per_split; ks1 = min(ks0 + ks_per_split, ks_total); ks = ks0; ntb = ntb_; chunk_len = cl_;
+        chunk = ks0 / ntb; tb = ks0 - chunk * ntb;
+        cl = chunk < WT_MAX_CHUNKS ? chunk_len[chunk] : (1 << 30);
+    }
+    __device__ __forceinline__ bool more() const { return ks < ks1; }
+    __device__ __forceinline__ bool on() const { return ks == ks0 || tb * 128 < cl; }
+    __device__ __forceinline__ void next() {
+        ++ks;
+        if (++tb == ntb) { tb = 0; ++chunk; cl = chunk < WT_MAX_CHUNKS ? chunk_len[chunk] : (1 << 30); }
+    }
+};
+// ring position: stage index and phase parity, advanced without a modulo
+struct Ring {
+    int s = 0, ph = 0;
+    __device__ __forceinline__ void advance() { if (++s == WT_STAGES) { s = 0; ph ^= 1; } }
+};
 
 template <typename TG, typename TX>
 __global__ void __launch_bounds__(WT_THREADS, 1)
@@ -103,9 +122,10 @@ dw_wgrad_tc_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_consta
     uint64_t* acc_empty = acc_full + 2;        // [2]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     int* chunk_len = reinterpret_cast<int*>(tmem_slot + 2);                 // [WT_MAX_CHUNKS]
-    float* stg_all = reinterpret_cast<float*>(chunk_len + WT_MAX_CHUNKS);   // [4][32][33]
-    float* xw = stg_all + 4 * 32 * WT_STG_PITCH;                            // [4][128]
-    int* epi_fail = reinterpret_cast<int*>(xw + 4 * 128);                   // set when an epilogue wait expired
+    // staging rows are read with 16-byte loads: keep the block 16-byte aligned (barriers etc. take < 512 bytes)
+    float* stg_all = reinterpret_cast<float*>(smem + WT_STAGES * WT_STAGE_BYTES + 512);   // [4][63][36]
+    float* xw = stg_all + 4 * WT_STG_FLOATS;                                // [4][160]
+    int* epi_fail = reinterpret_cast<int*>(xw + 4 * WT_XW);                 // set when an epilogue wait expired
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g_bytes = 2 * p.BB * 128, box_bytes = p.BB * 128;
@@ -125,6 +145,8 @@ dw_wgrad_tc_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_consta
         for (int b = ch * p.BB; b < min(p.B, (ch + 1) * p.BB); ++b) m = max(m, min(p.len_out[b], p.T));
         chunk_len[ch] = m;
     }
+    // the skewed staging is written on the same parallelogram every time; the rest stays zero
+    for (int i = tid; i < 4 * WT_STG_FLOATS; i += WT_THREADS) stg_all[i] = 0.f;
     if (warp == 0) { ptx::tmem_alloc(tmem_slot, 2 * WT_ACC_COLS); ptx::tmem_relinquish(); }
     ptx::tc_fence_before();
     __syncthreads();
@@ -132,148 +154,176 @@ dw_wgrad_tc_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_consta
     const uint32_t tmem = *tmem_slot;
     const int ks_total = p.nchunks * p.ntb;
 
-    // contraction step ks of a unit that starts at ks0: skipped when its time block lies past every
-    // sample of its chunk (never the unit's first step, so that an accumulator is always written)
-    auto step_on = [&](int ks, int ks0, int& chunk, int& tb) -> bool {
-        chunk = ks / p.ntb; tb = ks - chunk * p.ntb;
-        if (ks == ks0 || chunk >= WT_MAX_CHUNKS) return true;
-        return tb * 128 < chunk_len[chunk];
-    };
-
-    if (warp == 8) {
-        if (lane == 0) {                               // ---- TMA producer ----
-            int it = 0; bool dead = false;
-            for (int unit = blockIdx.x; unit < p.units && !dead; unit += gridDim.x) {
-                const int c = unit / p.S, sp = unit - c * p.S;
-                const int ks0 = sp * p.ks_per_split, ks1 = min(ks0 + p.ks_per_split, ks_total);
-                for (int ks = ks0; ks < ks1; ++ks) {
-                    int chunk, tb;
-                    if (!step_on(ks, ks0, chunk, tb)) continue;
-                    const int s = it % WT_STAGES, ph = (it / WT_STAGES) & 1;
-                    if (!ptx::mbar_wait(&empty[s], ph ^ 1)) { raise_status(p.status, kErrTimeout); dead = true; break; }
-                    ptx::mbar_arrive_expect_tx(&full[s], stage_tx);
-                    uint8_t* sG = smem + s * WT_STAGE_BYTES;
-                    uint8_t* sX = sG + g_bytes;
-                    const int b0 = chunk * p.BB, t0 = tb * 128;
-                    ptx::tma_load_3d(sG, &mapG, &full[s], t0, c, b0);
-                    ptx::tma_load_3d(sG + box_bytes, &mapG, &full[s], t0 + 64, c, b0);
-                    for (int q = 0; q < p.nxb; ++q)
-                        ptx::tma_load_3d(sX + q * box_bytes, &mapX, &full[s], t0 - p.Pa + 64 * q, c, b0);
-                    ++it;
+    if (warp == 12) {                                  // ---- TMA producer: one box per lane ----
+        Ring rg; bool dead = false;
+        const bool is_g = lane < 2;
+        const int q = lane - 2;
+        const bool active = lane < 2 + p.nxb;
+        const void* map = is_g ? (const void*)&mapG : (const void*)&mapX;
+        const int dst_off = is_g ? lane * box_bytes : g_bytes + q * box_bytes;
+        const int t_off = is_g ? 64 * lane : 64 * q - p.Pa;
+        for (int unit = blockIdx.x; unit < p.units && !dead; unit += gridDim.x) {
+            const int c = unit / p.S, sp = unit - c * p.S;
+            StepWalk w; w.begin(sp, p.ks_per_split, ks_total, p.ntb, chunk_len);
+            for (; w.more(); w.next()) {
+                if (!w.on()) continue;
+                bool ok = true;
+                if (lane == 0) {
+                    ok = ptx::mbar_wait(&empty[rg.s], rg.ph ^ 1);
+                    if (ok) ptx::mbar_arrive_expect_tx(&full[rg.s], stage_tx);
                 }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) { if (lane == 0) raise_status(p.status, kErrTimeout); dead = true; break; }
+                if (active)
+                    ptx::tma_load_3d(smem + rg.s * WT_STAGE_BYTES + dst_off, map, &full[rg.s], w.tb * 128 + t_off, c,
+                                     w.chunk * p.BB);
+                rg.advance();
             }
         }
-        __syncwarp();
-    } else if (warp == 9) {
+    } else if (warp == 13) {
         if (lane == 0) {                               // ---- MMA issuer ----
             const uint32_t idesc = ptx::instr_desc(FmtW<TG>::v, 1u, 1u, 128, (uint32_t)p.N);
-            int it = 0, j = 0; bool dead = false;
+            // descriptors differ from step to step only in the start-address field
+            const uint64_t dbase = ptx::smem_desc(0, box_bytes, 1024);
+            const uint32_t smem_a = ptx::smem_u32(smem);
+            const int nkk = p.BB / 16;
+            Ring rg; int j = 0; bool dead = false;
             for (int unit = blockIdx.x; unit < p.units && !dead; unit += gridDim.x, ++j) {
                 const int c = unit / p.S, sp = unit - c * p.S;
-                const int ks0 = sp * p.ks_per_split, ks1 = min(ks0 + p.ks_per_split, ks_total);
+                (void)c;
                 const int buf = j & 1;
                 if (!ptx::mbar_wait(&acc_empty[buf], ((j >> 1) & 1) ^ 1)) { raise_status(p.status, kErrTimeout); break; }
                 ptx::tc_fence_after();
-                int done = 0;
-                for (int ks = ks0; ks < ks1; ++ks) {
-                    int chunk, tb;
-                    if (!step_on(ks, ks0, chunk, tb)) continue;
-                    const int s = it % WT_STAGES, ph = (it / WT_STAGES) & 1;
-                    if (!ptx::mbar_wait(&full[s], ph) || !ptx::mbar_wait(&conv[s], ph)) {
+                uint32_t accum = 0;
+                StepWalk w; w.begin(sp, p.ks_per_split, ks_total, p.ntb, chunk_len);
+                for (; w.more(); w.next()) {
+                    if (!w.on()) continue;
+                    // conv[s] completes only after the preparation warps have seen full[s] complete
+                    if (!ptx::mbar_wait(&conv[rg.s], rg.ph)) {
                         raise_status(p.status, kErrTimeout); dead = true; break;
                     }
                     ptx::tc_fence_after();
-                    const uint32_t aG = ptx::smem_u32(smem + s * WT_STAGE_BYTES), aX = aG + g_bytes;
-                    for (int kk = 0; kk < p.BB / 16; ++kk) {
-                        const uint64_t adesc = ptx::smem_desc(aG + kk * 2048, box_bytes, 1024);
-                        const uint64_t bdesc = ptx::smem_desc(aX + kk * 2048, box_bytes, 1024);
-                        ptx::mma_f16(tmem + buf * WT_ACC_COLS, adesc, bdesc, idesc, (done > 0 || kk > 0) ? 1u : 0u);
+                    const uint32_t aG = smem_a + rg.s * WT_STAGE_BYTES;
+                    uint64_t dG = dbase | (uint64_t)((aG & 0x3FFFFu) >> 4);
+                    uint64_t dX = dbase | (uint64_t)(((aG + g_bytes) & 0x3FFFFu) >> 4);
+                    for (int kk = 0; kk < nkk; ++kk) {
+                        ptx::mma_f16(tmem + buf * WT_ACC_COLS, dG, dX, idesc, accum);
+                        accum = 1u; dG += 2048 >> 4; dX += 2048 >> 4;
                     }
-                    ptx::mma_commit(&empty[s]);
-                    ++done; ++it;
+                    ptx::mma_commit(&empty[rg.s]);
+                    rg.advance();
                 }
                 if (!dead) ptx::mma_commit(&acc_full[buf]);
             }
         }
         __syncwarp();
-    } else if (warp >= 4) {                            // ---- operand preparation (warps 4-7) ----
-        const int ctid = tid - 128;
-        int it = 0; bool dead = false; bool over = false;
+    } else if (warp >= 4) {                            // ---- operand preparation: two groups of four warps ----
+        // group 0 (warps 4-7) takes the even ring steps, group 1 (warps 8-11) the odd ones
+        const int grp = (warp - 4) >> 2;
+        const int ctid = tid - 128 - 128 * grp;
+        // Vector v = ctid + 128 i of the window sits in box v / (8 BB), sample row (v / 8) % BB, 16-byte slot
+        // v % 8.  The slot and the row's low bits do not depend on i, so the frame offset inside a box is
+        // a per-thread constant (128-byte swizzle: logical slot = physical slot ^ (row % 8)).
+        const int lb = (p.BB == 32) ? 5 : 4;
+        const int nvec_t = (p.nxb * p.BB) >> 4;                 // vectors per thread and step (<= 8)
+        const int r0 = ctid >> 3;
+        const int toff = 8 * ((ctid & 7) ^ (r0 & 7));
+        Ring rg; int it = 0; bool dead = false; float amax = 0.f;
         for (int unit = blockIdx.x; unit < p.units && !dead; unit += gridDim.x) {
             const int c = unit / p.S, sp = unit - c * p.S;
             (void)c;
-            const int ks0 = sp * p.ks_per_split, ks1 = min(ks0 + p.ks_per_split, ks_total);
-            for (int ks = ks0; ks < ks1; ++ks) {
-                int chunk, tb;
-                if (!step_on(ks, ks0, chunk, tb)) continue;
-                const int s = it % WT_STAGES, ph = (it / WT_STAGES) & 1;
-                bool ok = ptx::mbar_wait(&full[s], ph);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) { if (lane == 0) raise_status(p.status, kErrTimeout); dead = true; break; }
-                if (p.prep) {
-                    uint4* sX = reinterpret_cast<uint4*>(smem + s * WT_STAGE_BYTES + g_bytes);
-                    const int nvec = p.nxb * p.BB * 8;
-                    const int tx0 = tb * 128 - p.Pa, b0 = chunk * p.BB;
-                    for (int v = ctid; v < nvec; v += 128) {
-                        const int q = v / (p.BB * 8), r = (v >> 3) % p.BB, pv = v & 7;
-                        const int lv = pv ^ (r & 7);                       // 128-byte swizzle: logical 16-byte slot
-                        const int t = tx0 + 64 * q + 8 * lv;
-                        const int b = b0 + r;
-                        int nvalid = 8;
-                        if (p.mask) nvalid = (b < p.B) ? (min(p.len_in[b], p.T) - t) : 0;
-                        sX[v] = prep8<TG, TX>(sX[v], nvalid, over);
+            StepWalk w; w.begin(sp, p.ks_per_split, ks_total, p.ntb, chunk_len);
+            for (; w.more(); w.next()) {
+                if (!w.on()) continue;
+                if ((it & 1) == grp) {
+                    const bool ok = ptx::mbar_wait_warp(&full[rg.s], rg.ph);
+                    if (!ok) { if (lane == 0) raise_status(p.status, kErrTimeout); dead = true; break; }
+                    if (p.prep) {
+                        uint4* sX = reinterpret_cast<uint4*>(smem + rg.s * WT_STAGE_BYTES + g_bytes);
+                        const int tx0 = w.tb * 128 - p.Pa + toff, b0 = w.chunk * p.BB;
+                        // frames left before the sample's end, for this thread's (at most two) rows
+                        int left0 = 1 << 30, left1 = 1 << 30;
+                        if (p.mask) {
+                            const int ba = b0 + r0, bb = b0 + r0 + 16;
+                            left0 = (ba < p.B ? min(p.len_in[ba], p.T) : 0) - tx0;
+                            left1 = (bb < p.B ? min(p.len_in[bb], p.T) : 0) - tx0;
+                        }
+                        uint4 raw[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) if (i < nvec_t) raw[i] = sX[ctid + 128 * i];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            if (i < nvec_t) {
+                                const int v = ctid + 128 * i;
+                                const int left = (((v >> 3) & 16) & (p.BB - 1)) ? left1 : left0;
+                                sX[v] = prep8<TG, TX>(raw[i], left - 64 * (v >> (3 + lb)), amax);
+                            }
+                        }
+                        ptx::fence_proxy_async();
                     }
-                    ptx::fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(&conv[rg.s]);
                 }
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&conv[s]);
-                ++it;
+                rg.advance(); ++it;
             }
         }
-        if (over) raise_status(p.status, kErrRange);
+        if (amax >= 65536.f) raise_status(p.status, kErrRange);
     } else {                                           // ---- epilogue (warps 0-3) ----
-        float* stg = stg_all + warp * 32 * WT_STG_PITCH;
-        const int nq = (31 + p.delta + p.K + 31) / 32;     // 32-column chunks this warp reads
+        // Warp e owns accumulator rows j = 32 e + l (lane l) and reads them in 32-column chunks
+        // (columns 32 e + 32 q + i).  The entry of tap k in row j is column j + delta + k, so inside a chunk
+        // it lies on the diagonal d = i - l + 31 = delta + k - 32 q + 31.  Each lane scatters its 32 values
+        // to staging row d (pitch 36 floats: conflict-free both ways), and a lane then sums whole staging
+        // rows d = lane and d = lane + 32 with 16-byte loads: all of them belong to taps
+        // k = lane + 1 - delta + 32 n with n = q - 1 and n = q.
+        float* stg = stg_all + warp * WT_STG_FLOATS;
+        const int nq = (62 + p.delta + p.K) / 32;          // 32-column chunks this warp reads (<= 6)
         int j = 0;
         for (int unit = blockIdx.x; unit < p.units; unit += gridDim.x, ++j) {
             const int c = unit / p.S, sp = unit - c * p.S;
             const int buf = j & 1;
-            bool ok = ptx::mbar_wait(&acc_full[buf], (j >> 1) & 1);
-            ok = __all_sync(0xffffffffu, ok);
+            const bool ok = ptx::mbar_wait_warp(&acc_full[buf], (j >> 1) & 1, 64);
             if (!ok && lane == 0) { raise_status(p.status, kErrTimeout); atomicExch(epi_fail, 1); }
             bar_sync_named(1, 128);                        // the four warps leave together or not at all
             if (*reinterpret_cast<volatile int*>(epi_fail)) break;
             ptx::tc_fence_after();
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};           // taps lane, lane+32, lane+64, lane+96
-            for (int q = 0; q < nq; ++q) {
-                uint32_t r[32];
-                ptx::tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + buf * WT_ACC_COLS + warp * 32 + q * 32, r);
-                ptx::tmem_ld_wait();
-                __syncwarp();
+            float acc[7] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};   // acc[n + 1]: tap lane + 1 - delta + 32 n
 #pragma unroll
-                for (int i = 0; i < 32; ++i) stg[lane * WT_STG_PITCH + i] = __uint_as_float(r[i]);
-                __syncwarp();
-                // row l of this warp is frame j = 32 warp + l; it holds columns 32 warp + 32 q + i, and the
-                // entry of tap k sits at column j + delta + k, i.e. i = l + delta + k - 32 q
+            for (int q = 0; q < 6; ++q) {
+                if (q < nq) {
+                    uint32_t r[32];
+                    ptx::tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + buf * WT_ACC_COLS + warp * 32 + q * 32, r);
+                    ptx::tmem_ld_wait();
+                    __syncwarp();
 #pragma unroll
-                for (int m = 0; m < 4; ++m) {
-                    const int k = lane + 32 * m;
-                    if (k < p.K) {
-                        const int off = p.delta + k - 32 * q;
-                        const int lo = max(0, -off), hi = min(31, 31 - off);
-                        float a = acc[m];
-                        for (int l = lo; l <= hi; ++l) a += stg[l * WT_STG_PITCH + l + off];
-                        acc[m] = a;
+                    for (int i = 0; i < 32; ++i) stg[(i + 31 - lane) * WT_STG_PITCH + lane] = __uint_as_float(r[i]);
+                    __syncwarp();
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int d = lane + 32 * h;
+                        if (d < 63) {
+                            const float4* row = reinterpret_cast<const float4*>(stg + d * WT_STG_PITCH);
+                            float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                            for (int v = 0; v < 8; v += 2) {
+                                const float4 x0 = row[v], x1 = row[v + 1];
+                                s0 += (x0.x + x0.y) + (x0.z + x0.w);
+                                s1 += (x1.x + x1.y) + (x1.z + x1.w);
+                            }
+                            acc[q + h] += s0 + s1;
+                        }
                     }
                 }
             }
             ptx::tc_fence_before();
             ptx::mbar_arrive(&acc_empty[buf]);             // accumulator buffer may be overwritten
 #pragma unroll
-            for (int m = 0; m < 4; ++m) xw[warp * 128 + lane + 32 * m] = acc[m];
+            for (int n = 0; n < 7; ++n) {
+                const int k = lane + 1 - p.delta + 32 * (n - 1);
+                if (k >= 0 && k < p.K) xw[warp * WT_XW + k] = acc[n];
+            }
             bar_sync_named(1, 128);
             if (tid < p.K) {
-                const float v = ((xw[tid] + xw[128 + tid]) + xw[256 + tid]) + xw[384 + tid];
+                const float v = ((xw[tid] + xw[WT_XW + tid]) + xw[2 * WT_XW + tid]) + xw[3 * WT_XW + tid];
                 p.partials[((size_t)sp * p.C + c) * p.K + tid] = v;
             }
             bar_sync_named(1, 128);
@@ -284,8 +334,9 @@ dw_wgrad_tc_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_consta
     if (warp == 0) ptx::tmem_dealloc(tmem, 2 * WT_ACC_COLS);
 }
 
-constexpr int kWtSmem = WT_STAGES * WT_STAGE_BYTES + 1024 /* alignment */ + 256 /* barriers */ +
-                        WT_MAX_CHUNKS * 4 + 4 * 32 * WT_STG_PITCH * 4 + 4 * 128 * 4 + 16;
+constexpr int kWtSmem = WT_STAGES * WT_STAGE_BYTES + 1024 /* alignment */ + 512 /* barriers, chunk lengths */ +
+                        4 * WT_STG_FLOATS * 4 + 4 * WT_XW * 4 + 16;
+static_assert((3 * WT_STAGES + 4) * 8 + 8 + WT_MAX_CHUNKS * 4 <= 512, "barrier block");
 
 template <typename TG, typename TX>
 void launch_wt(const Launch& L, int grid, const CUtensorMap& mg, const CUtensorMap& mx, const WtParams& p) {

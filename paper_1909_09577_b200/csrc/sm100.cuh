@@ -45,6 +45,24 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     return false;
 }
 
+// Whole-warp wait: lane 0 polls and the other lanes follow it.  Thirty-two lanes polling one mbarrier are
+// thirty-two serialised requests to the same word on every poll, which delays the mbarrier, TMA and MMA
+// instructions of the single-thread roles that share the SM.  `sleep_ns` > 0 backs off between polls.
+// Call with all 32 lanes.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, uint32_t sleep_ns = 0) {
+    uint32_t ok = 1;
+    if ((threadIdx.x & 31) == 0) {
+        ok = 0;
+        for (uint32_t i = 0; i < kWaitPolls; ++i) {
+            if (mbar_try_wait(bar, parity)) { ok = 1; break; }
+            if (sleep_ns) __nanosleep(sleep_ns);
+        }
+    }
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    __syncwarp();                       // orders every lane's later accesses after lane 0's acquire
+    return ok != 0;
+}
+
 // ---- TMA tiled loads (global -> this CTA's shared memory), completion on an mbarrier -----------
 __device__ __forceinline__ void tma_load_2d(void* dst, const void* map, uint64_t* bar, int x, int y) {
     asm volatile(
