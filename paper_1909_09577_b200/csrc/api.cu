@@ -140,7 +140,11 @@ int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
     const int odt = op_dtype(d);
     const void* u;
     if (d->has_dw) {
-        dw_fwd(L, dt, odt, io.x, p->wd, sv->u, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s);
+        if (ctx->gemm_mode == 0 && dw_tma_supported(&ctx->tc, dt, m.B, m.T, m.K, m.s))
+            dw_tma_fwd(&ctx->tc, L, dt, odt, io.x, p->wd, sv->u, io.len_in, io.len_out, m.B, m.Cin, m.T, m.K,
+                       io.x_clean ? 1 : 0);
+        else
+            dw_fwd(L, dt, odt, io.x, p->wd, sv->u, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s);
         u = sv->u;
     } else if (io.x_clean) {
         u = io.x;
@@ -292,9 +296,14 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
                         m.T, m.K, io.x_clean ? 1 : 0);
         else
             dw_wgrad(L, dt, odt, s.gu, io.x, g->dwd, s.wpart, acc, gmax, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s);
-        if (io.dx)
-            dw_dgrad(L, dt, odt, s.gu, p->wd, io.dx, io.dx_add, extra, gmax, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp,
-                     m.K, m.s);
+        if (io.dx) {
+            if (ctx->gemm_mode == 0 && dw_tma_supported(&ctx->tc, dt, m.B, m.T, m.K, m.s))
+                dw_tma_dgrad(&ctx->tc, L, dt, odt, s.gu, p->wd, io.dx, io.dx_add, extra, gmax, io.len_in, io.len_out, m.B,
+                             m.Cin, m.T, m.K);
+            else
+                dw_dgrad(L, dt, odt, s.gu, p->wd, io.dx, io.dx_add, extra, gmax, io.len_in, io.len_out, m.B, m.Cin, m.T,
+                         m.Tp, m.K, m.s);
+        }
     } else if (io.dx) {
         if (!io.dx_add && !extra) {
             pointwise_dgrad(ctx, L, dt, p->wp, s.gv, io.dx, m.B, m.Cin, m.Cout, m.Tp, io.len_out);

@@ -1,0 +1,472 @@
+// Stride-1 depthwise correlation (forward and input gradient) on the tensor cores, fed by TMA.
+//
+// For one channel the K-tap correlation over time is a banded Toeplitz product.  Time is cut into blocks
+// of 128 output frames; the MMA tile has one (sample, time block) pair per row:
+//     D[(b,tb), j] = sum_{j'} X[(b,tb), j'] * Tz[j', j],   X[(b,tb), j'] = x[b, c, 128 tb - Pa + j'],
+//     Tz[j', j] = w[j' - j - (Pa - P)]  (zero outside the taps),   Pa = P rounded up to a multiple of 8
+// so that every window starts on a 16-byte boundary.  The band is the same for output positions j and
+// j + 64 up to a shift of 64 in j', so only the 64-column block Tz64 is built (per channel, by four
+// builder warps, double-buffered) and the two halves of a tile are  D[:, 64 h + j] = X[:, 64 h + j'] * Tz64,
+// i.e. the same B operand with the A operand's start address moved by one 64-element chunk.
+// A (the windows) comes straight from HBM: TMA boxes of (64 frames x 1 channel x BB samples), K-major,
+// 128-byte swizzle; frames outside [0, T) are zero-filled by the TMA unit, which is the "same" padding.
+// Each input element is read from HBM once (window overlaps hit L2).  Rows of a tile are
+// (time block within a group of 128/BB, sample within a chunk of BB).
+// Warps: 0-7 epilogue (TMEM lane quarter w%4, column half w/4), 8-9 input masking (only when the input
+// may be non-zero beyond a sample's length), 10-13 Toeplitz builders, 14 TMA producer (one box per lane),
+// 15 MMA issuer.  Accumulators are quadruple-buffered in tensor memory.  The epilogue transposes the
+// accumulator through shared memory so that global accesses are whole 32-byte sectors: already rounded
+// to the 16-bit output type when nothing is added to the result, in fp32 otherwise.
+// Every wait is bounded; on expiry the CTA raises the status word and leaves.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <type_traits>
+
+#include "common.cuh"
+#include "kernels.h"
+#include "sm100.cuh"
+#include "tc_gemm.h"
+
+namespace sc {
+namespace {
+
+constexpr int DT_THREADS = 512;
+constexpr int DT_AB_BYTES = 180224;        // A ring (3 x 48 KiB or 2 x 64 KiB) + two Toeplitz blocks (16 or 24 KiB each)
+constexpr int DT_ACC_COLS = 128;
+constexpr int DT_NACC = 4;
+constexpr int DT_STG_BYTES = 5120;         // per epilogue warp: 2 x 32 rows x 80 bytes (16-bit) or 32 rows x 144 bytes (fp32)
+constexpr int DT_WOFF = 80;                // index of tap 0 in the padded tap arrays
+constexpr int DT_WLEN = 288;
+constexpr int DT_MAX_STAGES = 3;
+
+struct DtParams {
+    const void* w; void* out; const void* add1; const void* add2; const float* gmax;
+    const int* len_src; const int* len_dst; int* status;
+    int B, C, T, K, Pa, delta;
+    int BB, TBL;          // samples per chunk, time blocks per group (BB * TBL = 128)
+    int nxb;              // 64-element chunks of the window (2 to 4)
+    int NK2;              // contraction length of one half (multiple of 16, <= 192)
+    int ntb, ngrp, nchunks, tpc;   // time blocks, groups, sample chunks, tiles per channel
+    int nstages, stage_bytes;
+    int b_stride;         // bytes per Toeplitz buffer: 64 rows x 128 bytes per 64-element chunk of NK2
+    int mask;             // 1: zero input frames at or beyond len_src
+    int flip;             // 1: taps reversed (input gradient)
+};
+
+template <typename T> struct FmtD;
+template <> struct FmtD<__half> { static constexpr uint32_t v = 0; };
+template <> struct FmtD<__nv_bfloat16> { static constexpr uint32_t v = 1; };
+
+template <typename T> __device__ __forceinline__ unsigned short to_bits16(float v);
+template <> __device__ __forceinline__ unsigned short to_bits16<__half>(float v) { return __half_as_ushort(__float2half_rn(v)); }
+template <> __device__ __forceinline__ unsigned short to_bits16<__nv_bfloat16>(float v) { return __bfloat16_as_ushort(__float2bfloat16_rn(v)); }
+
+template <typename T> __device__ __forceinline__ uint32_t pack2(float a, float b);
+template <> __device__ __forceinline__ uint32_t pack2<__half>(float a, float b) {
+    const __half2 h = __floats2half2_rn(a, b); return *reinterpret_cast<const uint32_t*>(&h);
+}
+template <> __device__ __forceinline__ uint32_t pack2<__nv_bfloat16>(float a, float b) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(a, b); return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+__device__ __forceinline__ void named_bar(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// TI: type of the input tensor and of both MMA operands; TW: stored tap type; TO: output / addend type.
+template <typename TI, typename TW, typename TO>
+__global__ void __launch_bounds__(DT_THREADS, 1)
+dw_tma_kernel(const __grid_constant__ CUtensorMap mapX, DtParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    uint8_t* sB = smem + p.nstages * p.stage_bytes;                         // [2][b_stride], 1024-byte aligned
+    uint8_t* stg_all = smem + DT_AB_BYTES;                                  // [8][DT_STG_BYTES]
+    unsigned short* wpadE = reinterpret_cast<unsigned short*>(stg_all + 8 * DT_STG_BYTES);   // [DT_WLEN] taps
+    unsigned short* wpadO = wpadE + DT_WLEN;                                // the same, shifted by one element
+    uint64_t* full = reinterpret_cast<uint64_t*>(wpadO + DT_WLEN);          // [DT_MAX_STAGES]
+    uint64_t* prep = full + DT_MAX_STAGES;
+    uint64_t* empty = prep + DT_MAX_STAGES;
+    uint64_t* acc_full = empty + DT_MAX_STAGES;     // [DT_NACC]
+    uint64_t* acc_empty = acc_full + DT_NACC;       // [DT_NACC]
+    uint64_t* b_full = acc_empty + DT_NACC;         // [2]
+    uint64_t* b_empty = b_full + 2;                 // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(b_empty + 2);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int s = 0; s < DT_MAX_STAGES; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&prep[s], 2); ptx::mbar_init(&empty[s], 1); }
+        for (int i = 0; i < DT_NACC; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 256); }
+        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&b_full[i], 4); ptx::mbar_init(&b_empty[i], 1); }
+        ptx::fence_barrier_init();
+        ptx::prefetch_tensormap(&mapX);
+    }
+    if (warp == 0) { ptx::tmem_alloc(tmem_slot, DT_NACC * DT_ACC_COLS); ptx::tmem_relinquish(); }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    const int box_bytes = p.BB * 128;
+
+    if (warp == 14) {                                  // ---- TMA producer: one box per lane ----
+        // box (q, tbl): window chunk q of time block tbl of the group, all BB samples of the chunk
+        const int nbox = p.nxb * p.TBL;
+        const int q = lane / p.TBL, tbl = lane - q * p.TBL;
+        const bool active = lane < nbox;
+        const int dst_off = q * 16384 + tbl * box_bytes;
+        int s = 0, ph = 0; bool dead = false;
+        for (int c = blockIdx.x; c < p.C && !dead; c += gridDim.x) {
+            for (int chunk = 0; chunk < p.nchunks && !dead; ++chunk) {
+                for (int g = 0; g < p.ngrp; ++g) {
+                    uint32_t ok = 1;
+                    if (lane == 0) {
+                        ok = ptx::mbar_wait(&empty[s], ph ^ 1) ? 1u : 0u;
+                        if (ok) ptx::mbar_arrive_expect_tx(&full[s], (uint32_t)(nbox * box_bytes));
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) { if (lane == 0) raise_status(p.status, kErrTimeout); dead = true; break; }
+                    if (active)
+                        ptx::tma_load_3d(smem + s * p.stage_bytes + dst_off, &mapX, &full[s],
+                                         128 * (g * p.TBL + tbl) - p.Pa + 64 * q, c, chunk * p.BB);
+                    if (++s == p.nstages) { s = 0; ph ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 15) {
+        if (lane == 0) {                               // ---- MMA issuer ----
+            const uint32_t idesc = ptx::instr_desc(FmtD<TI>::v, 0u, 0u, 128, 64);
+            const uint64_t dk = ptx::smem_desc(0, 16, 1024);
+            const uint32_t smem_a = ptx::smem_u32(smem), smem_b = ptx::smem_u32(sB);
+            const int nkk = p.NK2 / 16;
+            int s = 0, ph = 0, j = 0, ci = 0; bool dead = false;
+            for (int c = blockIdx.x; c < p.C && !dead; c += gridDim.x, ++ci) {
+                const int bb = ci & 1;
+                if (!ptx::mbar_wait(&b_full[bb], (ci >> 1) & 1)) { raise_status(p.status, kErrTimeout); break; }
+                for (int t = 0; t < p.tpc; ++t, ++j) {
+                    const int buf = j & (DT_NACC - 1);
+                    if (!ptx::mbar_wait(&acc_empty[buf], ((j / DT_NACC) & 1) ^ 1)) { raise_status(p.status, kErrTimeout); dead = true; break; }
+                    if (!ptx::mbar_wait(p.mask ? &prep[s] : &full[s], ph)) { raise_status(p.status, kErrTimeout); dead = true; break; }
+                    ptx::tc_fence_after();
+                    const uint32_t aA = smem_a + s * p.stage_bytes, aB = smem_b + bb * p.b_stride;
+                    const uint64_t dB0 = dk | (uint64_t)((aB & 0x3FFFFu) >> 4);
+#pragma unroll 1
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t d = tmem + buf * DT_ACC_COLS + 64 * h;
+                        uint64_t dA = dk | (uint64_t)(((aA + h * 16384) & 0x3FFFFu) >> 4), dB = dB0;
+                        for (int kk = 0; kk < nkk; ++kk) {
+                            ptx::mma_f16(d, dA, dB, idesc, kk > 0 ? 1u : 0u);
+                            // 16 contraction elements on: 32 bytes inside a 64-element chunk, else the next chunk
+                            if ((kk & 3) == 3) { dA += (16384 - 96) >> 4; dB += (8192 - 96) >> 4; }
+                            else { dA += 32 >> 4; dB += 32 >> 4; }
+                        }
+                    }
+                    ptx::mma_commit(&empty[s]);
+                    ptx::mma_commit(&acc_full[buf]);
+                    if (++s == p.nstages) { s = 0; ph ^= 1; }
+                }
+                if (!dead) ptx::mma_commit(&b_empty[bb]);      // the Toeplitz buffer may be rebuilt
+            }
+        }
+        __syncwarp();
+    } else if (warp >= 10) {                           // ---- Toeplitz builders (warps 10-13) ----
+        const int bt = tid - 320;                      // 0 .. 127
+        const int j = bt & 63, hv = bt >> 6;           // row of Tz64 (output position inside a half); vector parity
+        const int nvec = p.NK2 / 8;
+        // element (j', j) = tap j' - j - delta = padded tap index base + j'; 32-bit loads need an even
+        // index, so rows with an odd base read the copy that is shifted by one element
+        const int base = DT_WOFF - j - p.delta;
+        const uint32_t* src0 = reinterpret_cast<const uint32_t*>((base & 1) ? (wpadO + base - 1) : (wpadE + base));
+        int ci = 0; bool dead = false;
+        for (int c = blockIdx.x; c < p.C && !dead; c += gridDim.x, ++ci) {
+            const int bb = ci & 1;
+            named_bar(2, 128);                         // everyone is done reading the previous channel's taps
+            for (int i = bt; i < DT_WLEN; i += 128) {
+                const int k = i - DT_WOFF;
+                float v = 0.f;
+                if (k >= 0 && k < p.K) v = ldf(reinterpret_cast<const TW*>(p.w) + (size_t)c * p.K + (p.flip ? p.K - 1 - k : k));
+                const unsigned short bits = to_bits16<TI>(v);
+                wpadE[i] = bits;
+                if (i > 0) wpadO[i - 1] = bits;
+                if (i == DT_WLEN - 1) wpadO[i] = 0;
+            }
+            named_bar(2, 128);
+            const bool ok = ptx::mbar_wait_warp(&b_empty[bb], ((ci >> 1) & 1) ^ 1, 32);
+            if (!ok) { if (lane == 0) raise_status(p.status, kErrTimeout); dead = true; break; }
+            uint4* rowbase = reinterpret_cast<uint4*>(sB + bb * p.b_stride + j * 128);
+            for (int v = hv; v < nvec; v += 2) {       // vector v holds j' = 8 v .. 8 v + 7
+                const uint32_t* src = src0 + 4 * v;
+                // chunk v / 8 (8192 bytes apart), 16-byte slot (v % 8) ^ (row % 8)
+                rowbase[(v >> 3) * 512 + ((v & 7) ^ (j & 7))] = make_uint4(src[0], src[1], src[2], src[3]);
+            }
+            ptx::fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&b_full[bb]);
+        }
+    } else if (warp >= 8) {                            // ---- input masking (warps 8-9): rows mt and mt + 64 ----
+        if (p.mask) {
+            const int mt = tid - 256;                  // 0 .. 63
+            int s = 0, ph = 0; bool dead = false;
+            for (int c = blockIdx.x; c < p.C && !dead; c += gridDim.x) {
+                for (int chunk = 0; chunk < p.nchunks && !dead; ++chunk) {
+                    for (int g = 0; g < p.ngrp; ++g) {
+                        const bool ok = ptx::mbar_wait_warp(&full[s], ph);
+                        if (!ok) { if (lane == 0) raise_status(p.status, kErrTimeout); dead = true; break; }
+                        bool wrote = false;
+#pragma unroll 1
+                        for (int rsel = 0; rsel < 2; ++rsel) {
+                            const int r = mt + 64 * rsel;
+                            const int tbl = r / p.BB, bi = r - tbl * p.BB;
+                            const int b = chunk * p.BB + bi;
+                            const int len = b < p.B ? min(p.len_src[b], p.T) : 0;
+                            const int t0 = 128 * (g * p.TBL + tbl) - p.Pa;      // first frame of this row's window
+                            if (t0 + 64 * p.nxb <= len) continue;
+                            uint8_t* row = smem + s * p.stage_bytes + r * 128;
+                            for (int v = 0; v < 8 * p.nxb; ++v) {
+                                const int t = t0 + 8 * v;                    // logical vector v: frames t .. t + 7
+                                if (t + 8 <= len) continue;
+                                uint4* pv = reinterpret_cast<uint4*>(row + (v >> 3) * 16384) + ((v & 7) ^ (r & 7));
+                                wrote = true;
+                                if (t >= len) { *pv = make_uint4(0, 0, 0, 0); continue; }
+                                uint4 x = *pv;
+                                uint32_t wv[4] = {x.x, x.y, x.z, x.w};
+                                const int nv = len - t;
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    if (2 * i >= nv) wv[i] = 0u;
+                                    else if (2 * i + 1 >= nv) wv[i] &= 0x0000FFFFu;
+                                }
+                                *pv = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+                            }
+                        }
+                        if (wrote) ptx::fence_proxy_async();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(&prep[s]);
+                        if (++s == p.nstages) { s = 0; ph ^= 1; }
+                    }
+                }
+            }
+        }
+    } else {                                           // ---- epilogue (warps 0-7) ----
+        const int wq = warp & 3, half = warp >> 2;
+        uint8_t* stg = stg_all + warp * DT_STG_BYTES;
+        const float inv = p.gmax ? 1.f / pow2_scale(*p.gmax) : 1.f;
+        const bool has_add = p.add1 != nullptr || p.add2 != nullptr;
+        TO* out = reinterpret_cast<TO*>(p.out);
+        const TO* add1 = reinterpret_cast<const TO*>(p.add1);
+        const TO* add2 = reinterpret_cast<const TO*>(p.add2);
+        // this lane's own accumulator row (what it reads from tensor memory)
+        const int my_tbl = (wq * 32 + lane) / p.BB, my_bi = (wq * 32 + lane) - my_tbl * p.BB;
+        // store phase: in pass `it` this lane stores 8 columns (cs .. cs + 7) of warp row 8 it + lane / 4.
+        // Which (time block, sample) that row is never changes, so it is worked out once.
+        const int rr = lane >> 2, cs = (lane & 3) * 8;
+        int tbl_of[4], bi_of[4];
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int row = wq * 32 + it * 8 + rr;
+            tbl_of[it] = row / p.BB; bi_of[it] = row - tbl_of[it] * p.BB;
+        }
+        int j = 0; float amax = 0.f;
+        for (int c = blockIdx.x; c < p.C; c += gridDim.x) {
+            for (int chunk = 0; chunk < p.nchunks; ++chunk) {
+                int ld_of[4]; long long base_of[4];       // valid output length and element offset of frame 0
+#pragma unroll
+                for (int it = 0; it < 4; ++it) {
+                    const int b = chunk * p.BB + bi_of[it];
+                    ld_of[it] = b < p.B ? min(p.len_dst[b], p.T) : -1;          // -1: no such sample
+                    base_of[it] = ((long long)b * p.C + c) * p.T;
+                }
+                const int my_b = chunk * p.BB + my_bi;
+                const int my_ld = my_b < p.B ? min(p.len_dst[my_b], p.T) : 0;
+                for (int g = 0; g < p.ngrp; ++g, ++j) {
+                    const int buf = j & (DT_NACC - 1);
+                    const bool ok = ptx::mbar_wait_warp(&acc_full[buf], (j / DT_NACC) & 1, 32);
+                    if (!ok) { if (lane == 0) raise_status(p.status, kErrTimeout); goto done; }
+                    ptx::tc_fence_after();
+                    const uint32_t taddr = tmem + ((uint32_t)(wq * 32) << 16) + buf * DT_ACC_COLS + 64 * half;
+                    const int tcol0 = 128 * (g * p.TBL) + 64 * half;            // frame of column 0 of this half, time block 0
+                    if (!has_add) {
+                        // ---- round first, transpose 16-bit values: both 32-column chunks in one go ----
+                        uint32_t v0[32], v1[32];
+                        ptx::tmem_ld32(taddr, v0);
+                        ptx::tmem_ld32(taddr + 32, v1);
+                        ptx::tmem_ld_wait();
+                        const int nv = my_ld - (tcol0 + 128 * my_tbl);          // valid columns of this lane's row
+                        __syncwarp();
+#pragma unroll
+                        for (int cc = 0; cc < 2; ++cc) {
+                            uint32_t (&v)[32] = cc ? v1 : v0;
+                            float f[32];
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) * inv;
+                            if (nv < 32 * cc + 32) {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) if (32 * cc + i >= nv) f[i] = 0.f;
+                            }
+                            if (std::is_same<TO, __half>::value) {   // range guard: clamp only when hit
+                                float m = 0.f;
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) m = fmaxf(m, fabsf(f[i]));
+                                if (m > 65504.f) {
+#pragma unroll
+                                    for (int i = 0; i < 32; ++i) f[i] = fminf(fmaxf(f[i], -65504.f), 65504.f);
+                                }
+                                amax = fmaxf(amax, m);
+                            }
+                            uint4* dst = reinterpret_cast<uint4*>(stg + cc * 2560 + lane * 80);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                dst[i] = make_uint4(pack2<TO>(f[8 * i], f[8 * i + 1]), pack2<TO>(f[8 * i + 2], f[8 * i + 3]),
+                                                    pack2<TO>(f[8 * i + 4], f[8 * i + 5]), pack2<TO>(f[8 * i + 6], f[8 * i + 7]));
+                        }
+                        __syncwarp();
+#pragma unroll
+                        for (int cc = 0; cc < 2; ++cc) {
+#pragma unroll
+                            for (int it = 0; it < 4; ++it) {
+                                const int t = tcol0 + 128 * tbl_of[it] + 32 * cc + cs;
+                                if (ld_of[it] < 0 || t >= p.T) continue;
+                                const uint4 x = *reinterpret_cast<const uint4*>(stg + cc * 2560 + (it * 8 + rr) * 80 + 2 * cs);
+                                *reinterpret_cast<uint4*>(out + base_of[it] + t) = x;
+                            }
+                        }
+                    } else {
+                        // ---- something is added to the result: transpose fp32, add, then round ----
+#pragma unroll 1
+                        for (int cc = 0; cc < 2; ++cc) {
+                            uint32_t v[32];
+                            ptx::tmem_ld32(taddr + 32 * cc, v);
+                            ptx::tmem_ld_wait();
+                            __syncwarp();
+                            float* sf = reinterpret_cast<float*>(stg);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                *reinterpret_cast<float4*>(sf + lane * 36 + 4 * i) =
+                                    make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                                                __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+                            __syncwarp();
+#pragma unroll
+                            for (int it = 0; it < 4; ++it) {
+                                const int t = tcol0 + 128 * tbl_of[it] + 32 * cc + cs;
+                                const int ld = ld_of[it];
+                                if (ld < 0 || t >= p.T) continue;
+                                const long long off = base_of[it] + t;
+                                float f[8];
+                                if (t >= ld) {
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) f[e] = 0.f;
+                                } else {
+                                    const float4 a = *reinterpret_cast<const float4*>(sf + (it * 8 + rr) * 36 + cs);
+                                    const float4 bq = *reinterpret_cast<const float4*>(sf + (it * 8 + rr) * 36 + cs + 4);
+                                    f[0] = a.x * inv; f[1] = a.y * inv; f[2] = a.z * inv; f[3] = a.w * inv;
+                                    f[4] = bq.x * inv; f[5] = bq.y * inv; f[6] = bq.z * inv; f[7] = bq.w * inv;
+                                    if (add1) { float q8[8]; ld8<TO>(add1 + off, q8);
+#pragma unroll
+                                        for (int e = 0; e < 8; ++e) f[e] += q8[e]; }
+                                    if (add2) { float q8[8]; ld8<TO>(add2 + off, q8);
+#pragma unroll
+                                        for (int e = 0; e < 8; ++e) f[e] += q8[e]; }
+                                    if (t + 8 > ld) {
+#pragma unroll
+                                        for (int e = 0; e < 8; ++e) if (t + e >= ld) f[e] = 0.f;
+                                    }
+                                    if (std::is_same<TO, __half>::value) {
+                                        float m = 0.f;
+#pragma unroll
+                                        for (int e = 0; e < 8; ++e) m = fmaxf(m, fabsf(f[e]));
+                                        if (m > 65504.f) {
+#pragma unroll
+                                            for (int e = 0; e < 8; ++e) f[e] = fminf(fmaxf(f[e], -65504.f), 65504.f);
+                                        }
+                                        amax = fmaxf(amax, m);
+                                    }
+                                }
+                                st8<TO>(out + off, f);
+                            }
+                        }
+                    }
+                    ptx::tc_fence_before();
+                    ptx::mbar_arrive(&acc_empty[buf]);
+                }
+            }
+        }
+    done:
+        if (amax > 65504.f) raise_status(p.status, kErrRange);
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 0) ptx::tmem_dealloc(tmem, DT_NACC * DT_ACC_COLS);
+}
+
+constexpr int kDtSmem = 1024 + DT_AB_BYTES + 8 * DT_STG_BYTES + 2 * DT_WLEN * 2 + 512;
+static_assert(kDtSmem <= 232448, "shared memory per CTA");
+
+template <typename TI, typename TW, typename TO>
+void launch_dt(const Launch& L, int grid, const CUtensorMap& mx, const DtParams& p) {
+    auto kern = dw_tma_kernel<TI, TW, TO>;
+    static bool configured = false;
+    if (!configured) {
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kDtSmem);
+        configured = true;
+    }
+    kern<<<grid, DT_THREADS, kDtSmem, L.stream>>>(mx, p);
+    L.count();
+}
+
+// in_dtype: type of the input tensor; w_dtype: stored tap type; out_dtype: output / addend type
+void run(const TcState* st, const Launch& L, int in_dtype, int w_dtype, int out_dtype, const void* in, const void* w,
+         void* out, const void* add1, const void* add2, const float* gmax, const int* len_src, const int* len_dst,
+         int B, int C, int T, int K, int mask, int flip) {
+    DtParams p{};
+    const int P = (K - 1) / 2;
+    p.w = w; p.out = out; p.add1 = add1; p.add2 = add2; p.gmax = gmax; p.len_src = len_src; p.len_dst = len_dst;
+    p.status = L.status;
+    p.B = B; p.C = C; p.T = T; p.K = K;
+    p.Pa = (P + 7) / 8 * 8; p.delta = p.Pa - P;
+    p.BB = B >= 32 ? 32 : 16; p.TBL = 128 / p.BB;
+    p.NK2 = (63 + K + p.delta + 15) / 16 * 16;
+    p.nxb = (p.NK2 + 63) / 64 + 1;
+    p.ntb = (T + 127) / 128; p.ngrp = (p.ntb + p.TBL - 1) / p.TBL; p.nchunks = (B + p.BB - 1) / p.BB;
+    p.tpc = p.nchunks * p.ngrp;
+    p.stage_bytes = p.nxb * 16384;
+    p.b_stride = ((p.NK2 + 63) / 64) * 8192;
+    p.nstages = std::min(DT_MAX_STAGES, (DT_AB_BYTES - 2 * p.b_stride) / p.stage_bytes);
+    p.mask = mask; p.flip = flip;
+    CUtensorMap mx;
+    const uint64_t dims[3] = {(uint64_t)T, (uint64_t)C, (uint64_t)B};
+    const uint32_t box[3] = {64, 1, (uint32_t)p.BB};
+    if (!tc_make_map(st, &mx, in_dtype, in, 3, dims, box)) return;
+    const int grid = std::min(std::max(1, st->sm_count), C);
+    if (in_dtype == F16 && w_dtype == F16) launch_dt<__half, __half, __half>(L, grid, mx, p);
+    else if (in_dtype == F16 && out_dtype == BF16) launch_dt<__half, __nv_bfloat16, __nv_bfloat16>(L, grid, mx, p);
+    else if (out_dtype == F16) launch_dt<__nv_bfloat16, __nv_bfloat16, __half>(L, grid, mx, p);
+    else launch_dt<__nv_bfloat16, __nv_bfloat16, __nv_bfloat16>(L, grid, mx, p);
+}
+
+}  // namespace
+
+bool dw_tma_supported(const TcState* st, int dtype, int B, int T, int K, int s) {
+    if (!st || !st->ready || dtype == F32 || s != 1) return false;
+    if (B < 16 || T % 8 != 0 || T < 64 || (K & 1) == 0) return false;
+    const int P = (K - 1) / 2, Pa = (P + 7) / 8 * 8;
+    return 63 + K + (Pa - P) <= 192;
+}
+
+void dw_tma_fwd(const TcState* st, const Launch& L, int dtype, int odt, const void* x, const void* wd, void* u,
+                const int* len_in, const int* len_out, int B, int C, int T, int K, int x_clean) {
+    KScope ks_(L, KC_DW_FWD, (double)B * C * T * (dtype_size(dtype) + dtype_size(odt)), 2.0 * B * C * T * K);
+    run(st, L, dtype, dtype, odt, x, wd, u, nullptr, nullptr, nullptr, len_in, len_out, B, C, T, K, x_clean ? 0 : 1, 0);
+}
+
+void dw_tma_dgrad(const TcState* st, const Launch& L, int dtype, int odt, const void* gu, const void* wd, void* dx,
+                  const void* add1, const void* add2, const float* gmax, const int* len_in, const int* len_out, int B,
+                  int C, int T, int K) {
+    KScope ks_(L, KC_DW_DGRAD, (double)B * C * T * (dtype_size(dtype) * (1 + (add1 ? 1 : 0) + (add2 ? 1 : 0)) + dtype_size(odt)),
+               2.0 * B * C * T * K);
+    // gu is produced by the library and is zero at and beyond len_out: no input masking
+    run(st, L, odt, dtype, dtype, gu, wd, dx, add1, add2, gmax, len_out, len_in, B, C, T, K, 0, 1);
+}
+
+}  // namespace sc

@@ -75,6 +75,15 @@ bool dw_wgrad_tc_supported(const TcState* st, int dtype, int B, int T, int K, in
 void dw_wgrad_tc(const TcState* st, const Launch& L, int dtype, int odt, const void* gu, const void* x, float* dwd,
                  float* partials, int accumulate, const float* gmax, const int* len_in, const int* len_out, int B,
                  int C, int T, int K, int x_clean);
+// TMA-fed tensor-core forms of the stride-1 depthwise forward / input gradient (16-bit types, B >= 16,
+// K + padding slack <= 129): same results as dw_fwd / dw_dgrad.  x_clean != 0 promises that x is already
+// zero at and beyond len_in.
+bool dw_tma_supported(const TcState* st, int dtype, int B, int T, int K, int s);
+void dw_tma_fwd(const TcState* st, const Launch& L, int dtype, int odt, const void* x, const void* wd, void* u,
+                const int* len_in, const int* len_out, int B, int C, int T, int K, int x_clean);
+void dw_tma_dgrad(const TcState* st, const Launch& L, int dtype, int odt, const void* gu, const void* wd, void* dx,
+                  const void* add1, const void* add2, const float* gmax, const int* len_in, const int* len_out, int B,
+                  int C, int T, int K);
 // Tensor-core forms of the stride-1 depthwise forward / input gradient (16-bit types, K <= 129).
 bool dw_tc_supported(int dtype, int T, int K, int s);
 void dw_tc_fwd(const Launch& L, int dtype, int odt, const void* x, const void* wd, void* u, const int* len_in,
