@@ -12,11 +12,16 @@
 // 128-byte swizzle; frames outside [0, T) are zero-filled by the TMA unit, which is the "same" padding.
 // Each input element is read from HBM once (window overlaps hit L2).  Rows of a tile are
 // (time block within a group of 128/BB, sample within a chunk of BB).
-// Warps: 0-7 epilogue (TMEM lane quarter w%4, column half w/4), 8-9 input masking (only when the input
+// Warps: 0-7 epilogue (TMEM lane quarter w%4, column half w/4), 8 input masking (only when the input
 // may be non-zero beyond a sample's length), 10-13 Toeplitz builders, 14 TMA producer (one box per lane),
-// 15 MMA issuer.  Accumulators are quadruple-buffered in tensor memory.  The epilogue transposes the
-// accumulator through shared memory so that global accesses are whole 32-byte sectors: already rounded
-// to the 16-bit output type when nothing is added to the result, in fp32 otherwise.
+// 15 and 9 MMA issuers for the even and odd tiles (a tile costs its issuer about twenty barrier, MMA and
+// commit instructions of a hundred cycles or more each, so two issuers alternate; their tiles use
+// different accumulators and stages).  Accumulators are quadruple-buffered in tensor memory.  In the epilogue a
+// lane owns 64 consecutive output frames of one row: it rounds them and parks the 128 bytes in shared
+// memory, and one TMA store per (64 frames x BB samples) box writes them out (whole 128-byte lines, no
+// per-thread global stores; frames beyond T and samples beyond B are clipped by the TMA unit).  When
+// something is added to the result the accumulator is instead transposed through shared memory in fp32
+// so that addends are read and results written as whole 32-byte sectors.
 // Every wait is bounded; on expiry the CTA raises the status word and leaves.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -38,7 +43,7 @@ constexpr int DT_THREADS = 512;
 constexpr int DT_AB_BYTES = 180224;        // A ring (3 x 48 KiB or 2 x 64 KiB) + two Toeplitz blocks (16 or 24 KiB each)
 constexpr int DT_ACC_COLS = 128;
 constexpr int DT_NACC = 4;
-constexpr int DT_STG_BYTES = 5120;         // per epilogue warp: 2 x 32 rows x 80 bytes (16-bit) or 32 rows x 144 bytes (fp32)
+constexpr int DT_STG_BYTES = 4608;         // per epilogue warp: 32 rows x 144 bytes (128 bytes of 16-bit values, or one fp32 chunk)
 constexpr int DT_WOFF = 80;                // index of tap 0 in the padded tap arrays
 constexpr int DT_WLEN = 288;
 constexpr int DT_MAX_STAGES = 3;
@@ -80,7 +85,7 @@ __device__ __forceinline__ void named_bar(int id, int nthreads) {
 // TI: type of the input tensor and of both MMA operands; TW: stored tap type; TO: output / addend type.
 template <typename TI, typename TW, typename TO>
 __global__ void __launch_bounds__(DT_THREADS, 1)
-dw_tma_kernel(const __grid_constant__ CUtensorMap mapX, DtParams p) {
+dw_tma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapO, DtParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint8_t* sB = smem + p.nstages * p.stage_bytes;                         // [2][b_stride], 1024-byte aligned
@@ -98,11 +103,12 @@ dw_tma_kernel(const __grid_constant__ CUtensorMap mapX, DtParams p) {
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
-        for (int s = 0; s < DT_MAX_STAGES; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&prep[s], 2); ptx::mbar_init(&empty[s], 1); }
+        for (int s = 0; s < DT_MAX_STAGES; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&prep[s], 1); ptx::mbar_init(&empty[s], 1); }
         for (int i = 0; i < DT_NACC; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 256); }
-        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&b_full[i], 4); ptx::mbar_init(&b_empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&b_full[i], 4); ptx::mbar_init(&b_empty[i], 2); }
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&mapX);
+        ptx::prefetch_tensormap(&mapO);
     }
     if (warp == 0) { ptx::tmem_alloc(tmem_slot, DT_NACC * DT_ACC_COLS); ptx::tmem_relinquish(); }
     ptx::tc_fence_before();
@@ -135,8 +141,9 @@ dw_tma_kernel(const __grid_constant__ CUtensorMap mapX, DtParams p) {
                 }
             }
         }
-    } else if (warp == 15) {
-        if (lane == 0) {                               // ---- MMA issuer ----
+    } else if (warp == 15 || warp == 9) {
+        if (lane == 0) {                               // ---- MMA issuers: warp 15 even tiles, warp 9 odd tiles ----
+            const int mine = (warp == 15) ? 0 : 1;
             const uint32_t idesc = ptx::instr_desc(FmtD<TI>::v, 0u, 0u, 128, 64);
             const uint64_t dk = ptx::smem_desc(0, 16, 1024);
             const uint32_t smem_a = ptx::smem_u32(smem), smem_b = ptx::smem_u32(sB);
@@ -146,6 +153,7 @@ dw_tma_kernel(const __grid_constant__ CUtensorMap mapX, DtParams p) {
                 const int bb = ci & 1;
                 if (!ptx::mbar_wait(&b_full[bb], (ci >> 1) & 1)) { raise_status(p.status, kErrTimeout); break; }
                 for (int t = 0; t < p.tpc; ++t, ++j) {
+                    if ((j & 1) != mine) { if (++s == p.nstages) { s = 0; ph ^= 1; } continue; }
                     const int buf = j & (DT_NACC - 1);
                     if (!ptx::mbar_wait(&acc_empty[buf], ((j / DT_NACC) & 1) ^ 1)) { raise_status(p.status, kErrTimeout); dead = true; break; }
                     if (!ptx::mbar_wait(p.mask ? &prep[s] : &full[s], ph)) { raise_status(p.status, kErrTimeout); dead = true; break; }
@@ -205,9 +213,9 @@ dw_tma_kernel(const __grid_constant__ CUtensorMap mapX, DtParams p) {
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&b_full[bb]);
         }
-    } else if (warp >= 8) {                            // ---- input masking (warps 8-9): rows mt and mt + 64 ----
+    } else if (warp == 8) {                            // ---- input masking (warp 8): rows mt, mt + 32, mt + 64, mt + 96 ----
         if (p.mask) {
-            const int mt = tid - 256;                  // 0 .. 63
+            const int mt = tid - 256;                  // 0 .. 31
             int s = 0, ph = 0; bool dead = false;
             for (int c = blockIdx.x; c < p.C && !dead; c += gridDim.x) {
                 for (int chunk = 0; chunk < p.nchunks && !dead; ++chunk) {
@@ -216,8 +224,8 @@ dw_tma_kernel(const __grid_constant__ CUtensorMap mapX, DtParams p) {
                         if (!ok) { if (lane == 0) raise_status(p.status, kErrTimeout); dead = true; break; }
                         bool wrote = false;
 #pragma unroll 1
-                        for (int rsel = 0; rsel < 2; ++rsel) {
-                            const int r = mt + 64 * rsel;
+                        for (int rsel = 0; rsel < 4; ++rsel) {
+                            const int r = mt + 32 * rsel;
                             const int tbl = r / p.BB, bi = r - tbl * p.BB;
                             const int b = chunk * p.BB + bi;
                             const int len = b < p.B ? min(p.len_src[b], p.T) : 0;
@@ -288,49 +296,57 @@ dw_tma_kernel(const __grid_constant__ CUtensorMap mapX, DtParams p) {
                     const uint32_t taddr = tmem + ((uint32_t)(wq * 32) << 16) + buf * DT_ACC_COLS + 64 * half;
                     const int tcol0 = 128 * (g * p.TBL) + 64 * half;            // frame of column 0 of this half, time block 0
                     if (!has_add) {
-                        // ---- round first, transpose 16-bit values: both 32-column chunks in one go ----
+                        // ---- nothing to add: round, park the lane's own 64 columns (one 128-byte row of a
+                        // 128-byte-swizzled box) in shared memory; one TMA store per box writes them out ----
                         uint32_t v0[32], v1[32];
                         ptx::tmem_ld32(taddr, v0);
                         ptx::tmem_ld32(taddr + 32, v1);
                         ptx::tmem_ld_wait();
                         const int nv = my_ld - (tcol0 + 128 * my_tbl);          // valid columns of this lane's row
+                        // the previous tile's stores must have read their source before it is overwritten
+                        if (lane == 0) ptx::bulk_wait_read();
                         __syncwarp();
+                        uint4* dst = reinterpret_cast<uint4*>(stg_all + warp * 4096 + lane * 128);
 #pragma unroll
                         for (int cc = 0; cc < 2; ++cc) {
                             uint32_t (&v)[32] = cc ? v1 : v0;
                             float f[32];
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) * inv;
+                            for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]);
+                            if (p.gmax) {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) f[i] *= inv;
+                            }
                             if (nv < 32 * cc + 32) {
 #pragma unroll
                                 for (int i = 0; i < 32; ++i) if (32 * cc + i >= nv) f[i] = 0.f;
                             }
                             if (std::is_same<TO, __half>::value) {   // range guard: clamp only when hit
-                                float m = 0.f;
+                                float m4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                                for (int i = 0; i < 32; ++i) m = fmaxf(m, fabsf(f[i]));
+                                for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], fabsf(f[i]));
+                                const float m = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
                                 if (m > 65504.f) {
 #pragma unroll
                                     for (int i = 0; i < 32; ++i) f[i] = fminf(fmaxf(f[i], -65504.f), 65504.f);
                                 }
                                 amax = fmaxf(amax, m);
                             }
-                            uint4* dst = reinterpret_cast<uint4*>(stg + cc * 2560 + lane * 80);
 #pragma unroll
-                            for (int i = 0; i < 4; ++i)
-                                dst[i] = make_uint4(pack2<TO>(f[8 * i], f[8 * i + 1]), pack2<TO>(f[8 * i + 2], f[8 * i + 3]),
-                                                    pack2<TO>(f[8 * i + 4], f[8 * i + 5]), pack2<TO>(f[8 * i + 6], f[8 * i + 7]));
+                            for (int i = 0; i < 4; ++i)     // 16-byte slot 4 cc + i of the row, swizzled by the row index
+                                dst[(4 * cc + i) ^ (lane & 7)] =
+                                    make_uint4(pack2<TO>(f[8 * i], f[8 * i + 1]), pack2<TO>(f[8 * i + 2], f[8 * i + 3]),
+                                               pack2<TO>(f[8 * i + 4], f[8 * i + 5]), pack2<TO>(f[8 * i + 6], f[8 * i + 7]));
                         }
+                        ptx::fence_proxy_async();
                         __syncwarp();
-#pragma unroll
-                        for (int cc = 0; cc < 2; ++cc) {
-#pragma unroll
-                            for (int it = 0; it < 4; ++it) {
-                                const int t = tcol0 + 128 * tbl_of[it] + 32 * cc + cs;
-                                if (ld_of[it] < 0 || t >= p.T) continue;
-                                const uint4 x = *reinterpret_cast<const uint4*>(stg + cc * 2560 + (it * 8 + rr) * 80 + 2 * cs);
-                                *reinterpret_cast<uint4*>(out + base_of[it] + t) = x;
+                        if (lane == 0) {
+                            // the warp's 32 rows are 32 / BB boxes of (64 frames x 1 channel x BB samples)
+                            for (int i = 0; i < 32 / p.BB; ++i) {
+                                const int x = tcol0 + 128 * ((wq * 32) / p.BB + i);
+                                if (x < p.T) ptx::tma_store_3d(&mapO, stg_all + warp * 4096 + i * p.BB * 128, x, c, chunk * p.BB);
                             }
+                            ptx::bulk_commit();
                         }
                     } else {
                         // ---- something is added to the result: transpose fp32, add, then round ----
@@ -393,6 +409,7 @@ dw_tma_kernel(const __grid_constant__ CUtensorMap mapX, DtParams p) {
             }
         }
     done:
+        ptx::bulk_wait_all();                              // this thread's output stores have completed
         if (amax > 65504.f) raise_status(p.status, kErrRange);
     }
     ptx::tc_fence_before();
@@ -404,14 +421,14 @@ constexpr int kDtSmem = 1024 + DT_AB_BYTES + 8 * DT_STG_BYTES + 2 * DT_WLEN * 2 
 static_assert(kDtSmem <= 232448, "shared memory per CTA");
 
 template <typename TI, typename TW, typename TO>
-void launch_dt(const Launch& L, int grid, const CUtensorMap& mx, const DtParams& p) {
+void launch_dt(const Launch& L, int grid, const CUtensorMap& mx, const CUtensorMap& mo, const DtParams& p) {
     auto kern = dw_tma_kernel<TI, TW, TO>;
     static bool configured = false;
     if (!configured) {
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kDtSmem);
         configured = true;
     }
-    kern<<<grid, DT_THREADS, kDtSmem, L.stream>>>(mx, p);
+    kern<<<grid, DT_THREADS, kDtSmem, L.stream>>>(mx, mo, p);
     L.count();
 }
 
@@ -437,12 +454,13 @@ void run(const TcState* st, const Launch& L, int in_dtype, int w_dtype, int out_
     CUtensorMap mx;
     const uint64_t dims[3] = {(uint64_t)T, (uint64_t)C, (uint64_t)B};
     const uint32_t box[3] = {64, 1, (uint32_t)p.BB};
-    if (!tc_make_map(st, &mx, in_dtype, in, 3, dims, box)) return;
+    CUtensorMap mo;
+    if (!tc_make_map(st, &mx, in_dtype, in, 3, dims, box) || !tc_make_map(st, &mo, out_dtype, out, 3, dims, box)) return;
     const int grid = std::min(std::max(1, st->sm_count), C);
-    if (in_dtype == F16 && w_dtype == F16) launch_dt<__half, __half, __half>(L, grid, mx, p);
-    else if (in_dtype == F16 && out_dtype == BF16) launch_dt<__half, __nv_bfloat16, __nv_bfloat16>(L, grid, mx, p);
-    else if (out_dtype == F16) launch_dt<__nv_bfloat16, __nv_bfloat16, __half>(L, grid, mx, p);
-    else launch_dt<__nv_bfloat16, __nv_bfloat16, __nv_bfloat16>(L, grid, mx, p);
+    if (in_dtype == F16 && w_dtype == F16) launch_dt<__half, __half, __half>(L, grid, mx, mo, p);
+    else if (in_dtype == F16 && out_dtype == BF16) launch_dt<__half, __nv_bfloat16, __nv_bfloat16>(L, grid, mx, mo, p);
+    else if (out_dtype == F16) launch_dt<__nv_bfloat16, __nv_bfloat16, __half>(L, grid, mx, mo, p);
+    else launch_dt<__nv_bfloat16, __nv_bfloat16, __nv_bfloat16>(L, grid, mx, mo, p);
 }
 
 }  // namespace
