@@ -86,32 +86,35 @@ bn_stats_kernel(const T* __restrict__ v, const int* __restrict__ len_out, int nr
     if (lane == 0) partials[row] = make_float2(s[0], q[0]);
 }
 
-// 32 channels x 32 part-slices per CTA.  Pass 1 sums the partial sums (slice s takes parts s, s+32, ...
-// in increasing order; the slice results are then added in slice order), which gives the mean; pass 2
-// sums M2_p + n_p (mean_p - mean)^2 the same way.  The order is fixed, so the result is bit-repeatable,
-// and no term depends on the previous one, so the loads and divisions pipeline.
-constexpr int kFinSlices = 32;
-__global__ void __launch_bounds__(32 * kFinSlices)
+// One warp per channel.  Lane l takes parts l, l + 32, ... in increasing order and the 32 lane results
+// are combined by a fixed butterfly, so the result is bit-repeatable.  Pass 1 sums the partial sums,
+// which gives the mean; pass 2 sums M2_p + n_p (mean_p - mean)^2 = M2_p + (sum_p - n_p mean)^2 / n_p.
+// No term depends on the previous one, so a lane's loads are all in flight together; the parts are
+// kept in registers between the passes when there are at most kFinKeep per lane.
+constexpr int kFinKeep = 8;
+constexpr int kFinWarps = 8;
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__global__ void __launch_bounds__(32 * kFinWarps)
 bn_finalize_kernel(const float2* __restrict__ partials, int parts_per_b, int tile_w,
                    const int* __restrict__ len_out, const int* __restrict__ nvalid, int B,
                    int C, float eps, float momentum, float* __restrict__ mean_out,
                    float* __restrict__ invstd_out, float* running_mean, float* running_var) {
-    __shared__ double sh[kFinSlices][33];
-    __shared__ double sh_mean[32];
-    const int cx = threadIdx.x & 31, sl = threadIdx.x >> 5;
-    const int o = blockIdx.x * 32 + cx;
+    const int lane = threadIdx.x & 31;
+    const int o = blockIdx.x * kFinWarps + (threadIdx.x >> 5);
+    if (o >= C) return;
     const int nparts = B * parts_per_b;
     const double N = (double)(*nvalid);
-    // this thread's parts: sl, sl+32, ...; the first eight are kept in registers between the two passes
-    constexpr int kKeep = 8;
-    float2 keep[kKeep];
-    int cnts[kKeep];
+    float2 keep[kFinKeep];
+    int cnts[kFinKeep];
 #pragma unroll
-    for (int i = 0; i < kKeep; ++i) {
-        const int pi = sl + i * kFinSlices;
-        cnts[i] = 0;
-        keep[i] = make_float2(0.f, 0.f);
-        if (o < C && pi < nparts) {
+    for (int i = 0; i < kFinKeep; ++i) {
+        const int pi = lane + 32 * i;
+        cnts[i] = 0; keep[i] = make_float2(0.f, 0.f);
+        if (pi < nparts) {
             const int b = pi / parts_per_b, j = pi - b * parts_per_b;
             cnts[i] = max(0, min(len_out[b] - j * tile_w, tile_w));
             if (cnts[i] > 0) keep[i] = partials[(size_t)pi * C + o];
@@ -119,42 +122,29 @@ bn_finalize_kernel(const float2* __restrict__ partials, int parts_per_b, int til
     }
     double s1 = 0.0;
 #pragma unroll
-    for (int i = 0; i < kKeep; ++i) if (cnts[i] > 0) s1 += (double)keep[i].x;
-    if (o < C)
-        for (int pi = sl + kKeep * kFinSlices; pi < nparts; pi += kFinSlices) {
-            const int b = pi / parts_per_b, j = pi - b * parts_per_b;
-            if (len_out[b] - j * tile_w > 0) s1 += (double)partials[(size_t)pi * C + o].x;
-        }
-    sh[sl][cx] = s1;
-    __syncthreads();
-    if (sl == 0) {
-        double t = 0.0;
-        for (int k = 0; k < kFinSlices; ++k) t += sh[k][cx];
-        sh_mean[cx] = N > 0 ? t / N : 0.0;
+    for (int i = 0; i < kFinKeep; ++i) if (cnts[i] > 0) s1 += (double)keep[i].x;
+    for (int pi = lane + 32 * kFinKeep; pi < nparts; pi += 32) {
+        const int b = pi / parts_per_b, j = pi - b * parts_per_b;
+        if (len_out[b] - j * tile_w > 0) s1 += (double)partials[(size_t)pi * C + o].x;
     }
-    __syncthreads();
-    const double mean = sh_mean[cx];
+    const double mean = N > 0 ? warp_sum_d(s1) / N : 0.0;
     double q = 0.0;
 #pragma unroll
-    for (int i = 0; i < kKeep; ++i)
+    for (int i = 0; i < kFinKeep; ++i)
         if (cnts[i] > 0) {
-            const double d = (double)keep[i].x / (double)cnts[i] - mean;
-            q += (double)keep[i].y + (double)cnts[i] * d * d;
+            const double d = (double)keep[i].x - (double)cnts[i] * mean;
+            q += (double)keep[i].y + (double)((float)(d * d) / (float)cnts[i]);
         }
-    if (o < C)
-        for (int pi = sl + kKeep * kFinSlices; pi < nparts; pi += kFinSlices) {
-            const int b = pi / parts_per_b, j = pi - b * parts_per_b;
-            const int cnt = min(len_out[b] - j * tile_w, tile_w);
-            if (cnt <= 0) continue;
-            const float2 p = partials[(size_t)pi * C + o];
-            const double d = (double)p.x / (double)cnt - mean;
-            q += (double)p.y + (double)cnt * d * d;
-        }
-    sh[sl][cx] = q;
-    __syncthreads();
-    if (sl != 0 || o >= C) return;
-    double m2 = 0.0;
-    for (int k = 0; k < kFinSlices; ++k) m2 += sh[k][cx];
+    for (int pi = lane + 32 * kFinKeep; pi < nparts; pi += 32) {
+        const int b = pi / parts_per_b, j = pi - b * parts_per_b;
+        const int cnt = min(len_out[b] - j * tile_w, tile_w);
+        if (cnt <= 0) continue;
+        const float2 p = partials[(size_t)pi * C + o];
+        const double d = (double)p.x - (double)cnt * mean;
+        q += (double)p.y + (double)((float)(d * d) / (float)cnt);
+    }
+    const double m2 = warp_sum_d(q);
+    if (lane != 0) return;
     const double var = N > 0 ? m2 / N : 0.0;
     const float invstd = (float)(1.0 / sqrt(var + (double)eps));
     const float mu = (float)mean;
@@ -290,33 +280,34 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_reduce_kernel(BnBwdArgs a)
     }
 }
 
-__global__ void __launch_bounds__(32 * kFinSlices)
+// One warp per channel: lane l takes the (sample, slot) partials l, l + 32, ... in increasing order; the
+// lane sums are combined by a fixed butterfly.
+__global__ void __launch_bounds__(32 * kFinWarps)
 bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const float* gamma_r, float* dgamma, float* dbeta,
                        float* dgamma_r, float* dbeta_r, float* dbias, int accumulate) {
-    __shared__ float4 shs[kFinSlices][32];
-    const int cx = threadIdx.x & 31, sl = threadIdx.x >> 5;
-    const int o = blockIdx.x * 32 + cx;
-    __shared__ float shmax[kFinSlices][32];
+    const int lane = threadIdx.x & 31;
+    const int o = blockIdx.x * kFinWarps + (threadIdx.x >> 5);
+    if (o >= a.C) return;
     double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
     float amax = 0.f;
-    if (o < a.C) {
+    {
         const int vpr = a.Tp / 8;
         const int np = a.B * a.nslots;
-        for (int base = sl; base < np; base += 8 * kFinSlices) {
-            float4 pv[8]; float am[8]; bool use[8];
+        for (int base = lane; base < np; base += 8 * 32) {
+            float4 pv[8]; float am[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) {          // issue every load before the first add
-                const int pi = base + i * kFinSlices;
-                use[i] = pi < np;
+                const int pi = base + i * 32;
+                bool use = pi < np;
                 pv[i] = make_float4(0.f, 0.f, 0.f, 0.f); am[i] = 0.f;
-                if (use[i]) {
+                if (use) {
                     const int b = pi / a.nslots, slot = pi - b * a.nslots;
                     const long long r = (long long)b * a.C + o;
                     if (a.nslots > 1) {      // slots in use for this row (see bn_bwd_reduce_fast_kernel)
                         const int used = (int)((((r + 1) * vpr - 1) >> 5) - ((r * vpr) >> 5)) + 1;
-                        use[i] = slot < used;
+                        use = slot < used;
                     }
-                    if (use[i]) {
+                    if (use) {
                         pv[i] = a.partials[(size_t)r * a.nslots + slot];
                         if (a.gmax) am[i] = a.amax_part[(size_t)r * a.nslots + slot];
                     }
@@ -329,15 +320,9 @@ bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const float* gamma_r, fl
             }
         }
     }
-    shs[sl][cx] = make_float4((float)s0, (float)s1, (float)s2, (float)s3);
-    shmax[sl][cx] = amax;
-    __syncthreads();
-    if (sl != 0 || o >= a.C) return;
-    for (int k = 1; k < kFinSlices; ++k) {
-        const float4 t = shs[k][cx];
-        s0 += t.x; s1 += t.y; s2 += t.z; s3 += t.w;
-        amax = fmaxf(amax, shmax[k][cx]);
-    }
+    s0 = warp_sum_d(s0); s1 = warp_sum_d(s1); s2 = warp_sum_d(s2); s3 = warp_sum_d(s3);
+    amax = warp_max(amax);
+    if (lane != 0) return;
     const float N = (float)(*a.nvalid);
     if (a.gmax) {
         // |gv| <= |k| (max|ga| + |c1| + max|vhat| |c2|) and max|vhat| <= sqrt(N); a maximum is order-free,
@@ -448,9 +433,17 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_fast_kernel(BnBwdArgs a, int
     if (t0 < len) {
         float g[8], y[8], vn[8], vnr[8];
         ld8<T>((const T*)a.g + off, g);
-        ld8<T>((const T*)a.y + off, y);
         ld8<NT>((const NT*)a.vhat + off, vn);
         if (RES == 2) ld8<NT>((const NT*)a.vhat_r + off, vnr);
+        if (RES == 0) {
+            // without a residual the forward output is relu(gamma * vhat + beta) of the STORED vhat, rounded
+            // to the activation type: the gate is recomputed from vhat and the output need not be read
+            const float ga_ = a.gamma[o], be_ = a.beta[o];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) y[i] = round_io<T>(fmaf(ga_, vn[i], be_));
+        } else {
+            ld8<T>((const T*)a.y + off, y);
+        }
         float4 cf = a.coef[o];
         if (a.gmax) cf.x *= pow2_scale(*a.gmax);
         float4 cr = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -494,9 +487,16 @@ __global__ void __launch_bounds__(256) bn_bwd_reduce_fast_kernel(BnBwdArgs a, in
         const size_t off = (size_t)row * a.Tp + t0;
         float g[8], y[8], vn[8], vnr[8];
         ld8<T>((const T*)a.g + off, g);
-        ld8<T>((const T*)a.y + off, y);
         ld8<NT>((const NT*)a.vhat + off, vn);
         if (RES == 2) ld8<NT>((const NT*)a.vhat_r + off, vnr);
+        if (RES == 0) {          // gate from the stored vhat (see bn_bwd_apply_fast_kernel)
+            const int o = row - b * a.C;
+            const float ga_ = a.gamma[o], be_ = a.beta[o];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) y[i] = round_io<T>(fmaf(ga_, vn[i], be_));
+        } else {
+            ld8<T>((const T*)a.y + off, y);
+        }
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const float ga = (t0 + i < len && y[i] > 0.f) ? g[i] : 0.f;
@@ -584,7 +584,7 @@ void bn_finalize(const Launch& L, const float2* partials, int parts_per_b, int t
                  const int* nvalid, int B, int C, float eps, float momentum, float* mean, float* invstd,
                  float* running_mean, float* running_var) {
     KScope ks_(L, KC_BN_FINALIZE, 8.0 * B * parts_per_b * C, 0.0);
-    bn_finalize_kernel<<<(C + 31) / 32, 32 * kFinSlices, 0, L.stream>>>(partials, parts_per_b, tile_w, len_out, nvalid, B, C,
+    bn_finalize_kernel<<<(C + kFinWarps - 1) / kFinWarps, 32 * kFinWarps, 0, L.stream>>>(partials, parts_per_b, tile_w, len_out, nvalid, B, C,
                                                             eps, momentum, mean, invstd, running_mean, running_var);
     L.count();
 }
@@ -608,12 +608,13 @@ void bn_apply(const Launch& L, int dtype, const ApplyArgs& a) {
 void bn_bwd_reduce(const Launch& L, int dtype, BnBwdArgs& a) {
     a.nslots = 1;
     if (a.Tp % 8 == 0 && a.Tp >= 256 && a.has_bn && a.has_relu && a.res_before_relu) {
-        KScope ks2_(L, KC_BN_BWD_REDUCE, (double)a.B * a.C * a.Tp * (dtype_size(dtype) * 2 + dtype_size(ntype_of(dtype)) * (a.residual == 2 ? 2 : 1)), 0.0);
+        KScope ks2_(L, KC_BN_BWD_REDUCE, (double)a.B * a.C * a.Tp * (dtype_size(dtype) * (a.residual == 0 ? 1 : 2) + dtype_size(ntype_of(dtype)) * (a.residual == 2 ? 2 : 1)), 0.0);
         const int vpr = a.Tp / 8;
         a.nslots = bn_bwd_max_slots(a.Tp);
         const long long total = (long long)a.B * a.C * vpr;
         const unsigned grid = (unsigned)((total + 255) / 256);
         if (a.residual == 2) { SC_DISPATCH3(dtype, (bn_bwd_reduce_fast_kernel<T, NT, 2><<<grid, 256, 0, L.stream>>>(a, vpr, total))); }
+        else if (a.residual == 1) { SC_DISPATCH3(dtype, (bn_bwd_reduce_fast_kernel<T, NT, 1><<<grid, 256, 0, L.stream>>>(a, vpr, total))); }
         else { SC_DISPATCH3(dtype, (bn_bwd_reduce_fast_kernel<T, NT, 0><<<grid, 256, 0, L.stream>>>(a, vpr, total))); }
         L.count();
         return;
@@ -627,13 +628,14 @@ void bn_bwd_finalize(const Launch& L, const BnBwdArgs& a, const float* gamma, co
                      float* dgamma, float* dbeta, float* dgamma_r, float* dbeta_r, float* dbias,
                      int accumulate) {
     KScope ks_(L, KC_BN_BWD_FINALIZE, 16.0 * a.B * a.C, 0.0);
-    bn_bwd_finalize_kernel<<<(a.C + 31) / 32, 32 * kFinSlices, 0, L.stream>>>(a, gamma, gamma_r, dgamma, dbeta, dgamma_r,
+    bn_bwd_finalize_kernel<<<(a.C + kFinWarps - 1) / kFinWarps, 32 * kFinWarps, 0, L.stream>>>(a, gamma, gamma_r, dgamma, dbeta, dgamma_r,
                                                                   dbeta_r, dbias, accumulate);
     L.count();
 }
 
 void bn_bwd_apply(const Launch& L, int dtype, const BnBwdArgs& a) {
-    KScope ks_(L, KC_BN_BWD_APPLY, (double)a.B * a.C * a.Tp * (dtype_size(dtype) * (a.has_relu && a.res_before_relu ? 2 : 1) + (a.has_bn ? dtype_size(ntype_of(dtype)) : 0) + (a.residual == 2 ? dtype_size(ntype_of(dtype)) : 0) + dtype_size(dtype) * (1 + (a.residual != 0 ? 1 : 0))), 0.0);
+    const bool fast_apply = a.Tp % 8 == 0 && a.has_bn && a.has_relu && a.res_before_relu;
+    KScope ks_(L, KC_BN_BWD_APPLY, (double)a.B * a.C * a.Tp * (dtype_size(dtype) * (a.has_relu && a.res_before_relu && !(fast_apply && a.residual == 0) ? 2 : 1) + (a.has_bn ? dtype_size(ntype_of(dtype)) : 0) + (a.residual == 2 ? dtype_size(ntype_of(dtype)) : 0) + dtype_size(dtype) * (1 + (a.residual != 0 ? 1 : 0))), 0.0);
     if (a.Tp % 8 == 0 && a.has_bn && a.has_relu && a.res_before_relu) {
         const int vpr = a.Tp / 8;
         const long long total = (long long)a.B * a.C * vpr;

@@ -31,8 +31,8 @@
 namespace sc {
 namespace {
 
-constexpr int WT_STAGES = 6;
-constexpr int WT_STAGE_BYTES = 24576;      // 128 frames of gu + up to 256 frames of x, 32 samples, 16-bit
+constexpr int WT_STAGES = 4;               // at most; 3 when the x window needs four 64-frame boxes
+constexpr int WT_RING_BYTES = 163840;      // stage = two time blocks x (128 frames of gu + 192 or 256 frames of x) x 32 samples
 constexpr int WT_THREADS = 448;
 constexpr int WT_ACC_COLS = 256;
 constexpr int WT_MAX_CHUNKS = 64;
@@ -42,11 +42,13 @@ constexpr int WT_XW = 128;
 
 struct WtParams {
     float* partials; const int* len_in; const int* len_out; int* status;
+    float* dwd; const float* gmax; int accumulate;   // used when a channel is not split: the result is written directly
     int B, C, T, K, Pa, delta;
     int BB;              // samples per contraction step (16 or 32)
     int nxb;             // 64-frame boxes in the x window
     int N;               // accumulator columns in use
-    int nchunks, ntb;    // contraction steps per channel = nchunks * ntb
+    int nchunks, ntb;    // contraction steps per channel = nchunks * ntb; a step is a PAIR of 128-frame time blocks
+    int nstages, stage_bytes;
     int S, ks_per_split; // splits per channel
     int units;           // C * S
     int prep;            // 1: the x window needs converting and/or masking
@@ -98,7 +100,7 @@ struct StepWalk {
         cl = chunk < WT_MAX_CHUNKS ? chunk_len[chunk] : (1 << 30);
     }
     __device__ __forceinline__ bool more() const { return ks < ks1; }
-    __device__ __forceinline__ bool on() const { return ks == ks0 || tb * 128 < cl; }
+    __device__ __forceinline__ bool on() const { return ks == ks0 || tb * 256 < cl; }
     __device__ __forceinline__ void next() {
         ++ks;
         if (++tb == ntb) { tb = 0; ++chunk; cl = chunk < WT_MAX_CHUNKS ? chunk_len[chunk] : (1 << 30); }
@@ -106,8 +108,9 @@ struct StepWalk {
 };
 // ring position: stage index and phase parity, advanced without a modulo
 struct Ring {
-    int s = 0, ph = 0;
-    __device__ __forceinline__ void advance() { if (++s == WT_STAGES) { s = 0; ph ^= 1; } }
+    int s = 0, ph = 0, n;
+    __device__ __forceinline__ explicit Ring(int nstages) : n(nstages) {}
+    __device__ __forceinline__ void advance() { if (++s == n) { s = 0; ph ^= 1; } }
 };
 
 template <typename TG, typename TX>
@@ -115,7 +118,7 @@ __global__ void __launch_bounds__(WT_THREADS, 1)
 dw_wgrad_tc_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_constant__ CUtensorMap mapX, WtParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + WT_STAGES * WT_STAGE_BYTES);
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + WT_RING_BYTES);
     uint64_t* conv = full + WT_STAGES;
     uint64_t* empty = conv + WT_STAGES;
     uint64_t* acc_full = empty + WT_STAGES;    // [2]
@@ -123,13 +126,14 @@ dw_wgrad_tc_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_consta
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     int* chunk_len = reinterpret_cast<int*>(tmem_slot + 2);                 // [WT_MAX_CHUNKS]
     // staging rows are read with 16-byte loads: keep the block 16-byte aligned (barriers etc. take < 512 bytes)
-    float* stg_all = reinterpret_cast<float*>(smem + WT_STAGES * WT_STAGE_BYTES + 512);   // [4][63][36]
+    float* stg_all = reinterpret_cast<float*>(smem + WT_RING_BYTES + 512);   // [4][63][36]
     float* xw = stg_all + 4 * WT_STG_FLOATS;                                // [4][160]
     int* epi_fail = reinterpret_cast<int*>(xw + 4 * WT_XW);                 // set when an epilogue wait expired
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g_bytes = 2 * p.BB * 128, box_bytes = p.BB * 128;
-    const int stage_tx = g_bytes + p.nxb * box_bytes;
+    const int x_bytes = p.nxb * box_bytes;
+    const int stage_tx = 2 * (g_bytes + x_bytes);
 
     if (tid == 0) {
         for (int s = 0; s < WT_STAGES; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&conv[s], 4); ptx::mbar_init(&empty[s], 1); }
@@ -155,13 +159,16 @@ dw_wgrad_tc_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_consta
     const int ks_total = p.nchunks * p.ntb;
 
     if (warp == 12) {                                  // ---- TMA producer: one box per lane ----
-        Ring rg; bool dead = false;
-        const bool is_g = lane < 2;
-        const int q = lane - 2;
-        const bool active = lane < 2 + p.nxb;
+        Ring rg(p.nstages); bool dead = false;
+        // lane -> (time block of the pair, box): boxes 0-1 are gu, boxes 2.. the x window
+        const int per = 2 + p.nxb;
+        const int hb = lane / per, bx = lane - hb * per;
+        const bool is_g = bx < 2;
+        const int q = bx - 2;
+        const bool active = lane < 2 * per;
         const void* map = is_g ? (const void*)&mapG : (const void*)&mapX;
-        const int dst_off = is_g ? lane * box_bytes : g_bytes + q * box_bytes;
-        const int t_off = is_g ? 64 * lane : 64 * q - p.Pa;
+        const int dst_off = is_g ? hb * g_bytes + bx * box_bytes : 2 * g_bytes + hb * x_bytes + q * box_bytes;
+        const int t_off = 128 * hb + (is_g ? 64 * bx : 64 * q - p.Pa);
         for (int unit = blockIdx.x; unit < p.units && !dead; unit += gridDim.x) {
             const int c = unit / p.S, sp = unit - c * p.S;
             StepWalk w; w.begin(sp, p.ks_per_split, ks_total, p.ntb, chunk_len);
@@ -175,7 +182,7 @@ dw_wgrad_tc_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_consta
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) { if (lane == 0) raise_status(p.status, kErrTimeout); dead = true; break; }
                 if (active)
-                    ptx::tma_load_3d(smem + rg.s * WT_STAGE_BYTES + dst_off, map, &full[rg.s], w.tb * 128 + t_off, c,
+                    ptx::tma_load_3d(smem + rg.s * p.stage_bytes + dst_off, map, &full[rg.s], w.tb * 256 + t_off, c,
                                      w.chunk * p.BB);
                 rg.advance();
             }
@@ -187,7 +194,7 @@ dw_wgrad_tc_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_consta
             const uint64_t dbase = ptx::smem_desc(0, box_bytes, 1024);
             const uint32_t smem_a = ptx::smem_u32(smem);
             const int nkk = p.BB / 16;
-            Ring rg; int j = 0; bool dead = false;
+            Ring rg(p.nstages); int j = 0; bool dead = false;
             for (int unit = blockIdx.x; unit < p.units && !dead; unit += gridDim.x, ++j) {
                 const int c = unit / p.S, sp = unit - c * p.S;
                 (void)c;
@@ -203,12 +210,15 @@ dw_wgrad_tc_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_consta
                         raise_status(p.status, kErrTimeout); dead = true; break;
                     }
                     ptx::tc_fence_after();
-                    const uint32_t aG = smem_a + rg.s * WT_STAGE_BYTES;
-                    uint64_t dG = dbase | (uint64_t)((aG & 0x3FFFFu) >> 4);
-                    uint64_t dX = dbase | (uint64_t)(((aG + g_bytes) & 0x3FFFFu) >> 4);
-                    for (int kk = 0; kk < nkk; ++kk) {
-                        ptx::mma_f16(tmem + buf * WT_ACC_COLS, dG, dX, idesc, accum);
-                        accum = 1u; dG += 2048 >> 4; dX += 2048 >> 4;
+                    const uint32_t aG = smem_a + rg.s * p.stage_bytes;
+#pragma unroll 1
+                    for (int hb = 0; hb < 2; ++hb) {
+                        uint64_t dG = dbase | (uint64_t)(((aG + hb * g_bytes) & 0x3FFFFu) >> 4);
+                        uint64_t dX = dbase | (uint64_t)(((aG + 2 * g_bytes + hb * x_bytes) & 0x3FFFFu) >> 4);
+                        for (int kk = 0; kk < nkk; ++kk) {
+                            ptx::mma_f16(tmem + buf * WT_ACC_COLS, dG, dX, idesc, accum);
+                            accum = 1u; dG += 2048 >> 4; dX += 2048 >> 4;
+                        }
                     }
                     ptx::mma_commit(&empty[rg.s]);
                     rg.advance();
@@ -228,7 +238,7 @@ dw_wgrad_tc_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_consta
         const int nvec_t = (p.nxb * p.BB) >> 4;                 // vectors per thread and step (<= 8)
         const int r0 = ctid >> 3;
         const int toff = 8 * ((ctid & 7) ^ (r0 & 7));
-        Ring rg; int it = 0; bool dead = false; float amax = 0.f;
+        Ring rg(p.nstages); int it = 0; bool dead = false; float amax = 0.f;
         for (int unit = blockIdx.x; unit < p.units && !dead; unit += gridDim.x) {
             const int c = unit / p.S, sp = unit - c * p.S;
             (void)c;
@@ -239,24 +249,27 @@ dw_wgrad_tc_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_consta
                     const bool ok = ptx::mbar_wait_warp(&full[rg.s], rg.ph);
                     if (!ok) { if (lane == 0) raise_status(p.status, kErrTimeout); dead = true; break; }
                     if (p.prep) {
-                        uint4* sX = reinterpret_cast<uint4*>(smem + rg.s * WT_STAGE_BYTES + g_bytes);
-                        const int tx0 = w.tb * 128 - p.Pa + toff, b0 = w.chunk * p.BB;
-                        // frames left before the sample's end, for this thread's (at most two) rows
-                        int left0 = 1 << 30, left1 = 1 << 30;
-                        if (p.mask) {
-                            const int ba = b0 + r0, bb = b0 + r0 + 16;
-                            left0 = (ba < p.B ? min(p.len_in[ba], p.T) : 0) - tx0;
-                            left1 = (bb < p.B ? min(p.len_in[bb], p.T) : 0) - tx0;
-                        }
-                        uint4 raw[8];
+#pragma unroll 1
+                        for (int hb = 0; hb < 2; ++hb) {
+                            uint4* sX = reinterpret_cast<uint4*>(smem + rg.s * p.stage_bytes + 2 * g_bytes + hb * x_bytes);
+                            const int tx0 = w.tb * 256 + 128 * hb - p.Pa + toff, b0 = w.chunk * p.BB;
+                            // frames left before the sample's end, for this thread's (at most two) rows
+                            int left0 = 1 << 30, left1 = 1 << 30;
+                            if (p.mask) {
+                                const int ba = b0 + r0, bb = b0 + r0 + 16;
+                                left0 = (ba < p.B ? min(p.len_in[ba], p.T) : 0) - tx0;
+                                left1 = (bb < p.B ? min(p.len_in[bb], p.T) : 0) - tx0;
+                            }
+                            uint4 raw[8];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) if (i < nvec_t) raw[i] = sX[ctid + 128 * i];
+                            for (int i = 0; i < 8; ++i) if (i < nvec_t) raw[i] = sX[ctid + 128 * i];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            if (i < nvec_t) {
-                                const int v = ctid + 128 * i;
-                                const int left = (((v >> 3) & 16) & (p.BB - 1)) ? left1 : left0;
-                                sX[v] = prep8<TG, TX>(raw[i], left - 64 * (v >> (3 + lb)), amax);
+                            for (int i = 0; i < 8; ++i) {
+                                if (i < nvec_t) {
+                                    const int v = ctid + 128 * i;
+                                    const int left = (((v >> 3) & 16) & (p.BB - 1)) ? left1 : left0;
+                                    sX[v] = prep8<TG, TX>(raw[i], left - 64 * (v >> (3 + lb)), amax);
+                                }
                             }
                         }
                         ptx::fence_proxy_async();
@@ -324,7 +337,13 @@ dw_wgrad_tc_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_consta
             bar_sync_named(1, 128);
             if (tid < p.K) {
                 const float v = ((xw[tid] + xw[WT_XW + tid]) + xw[2 * WT_XW + tid]) + xw[3 * WT_XW + tid];
-                p.partials[((size_t)sp * p.C + c) * p.K + tid] = v;
+                if (p.S == 1) {        // no split: finish here (undo the gradient scale, accumulate) and skip the reduction pass
+                    const float r = p.gmax ? v * (1.f / pow2_scale(*p.gmax)) : v;
+                    float* dst = p.dwd + (size_t)c * p.K + tid;
+                    *dst = p.accumulate ? *dst + r : r;
+                } else {
+                    p.partials[((size_t)sp * p.C + c) * p.K + tid] = v;
+                }
             }
             bar_sync_named(1, 128);
         }
@@ -334,7 +353,7 @@ dw_wgrad_tc_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_consta
     if (warp == 0) ptx::tmem_dealloc(tmem, 2 * WT_ACC_COLS);
 }
 
-constexpr int kWtSmem = WT_STAGES * WT_STAGE_BYTES + 1024 /* alignment */ + 512 /* barriers, chunk lengths */ +
+constexpr int kWtSmem = WT_RING_BYTES + 1024 /* alignment */ + 512 /* barriers, chunk lengths */ +
                         4 * WT_STG_FLOATS * 4 + 4 * WT_XW * 4 + 16;
 static_assert((3 * WT_STAGES + 4) * 8 + 8 + WT_MAX_CHUNKS * 4 <= 512, "barrier block");
 
@@ -367,13 +386,16 @@ void dw_wgrad_tc(const TcState* st, const Launch& L, int dtype, int odt, const v
         KScope ks_(L, KC_DW_WGRAD, (double)B * C * T * (dtype_size(dtype) + dtype_size(odt)), 2.0 * B * C * T * K);
         const int P = (K - 1) / 2;
         p.partials = partials; p.len_in = len_in; p.len_out = len_out; p.status = L.status;
+        p.dwd = dwd; p.gmax = gmax; p.accumulate = accumulate;
         p.B = B; p.C = C; p.T = T; p.K = K;
         p.Pa = (P + 7) / 8 * 8; p.delta = p.Pa - P;
         p.BB = B >= 32 ? 32 : 16;
         p.N = (127 + K + p.delta + 15) / 16 * 16;
         p.nxb = (p.N + 63) / 64;
+        p.stage_bytes = 2 * (2 + p.nxb) * p.BB * 128;
+        p.nstages = std::min(WT_STAGES, WT_RING_BYTES / p.stage_bytes);
         p.nchunks = (B + p.BB - 1) / p.BB;
-        p.ntb = (T + 127) / 128;
+        p.ntb = (T + 255) / 256;                              // pairs of 128-frame time blocks
         const int steps = p.nchunks * p.ntb;
         // splits per channel: the count that minimises (rounds of units over the SMs) x (steps + epilogue)
         const int sms = std::max(1, st->sm_count);
@@ -398,7 +420,7 @@ void dw_wgrad_tc(const TcState* st, const Launch& L, int dtype, int odt, const v
         else if (odt == F16) launch_wt<__half, __nv_bfloat16>(L, grid, mg, mx, p);
         else launch_wt<__nv_bfloat16, __nv_bfloat16>(L, grid, mg, mx, p);
     }
-    reduce_partials(L, partials, p.S, (int64_t)C * K, dwd, accumulate, gmax);
+    if (p.S > 1) reduce_partials(L, partials, p.S, (int64_t)C * K, dwd, accumulate, gmax);
 }
 
 }  // namespace sc
