@@ -29,10 +29,12 @@ import synth_inputs as si  # noqa: E402
 METRIC = "encoder fwd+bwd audio frames/sec"
 UNIT = "frames/s"
 # The kernel class that takes the largest share of the step (see profiles/); its roofline is reported.
-DOMINANT_CLASS = "dw_wgrad"
+DOMINANT_CLASS = "pw_fwd"
 # measured DRAM bytes / algorithmic bytes of that class's kernel (profiles/block512_dram_traffic.txt:
-# dw_wgrad_reg16_kernel read 52.5 MB for 52.4 MB of operands); scales with the elements processed
-TRAFFIC_RATIO = {"dw_wgrad": 52.5 / 52.4}
+# the 512->512 forward contraction read 26.8 MB and wrote 0.1 MB to DRAM for 78.6 MB of operands and
+# results -- the fp32 result stays in the 126 MB L2 for the kernel that consumes it); scales with the
+# elements processed
+TRAFFIC_RATIO = {"pw_fwd": 26.9 / 78.6}
 
 
 def measured_peaks():
@@ -341,14 +343,22 @@ def main():
                                             if args.profile_class in TRAFFIC_RATIO else None),
                                 "hbm_gbs": gbs, "hbm_frac": gbs / peaks["hbm_gbs"], "peak_source": "derived: 148 SMs x 128 lanes x 1.965 GHz",
                                 "launches": pc["launches"], "avg_ms": per_ms}
-        elif args.profile_class.startswith("pw_") and args.gemm_mode == 0 and tfs > 0.2 * peaks["hbm_gbs"] * 1e-3 * 212:
+        elif (args.profile_class.startswith("pw_") and args.gemm_mode == 0
+              and tfs / peaks["bf16_tflops_sustained"] > gbs / peaks["hbm_gbs"]):
+            # the class's FLOPs at the tensor peak take longer than its bytes at the HBM peak
             line["roofline"] = {"kernel": args.profile_class, "bound": "tensor", "achieved": tfs,
                                 "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                                "frac": tfs / peaks["bf16_tflops_sustained"], "traffic": None,
+                                "frac": tfs / peaks["bf16_tflops_sustained"],
+                                "traffic": (TRAFFIC_RATIO[args.profile_class] * pc["bytes"] / pc["launches"]
+                                            if args.profile_class in TRAFFIC_RATIO else None),
+                                "hbm_gbs": gbs, "hbm_frac": gbs / peaks["hbm_gbs"],
                                 "peak_source": peaks["source"], "launches": pc["launches"], "avg_ms": per_ms}
         else:
             line["roofline"] = {"kernel": args.profile_class, "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"],
-                                "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                                "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                                "traffic": (TRAFFIC_RATIO[args.profile_class] * pc["bytes"] / pc["launches"]
+                                            if args.profile_class in TRAFFIC_RATIO else None),
+                                "tflops": tfs, "tensor_frac": tfs / peaks["bf16_tflops_sustained"],
                                 "peak_source": peaks["source"], "launches": pc["launches"], "avg_ms": per_ms}
     if not args.no_cpu_baseline and world == 1:
         v, cores, dt, desc = oracle_sample(w, 1)
