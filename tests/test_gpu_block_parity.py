@@ -78,6 +78,12 @@ TC_SHAPES = [
     (dict(C_in=16, C_out=24, K=121, residual="proj"), 40, 136, True),
     (dict(C_in=160, C_out=8, K=39, residual="none"), 33, 1000, True),
     (dict(C_in=8, C_out=8, K=5, residual="identity"), 16, 128, False),
+    # TMA-fed depthwise: a single tap, the widest supported halo (tap gradient falls back to SIMT), rows
+    # shorter than one 128-frame block, two sample chunks of 32 with time-block groups cut short by T
+    (dict(C_in=8, C_out=16, K=1, residual="none"), 16, 64, True),
+    (dict(C_in=8, C_out=8, K=129, residual="none"), 17, 264, True),
+    (dict(C_in=16, C_out=8, K=33, residual="proj"), 18, 72, True),
+    (dict(C_in=8, C_out=8, K=75, residual="identity"), 64, 1160, True),
 ]
 
 
