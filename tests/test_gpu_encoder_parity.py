@@ -40,7 +40,7 @@ def run_encoder(ctx, api, w, d, want_dx=True):
 @pytest.mark.parametrize("ragged", [False, True])
 def test_tiny_encoder(api, ctx, dtype, ragged):
     # enough frames that the weight-gradient sums are not dominated by a handful of terms
-    w = si.tiny_encoder(dtype=dtype, B=6, T=320, ragged=ragged, width=32)
+    w = si.tiny_encoder(dtype=dtype, B=8, T=512, ragged=ragged, width=32)
     d = si.draw(w)
     reports, chain = U.run_chain(ctx, api, w, d)
     spec, logits, out_len, gblob, dx = run_encoder(ctx, api, w, d)
