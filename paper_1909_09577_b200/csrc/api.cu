@@ -193,6 +193,7 @@ struct BwdScratch {
     float4 *partials, *coef, *coef_r;
     float *amax_part, *gmax;
     void *gv, *gvr, *gres, *gu, *gxr, *xr, *w16;
+    void *gv16, *gvr16, *x16, *xr16;     // half copies for the weight gradients of bf16 layers (see block_bwd_impl)
     float* wpart; size_t wpart_bytes;
 };
 
@@ -213,6 +214,11 @@ void plan_bwd(const sc_block_desc* d, const Dims& m, Bump& ws, BwdScratch* s, co
     s->gu = ws.take(act_in);
     s->gxr = d->residual == SC_RES_PROJ ? ws.take(e * m.B * m.Cres * m.Tp) : nullptr;
     s->xr = d->residual == SC_RES_PROJ ? ws.take(e * m.B * m.Cres * m.Tp) : nullptr;
+    const bool bf = d->io_dtype == SC_BF16 && d->has_bn;
+    s->gv16 = (bf && !d->has_dw) ? ws.take(act_out) : nullptr;
+    s->x16 = (bf && !d->has_dw) ? ws.take(act_in) : nullptr;
+    s->gvr16 = (bf && d->residual == SC_RES_PROJ) ? ws.take(act_out) : nullptr;
+    s->xr16 = (bf && d->residual == SC_RES_PROJ) ? ws.take(e * m.B * m.Cres * m.Tp) : nullptr;
     size_t wb = gemm_wgrad_simt_scratch_bytes(m.B, std::max(m.Cin, m.Cres), m.Cout);
     wb = std::max(wb, tc_wgrad_scratch_bytes(tc, std::max(m.Cin, m.Cres), m.Cout));
     wb = std::max(wb, dw_wgrad_scratch_bytes(m.B, m.Cin, m.K));
@@ -251,10 +257,20 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
     const int odt = op_dtype(d);
     // gv (and gu after it) is kept scaled by a power of two whenever it is a library-internal 16-bit
     // tensor, so that neither a tiny nor a huge upstream gradient leaves the half range
-    float* gmax = (dt != SC_F32 && d->has_dw && d->has_bn) ? s.gmax : nullptr;
+    // bf16 layers whose gv / gvr stay in bf16 (no depthwise step; the residual projection) get a scaled
+    // half copy of that gradient, and of the other operand, for their weight-gradient contraction: with
+    // 8 significand bits the rounding of the gradient alone uses most of the error budget of dwp / dwr
+    const bool tc_ok = ctx->gemm_mode == 0;
+    const bool half_gv = dt == SC_BF16 && d->has_bn && !d->has_dw && s.gv16 && tc_ok &&
+                         tc_wgrad_supported(&ctx->tc, SC_F16, m.Cin, m.Cout, m.Tp);
+    const bool half_gvr = dt == SC_BF16 && d->has_bn && d->residual == SC_RES_PROJ && s.gvr16 && tc_ok &&
+                          tc_wgrad_supported(&ctx->tc, SC_F16, m.Cres, m.Cout, m.Tp);
+    float* gmax = (dt != SC_F32 && d->has_bn && (d->has_dw || half_gv || half_gvr)) ? s.gmax : nullptr;
     if (gmax) cudaMemsetAsync(gmax, 0, sizeof(float), L.stream);
     BnBwdArgs a{};
     a.amax_part = s.amax_part; a.gmax = gmax; a.gv_dtype = odt;
+    a.gv_scaled = (gmax && d->has_dw) ? 1 : 0;
+    a.gv16 = half_gv ? s.gv16 : nullptr; a.gvr16 = half_gvr ? s.gvr16 : nullptr;
     a.g = io.dy; a.y = io.y; a.vhat = sv->vhat; a.vhat_r = sv->vhat_r;
     a.invstd = sv->invstd; a.invstd_r = sv->invstd_r; a.gamma = p->gamma; a.beta = p->beta;
     a.len_out = io.len_out; a.nvalid = io.nvalid;
@@ -270,7 +286,13 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
     bn_bwd_apply(L, dt, a);
 
     const void* u = d->has_dw ? sv->u : (io.x_clean ? io.x : sv->u);
-    pointwise_wgrad(ctx, L, odt, s.gv, u, g->dwp, s.wpart, acc, m.B, m.Cin, m.Cout, m.Tp, io.len_out, gmax);
+    if (half_gv) {
+        mask_convert_f16(L, s.x16, io.x, io.len_in, m.B, m.Cin, m.T);
+        pointwise_wgrad(ctx, L, SC_F16, s.gv16, s.x16, g->dwp, s.wpart, acc, m.B, m.Cin, m.Cout, m.Tp, io.len_out, gmax);
+    } else {
+        pointwise_wgrad(ctx, L, odt, s.gv, u, g->dwp, s.wpart, acc, m.B, m.Cin, m.Cout, m.Tp, io.len_out,
+                        a.gv_scaled ? gmax : nullptr);
+    }
     const void* wp_op = p->wp;
     if (odt != dt) {
         if (io.w16_kept) wp_op = io.w16_kept;
@@ -281,7 +303,12 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
     if (d->residual == SC_RES_PROJ) {
         const void* xr = io.xres;
         if (!io.res_clean) { mask_copy(L, dt, s.xr, io.xres, io.len_out, m.B, m.Cres, m.Tp); xr = s.xr; }
-        pointwise_wgrad(ctx, L, dt, s.gvr, xr, g->dwr, s.wpart, acc, m.B, m.Cres, m.Cout, m.Tp, io.len_out, nullptr);
+        if (half_gvr) {
+            mask_convert_f16(L, s.xr16, io.xres, io.len_out, m.B, m.Cres, m.Tp);
+            pointwise_wgrad(ctx, L, SC_F16, s.gvr16, s.xr16, g->dwr, s.wpart, acc, m.B, m.Cres, m.Cout, m.Tp, io.len_out, gmax);
+        } else {
+            pointwise_wgrad(ctx, L, dt, s.gvr, xr, g->dwr, s.wpart, acc, m.B, m.Cres, m.Cout, m.Tp, io.len_out, nullptr);
+        }
         void* tgt = io.dx_res ? io.dx_res : s.gxr;
         if (io.dx_res || io.dx) pointwise_dgrad(ctx, L, dt, p->wr, s.gvr, tgt, m.B, m.Cres, m.Cout, m.Tp, io.len_out);
         if (!io.dx_res) extra = s.gxr;

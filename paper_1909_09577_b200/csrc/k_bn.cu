@@ -269,7 +269,7 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_reduce_kernel(BnBwdArgs a)
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             s[0] += ga[i]; s[1] += ga[i] * vh[i]; s[2] += gr[i]; s[3] += gr[i] * vhr[i];
-            amax = fmaxf(amax, fabsf(ga[i]));
+            amax = fmaxf(amax, fmaxf(fabsf(ga[i]), fabsf(gr[i])));
         }
     }
     block_sum(s);
@@ -330,6 +330,9 @@ bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const float* gamma_r, fl
         float bound = amax;
         if (a.has_bn)
             bound = fabsf(gamma[o] * a.invstd[o]) * (amax + fabsf((float)s0) / N + sqrtf(N) * fabsf((float)s1) / N);
+        if (a.residual == 2)     // the residual branch's gradient shares the scale
+            bound = fmaxf(bound, fabsf(gamma_r[o] * a.invstd_r[o]) *
+                                     (amax + fabsf((float)s2) / N + sqrtf(N) * fabsf((float)s3) / N));
         if (bound < 3.0e38f) atomicMax(reinterpret_cast<unsigned int*>(a.gmax), __float_as_uint(bound));
     }
     auto put = [&](float* dst, double val) {
@@ -353,9 +356,11 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_apply_kernel(BnBwdArgs a) 
     SC_ROW_SETUP(a.B * a.C)
     const int b = row / a.C, o = row % a.C;
     BwdRow<T, NT> R(a, row, b, o);
-    float4 cf = a.coef[o];
-    if (a.gmax) cf.x *= pow2_scale(*a.gmax);        // exact: a power of two
+    const float4 cf = a.coef[o];
+    const float sc = a.gmax ? pow2_scale(*a.gmax) : 1.f;      // multiplying by it is exact: a power of two
     const float4 cr = (a.residual == 2) ? a.coef_r[o] : make_float4(0.f, 0.f, 0.f, 0.f);
+    __half* __restrict__ gv16 = a.gv16 ? (__half*)a.gv16 + (size_t)row * R.Tp : nullptr;
+    __half* __restrict__ gvr16 = a.gvr16 ? (__half*)a.gvr16 + (size_t)row * R.Tp : nullptr;
     GT* __restrict__ gv = (GT*)a.gv + (size_t)row * R.Tp;
     T* __restrict__ gvr = (a.residual == 2) ? (T*)a.gvr + (size_t)row * R.Tp : nullptr;
     T* __restrict__ gres = (a.residual == 1) ? (T*)a.gres + (size_t)row * R.Tp : nullptr;
@@ -371,11 +376,32 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_apply_kernel(BnBwdArgs a) 
                 if (a.residual == 2) o2[i] = in ? cr.x * (gr[i] - cr.y - vhr[i] * cr.z) : 0.f;
                 else o2[i] = gr[i];
             }
-            diffuse8<GT>(o1, R.len - t0);
-            if (a.residual == 2) diffuse8<T>(o2, R.len - t0);
         } else {
 #pragma unroll
             for (int i = 0; i < 8; ++i) { o1[i] = 0.f; o2[i] = 0.f; }
+        }
+        const int nin = R.len - t0;
+        if (gv16) {              // half copy for the weight gradient; gv itself keeps plain rounding
+            float h[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) h[i] = o1[i] * sc;
+            diffuse8<__half>(h, nin);
+            store_chunk(gv16, t0, R.Tp, R.vec, h);
+        } else {
+            if (a.gv_scaled) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) o1[i] *= sc;
+            }
+            diffuse8<GT>(o1, nin);
+        }
+        if (gvr16) {
+            float h[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) h[i] = o2[i] * sc;
+            diffuse8<__half>(h, nin);
+            store_chunk(gvr16, t0, R.Tp, R.vec, h);
+        } else if (a.residual == 2) {
+            diffuse8<T>(o2, nin);
         }
         store_chunk(gv, t0, R.Tp, R.vec, o1);
         if (gvr) store_chunk(gvr, t0, R.Tp, R.vec, o2);
@@ -444,8 +470,7 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_fast_kernel(BnBwdArgs a, int
         } else {
             ld8<T>((const T*)a.y + off, y);
         }
-        float4 cf = a.coef[o];
-        if (a.gmax) cf.x *= pow2_scale(*a.gmax);
+        const float4 cf = a.coef[o];
         float4 cr = make_float4(0.f, 0.f, 0.f, 0.f);
         if (RES == 2) cr = a.coef_r[o];
 #pragma unroll
@@ -456,11 +481,37 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_fast_kernel(BnBwdArgs a, int
             if (RES == 2) o2[i] = in ? cr.x * (ga - cr.y - vnr[i] * cr.z) : 0.f;
             if (RES == 1) o2[i] = ga;
         }
-        diffuse8<GT>(o1, len - t0);
-        if (RES == 2) diffuse8<T>(o2, len - t0);
     } else {
 #pragma unroll
         for (int i = 0; i < 8; ++i) { o1[i] = 0.f; o2[i] = 0.f; }
+    }
+    {
+        const float sc = a.gmax ? pow2_scale(*a.gmax) : 1.f;      // exact: a power of two
+        const int nin = len - t0;
+        if (a.gv16) {            // half copy for the weight gradient; gv itself keeps plain rounding
+            float h[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) h[i] = o1[i] * sc;
+            diffuse8<__half>(h, nin);
+            st8<__half>((__half*)a.gv16 + off, h);
+        } else {
+            if (a.gv_scaled) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) o1[i] *= sc;
+            }
+            diffuse8<GT>(o1, nin);
+        }
+        if (RES == 2) {
+            if (a.gvr16) {
+                float h[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) h[i] = o2[i] * sc;
+                diffuse8<__half>(h, nin);
+                st8<__half>((__half*)a.gvr16 + off, h);
+            } else {
+                diffuse8<T>(o2, nin);
+            }
+        }
     }
     st8<GT>((GT*)a.gv + off, o1);
     if (RES == 2) st8<T>((T*)a.gvr + off, o2);
@@ -689,6 +740,51 @@ void convert_bf16_to_f16_many(const Launch& L, const ConvertList& list) {
     for (int i = 0; i < list.count; ++i) total += list.n[i];
     KScope ks_(L, KC_EW, 4.0 * total, 0.0);
     convert_many_kernel<<<dim3(64, list.count), 256, 0, L.stream>>>(list);
+    L.count();
+}
+
+namespace {
+// one 8-frame vector per thread (rows are a multiple of 8 frames) or one element per thread
+__global__ void __launch_bounds__(256)
+mask_convert_f16_kernel(__half* __restrict__ out, const __nv_bfloat16* __restrict__ in, const int* __restrict__ len,
+                        int C, int Tt, long long total, int vec, int* status) {
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (idx >= total) return;
+    const int per_row = vec ? Tt / 8 : Tt;
+    const long long row = idx / per_row;
+    const int t0 = (int)(idx - row * per_row) * (vec ? 8 : 1);
+    const int l = min(len[row / C], Tt);
+    const size_t off = (size_t)row * Tt + t0;
+    bool over = false;
+    if (vec) {
+        float f[8];
+        if (t0 < l) {
+            ld8<__nv_bfloat16>(in + off, f);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (t0 + i >= l) f[i] = 0.f;
+                if (fabsf(f[i]) > 65504.f) { f[i] = copysignf(65504.f, f[i]); over = true; }
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) f[i] = 0.f;
+        }
+        st8<__half>(out + off, f);
+    } else {
+        float f = t0 < l ? __bfloat162float(in[off]) : 0.f;
+        if (fabsf(f) > 65504.f) { f = copysignf(65504.f, f); over = true; }
+        out[off] = __float2half_rn(f);
+    }
+    if (over) raise_status(status, kErrRange);
+}
+}  // namespace
+
+void mask_convert_f16(const Launch& L, void* out, const void* in, const int* len, int B, int C, int Tt) {
+    KScope ks_(L, KC_EW, 4.0 * B * C * Tt, 0.0);
+    const int vec = (Tt % 8 == 0) ? 1 : 0;
+    const long long total = (long long)B * C * (vec ? Tt / 8 : Tt);
+    mask_convert_f16_kernel<<<(unsigned)((total + 255) / 256), 256, 0, L.stream>>>((__half*)out, (const __nv_bfloat16*)in, len,
+                                                                                C, Tt, total, vec, L.status);
     L.count();
 }
 

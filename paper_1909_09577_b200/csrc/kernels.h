@@ -164,7 +164,10 @@ struct BnBwdArgs {
     int gv_dtype;                                  // storage type of gv (OT)
     float4* coef; float4* coef_r;                  // [C]: (k, c1, c2, unused)
     void* gv; void* gvr; void* gres;               // outputs of the apply step (gvr: proj, gres: identity)
-                                                   // gv is multiplied by pow2_scale(*gmax) when gmax is set
+    int gv_scaled;                                 // gv is multiplied by pow2_scale(*gmax) (gmax must be set)
+    // Optional half copies for the weight-gradient contractions of bf16 layers whose gv / gvr stay in
+    // bf16 (8 significand bits): multiplied by pow2_scale(*gmax), rounded with error diffusion.
+    void* gv16; void* gvr16;
 };
 void bn_bwd_reduce(const Launch& L, int dtype, BnBwdArgs& a);
 // partial slots per row that bn_bwd_reduce may use for rows of Tp frames (for scratch sizing)
@@ -174,6 +177,8 @@ void bn_bwd_finalize(const Launch& L, const BnBwdArgs& a, const float* gamma, co
                      int accumulate);
 void bn_bwd_apply(const Launch& L, int dtype, const BnBwdArgs& a);
 
+// out (half) = [t<len[b]] ? in (bf16) : 0; values beyond the half range are clamped and flagged
+void mask_convert_f16(const Launch& L, void* out, const void* in, const int* len, int B, int C, int T);
 // masked copy: out = [t<len[b]] ? in : 0
 void mask_copy(const Launch& L, int dtype, void* out, const void* in, const int* len, int B, int C, int T);
 
