@@ -414,10 +414,10 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_apply_kernel(BnBwdArgs a) 
 // warps and many 16-byte loads in flight per SM.
 template <typename T, typename VT, typename NT, int RES>
 __global__ void __launch_bounds__(256) bn_apply_fast_kernel(ApplyArgs a, int vpr, long long total) {
-    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
-    if (idx >= total) return;
-    const int row = (int)(idx / vpr), t0 = (int)(idx - (long long)row * vpr) * 8;
-    const int b = row / a.C, o = row - b * a.C;
+    const uint32_t idx = blockIdx.x * 256u + threadIdx.x;       // the launcher guarantees total < 2^31
+    if (idx >= (uint32_t)total) return;
+    const int row = (int)a.dvpr.div(idx), t0 = ((int)idx - row * vpr) * 8;
+    const int b = (int)a.dC.div((uint32_t)row), o = row - b * a.C;
     const int len = min(a.len_out[b], a.Tp);
     const size_t off = (size_t)row * a.Tp + t0;
     float out[8], n1[8], n2[8];
@@ -449,10 +449,10 @@ __global__ void __launch_bounds__(256) bn_apply_fast_kernel(ApplyArgs a, int vpr
 
 template <typename T, typename NT, typename GT, int RES>
 __global__ void __launch_bounds__(256) bn_bwd_apply_fast_kernel(BnBwdArgs a, int vpr, long long total) {
-    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
-    if (idx >= total) return;
-    const int row = (int)(idx / vpr), t0 = (int)(idx - (long long)row * vpr) * 8;
-    const int b = row / a.C, o = row - b * a.C;
+    const uint32_t idx = blockIdx.x * 256u + threadIdx.x;       // the launcher guarantees total < 2^31
+    if (idx >= (uint32_t)total) return;
+    const int row = (int)a.dvpr.div(idx), t0 = ((int)idx - row * vpr) * 8;
+    const int b = (int)a.dC.div((uint32_t)row), o = row - b * a.C;
     const int len = min(a.len_out[b], a.Tp);
     const size_t off = (size_t)row * a.Tp + t0;
     float o1[8], o2[8];
@@ -524,14 +524,14 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_fast_kernel(BnBwdArgs a, int
 // assignment, summed later in slot order.
 template <typename T, typename NT, int RES>
 __global__ void __launch_bounds__(256) bn_bwd_reduce_fast_kernel(BnBwdArgs a, int vpr, long long total) {
-    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    const uint32_t idx = blockIdx.x * 256u + threadIdx.x;       // the launcher guarantees total < 2^31
     const int lane = threadIdx.x & 31;
-    const long long warp_first = idx - lane;
-    if (warp_first >= total) return;
-    const bool valid = idx < total;
-    const long long cidx = valid ? idx : total - 1;
-    const int row = (int)(cidx / vpr), t0 = (int)(cidx - (long long)row * vpr) * 8;
-    const int b = row / a.C;
+    const uint32_t warp_first = idx - lane, tot = (uint32_t)total;
+    if (warp_first >= tot) return;
+    const bool valid = idx < tot;
+    const uint32_t cidx = valid ? idx : tot - 1;
+    const int row = (int)a.dvpr.div(cidx), t0 = ((int)cidx - row * vpr) * 8;
+    const int b = (int)a.dC.div((uint32_t)row);
     const int len = min(a.len_out[b], a.Tp);
     float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f, amax = 0.f;
     if (valid && t0 < len) {
@@ -556,19 +556,20 @@ __global__ void __launch_bounds__(256) bn_bwd_reduce_fast_kernel(BnBwdArgs a, in
             amax = fmaxf(amax, fabsf(ga));
         }
     }
-    const int row0 = (int)(warp_first / vpr);
-    const long long wg = warp_first >> 5;                    // global warp index
+    const int row0 = (int)a.dvpr.div(warp_first);
+    const uint32_t wg = warp_first >> 5;                     // global warp index
 #pragma unroll
     for (int seg = 0; seg < 2; ++seg) {
         const int r = row0 + seg;
-        if (seg == 1 && (long long)r * vpr >= warp_first + 32) break;     // warp lies inside one row (uniform)
+        const uint32_t rfirst = (uint32_t)r * (uint32_t)vpr;           // first vector of row r
+        if (seg == 1 && rfirst >= warp_first + 32) break;              // warp lies inside one row (uniform)
         const bool mine = valid && row == r;
         float v[4] = {mine ? s0 : 0.f, mine ? s1 : 0.f, mine ? s2 : 0.f, mine ? s3 : 0.f};
 #pragma unroll
-        for (int i = 0; i < 4; ++i) v[i] = warp_sum(v[i]);
+        for (int i = 0; i < (RES == 2 ? 4 : 2); ++i) v[i] = warp_sum(v[i]);      // v[2], v[3] are zero otherwise
         const float m = a.gmax ? warp_max(mine ? amax : 0.f) : 0.f;
-        if (lane == 0 && (long long)r * vpr < total) {
-            const int slot = (int)(wg - (((long long)r * vpr) >> 5));
+        if (lane == 0 && rfirst < tot) {
+            const int slot = (int)(wg - (rfirst >> 5));
             a.partials[(size_t)r * a.nslots + slot] = make_float4(v[0], v[1], v[2], v[3]);
             if (a.gmax) a.amax_part[(size_t)r * a.nslots + slot] = m;
         }
@@ -640,10 +641,15 @@ void bn_finalize(const Launch& L, const float2* partials, int parts_per_b, int t
     L.count();
 }
 
-void bn_apply(const Launch& L, int dtype, const ApplyArgs& a) {
+// the flattened kernels index with 32 bits
+static bool fits32(int B, int C, int Tp) { return (long long)B * C * (Tp / 8) < (1ll << 31) && (long long)B * C * Tp < (1ll << 31); }
+
+void bn_apply(const Launch& L, int dtype, const ApplyArgs& a_in) {
+    ApplyArgs a = a_in;
     KScope ks_(L, KC_BN_APPLY, (double)a.B * a.C * a.Tp * (dtype_size(vtype_of(dtype)) + dtype_size(dtype) + dtype_size(ntype_of(dtype)) + (a.residual == 1 ? dtype_size(dtype) : 0) + (a.residual == 2 ? dtype_size(vtype_of(dtype)) + dtype_size(ntype_of(dtype)) : 0)), 0.0);
-    if (a.Tp % 8 == 0 && a.has_relu && a.res_before_relu) {
+    if (a.Tp % 8 == 0 && a.has_relu && a.res_before_relu && fits32(a.B, a.C, a.Tp)) {
         const int vpr = a.Tp / 8;
+        a.dvpr = FastDiv((uint32_t)vpr); a.dC = FastDiv((uint32_t)a.C);
         const long long total = (long long)a.B * a.C * vpr;
         const unsigned grid = (unsigned)((total + 255) / 256);
 #define SC_APPLY_FAST(RES) SC_DISPATCH3(dtype, (bn_apply_fast_kernel<T, VT, NT, RES><<<grid, 256, 0, L.stream>>>(a, vpr, total)))
@@ -658,7 +664,8 @@ void bn_apply(const Launch& L, int dtype, const ApplyArgs& a) {
 
 void bn_bwd_reduce(const Launch& L, int dtype, BnBwdArgs& a) {
     a.nslots = 1;
-    if (a.Tp % 8 == 0 && a.Tp >= 256 && a.has_bn && a.has_relu && a.res_before_relu) {
+    if (a.Tp % 8 == 0 && a.Tp >= 256 && a.has_bn && a.has_relu && a.res_before_relu && fits32(a.B, a.C, a.Tp)) {
+        a.dvpr = FastDiv((uint32_t)(a.Tp / 8)); a.dC = FastDiv((uint32_t)a.C);
         KScope ks2_(L, KC_BN_BWD_REDUCE, (double)a.B * a.C * a.Tp * (dtype_size(dtype) * (a.residual == 0 ? 1 : 2) + dtype_size(ntype_of(dtype)) * (a.residual == 2 ? 2 : 1)), 0.0);
         const int vpr = a.Tp / 8;
         a.nslots = bn_bwd_max_slots(a.Tp);
@@ -684,11 +691,13 @@ void bn_bwd_finalize(const Launch& L, const BnBwdArgs& a, const float* gamma, co
     L.count();
 }
 
-void bn_bwd_apply(const Launch& L, int dtype, const BnBwdArgs& a) {
-    const bool fast_apply = a.Tp % 8 == 0 && a.has_bn && a.has_relu && a.res_before_relu;
+void bn_bwd_apply(const Launch& L, int dtype, const BnBwdArgs& a_in) {
+    BnBwdArgs a = a_in;
+    const bool fast_apply = a.Tp % 8 == 0 && a.has_bn && a.has_relu && a.res_before_relu && fits32(a.B, a.C, a.Tp);
     KScope ks_(L, KC_BN_BWD_APPLY, (double)a.B * a.C * a.Tp * (dtype_size(dtype) * (a.has_relu && a.res_before_relu && !(fast_apply && a.residual == 0) ? 2 : 1) + (a.has_bn ? dtype_size(ntype_of(dtype)) : 0) + (a.residual == 2 ? dtype_size(ntype_of(dtype)) : 0) + dtype_size(dtype) * (1 + (a.residual != 0 ? 1 : 0))), 0.0);
-    if (a.Tp % 8 == 0 && a.has_bn && a.has_relu && a.res_before_relu) {
+    if (fast_apply) {
         const int vpr = a.Tp / 8;
+        a.dvpr = FastDiv((uint32_t)vpr); a.dC = FastDiv((uint32_t)a.C);
         const long long total = (long long)a.B * a.C * vpr;
         const unsigned grid = (unsigned)((total + 255) / 256);
 #define SC_BWD_FAST(RES)                                                                                          \

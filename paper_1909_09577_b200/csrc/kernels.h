@@ -139,6 +139,26 @@ inline size_t dtype_size(int dtype) { return dtype == 0 ? 4 : 2; }
 // whose contraction operand is the layer input.
 inline int otype_of(int dtype, int has_dw) { return (dtype == 2 && has_dw) ? 1 : dtype; }
 
+// Division of a 32-bit index by a run-time constant without a divide instruction (multiply-high and two
+// shifts; exact for every 32-bit numerator).  The flattened elementwise kernels split their thread index
+// into (row, position) and a row into (sample, channel) with it.
+struct FastDiv {
+    uint32_t mul = 1, sh1 = 0, sh2 = 0;
+    FastDiv() = default;
+    explicit FastDiv(uint32_t d) {
+        uint32_t l = 0;
+        while (l < 32 && (1ull << l) < d) ++l;
+        mul = (uint32_t)(((1ull << 32) * ((1ull << l) - d)) / d + 1);
+        sh1 = l < 1 ? l : 1; sh2 = l > 0 ? l - 1 : 0;
+    }
+#ifdef __CUDACC__
+    __device__ __forceinline__ uint32_t div(uint32_t n) const {
+        const uint32_t t = __umulhi(n, mul);
+        return (t + ((n - t) >> sh1)) >> sh2;
+    }
+#endif
+};
+
 struct ApplyArgs {
     const void* v; const float *mean, *invstd, *gamma, *beta;          // main branch (v in VT)
     void* vhat;                                                        // out, NT
@@ -148,6 +168,7 @@ struct ApplyArgs {
     void* vhat_r;                                                      // out, NT
     void* y; const int* len_out;
     int B, C, Tp, has_relu, res_before_relu;
+    FastDiv dvpr, dC;                              // by Tp / 8 and by C (set by bn_apply)
 };
 void bn_apply(const Launch& L, int dtype, const ApplyArgs& a);
 
@@ -168,6 +189,7 @@ struct BnBwdArgs {
     // Optional half copies for the weight-gradient contractions of bf16 layers whose gv / gvr stay in
     // bf16 (8 significand bits): multiplied by pow2_scale(*gmax), rounded with error diffusion.
     void* gv16; void* gvr16;
+    FastDiv dvpr, dC;                              // by Tp / 8 and by C (set by the launchers)
 };
 void bn_bwd_reduce(const Launch& L, int dtype, BnBwdArgs& a);
 // partial slots per row that bn_bwd_reduce may use for rows of Tp frames (for scratch sizing)
