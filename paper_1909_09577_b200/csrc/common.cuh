@@ -61,6 +61,16 @@ template <> __device__ __forceinline__ float round_io<__nv_bfloat16>(float v) { 
 template <typename ST> __device__ __forceinline__ void diffuse8(float (&v)[8], int n) {
     if (sizeof(ST) == 4) return;
     float r = 0.f;
+    if (n >= 8) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float t = v[i] + r;
+            const float q = round_io<ST>(t);
+            r = t - q;
+            v[i] = q;
+        }
+        return;
+    }
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         if (i < n) {

@@ -456,6 +456,9 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_fast_kernel(BnBwdArgs a, int
     const int len = min(a.len_out[b], a.Tp);
     const size_t off = (size_t)row * a.Tp + t0;
     float o1[8], o2[8];
+    const int nin = len - t0;                                      // frames of this vector inside the sample
+    const float sc = a.gmax ? pow2_scale(*a.gmax) : 1.f;          // multiplying by it is exact: a power of two
+    const bool fold = !a.gv16 && a.gv_scaled;
     if (t0 < len) {
         float g[8], y[8], vn[8], vnr[8];
         ld8<T>((const T*)a.g + off, g);
@@ -470,24 +473,36 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_fast_kernel(BnBwdArgs a, int
         } else {
             ld8<T>((const T*)a.y + off, y);
         }
+        // gv = k (ga - c1 - c2 vhat) as two fused multiply-adds; when gv itself is the scaled half tensor the
+        // power-of-two scale is folded into k (exact)
         const float4 cf = a.coef[o];
-        float4 cr = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (RES == 2) cr = a.coef_r[o];
+        const float kx = (fold ? sc : 1.f) * cf.x;
+        const float k0 = -kx * cf.y, k2 = -kx * cf.z;
+        float kr = 0.f, r0 = 0.f, r2 = 0.f;
+        if (RES == 2) { const float4 cr = a.coef_r[o]; kr = cr.x; r0 = -kr * cr.y; r2 = -kr * cr.z; }
+        if (nin >= 8) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const bool in = t0 + i < len;
-            const float ga = (in && y[i] > 0.f) ? g[i] : 0.f;
-            o1[i] = in ? cf.x * (ga - cf.y - vn[i] * cf.z) : 0.f;
-            if (RES == 2) o2[i] = in ? cr.x * (ga - cr.y - vnr[i] * cr.z) : 0.f;
-            if (RES == 1) o2[i] = ga;
+            for (int i = 0; i < 8; ++i) {
+                const float ga = y[i] > 0.f ? g[i] : 0.f;
+                o1[i] = fmaf(k2, vn[i], fmaf(kx, ga, k0));
+                if (RES == 2) o2[i] = fmaf(r2, vnr[i], fmaf(kr, ga, r0));
+                if (RES == 1) o2[i] = ga;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const bool in = i < nin;
+                const float ga = (in && y[i] > 0.f) ? g[i] : 0.f;
+                o1[i] = in ? fmaf(k2, vn[i], fmaf(kx, ga, k0)) : 0.f;
+                if (RES == 2) o2[i] = in ? fmaf(r2, vnr[i], fmaf(kr, ga, r0)) : 0.f;
+                if (RES == 1) o2[i] = ga;
+            }
         }
     } else {
 #pragma unroll
         for (int i = 0; i < 8; ++i) { o1[i] = 0.f; o2[i] = 0.f; }
     }
     {
-        const float sc = a.gmax ? pow2_scale(*a.gmax) : 1.f;      // exact: a power of two
-        const int nin = len - t0;
         if (a.gv16) {            // half copy for the weight gradient; gv itself keeps plain rounding
             float h[8];
 #pragma unroll
@@ -495,10 +510,6 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_fast_kernel(BnBwdArgs a, int
             diffuse8<__half>(h, nin);
             st8<__half>((__half*)a.gv16 + off, h);
         } else {
-            if (a.gv_scaled) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) o1[i] *= sc;
-            }
             diffuse8<GT>(o1, nin);
         }
         if (RES == 2) {
