@@ -144,7 +144,25 @@ def bn_bwd(ga, vhat, valid, gamma, invstd, N):
 
 
 # ----------------------------------------------------------------------------
+# Decoder tail: log-softmax over the class (channel) axis.  The paper's CTC decoder module turns
+# the encoder output into ``log_probs`` (section 4.1.1); its last step, after the 1x1 convolution
+# that produces the class scores z, is  log_probs[b,c,t] = z[b,c,t] - log(sum_c' exp(z[b,c',t])).
+# ----------------------------------------------------------------------------
+def log_softmax_fwd(z):
+    """Per (b, t) position over axis 1, written as the definition with the usual max shift
+    (exp(z - max) is the same ratio; it only avoids overflow)."""
+    zmax = np.max(z, axis=1, keepdims=True)
+    return z - zmax - np.log(np.sum(np.exp(z - zmax), axis=1, keepdims=True))
+
+
+def log_softmax_bwd(g, logp):
+    """Adjoint: d z[c] = g[c] - softmax[c] * sum_c' g[c'],  softmax = exp(log_probs)."""
+    return g - np.exp(logp) * np.sum(g, axis=1, keepdims=True)
+
+
+# ----------------------------------------------------------------------------
 # One layer:  [mask] -> [depthwise] -> pointwise [+bias] -> [BN] -> [+residual] -> [ReLU] -> mask
+#             (or, for the decoder tail:  ... pointwise + bias -> log-softmax over channels -> mask)
 # ----------------------------------------------------------------------------
 def _p(params, name):
     return np.asarray(params[name], dtype=F64)
@@ -217,6 +235,10 @@ def block_fwd(L, x, lengths, params, res_src=None):
     y = np.maximum(a, 0.0) if L.has_relu else a
     if r is not None and not L.res_before_relu:
         y = y + r
+    if getattr(L, "log_softmax", False):
+        # decoder tail (only legal on a linear layer): reading: padded frames read as zero, like
+        # every other output of the path
+        y = log_softmax_fwd(y)
     S["y"] = np.where(valid, y, 0.0)
     return S
 
@@ -234,6 +256,8 @@ def block_bwd(L, g, lengths, params, S, gate=None):
     T = S["xm"].shape[2]
     G = {}
     gm = np.where(valid, g, 0.0)                        # output mask
+    if getattr(L, "log_softmax", False):
+        gm = np.where(valid, log_softmax_bwd(gm, S["y"]), 0.0)
     if L.has_relu:
         if gate is None:
             gate = S["a"] > 0.0

@@ -73,6 +73,7 @@ class LayerCfg:
     res_from: Optional[int] = None  # index of the layer whose INPUT feeds the residual (None: own input)
     res_before_relu: bool = True
     eps: float = 1e-3
+    log_softmax: bool = False       # decoder tail on a linear layer: log-softmax over the channels
 
     def param_shapes(self) -> Dict[str, tuple]:
         s: Dict[str, tuple] = {}
@@ -129,8 +130,9 @@ class Workload:
         return T
 
 
-def quartznet5x5_layers() -> List[LayerCfg]:
-    """QuartzNet-5x5-style encoder plus the two pointwise layers that end in 29 logits."""
+def quartznet5x5_layers(log_probs: bool = False) -> List[LayerCfg]:
+    """QuartzNet-5x5-style encoder plus the two pointwise layers that end in 29 logits
+    (log_probs=True: in 29 log-probabilities, the decoder module's output)."""
     layers: List[LayerCfg] = [LayerCfg(64, 256, K=33, stride=2)]
     plan = [(256, 33), (256, 39), (512, 51), (512, 63), (512, 75)]
     c_prev = 256
@@ -146,7 +148,8 @@ def quartznet5x5_layers() -> List[LayerCfg]:
         c_prev = c_out
     layers.append(LayerCfg(512, 512, K=87))
     layers.append(LayerCfg(512, 1024, K=1, has_dw=False))
-    layers.append(LayerCfg(1024, 29, K=1, has_dw=False, has_bn=False, has_relu=False, has_bias=True))
+    layers.append(LayerCfg(1024, 29, K=1, has_dw=False, has_bn=False, has_relu=False, has_bias=True,
+                           log_softmax=log_probs))
     return layers
 
 

@@ -435,6 +435,66 @@ def test_p7_hand_worked_example():
     np.testing.assert_allclose(O.block_fwd(L3, x, [4], p)["vhat"].ravel(), gold["eps1e-3.vhat"], **tol)
 
 
+# ----------------------------------------------------------------------------------------------
+# Decoder tail: log-softmax over the classes
+# ----------------------------------------------------------------------------------------------
+def test_log_softmax_matches_torch_and_closed_forms():
+    rng = np.random.default_rng(21)
+    z = rng.standard_normal((3, 29, 11)) * 3.0
+    lp = O.log_softmax_fwd(z)
+    zt = torch.tensor(z, requires_grad=True)
+    ref = F.log_softmax(zt, dim=1)
+    np.testing.assert_allclose(lp, ref.detach().numpy(), rtol=0, atol=1e-13)
+    # probabilities sum to one at every position; shifting z by a per-position constant changes nothing
+    np.testing.assert_allclose(np.exp(lp).sum(axis=1), 1.0, atol=1e-13)
+    np.testing.assert_allclose(O.log_softmax_fwd(z + rng.standard_normal((3, 1, 11)) * 50), lp, atol=1e-11)
+    # two classes: the closed form -log(1 + exp(z1 - z0))
+    z2 = rng.standard_normal((2, 2, 5))
+    np.testing.assert_allclose(O.log_softmax_fwd(z2)[:, 0], -np.log1p(np.exp(z2[:, 1] - z2[:, 0])), atol=1e-13)
+    # adjoint against autograd; rows of the gradient sum to zero
+    g = rng.standard_normal(z.shape)
+    ref.backward(torch.tensor(g))
+    dz = O.log_softmax_bwd(g, lp)
+    np.testing.assert_allclose(dz, zt.grad.numpy(), atol=1e-12)
+    np.testing.assert_allclose(dz.sum(axis=1), 0.0, atol=1e-12)
+
+
+def test_decoder_tail_layer_fwd_bwd():
+    """Linear + bias + log-softmax layer under a padding mask: against torch on the packed valid frames,
+    and every gradient against central differences."""
+    rng = np.random.default_rng(22)
+    L = si.LayerCfg(6, 5, K=1, has_dw=False, has_bn=False, has_relu=False, has_bias=True, log_softmax=True)
+    B, T = 3, 7
+    lengths = np.array([7, 3, 1])
+    x = rng.standard_normal((B, 6, T))
+    p = {"wp": rng.uniform(-1, 1, (5, 6)), "bias": rng.uniform(-1, 1, (5,))}
+    g = rng.standard_normal((B, 5, T))
+    S = O.block_fwd(L, x, lengths, p)
+    G = O.block_bwd(L, g, lengths, p, S)
+    valid = S["valid"]
+    assert np.all(S["y"][~np.broadcast_to(valid, S["y"].shape)] == 0)
+    xt = torch.tensor(x, requires_grad=True)
+    wt = torch.tensor(p["wp"], requires_grad=True)
+    bt = torch.tensor(p["bias"], requires_grad=True)
+    m = torch.tensor(np.broadcast_to(valid, (B, 5, T)).copy())
+    yt = torch.where(m, F.log_softmax(torch.einsum("oc,bct->bot", wt, xt) + bt[None, :, None], dim=1), torch.zeros(()).double())
+    np.testing.assert_allclose(S["y"], yt.detach().numpy(), atol=1e-12)
+    (yt * torch.tensor(g)).sum().backward()
+    np.testing.assert_allclose(G["dx"], xt.grad.numpy(), atol=1e-12)
+    np.testing.assert_allclose(G["dwp"], wt.grad.numpy(), atol=1e-12)
+    np.testing.assert_allclose(G["dbias"], bt.grad.numpy(), atol=1e-12)
+    # central differences of the loss sum(y * g) w.r.t. one weight and one input element
+    def loss(xx, pp):
+        return float(np.sum(O.block_fwd(L, xx, lengths, pp)["y"] * g))
+    h = 1e-6
+    pp = {k: v.copy() for k, v in p.items()}; pp["wp"][2, 3] += h
+    pm = {k: v.copy() for k, v in p.items()}; pm["wp"][2, 3] -= h
+    assert abs((loss(x, pp) - loss(x, pm)) / (2 * h) - G["dwp"][2, 3]) < 1e-6
+    xp = x.copy(); xp[1, 4, 2] += h
+    xm = x.copy(); xm[1, 4, 2] -= h
+    assert abs((loss(xp, p) - loss(xm, p)) / (2 * h) - G["dx"][1, 4, 2]) < 1e-6
+
+
 def test_running_stats():
     rm, rv = O.running_stats_update(np.zeros(2), np.ones(2), np.array([1.0, 2.0]), np.array([4.0, 9.0]), 10)
     np.testing.assert_allclose(rm, [0.1, 0.2])
