@@ -243,6 +243,62 @@ def block_fwd(L, x, lengths, params, res_src=None):
     return S
 
 
+def block_infer(L, x, lengths, params, running, res_src=None):
+    """Forward of one layer in evaluation mode (the paper's `eval` / `infer` actions, section 3.1): the
+    batch statistics are replaced by fixed running statistics,
+        bn = gamma * (v - running_mean) / sqrt(running_var + eps) + beta,
+    everything else as in block_fwd.  ``running`` = dict(mean, var[, mean_r, var_r]).  Returns y only
+    (plus out_len, valid)."""
+    x = np.asarray(x, dtype=F64)
+    B, C_in, T = x.shape
+    s = L.stride if L.has_dw else 1
+    K = L.K if L.has_dw else 1
+    Tp = out_time(T, K, s)
+    lengths = np.asarray(lengths, dtype=np.int64)
+    out_len = out_lengths(lengths, s)
+    valid = time_mask(out_len, Tp)
+    xm = np.where(time_mask(lengths, T), x, 0.0)
+    u = depthwise_fwd(xm, _p(params, "wd"), s) if L.has_dw else xm
+    u = np.where(valid, u, 0.0)
+    v = pointwise_fwd(u, _p(params, "wp"))
+    if L.has_bias:
+        v = v + _p(params, "bias")[None, :, None]
+
+    def fixed_bn(t, mean, var, gamma, beta):
+        k = gamma / np.sqrt(np.asarray(var, F64) + L.eps)
+        return k[None, :, None] * (t - np.asarray(mean, F64)[None, :, None]) + beta[None, :, None]
+
+    bn = fixed_bn(v, running["mean"], running["var"], _p(params, "gamma"), _p(params, "beta")) if L.has_bn else v
+    r = None
+    if L.residual != "none":
+        rs = x if res_src is None else np.asarray(res_src, dtype=F64)
+        xr = np.where(valid, rs, 0.0)
+        if L.residual == "identity":
+            r = xr
+        else:
+            r = fixed_bn(pointwise_fwd(xr, _p(params, "wr")), running["mean_r"], running["var_r"],
+                         _p(params, "gamma_r"), _p(params, "beta_r"))
+    a = bn + r if (r is not None and L.res_before_relu) else bn
+    y = np.maximum(a, 0.0) if L.has_relu else a
+    if r is not None and not L.res_before_relu:
+        y = y + r
+    if getattr(L, "log_softmax", False):
+        y = log_softmax_fwd(y)
+    return {"y": np.where(valid, y, 0.0), "out_len": out_len, "valid": valid}
+
+
+def encoder_infer(layers, x, lengths, params, running):
+    """Evaluation-mode forward through every layer; ``running[i]`` as for block_infer."""
+    acts = [np.asarray(x, dtype=F64)]
+    lens = [np.asarray(lengths, dtype=np.int64)]
+    for i, L in enumerate(layers):
+        res = acts[L.res_from if L.res_from is not None else i] if L.residual != "none" else None
+        S = block_infer(L, acts[i], lens[i], params[i], running[i], res_src=res)
+        acts.append(S["y"])
+        lens.append(S["out_len"])
+    return acts, lens
+
+
 def block_bwd(L, g, lengths, params, S, gate=None):
     """Backward of block_fwd.  ``g`` = dLoss/dy, ``S`` = block_fwd's dict.
     ``gate`` (bool [B,C_out,T'], optional) overrides the ReLU gate [a > 0]; derivative at a == 0

@@ -495,6 +495,50 @@ def test_decoder_tail_layer_fwd_bwd():
     assert abs((loss(xp, p) - loss(xm, p)) / (2 * h) - G["dx"][1, 4, 2]) < 1e-6
 
 
+# ----------------------------------------------------------------------------------------------
+# Evaluation mode: fixed running statistics
+# ----------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("residual", ["none", "identity", "proj"])
+def test_infer_matches_torch_eval_and_folded_weights(residual):
+    rng = np.random.default_rng(31)
+    Co = 6 if residual == "identity" else 5
+    L = si.LayerCfg(6, Co, K=5, residual=residual)
+    B, T = 3, 12
+    lengths = np.array([12, 5, 9])
+    x = rng.standard_normal((B, 6, T))
+    p = rand_params(rng, L)
+    run = {"mean": rng.standard_normal(Co), "var": rng.uniform(0.5, 2.0, Co),
+           "mean_r": rng.standard_normal(Co), "var_r": rng.uniform(0.5, 2.0, Co)}
+    S = O.block_infer(L, x, lengths, p, run)
+    valid = S["valid"]
+    # torch: grouped conv, 1x1 conv, batch_norm in eval mode, on the masked input
+    xm = torch.tensor(np.where(O.time_mask(lengths, T), x, 0.0))
+    u = F.conv1d(xm, torch.tensor(p["wd"])[:, None, :], padding=2, groups=6)
+    u = torch.where(torch.tensor(np.broadcast_to(valid, u.shape).copy()), u, torch.zeros(()).double())
+    v = F.conv1d(u, torch.tensor(p["wp"])[:, :, None])
+    bn = F.batch_norm(v, torch.tensor(run["mean"]), torch.tensor(run["var"]), torch.tensor(p["gamma"]),
+                      torch.tensor(p["beta"]), training=False, eps=L.eps)
+    if residual == "identity":
+        bn = bn + xm
+    if residual == "proj":
+        vr = F.conv1d(xm, torch.tensor(p["wr"])[:, :, None])
+        bn = bn + F.batch_norm(vr, torch.tensor(run["mean_r"]), torch.tensor(run["var_r"]), torch.tensor(p["gamma_r"]),
+                               torch.tensor(p["beta_r"]), training=False, eps=L.eps)
+    ref = torch.where(torch.tensor(np.broadcast_to(valid, bn.shape).copy()), F.relu(bn), torch.zeros(()).double())
+    np.testing.assert_allclose(S["y"], ref.numpy(), atol=1e-12)
+    # folding: the fixed normalisation is an affine map per channel, so it folds into the pointwise weights
+    k = p["gamma"] / np.sqrt(run["var"] + L.eps)
+    Lf = si.LayerCfg(6, Co, K=5, has_bn=False, has_relu=False, has_bias=True)
+    pf = {"wd": p["wd"], "wp": p["wp"] * k[:, None], "bias": p["beta"] - run["mean"] * k}
+    folded = O.block_fwd(Lf, x, lengths, pf)["y"]
+    if residual == "none":
+        np.testing.assert_allclose(S["y"], np.maximum(folded, 0.0), atol=1e-12)
+    # with the batch's own statistics as "running" statistics it is the training-mode forward
+    St = O.block_fwd(L, x, lengths, p)
+    own = {"mean": St["mean"], "var": St["var"], "mean_r": St.get("mean_r"), "var_r": St.get("var_r")}
+    np.testing.assert_allclose(O.block_infer(L, x, lengths, p, own)["y"], St["y"], atol=1e-12)
+
+
 def test_running_stats():
     rm, rv = O.running_stats_update(np.zeros(2), np.ones(2), np.array([1.0, 2.0]), np.array([4.0, 9.0]), 10)
     np.testing.assert_allclose(rm, [0.1, 0.2])
