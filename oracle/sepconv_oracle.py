@@ -41,10 +41,19 @@ F64 = np.float64
 # ----------------------------------------------------------------------------
 # Lengths and masks
 # ----------------------------------------------------------------------------
-def out_time(T: int, K: int, stride: int) -> int:
-    """Frames produced by a K-tap, "same"-padded (P=(K-1)/2) correlation with the given stride."""
-    P = (K - 1) // 2
-    return (T + 2 * P - K) // stride + 1
+def same_padding(K: int, dilation: int = 1):
+    """Zeros added left and right so that a stride-1 correlation keeps the length: dilation*(K-1) in
+    total.  reading: for an even total (odd K, or even dilation) it splits evenly; otherwise the extra
+    zero goes to the right (left = total // 2), the convention of the common "same" padding."""
+    total = dilation * (K - 1)
+    return total // 2, total - total // 2
+
+
+def out_time(T: int, K: int, stride: int, dilation: int = 1) -> int:
+    """Frames produced by a K-tap, "same"-padded correlation (taps `dilation` frames apart) with the
+    given stride: floor((T + pad_total - dilation*(K-1) - 1) / stride) + 1 = floor((T-1)/stride) + 1."""
+    pl, pr = same_padding(K, dilation)
+    return (T + pl + pr - dilation * (K - 1) - 1) // stride + 1
 
 
 def out_lengths(lengths, stride: int):
@@ -62,38 +71,39 @@ def time_mask(lengths, T: int):
 # ----------------------------------------------------------------------------
 # The four linear pieces and their adjoints
 # ----------------------------------------------------------------------------
-def depthwise_fwd(xm, wd, stride: int):
-    """u[b,c,t] = sum_k wd[c,k] * xm[b,c,t*stride + k - P], zero outside [0,T).
+def depthwise_fwd(xm, wd, stride: int, dilation: int = 1):
+    """u[b,c,t] = sum_k wd[c,k] * xm[b,c,t*stride + k*dilation - P], zero outside [0,T), P = left padding.
     reading: cross-correlation (taps are not flipped)."""
     B, C, T = xm.shape
     K = wd.shape[1]
-    P = (K - 1) // 2
-    Tp = out_time(T, K, stride)
-    xp = np.zeros((B, C, T + 2 * P), F64)
+    P, Pr = same_padding(K, dilation)
+    Tp = out_time(T, K, stride, dilation)
+    xp = np.zeros((B, C, T + P + Pr), F64)
     xp[:, :, P:P + T] = xm
     u = np.zeros((B, C, Tp), F64)
     span = (Tp - 1) * stride + 1
     for k in range(K):
-        u += wd[None, :, k, None] * xp[:, :, k:k + span:stride]
+        u += wd[None, :, k, None] * xp[:, :, k * dilation:k * dilation + span:stride]
     return u
 
 
-def depthwise_bwd(gu, xm, wd, stride: int):
+def depthwise_bwd(gu, xm, wd, stride: int, dilation: int = 1):
     """Adjoint of depthwise_fwd: returns (gx, dwd).
-    gx[b,c,tau] = sum over (k,t) with t*stride+k-P = tau of wd[c,k]*gu[b,c,t];
-    dwd[c,k]    = sum_{b,t} gu[b,c,t] * xm[b,c,t*stride+k-P]."""
+    gx[b,c,tau] = sum over (k,t) with t*stride+k*dilation-P = tau of wd[c,k]*gu[b,c,t];
+    dwd[c,k]    = sum_{b,t} gu[b,c,t] * xm[b,c,t*stride+k*dilation-P]."""
     B, C, T = xm.shape
     K = wd.shape[1]
-    P = (K - 1) // 2
+    P, Pr = same_padding(K, dilation)
     Tp = gu.shape[2]
-    xp = np.zeros((B, C, T + 2 * P), F64)
+    xp = np.zeros((B, C, T + P + Pr), F64)
     xp[:, :, P:P + T] = xm
     gxp = np.zeros_like(xp)
     dwd = np.zeros((C, K), F64)
     span = (Tp - 1) * stride + 1
     for k in range(K):
-        gxp[:, :, k:k + span:stride] += wd[None, :, k, None] * gu
-        dwd[:, k] = np.sum(gu * xp[:, :, k:k + span:stride], axis=(0, 2))
+        o = k * dilation
+        gxp[:, :, o:o + span:stride] += wd[None, :, k, None] * gu
+        dwd[:, k] = np.sum(gu * xp[:, :, o:o + span:stride], axis=(0, 2))
     return gxp[:, :, P:P + T], dwd
 
 
@@ -182,7 +192,8 @@ def block_fwd(L, x, lengths, params, res_src=None):
     B, C_in, T = x.shape
     s = L.stride if L.has_dw else 1
     K = L.K if L.has_dw else 1
-    Tp = out_time(T, K, s)
+    dil = getattr(L, "dilation", 1) if L.has_dw else 1
+    Tp = out_time(T, K, s, dil)
     lengths = np.asarray(lengths, dtype=np.int64)
     out_len = out_lengths(lengths, s)
     valid = time_mask(out_len, Tp)                      # m'
@@ -191,7 +202,7 @@ def block_fwd(L, x, lengths, params, res_src=None):
     # mask on the conv input
     xm = np.where(time_mask(lengths, T), x, 0.0)
     S["xm"] = xm
-    u = depthwise_fwd(xm, _p(params, "wd"), s) if L.has_dw else xm
+    u = depthwise_fwd(xm, _p(params, "wd"), s, dil) if L.has_dw else xm
     u = np.where(valid, u, 0.0)                         # frames beyond len' are never used
     S["u"] = u
     v = pointwise_fwd(u, _p(params, "wp"))
@@ -253,12 +264,13 @@ def block_infer(L, x, lengths, params, running, res_src=None):
     B, C_in, T = x.shape
     s = L.stride if L.has_dw else 1
     K = L.K if L.has_dw else 1
-    Tp = out_time(T, K, s)
+    dil = getattr(L, "dilation", 1) if L.has_dw else 1
+    Tp = out_time(T, K, s, dil)
     lengths = np.asarray(lengths, dtype=np.int64)
     out_len = out_lengths(lengths, s)
     valid = time_mask(out_len, Tp)
     xm = np.where(time_mask(lengths, T), x, 0.0)
-    u = depthwise_fwd(xm, _p(params, "wd"), s) if L.has_dw else xm
+    u = depthwise_fwd(xm, _p(params, "wd"), s, dil) if L.has_dw else xm
     u = np.where(valid, u, 0.0)
     v = pointwise_fwd(u, _p(params, "wp"))
     if L.has_bias:
@@ -335,7 +347,7 @@ def block_bwd(L, g, lengths, params, S, gate=None):
         G["dbias"] = np.sum(gv, axis=(0, 2))
     gu, G["dwp"] = pointwise_bwd(gv, S["u"], _p(params, "wp"))
     if L.has_dw:
-        gx, G["dwd"] = depthwise_bwd(gu, S["xm"], _p(params, "wd"), s)
+        gx, G["dwd"] = depthwise_bwd(gu, S["xm"], _p(params, "wd"), s, getattr(L, "dilation", 1))
     else:
         gx = gu
     G["dx"] = np.where(time_mask(lengths, T), gx, 0.0)

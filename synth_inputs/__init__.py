@@ -74,6 +74,7 @@ class LayerCfg:
     res_before_relu: bool = True
     eps: float = 1e-3
     log_softmax: bool = False       # decoder tail on a linear layer: log-softmax over the channels
+    dilation: int = 1               # frames between neighbouring taps of the depthwise step
 
     def param_shapes(self) -> Dict[str, tuple]:
         s: Dict[str, tuple] = {}
@@ -125,8 +126,7 @@ class Workload:
         T = self.T
         for L in self.layers:
             if L.has_dw:
-                P = (L.K - 1) // 2
-                T = (T + 2 * P - L.K) // L.stride + 1
+                T = (T - 1) // L.stride + 1      # "same" padding: dilation * (K - 1) zeros in total
         return T
 
 

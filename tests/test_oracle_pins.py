@@ -33,8 +33,9 @@ def brute_block(L, x, lengths, p, res_src=None):
     B, Ci, T = x.shape
     s = L.stride if L.has_dw else 1
     K = L.K if L.has_dw else 1
-    P = (K - 1) // 2
-    Tp = (T + 2 * P - K) // s + 1
+    dil = L.dilation if L.has_dw else 1
+    P = (dil * (K - 1)) // 2                 # zeros on the left; the right side gets the rest
+    Tp = (T - 1) // s + 1
     Co = L.C_out
     lenp = [-(-int(l) // s) for l in lengths]
     xt = lambda b, c, t: (x[b][c][t] if 0 <= t < T and t < lengths[b] else 0.0)
@@ -43,7 +44,7 @@ def brute_block(L, x, lengths, p, res_src=None):
         if t >= lenp[b]:
             continue
         if L.has_dw:
-            u[b][c][t] = sum(p["wd"][c][k] * xt(b, c, t * s + k - P) for k in range(K))
+            u[b][c][t] = sum(p["wd"][c][k] * xt(b, c, t * s + k * dil - P) for k in range(K))
         else:
             u[b][c][t] = xt(b, c, t)
 
@@ -93,6 +94,9 @@ TINY = [
     dict(C_in=3, C_out=3, K=1, stride=1, residual="identity", res_before_relu=False),
     dict(C_in=3, C_out=2, K=1, has_dw=False, has_bn=False, has_relu=False, has_bias=True),
     dict(C_in=2, C_out=4, K=3, stride=1, residual="proj", res_before_relu=False),
+    dict(C_in=3, C_out=3, K=4, stride=1, residual="identity"),            # even K: one more zero on the right
+    dict(C_in=2, C_out=3, K=3, stride=1, dilation=2, residual="proj"),
+    dict(C_in=2, C_out=2, K=2, stride=2, dilation=3, residual="none"),
 ]
 
 
@@ -537,6 +541,25 @@ def test_infer_matches_torch_eval_and_folded_weights(residual):
     St = O.block_fwd(L, x, lengths, p)
     own = {"mean": St["mean"], "var": St["var"], "mean_r": St.get("mean_r"), "var_r": St.get("var_r")}
     np.testing.assert_allclose(O.block_infer(L, x, lengths, p, own)["y"], St["y"], atol=1e-12)
+
+
+@pytest.mark.parametrize("K,dil", [(4, 1), (3, 2), (2, 3), (6, 2), (5, 3)])
+def test_same_padding_convention_matches_torch(K, dil):
+    """Even K and dilated taps against torch's grouped conv1d with padding='same' (stride 1), forward and both
+    gradients: pins where the zeros go when dilation*(K-1) is odd."""
+    rng = np.random.default_rng(40 + K + dil)
+    x = rng.standard_normal((2, 3, 11))
+    w = rng.standard_normal((3, K))
+    g = rng.standard_normal((2, 3, 11))
+    u = O.depthwise_fwd(x, w, 1, dil)
+    xt, wt = torch.tensor(x, requires_grad=True), torch.tensor(w, requires_grad=True)
+    ref = F.conv1d(xt, wt[:, None, :], padding="same", dilation=dil, groups=3)
+    np.testing.assert_allclose(u, ref.detach().numpy(), atol=1e-12)
+    ref.backward(torch.tensor(g))
+    gx, dwd = O.depthwise_bwd(g, x, w, 1, dil)
+    np.testing.assert_allclose(gx, xt.grad.numpy(), atol=1e-12)
+    np.testing.assert_allclose(dwd, wt.grad.numpy(), atol=1e-12)
+    assert O.out_time(11, K, 1, dil) == 11 and O.out_time(11, K, 2, dil) == 6
 
 
 def test_running_stats():
