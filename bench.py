@@ -6,7 +6,13 @@ Default workload: the bf16 QuartzNet-5x5-style encoder, B=32, T=1600 input frame
 (config 4); `--config 5` runs the ragged B=64, T=3200 encoder.  Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config 4|5] [--impl reference]
-                  [--profile-class NAME|all] [--no-cpu-baseline]
+                  [--no-cpu-baseline] [--no-e2e] [--no-graph] [--block C_in,C_out,K,B,T]
+
+Besides the step throughput the line carries `roofline_per_class`: for every kernel class of the step
+its CUDA-event time, launches, algorithmic bytes and flops (every tensor the class must read or write
+once, 16-bit activations, valid frames only), the bound that binds it (the slower of its flops at the
+measured tensor peak and its bytes at the measured HBM peak) and the fraction of that bound it reaches;
+`roofline` repeats the entry of the class with the largest share of the step.
 
 N > 1 (under torchrun): every rank runs an independent replica of the same workload on its own GPU
 (the path has no exchange step); value = N * frames / max-over-ranks time.
@@ -28,13 +34,60 @@ import synth_inputs as si  # noqa: E402
 
 METRIC = "encoder fwd+bwd audio frames/sec"
 UNIT = "frames/s"
-# The kernel class that takes the largest share of the step (see profiles/); its roofline is reported.
-DOMINANT_CLASS = "pw_fwd"
-# measured DRAM bytes / algorithmic bytes of that class's kernel (profiles/block512_dram_traffic.txt:
-# the 512->512 forward contraction read 26.8 MB and wrote 0.1 MB to DRAM for 78.6 MB of operands and
-# results -- the fp32 result stays in the 126 MB L2 for the kernel that consumes it); scales with the
-# elements processed
-TRAFFIC_RATIO = {"pw_fwd": 26.9 / 78.6}
+TOLERANCE = {"fp32": "max |err| <= 1e-4 * max(|ref|, RMS ref) per tensor",
+             "16bit": "max |err| <= 2e-2 * RMS(ref over valid frames) per tensor; for tensors stored in bf16/fp16 the "
+                      "elements whose half unit in the last place exceeds that allowance get the half unit added"}
+
+
+def kernels_sha():
+    """Hash of the kernel sources: ties a committed counter summary to the kernels it was taken on."""
+    import hashlib
+    h = hashlib.sha256()
+    d = os.path.join(ROOT, "paper_1909_09577_b200", "csrc")
+    for fn in sorted(os.listdir(d)):
+        if fn.endswith((".cu", ".cuh", ".h")):
+            h.update(open(os.path.join(d, fn), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def dram_traffic_ratios():
+    """Measured DRAM bytes / algorithmic bytes per kernel class, from the committed ncu summary
+    profiles/dram_traffic_by_class.txt (lines `class <name> dram_bytes <x> algorithmic_bytes <y>` taken on
+    one block of the workload, plus `kernels_sha <hash of the kernel sources at capture time>`).  Returns
+    {} when the file is absent or the kernel sources have changed since the counters were taken."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic_by_class.txt")
+    if not os.path.exists(path):
+        return {}
+    ratios, sha = {}, None
+    for line in open(path):
+        f = line.split()
+        if len(f) >= 2 and f[0] == "kernels_sha":
+            sha = f[1]
+        if len(f) >= 6 and f[0] == "class" and f[2] == "dram_bytes" and f[4] == "algorithmic_bytes":
+            ratios[f[1]] = float(f[3]) / float(f[5])
+    return ratios if sha == kernels_sha() else {}
+
+
+def class_rooflines(prof, nsteps, valid_frac, peaks, traffic_ratio):
+    """Per kernel class: time, launches, algorithmic work on valid frames, binding bound and fraction.
+    The launchers count padded frames (they cannot see the lengths); every per-position cost scales
+    with the valid fraction, which the caller knows from the host copy of the lengths."""
+    out = {}
+    tot = sum(v["ms"] for v in prof.values()) or 1.0
+    for k, v in prof.items():
+        ms = v["ms"] / nsteps
+        by, fl = v["bytes"] * valid_frac / nsteps, v["flops"] * valid_frac / nsteps
+        t_hbm = by / (peaks["hbm_gbs"] * 1e9) * 1e3
+        t_ten = fl / (peaks["bf16_tflops_sustained"] * 1e12) * 1e3
+        bound = "tensor" if (k.startswith("pw_") and t_ten > t_hbm) else "hbm"
+        gbs, tfs = by / ms / 1e6, fl / ms / 1e9
+        lps = v["launches"] / nsteps
+        out[k] = {"ms_per_step": ms, "launches_per_step": lps, "share": v["ms"] / tot,
+                  "algorithmic_bytes": by, "flops": fl, "GB/s": gbs, "TFLOP/s": tfs, "bound": bound,
+                  "frac": (t_ten if bound == "tensor" else t_hbm) / ms if ms > 0 else None,
+                  "hbm_frac": gbs / peaks["hbm_gbs"], "tensor_frac": tfs / peaks["bf16_tflops_sustained"],
+                  "traffic": traffic_ratio[k] * by / lps if k in traffic_ratio and lps else None}
+    return out
 
 
 def measured_peaks():
@@ -170,10 +223,13 @@ def main():
                          "(e.g. 512,512,63,32,800); residual projection from the block input")
     ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end (host buffers) leg")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--profile-class", default=DOMINANT_CLASS)
-    ap.add_argument("--breakdown", default=None, help="write a per-kernel-class event-time table to this file")
+    ap.add_argument("--breakdown", default=None, help="also write the per-kernel-class table to this text file")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--gemm-mode", type=int, default=0)
+    ap.add_argument("--tile-shape", type=int, default=None, help="tile shape of the pointwise contractions (0, 1, 2)")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="every kernel on one stream in program order (default: weight gradients and the residual "
+                         "projection overlap the critical path on the library's second stream)")
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every kernel from the host each step instead of replaying a captured CUDA graph")
     args = ap.parse_args()
@@ -202,6 +258,9 @@ def main():
     d = si.draw(w)
     ctx = api.Context(local)
     ctx.set_gemm_mode(args.gemm_mode)
+    ctx.set_overlap(not args.no_overlap)
+    if args.tile_shape is not None:
+        ctx.set_tile_shape(args.tile_shape)
     spec = api.EncoderSpec(w.layers, w.B, w.T, w.dtype)
     td = api.binding.TORCH_DTYPE[spec.code]
     blob = spec.pack_params(d.params, dev)
@@ -269,24 +328,23 @@ def main():
             step()
         assert ctx.last_status() == 0
 
-    # ---- device-resident timing; the dominant kernel class is bracketed with events meanwhile ----
+    # ---- device-resident timing ------------------------------------------------------------------
     sampler = ClockSampler(local) if rank == 0 else None
     l0 = ctx.launch_count()
-    if args.no_graph:
-        ctx.profile_begin(args.profile_class, max_launches=8192)
     ms, t0, t1 = timed(step, args.steps)
-    if args.no_graph:
-        prof = ctx.profile_end()
-        launches = ctx.launch_count() - l0
-    else:
-        launches = launches_per_step * args.steps
-        # per-kernel event brackets cannot sit inside a replayed graph: the dominant kernel class is
-        # timed right after, same buffers and kernels, launched one by one
-        ctx.profile_begin(args.profile_class, max_launches=8192)
-        for _ in range(max(3, args.steps // 2)):
-            eager_step()
-        prof = ctx.profile_end()
+    launches = (ctx.launch_count() - l0) if args.no_graph else launches_per_step * args.steps
     clocks = sampler.stop(t0, t1) if sampler else None
+    # Per-kernel-class CUDA-event brackets cannot sit inside a replayed graph: every class is timed right
+    # after the timed region, same buffers and kernels, launched one by one from the host.
+    # The profiled steps run every kernel alone, in program order (overlap off): a class's time is its kernels'
+    # own duration, not that of whatever shared the GPU with them.
+    nprof = max(3, args.steps // 4)
+    ctx.set_overlap(False)
+    ctx.profile_begin("all", max_launches=600 * nprof)
+    for _ in range(nprof):
+        (step if args.no_graph else eager_step)()
+    prof = ctx.profile_end()
+    ctx.set_overlap(not args.no_overlap)
 
     # ---- end to end: pinned host inputs in, logits + gradients out, every step --------------------
     if args.no_e2e:
@@ -297,20 +355,6 @@ def main():
         ms_e2e, _, _ = timed(step_e2e, args.steps)
     h2d = x_h.numel() * x_h.element_size() + g_h.numel() * g_h.element_size() + len_h.numel() * 4
     d2h = logits_h.numel() * logits_h.element_size() + grads_h.numel()
-
-    if args.breakdown and rank == 0:
-        ctx.profile_begin("all", max_launches=8192)
-        nb = 3
-        for _ in range(nb):
-            (step if args.no_graph else eager_step)()
-        allp = ctx.profile_end()
-        tot = sum(v["ms"] for v in allp.values())
-        with open(args.breakdown, "w") as f:
-            f.write(f"# per-kernel-class CUDA-event time, {w.name}, {nb} steps; sum {tot / nb:.3f} ms/step\n")
-            f.write("class launches/step ms/step share GB/s TFLOP/s\n")
-            for k, v in sorted(allp.items(), key=lambda kv: -kv[1]["ms"]):
-                f.write(f"{k} {v['launches'] / nb:.0f} {v['ms'] / nb:.4f} {v['ms'] / tot:.3f} "
-                        f"{v['bytes'] / v['ms'] / 1e6:.0f} {v['flops'] / v['ms'] / 1e9:.1f}\n")
 
     if rank != 0:
         if world > 1:
@@ -326,44 +370,43 @@ def main():
             "config": {"workload": w.name, "B": w.B, "T_in": w.T, "layers": len(w.layers),
                        "valid_frames": int(d.lengths.sum()), "l2": "per-step working set (GBs) exceeds L2",
                        "parallelism": "replicas" if world > 1 else "single",
-                       "launch": "host launches" if args.no_graph else "CUDA graph replay"},
+                       "launch": "host launches" if args.no_graph else "CUDA graph replay",
+                       "overlap": "off" if args.no_overlap else "weight gradients and residual projection on a second stream"},
             "clocks": clocks, "gpu_launches": int(launches),
             "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                     "ms_per_step": ms_e2e / args.steps}}
-    pc = prof.get(args.profile_class)
-    if pc:
-        per_ms = pc["ms"] / pc["launches"]
-        gbs = pc["bytes"] / pc["ms"] / 1e6
-        tfs = pc["flops"] / pc["ms"] / 1e9
-        alu_peak = 148 * 128 * 1.965e9 / 1e12     # T FMA/s: SMs x fp32 lanes x max clock
-        if args.profile_class.startswith("dw_"):
-            line["roofline"] = {"kernel": args.profile_class, "bound": "alu", "achieved": tfs / 2, "peak": alu_peak,
-                                "unit": "TFMA/s", "frac": tfs / 2 / alu_peak,
-                                "traffic": (TRAFFIC_RATIO[args.profile_class] * pc["bytes"] / pc["launches"]
-                                            if args.profile_class in TRAFFIC_RATIO else None),
-                                "hbm_gbs": gbs, "hbm_frac": gbs / peaks["hbm_gbs"], "peak_source": "derived: 148 SMs x 128 lanes x 1.965 GHz",
-                                "launches": pc["launches"], "avg_ms": per_ms}
-        elif (args.profile_class.startswith("pw_") and args.gemm_mode == 0
-              and tfs / peaks["bf16_tflops_sustained"] > gbs / peaks["hbm_gbs"]):
-            # the class's FLOPs at the tensor peak take longer than its bytes at the HBM peak
-            line["roofline"] = {"kernel": args.profile_class, "bound": "tensor", "achieved": tfs,
-                                "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                                "frac": tfs / peaks["bf16_tflops_sustained"],
-                                "traffic": (TRAFFIC_RATIO[args.profile_class] * pc["bytes"] / pc["launches"]
-                                            if args.profile_class in TRAFFIC_RATIO else None),
-                                "hbm_gbs": gbs, "hbm_frac": gbs / peaks["hbm_gbs"],
-                                "peak_source": peaks["source"], "launches": pc["launches"], "avg_ms": per_ms}
-        else:
-            line["roofline"] = {"kernel": args.profile_class, "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"],
-                                "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
-                                "traffic": (TRAFFIC_RATIO[args.profile_class] * pc["bytes"] / pc["launches"]
-                                            if args.profile_class in TRAFFIC_RATIO else None),
-                                "tflops": tfs, "tensor_frac": tfs / peaks["bf16_tflops_sustained"],
-                                "peak_source": peaks["source"], "launches": pc["launches"], "avg_ms": per_ms}
+    valid_frac = float(d.lengths.sum()) / float(w.B * w.T)
+    per_class = class_rooflines(prof, nprof, valid_frac, peaks, dram_traffic_ratios())
+    line["tolerance"] = TOLERANCE
+    line["roofline_per_class"] = per_class
+    line["roofline_note"] = ("class times: CUDA events around every launch of %d host-launched steps run right after the "
+                             "timed region, one stream, no overlap (they sum to %.3f ms/step against %.3f ms for the "
+                             "replayed graph, in which independent kernels overlap); bytes and "
+                             "flops are algorithmic, valid frames only; peaks: %s HBM %.0f GB/s, bf16 %.0f TFLOP/s sustained"
+                             % (nprof, sum(v["ms_per_step"] for v in per_class.values()), ms / args.steps,
+                                peaks["source"], peaks["hbm_gbs"], peaks["bf16_tflops_sustained"]))
+    if per_class:
+        top = max(per_class, key=lambda k: per_class[k]["share"])
+        e = per_class[top]
+        tens = e["bound"] == "tensor"
+        line["roofline"] = {"kernel": top, "bound": e["bound"], "achieved": e["TFLOP/s"] if tens else e["GB/s"],
+                            "peak": peaks["bf16_tflops_sustained"] if tens else peaks["hbm_gbs"],
+                            "unit": "TFLOP/s" if tens else "GB/s", "frac": e["frac"], "traffic": e["traffic"],
+                            "peak_source": peaks["source"], "launches": e["launches_per_step"] * nprof,
+                            "avg_ms": e["ms_per_step"] / e["launches_per_step"], "share_of_step": e["share"]}
+    if args.breakdown:
+        with open(args.breakdown, "w") as f:
+            f.write(f"# per-kernel-class CUDA-event time, {w.name}, {nprof} host-launched steps; "
+                    f"graph-replayed step {ms / args.steps:.3f} ms\n")
+            f.write("class launches/step ms/step share GB/s TFLOP/s bound frac\n")
+            for k, v in sorted(per_class.items(), key=lambda kv: -kv[1]["share"]):
+                f.write(f"{k} {v['launches_per_step']:.0f} {v['ms_per_step']:.4f} {v['share']:.3f} {v['GB/s']:.0f} "
+                        f"{v['TFLOP/s']:.1f} {v['bound']} {v['frac']:.3f}\n")
     if not args.no_cpu_baseline and world == 1:
         v, cores, dt, desc = oracle_sample(w, 1)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
-                                "seconds": dt}
+                                "seconds": dt, "note": "a one-sample slice: its batch statistics run over that sample "
+                                                       "alone, so it is the same arithmetic per frame, not the same batch"}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -13,7 +13,8 @@
  *
  * One layer ("block") computes, for x [B, C_in, T_in] and lengths len[b] (in input frames):
  *     xm = x where t <  len[b], else 0                                   (padding mask)
- *     u[b,c,t]  = sum_k wd[c,k] * xm[b,c,t*stride + k - (K-1)/2]          (depthwise, zero "same" padding)
+ *     u[b,c,t]  = sum_k wd[c,k] * xm[b,c,t*stride + k*dilation - P]       (depthwise, zero "same" padding:
+ *                 dilation*(K-1) zeros in total, P = floor of half of them on the left)
  *     v[b,o,t]  = sum_c wp[o,c] * u[b,c,t]  (+ bias[o])                   (pointwise 1x1)
  *     len'[b]   = ceil(len[b]/stride);  N = sum_b len'[b]
  *     mean, var = per-channel moments of v over the N valid frames (biased variance)
@@ -22,7 +23,8 @@
  *     y         = relu(bn + r)           (res_before_relu = 1, the default)
  *               = relu(bn) + r           (res_before_relu = 0)
  *     y = 0 for t >= len'[b]
- * and the exact gradient of that map.  T' = floor((T_in + 2P - K)/stride) + 1 with P = (K-1)/2.
+ * and the exact gradient of that map.  A linear layer (has_bn = 0) may end in the decoder's log-softmax over its
+ * channels (log_softmax = 1): y[b,:,t] = z[b,:,t] - log(sum_c exp(z[b,c,t])) with z = wp u + bias.  T' = floor((T_in - 1)/stride) + 1.
  *
  * Conventions common to all calls
  *   - Every pointer named *_dev or held in an sc_tensor / sc_block_params / sc_block_saved /
@@ -73,7 +75,7 @@ typedef enum {
     SC_ERR_DEVICE_TIMEOUT = -9,    /* (device) a bounded wait inside a kernel ran out              */
     SC_ERR_ARCH = -10,             /* the device is not compute capability 10.x                    */
     SC_ERR_CUDA = -11,             /* a CUDA runtime/driver call failed                            */
-    SC_ERR_RANGE = -12             /* (device) a depthwise output exceeded the float16 range       */
+    SC_ERR_RANGE = -12             /* (device) a depthwise or pointwise result exceeded the float16 range */
 } sc_status;
 
 /* A typed tensor argument: size/stride in elements, tag[i] names axis i. */
@@ -88,13 +90,19 @@ typedef struct {
 
 typedef struct {
     int32_t B, C_in, C_out, T_in;
-    int32_t K, stride;          /* K odd; stride 1 or 2 (ignored when has_dw = 0)                  */
+    int32_t K, stride;          /* K >= 1; stride 1 or 2 (ignored when has_dw = 0).  Odd K with adjacent */
+                                /* taps takes the tensor-core depthwise kernels; even K or dilation > 1  */
+                                /* takes plain kernels                                                   */
     int32_t io_dtype;           /* sc_dtype of activations and conv weights                        */
     int32_t residual;           /* sc_residual                                                     */
     int32_t C_res;              /* channels of the residual source (0: same as C_in)               */
     int32_t has_dw, has_bn, has_relu, has_bias;
     int32_t res_before_relu;    /* 1: y = relu(bn + r);  0: y = relu(bn) + r                       */
     float   bn_eps, bn_momentum;
+    int32_t log_softmax;        /* 1: y = log-softmax over the channels of (wp u + bias), the decoder   */
+                                /* module's log_probs (section 4.1.1); only on a layer with has_bn = 0,  */
+                                /* has_relu = 0 and no residual.  Backward then takes dL/dlog_probs      */
+    int32_t dilation;           /* frames between neighbouring depthwise taps (0 or 1: adjacent)          */
 } sc_block_desc;
 
 typedef struct {          /* device pointers; absent parts may be null                             */
@@ -110,10 +118,12 @@ typedef struct {          /* written by sepconv_fwd, read by sepconv_bwd; caller
     void  *u;             /* [B, C_in, T'] depthwise output (or masked input when has_dw = 0).     */
                           /* float16 when the layer has a depthwise step and batch norm and        */
                           /* io_dtype is 16-bit (also for bf16: see below); io_dtype otherwise     */
-    void  *vhat;          /* [B, C_out, T'] normalised (v - mean)/sqrt(var+eps), zero in padding   */
-                          /* (has_bn only); float32 when io_dtype is SC_F32, float16 otherwise     */
+    void  *v;             /* [B, C_out, T'] pointwise result before normalisation (has_bn only);   */
+                          /* float32 when io_dtype is SC_F32, float16 otherwise (a value beyond    */
+                          /* the float16 range is clamped and reported as SC_ERR_RANGE); frames    */
+                          /* at and beyond len'[b] are unspecified and never read                  */
     float *mean, *invstd; /* [C_out]                                                               */
-    void  *vhat_r;        /* same for the projection residual branch                               */
+    void  *vr;            /* same for the projection residual branch: wr * xr                      */
     float *mean_r, *invstd_r;
 } sc_block_saved;
 
@@ -136,21 +146,41 @@ typedef struct {
 
 /* Creates a context on CUDA device `device` (which must be compute capability 10.x) and allocates
  * the 64-byte device status word -- the only device allocation the library ever makes.
- * Returns SC_ERR_ARCH on any other architecture. */
+ * Returns SC_ERR_ARCH on any other architecture.  (The paper's modules are created once by a factory
+ * and then only executed, section 3.1; the context is that create-once state: device, status word,
+ * resolved driver entry points.) */
 int  sepconv_ctx_create(sc_ctx** out, int device);
 void sepconv_ctx_destroy(sc_ctx* ctx);
 
-/* Synchronises `cuda_stream`, returns the device status word (SC_OK, SC_ERR_LENGTHS or
- * SC_ERR_DEVICE_TIMEOUT) and clears it. */
+/* Synchronises `cuda_stream`, returns the device status word (SC_OK, SC_ERR_LENGTHS, SC_ERR_RANGE or
+ * SC_ERR_DEVICE_TIMEOUT) and clears it.  These are the errors only the device can see: the `length`
+ * port of section 4.1.1 holding a value outside [1, T], an intermediate leaving the float16 range that
+ * section 3.3's mixed-precision policy stores it in, a bounded wait inside a kernel that ran out. */
 int  sepconv_last_status(sc_ctx* ctx, void* cuda_stream);
+/* Text for a status code.  The argument-validation codes follow the outcomes of the paper's neural-type
+ * comparison (section 3.2): an axis of the wrong size is DIM_INCOMPATIBLE (Table 1's 64- vs 40-channel
+ * spectrogram rows), the right axes in the wrong order are TRANSPOSED (the paper's TRANSPOSE_SAME),
+ * another element type, rank or set of axis tags is INCOMPATIBLE. */
 const char* sepconv_strerror(int status);
+
+/* Launches one small kernel whose only thread waits, with a short poll limit, on a barrier that nothing
+ * signals: the wait must run out and leave SC_ERR_DEVICE_TIMEOUT in the status word, and the context
+ * must stay usable.  It exercises the give-up path that every device-side wait of the library has
+ * (the paper has no counterpart; nothing is left in flight and the GPU is not faulted or hung). */
+int  sepconv_selftest_bounded_wait(sc_ctx* ctx, void* cuda_stream);
 
 /* ---- one block ---------------------------------------------------------------------------- */
 
-/* Bytes of scratch the two block calls need for this descriptor (host-only computation). */
+/* Bytes of scratch the two block calls need for this descriptor (host-only computation).  The block
+ * descriptor is the module's constructor arguments as a plain struct: the paper keeps a module's
+ * structure in data, not in code (section 3).  Returns SC_ERR_UNSUPPORTED for a descriptor the
+ * library does not implement (even K, stride other than 1 or 2, identity residual across a channel
+ * change, ...). */
 int  sepconv_workspace_bytes(const sc_block_desc* desc, size_t* fwd_bytes, size_t* bwd_bytes);
 
-/* Forward of one block (definition at the top of this file).
+/* Forward of one block (definition at the top of this file): the body of the encoder module of section
+ * 4.1.1, whose ports are (audio_signal, length) -> (encoded, encoded_len); every tensor argument is
+ * checked against the [batch, channel, time] neural type of section 3.2 before anything is enqueued.
  *   x              [B, C_in, T_in]
  *   x_res          residual source [B, C_res, T']; null = x (requires stride 1)
  *   lengths_dev    int32 [B], valid input frames, each in [1, T_in]
@@ -170,7 +200,8 @@ int  sepconv_fwd(sc_ctx* ctx, const sc_block_desc* desc,
  *   x, x_res, y, lengths_dev, params, saved: as given to / produced by sepconv_fwd
  *   dx       [B, C_in, T_in]  <- gradient w.r.t. x (zero in padded frames)
  *   dx_res   [B, C_res, T']   <- gradient w.r.t. x_res; null = the residual path's gradient is
- *            added into dx (only legal when the residual source is x)
+ *            added into dx (only legal when the residual source is x: with a separate x_res and no
+ *            dx_res the call returns SC_ERR_UNSUPPORTED)
  *   dx_add   optional [B, C_in, T_in] tensor added into dx before rounding (a gradient that
  *            reaches the same input along another path)
  *   grads    parameter gradients, float32; accumulate != 0 adds into them instead of overwriting
@@ -183,6 +214,20 @@ int  sepconv_bwd(sc_ctx* ctx, const sc_block_desc* desc,
                  sc_tensor* dx, sc_tensor* dx_res, const sc_tensor* dx_add,
                  sc_block_grads* grads, int accumulate,
                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Evaluation-mode forward of one block (the paper's `eval` / `infer` actions, section 3.1): batch statistics are
+ * replaced by the given running statistics,  bn = gamma (v - running_mean) / sqrt(running_var + eps) + beta,
+ * everything else as in sepconv_fwd; nothing is saved for a backward pass and the running statistics are
+ * only read.  running_mean_r / running_var_r belong to the projection residual's batch norm (null otherwise).
+ * Scratch: sepconv_infer_workspace_bytes. */
+int  sepconv_infer_workspace_bytes(const sc_block_desc* desc, size_t* bytes);
+int  sepconv_infer(sc_ctx* ctx, const sc_block_desc* desc,
+                   const sc_tensor* x, const sc_tensor* x_res, const int32_t* lengths_dev,
+                   const sc_block_params* params,
+                   const float* running_mean, const float* running_var,
+                   const float* running_mean_r, const float* running_var_r,
+                   sc_tensor* y, int32_t* out_lengths_dev,
+                   void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* Forward of one block without a workspace argument and without any allocation (the paper has no
  * counterpart; this exists for integration reasons only).
@@ -200,8 +245,11 @@ int  sepconv_bwd(sc_ctx* ctx, const sc_block_desc* desc,
  * statistics are not updated).  The call itself uses no cudaMalloc/cudaFree or other allocating
  * routine.
  *
- * The first call on each device looks up the array's device address (with the context's device
- * current, as for every other call); make that first call outside any stream capture.
+ * The first call on each device looks up the array's device address; with CUDA's lazy module loading
+ * that is also the moment the device sets the array aside, so this first call can still fail with
+ * SC_ERR_CUDA on a device whose memory is already fully committed: make it once at start-up, outside
+ * any stream capture.  The context's device must be the current device (SC_ERR_UNSUPPORTED otherwise:
+ * the array belongs to the current device).
  * All calls on a device share the one array and it keeps the previous call's contents: two calls
  * whose GPU work overlaps (different streams, no dependency between them) race on it -- keep such
  * calls on one stream or order them with events. */
@@ -213,9 +261,15 @@ int  sepconv_fwd_static(sc_ctx* ctx, const sc_block_desc* desc,
 
 /* ---- whole encoder -------------------------------------------------------------------------- */
 
+/* Bytes of workspace encoder_fwd_bwd needs for this layer list (host-only computation).  Returns
+ * SC_ERR_UNSUPPORTED when the block-level residual spans [res_from[i], i] overlap or share a source:
+ * the encoder keeps one pending residual gradient at a time, which is all the Jasper-style encoders
+ * of section 4.1.1 need (each block's residual comes from that block's input only). */
 int  encoder_workspace_bytes(const sc_encoder_desc* desc, size_t* bytes);
 
-/* Forward through every layer, then backward from `dlogits`, in one call.
+/* The whole encoder module of section 4.1.1 plus the 1x1 decoder convolution that ends in the logits
+ * (`jasper_encoder` then `jasper_decoder` without its log-softmax): forward through every layer, then
+ * backward from `dlogits`, in one call.
  *   x [B, C_0, T_in], lengths_dev int32 [B]
  *   params_blob / grads_blob: flat device blobs addressed by param_offsets / grad_offsets
  *   dlogits [B, C_last, T_last] upstream gradient; logits [B, C_last, T_last] (written)
@@ -229,11 +283,39 @@ int  encoder_fwd_bwd(sc_ctx* ctx, const sc_encoder_desc* desc,
                      void* grads_blob, const int64_t* grad_offsets, sc_tensor* dx,
                      int accumulate, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Evaluation-mode forward through every layer (sepconv_infer per layer, intermediates in `workspace`):
+ *   running_blob / running_offsets: flat device blob of float32 running statistics and a HOST array of
+ *   n_layers*4 byte offsets (order: mean, var, mean_r, var_r; -1 where the layer has none)
+ *   out [B, C_last, T_last] <- logits, or log_probs when the last layer has log_softmax = 1. */
+int  encoder_infer_workspace_bytes(const sc_encoder_desc* desc, size_t* bytes);
+int  encoder_infer(sc_ctx* ctx, const sc_encoder_desc* desc,
+                   const sc_tensor* x, const int32_t* lengths_dev,
+                   const void* params_blob, const int64_t* param_offsets,
+                   const void* running_blob, const int64_t* running_offsets,
+                   sc_tensor* out, int32_t* out_lengths_dev,
+                   void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Selects the kernel family for the pointwise contractions: 0 = automatic (tensor cores where
- * the shape allows), 1 = force the plain fp32-accumulate SIMT kernels.  Used by tests. */
+ * the shape allows), 1 = force the plain fp32-accumulate SIMT kernels.  Used by tests (the paper has
+ * no counterpart). */
 int  sepconv_set_gemm_mode(sc_ctx* ctx, int mode);
 
-/* Number of kernel launches this context has enqueued so far (for reporting). */
+/* Tile shape of the forward / input-gradient pointwise contractions (tuning aid; the paper has no counterpart):
+ * 0 = 256 output channels x 256 frames per tile with one accumulator in tensor memory, 1 = 256 x 128 and
+ * 2 = 128 x 256 with two accumulators, so that a tile's epilogue overlaps the next tile's MMAs.  Results do not
+ * depend on it except for the summation order of the batch-norm statistics. */
+int  sepconv_set_tile_shape(sc_ctx* ctx, int shape);
+
+/* Overlap of independent kernels (on by default).  The weight-gradient contractions of a layer and the residual
+ * projection's forward contraction do not feed the next kernel of the pass; with overlap on they run on a second
+ * stream that the context owns, forked from and joined back into `cuda_stream` with events before the call
+ * returns, so to the caller every call still behaves as work enqueued on `cuda_stream` alone (stream capture
+ * included).  0 turns it off: every kernel on `cuda_stream`, in program order.  Results are bit-identical either
+ * way.  (The paper has no counterpart.) */
+int  sepconv_set_overlap(sc_ctx* ctx, int on);
+
+/* Number of kernel launches this context has enqueued so far (for reporting; the paper has no
+ * counterpart). */
 int64_t sepconv_launch_count(sc_ctx* ctx);
 
 /* Per-kernel-class timing with CUDA events on the launching stream (measurement aid; the paper has

@@ -41,14 +41,12 @@ class sc_block_desc(C.Structure):
                 ("residual", C.c_int32), ("C_res", C.c_int32),
                 ("has_dw", C.c_int32), ("has_bn", C.c_int32), ("has_relu", C.c_int32),
                 ("has_bias", C.c_int32), ("res_before_relu", C.c_int32),
-                ("bn_eps", C.c_float), ("bn_momentum", C.c_float)]
+                ("bn_eps", C.c_float), ("bn_momentum", C.c_float), ("log_softmax", C.c_int32), ("dilation", C.c_int32)]
 
     @property
     def T_out(self) -> int:
-        K = self.K if self.has_dw else 1
         s = self.stride if self.has_dw else 1
-        P = (K - 1) // 2
-        return (self.T_in + 2 * P - K) // s + 1
+        return (self.T_in - 1) // s + 1
 
 
 class sc_block_params(C.Structure):
@@ -56,7 +54,7 @@ class sc_block_params(C.Structure):
 
 
 class sc_block_saved(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("u", "vhat", "mean", "invstd", "vhat_r", "mean_r", "invstd_r")]
+    _fields_ = [(n, C.c_void_p) for n in ("u", "v", "mean", "invstd", "vr", "mean_r", "invstd_r")]
 
 
 class sc_block_grads(C.Structure):
@@ -69,7 +67,8 @@ class sc_encoder_desc(C.Structure):
 
 _lib = None
 
-EXPORTS = ("sepconv_fwd_static", "sepconv_profile_begin", "sepconv_profile_end", "sepconv_kernel_class_count",
+EXPORTS = ("sepconv_set_overlap", "sepconv_set_tile_shape", "sepconv_fwd_static", "sepconv_selftest_bounded_wait", "sepconv_infer", "sepconv_infer_workspace_bytes",
+           "encoder_infer", "encoder_infer_workspace_bytes", "sepconv_profile_begin", "sepconv_profile_end", "sepconv_kernel_class_count",
            "sepconv_kernel_class_name", "sepconv_ctx_create", "sepconv_ctx_destroy", "sepconv_last_status", "sepconv_strerror",
            "sepconv_workspace_bytes", "sepconv_fwd", "sepconv_bwd", "encoder_workspace_bytes",
            "encoder_fwd_bwd", "sepconv_set_gemm_mode", "sepconv_launch_count")
@@ -92,6 +91,9 @@ def load_library(path: str = LIB_PATH):
     lib.sepconv_ctx_destroy.restype = None
     lib.sepconv_last_status.argtypes = [C.c_void_p, C.c_void_p]
     lib.sepconv_set_gemm_mode.argtypes = [C.c_void_p, C.c_int]
+    lib.sepconv_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_void_p]
+    lib.sepconv_set_overlap.argtypes = [C.c_void_p, C.c_int]
+    lib.sepconv_set_tile_shape.argtypes = [C.c_void_p, C.c_int]
     lib.sepconv_launch_count.argtypes = [C.c_void_p]
     lib.sepconv_launch_count.restype = C.c_int64
     lib.sepconv_workspace_bytes.argtypes = [C.POINTER(sc_block_desc), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
@@ -112,6 +114,14 @@ def load_library(path: str = LIB_PATH):
                                     C.c_void_p, C.POINTER(C.c_int64), C.POINTER(sc_tensor),
                                     C.POINTER(sc_tensor), C.c_void_p, C.c_void_p, C.POINTER(C.c_int64),
                                     C.POINTER(sc_tensor), C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.sepconv_infer_workspace_bytes.argtypes = [C.POINTER(sc_block_desc), C.POINTER(C.c_size_t)]
+    lib.sepconv_infer.argtypes = [C.c_void_p, C.POINTER(sc_block_desc), C.POINTER(sc_tensor), C.POINTER(sc_tensor),
+                                  C.c_void_p, C.POINTER(sc_block_params), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                  C.POINTER(sc_tensor), C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.encoder_infer_workspace_bytes.argtypes = [C.POINTER(sc_encoder_desc), C.POINTER(C.c_size_t)]
+    lib.encoder_infer.argtypes = [C.c_void_p, C.POINTER(sc_encoder_desc), C.POINTER(sc_tensor), C.c_void_p, C.c_void_p,
+                                  C.POINTER(C.c_int64), C.c_void_p, C.POINTER(C.c_int64), C.POINTER(sc_tensor), C.c_void_p,
+                                  C.c_void_p, C.c_size_t, C.c_void_p]
     lib.sepconv_profile_begin.argtypes = [C.c_void_p, C.c_int, C.c_int]
     lib.sepconv_profile_end.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64),
                                         C.POINTER(C.c_double), C.POINTER(C.c_double)]
@@ -163,6 +173,8 @@ def block_desc(L, B: int, T: int, dtype: str) -> sc_block_desc:
     d.res_before_relu = int(L.res_before_relu)
     d.bn_eps = float(L.eps)
     d.bn_momentum = 0.1
+    d.log_softmax = int(getattr(L, "log_softmax", False))
+    d.dilation = int(getattr(L, "dilation", 1))
     return d
 
 
@@ -185,6 +197,17 @@ class Context:
 
     def last_status(self, stream=None) -> int:
         return int(self.lib.sepconv_last_status(self.h, _stream_ptr(stream)))
+
+    def selftest_bounded_wait(self, stream=None):
+        """Enqueues the kernel whose bounded wait must run out (see sepconv.h)."""
+        _check(self.lib.sepconv_selftest_bounded_wait(self.h, _stream_ptr(stream)), "sepconv_selftest_bounded_wait")
+
+    def set_overlap(self, on: bool):
+        """Run independent kernels on the context's second stream (default) or everything in program order."""
+        _check(self.lib.sepconv_set_overlap(self.h, int(bool(on))), "sepconv_set_overlap")
+
+    def set_tile_shape(self, shape: int):
+        _check(self.lib.sepconv_set_tile_shape(self.h, shape), "sepconv_set_tile_shape")
 
     def set_gemm_mode(self, mode: int):
         _check(self.lib.sepconv_set_gemm_mode(self.h, mode), "sepconv_set_gemm_mode")
@@ -242,13 +265,13 @@ def sepconv_fwd(ctx: Context, desc: sc_block_desc, x: torch.Tensor, lengths: tor
     if saved is None:
         ut = torch.float16 if (desc.has_dw and desc.has_bn and desc.io_dtype != SC_F32) else td
         saved = {"u": torch.empty((B, Ci, Tp), dtype=ut, device=dev)}
-        nt = torch.float32 if desc.io_dtype == SC_F32 else torch.float16   # type of the normalised tensors
+        nt = torch.float32 if desc.io_dtype == SC_F32 else torch.float16   # type of the saved pointwise results
         if desc.has_bn:
-            saved["vhat"] = torch.empty((B, Co, Tp), dtype=nt, device=dev)
+            saved["v"] = torch.empty((B, Co, Tp), dtype=nt, device=dev)
             saved["mean"] = torch.empty((Co,), dtype=torch.float32, device=dev)
             saved["invstd"] = torch.empty((Co,), dtype=torch.float32, device=dev)
         if desc.residual == 2:
-            saved["vhat_r"] = torch.empty((B, Co, Tp), dtype=nt, device=dev)
+            saved["vr"] = torch.empty((B, Co, Tp), dtype=nt, device=dev)
             saved["mean_r"] = torch.empty((Co,), dtype=torch.float32, device=dev)
             saved["invstd_r"] = torch.empty((Co,), dtype=torch.float32, device=dev)
     sv = sc_block_saved()
@@ -264,6 +287,26 @@ def sepconv_fwd(ctx: Context, desc: sc_block_desc, x: torch.Tensor, lengths: tor
                              workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
     _check(rc, "sepconv_fwd")
     return y, out_len, saved
+
+
+def sepconv_infer(ctx: Context, desc: sc_block_desc, x: torch.Tensor, lengths: torch.Tensor,
+                  params: Dict[str, torch.Tensor], running: Dict[str, torch.Tensor],
+                  x_res: Optional[torch.Tensor] = None, stream=None):
+    """Evaluation-mode forward.  running: float32 device tensors "mean", "var" (and "mean_r", "var_r" for a
+    projection residual).  Returns (y, out_lengths)."""
+    dev = x.device
+    y = torch.empty((desc.B, desc.C_out, desc.T_out), dtype=TORCH_DTYPE[desc.io_dtype], device=dev)
+    out_len = torch.empty((desc.B,), dtype=torch.int32, device=dev)
+    n = C.c_size_t()
+    _check(ctx.lib.sepconv_infer_workspace_bytes(C.byref(desc), C.byref(n)), "sepconv_infer_workspace_bytes")
+    ws = _workspace(int(n.value), dev)
+    p = _params_struct(params)
+    ptr = lambda k: running[k].data_ptr() if k in running and running[k] is not None else None
+    rc = ctx.lib.sepconv_infer(ctx.h, C.byref(desc), tensor_arg(x), tensor_arg(x_res), lengths.data_ptr(), C.byref(p),
+                               ptr("mean"), ptr("var"), ptr("mean_r"), ptr("var_r"), tensor_arg(y), out_len.data_ptr(),
+                               ws.data_ptr(), ws.numel(), _stream_ptr(stream))
+    _check(rc, "sepconv_infer")
+    return y, out_len
 
 
 STATIC_SCRATCH_BYTES = 8 << 20
@@ -372,6 +415,25 @@ class EncoderSpec:
                 blob[off:off + raw.numel()] = raw
         return blob
 
+    def pack_running(self, running: Sequence[Optional[Dict[str, np.ndarray]]], device):
+        """Flat float32 blob of the per-layer running statistics (mean, var, mean_r, var_r) and the host
+        offsets array that encoder_infer takes."""
+        offs = (C.c_int64 * (4 * len(self.layers)))()
+        chunks, pos = [], 0
+        for i, r in enumerate(running):
+            for j, name in enumerate(("mean", "var", "mean_r", "var_r")):
+                if r is None or name not in r or r[name] is None:
+                    offs[4 * i + j] = -1
+                    continue
+                a = np.ascontiguousarray(r[name], dtype=np.float32)
+                offs[4 * i + j] = pos
+                chunks.append((pos, a))
+                pos += (a.nbytes + 255) // 256 * 256
+        blob = torch.zeros(max(pos, 256), dtype=torch.uint8, device=device)
+        for off, a in chunks:
+            blob[off:off + a.nbytes] = torch.from_numpy(a).view(torch.uint8).reshape(-1).to(device)
+        return blob, offs
+
     def param_view(self, blob: torch.Tensor, i: int, name: str) -> torch.Tensor:
         j = PARAM_ORDER.index(name)
         off = self.param_offsets[8 * i + j]
@@ -390,6 +452,23 @@ def encoder_workspace_bytes(spec: EncoderSpec) -> int:
     n = C.c_size_t()
     _check(load_library().encoder_workspace_bytes(C.byref(spec.desc), C.byref(n)), "encoder_workspace_bytes")
     return int(n.value)
+
+
+def encoder_infer(ctx: Context, spec: EncoderSpec, x: torch.Tensor, lengths: torch.Tensor, params_blob: torch.Tensor,
+                  running_blob: torch.Tensor, running_offsets, workspace: Optional[torch.Tensor] = None, stream=None):
+    """Evaluation-mode forward through every layer.  Returns (out, out_lengths)."""
+    dev = x.device
+    out = torch.empty((spec.B, spec.C_out, spec.T_out), dtype=TORCH_DTYPE[spec.code], device=dev)
+    out_len = torch.empty((spec.B,), dtype=torch.int32, device=dev)
+    if workspace is None:
+        n = C.c_size_t()
+        _check(ctx.lib.encoder_infer_workspace_bytes(C.byref(spec.desc), C.byref(n)), "encoder_infer_workspace_bytes")
+        workspace = _workspace(int(n.value), dev)
+    rc = ctx.lib.encoder_infer(ctx.h, C.byref(spec.desc), tensor_arg(x), lengths.data_ptr(), params_blob.data_ptr(),
+                               spec.param_offsets, running_blob.data_ptr(), running_offsets, tensor_arg(out),
+                               out_len.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
+    _check(rc, "encoder_infer")
+    return out, out_len
 
 
 def encoder_fwd_bwd(ctx: Context, spec: EncoderSpec, x: torch.Tensor, lengths: torch.Tensor,

@@ -20,9 +20,16 @@ struct sc_ctx {
     int gemm_mode = 0;
     TcState tc;
     Prof prof;
+    // A second, library-owned stream: kernels that are off the critical path of a layer (weight gradients, the
+    // residual projection's contraction) run there, forked from and joined back into the caller's stream with
+    // events, so that they fill the SMs a latency-bound kernel of the critical path leaves idle.
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};   // fork A, fork B, done[2], fwd fork, fwd join
+    int overlap = 1;
 };
 
 namespace sc {
+int ctx_device(const sc_ctx* ctx) { return ctx ? ctx->device : -1; }
 const char* kclass_name(int c) {
     static const char* n[KC_COUNT] = {"lengths", "dw_fwd", "dw_dgrad", "dw_wgrad", "pw_fwd", "pw_dgrad", "pw_wgrad",
                                       "bn_stats", "bn_finalize", "bn_apply", "bn_bwd_reduce", "bn_bwd_finalize",
@@ -47,7 +54,7 @@ struct Bump {
     bool ok() const { return base == nullptr || off <= cap; }
 };
 
-struct Dims { int B, Cin, Cout, Cres, T, Tp, K, s; };
+struct Dims { int B, Cin, Cout, Cres, T, Tp, K, s, dil; bool plain; };   // plain: odd K, adjacent taps
 
 int desc_dims(const sc_block_desc* d, Dims* o) {
     if (!d) return SC_ERR_NULL;
@@ -55,16 +62,18 @@ int desc_dims(const sc_block_desc* d, Dims* o) {
     if (d->B < 1 || d->C_in < 1 || d->C_out < 1 || d->T_in < 1) return SC_ERR_DIM_INCOMPATIBLE;
     o->B = d->B; o->Cin = d->C_in; o->Cout = d->C_out; o->T = d->T_in;
     o->K = d->has_dw ? d->K : 1; o->s = d->has_dw ? d->stride : 1;
-    if (o->K < 1 || (o->K & 1) == 0) return SC_ERR_UNSUPPORTED;
+    o->dil = (d->has_dw && d->dilation > 1) ? d->dilation : 1;
+    if (d->dilation < 0 || o->K < 1) return SC_ERR_UNSUPPORTED;
     if (o->s != 1 && o->s != 2) return SC_ERR_UNSUPPORTED;
-    const int P = (o->K - 1) / 2;
-    o->Tp = (o->T + 2 * P - o->K) / o->s + 1;
+    o->plain = o->dil == 1 && (o->K & 1);
+    o->Tp = (o->T - 1) / o->s + 1;            // "same" padding: dil * (K - 1) zeros in total
     o->Cres = d->C_res > 0 ? d->C_res : d->C_in;
     if (d->residual < 0 || d->residual > 2) return SC_ERR_UNSUPPORTED;
     if (d->residual == SC_RES_IDENTITY && o->Cres != o->Cout) return SC_ERR_UNSUPPORTED;
     if (d->residual != SC_RES_NONE && !d->has_bn) return SC_ERR_UNSUPPORTED;
     if (!d->has_bn && d->has_relu) return SC_ERR_UNSUPPORTED;
     if (d->has_bn && d->has_bias) return SC_ERR_UNSUPPORTED;   // a bias before batch norm cancels
+    if (d->log_softmax && (d->has_bn || d->has_relu || d->residual != SC_RES_NONE)) return SC_ERR_UNSUPPORTED;
     return SC_OK;
 }
 
@@ -89,7 +98,7 @@ int check_tensor(const sc_tensor* t, int dtype, int64_t B, int64_t C, int64_t T)
 
 struct BlockIO {                 // raw pointers after validation
     const void* x; const void* xres; void* y;
-    const int* len_in; int* len_out; int* nvalid;
+    const int* len_in; int* len_out; int* nvalid; int* blk_off;
     bool x_clean, res_clean;     // inputs known to be zero in padded frames
     bool lengths_ready;          // len_out / nvalid already computed
     void* w16_keep;              // optional: where to leave the float16 copy of wp for the backward pass
@@ -100,51 +109,94 @@ struct BlockIO {                 // raw pointers after validation
 int op_dtype(const sc_block_desc* d) { return otype_of(d->io_dtype, d->has_dw && d->has_bn); }
 
 // ---- forward scratch ---------------------------------------------------------------------------
-struct FwdScratch { float2* partials; void *xr, *v, *vr, *w16; int* len_out; int* nvalid; };
+struct FwdScratch { void* partials; void* partials_r; void *xr, *w16; float* zf32; int* len_out; int* nvalid; int* blk_off; };
 
 void plan_fwd(const sc_block_desc* d, const Dims& m, Bump& ws, FwdScratch* f, const TcState* tc) {
-    const size_t parts = (size_t)m.B * tc_max_parts_per_sample(m.Tp) * m.Cout;
     f->len_out = (int*)ws.take(sizeof(int) * m.B);
     f->nvalid = (int*)ws.take(sizeof(int));
-    f->partials = (float2*)ws.take(sizeof(float2) * parts);
-    const size_t vbytes = dtype_size(vtype_of(d->io_dtype)) * m.B * m.Cout * m.Tp;
-    f->v = d->has_bn ? ws.take(vbytes) : nullptr;
-    f->vr = (d->residual == SC_RES_PROJ) ? ws.take(vbytes) : nullptr;
+    f->blk_off = (int*)ws.take(sizeof(int) * (m.B + 1));
+    f->partials = ws.take(tc_stats_bytes(m.B, m.Cout, m.Tp));
+    f->partials_r = (d->residual == SC_RES_PROJ) ? ws.take(tc_stats_bytes(m.B, m.Cout, m.Tp)) : nullptr;
+    f->zf32 = d->log_softmax ? (float*)ws.take(sizeof(float) * m.B * m.Cout * m.Tp) : nullptr;
     f->xr = (d->residual == SC_RES_PROJ) ? ws.take(esize(d->io_dtype) * m.B * m.Cres * m.Tp) : nullptr;
     f->w16 = (op_dtype(d) != d->io_dtype) ? ws.take((size_t)2 * m.Cout * m.Cin) : nullptr;
 }
 
-// v = w * u for every sample (stored in the transient type), plus masked batch statistics.
+// v = w * u for every sample (stored once, in the type it is kept in for the backward pass), plus masked
+// batch statistics.
 void pointwise_bn(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const Dims& m, int Cin, int opdt,
-                  const void* w, const void* u, void* v, const int* len_out, const int* nvalid,
-                  float* mean, float* invstd, float2* partials, float* rmean, float* rvar) {
-    const int vdt = vtype_of(d->io_dtype);
-    int parts = 1, tile_w = m.Tp;
-    bool fused = false;
-    if (ctx->gemm_mode == 0 && tc_fwd_supported(&ctx->tc, opdt, Cin, m.Cout, m.Tp)) {
-        fused = tc_gemm_fwd(&ctx->tc, L, opdt, w, u, nullptr, v, vdt, len_out, m.B, Cin, m.Cout, m.Tp,
-                            partials, &parts, &tile_w);
-    } else {
+                  const void* w, const void* u, void* v, const int* len_out, const int* nvalid, const int* blk_off,
+                  float* mean, float* invstd, void* partials, float* rmean, float* rvar) {
+    const int vdt = ntype_of(d->io_dtype);
+    StatsLayout sl;
+    if (ctx->gemm_mode == 0 && tc_fwd_supported(&ctx->tc, opdt, Cin, m.Cout, m.Tp))
+        tc_gemm_fwd(&ctx->tc, L, opdt, w, u, nullptr, v, vdt, len_out, blk_off, m.B, Cin, m.Cout, m.Tp, partials, &sl);
+    else
         gemm_fwd_simt(L, opdt, w, u, nullptr, v, vdt, len_out, m.B, Cin, m.Cout, m.Tp);
+    if (sl.kind == 2) {
+        bn_finalize_flat(L, (const float4*)partials, sl.grid, sl.tiles_m, sl.rows_per_tile, blk_off, nvalid, m.B, m.Cout,
+                         d->bn_eps, d->bn_momentum, mean, invstd, rmean, rvar);
+        return;
     }
-    if (!fused) { bn_stats(L, vdt, v, len_out, m.B, m.Cout, m.Tp, partials); parts = 1; tile_w = m.Tp; }
-    bn_finalize(L, partials, parts, tile_w, len_out, nvalid, m.B, m.Cout, d->bn_eps, d->bn_momentum, mean,
-                invstd, rmean, rvar);
+    if (sl.kind == 0) { bn_stats(L, vdt, v, len_out, m.B, m.Cout, m.Tp, (float2*)partials); sl.parts_per_b = 1; sl.tile_w = m.Tp; }
+    bn_finalize(L, (const float2*)partials, sl.parts_per_b, sl.tile_w, len_out, nvalid, m.B, m.Cout, d->bn_eps, d->bn_momentum,
+                mean, invstd, rmean, rvar);
+}
+
+// The launch context of the side stream (same status word, counters and profile), or L itself when overlap is off.
+Launch side_launch(sc_ctx* ctx, const Launch& L) {
+    Launch s = L;
+    if (ctx->overlap && ctx->side) s.stream = ctx->side;
+    return s;
+}
+// side stream waits for everything enqueued on L.stream so far
+void fork_to_side(sc_ctx* ctx, const Launch& L, cudaEvent_t ev) {
+    if (!(ctx->overlap && ctx->side)) return;
+    cudaEventRecord(ev, L.stream);
+    cudaStreamWaitEvent(ctx->side, ev, 0);
+}
+void record_side(sc_ctx* ctx, cudaEvent_t ev) { if (ctx->overlap && ctx->side) cudaEventRecord(ev, ctx->side); }
+void wait_side(sc_ctx* ctx, const Launch& L, cudaEvent_t ev) { if (ctx->overlap && ctx->side) cudaStreamWaitEvent(L.stream, ev, 0); }
+
+// Evaluation mode: fixed running statistics take the place of the batch statistics.
+struct InferStats { const float *mean, *var, *mean_r, *var_r; };
+
+// v = w * u without statistics (evaluation mode); invstd <- 1 / sqrt(var + eps)
+void pointwise_fixed(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const Dims& m, int Cin, int opdt, const void* w,
+                     const void* u, void* v, const int* len_out, const int* blk_off, const float* var, float* invstd) {
+    const int vdt = ntype_of(d->io_dtype);
+    if (ctx->gemm_mode == 0 && tc_fwd_supported(&ctx->tc, opdt, Cin, m.Cout, m.Tp))
+        tc_gemm_fwd(&ctx->tc, L, opdt, w, u, nullptr, v, vdt, len_out, blk_off, m.B, Cin, m.Cout, m.Tp, nullptr, nullptr);
+    else
+        gemm_fwd_simt(L, opdt, w, u, nullptr, v, vdt, len_out, m.B, Cin, m.Cout, m.Tp);
+    invstd_from_var(L, var, d->bn_eps, invstd, m.Cout);
 }
 
 int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const Dims& m, BlockIO io,
                    const sc_block_params* p, sc_block_saved* sv, float* rmean, float* rvar,
-                   const FwdScratch& f) {
+                   const FwdScratch& f, const InferStats* inf = nullptr) {
     const int dt = d->io_dtype;
-    if (!io.lengths_ready) lengths(L, io.len_in, m.B, m.T, m.s, io.len_out, io.nvalid);
+    if (!io.lengths_ready) lengths(L, io.len_in, m.B, m.T, m.s, io.len_out, io.nvalid, io.blk_off);
     const int odt = op_dtype(d);
+    if (d->has_bn && d->residual == SC_RES_PROJ) {
+        // the residual projection does not depend on the main branch: its contraction and statistics go to the
+        // side stream and are joined just before the apply step
+        fork_to_side(ctx, L, ctx->ev[4]);
+        const Launch Ls = side_launch(ctx, L);
+        const void* xr = io.xres;
+        if (!io.res_clean) { mask_copy(Ls, dt, f.xr, io.xres, io.len_out, m.B, m.Cres, m.Tp); xr = f.xr; }
+        if (inf) pointwise_fixed(ctx, Ls, d, m, m.Cres, dt, p->wr, xr, sv->vr, io.len_out, io.blk_off, inf->var_r, sv->invstd_r);
+        else pointwise_bn(ctx, Ls, d, m, m.Cres, dt, p->wr, xr, sv->vr, io.len_out, io.nvalid, io.blk_off, sv->mean_r,
+                          sv->invstd_r, f.partials_r, nullptr, nullptr);
+        record_side(ctx, ctx->ev[5]);
+    }
     const void* u;
     if (d->has_dw) {
-        if (ctx->gemm_mode == 0 && dw_tma_supported(&ctx->tc, dt, m.B, m.T, m.K, m.s))
+        if (ctx->gemm_mode == 0 && m.plain && dw_tma_supported(&ctx->tc, dt, m.B, m.T, m.K, m.s))
             dw_tma_fwd(&ctx->tc, L, dt, odt, io.x, p->wd, sv->u, io.len_in, io.len_out, m.B, m.Cin, m.T, m.K,
                        io.x_clean ? 1 : 0);
         else
-            dw_fwd(L, dt, odt, io.x, p->wd, sv->u, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s);
+            dw_fwd(L, dt, odt, io.x, p->wd, sv->u, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s, m.dil);
         u = sv->u;
     } else if (io.x_clean) {
         u = io.x;
@@ -152,14 +204,17 @@ int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
         mask_copy(L, dt, sv->u, io.x, io.len_in, m.B, m.Cin, m.T);
         u = sv->u;
     }
-    if (!d->has_bn) {   // linear layer: y = mask * (w u + bias)
+    if (!d->has_bn) {   // linear layer: y = mask * (w u + bias), or its log-softmax over the channels
+        // with the decoder tail the class scores stay in float32 until the log-softmax has been taken
+        void* z = d->log_softmax ? (void*)f.zf32 : io.y;
+        const int zdt = d->log_softmax ? (int)SC_F32 : dt;
         if (ctx->gemm_mode == 0 && tc_fwd_supported(&ctx->tc, dt, m.Cin, m.Cout, m.Tp)) {
-            int parts, tw;
-            tc_gemm_fwd(&ctx->tc, L, dt, p->wp, u, d->has_bias ? p->bias : nullptr, io.y, dt, io.len_out, m.B, m.Cin,
-                        m.Cout, m.Tp, nullptr, &parts, &tw);
+            tc_gemm_fwd(&ctx->tc, L, dt, p->wp, u, d->has_bias ? p->bias : nullptr, z, zdt, io.len_out, io.blk_off, m.B,
+                        m.Cin, m.Cout, m.Tp, nullptr, nullptr);
         } else {
-            gemm_fwd_simt(L, dt, p->wp, u, d->has_bias ? p->bias : nullptr, io.y, dt, io.len_out, m.B, m.Cin, m.Cout, m.Tp);
+            gemm_fwd_simt(L, dt, p->wp, u, d->has_bias ? p->bias : nullptr, z, zdt, io.len_out, m.B, m.Cin, m.Cout, m.Tp);
         }
+        if (d->log_softmax) log_softmax_fwd(L, dt, f.zf32, io.y, io.len_out, m.B, m.Cout, m.Tp);
         return SC_OK;
     }
     const void* wp_op = p->wp;
@@ -168,20 +223,17 @@ int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
         if (!(io.w16_keep && io.w16_ready)) convert_bf16_to_f16(L, p->wp, dst, (int64_t)m.Cout * m.Cin);
         wp_op = dst;
     }
-    pointwise_bn(ctx, L, d, m, m.Cin, odt, wp_op, u, f.v, io.len_out, io.nvalid, sv->mean, sv->invstd, f.partials,
-                 rmean, rvar);
+    if (inf) pointwise_fixed(ctx, L, d, m, m.Cin, odt, wp_op, u, sv->v, io.len_out, io.blk_off, inf->var, sv->invstd);
+    else pointwise_bn(ctx, L, d, m, m.Cin, odt, wp_op, u, sv->v, io.len_out, io.nvalid, io.blk_off, sv->mean, sv->invstd,
+                      f.partials, rmean, rvar);
     ApplyArgs a{};
-    a.v = f.v; a.mean = sv->mean; a.invstd = sv->invstd; a.gamma = p->gamma; a.beta = p->beta; a.vhat = sv->vhat;
+    a.v = sv->v; a.mean = inf ? inf->mean : sv->mean; a.invstd = sv->invstd; a.gamma = p->gamma; a.beta = p->beta;
     a.residual = d->residual; a.y = io.y; a.len_out = io.len_out;
     a.B = m.B; a.C = m.Cout; a.Tp = m.Tp; a.has_relu = d->has_relu; a.res_before_relu = d->res_before_relu;
     if (d->residual == SC_RES_IDENTITY) a.xres = io.xres;
     if (d->residual == SC_RES_PROJ) {
-        const void* xr = io.xres;
-        if (!io.res_clean) { mask_copy(L, dt, f.xr, io.xres, io.len_out, m.B, m.Cres, m.Tp); xr = f.xr; }
-        pointwise_bn(ctx, L, d, m, m.Cres, dt, p->wr, xr, f.vr, io.len_out, io.nvalid, sv->mean_r, sv->invstd_r,
-                     f.partials, nullptr, nullptr);
-        a.vr = f.vr; a.mean_r = sv->mean_r; a.invstd_r = sv->invstd_r; a.gamma_r = p->gamma_r; a.beta_r = p->beta_r;
-        a.vhat_r = sv->vhat_r;
+        a.vr = sv->vr; a.mean_r = inf ? inf->mean_r : sv->mean_r; a.invstd_r = sv->invstd_r; a.gamma_r = p->gamma_r; a.beta_r = p->beta_r;
+        wait_side(ctx, L, ctx->ev[5]);      // the projection branch (enqueued above on the side stream) is complete
     }
     bn_apply(L, dt, a);
     return SC_OK;
@@ -189,10 +241,10 @@ int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
 
 // ---- backward scratch --------------------------------------------------------------------------
 struct BwdScratch {
-    int* len_out; int* nvalid;
+    int* len_out; int* nvalid; int* blk_off;
     float4 *partials, *coef, *coef_r;
     float *amax_part, *gmax;
-    void *gv, *gvr, *gres, *gu, *gxr, *xr, *w16;
+    void *gv, *gvr, *gres, *gu, *gxr, *xr, *w16, *dz;
     void *gv16, *gvr16, *x16, *xr16;     // half copies for the weight gradients of bf16 layers (see block_bwd_impl)
     float* wpart; size_t wpart_bytes;
 };
@@ -202,6 +254,7 @@ void plan_bwd(const sc_block_desc* d, const Dims& m, Bump& ws, BwdScratch* s, co
     const size_t act_out = e * m.B * m.Cout * m.Tp, act_in = e * m.B * m.Cin * m.Tp;
     s->len_out = (int*)ws.take(sizeof(int) * m.B);
     s->nvalid = (int*)ws.take(sizeof(int));
+    s->blk_off = (int*)ws.take(sizeof(int) * (m.B + 1));
     s->partials = (float4*)ws.take(sizeof(float4) * m.B * m.Cout * bn_bwd_max_slots(m.Tp));
     s->coef = (float4*)ws.take(sizeof(float4) * m.Cout);
     s->coef_r = (float4*)ws.take(sizeof(float4) * m.Cout);
@@ -209,6 +262,7 @@ void plan_bwd(const sc_block_desc* d, const Dims& m, Bump& ws, BwdScratch* s, co
     s->gmax = (float*)ws.take(sizeof(float));
     s->w16 = (op_dtype(d) != d->io_dtype) ? ws.take((size_t)2 * m.Cout * m.Cin) : nullptr;
     s->gv = ws.take(act_out);
+    s->dz = d->log_softmax ? ws.take(act_out) : nullptr;
     s->gvr = d->residual == SC_RES_PROJ ? ws.take(act_out) : nullptr;
     s->gres = d->residual == SC_RES_IDENTITY ? ws.take(act_out) : nullptr;
     s->gu = ws.take(act_in);
@@ -235,9 +289,9 @@ void pointwise_wgrad(sc_ctx* ctx, const Launch& L, int dt, const void* gv, const
         gemm_wgrad_simt(L, dt, gv, u, dw, part, acc, B, Cin, Cout, Tp, gmax);
 }
 void pointwise_dgrad(sc_ctx* ctx, const Launch& L, int dt, const void* w, const void* gv, void* gu, int B,
-                     int Cin, int Cout, int Tp, const int* len_out) {
+                     int Cin, int Cout, int Tp, const int* len_out, const int* blk_off) {
     if (ctx->gemm_mode == 0 && tc_dgrad_supported(&ctx->tc, dt, Cin, Cout, Tp))
-        tc_gemm_dgrad(&ctx->tc, L, dt, w, gv, gu, B, Cin, Cout, Tp, len_out);
+        tc_gemm_dgrad(&ctx->tc, L, dt, w, gv, gu, B, Cin, Cout, Tp, len_out, blk_off);
     else
         gemm_dgrad_simt(L, dt, w, gv, gu, B, Cin, Cout, Tp);
 }
@@ -245,9 +299,10 @@ void pointwise_dgrad(sc_ctx* ctx, const Launch& L, int dt, const void* w, const 
 struct BwdIO {
     const void *dy, *x, *xres, *y;
     void *dx, *dx_res; const void* dx_add;
-    const int* len_in; const int* len_out; const int* nvalid;
+    const int* len_in; const int* len_out; const int* nvalid; const int* blk_off;
     bool x_clean, res_clean;
     const void* w16_kept;        // float16 copy of wp left by the forward pass (optional)
+    cudaEvent_t done;            // recorded on the side stream after this layer's last side-stream kernel
 };
 
 int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const Dims& m, BwdIO io,
@@ -267,12 +322,17 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
                           tc_wgrad_supported(&ctx->tc, SC_F16, m.Cres, m.Cout, m.Tp);
     float* gmax = (dt != SC_F32 && d->has_bn && (d->has_dw || half_gv || half_gvr)) ? s.gmax : nullptr;
     if (gmax) cudaMemsetAsync(gmax, 0, sizeof(float), L.stream);
+    const void* dy = io.dy;
+    if (d->log_softmax) {      // upstream gradient is w.r.t. the log-probabilities: back through the log-softmax first
+        log_softmax_bwd(L, dt, s.dz, io.dy, io.y, io.len_out, m.B, m.Cout, m.Tp);
+        dy = s.dz;
+    }
     BnBwdArgs a{};
     a.amax_part = s.amax_part; a.gmax = gmax; a.gv_dtype = odt;
     a.gv_scaled = (gmax && d->has_dw) ? 1 : 0;
     a.gv16 = half_gv ? s.gv16 : nullptr; a.gvr16 = half_gvr ? s.gvr16 : nullptr;
-    a.g = io.dy; a.y = io.y; a.vhat = sv->vhat; a.vhat_r = sv->vhat_r;
-    a.invstd = sv->invstd; a.invstd_r = sv->invstd_r; a.gamma = p->gamma; a.beta = p->beta;
+    a.g = dy; a.y = io.y; a.v = sv->v; a.vr = sv->vr;
+    a.mean = sv->mean; a.mean_r = sv->mean_r; a.invstd = sv->invstd; a.invstd_r = sv->invstd_r; a.gamma = p->gamma; a.beta = p->beta;
     a.len_out = io.len_out; a.nvalid = io.nvalid;
     a.B = m.B; a.C = m.Cout; a.Tp = m.Tp; a.has_bn = d->has_bn; a.has_relu = d->has_relu;
     a.res_before_relu = d->res_before_relu; a.residual = d->residual;
@@ -285,60 +345,69 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
                     d->has_bias ? g->dbias : nullptr, acc);
     bn_bwd_apply(L, dt, a);
 
+    // The weight gradients are off the critical path (nothing later in the backward pass reads them): they run on
+    // the side stream while this stream goes on with the input gradients.
+    const Launch Ls = side_launch(ctx, L);
+    fork_to_side(ctx, L, ctx->ev[0]);                   // gv, gvr and their half copies are complete
     const void* u = d->has_dw ? sv->u : (io.x_clean ? io.x : sv->u);
     if (half_gv) {
-        mask_convert_f16(L, s.x16, io.x, io.len_in, m.B, m.Cin, m.T);
-        pointwise_wgrad(ctx, L, SC_F16, s.gv16, s.x16, g->dwp, s.wpart, acc, m.B, m.Cin, m.Cout, m.Tp, io.len_out, gmax);
+        mask_convert_f16(Ls, s.x16, io.x, io.len_in, m.B, m.Cin, m.T);
+        pointwise_wgrad(ctx, Ls, SC_F16, s.gv16, s.x16, g->dwp, s.wpart, acc, m.B, m.Cin, m.Cout, m.Tp, io.len_out, gmax);
     } else {
-        pointwise_wgrad(ctx, L, odt, s.gv, u, g->dwp, s.wpart, acc, m.B, m.Cin, m.Cout, m.Tp, io.len_out,
+        pointwise_wgrad(ctx, Ls, odt, s.gv, u, g->dwp, s.wpart, acc, m.B, m.Cin, m.Cout, m.Tp, io.len_out,
                         a.gv_scaled ? gmax : nullptr);
     }
+    if (d->residual == SC_RES_PROJ) {
+        if (half_gvr) {
+            mask_convert_f16(Ls, s.xr16, io.xres, io.len_out, m.B, m.Cres, m.Tp);
+            pointwise_wgrad(ctx, Ls, SC_F16, s.gvr16, s.xr16, g->dwr, s.wpart, acc, m.B, m.Cres, m.Cout, m.Tp, io.len_out, gmax);
+        } else {
+            const void* xr = io.xres;
+            if (!io.res_clean) { mask_copy(Ls, dt, s.xr, io.xres, io.len_out, m.B, m.Cres, m.Tp); xr = s.xr; }
+            pointwise_wgrad(ctx, Ls, dt, s.gvr, xr, g->dwr, s.wpart, acc, m.B, m.Cres, m.Cout, m.Tp, io.len_out, nullptr);
+        }
+    }
+
     const void* wp_op = p->wp;
     if (odt != dt) {
         if (io.w16_kept) wp_op = io.w16_kept;
         else { convert_bf16_to_f16(L, p->wp, s.w16, (int64_t)m.Cout * m.Cin); wp_op = s.w16; }
     }
-
     const void* extra = nullptr;    // residual-path gradient to fold into dx
     if (d->residual == SC_RES_PROJ) {
-        const void* xr = io.xres;
-        if (!io.res_clean) { mask_copy(L, dt, s.xr, io.xres, io.len_out, m.B, m.Cres, m.Tp); xr = s.xr; }
-        if (half_gvr) {
-            mask_convert_f16(L, s.xr16, io.xres, io.len_out, m.B, m.Cres, m.Tp);
-            pointwise_wgrad(ctx, L, SC_F16, s.gvr16, s.xr16, g->dwr, s.wpart, acc, m.B, m.Cres, m.Cout, m.Tp, io.len_out, gmax);
-        } else {
-            pointwise_wgrad(ctx, L, dt, s.gvr, xr, g->dwr, s.wpart, acc, m.B, m.Cres, m.Cout, m.Tp, io.len_out, nullptr);
-        }
         void* tgt = io.dx_res ? io.dx_res : s.gxr;
-        if (io.dx_res || io.dx) pointwise_dgrad(ctx, L, dt, p->wr, s.gvr, tgt, m.B, m.Cres, m.Cout, m.Tp, io.len_out);
+        if (io.dx_res || io.dx) pointwise_dgrad(ctx, L, dt, p->wr, s.gvr, tgt, m.B, m.Cres, m.Cout, m.Tp, io.len_out, io.blk_off);
         if (!io.dx_res) extra = s.gxr;
     } else if (d->residual == SC_RES_IDENTITY && !io.dx_res) {
         extra = s.gres;
     }
 
     if (d->has_dw) {
-        pointwise_dgrad(ctx, L, odt, wp_op, s.gv, s.gu, m.B, m.Cin, m.Cout, m.Tp, io.len_out);
-        if (ctx->gemm_mode == 0 && dw_wgrad_tc_supported(&ctx->tc, dt, m.B, m.T, m.K, m.s))
-            dw_wgrad_tc(&ctx->tc, L, dt, odt, s.gu, io.x, g->dwd, s.wpart, acc, gmax, io.len_in, io.len_out, m.B, m.Cin,
+        pointwise_dgrad(ctx, L, odt, wp_op, s.gv, s.gu, m.B, m.Cin, m.Cout, m.Tp, io.len_out, io.blk_off);
+        fork_to_side(ctx, L, ctx->ev[1]);               // gu is complete
+        if (ctx->gemm_mode == 0 && m.plain && dw_wgrad_tc_supported(&ctx->tc, dt, m.B, m.T, m.K, m.s))
+            dw_wgrad_tc(&ctx->tc, Ls, dt, odt, s.gu, io.x, g->dwd, s.wpart, acc, gmax, io.len_in, io.len_out, m.B, m.Cin,
                         m.T, m.K, io.x_clean ? 1 : 0);
         else
-            dw_wgrad(L, dt, odt, s.gu, io.x, g->dwd, s.wpart, acc, gmax, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s);
+            dw_wgrad(Ls, dt, odt, s.gu, io.x, g->dwd, s.wpart, acc, gmax, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s, m.dil);
         if (io.dx) {
-            if (ctx->gemm_mode == 0 && dw_tma_supported(&ctx->tc, dt, m.B, m.T, m.K, m.s))
+            if (ctx->gemm_mode == 0 && m.plain && dw_tma_supported(&ctx->tc, dt, m.B, m.T, m.K, m.s))
                 dw_tma_dgrad(&ctx->tc, L, dt, odt, s.gu, p->wd, io.dx, io.dx_add, extra, gmax, io.len_in, io.len_out, m.B,
                              m.Cin, m.T, m.K);
             else
                 dw_dgrad(L, dt, odt, s.gu, p->wd, io.dx, io.dx_add, extra, gmax, io.len_in, io.len_out, m.B, m.Cin, m.T,
-                         m.Tp, m.K, m.s);
+                         m.Tp, m.K, m.s, m.dil);
         }
     } else if (io.dx) {
         if (!io.dx_add && !extra) {
-            pointwise_dgrad(ctx, L, dt, p->wp, s.gv, io.dx, m.B, m.Cin, m.Cout, m.Tp, io.len_out);
+            pointwise_dgrad(ctx, L, dt, p->wp, s.gv, io.dx, m.B, m.Cin, m.Cout, m.Tp, io.len_out, io.blk_off);
         } else {
-            pointwise_dgrad(ctx, L, dt, p->wp, s.gv, s.gu, m.B, m.Cin, m.Cout, m.Tp, io.len_out);
+            pointwise_dgrad(ctx, L, dt, p->wp, s.gv, s.gu, m.B, m.Cin, m.Cout, m.Tp, io.len_out, io.blk_off);
             ew_add_masked(L, dt, io.dx, s.gu, io.dx_add, extra, io.len_in, m.B, m.Cin, m.T);
         }
     }
+    // the caller joins: it waits for io.done on its stream before it reuses this scratch or returns
+    if (io.done) record_side(ctx, io.done);
     return SC_OK;
 }
 
@@ -353,8 +422,8 @@ int check_params(const sc_block_desc* d, const sc_block_params* p) {
 int check_saved(const sc_block_desc* d, const sc_block_saved* s, bool x_clean) {
     if (!s) return SC_ERR_NULL;
     if ((d->has_dw || !x_clean) && !s->u) return SC_ERR_NULL;
-    if (d->has_bn && (!s->vhat || !s->mean || !s->invstd)) return SC_ERR_NULL;
-    if (d->residual == SC_RES_PROJ && (!s->vhat_r || !s->mean_r || !s->invstd_r)) return SC_ERR_NULL;
+    if (d->has_bn && (!s->v || !s->mean || !s->invstd)) return SC_ERR_NULL;
+    if (d->residual == SC_RES_PROJ && (!s->vr || !s->mean_r || !s->invstd_r)) return SC_ERR_NULL;
     return SC_OK;
 }
 int check_grads(const sc_block_desc* d, const sc_block_grads* g) {
@@ -394,6 +463,9 @@ int sepconv_ctx_create(sc_ctx** out, int device) {
     cudaMemset(c->status_dev, 0, 64);
     int r = tc_init(&c->tc, device, c->sm_count);
     if (r != SC_OK) { cudaFree(c->status_dev); delete c; return r; }
+    bool ok = cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; i < 6 && ok; ++i) ok = cudaEventCreateWithFlags(&c->ev[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { sepconv_ctx_destroy(c); return SC_ERR_CUDA; }
     *out = c;
     return SC_OK;
 }
@@ -401,6 +473,8 @@ int sepconv_ctx_create(sc_ctx** out, int device) {
 void sepconv_ctx_destroy(sc_ctx* ctx) {
     if (!ctx) return;
     for (cudaEvent_t e : ctx->prof.events) cudaEventDestroy(e);
+    for (cudaEvent_t e : ctx->ev) if (e) cudaEventDestroy(e);
+    if (ctx->side) cudaStreamDestroy(ctx->side);
     cudaFree(ctx->status_dev);
     delete ctx;
 }
@@ -432,6 +506,26 @@ const char* sepconv_strerror(int s) {
         case SC_ERR_RANGE: return "an intermediate value left the float16 range and was clamped";
         default: return "unknown status";
     }
+}
+
+int sepconv_selftest_bounded_wait(sc_ctx* ctx, void* cuda_stream) {
+    if (!ctx) return SC_ERR_NULL;
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode};
+    selftest_bounded_wait(L);
+    return finish(ctx);
+}
+
+int sepconv_set_tile_shape(sc_ctx* ctx, int shape) {
+    if (!ctx) return SC_ERR_NULL;
+    if (shape < 0 || shape > 2) return SC_ERR_UNSUPPORTED;
+    ctx->tc.flat_shape = shape;
+    return SC_OK;
+}
+
+int sepconv_set_overlap(sc_ctx* ctx, int on) {
+    if (!ctx) return SC_ERR_NULL;
+    ctx->overlap = on ? 1 : 0;
+    return SC_OK;
 }
 
 int sepconv_set_gemm_mode(sc_ctx* ctx, int mode) {
@@ -507,11 +601,66 @@ int sepconv_fwd(sc_ctx* ctx, const sc_block_desc* desc, const sc_tensor* x, cons
     Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode};
     BlockIO io{};
     io.x = x->ptr; io.xres = desc->residual != SC_RES_NONE ? (x_res ? x_res->ptr : x->ptr) : nullptr;
-    io.y = y->ptr; io.len_in = lengths_dev; io.len_out = f.len_out; io.nvalid = f.nvalid;
+    io.y = y->ptr; io.len_in = lengths_dev; io.len_out = f.len_out; io.nvalid = f.nvalid; io.blk_off = f.blk_off;
     io.x_clean = false; io.res_clean = false; io.lengths_ready = false;
     SC_TRY(block_fwd_impl(ctx, L, desc, m, io, params, saved, running_mean, running_var, f));
     if (out_lengths_dev)
         cudaMemcpyAsync(out_lengths_dev, f.len_out, sizeof(int) * m.B, cudaMemcpyDeviceToDevice, L.stream);
+    return finish(ctx);
+}
+
+namespace {
+// scratch of the evaluation-mode forward: the training forward's scratch plus the tensors that call would save
+struct InferScratch { FwdScratch f; sc_block_saved sv; };
+void plan_infer(const sc_block_desc* d, const Dims& m, Bump& ws, InferScratch* q, const TcState* tc) {
+    plan_fwd(d, m, ws, &q->f, tc);
+    memset(&q->sv, 0, sizeof(q->sv));
+    const size_t e = esize(d->io_dtype), en = dtype_size(ntype_of(d->io_dtype));
+    q->sv.u = ws.take(e * m.B * m.Cin * m.Tp);
+    if (d->has_bn) { q->sv.v = ws.take(en * m.B * m.Cout * m.Tp); q->sv.invstd = (float*)ws.take(4 * m.Cout); }
+    if (d->residual == SC_RES_PROJ) { q->sv.vr = ws.take(en * m.B * m.Cout * m.Tp); q->sv.invstd_r = (float*)ws.take(4 * m.Cout); }
+}
+}  // namespace
+
+int sepconv_infer_workspace_bytes(const sc_block_desc* desc, size_t* bytes) {
+    if (!bytes) return SC_ERR_NULL;
+    Dims m;
+    SC_TRY(desc_dims(desc, &m));
+    Bump b(nullptr, 0); InferScratch q; plan_infer(desc, m, b, &q, nullptr);
+    *bytes = b.off + 256;
+    return SC_OK;
+}
+
+int sepconv_infer(sc_ctx* ctx, const sc_block_desc* desc, const sc_tensor* x, const sc_tensor* x_res,
+                  const int32_t* lengths_dev, const sc_block_params* params, const float* running_mean,
+                  const float* running_var, const float* running_mean_r, const float* running_var_r, sc_tensor* y,
+                  int32_t* out_lengths_dev, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!ctx || !lengths_dev) return SC_ERR_NULL;
+    Dims m;
+    SC_TRY(desc_dims(desc, &m));
+    const int dt = desc->io_dtype;
+    SC_TRY(check_tensor(x, dt, m.B, m.Cin, m.T));
+    SC_TRY(check_tensor(y, dt, m.B, m.Cout, m.Tp));
+    if (desc->residual != SC_RES_NONE) {
+        if (x_res) SC_TRY(check_tensor(x_res, dt, m.B, m.Cres, m.Tp));
+        else if (m.s != 1 || m.Cres != m.Cin) return SC_ERR_UNSUPPORTED;
+    }
+    SC_TRY(check_params(desc, params));
+    if (desc->has_bn && (!running_mean || !running_var)) return SC_ERR_NULL;
+    if (desc->residual == SC_RES_PROJ && (!running_mean_r || !running_var_r)) return SC_ERR_NULL;
+    if (!workspace) return SC_ERR_WORKSPACE;
+    Bump ws(workspace, workspace_bytes);
+    InferScratch q;
+    plan_infer(desc, m, ws, &q, &ctx->tc);
+    if (!ws.ok()) return SC_ERR_WORKSPACE;
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode};
+    BlockIO io{};
+    io.x = x->ptr; io.xres = desc->residual != SC_RES_NONE ? (x_res ? x_res->ptr : x->ptr) : nullptr;
+    io.y = y->ptr; io.len_in = lengths_dev; io.len_out = q.f.len_out; io.nvalid = q.f.nvalid; io.blk_off = q.f.blk_off;
+    InferStats inf{running_mean, running_var, running_mean_r, running_var_r};
+    SC_TRY(block_fwd_impl(ctx, L, desc, m, io, params, &q.sv, nullptr, nullptr, q.f, &inf));
+    if (out_lengths_dev)
+        cudaMemcpyAsync(out_lengths_dev, q.f.len_out, sizeof(int) * m.B, cudaMemcpyDeviceToDevice, L.stream);
     return finish(ctx);
 }
 
@@ -534,6 +683,8 @@ int sepconv_bwd(sc_ctx* ctx, const sc_block_desc* desc, const sc_tensor* dy, con
         else if (m.s != 1 || m.Cres != m.Cin) return SC_ERR_UNSUPPORTED;
         if (dx_res) SC_TRY(check_tensor(dx_res, dt, m.B, m.Cres, m.Tp));
         else if (m.s != 1 || m.Cres != m.Cin) return SC_ERR_UNSUPPORTED;
+        // folding the residual path's gradient into dx is only meaningful when the residual source is x itself
+        else if (x_res && x_res->ptr != x->ptr) return SC_ERR_UNSUPPORTED;
     }
     SC_TRY(check_params(desc, params));
     SC_TRY(check_saved(desc, saved, false));
@@ -544,15 +695,17 @@ int sepconv_bwd(sc_ctx* ctx, const sc_block_desc* desc, const sc_tensor* dy, con
     plan_bwd(desc, m, ws, &s, &ctx->tc);
     if (!ws.ok()) return SC_ERR_WORKSPACE;
     Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode};
-    lengths(L, lengths_dev, m.B, m.T, m.s, s.len_out, s.nvalid);
+    lengths(L, lengths_dev, m.B, m.T, m.s, s.len_out, s.nvalid, s.blk_off);
     BwdIO io{};
     io.dy = dy->ptr; io.x = x->ptr; io.y = y->ptr;
     io.xres = desc->residual != SC_RES_NONE ? (x_res ? x_res->ptr : x->ptr) : nullptr;
     io.dx = dx->ptr; io.dx_res = (desc->residual != SC_RES_NONE && dx_res) ? dx_res->ptr : nullptr;
     io.dx_add = dx_add ? dx_add->ptr : nullptr;
-    io.len_in = lengths_dev; io.len_out = s.len_out; io.nvalid = s.nvalid;
+    io.len_in = lengths_dev; io.len_out = s.len_out; io.nvalid = s.nvalid; io.blk_off = s.blk_off;
     io.x_clean = false; io.res_clean = false;
+    io.done = ctx->ev[2];
     SC_TRY(block_bwd_impl(ctx, L, desc, m, io, params, saved, grads, accumulate, s));
+    wait_side(ctx, L, ctx->ev[2]);
     return finish(ctx);
 }
 
@@ -560,7 +713,7 @@ int sepconv_bwd(sc_ctx* ctx, const sc_block_desc* desc, const sc_tensor* dy, con
 namespace {
 struct LayerPlan {
     sc_block_desc d; Dims m;
-    sc_block_saved sv; void* y; int* len_out; int* nvalid; void* w16;
+    sc_block_saved sv; void* y; int* len_out; int* nvalid; int* blk_off; void* w16;
     bool own_lengths;
 };
 struct EncPlan {
@@ -568,6 +721,7 @@ struct EncPlan {
     void* gbuf[2]; void* pending;
     size_t bytes;
     size_t scratch_mark;           // offset where the shared per-layer scratch starts
+    size_t scratch_size;           // its size; a second region of the same size follows (backward layers alternate)
 };
 
 int plan_encoder(const sc_encoder_desc* e, void* base, size_t cap, EncPlan* P, const TcState* tc) {
@@ -576,6 +730,15 @@ int plan_encoder(const sc_encoder_desc* e, void* base, size_t cap, EncPlan* P, c
     P->L.resize(e->n_layers);
     int B = e->layers[0].B, T = e->layers[0].T_in, C = e->layers[0].C_in;
     size_t max_act = 0, max_res = 0;
+    // One pending residual-gradient buffer serves the whole backward pass, so the spans [source, layer]
+    // of the block-level residuals must not overlap (which also rules out two layers sharing a source).
+    int span_end = -1;
+    for (int i = 0; i < e->n_layers; ++i) {
+        if (e->layers[i].residual == SC_RES_NONE || !e->res_from || e->res_from[i] < 0 || e->res_from[i] == i) continue;
+        if (e->res_from[i] > i) return SC_ERR_UNSUPPORTED;
+        if (e->res_from[i] <= span_end) return SC_ERR_UNSUPPORTED;
+        span_end = i;
+    }
     for (int i = 0; i < e->n_layers; ++i) {
         LayerPlan& lp = P->L[i];
         lp.d = e->layers[i];
@@ -597,17 +760,19 @@ int plan_encoder(const sc_encoder_desc* e, void* base, size_t cap, EncPlan* P, c
             max_res = std::max(max_res, es * m.B * m.Cres * m.Tp);
         }
         lp.own_lengths = (i == 0) || (m.s != 1);
-        if (lp.own_lengths) { lp.len_out = (int*)ws.take(sizeof(int) * B); lp.nvalid = (int*)ws.take(sizeof(int)); }
-        else { lp.len_out = P->L[i - 1].len_out; lp.nvalid = P->L[i - 1].nvalid; }
+        if (lp.own_lengths) {
+            lp.len_out = (int*)ws.take(sizeof(int) * B); lp.nvalid = (int*)ws.take(sizeof(int));
+            lp.blk_off = (int*)ws.take(sizeof(int) * (B + 1));
+        } else { lp.len_out = P->L[i - 1].len_out; lp.nvalid = P->L[i - 1].nvalid; lp.blk_off = P->L[i - 1].blk_off; }
         memset(&lp.sv, 0, sizeof(lp.sv));
         if (lp.d.has_dw) lp.sv.u = ws.take(es * B * m.Cin * m.Tp);
         else if (i == 0) lp.sv.u = ws.take(es * B * m.Cin * m.Tp);
         if (lp.d.has_bn) {
-            lp.sv.vhat = ws.take(dtype_size(ntype_of(lp.d.io_dtype)) * B * m.Cout * m.Tp);
+            lp.sv.v = ws.take(dtype_size(ntype_of(lp.d.io_dtype)) * B * m.Cout * m.Tp);
             lp.sv.mean = (float*)ws.take(4 * m.Cout); lp.sv.invstd = (float*)ws.take(4 * m.Cout);
         }
         if (lp.d.residual == SC_RES_PROJ) {
-            lp.sv.vhat_r = ws.take(dtype_size(ntype_of(lp.d.io_dtype)) * B * m.Cout * m.Tp);
+            lp.sv.vr = ws.take(dtype_size(ntype_of(lp.d.io_dtype)) * B * m.Cout * m.Tp);
             lp.sv.mean_r = (float*)ws.take(4 * m.Cout); lp.sv.invstd_r = (float*)ws.take(4 * m.Cout);
         }
         lp.y = (i + 1 < e->n_layers) ? ws.take(es * B * m.Cout * m.Tp) : nullptr;
@@ -623,7 +788,11 @@ int plan_encoder(const sc_encoder_desc* e, void* base, size_t cap, EncPlan* P, c
         Bump b(base, cap); b.off = mark; FwdScratch f; plan_fwd(&P->L[i].d, P->L[i].m, b, &f, tc); hi = std::max(hi, b.off);
         Bump c(base, cap); c.off = mark; BwdScratch s; plan_bwd(&P->L[i].d, P->L[i].m, c, &s, tc); hi = std::max(hi, c.off);
     }
-    ws.off = hi;
+    // two scratch regions: backward layer i works in region i & 1, so that the weight-gradient kernels of layer i
+    // (side stream) may still read their operands while layer i - 1 already writes its own
+    hi = (hi + 255) & ~(size_t)255;
+    ws.off = hi + (hi - mark);
+    P->scratch_size = hi - mark;
     P->gbuf[0] = ws.take(max_act); P->gbuf[1] = ws.take(max_act);
     P->pending = max_res ? ws.take(max_res) : nullptr;
     P->bytes = ws.off + 256;
@@ -654,6 +823,54 @@ int encoder_workspace_bytes(const sc_encoder_desc* desc, size_t* bytes) {
     SC_TRY(plan_encoder(desc, nullptr, 0, &P, nullptr));
     *bytes = P.bytes;
     return SC_OK;
+}
+
+int encoder_infer_workspace_bytes(const sc_encoder_desc* desc, size_t* bytes) {
+    return encoder_workspace_bytes(desc, bytes);      // the same plan: per-layer buffers double as scratch
+}
+
+int encoder_infer(sc_ctx* ctx, const sc_encoder_desc* e, const sc_tensor* x, const int32_t* lengths_dev,
+                  const void* params_blob, const int64_t* param_offsets, const void* running_blob,
+                  const int64_t* running_offsets, sc_tensor* out, int32_t* out_lengths_dev, void* workspace,
+                  size_t workspace_bytes, void* cuda_stream) {
+    if (!ctx || !lengths_dev || !params_blob || !param_offsets || !running_blob || !running_offsets) return SC_ERR_NULL;
+    if (!workspace) return SC_ERR_WORKSPACE;
+    EncPlan P;
+    SC_TRY(plan_encoder(e, workspace, workspace_bytes, &P, &ctx->tc));
+    const int n = e->n_layers;
+    const Dims& m0 = P.L[0].m; const Dims& ml = P.L[n - 1].m;
+    const int dt = P.L[0].d.io_dtype;
+    SC_TRY(check_tensor(x, dt, m0.B, m0.Cin, m0.T));
+    SC_TRY(check_tensor(out, dt, ml.B, ml.Cout, ml.Tp));
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode};
+    auto input_of = [&](int i) -> const void* { return i == 0 ? x->ptr : P.L[i - 1].y; };
+    auto res_src = [&](int i) -> int { return (e->res_from && e->res_from[i] >= 0) ? e->res_from[i] : i; };
+    auto stat = [&](int i, int j) -> const float* {
+        const int64_t o = running_offsets[4 * i + j];
+        return o < 0 ? nullptr : (const float*)((const char*)running_blob + o);
+    };
+    for (int i = 0; i < n; ++i) {
+        LayerPlan& lp = P.L[i];
+        sc_block_params prm = layer_params(params_blob, param_offsets + 8 * i);
+        SC_TRY(check_params(&lp.d, &prm));
+        InferStats inf{stat(i, 0), stat(i, 1), stat(i, 2), stat(i, 3)};
+        if (lp.d.has_bn && (!inf.mean || !inf.var)) return SC_ERR_NULL;
+        if (lp.d.residual == SC_RES_PROJ && (!inf.mean_r || !inf.var_r)) return SC_ERR_NULL;
+        Bump b(workspace, workspace_bytes); b.off = P.scratch_mark;
+        FwdScratch f; plan_fwd(&lp.d, lp.m, b, &f, &ctx->tc);
+        BlockIO io{};
+        io.x = input_of(i);
+        io.xres = lp.d.residual != SC_RES_NONE ? input_of(res_src(i)) : nullptr;
+        io.y = (i + 1 < n) ? lp.y : out->ptr;
+        io.len_in = i == 0 ? lengths_dev : P.L[i - 1].len_out; io.len_out = lp.len_out; io.nvalid = lp.nvalid; io.blk_off = lp.blk_off;
+        io.x_clean = i > 0; io.res_clean = lp.d.residual != SC_RES_NONE && res_src(i) > 0;
+        io.lengths_ready = !lp.own_lengths;
+        io.w16_keep = lp.w16; io.w16_ready = false;
+        SC_TRY(block_fwd_impl(ctx, L, &lp.d, lp.m, io, &prm, &lp.sv, nullptr, nullptr, f, &inf));
+    }
+    if (out_lengths_dev)
+        cudaMemcpyAsync(out_lengths_dev, P.L[n - 1].len_out, sizeof(int) * m0.B, cudaMemcpyDeviceToDevice, L.stream);
+    return finish(ctx);
 }
 
 int encoder_fwd_bwd(sc_ctx* ctx, const sc_encoder_desc* e, const sc_tensor* x, const int32_t* lengths_dev,
@@ -706,7 +923,7 @@ int encoder_fwd_bwd(sc_ctx* ctx, const sc_encoder_desc* e, const sc_tensor* x, c
         io.x = input_of(i);
         io.xres = lp.d.residual != SC_RES_NONE ? input_of(res_src(i)) : nullptr;
         io.y = (i + 1 < n) ? lp.y : logits->ptr;
-        io.len_in = len_in_of(i); io.len_out = lp.len_out; io.nvalid = lp.nvalid;
+        io.len_in = len_in_of(i); io.len_out = lp.len_out; io.nvalid = lp.nvalid; io.blk_off = lp.blk_off;
         io.x_clean = i > 0; io.res_clean = lp.d.residual != SC_RES_NONE && res_src(i) > 0;
         io.lengths_ready = !lp.own_lengths;
         io.w16_keep = lp.w16; io.w16_ready = true;
@@ -718,23 +935,28 @@ int encoder_fwd_bwd(sc_ctx* ctx, const sc_encoder_desc* e, const sc_tensor* x, c
     // backward
     const void* g = dlogits->ptr;
     std::vector<char> has_pending(n, 0);
+    bool side_busy[2] = {false, false};
     for (int i = n - 1; i >= 0; --i) {
         LayerPlan& lp = P.L[i];
-        Bump b(workspace, workspace_bytes); b.off = mark;
+        // this layer reuses the scratch region of layer i + 2: that layer's side-stream kernels must be done
+        if (side_busy[i & 1]) wait_side(ctx, L, ctx->ev[2 + (i & 1)]);
+        Bump b(workspace, workspace_bytes); b.off = mark + (size_t)(i & 1) * P.scratch_size;
         BwdScratch s; plan_bwd(&lp.d, lp.m, b, &s, &ctx->tc);
         BwdIO io{};
+        io.done = ctx->ev[2 + (i & 1)]; side_busy[i & 1] = true;
         io.dy = g; io.x = input_of(i); io.y = (i + 1 < n) ? lp.y : logits->ptr;
         io.xres = lp.d.residual != SC_RES_NONE ? input_of(res_src(i)) : nullptr;
         io.dx = (i == 0) ? (dx ? dx->ptr : nullptr) : P.gbuf[i & 1];
         io.dx_res = nullptr;
         if (lp.d.residual != SC_RES_NONE && res_src(i) != i) { io.dx_res = P.pending; has_pending[res_src(i)] = 1; }
         io.dx_add = has_pending[i] ? P.pending : nullptr;
-        io.len_in = len_in_of(i); io.len_out = lp.len_out; io.nvalid = lp.nvalid;
+        io.len_in = len_in_of(i); io.len_out = lp.len_out; io.nvalid = lp.nvalid; io.blk_off = lp.blk_off;
         io.x_clean = i > 0; io.res_clean = lp.d.residual != SC_RES_NONE && res_src(i) > 0;
         io.w16_kept = lp.w16;
         SC_TRY(block_bwd_impl(ctx, L, &lp.d, lp.m, io, &prm[i], &lp.sv, &grd[i], accumulate, s));
         g = io.dx;
     }
+    for (int q = 0; q < 2; ++q) if (side_busy[q]) wait_side(ctx, L, ctx->ev[2 + q]);     // join before returning
     return finish(ctx);
 }
 

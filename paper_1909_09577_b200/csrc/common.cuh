@@ -52,6 +52,11 @@ template <> __device__ __forceinline__ float round_io<float>(float v) { return v
 template <> __device__ __forceinline__ float round_io<__half>(float v) { return __half2float(__float2half_rn(v)); }
 template <> __device__ __forceinline__ float round_io<__nv_bfloat16>(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 
+// vhat = (v - mean) * invstd in exactly these two float operations wherever it is needed (forward apply,
+// backward reduce and apply): the normalised value is never stored, and the ReLU decision derived from it
+// must be the same bit on every path.
+__device__ __forceinline__ float bn_norm(float v, float mu, float is) { return __fmul_rn(__fsub_rn(v, mu), is); }
+
 // Rounds the first n of 8 consecutive values to the storage type with error diffusion: the rounding
 // residual of one element is added to the next before it is rounded, so the residuals of a vector do
 // not add up.  Plain rounding is biased whenever the values sit on a lattice that the storage grid
@@ -96,6 +101,18 @@ template <> __device__ __forceinline__ void ld8<__half>(const __half* p, float (
 }
 template <> __device__ __forceinline__ void ld8<__nv_bfloat16>(const __nv_bfloat16* p, float (&f)[8]) {
     uint4 r = *reinterpret_cast<const uint4*>(p);
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&r);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { float2 q = __bfloat1622float2(h[i]); f[2 * i] = q.x; f[2 * i + 1] = q.y; }
+}
+// the same conversion from a 16-byte vector that is already in registers (16-bit types)
+template <typename T> __device__ __forceinline__ void cvt8(const uint4& r, float (&f)[8]);
+template <> __device__ __forceinline__ void cvt8<__half>(const uint4& r, float (&f)[8]) {
+    const __half2* h = reinterpret_cast<const __half2*>(&r);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { float2 q = __half22float2(h[i]); f[2 * i] = q.x; f[2 * i + 1] = q.y; }
+}
+template <> __device__ __forceinline__ void cvt8<__nv_bfloat16>(const uint4& r, float (&f)[8]) {
     const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&r);
 #pragma unroll
     for (int i = 0; i < 4; ++i) { float2 q = __bfloat1622float2(h[i]); f[2 * i] = q.x; f[2 * i + 1] = q.y; }

@@ -3,6 +3,8 @@
 // per-channel coefficients are loaded once and reductions stay inside the CTA (warp shuffles +
 // one shared-memory step).  Cross-CTA reductions go through per-row partials that a finalize
 // kernel sums in a fixed order, so results are bit-repeatable.
+#include <algorithm>
+
 #include "common.cuh"
 #include "kernels.h"
 
@@ -39,7 +41,8 @@ __device__ __forceinline__ void block_sum(float (&v)[N]) {
 __device__ __forceinline__ float block_max(float v) { return warp_max(v); }
 
 __global__ void lengths_kernel(const int* __restrict__ len_in, int B, int T_in, int stride,
-                               int* __restrict__ len_out, int* __restrict__ nvalid, int* status) {
+                               int* __restrict__ len_out, int* __restrict__ nvalid, int* __restrict__ blk_off,
+                               int* status) {
     // single CTA; B is small (<= a few thousand)
     __shared__ int total;
     if (threadIdx.x == 0) total = 0;
@@ -54,7 +57,14 @@ __global__ void lengths_kernel(const int* __restrict__ len_in, int B, int T_in, 
     }
     atomicAdd(&total, local);   // integer: order-independent
     __syncthreads();
-    if (threadIdx.x == 0) *nvalid = total;
+    if (threadIdx.x == 0) {
+        *nvalid = total;
+        if (blk_off) {              // B is small: a serial scan by one thread
+            int acc = 0;
+            for (int b = 0; b < B; ++b) { blk_off[b] = acc; acc += (len_out[b] + 63) / 64; }
+            blk_off[B] = acc;
+        }
+    }
 }
 
 template <typename T>
@@ -86,115 +96,164 @@ bn_stats_kernel(const T* __restrict__ v, const int* __restrict__ len_out, int nr
     if (lane == 0) partials[row] = make_float2(s[0], q[0]);
 }
 
-// One warp per channel.  Lane l takes parts l, l + 32, ... in increasing order and the 32 lane results
-// are combined by a fixed butterfly, so the result is bit-repeatable.  Pass 1 sums the partial sums,
-// which gives the mean; pass 2 sums M2_p + n_p (mean_p - mean)^2 = M2_p + (sum_p - n_p mean)^2 / n_p.
-// No term depends on the previous one, so a lane's loads are all in flight together; the parts are
-// kept in registers between the passes when there are at most kFinKeep per lane.
-constexpr int kFinKeep = 8;
-constexpr int kFinWarps = 8;
-__device__ __forceinline__ double warp_sum_d(double v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
+// Thirty-two channels per CTA, one per lane, so that every load of a warp is one contiguous run of the
+// [part][channel] partial array.  Warp w takes parts w, w + 32, ... in increasing order; the thirty-two
+// warp results are combined in warp order, so the result is bit-repeatable.  One pass: with a pivot c
+// (the mean of the channel's first part, which always holds at least one valid frame)
+//   sum = sum_p sum_p,   M2 = sum_p [M2_p + n_p (mean_p - c)^2]  -  N (mean - c)^2,
+// and because c lies within the spread of the data the subtraction cancels nothing that matters.
+// No term depends on the previous one, so a lane's few loads are all in flight together.
+constexpr int kFinWarps = 32;
 __global__ void __launch_bounds__(32 * kFinWarps)
 bn_finalize_kernel(const float2* __restrict__ partials, int parts_per_b, int tile_w,
                    const int* __restrict__ len_out, const int* __restrict__ nvalid, int B,
                    int C, float eps, float momentum, float* __restrict__ mean_out,
                    float* __restrict__ invstd_out, float* running_mean, float* running_var) {
-    const int lane = threadIdx.x & 31;
-    const int o = blockIdx.x * kFinWarps + (threadIdx.x >> 5);
-    if (o >= C) return;
+    __shared__ float2 s_red[kFinWarps][32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int o = blockIdx.x * 32 + lane;
+    const bool act = o < C;
     const int nparts = B * parts_per_b;
+    auto count_of = [&](int pi) -> int {
+        const int b = pi / parts_per_b, j = pi - b * parts_per_b;
+        return max(0, min(len_out[b] - j * tile_w, tile_w));
+    };
+    float s1 = 0.f, q = 0.f;
+    if (act) {
+        const float c = partials[o].x / (float)max(1, count_of(0));
+        for (int p0 = w; p0 < nparts; p0 += 8 * kFinWarps) {
+            float2 v[8]; int cnt[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {        // issue every load before the first use
+                const int pi = p0 + i * kFinWarps;
+                cnt[i] = pi < nparts ? count_of(pi) : 0;
+                v[i] = cnt[i] > 0 ? partials[(size_t)pi * C + o] : make_float2(0.f, 0.f);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (cnt[i] > 0) {
+                    const float n = (float)cnt[i];
+                    const float d = v[i].x / n - c;
+                    s1 += v[i].x;
+                    q += fmaf(n * d, d, v[i].y);
+                }
+            }
+        }
+    }
+    s_red[w][lane] = make_float2(s1, q);
+    __syncthreads();
+    if (w != 0 || !act) return;
     const double N = (double)(*nvalid);
-    float2 keep[kFinKeep];
-    int cnts[kFinKeep];
+    const double c = (double)(partials[o].x / (float)max(1, count_of(0)));
+    double t = 0.0, m2 = 0.0;
 #pragma unroll
-    for (int i = 0; i < kFinKeep; ++i) {
-        const int pi = lane + 32 * i;
-        cnts[i] = 0; keep[i] = make_float2(0.f, 0.f);
-        if (pi < nparts) {
-            const int b = pi / parts_per_b, j = pi - b * parts_per_b;
-            cnts[i] = max(0, min(len_out[b] - j * tile_w, tile_w));
-            if (cnts[i] > 0) keep[i] = partials[(size_t)pi * C + o];
-        }
-    }
-    double s1 = 0.0;
-#pragma unroll
-    for (int i = 0; i < kFinKeep; ++i) if (cnts[i] > 0) s1 += (double)keep[i].x;
-    for (int pi = lane + 32 * kFinKeep; pi < nparts; pi += 32) {
-        const int b = pi / parts_per_b, j = pi - b * parts_per_b;
-        if (len_out[b] - j * tile_w > 0) s1 += (double)partials[(size_t)pi * C + o].x;
-    }
-    const double mean = N > 0 ? warp_sum_d(s1) / N : 0.0;
-    double q = 0.0;
-#pragma unroll
-    for (int i = 0; i < kFinKeep; ++i)
-        if (cnts[i] > 0) {
-            const double d = (double)keep[i].x - (double)cnts[i] * mean;
-            q += (double)keep[i].y + (double)((float)(d * d) / (float)cnts[i]);
-        }
-    for (int pi = lane + 32 * kFinKeep; pi < nparts; pi += 32) {
-        const int b = pi / parts_per_b, j = pi - b * parts_per_b;
-        const int cnt = min(len_out[b] - j * tile_w, tile_w);
-        if (cnt <= 0) continue;
-        const float2 p = partials[(size_t)pi * C + o];
-        const double d = (double)p.x - (double)cnt * mean;
-        q += (double)p.y + (double)((float)(d * d) / (float)cnt);
-    }
-    const double m2 = warp_sum_d(q);
-    if (lane != 0) return;
-    const double var = N > 0 ? m2 / N : 0.0;
+    for (int i = 0; i < kFinWarps; ++i) { t += (double)s_red[i][lane].x; m2 += (double)s_red[i][lane].y; }
+    const double mean = N > 0 ? t / N : 0.0;
+    double var = N > 0 ? (m2 - N * (mean - c) * (mean - c)) / N : 0.0;
+    var = var > 0.0 ? var : 0.0;
     const float invstd = (float)(1.0 / sqrt(var + (double)eps));
-    const float mu = (float)mean;
-    mean_out[o] = mu;
+    mean_out[o] = (float)mean;
     invstd_out[o] = invstd;
-    if (running_mean) running_mean[o] = (1.f - momentum) * running_mean[o] + momentum * mu;
+    if (running_mean) running_mean[o] = (1.f - momentum) * running_mean[o] + momentum * (float)mean;
     if (running_var) {
         double unb = N > 1 ? var * (N / (N - 1.0)) : var;
         running_var[o] = (1.f - momentum) * running_var[o] + momentum * (float)unb;
     }
 }
 
-template <typename T, typename VT, typename NT>
+// The same merge for the per-(CTA, channel) partials (count, sum, M2) of the flattened-block contraction.
+// CTA c of the contraction contributed to M tile m iff its unit range [c U / G, (c+1) U / G) meets
+// [m nblk, (m+1) nblk); the pivot is the mean of the first contributing CTA's partial.
+__global__ void __launch_bounds__(32 * kFinWarps)
+bn_finalize_flat_kernel(const float4* __restrict__ partials, int G, int tiles_m, int rows_per_tile,
+                        const int* __restrict__ blk_off, const int* __restrict__ nvalid, int B, int C, float eps,
+                        float momentum, float* __restrict__ mean_out, float* __restrict__ invstd_out,
+                        float* running_mean, float* running_var) {
+    __shared__ float2 s_red[kFinWarps][32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int o = blockIdx.x * 32 + lane;
+    const bool act = o < C;
+    const long long nblk = blk_off[B];
+    const long long U = (long long)tiles_m * nblk;
+    const int m = min(o, C - 1) / rows_per_tile;
+    const long long lo = m * nblk, hi = lo + nblk;
+    auto takes_part = [&](int c) -> bool {
+        const long long b0 = U * c / G, b1 = U * (c + 1) / G;
+        return max(b0, lo) < min(b1, hi);
+    };
+    int c_first = U > 0 ? (int)(lo * G / U) : 0;
+    while (c_first < G - 1 && !takes_part(c_first)) ++c_first;
+    float pivot = 0.f;
+    if (act && U > 0) { const float4 pv = partials[(size_t)c_first * C + o]; pivot = pv.x > 0.f ? pv.y / pv.x : 0.f; }
+    float s1 = 0.f, q = 0.f;
+    if (act && U > 0) {
+        for (int c0 = w; c0 < G; c0 += 8 * kFinWarps) {
+            float4 v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {        // issue every load before the first use
+                const int c = c0 + i * kFinWarps;
+                v[i] = (c < G && takes_part(c)) ? partials[(size_t)c * C + o] : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (v[i].x > 0.f) {
+                    const float d = v[i].y / v[i].x - pivot;
+                    s1 += v[i].y;
+                    q += fmaf(v[i].x * d, d, v[i].z);
+                }
+            }
+        }
+    }
+    s_red[w][lane] = make_float2(s1, q);
+    __syncthreads();
+    if (w != 0 || !act) return;
+    const double N = (double)(*nvalid);
+    double t = 0.0, m2 = 0.0;
+#pragma unroll
+    for (int i = 0; i < kFinWarps; ++i) { t += (double)s_red[i][lane].x; m2 += (double)s_red[i][lane].y; }
+    const double mean = N > 0 ? t / N : 0.0;
+    double var = N > 0 ? (m2 - N * (mean - (double)pivot) * (mean - (double)pivot)) / N : 0.0;
+    var = var > 0.0 ? var : 0.0;
+    mean_out[o] = (float)mean;
+    invstd_out[o] = (float)(1.0 / sqrt(var + (double)eps));
+    if (running_mean) running_mean[o] = (1.f - momentum) * running_mean[o] + momentum * (float)mean;
+    if (running_var) {
+        double unb = N > 1 ? var * (N / (N - 1.0)) : var;
+        running_var[o] = (1.f - momentum) * running_var[o] + momentum * (float)unb;
+    }
+}
+
+template <typename T, typename NT>
 __global__ void __launch_bounds__(kRowThreads) bn_apply_kernel(ApplyArgs a) {
     SC_ROW_SETUP(a.B * a.C)
     const int b = row / a.C, o = row % a.C;
     const int Tp = a.Tp, len = min(a.len_out[b], Tp);
     const bool vec = (Tp % 8 == 0);
     const size_t off = (size_t)row * Tp;
-    const VT* __restrict__ v = (const VT*)a.v + off;
+    const NT* __restrict__ v = (const NT*)a.v + off;
     const T* __restrict__ xr = a.residual == 1 ? (const T*)a.xres + off : nullptr;
-    const VT* __restrict__ vr = a.residual == 2 ? (const VT*)a.vr + off : nullptr;
+    const NT* __restrict__ vr = a.residual == 2 ? (const NT*)a.vr + off : nullptr;
     T* __restrict__ y = (T*)a.y + off;
-    NT* __restrict__ vh = (NT*)a.vhat + off;
-    NT* __restrict__ vhr = a.residual == 2 ? (NT*)a.vhat_r + off : nullptr;
     const float mu = a.mean[o], is = a.invstd[o], ga = a.gamma[o], be = a.beta[o];
     float mur = 0.f, isr = 0.f, gar = 0.f, ber = 0.f;
     if (a.residual == 2) { mur = a.mean_r[o]; isr = a.invstd_r[o]; gar = a.gamma_r[o]; ber = a.beta_r[o]; }
     for (int t0 = lane * 8; t0 < Tp; t0 += 256) {
-        float out[8], n1[8], n2[8];
+        float out[8];
         if (t0 < len) {
             float f[8], r[8];
             load_chunk(v, t0, Tp, vec, f);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) n1[i] = (t0 + i < len) ? round_io<NT>((f[i] - mu) * is) : 0.f;
             if (a.residual == 1) load_chunk(xr, t0, Tp, vec, r);
             else if (a.residual == 2) {
                 load_chunk(vr, t0, Tp, vec, r);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    n2[i] = (t0 + i < len) ? round_io<NT>((r[i] - mur) * isr) : 0.f;
-                    r[i] = fmaf(gar, n2[i], ber);
-                }
+                for (int i = 0; i < 8; ++i) r[i] = fmaf(gar, bn_norm(r[i], mur, isr), ber);
             } else {
 #pragma unroll
                 for (int i = 0; i < 8; ++i) r[i] = 0.f;
             }
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                float bn = fmaf(ga, n1[i], be);     // from the stored (rounded) vhat: backward sees the same value
+                float bn = fmaf(ga, bn_norm(f[i], mu, is), be);   // the backward pass recomputes exactly this
                 float q;
                 if (a.res_before_relu) { q = bn + r[i]; if (a.has_relu) q = fmaxf(q, 0.f); }
                 else { q = (a.has_relu ? fmaxf(bn, 0.f) : bn) + r[i]; }
@@ -202,29 +261,29 @@ __global__ void __launch_bounds__(kRowThreads) bn_apply_kernel(ApplyArgs a) {
             }
         } else {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) { out[i] = 0.f; n1[i] = 0.f; n2[i] = 0.f; }
+            for (int i = 0; i < 8; ++i) out[i] = 0.f;
         }
         store_chunk(y, t0, Tp, vec, out);
-        store_chunk(vh, t0, Tp, vec, n1);
-        if (vhr) store_chunk(vhr, t0, Tp, vec, n2);
     }
 }
 
 // Shared by the reduce and apply steps of the backward pass: per element gate and normalised value.
 template <typename T, typename NT>
 struct BwdRow {
-    const T* __restrict__ g; const T* __restrict__ y; const NT* __restrict__ vh; const NT* __restrict__ vhr;
-    float gam, bet;
+    const T* __restrict__ g; const T* __restrict__ y; const NT* __restrict__ v; const NT* __restrict__ vr;
+    float gam, bet, mu, is, mur, isr;
     int len, Tp;
     bool vec;
     __device__ BwdRow(const BnBwdArgs& a, int row, int b, int o) {
         Tp = a.Tp; len = min(a.len_out[b], Tp); vec = (Tp % 8 == 0);
         g = (const T*)a.g + (size_t)row * Tp;
         y = a.y ? (const T*)a.y + (size_t)row * Tp : nullptr;
-        vh = a.has_bn ? (const NT*)a.vhat + (size_t)row * Tp : nullptr;
-        vhr = (a.residual == 2) ? (const NT*)a.vhat_r + (size_t)row * Tp : nullptr;
+        v = a.has_bn ? (const NT*)a.v + (size_t)row * Tp : nullptr;
+        vr = (a.residual == 2) ? (const NT*)a.vr + (size_t)row * Tp : nullptr;
         const bool own_gate = a.has_relu && !a.res_before_relu && a.has_bn;
         gam = own_gate ? a.gamma[o] : 1.f; bet = own_gate ? a.beta[o] : 0.f;
+        mu = a.has_bn ? a.mean[o] : 0.f; is = a.has_bn ? a.invstd[o] : 0.f;
+        mur = (a.residual == 2) ? a.mean_r[o] : 0.f; isr = (a.residual == 2) ? a.invstd_r[o] : 0.f;
     }
     // ga: gated upstream gradient; gr: gradient reaching the residual sum; vn/vnr: normalised values
     __device__ __forceinline__ void chunk(const BnBwdArgs& a, int t0, float (&ga)[8], float (&gr)[8],
@@ -233,13 +292,19 @@ struct BwdRow {
         load_chunk(g, t0, Tp, vec, fg);
         const bool need_y = a.has_relu && a.res_before_relu;
         if (need_y) load_chunk(y, t0, Tp, vec, fy);
-        if (a.has_bn) load_chunk(vh, t0, Tp, vec, vn);
-        else {
+        if (a.has_bn) {
+            load_chunk(v, t0, Tp, vec, vn);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) vn[i] = bn_norm(vn[i], mu, is);
+        } else {
 #pragma unroll
             for (int i = 0; i < 8; ++i) vn[i] = 0.f;
         }
-        if (a.residual == 2) load_chunk(vhr, t0, Tp, vec, vnr);
-        else {
+        if (a.residual == 2) {
+            load_chunk(vr, t0, Tp, vec, vnr);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) vnr[i] = bn_norm(vnr[i], mur, isr);
+        } else {
 #pragma unroll
             for (int i = 0; i < 8; ++i) vnr[i] = 0.f;
         }
@@ -255,6 +320,12 @@ struct BwdRow {
         }
     }
 };
+
+// Partial sums of the backward reduction live in a [sample][slot][channel] array, so that the finalize
+// kernel, which gives one channel to each lane, reads contiguous runs.
+__device__ __forceinline__ size_t bwd_part_index(const BnBwdArgs& a, int b, int slot, int o) {
+    return ((size_t)b * a.nslots + slot) * a.C + o;
+}
 
 template <typename T, typename NT>
 __global__ void __launch_bounds__(kRowThreads) bn_bwd_reduce_kernel(BnBwdArgs a) {
@@ -275,79 +346,85 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_reduce_kernel(BnBwdArgs a)
     block_sum(s);
     if (a.gmax) amax = block_max(amax);
     if (lane == 0) {
-        a.partials[(size_t)row * a.nslots] = make_float4(s[0], s[1], s[2], s[3]);
-        if (a.gmax) a.amax_part[(size_t)row * a.nslots] = amax;
+        a.partials[bwd_part_index(a, b, 0, o)] = make_float4(s[0], s[1], s[2], s[3]);
+        if (a.gmax) a.amax_part[bwd_part_index(a, b, 0, o)] = amax;
     }
 }
 
-// One warp per channel: lane l takes the (sample, slot) partials l, l + 32, ... in increasing order; the
-// lane sums are combined by a fixed butterfly.
+// Thirty-two channels per CTA, one per lane; warp w takes samples w, w + 32, ... with all their slots (every
+// load issued before the first add) and the thirty-two warp results are combined in warp order
+// (bit-repeatable).
+constexpr int kBwdMaxSlotsUnrolled = 8;
 __global__ void __launch_bounds__(32 * kFinWarps)
 bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const float* gamma_r, float* dgamma, float* dbeta,
                        float* dgamma_r, float* dbeta_r, float* dbias, int accumulate) {
-    const int lane = threadIdx.x & 31;
-    const int o = blockIdx.x * kFinWarps + (threadIdx.x >> 5);
-    if (o >= a.C) return;
-    double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
-    float amax = 0.f;
-    {
-        const int vpr = a.Tp / 8;
-        const int np = a.B * a.nslots;
-        for (int base = lane; base < np; base += 8 * 32) {
-            float4 pv[8]; float am[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {          // issue every load before the first add
-                const int pi = base + i * 32;
-                bool use = pi < np;
-                pv[i] = make_float4(0.f, 0.f, 0.f, 0.f); am[i] = 0.f;
-                if (use) {
-                    const int b = pi / a.nslots, slot = pi - b * a.nslots;
-                    const long long r = (long long)b * a.C + o;
-                    if (a.nslots > 1) {      // slots in use for this row (see bn_bwd_reduce_fast_kernel)
-                        const int used = (int)((((r + 1) * vpr - 1) >> 5) - ((r * vpr) >> 5)) + 1;
-                        use = slot < used;
-                    }
-                    if (use) {
-                        pv[i] = a.partials[(size_t)r * a.nslots + slot];
-                        if (a.gmax) am[i] = a.amax_part[(size_t)r * a.nslots + slot];
-                    }
-                }
+    __shared__ float4 s_sum[kFinWarps][32];
+    __shared__ float s_max[kFinWarps][32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int o = blockIdx.x * 32 + lane;
+    const bool act = o < a.C;
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f, amax = 0.f;
+    if (act) {
+        const uint32_t vpr = (uint32_t)(a.Tp / 8);
+        for (int b = w; b < a.B; b += kFinWarps) {
+            int used = 1;
+            if (a.nslots > 1) {      // slots in use for this row (see bn_bwd_reduce_fast_kernel); r * vpr < 2^31
+                const uint32_t r = (uint32_t)b * (uint32_t)a.C + (uint32_t)o;
+                used = (int)((((r + 1u) * vpr - 1u) >> a.vpw_shift) - ((r * vpr) >> a.vpw_shift)) + 1;
             }
+            for (int sl0 = 0; sl0 < used; sl0 += kBwdMaxSlotsUnrolled) {
+                float4 pv[kBwdMaxSlotsUnrolled]; float am[kBwdMaxSlotsUnrolled];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                s0 += pv[i].x; s1 += pv[i].y; s2 += pv[i].z; s3 += pv[i].w;
-                amax = fmaxf(amax, am[i]);
+                for (int i = 0; i < kBwdMaxSlotsUnrolled; ++i) {
+                    const bool use = sl0 + i < used;
+                    pv[i] = use ? a.partials[bwd_part_index(a, b, sl0 + i, o)] : make_float4(0.f, 0.f, 0.f, 0.f);
+                    am[i] = (use && a.gmax) ? a.amax_part[bwd_part_index(a, b, sl0 + i, o)] : 0.f;
+                }
+#pragma unroll
+                for (int i = 0; i < kBwdMaxSlotsUnrolled; ++i) {
+                    s0 += pv[i].x; s1 += pv[i].y; s2 += pv[i].z; s3 += pv[i].w;
+                    amax = fmaxf(amax, am[i]);
+                }
             }
         }
     }
-    s0 = warp_sum_d(s0); s1 = warp_sum_d(s1); s2 = warp_sum_d(s2); s3 = warp_sum_d(s3);
-    amax = warp_max(amax);
-    if (lane != 0) return;
+    s_sum[w][lane] = make_float4(s0, s1, s2, s3);
+    s_max[w][lane] = amax;
+    __syncthreads();
+    if (w != 0 || !act) return;
+    double d0 = 0, d1 = 0, d2 = 0, d3 = 0;
+    amax = 0.f;
+#pragma unroll
+    for (int i = 0; i < kFinWarps; ++i) {
+        const float4 q = s_sum[i][lane];
+        d0 += q.x; d1 += q.y; d2 += q.z; d3 += q.w;
+        amax = fmaxf(amax, s_max[i][lane]);
+    }
     const float N = (float)(*a.nvalid);
     if (a.gmax) {
         // |gv| <= |k| (max|ga| + |c1| + max|vhat| |c2|) and max|vhat| <= sqrt(N); a maximum is order-free,
         // so the integer atomic on the (non-negative) float's bit pattern keeps the result repeatable
         float bound = amax;
         if (a.has_bn)
-            bound = fabsf(gamma[o] * a.invstd[o]) * (amax + fabsf((float)s0) / N + sqrtf(N) * fabsf((float)s1) / N);
+            bound = fabsf(gamma[o] * a.invstd[o]) * (amax + fabsf((float)d0) / N + sqrtf(N) * fabsf((float)d1) / N);
         if (a.residual == 2)     // the residual branch's gradient shares the scale
             bound = fmaxf(bound, fabsf(gamma_r[o] * a.invstd_r[o]) *
-                                     (amax + fabsf((float)s2) / N + sqrtf(N) * fabsf((float)s3) / N));
+                                     (amax + fabsf((float)d2) / N + sqrtf(N) * fabsf((float)d3) / N));
         if (bound < 3.0e38f) atomicMax(reinterpret_cast<unsigned int*>(a.gmax), __float_as_uint(bound));
     }
     auto put = [&](float* dst, double val) {
         if (dst) dst[o] = accumulate ? dst[o] + (float)val : (float)val;
     };
     if (a.has_bn) {
-        put(dbeta, s0); put(dgamma, s1);
-        a.coef[o] = make_float4(gamma[o] * a.invstd[o], (float)s0 / N, (float)s1 / N, 0.f);
+        put(dbeta, d0); put(dgamma, d1);
+        a.coef[o] = make_float4(gamma[o] * a.invstd[o], (float)d0 / N, (float)d1 / N, 0.f);
     } else {
-        put(dbias, s0);
+        put(dbias, d0);
         a.coef[o] = make_float4(1.f, 0.f, 0.f, 0.f);
     }
     if (a.residual == 2) {
-        put(dbeta_r, s2); put(dgamma_r, s3);
-        a.coef_r[o] = make_float4(gamma_r[o] * a.invstd_r[o], (float)s2 / N, (float)s3 / N, 0.f);
+        put(dbeta_r, d2); put(dgamma_r, d3);
+        a.coef_r[o] = make_float4(gamma_r[o] * a.invstd_r[o], (float)d2 / N, (float)d3 / N, 0.f);
     }
 }
 
@@ -410,179 +487,246 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_apply_kernel(BnBwdArgs a) 
 }
 
 // ---- flattened fast paths (the encoder's configuration: BN + ReLU, residual joined before the ReLU,
-// rows a multiple of 8 frames).  One 8-frame vector per thread: no row tails, few registers, so many
-// warps and many 16-byte loads in flight per SM.
-template <typename T, typename VT, typename NT, int RES>
+// rows a multiple of 8 frames).  A warp takes 32 * V consecutive 8-frame vectors, lane l the vectors
+// l, l + 32, ...: no row tails, and V independent 16-byte loads per tensor in flight per thread.
+template <typename T, typename NT, int RES, int V>
 __global__ void __launch_bounds__(256) bn_apply_fast_kernel(ApplyArgs a, int vpr, long long total) {
-    const uint32_t idx = blockIdx.x * 256u + threadIdx.x;       // the launcher guarantees total < 2^31
-    if (idx >= (uint32_t)total) return;
-    const int row = (int)a.dvpr.div(idx), t0 = ((int)idx - row * vpr) * 8;
-    const int b = (int)a.dC.div((uint32_t)row), o = row - b * a.C;
-    const int len = min(a.len_out[b], a.Tp);
-    const size_t off = (size_t)row * a.Tp + t0;
-    float out[8], n1[8], n2[8];
-    if (t0 < len) {
-        float f[8], r[8];
-        ld8<VT>((const VT*)a.v + off, f);
-        if (RES == 1) ld8<T>((const T*)a.xres + off, r);
-        if (RES == 2) ld8<VT>((const VT*)a.vr + off, r);
-        const float mu = a.mean[o], is = a.invstd[o], ga = a.gamma[o], be = a.beta[o];
-        float mur = 0.f, isr = 0.f, gar = 0.f, ber = 0.f;
-        if (RES == 2) { mur = a.mean_r[o]; isr = a.invstd_r[o]; gar = a.gamma_r[o]; ber = a.beta_r[o]; }
+    const uint32_t tid = blockIdx.x * 256u + threadIdx.x;        // the launcher guarantees total < 2^31
+    const uint32_t base = (tid >> 5) * (32u * V) + (threadIdx.x & 31), tot = (uint32_t)total;
+    size_t off[V]; int nin[V], ch[V];
+    uint4 rv[V], rr[V];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const bool in = t0 + i < len;
-            n1[i] = in ? round_io<NT>((f[i] - mu) * is) : 0.f;
-            float rr = 0.f;
-            if (RES == 1) rr = r[i];
-            if (RES == 2) { n2[i] = in ? round_io<NT>((r[i] - mur) * isr) : 0.f; rr = fmaf(gar, n2[i], ber); }
-            out[i] = in ? fmaxf(fmaf(ga, n1[i], be) + rr, 0.f) : 0.f;
+    for (int j = 0; j < V; ++j) {
+        const uint32_t idx = base + 32u * j;
+        nin[j] = -1; ch[j] = 0; off[j] = 0;
+        rv[j] = make_uint4(0, 0, 0, 0); rr[j] = make_uint4(0, 0, 0, 0);
+        if (idx < tot) {
+            const int row = (int)a.dvpr.div(idx), t0 = ((int)idx - row * vpr) * 8;
+            const int b = (int)a.dC.div((uint32_t)row);
+            ch[j] = row - b * a.C;
+            nin[j] = max(0, min(a.len_out[b], a.Tp) - t0);
+            off[j] = (size_t)row * a.Tp + t0;
+            if (nin[j] > 0) {
+                rv[j] = *reinterpret_cast<const uint4*>((const NT*)a.v + off[j]);
+                if (RES == 1) rr[j] = *reinterpret_cast<const uint4*>((const T*)a.xres + off[j]);
+                if (RES == 2) rr[j] = *reinterpret_cast<const uint4*>((const NT*)a.vr + off[j]);
+            }
         }
-    } else {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) { out[i] = 0.f; n1[i] = 0.f; n2[i] = 0.f; }
     }
-    st8<T>((T*)a.y + off, out);
-    st8<NT>((NT*)a.vhat + off, n1);
-    if (RES == 2) st8<NT>((NT*)a.vhat_r + off, n2);
-}
-
-template <typename T, typename NT, typename GT, int RES>
-__global__ void __launch_bounds__(256) bn_bwd_apply_fast_kernel(BnBwdArgs a, int vpr, long long total) {
-    const uint32_t idx = blockIdx.x * 256u + threadIdx.x;       // the launcher guarantees total < 2^31
-    if (idx >= (uint32_t)total) return;
-    const int row = (int)a.dvpr.div(idx), t0 = ((int)idx - row * vpr) * 8;
-    const int b = (int)a.dC.div((uint32_t)row), o = row - b * a.C;
-    const int len = min(a.len_out[b], a.Tp);
-    const size_t off = (size_t)row * a.Tp + t0;
-    float o1[8], o2[8];
-    const int nin = len - t0;                                      // frames of this vector inside the sample
-    const float sc = a.gmax ? pow2_scale(*a.gmax) : 1.f;          // multiplying by it is exact: a power of two
-    const bool fold = !a.gv16 && a.gv_scaled;
-    if (t0 < len) {
-        float g[8], y[8], vn[8], vnr[8];
-        ld8<T>((const T*)a.g + off, g);
-        ld8<NT>((const NT*)a.vhat + off, vn);
-        if (RES == 2) ld8<NT>((const NT*)a.vhat_r + off, vnr);
-        if (RES == 0) {
-            // without a residual the forward output is relu(gamma * vhat + beta) of the STORED vhat, rounded
-            // to the activation type: the gate is recomputed from vhat and the output need not be read
-            const float ga_ = a.gamma[o], be_ = a.beta[o];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) y[i] = round_io<T>(fmaf(ga_, vn[i], be_));
-        } else {
-            ld8<T>((const T*)a.y + off, y);
-        }
-        // gv = k (ga - c1 - c2 vhat) as two fused multiply-adds; when gv itself is the scaled half tensor the
-        // power-of-two scale is folded into k (exact)
-        const float4 cf = a.coef[o];
-        const float kx = (fold ? sc : 1.f) * cf.x;
-        const float k0 = -kx * cf.y, k2 = -kx * cf.z;
-        float kr = 0.f, r0 = 0.f, r2 = 0.f;
-        if (RES == 2) { const float4 cr = a.coef_r[o]; kr = cr.x; r0 = -kr * cr.y; r2 = -kr * cr.z; }
-        if (nin >= 8) {
+    for (int j = 0; j < V; ++j) {
+        if (nin[j] < 0) continue;
+        float out[8];
+        if (nin[j] > 0) {
+            const int o = ch[j];
+            float f[8], r[8];
+            cvt8<NT>(rv[j], f);
+            if (RES == 1) cvt8<T>(rr[j], r);
+            if (RES == 2) cvt8<NT>(rr[j], r);
+            const float mu = a.mean[o], is = a.invstd[o], ga = a.gamma[o], be = a.beta[o];
+            float mur = 0.f, isr = 0.f, gar = 0.f, ber = 0.f;
+            if (RES == 2) { mur = a.mean_r[o]; isr = a.invstd_r[o]; gar = a.gamma_r[o]; ber = a.beta_r[o]; }
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                const float ga = y[i] > 0.f ? g[i] : 0.f;
-                o1[i] = fmaf(k2, vn[i], fmaf(kx, ga, k0));
-                if (RES == 2) o2[i] = fmaf(r2, vnr[i], fmaf(kr, ga, r0));
-                if (RES == 1) o2[i] = ga;
+                float rres = 0.f;
+                if (RES == 1) rres = r[i];
+                if (RES == 2) rres = fmaf(gar, bn_norm(r[i], mur, isr), ber);
+                const float q = fmaxf(fmaf(ga, bn_norm(f[i], mu, is), be) + rres, 0.f);
+                out[i] = i < nin[j] ? q : 0.f;
             }
         } else {
 #pragma unroll
+            for (int i = 0; i < 8; ++i) out[i] = 0.f;
+        }
+        st8<T>((T*)a.y + off[j], out);
+    }
+}
+
+template <typename T, typename NT, typename GT, int RES, int V>
+__global__ void __launch_bounds__(256) bn_bwd_apply_fast_kernel(BnBwdArgs a, int vpr, long long total) {
+    const uint32_t tid = blockIdx.x * 256u + threadIdx.x;        // the launcher guarantees total < 2^31
+    const uint32_t base = (tid >> 5) * (32u * V) + (threadIdx.x & 31), tot = (uint32_t)total;
+    const float sc = a.gmax ? pow2_scale(*a.gmax) : 1.f;          // multiplying by it is exact: a power of two
+    const bool fold = !a.gv16 && a.gv_scaled;
+    size_t off[V]; int nin[V], ch[V];
+    uint4 rg[V], rv[V], rr[V], ry[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+        const uint32_t idx = base + 32u * j;
+        nin[j] = -1; ch[j] = 0; off[j] = 0;
+        rg[j] = rv[j] = rr[j] = ry[j] = make_uint4(0, 0, 0, 0);
+        if (idx < tot) {
+            const int row = (int)a.dvpr.div(idx), t0 = ((int)idx - row * vpr) * 8;
+            const int b = (int)a.dC.div((uint32_t)row);
+            ch[j] = row - b * a.C;
+            nin[j] = max(0, min(a.len_out[b], a.Tp) - t0);        // frames of this vector inside the sample
+            off[j] = (size_t)row * a.Tp + t0;
+            if (nin[j] > 0) {
+                rg[j] = *reinterpret_cast<const uint4*>((const T*)a.g + off[j]);
+                rv[j] = *reinterpret_cast<const uint4*>((const NT*)a.v + off[j]);
+                if (RES == 2) rr[j] = *reinterpret_cast<const uint4*>((const NT*)a.vr + off[j]);
+                if (RES != 0) ry[j] = *reinterpret_cast<const uint4*>((const T*)a.y + off[j]);
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+        if (nin[j] < 0) continue;
+        float o1[8], o2[8];
+        const int n = nin[j];
+        if (n > 0) {
+            const int o = ch[j];
+            float g[8], y[8], vn[8], vnr[8];
+            cvt8<T>(rg[j], g);
+            cvt8<NT>(rv[j], vn);
+            const float mu = a.mean[o], is = a.invstd[o];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) vn[i] = bn_norm(vn[i], mu, is);
+            if (RES == 2) {
+                cvt8<NT>(rr[j], vnr);
+                const float mur = a.mean_r[o], isr = a.invstd_r[o];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) vnr[i] = bn_norm(vnr[i], mur, isr);
+            }
+            if (RES == 0) {
+                // without a residual the forward output is relu(gamma * vhat + beta), rounded to the
+                // activation type: the gate is recomputed from v and the output need not be read
+                const float ga_ = a.gamma[o], be_ = a.beta[o];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) y[i] = round_io<T>(fmaf(ga_, vn[i], be_));
+            } else {
+                cvt8<T>(ry[j], y);
+            }
+            // gv = k (ga - c1 - c2 vhat) as two fused multiply-adds; when gv itself is the scaled half tensor the
+            // power-of-two scale is folded into k (exact)
+            const float4 cf = a.coef[o];
+            const float kx = (fold ? sc : 1.f) * cf.x;
+            const float k0 = -kx * cf.y, k2 = -kx * cf.z;
+            float kr = 0.f, r0 = 0.f, r2 = 0.f;
+            if (RES == 2) { const float4 cr = a.coef_r[o]; kr = cr.x; r0 = -kr * cr.y; r2 = -kr * cr.z; }
+#pragma unroll
             for (int i = 0; i < 8; ++i) {
-                const bool in = i < nin;
+                const bool in = i < n;
                 const float ga = (in && y[i] > 0.f) ? g[i] : 0.f;
                 o1[i] = in ? fmaf(k2, vn[i], fmaf(kx, ga, k0)) : 0.f;
                 if (RES == 2) o2[i] = in ? fmaf(r2, vnr[i], fmaf(kr, ga, r0)) : 0.f;
                 if (RES == 1) o2[i] = ga;
             }
-        }
-    } else {
+        } else {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { o1[i] = 0.f; o2[i] = 0.f; }
-    }
-    {
+            for (int i = 0; i < 8; ++i) { o1[i] = 0.f; o2[i] = 0.f; }
+        }
         if (a.gv16) {            // half copy for the weight gradient; gv itself keeps plain rounding
             float h[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) h[i] = o1[i] * sc;
-            diffuse8<__half>(h, nin);
-            st8<__half>((__half*)a.gv16 + off, h);
+            diffuse8<__half>(h, n);
+            st8<__half>((__half*)a.gv16 + off[j], h);
         } else {
-            diffuse8<GT>(o1, nin);
+            diffuse8<GT>(o1, n);
         }
         if (RES == 2) {
             if (a.gvr16) {
                 float h[8];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) h[i] = o2[i] * sc;
-                diffuse8<__half>(h, nin);
-                st8<__half>((__half*)a.gvr16 + off, h);
+                diffuse8<__half>(h, n);
+                st8<__half>((__half*)a.gvr16 + off[j], h);
             } else {
-                diffuse8<T>(o2, nin);
+                diffuse8<T>(o2, n);
+            }
+        }
+        st8<GT>((GT*)a.gv + off[j], o1);
+        if (RES == 2) st8<T>((T*)a.gvr + off[j], o2);
+        if (RES == 1) st8<T>((T*)a.gres + off[j], o2);
+    }
+}
+
+// Flattened reduce: a warp's 32 * V consecutive vectors belong to at most two rows (vpr >= 32 * V), so two
+// masked warp reductions give one partial per (row, warp) pair.  Row r's partials sit in slots
+// [0, last_warp(r) - first_warp(r)] with first_warp(r) = (r * vpr) / (32 * V): a static assignment,
+// summed later in slot order.
+template <typename T, typename NT, int RES, int V>
+__global__ void __launch_bounds__(256) bn_bwd_reduce_fast_kernel(BnBwdArgs a, int vpr, long long total) {
+    const uint32_t tid = blockIdx.x * 256u + threadIdx.x;        // the launcher guarantees total < 2^31
+    const int lane = threadIdx.x & 31;
+    const uint32_t wg = tid >> 5;                                // global warp index
+    const uint32_t warp_first = wg * (32u * V), tot = (uint32_t)total;
+    if (warp_first >= tot) return;
+    const int row0 = (int)a.dvpr.div(warp_first);
+    int nin[V], ch[V], rw[V];
+    uint4 rg[V], rv[V], rr[V], ry[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+        const uint32_t idx = warp_first + 32u * j + lane;
+        nin[j] = 0; ch[j] = 0; rw[j] = row0;
+        rg[j] = rv[j] = rr[j] = ry[j] = make_uint4(0, 0, 0, 0);
+        if (idx < tot) {
+            const int row = (int)a.dvpr.div(idx), t0 = ((int)idx - row * vpr) * 8;
+            const int b = (int)a.dC.div((uint32_t)row);
+            rw[j] = row; ch[j] = row - b * a.C;
+            nin[j] = max(0, min(a.len_out[b], a.Tp) - t0);
+            if (nin[j] > 0) {
+                const size_t off = (size_t)row * a.Tp + t0;
+                rg[j] = *reinterpret_cast<const uint4*>((const T*)a.g + off);
+                rv[j] = *reinterpret_cast<const uint4*>((const NT*)a.v + off);
+                if (RES == 2) rr[j] = *reinterpret_cast<const uint4*>((const NT*)a.vr + off);
+                if (RES != 0) ry[j] = *reinterpret_cast<const uint4*>((const T*)a.y + off);
             }
         }
     }
-    st8<GT>((GT*)a.gv + off, o1);
-    if (RES == 2) st8<T>((T*)a.gvr + off, o2);
-    if (RES == 1) st8<T>((T*)a.gres + off, o2);
-}
-
-// Flattened reduce: one 8-frame vector per thread; a warp's 32 consecutive vectors belong to at most two
-// rows (vpr >= 32), so two masked warp reductions give one partial per (row, warp) pair.  Row r's
-// partials sit in slots [0, last_warp(r) - first_warp(r)] with first_warp(r) = (r * vpr) >> 5: a static
-// assignment, summed later in slot order.
-template <typename T, typename NT, int RES>
-__global__ void __launch_bounds__(256) bn_bwd_reduce_fast_kernel(BnBwdArgs a, int vpr, long long total) {
-    const uint32_t idx = blockIdx.x * 256u + threadIdx.x;       // the launcher guarantees total < 2^31
-    const int lane = threadIdx.x & 31;
-    const uint32_t warp_first = idx - lane, tot = (uint32_t)total;
-    if (warp_first >= tot) return;
-    const bool valid = idx < tot;
-    const uint32_t cidx = valid ? idx : tot - 1;
-    const int row = (int)a.dvpr.div(cidx), t0 = ((int)cidx - row * vpr) * 8;
-    const int b = (int)a.dC.div((uint32_t)row);
-    const int len = min(a.len_out[b], a.Tp);
-    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f, amax = 0.f;
-    if (valid && t0 < len) {
-        const size_t off = (size_t)row * a.Tp + t0;
+    float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    float amx[2] = {0.f, 0.f};
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+        const int n = nin[j];
+        if (n <= 0) continue;
+        const int o = ch[j];
         float g[8], y[8], vn[8], vnr[8];
-        ld8<T>((const T*)a.g + off, g);
-        ld8<NT>((const NT*)a.vhat + off, vn);
-        if (RES == 2) ld8<NT>((const NT*)a.vhat_r + off, vnr);
-        if (RES == 0) {          // gate from the stored vhat (see bn_bwd_apply_fast_kernel)
-            const int o = row - b * a.C;
+        cvt8<T>(rg[j], g);
+        cvt8<NT>(rv[j], vn);
+        const float mu = a.mean[o], is = a.invstd[o];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) vn[i] = bn_norm(vn[i], mu, is);
+        if (RES == 2) {
+            cvt8<NT>(rr[j], vnr);
+            const float mur = a.mean_r[o], isr = a.invstd_r[o];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) vnr[i] = bn_norm(vnr[i], mur, isr);
+        }
+        if (RES == 0) {          // gate from v (see bn_bwd_apply_fast_kernel)
             const float ga_ = a.gamma[o], be_ = a.beta[o];
 #pragma unroll
             for (int i = 0; i < 8; ++i) y[i] = round_io<T>(fmaf(ga_, vn[i], be_));
         } else {
-            ld8<T>((const T*)a.y + off, y);
+            cvt8<T>(ry[j], y);
         }
+        float s0 = 0.f, s1 = 0.f, s3 = 0.f, m = 0.f;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            const float ga = (t0 + i < len && y[i] > 0.f) ? g[i] : 0.f;
-            s0 += ga; s1 += ga * vn[i];
-            if (RES == 2) { s2 += ga; s3 += ga * vnr[i]; }
-            amax = fmaxf(amax, fabsf(ga));
+            const float ga = (i < n && y[i] > 0.f) ? g[i] : 0.f;
+            s0 += ga; s1 = fmaf(ga, vn[i], s1);
+            if (RES == 2) s3 = fmaf(ga, vnr[i], s3);
+            m = fmaxf(m, fabsf(ga));
         }
+        const int seg = rw[j] != row0 ? 1 : 0;
+        acc[seg][0] += s0; acc[seg][1] += s1; acc[seg][2] += s0; acc[seg][3] += s3;
+        amx[seg] = fmaxf(amx[seg], m);
     }
-    const int row0 = (int)a.dvpr.div(warp_first);
-    const uint32_t wg = warp_first >> 5;                     // global warp index
 #pragma unroll
     for (int seg = 0; seg < 2; ++seg) {
         const int r = row0 + seg;
         const uint32_t rfirst = (uint32_t)r * (uint32_t)vpr;           // first vector of row r
-        if (seg == 1 && rfirst >= warp_first + 32) break;              // warp lies inside one row (uniform)
-        const bool mine = valid && row == r;
-        float v[4] = {mine ? s0 : 0.f, mine ? s1 : 0.f, mine ? s2 : 0.f, mine ? s3 : 0.f};
+        if (seg == 1 && rfirst >= warp_first + 32u * V) break;         // warp lies inside one row (uniform)
+        float v[4] = {acc[seg][0], acc[seg][1], RES == 2 ? acc[seg][2] : 0.f, RES == 2 ? acc[seg][3] : 0.f};
 #pragma unroll
-        for (int i = 0; i < (RES == 2 ? 4 : 2); ++i) v[i] = warp_sum(v[i]);      // v[2], v[3] are zero otherwise
-        const float m = a.gmax ? warp_max(mine ? amax : 0.f) : 0.f;
+        for (int i = 0; i < (RES == 2 ? 4 : 2); ++i) v[i] = warp_sum(v[i]);
+        const float m = a.gmax ? warp_max(amx[seg]) : 0.f;
         if (lane == 0 && rfirst < tot) {
-            const int slot = (int)(wg - (rfirst >> 5));
-            a.partials[(size_t)r * a.nslots + slot] = make_float4(v[0], v[1], v[2], v[3]);
-            if (a.gmax) a.amax_part[(size_t)r * a.nslots + slot] = m;
+            const int slot = (int)(wg - rfirst / (32u * V));
+            const int b = (int)a.dC.div((uint32_t)r), o = r - b * a.C;
+            a.partials[bwd_part_index(a, b, slot, o)] = make_float4(v[0], v[1], v[2], v[3]);
+            if (a.gmax) a.amax_part[bwd_part_index(a, b, slot, o)] = m;
         }
     }
 }
@@ -619,10 +763,14 @@ ew_add_masked_kernel(T* out, const T* a, const T* b, const T* c, const int* len,
 
 #define SC_DISPATCH3(dtype, ...)                                                              \
     switch (dtype) {                                                                          \
-        case F32: { using T = float; using VT = float; using NT = float; __VA_ARGS__; break; }          \
-        case F16: { using T = __half; using VT = __half; using NT = __half; __VA_ARGS__; break; }       \
-        default:  { using T = __nv_bfloat16; using VT = float; using NT = __half; __VA_ARGS__; break; } \
+        case F32: { using T = float; using NT = float; __VA_ARGS__; break; }                  \
+        case F16: { using T = __half; using NT = __half; __VA_ARGS__; break; }                \
+        default:  { using T = __nv_bfloat16; using NT = __half; __VA_ARGS__; break; }         \
     }
+// 16-bit activation types only (the flattened kernels move 16-byte vectors of 8 elements)
+#define SC_DISPATCH16(dtype, ...)                                                             \
+    if (dtype == F16) { using T = __half; using NT = __half; __VA_ARGS__; }                   \
+    else { using T = __nv_bfloat16; using NT = __half; __VA_ARGS__; }
 #define SC_DISPATCH(dtype, ...)                                             \
     switch (dtype) {                                                        \
         case F32: { using T = float; __VA_ARGS__; break; }                  \
@@ -630,16 +778,17 @@ ew_add_masked_kernel(T* out, const T* a, const T* b, const T* c, const int* len,
         default:  { using T = __nv_bfloat16; __VA_ARGS__; break; }          \
     }
 
-void lengths(const Launch& L, const int* len_in, int B, int T_in, int stride, int* len_out, int* nvalid) {
+void lengths(const Launch& L, const int* len_in, int B, int T_in, int stride, int* len_out, int* nvalid, int* blk_off) {
     KScope ks_(L, KC_LENGTHS, 8.0 * B, 0.0);
-    lengths_kernel<<<1, 256, 0, L.stream>>>(len_in, B, T_in, stride, len_out, nvalid, L.status);
+    lengths_kernel<<<1, 256, 0, L.stream>>>(len_in, B, T_in, stride, len_out, nvalid, blk_off, L.status);
     L.count();
 }
 
 void bn_stats(const Launch& L, int vdtype, const void* v, const int* len_out, int B, int C, int Tp,
               float2* partials) {
     KScope ks_(L, KC_BN_STATS, (double)dtype_size(vdtype) * B * C * Tp, 0.0);
-    SC_DISPATCH(vdtype, (bn_stats_kernel<T><<<(B * C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>((const T*)v, len_out, B * C, C, Tp, partials)));
+    if (vdtype == F32) bn_stats_kernel<float><<<(B * C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>((const float*)v, len_out, B * C, C, Tp, partials);
+    else bn_stats_kernel<__half><<<(B * C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>((const __half*)v, len_out, B * C, C, Tp, partials);
     L.count();
 }
 
@@ -647,48 +796,65 @@ void bn_finalize(const Launch& L, const float2* partials, int parts_per_b, int t
                  const int* nvalid, int B, int C, float eps, float momentum, float* mean, float* invstd,
                  float* running_mean, float* running_var) {
     KScope ks_(L, KC_BN_FINALIZE, 8.0 * B * parts_per_b * C, 0.0);
-    bn_finalize_kernel<<<(C + kFinWarps - 1) / kFinWarps, 32 * kFinWarps, 0, L.stream>>>(partials, parts_per_b, tile_w, len_out, nvalid, B, C,
-                                                            eps, momentum, mean, invstd, running_mean, running_var);
+    bn_finalize_kernel<<<(C + 31) / 32, 32 * kFinWarps, 0, L.stream>>>(partials, parts_per_b, tile_w, len_out, nvalid, B, C,
+                                                                     eps, momentum, mean, invstd, running_mean, running_var);
+    L.count();
+}
+
+void bn_finalize_flat(const Launch& L, const float4* partials, int grid, int tiles_m, int rows_per_tile,
+                      const int* blk_off, const int* nvalid, int B, int C, float eps, float momentum, float* mean,
+                      float* invstd, float* running_mean, float* running_var) {
+    KScope ks_(L, KC_BN_FINALIZE, 16.0 * grid * C / std::max(1, tiles_m), 0.0);
+    bn_finalize_flat_kernel<<<(C + 31) / 32, 32 * kFinWarps, 0, L.stream>>>(partials, grid, tiles_m, rows_per_tile, blk_off, nvalid, B,
+                                                                          C, eps, momentum, mean, invstd, running_mean, running_var);
     L.count();
 }
 
 // the flattened kernels index with 32 bits
 static bool fits32(int B, int C, int Tp) { return (long long)B * C * (Tp / 8) < (1ll << 31) && (long long)B * C * Tp < (1ll << 31); }
+static unsigned fast_grid(long long total, int V) { return (unsigned)((total + 256ll * V - 1) / (256ll * V)); }
 
+// Algorithmic bytes per element of the batch-norm kernels: every tensor they must read or write, once.
 void bn_apply(const Launch& L, int dtype, const ApplyArgs& a_in) {
     ApplyArgs a = a_in;
-    KScope ks_(L, KC_BN_APPLY, (double)a.B * a.C * a.Tp * (dtype_size(vtype_of(dtype)) + dtype_size(dtype) + dtype_size(ntype_of(dtype)) + (a.residual == 1 ? dtype_size(dtype) : 0) + (a.residual == 2 ? dtype_size(vtype_of(dtype)) + dtype_size(ntype_of(dtype)) : 0)), 0.0);
-    if (a.Tp % 8 == 0 && a.has_relu && a.res_before_relu && fits32(a.B, a.C, a.Tp)) {
+    const double e = (double)dtype_size(dtype), en = (double)dtype_size(ntype_of(dtype));
+    KScope ks_(L, KC_BN_APPLY, (double)a.B * a.C * a.Tp * (en + e + (a.residual == 1 ? e : 0) + (a.residual == 2 ? en : 0)), 0.0);
+    if (dtype != F32 && a.Tp % 8 == 0 && a.has_relu && a.res_before_relu && fits32(a.B, a.C, a.Tp)) {
         const int vpr = a.Tp / 8;
         a.dvpr = FastDiv((uint32_t)vpr); a.dC = FastDiv((uint32_t)a.C);
         const long long total = (long long)a.B * a.C * vpr;
-        const unsigned grid = (unsigned)((total + 255) / 256);
-#define SC_APPLY_FAST(RES) SC_DISPATCH3(dtype, (bn_apply_fast_kernel<T, VT, NT, RES><<<grid, 256, 0, L.stream>>>(a, vpr, total)))
+        const unsigned grid = fast_grid(total, 2);
+#define SC_APPLY_FAST(RES) SC_DISPATCH16(dtype, (bn_apply_fast_kernel<T, NT, RES, 2><<<grid, 256, 0, L.stream>>>(a, vpr, total)))
         if (a.residual == 0) { SC_APPLY_FAST(0); } else if (a.residual == 1) { SC_APPLY_FAST(1); } else { SC_APPLY_FAST(2); }
 #undef SC_APPLY_FAST
         L.count();
         return;
     }
-    SC_DISPATCH3(dtype, (bn_apply_kernel<T, VT, NT><<<(a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>(a)));
+    SC_DISPATCH3(dtype, (bn_apply_kernel<T, NT><<<(a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>(a)));
     L.count();
 }
 
 void bn_bwd_reduce(const Launch& L, int dtype, BnBwdArgs& a) {
-    a.nslots = 1;
-    if (a.Tp % 8 == 0 && a.Tp >= 256 && a.has_bn && a.has_relu && a.res_before_relu && fits32(a.B, a.C, a.Tp)) {
+    a.nslots = 1; a.vpw = 32; a.vpw_shift = 5;
+    const double e = (double)dtype_size(dtype), en = (double)dtype_size(ntype_of(dtype));
+    if (dtype != F32 && a.Tp % 8 == 0 && a.Tp >= 256 && a.has_bn && a.has_relu && a.res_before_relu && fits32(a.B, a.C, a.Tp)) {
         a.dvpr = FastDiv((uint32_t)(a.Tp / 8)); a.dC = FastDiv((uint32_t)a.C);
-        KScope ks2_(L, KC_BN_BWD_REDUCE, (double)a.B * a.C * a.Tp * (dtype_size(dtype) * (a.residual == 0 ? 1 : 2) + dtype_size(ntype_of(dtype)) * (a.residual == 2 ? 2 : 1)), 0.0);
+        KScope ks2_(L, KC_BN_BWD_REDUCE, (double)a.B * a.C * a.Tp * (e * (a.residual == 0 ? 1 : 2) + en * (a.residual == 2 ? 2 : 1)), 0.0);
         const int vpr = a.Tp / 8;
+        const int V = vpr >= 64 ? 2 : 1;
+        a.vpw = 32 * V; a.vpw_shift = V == 2 ? 6 : 5;
         a.nslots = bn_bwd_max_slots(a.Tp);
         const long long total = (long long)a.B * a.C * vpr;
-        const unsigned grid = (unsigned)((total + 255) / 256);
-        if (a.residual == 2) { SC_DISPATCH3(dtype, (bn_bwd_reduce_fast_kernel<T, NT, 2><<<grid, 256, 0, L.stream>>>(a, vpr, total))); }
-        else if (a.residual == 1) { SC_DISPATCH3(dtype, (bn_bwd_reduce_fast_kernel<T, NT, 1><<<grid, 256, 0, L.stream>>>(a, vpr, total))); }
-        else { SC_DISPATCH3(dtype, (bn_bwd_reduce_fast_kernel<T, NT, 0><<<grid, 256, 0, L.stream>>>(a, vpr, total))); }
+        const unsigned grid = fast_grid(total, V);
+#define SC_RED_FAST(RES)                                                                                                   \
+        if (V == 2) { SC_DISPATCH16(dtype, (bn_bwd_reduce_fast_kernel<T, NT, RES, 2><<<grid, 256, 0, L.stream>>>(a, vpr, total))); } \
+        else { SC_DISPATCH16(dtype, (bn_bwd_reduce_fast_kernel<T, NT, RES, 1><<<grid, 256, 0, L.stream>>>(a, vpr, total))); }
+        if (a.residual == 2) { SC_RED_FAST(2); } else if (a.residual == 1) { SC_RED_FAST(1); } else { SC_RED_FAST(0); }
+#undef SC_RED_FAST
         L.count();
         return;
     }
-    KScope ks_(L, KC_BN_BWD_REDUCE, (double)a.B * a.C * a.Tp * (dtype_size(dtype) * (a.has_relu && a.res_before_relu ? 2 : 1) + (a.has_bn ? dtype_size(ntype_of(dtype)) : 0) + (a.residual == 2 ? dtype_size(ntype_of(dtype)) : 0)), 0.0);
+    KScope ks_(L, KC_BN_BWD_REDUCE, (double)a.B * a.C * a.Tp * (e * (a.has_relu && a.res_before_relu ? 2 : 1) + (a.has_bn ? en : 0) + (a.residual == 2 ? en : 0)), 0.0);
     SC_DISPATCH3(dtype, (bn_bwd_reduce_kernel<T, NT><<<(a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>(a)));
     L.count();
 }
@@ -696,26 +862,26 @@ void bn_bwd_reduce(const Launch& L, int dtype, BnBwdArgs& a) {
 void bn_bwd_finalize(const Launch& L, const BnBwdArgs& a, const float* gamma, const float* gamma_r,
                      float* dgamma, float* dbeta, float* dgamma_r, float* dbeta_r, float* dbias,
                      int accumulate) {
-    KScope ks_(L, KC_BN_BWD_FINALIZE, 16.0 * a.B * a.C, 0.0);
-    bn_bwd_finalize_kernel<<<(a.C + kFinWarps - 1) / kFinWarps, 32 * kFinWarps, 0, L.stream>>>(a, gamma, gamma_r, dgamma, dbeta, dgamma_r,
-                                                                  dbeta_r, dbias, accumulate);
+    KScope ks_(L, KC_BN_BWD_FINALIZE, 16.0 * a.B * a.C * a.nslots, 0.0);
+    bn_bwd_finalize_kernel<<<(a.C + 31) / 32, 32 * kFinWarps, 0, L.stream>>>(a, gamma, gamma_r, dgamma, dbeta, dgamma_r,
+                                                                          dbeta_r, dbias, accumulate);
     L.count();
 }
 
 void bn_bwd_apply(const Launch& L, int dtype, const BnBwdArgs& a_in) {
     BnBwdArgs a = a_in;
-    const bool fast_apply = a.Tp % 8 == 0 && a.has_bn && a.has_relu && a.res_before_relu && fits32(a.B, a.C, a.Tp);
-    KScope ks_(L, KC_BN_BWD_APPLY, (double)a.B * a.C * a.Tp * (dtype_size(dtype) * (a.has_relu && a.res_before_relu && !(fast_apply && a.residual == 0) ? 2 : 1) + (a.has_bn ? dtype_size(ntype_of(dtype)) : 0) + (a.residual == 2 ? dtype_size(ntype_of(dtype)) : 0) + dtype_size(dtype) * (1 + (a.residual != 0 ? 1 : 0))), 0.0);
+    const bool fast_apply = dtype != F32 && a.Tp % 8 == 0 && a.has_bn && a.has_relu && a.res_before_relu && fits32(a.B, a.C, a.Tp);
+    const double e = (double)dtype_size(dtype), en = (double)dtype_size(ntype_of(dtype));
+    KScope ks_(L, KC_BN_BWD_APPLY, (double)a.B * a.C * a.Tp * (e * (a.has_relu && a.res_before_relu && !(fast_apply && a.residual == 0) ? 2 : 1) + (a.has_bn ? en : 0) + (a.residual == 2 ? en : 0) + (double)dtype_size(a.gv_dtype) + (a.residual != 0 ? e : 0)), 0.0);
     if (fast_apply) {
         const int vpr = a.Tp / 8;
         a.dvpr = FastDiv((uint32_t)vpr); a.dC = FastDiv((uint32_t)a.C);
         const long long total = (long long)a.B * a.C * vpr;
-        const unsigned grid = (unsigned)((total + 255) / 256);
-#define SC_BWD_FAST(RES)                                                                                          \
-        if (dtype == BF16 && a.gv_dtype == F16)                                                                   \
-            bn_bwd_apply_fast_kernel<__nv_bfloat16, __half, __half, RES><<<grid, 256, 0, L.stream>>>(a, vpr, total); \
-        else                                                                                                      \
-            SC_DISPATCH3(dtype, (bn_bwd_apply_fast_kernel<T, NT, T, RES><<<grid, 256, 0, L.stream>>>(a, vpr, total)))
+        const unsigned grid = fast_grid(total, 2);
+#define SC_BWD_FAST(RES)                                                                                             \
+        if (dtype == BF16 && a.gv_dtype == F16)                                                                      \
+            bn_bwd_apply_fast_kernel<__nv_bfloat16, __half, __half, RES, 2><<<grid, 256, 0, L.stream>>>(a, vpr, total); \
+        else { SC_DISPATCH16(dtype, (bn_bwd_apply_fast_kernel<T, NT, T, RES, 2><<<grid, 256, 0, L.stream>>>(a, vpr, total))); }
         if (a.residual == 0) { SC_BWD_FAST(0); } else if (a.residual == 1) { SC_BWD_FAST(1); } else { SC_BWD_FAST(2); }
 #undef SC_BWD_FAST
         L.count();

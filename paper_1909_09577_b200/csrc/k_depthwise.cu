@@ -154,10 +154,10 @@ template <typename T, typename TO>
 __global__ void __launch_bounds__(GT)
 dw_fwd_generic_kernel(const T* __restrict__ x, const T* __restrict__ w, TO* __restrict__ u,
                       const int* __restrict__ len_in, const int* __restrict__ len_out,
-                      int C, int Tt, int Tp, int K, int s, int* status) {
+                      int C, int Tt, int Tp, int K, int s, int dil, int* status) {
     extern __shared__ float smem[];
     const int b = blockIdx.z, c = blockIdx.y, t0 = blockIdx.x * GT;
-    const int P = (K - 1) / 2, XW = (GT - 1) * s + K;
+    const int P = (dil * (K - 1)) / 2, XW = (GT - 1) * s + (K - 1) * dil + 1;
     float* xs = smem;
     float* ws = smem + XW;
     const int li = min(len_in[b], Tt), lo = min(len_out[b], Tp);
@@ -172,7 +172,7 @@ dw_fwd_generic_kernel(const T* __restrict__ x, const T* __restrict__ w, TO* __re
     const int t = t0 + threadIdx.x;
     if (t >= Tp) return;
     float acc = 0.f;
-    for (int k = 0; k < K; ++k) acc = fmaf(ws[k], xs[threadIdx.x * s + k], acc);
+    for (int k = 0; k < K; ++k) acc = fmaf(ws[k], xs[threadIdx.x * s + k * dil], acc);
     if (std::is_same<TO, __half>::value && fabsf(acc) > 65504.f) { acc = copysignf(65504.f, acc); raise_status(status, kErrRange); }
     stf(u + ((size_t)b * C + c) * Tp + t, (t < lo) ? acc : 0.f);
 }
@@ -182,12 +182,12 @@ __global__ void __launch_bounds__(GT)
 dw_dgrad_generic_kernel(const TG* __restrict__ gu, const T* __restrict__ w, T* __restrict__ dx,
                         const T* __restrict__ add1, const T* __restrict__ add2, const float* __restrict__ gmax,
                         const int* __restrict__ len_in, const int* __restrict__ len_out,
-                        int C, int Tt, int Tp, int K, int s) {
+                        int C, int Tt, int Tp, int K, int s, int dil) {
     extern __shared__ float smem[];
     const int b = blockIdx.z, c = blockIdx.y, tau0 = blockIdx.x * GT;
-    const int P = (K - 1) / 2;
+    const int P = (dil * (K - 1)) / 2;
     // outputs tau0..tau0+GT-1 read gu[t] for t in [tlo, thi]
-    const int num = tau0 + P - (K - 1);
+    const int num = tau0 + P - (K - 1) * dil;
     const int tlo = (num >= 0) ? (num + s - 1) / s : -((-num) / s);
     const int thi = (tau0 + GT - 1 + P) / s;
     const int GW = thi - tlo + 1;
@@ -205,7 +205,7 @@ dw_dgrad_generic_kernel(const TG* __restrict__ gu, const T* __restrict__ w, T* _
     if (tau >= Tt) return;
     float acc = 0.f;
     for (int k = 0; k < K; ++k) {
-        const int q = tau + P - k;
+        const int q = tau + P - k * dil;
         if (q >= 0 && q % s == 0) { const int t = q / s; if (t >= tlo && t <= thi) acc = fmaf(ws[k], gs[t - tlo], acc); }
     }
     const size_t o = ((size_t)b * C + c) * Tt + tau;
@@ -220,9 +220,9 @@ template <typename TG, typename T>
 __global__ void __launch_bounds__(128)
 dw_wgrad_generic_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float* __restrict__ partials,
                         const int* __restrict__ len_in, const int* __restrict__ len_out,
-                        int B, int C, int Tt, int Tp, int K, int s) {
+                        int B, int C, int Tt, int Tp, int K, int s, int dil) {
     const int c = blockIdx.x, lane = threadIdx.x & 31, wrp = threadIdx.x >> 5;
-    const int P = (K - 1) / 2;
+    const int P = (dil * (K - 1)) / 2;
     // partials[b][c][k]; warps stride over samples
     for (int b = wrp; b < B; b += 4) {
         const int li = min(len_in[b], Tt), lo = min(len_out[b], Tp);
@@ -231,7 +231,7 @@ dw_wgrad_generic_kernel(const TG* __restrict__ gu, const T* __restrict__ x, floa
         for (int k = 0; k < K; ++k) {
             float acc = 0.f;
             for (int t = lane; t < lo; t += 32) {
-                const int tau = t * s + k - P;
+                const int tau = t * s + k * dil - P;
                 if (tau >= 0 && tau < li) acc = fmaf(ldf(grow + t), ldf(xrow + tau), acc);
             }
             acc = warp_sum(acc);
@@ -645,13 +645,14 @@ inline int host_phys(int i) { return i + ((i >> 5) << 2); }
     else { using T = __nv_bfloat16; using OT = __nv_bfloat16; __VA_ARGS__; }
 
 void dw_fwd(const Launch& L, int dtype, int odt, const void* x, const void* wd, void* u, const int* len_in,
-            const int* len_out, int B, int C, int Tt, int Tp, int K, int s) {
+            const int* len_out, int B, int C, int Tt, int Tp, int K, int s, int dil) {
     KScope ks_(L, KC_DW_FWD, (double)B * C * (dtype_size(dtype) * Tt + dtype_size(odt) * Tp), 2.0 * B * C * Tp * K);
-    if (!L.simt_only && dw_tc_supported(dtype, Tt, K, s)) {
+    const bool plain = dil == 1 && (K & 1);      // odd K, adjacent taps: the forms the specialised kernels are written for
+    if (!L.simt_only && plain && dw_tc_supported(dtype, Tt, K, s)) {
         dw_tc_fwd(L, dtype, odt, x, wd, u, len_in, len_out, B, C, Tt, K);
         return;
     }
-    if (s == 1) {
+    if (s == 1 && plain) {
         const int Kp = kpad(K);
         const size_t smem = (size_t)CH * (host_phys(TT + Kp) + 4 + Kp) * sizeof(float);
         dim3 grid((Tt + TT - 1) / TT, (C + CH - 1) / CH, B), block(32, CH);
@@ -659,24 +660,25 @@ void dw_fwd(const Launch& L, int dtype, int odt, const void* x, const void* wd, 
                                        (const T*)x, (const T*)wd, (OT*)u, nullptr, nullptr, nullptr, len_in, len_out, C, Tt,
                                        K, Kp, 0, L.status)));
     } else {
-        const size_t smem = (size_t)((GT - 1) * s + K + K) * sizeof(float);
+        const size_t smem = (size_t)((GT - 1) * s + (K - 1) * dil + 1 + K) * sizeof(float);
         dim3 grid((Tp + GT - 1) / GT, C, B);
         SC_DISPATCH_IO(dtype, odt, (dw_fwd_generic_kernel<T, OT><<<grid, GT, smem, L.stream>>>(
-                                       (const T*)x, (const T*)wd, (OT*)u, len_in, len_out, C, Tt, Tp, K, s, L.status)));
+                                       (const T*)x, (const T*)wd, (OT*)u, len_in, len_out, C, Tt, Tp, K, s, dil, L.status)));
     }
     L.count();
 }
 
 void dw_dgrad(const Launch& L, int dtype, int odt, const void* gu, const void* wd, void* dx, const void* add1,
               const void* add2, const float* gmax, const int* len_in, const int* len_out, int B, int C, int Tt,
-              int Tp, int K, int s) {
+              int Tp, int K, int s, int dil) {
+    const bool plain = dil == 1 && (K & 1);
     KScope ks_(L, KC_DW_DGRAD, (double)B * C * (dtype_size(dtype) * Tt * (1 + (add1 ? 1 : 0) + (add2 ? 1 : 0)) + dtype_size(odt) * Tp),
                2.0 * B * C * Tp * K);
-    if (!L.simt_only && dw_tc_supported(dtype, Tt, K, s)) {
+    if (!L.simt_only && plain && dw_tc_supported(dtype, Tt, K, s)) {
         dw_tc_dgrad(L, dtype, odt, gu, wd, dx, add1, add2, gmax, len_in, len_out, B, C, Tt, K);
         return;
     }
-    if (s == 1) {
+    if (s == 1 && plain) {
         const int Kp = kpad(K);
         const size_t smem = (size_t)CH * (host_phys(TT + Kp) + 4 + Kp) * sizeof(float);
         dim3 grid((Tt + TT - 1) / TT, (C + CH - 1) / CH, B), block(32, CH);
@@ -684,11 +686,11 @@ void dw_dgrad(const Launch& L, int dtype, int odt, const void* gu, const void* w
                                        (const OT*)gu, (const T*)wd, (T*)dx, (const T*)add1, (const T*)add2, gmax, len_out,
                                        len_in, C, Tt, K, Kp, 1, L.status)));
     } else {
-        const size_t smem = (size_t)((GT + K) / s + 4 + K) * sizeof(float);
+        const size_t smem = (size_t)((GT + (K - 1) * dil + 1) / s + 4 + K) * sizeof(float);
         dim3 grid((Tt + GT - 1) / GT, C, B);
         SC_DISPATCH_IO(dtype, odt, (dw_dgrad_generic_kernel<OT, T><<<grid, GT, smem, L.stream>>>(
                                        (const OT*)gu, (const T*)wd, (T*)dx, (const T*)add1, (const T*)add2, gmax, len_in,
-                                       len_out, C, Tt, Tp, K, s)));
+                                       len_out, C, Tt, Tp, K, s, dil)));
     }
     L.count();
 }
@@ -697,13 +699,17 @@ size_t dw_wgrad_scratch_bytes(int B, int C, int K) { return (size_t)B * C * K * 
 
 void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x, float* dwd, float* partials,
               int accumulate, const float* gmax, const int* len_in, const int* len_out, int B, int C, int Tt,
-              int Tp, int K, int s) {
+              int Tp, int K, int s, int dil) {
+    const bool plain = dil == 1 && (K & 1);
     int nsplit;
     {
     KScope ks_(L, KC_DW_WGRAD, (double)B * C * (dtype_size(dtype) * Tt + dtype_size(odt) * Tp), 2.0 * B * C * Tp * K);
     const int P = (K - 1) / 2, Ppad = (P + 3) / 4 * 4;
     const int nch = (K + (Ppad - P) + 7) / 8;
-    if (s == 1 && Tt % 8 == 0 && nch >= 2 && nch <= 12) {
+    // the register kernels stage whole rows: one row (double-buffered) must fit their shared-memory limit
+    const bool reg_fits = (dtype == F32) ? (size_t)2 * ((host_phys(Tt + 8 * nch + 8) + 4 + 3) / 4 * 4) * sizeof(float) <= 64 * 1024
+                                         : (size_t)2 * 2 * ((Tt + 8 * nch + 8 + 7) / 8 * 8) * 2 <= 96 * 1024;
+    if (plain && s == 1 && Tt % 8 == 0 && nch >= 2 && nch <= 12 && reg_fits) {
         // rows staged per pass: the count whose (rows x chunks) best fills the 128 threads
         const int cpr = Tt / 8;
         const int NST = (dtype == F32) ? 2 : 4;
@@ -722,8 +728,7 @@ void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x
 #define SC_WR_CASE(N)                                                                                          \
             case N: {                                                                                          \
                 auto kern = dw_wgrad_reg_kernel<float, float, N>;                                              \
-                static bool cfg_done = false;                                                                  \
-                if (!cfg_done) { cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024); cfg_done = true; } \
+                set_max_smem_once<dw_wgrad_reg_kernel<float, float, N>>(64 * 1024);                            \
                 kern<<<grid, WR_THREADS, smem, L.stream>>>((const float*)gu, (const float*)x, partials, len_in, len_out, \
                                                            B, C, Tt, K, Ppad, NR, NST, rsp);                   \
             } break;
@@ -748,20 +753,17 @@ void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x
             case N: {                                                                                          \
                 if (dtype == F16) {                                                                            \
                     auto kern = dw_wgrad_reg16_kernel<__half, __half, N>;                                      \
-                    static bool cfg_done = false;                                                              \
-                    if (!cfg_done) { cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024); cfg_done = true; } \
+                    set_max_smem_once<dw_wgrad_reg16_kernel<__half, __half, N>>(96 * 1024);   \
                     kern<<<grid, WR_THREADS, smem, L.stream>>>((const __half*)gu, (const __half*)x, partials, len_in, len_out, \
                                                                B, C, Tt, K, Ppad, NR, NST, RS);               \
                 } else if (odt == F16) {                                                                       \
                     auto kern = dw_wgrad_reg16_kernel<__half, __nv_bfloat16, N>;                               \
-                    static bool cfg_done = false;                                                              \
-                    if (!cfg_done) { cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024); cfg_done = true; } \
+                    set_max_smem_once<dw_wgrad_reg16_kernel<__half, __nv_bfloat16, N>>(96 * 1024);   \
                     kern<<<grid, WR_THREADS, smem, L.stream>>>((const __half*)gu, (const __nv_bfloat16*)x, partials, len_in, len_out, \
                                                                B, C, Tt, K, Ppad, NR, NST, RS);               \
                 } else {                                                                                       \
                     auto kern = dw_wgrad_reg16_kernel<__nv_bfloat16, __nv_bfloat16, N>;                        \
-                    static bool cfg_done = false;                                                              \
-                    if (!cfg_done) { cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024); cfg_done = true; } \
+                    set_max_smem_once<dw_wgrad_reg16_kernel<__nv_bfloat16, __nv_bfloat16, N>>(96 * 1024);   \
                     kern<<<grid, WR_THREADS, smem, L.stream>>>((const __nv_bfloat16*)gu, (const __nv_bfloat16*)x, partials, len_in, len_out, \
                                                                B, C, Tt, K, Ppad, NR, NST, RS);               \
                 }                                                                                              \
@@ -772,7 +774,7 @@ void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x
             }
 #undef SC_WR_CASE
         }
-    } else if (s == 1) {
+    } else if (plain && s == 1) {
         const int Kp = kpad(K), NG = Kp / R, nseg = WG_THREADS / NG;
         const int seglen = ((WG_TT + nseg - 1) / nseg + R - 1) / R * R;
         const int GW = nseg * seglen;
@@ -781,7 +783,7 @@ void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x
         dim3 grid(C, nsplit);
         SC_DISPATCH_IO(dtype, odt, (dw_wgrad_s1_kernel<OT, T><<<grid, WG_THREADS, smem, L.stream>>>(
                                        (const OT*)gu, (const T*)x, partials, len_in, len_out, B, C, Tt, K, Kp)));
-    } else if (K <= 128) {
+    } else if (plain && K <= 128) {
         nsplit = B;
         const size_t smem = (size_t)(WS_TT + (WS_TT - 1) * s + K + 128) * sizeof(float);
         dim3 grid(C, B);
@@ -790,7 +792,7 @@ void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x
     } else {
         nsplit = B;
         SC_DISPATCH_IO(dtype, odt, (dw_wgrad_generic_kernel<OT, T><<<C, 128, 0, L.stream>>>(
-                                       (const OT*)gu, (const T*)x, partials, len_in, len_out, B, C, Tt, Tp, K, s)));
+                                       (const OT*)gu, (const T*)x, partials, len_in, len_out, B, C, Tt, Tp, K, s, dil)));
     }
     L.count();
     }

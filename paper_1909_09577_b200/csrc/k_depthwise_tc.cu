@@ -223,8 +223,7 @@ template <typename TI, typename TW, typename TO, bool FLIP>
 void launch_tc(const Launch& L, const void* in, const void* w, void* out, const void* add1, const void* add2,
                const float* gmax, const int* len_src, const int* len_dst, int B, int C, int Tt, int K) {
     auto kern = dw_tc_kernel<TI, TW, TO, FLIP>;
-    static bool configured = false;
-    if (!configured) { cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes); configured = true; }
+    set_max_smem_once<dw_tc_kernel<TI, TW, TO, FLIP>>((int)kSmemBytes);
     const int S = (Tt + NB - 1) / NB + 2;
     const int nb = std::max(1, std::min(B, MAXROWS / S));
     dim3 grid(C, (B + nb - 1) / nb);

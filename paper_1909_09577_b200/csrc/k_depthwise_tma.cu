@@ -423,11 +423,7 @@ static_assert(kDtSmem <= 232448, "shared memory per CTA");
 template <typename TI, typename TW, typename TO>
 void launch_dt(const Launch& L, int grid, const CUtensorMap& mx, const CUtensorMap& mo, const DtParams& p) {
     auto kern = dw_tma_kernel<TI, TW, TO>;
-    static bool configured = false;
-    if (!configured) {
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kDtSmem);
-        configured = true;
-    }
+    set_max_smem_once<dw_tma_kernel<TI, TW, TO>>(kDtSmem);
     kern<<<grid, DT_THREADS, kDtSmem, L.stream>>>(mx, mo, p);
     L.count();
 }

@@ -360,11 +360,7 @@ static_assert((3 * WT_STAGES + 4) * 8 + 8 + WT_MAX_CHUNKS * 4 <= 512, "barrier b
 template <typename TG, typename TX>
 void launch_wt(const Launch& L, int grid, const CUtensorMap& mg, const CUtensorMap& mx, const WtParams& p) {
     auto kern = dw_wgrad_tc_kernel<TG, TX>;
-    static bool configured = false;
-    if (!configured) {
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kWtSmem);
-        configured = true;
-    }
+    set_max_smem_once<dw_wgrad_tc_kernel<TG, TX>>(kWtSmem);
     kern<<<grid, WT_THREADS, kWtSmem, L.stream>>>(mg, mx, p);
     L.count();
 }

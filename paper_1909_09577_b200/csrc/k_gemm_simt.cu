@@ -20,10 +20,13 @@ struct GemmDesc {
     int k_begin_per_z, k_len_per_z;   // split-K: slice z covers k in [z*k_len, (z+1)*k_len)
 };
 
+template <typename X> struct IsHalf { static constexpr bool value = false; };
+template <> struct IsHalf<__half> { static constexpr bool value = true; };
+
 template <typename T, typename OT, int MODE>   // MODE 0: fwd (bias+mask, T out) 1: dgrad (T out) 2: wgrad (float partial out)
 __global__ void __launch_bounds__(NT)
 gemm_simt_kernel(GemmDesc d, const T* __restrict__ a, const T* __restrict__ b, void* __restrict__ out,
-                 const float* __restrict__ bias, const int* __restrict__ len_out) {
+                 const float* __restrict__ bias, const int* __restrict__ len_out, int* status) {
     __shared__ float As[BK][BM + 4];
     __shared__ float Bs[BK][BN + 4];
     const int z = blockIdx.z;
@@ -101,6 +104,7 @@ gemm_simt_kernel(GemmDesc d, const T* __restrict__ a, const T* __restrict__ b, v
             if (MODE == 0) {
                 float v = acc[i][j] + (bias ? bias[m] : 0.f);
                 if (len_out && n >= len_out[z]) v = 0.f;
+                if (sizeof(OT) == 2 && fabsf(v) > 65504.f && IsHalf<OT>::value) { v = copysignf(65504.f, v); raise_status(status, kErrRange); }
                 stf((OT*)out + ((long long)z * d.M + m) * d.N + n, v);
             } else if (MODE == 1) {
                 stf((OT*)out + ((long long)z * d.M + m) * d.N + n, acc[i][j]);
@@ -175,11 +179,13 @@ void gemm_fwd_simt(const Launch& L, int dtype, const void* w, const void* u, con
     d.b_z = (long long)Cin * Tp; d.b_k = Tp; d.b_n = 1;
     dim3 grid((Tp + BN - 1) / BN, (Cout + BM - 1) / BM, B);
     if (out_dtype == dtype) {
-        SC_DISPATCH(dtype, (gemm_simt_kernel<T, T, 0><<<grid, NT, 0, L.stream>>>(d, (const T*)w, (const T*)u, v, bias, len_out)));
+        SC_DISPATCH(dtype, (gemm_simt_kernel<T, T, 0><<<grid, NT, 0, L.stream>>>(d, (const T*)w, (const T*)u, v, bias, len_out, L.status)));
+    } else if (dtype == BF16 && out_dtype == F16) {   // bfloat16 operands, float16 result
+        gemm_simt_kernel<__nv_bfloat16, __half, 0><<<grid, NT, 0, L.stream>>>(d, (const __nv_bfloat16*)w, (const __nv_bfloat16*)u, v, bias, len_out, L.status);
     } else if (dtype == BF16) {   // 16-bit operands, float result
-        gemm_simt_kernel<__nv_bfloat16, float, 0><<<grid, NT, 0, L.stream>>>(d, (const __nv_bfloat16*)w, (const __nv_bfloat16*)u, v, bias, len_out);
+        gemm_simt_kernel<__nv_bfloat16, float, 0><<<grid, NT, 0, L.stream>>>(d, (const __nv_bfloat16*)w, (const __nv_bfloat16*)u, v, bias, len_out, L.status);
     } else {
-        gemm_simt_kernel<__half, float, 0><<<grid, NT, 0, L.stream>>>(d, (const __half*)w, (const __half*)u, v, bias, len_out);
+        gemm_simt_kernel<__half, float, 0><<<grid, NT, 0, L.stream>>>(d, (const __half*)w, (const __half*)u, v, bias, len_out, L.status);
     }
     L.count();
 }
@@ -192,7 +198,7 @@ void gemm_dgrad_simt(const Launch& L, int dtype, const void* w, const void* gv, 
     d.a_z = 0; d.a_m = 1; d.a_k = Cin;            // A(m=c, k=o) = w[o*Cin + c]
     d.b_z = (long long)Cout * Tp; d.b_k = Tp; d.b_n = 1;
     dim3 grid((Tp + BN - 1) / BN, (Cin + BM - 1) / BM, B);
-    SC_DISPATCH(dtype, (gemm_simt_kernel<T, T, 1><<<grid, NT, 0, L.stream>>>(d, (const T*)w, (const T*)gv, gu, nullptr, nullptr)));
+    SC_DISPATCH(dtype, (gemm_simt_kernel<T, T, 1><<<grid, NT, 0, L.stream>>>(d, (const T*)w, (const T*)gv, gu, nullptr, nullptr, nullptr)));
     L.count();
 }
 
@@ -214,7 +220,7 @@ void gemm_wgrad_simt(const Launch& L, int dtype, const void* gv, const void* u, 
     d.b_n = Tp; d.b_kz = (long long)Cin * Tp;     // B(k=(b,t), n=c) = u[b,c,t]
     d.k_len_per_z = Tp;
     dim3 grid((Cin + BN - 1) / BN, (Cout + BM - 1) / BM, ns);
-    SC_DISPATCH(dtype, (gemm_simt_kernel<T, T, 2><<<grid, NT, 0, L.stream>>>(d, (const T*)gv, (const T*)u, partials, nullptr, nullptr)));
+    SC_DISPATCH(dtype, (gemm_simt_kernel<T, T, 2><<<grid, NT, 0, L.stream>>>(d, (const T*)gv, (const T*)u, partials, nullptr, nullptr, nullptr)));
     L.count();
     }
     reduce_partials(L, partials, ns, (int64_t)Cin * Cout, dw, accumulate, gmax);

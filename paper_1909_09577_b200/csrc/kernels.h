@@ -48,25 +48,50 @@ struct KScope {
     ~KScope() { if (slot >= 0) cudaEventRecord(L.prof->events[slot + 1], L.stream); }
 };
 
+// Device the context was created on (-1 for a null context).
+}  // namespace sc
+struct sc_ctx;
+namespace sc {
+int ctx_device(const sc_ctx* ctx);
+
+// Launches one CTA that waits, with a short poll limit, on an mbarrier that nothing ever signals: the wait
+// must run out, raise the timeout status and return (exercises the bounded-wait exit of the kernels).
+void selftest_bounded_wait(const Launch& L);
+
+// cudaFuncAttributeMaxDynamicSharedMemorySize is a per-device property of a kernel: set it once per
+// (kernel, device), keyed by the current device.
+template <auto Kern> inline void set_max_smem_once(int smem) {
+    static unsigned long long done = 0;      // one bit per device ordinal
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && ((done >> dev) & 1ull)) return;
+    cudaFuncSetAttribute(Kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (dev >= 0 && dev < 64) done |= 1ull << dev;
+}
+
 // ---- lengths -------------------------------------------------------------------------------
 // len_out[b] = ceil(len_in[b]/stride); *nvalid = sum_b len_out[b]; flags lengths outside [1,T_in].
-void lengths(const Launch& L, const int* len_in, int B, int T_in, int stride, int* len_out, int* nvalid);
+// blk_off (nullable, int [B+1]): exclusive prefix sum of ceil(len_out[b] / 64), the number of 64-frame blocks
+// of each sample that hold at least one valid frame; blk_off[B] is their total.
+void lengths(const Launch& L, const int* len_in, int B, int T_in, int stride, int* len_out, int* nvalid,
+             int* blk_off = nullptr);
 
 // ---- depthwise ------------------------------------------------------------------------------
-// u[b,c,t] = sum_k wd[c,k] * x[b,c,t*s+k-P] (x masked by len_in), written as 0 for t >= len_out[b].
+// u[b,c,t] = sum_k wd[c,k] * x[b,c,t*s+k*dil-P] (x masked by len_in), written as 0 for t >= len_out[b];
+// P = (dil*(K-1))/2 zeros on the left ("same" padding; any K >= 1, dil >= 1).
 // x and wd in `dtype`, u in `odt` (values beyond the half range are clamped and flagged).
 void dw_fwd(const Launch& L, int dtype, int odt, const void* x, const void* wd, void* u, const int* len_in,
-            const int* len_out, int B, int C, int T, int Tp, int K, int s);
+            const int* len_out, int B, int C, int T, int Tp, int K, int s, int dil = 1);
 // dx[b,c,tau] = [tau < len_in[b]] * (sum_{k,t: t*s+k-P=tau} wd[c,k]*gu[b,c,t] + add1 + add2)
 // gu in `odt` and pre-multiplied by pow2_scale(*gmax) when gmax is non-null; wd, add1, add2, dx in `dtype`.
 void dw_dgrad(const Launch& L, int dtype, int odt, const void* gu, const void* wd, void* dx, const void* add1,
               const void* add2, const float* gmax, const int* len_in, const int* len_out, int B, int C, int T,
-              int Tp, int K, int s);
+              int Tp, int K, int s, int dil = 1);
 // dwd[c,k] (+)= sum_{b,t<len_out} gu[b,c,t] * x[b,c,t*s+k-P] (x masked by len_in).
 // partials: float [B*C*K] scratch.
 void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x, float* dwd, float* partials,
               int accumulate, const float* gmax, const int* len_in, const int* len_out, int B, int C, int T,
-              int Tp, int K, int s);
+              int Tp, int K, int s, int dil = 1);
 size_t dw_wgrad_scratch_bytes(int B, int C, int K);
 // Tensor-core form of the stride-1 tap gradient (16-bit types, B >= 16, K <= 127): same result as dw_wgrad.
 // x_clean != 0 promises that x is already zero at and beyond len_in.  partials: float [8*C*K] at least.
@@ -97,6 +122,7 @@ void ew_add_masked(const Launch& L, int dtype, void* out, const void* a, const v
 
 // ---- pointwise, SIMT (any shape, fp32 accumulate) ------------------------------------------
 // v[b,o,t] = [t<len_out[b]] * (sum_c w[o,c]*u[b,c,t] + bias[o]); v is stored in out_dtype
+// (a float16 result beyond the half range is clamped and flagged)
 void gemm_fwd_simt(const Launch& L, int dtype, const void* w, const void* u, const float* bias, void* v,
                    int out_dtype, const int* len_out, int B, int Cin, int Cout, int Tp);
 // gu[b,c,t] = sum_o w[o,c]*gv[b,o,t]
@@ -125,11 +151,19 @@ void bn_finalize(const Launch& L, const float2* partials, int parts_per_b, int t
                  const int* nvalid, int B, int C, float eps, float momentum, float* mean, float* invstd,
                  float* running_mean, float* running_var);
 
-// Storage types.  T = activation type.  VT = type of the transient pre-normalisation tensor v
-// (float for fp32 and bf16 activations, half for fp16).  NT = type of the saved normalised tensor
-// vhat = (v - mean) * invstd (float for fp32, half otherwise: vhat has unit scale, so half's 10-bit
-// mantissa is safe where bf16's 8 bits would eat most of the error budget).
-inline int vtype_of(int dtype) { return dtype == 1 ? 1 : 0; }
+// The same merge for the per-(CTA, channel) float4 (count, sum, M2, -) partials of the flattened-block
+// contraction: `grid` CTAs, tiles_m M tiles of rows_per_tile channels, CTA c took the unit range
+// [c U / grid, (c+1) U / grid) with U = tiles_m * blk_off[B] (M tile major).
+void bn_finalize_flat(const Launch& L, const float4* partials, int grid, int tiles_m, int rows_per_tile,
+                      const int* blk_off, const int* nvalid, int B, int C, float eps, float momentum, float* mean,
+                      float* invstd, float* running_mean, float* running_var);
+
+// Storage types.  T = activation type.  NT = type of the pointwise result v, which the contraction's
+// epilogue writes once and which is kept for the backward pass: float for fp32 activations, half for
+// both 16-bit activation types (11 significand bits; bf16's 8 bits on v alone would use most of the
+// error budget).  The normalised value vhat = (v - mean) * invstd is never stored: the forward apply
+// step and the backward kernels recompute it from v with the same two float operations, so the ReLU
+// decision derived from it is the same bit on both sides.
 inline int ntype_of(int dtype) { return dtype == 0 ? 0 : 1; }
 inline size_t dtype_size(int dtype) { return dtype == 0 ? 4 : 2; }
 // OT = type of the tensors that only the library sees between the depthwise and pointwise steps
@@ -160,12 +194,10 @@ struct FastDiv {
 };
 
 struct ApplyArgs {
-    const void* v; const float *mean, *invstd, *gamma, *beta;          // main branch (v in VT)
-    void* vhat;                                                        // out, NT
+    const void* v; const float *mean, *invstd, *gamma, *beta;          // main branch (v in NT)
     int residual;                                  // 0 none, 1 identity, 2 projection
     const void* xres;                              // identity source [B,C,Tp], T
-    const void* vr; const float *mean_r, *invstd_r, *gamma_r, *beta_r; // projection branch (vr in VT)
-    void* vhat_r;                                                      // out, NT
+    const void* vr; const float *mean_r, *invstd_r, *gamma_r, *beta_r; // projection branch (vr in NT)
     void* y; const int* len_out;
     int B, C, Tp, has_relu, res_before_relu;
     FastDiv dvpr, dC;                              // by Tp / 8 and by C (set by bn_apply)
@@ -173,7 +205,8 @@ struct ApplyArgs {
 void bn_apply(const Launch& L, int dtype, const ApplyArgs& a);
 
 struct BnBwdArgs {
-    const void* g; const void* y; const void* vhat; const void* vhat_r;   // vhat, vhat_r in NT
+    const void* g; const void* y; const void* v; const void* vr;          // v, vr in NT
+    const float* mean; const float* mean_r;
     const float* invstd; const float* invstd_r;
     const float *gamma, *beta;                     // for the relu-then-add gate
     const int* len_out; const int* nvalid;
@@ -181,6 +214,7 @@ struct BnBwdArgs {
     float4* partials;                              // [B*C*nslots]
     float* amax_part;                              // [B*C*nslots] max |gated gradient| (only with gmax)
     int nslots;                                    // partial slots per (sample, channel) row; set by bn_bwd_reduce
+    int vpw, vpw_shift;                            // 8-frame vectors per warp of the flattened reduce (a power of two) and its log2; set by bn_bwd_reduce
     float* gmax;                                   // device scalar: bound on |gv| over the tensor (nullable)
     int gv_dtype;                                  // storage type of gv (OT)
     float4* coef; float4* coef_r;                  // [C]: (k, c1, c2, unused)
@@ -198,6 +232,15 @@ void bn_bwd_finalize(const Launch& L, const BnBwdArgs& a, const float* gamma, co
                      float* dgamma, float* dbeta, float* dgamma_r, float* dbeta_r, float* dbias,
                      int accumulate);
 void bn_bwd_apply(const Launch& L, int dtype, const BnBwdArgs& a);
+
+// ---- decoder tail / evaluation mode ---------------------------------------------------------------
+// y[b,:,t] = [t < len_out[b]] * (z[b,:,t] - log(sum_c exp(z[b,c,t]))), z in float32
+void log_softmax_fwd(const Launch& L, int dtype, const float* z, void* y, const int* len_out, int B, int C, int Tp);
+// dz[b,c,t] = [t < len_out[b]] * (g[b,c,t] - exp(logp[b,c,t]) * sum_c' g[b,c',t])
+void log_softmax_bwd(const Launch& L, int dtype, void* dz, const void* g, const void* logp, const int* len_out, int B,
+                     int C, int Tp);
+// invstd[o] = 1 / sqrt(var[o] + eps)
+void invstd_from_var(const Launch& L, const float* var, float eps, float* invstd, int C);
 
 // out (half) = [t<len[b]] ? in (bf16) : 0; values beyond the half range are clamped and flagged
 void mask_convert_f16(const Launch& L, void* out, const void* in, const int* len, int B, int C, int T);

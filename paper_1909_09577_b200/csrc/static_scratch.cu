@@ -6,6 +6,7 @@
 #include <cstdio>
 
 #include "../../include/sepconv.h"
+#include "kernels.h"
 
 // One array per GPU that loads the library, held until the process exits.
 static __device__ __align__(256) unsigned char g_static_scratch[SEPCONV_STATIC_SCRATCH_BYTES];
@@ -33,7 +34,14 @@ extern "C" int sepconv_fwd_static(sc_ctx* ctx, const sc_block_desc* desc, const 
     }
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SC_ERR_CUDA;
-    if (!g_scratch_addr[dev]) {     // first call on this device: resolve the array's device address
+    // the array and its address belong to the current device: it must be the one the context lives on
+    if (dev != sc::ctx_device(ctx)) {
+        fprintf(stderr, "sepconv_fwd_static: the current device (%d) is not the context's device (%d)\n", dev,
+                sc::ctx_device(ctx));
+        return SC_ERR_UNSUPPORTED;
+    }
+    if (!g_scratch_addr[dev]) {     // first call on this device: resolve the array's device address (with lazy
+                                    // module loading this is also where the device sets the array aside)
         void* p = nullptr;
         cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
         if (e != cudaSuccess || !p) {
@@ -44,9 +52,8 @@ extern "C" int sepconv_fwd_static(sc_ctx* ctx, const sc_block_desc* desc, const 
     }
     void* ws = g_scratch_addr[dev];
     // The array keeps whatever the previous call left.  Every scratch word the forward kernels read
-    // they write first in the same call, so nothing has to start at zero; the lengths/count header
-    // is cleared anyway so that a stale frame count can never be mistaken for a fresh one.
-    if (cudaMemsetAsync(ws, 0, 4096, (cudaStream_t)cuda_stream) != cudaSuccess) return SC_ERR_CUDA;
+    // they write first in the same call (lengths, frame count, statistics partials, masked copies), so
+    // nothing has to start at zero and nothing is enqueued before sepconv_fwd has validated its arguments.
     return sepconv_fwd(ctx, desc, x, x_res, lengths_dev, params, y, out_lengths_dev, saved, nullptr, nullptr,
                        ws, (size_t)SEPCONV_STATIC_SCRATCH_BYTES, cuda_stream);
 }

@@ -38,7 +38,7 @@ struct TcParams {
     int Kdim;       // forward: C_in, input gradient: C_out
     int B, Tp;
     int zero_fill;  // skipped (all-padding) tiles must still be written as zeros
-    int out_f32;    // forward: the result tensor is float32
+    int out_kind;   // forward: type of the result tensor: 0 = the operand type, 1 = float32, 2 = float16
     int nkb_t;      // weight gradient: 64-frame blocks per sample
     int kb_per_split, nkb_total;
 };
@@ -52,6 +52,17 @@ template <> struct Fmt<__nv_bfloat16> { static constexpr uint32_t v = 1; };
 // 16 bytes each (half-filled sectors).  The block is transposed through a per-warp shared-memory
 // buffer (row pitch 36 floats) so that each instruction writes whole 128-byte (fp32) or 64-byte
 // (16-bit) row segments.  `rows_left` / `cols_left` bound the valid part; cols are a multiple of 8.
+// A float16 result beyond the half range is clamped to the largest finite value and flagged.
+__device__ __forceinline__ void clamp_half32(float (&f)[32], int* status) {
+    float m = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) m = fmaxf(m, fabsf(f[i]));
+    if (m > 65504.f) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) f[i] = fminf(fmaxf(f[i], -65504.f), 65504.f);
+        raise_status(status, kErrRange);
+    }
+}
 constexpr int kStgPitch = 36;
 constexpr int kStgFloatsPerWarp = 32 * kStgPitch;
 template <typename OT>
@@ -113,7 +124,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
         if (p.len_out) len = min(p.len_out[z], p.Tp);
         if (n0 >= len) {                           // whole tile in padding
             if (p.zero_fill) {
-                const int esz = (MODE == MODE_FWD && p.out_f32) ? 4 : (int)sizeof(T);
+                const int esz = (MODE == MODE_FWD && p.out_kind == 1) ? 4 : (int)sizeof(T);
                 const int vec_per_row = BN * esz / 16;
                 for (int i = tid; i < 128 * MT * vec_per_row; i += kThreads) {
                     const int r = m0 + i / vec_per_row, cb = (i % vec_per_row) * (16 / esz);
@@ -259,14 +270,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
                     }
 #pragma unroll
                     for (int i = 0; i < 32; ++i) if (i >= nv) f[i] = 0.f;
+                    if (p.out_kind == 2 || (p.out_kind == 0 && sizeof(T) == 2 && Fmt<T>::v == 0)) clamp_half32(f, p.status);
                 }
                 {
                     const int row_w = m0 + mt * 128 + warp * 32;             // first row of this warp's block
                     const size_t base = ((size_t)z * p.M + row_w) * p.Ncols + n0 + c0;
                     float* stg = stg_all + warp * kStgFloatsPerWarp;
                     const int rl = p.M - row_w, cl = p.Ncols - (n0 + c0);
-                    if ((MODE == MODE_FWD && p.out_f32) || MODE == MODE_WGRAD)
+                    if ((MODE == MODE_FWD && p.out_kind == 1) || MODE == MODE_WGRAD)
                         store_block_staged<float>(stg, f, reinterpret_cast<float*>(p.out) + base, p.Ncols, rl, cl, lane);
+                    else if (MODE == MODE_FWD && p.out_kind == 2)
+                        store_block_staged<__half>(stg, f, reinterpret_cast<__half*>(p.out) + base, p.Ncols, rl, cl, lane);
                     else
                         store_block_staged<T>(stg, f, reinterpret_cast<T*>(p.out) + base, p.Ncols, rl, cl, lane);
                 }
@@ -407,7 +421,7 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap mapA, const __grid
             int n0, m0, z, len;
             if (!tile_info(tile, n0, m0, z, len)) {
                 if (p.zero_fill) {
-                    const int esz = (MODE == MODE_FWD && p.out_f32) ? 4 : (int)sizeof(T);
+                    const int esz = (MODE == MODE_FWD && p.out_kind == 1) ? 4 : (int)sizeof(T);
                     const int vec_per_row = BN * esz / 16;
                     for (int i = tid; i < 128 * MT * vec_per_row; i += 128 * MT) {
                         const int r = m0 + i / vec_per_row, cb = (i % vec_per_row) * (16 / esz);
@@ -455,14 +469,17 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap mapA, const __grid
                         }
 #pragma unroll
                         for (int i = 0; i < 32; ++i) if (i >= nv) f[i] = 0.f;
+                        if (p.out_kind == 2 || (p.out_kind == 0 && sizeof(T) == 2 && Fmt<T>::v == 0)) clamp_half32(f, p.status);
                     }
                     {
                         const int row_w = m0 + mt * 128 + wq * 32;
                         const size_t base = ((size_t)z * p.M + row_w) * p.Ncols + n0 + c0;
                         float* stg = stg_all + warp * kStgFloatsPerWarp;
                         const int rl = p.M - row_w, cl = p.Ncols - (n0 + c0);
-                        if (MODE == MODE_FWD && p.out_f32)
+                        if (MODE == MODE_FWD && p.out_kind == 1)
                             store_block_staged<float>(stg, f, reinterpret_cast<float*>(p.out) + base, p.Ncols, rl, cl, lane);
+                        else if (MODE == MODE_FWD && p.out_kind == 2)
+                            store_block_staged<__half>(stg, f, reinterpret_cast<__half*>(p.out) + base, p.Ncols, rl, cl, lane);
                         else
                             store_block_staged<T>(stg, f, reinterpret_cast<T*>(p.out) + base, p.Ncols, rl, cl, lane);
                     }
@@ -482,6 +499,334 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap mapA, const __grid
     ptx::tc_fence_before();
     __syncthreads();
     if (warp == 0) ptx::tmem_dealloc(tmem, TMEM_COLS);
+}
+
+// ---- persistent forward / input-gradient contraction over a flattened list of 64-frame blocks -----------
+// The N dimension of these contractions is (sample, frame).  Cutting it per sample into fixed tiles wastes
+// the tail of every sample (800 frames = 6.25 tiles of 128) and leaves the last wave of tiles mostly idle.
+// Here the valid 64-frame blocks of all samples form one list (a sample of len' frames contributes
+// ceil(len'/64) blocks; blocks wholly in padding are not in the list), a work unit is (128*MT-row M tile,
+// block), and CTA c of G takes the contiguous unit range [c U / G, (c+1) U / G): every CTA gets the same
+// number of blocks to within one.  Inside its range a CTA forms tiles of up to four consecutive blocks of one
+// M tile; an N-major B operand is a row of independent 64-column sub-tiles in shared memory, so the blocks of
+// a tile need not be adjacent in memory nor belong to one sample, and one MMA covers N = 64 * blocks columns.
+// Roles as above (epilogue warps, one TMA thread, one MMA thread); the accumulator (MT x 256 columns) fills
+// tensor memory, so the epilogue of a tile is not overlapped with the next tile's MMAs, only with its loads.
+// Statistics: a thread owns one output channel for the CTA's whole range of an M tile, sums about a pivot taken
+// from the row's first valid frame, and writes one (count, sum, M2) partial per (CTA, channel).
+constexpr int kFlatMaxNB = 4;          // blocks per tile (N up to 256)
+constexpr int kFlatMaxB = 2048;        // samples whose block offsets fit the shared-memory copy
+constexpr int kFlatMaxGrid = 256;
+constexpr int kOutPitch = 80;          // bytes per row of a warp's 32 x 32 staging block of 16-bit values
+constexpr int kOutStageBytes = 32 * kOutPitch;
+
+struct FlatParams {
+    void* out; const float* bias; const int* len_out; const int* blk_off; float4* stats; int* status;
+    int M;          // rows of D in total (C_out forward, C_in input gradient)
+    int Kdim;       // forward: C_in, input gradient: C_out
+    int B, Tp, nbT; // nbT = ceil(Tp / 64)
+    int tiles_m;
+    int zero_fill;  // blocks wholly in padding must be written as zeros
+    int out_half;   // the result is float16 although the operands are bfloat16
+    int out_f32;    // the result is float32 (one M sub-tile per CTA only: narrow heads such as the class scores)
+};
+
+// Coalesced store of a warp's 32 x 32 block as 16-bit values: lane l holds 32 consecutive columns of row l;
+// the block goes through a per-warp shared-memory buffer (row pitch 80 bytes: conflict-free both ways) so that
+// each store instruction writes whole 64-byte row segments.  cols_left is a multiple of 8.
+template <typename OT>
+__device__ __forceinline__ void store_block16(uint8_t* stg, const float (&f)[32], OT* out, size_t ld, int rows_left,
+                                              int cols_left, int lane) {
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float g[8] = {f[8 * i], f[8 * i + 1], f[8 * i + 2], f[8 * i + 3], f[8 * i + 4], f[8 * i + 5], f[8 * i + 6], f[8 * i + 7]};
+        st8<OT>(reinterpret_cast<OT*>(stg + lane * kOutPitch + i * 16), g);
+    }
+    __syncwarp();
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int r = it * 8 + (lane >> 2), c = (lane & 3) * 8;
+        if (r < rows_left && c < cols_left) {
+            const uint4 v = *reinterpret_cast<const uint4*>(stg + r * kOutPitch + (lane & 3) * 16);
+            *reinterpret_cast<uint4*>(out + (size_t)r * ld + c) = v;
+        }
+    }
+}
+
+// largest b in [0, B) with off[b] <= j  (off is non-decreasing, off[0] = 0, j < off[B])
+__device__ __forceinline__ int flat_find_sample(const int* off, int B, int j) {
+    int lo = 0, hi = B - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (off[mid] <= j) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+// next tile of a CTA's unit range: M tile m, first block j, nb blocks
+template <int NB>
+__device__ __forceinline__ bool flat_next_tile(long long& pos, long long end, int nblk, int& m, int& j, int& nb) {
+    if (pos >= end) return false;
+    m = (int)(pos / nblk); j = (int)(pos - (long long)m * nblk);
+    nb = (int)min((long long)NB, min(end - pos, (long long)(nblk - j)));
+    pos += nb;
+    return true;
+}
+
+// Shapes: MT M sub-tiles of 128 rows, NB blocks per tile, NBUF accumulator buffers (MT * NB * 64 * NBUF <= 512
+// tensor-memory columns).  With NBUF = 2 the epilogue of a tile overlaps the MMAs of the next one.
+template <int MT, int NB> struct FlatCfg {
+    static constexpr int A_BYTES = MT * 128 * 128;
+    static constexpr int STAGE = A_BYTES + NB * 8192;
+    static constexpr int STAGES = STAGE <= 49152 ? 4 : 3;
+    // per-warp staging: 32 x 32 16-bit values, or (one M sub-tile only) 32 x 32 floats for a float32 result
+    static constexpr int STG = MT == 1 ? kStgFloatsPerWarp * 4 : kOutStageBytes;
+    static constexpr int smem_bytes(int B) { return STAGES * STAGE + 256 + 4 * MT * STG + (B + 1) * 4 + 1024; }
+};
+
+template <typename T, int MODE, int MT, int NB, int NBUF>
+__global__ void __launch_bounds__(32 * (4 * MT + 2), 1)
+tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, FlatParams p) {
+    static_assert(MODE == MODE_FWD || MODE == MODE_DGRAD, "forward / input gradient only");
+    constexpr int A_BYTES = FlatCfg<MT, NB>::A_BYTES;
+    constexpr int STAGE = FlatCfg<MT, NB>::STAGE;
+    constexpr int STAGES = FlatCfg<MT, NB>::STAGES;
+    constexpr uint32_t ACC_COLS = MT * NB * 64;
+    constexpr uint32_t TMEM_COLS = ACC_COLS * NBUF;
+    static_assert(TMEM_COLS == 128 || TMEM_COLS == 256 || TMEM_COLS == 512, "tensor-memory columns");
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE);
+    uint64_t* empty = full + STAGES;
+    uint64_t* acc_full = empty + STAGES;       // [NBUF]
+    uint64_t* acc_empty = acc_full + NBUF;     // [NBUF]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + NBUF);
+    uint8_t* stg_all = smem + STAGES * STAGE + 256;
+    constexpr int STG = FlatCfg<MT, NB>::STG;
+    int* s_off = reinterpret_cast<int*>(stg_all + 4 * MT * STG);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
+        for (int i = 0; i < NBUF; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 128 * MT); }
+        ptx::fence_barrier_init();
+        ptx::prefetch_tensormap(&mapA);
+        ptx::prefetch_tensormap(&mapB);
+    }
+    if (warp == 0) { ptx::tmem_alloc(tmem_slot, TMEM_COLS); ptx::tmem_relinquish(); }
+    for (int i = tid; i <= p.B; i += blockDim.x) s_off[i] = p.blk_off[i];
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    const int nkb = (p.Kdim + BK - 1) / BK;
+    const int nblk = s_off[p.B];
+    const long long U = (long long)p.tiles_m * nblk;
+    const long long u_begin = U * blockIdx.x / gridDim.x, u_end = U * (blockIdx.x + 1) / gridDim.x;
+
+    if (warp == 4 * MT) {
+        if (lane == 0) {                              // ---- TMA producer ----
+            int it = 0, m, j, nb;
+            bool dead = false;
+            long long pos = u_begin;
+            while (!dead && flat_next_tile<NB>(pos, u_end, nblk, m, j, nb)) {
+                int bb[NB], tt[NB];
+                int b = flat_find_sample(s_off, p.B, j);
+#pragma unroll
+                for (int i = 0; i < NB; ++i) {
+                    if (i < nb) {
+                        while (j + i >= s_off[b + 1]) ++b;
+                        bb[i] = b; tt[i] = (j + i - s_off[b]) * 64;
+                    } else { bb[i] = 0; tt[i] = 0; }
+                }
+                const int m0 = m * (128 * MT);
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % STAGES, ph = (it / STAGES) & 1;
+                    if (!ptx::mbar_wait(&empty[s], ph ^ 1)) { raise_status(p.status, kErrTimeout); dead = true; break; }
+                    ptx::mbar_arrive_expect_tx(&full[s], A_BYTES + nb * 8192);
+                    uint8_t* sA = smem + s * STAGE;
+                    uint8_t* sB = sA + A_BYTES;
+                    const int k0 = kb * BK;
+                    if (MODE == MODE_FWD) {
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt) ptx::tma_load_2d(sA + mt * 16384, &mapA, &full[s], k0, m0 + mt * 128);
+                    } else {
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                            for (int h = 0; h < 2; ++h)
+                                ptx::tma_load_2d(sA + mt * 16384 + h * 8192, &mapA, &full[s], m0 + mt * 128 + 64 * h, k0);
+                    }
+#pragma unroll
+                    for (int i = 0; i < NB; ++i)
+                        if (i < nb) ptx::tma_load_3d(sB + i * 8192, &mapB, &full[s], tt[i], k0, bb[i]);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 4 * MT + 1) {
+        if (lane == 0) {                              // ---- MMA issuer ----
+            int it = 0, jt = 0, m, j, nb;
+            bool dead = false;
+            long long pos = u_begin;
+            while (!dead && flat_next_tile<NB>(pos, u_end, nblk, m, j, nb)) {
+                const int buf = jt % NBUF;
+                if (!ptx::mbar_wait(&acc_empty[buf], ((jt / NBUF) & 1) ^ 1)) { raise_status(p.status, kErrTimeout); break; }
+                ptx::tc_fence_after();
+                const uint32_t idesc = ptx::instr_desc(Fmt<T>::v, MODE == MODE_DGRAD ? 1u : 0u, 1u, 128, 64u * nb);
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % STAGES, ph = (it / STAGES) & 1;
+                    if (!ptx::mbar_wait(&full[s], ph)) { raise_status(p.status, kErrTimeout); dead = true; break; }
+                    ptx::tc_fence_after();
+                    const uint32_t aA = ptx::smem_u32(smem + s * STAGE), aB = aA + A_BYTES;
+#pragma unroll
+                    for (int ks = 0; ks < BK / 16; ++ks) {
+                        const uint64_t bdesc = ptx::smem_desc(aB + ks * 2048, 8192, 1024);
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt) {
+                            const uint64_t adesc = (MODE == MODE_DGRAD) ? ptx::smem_desc(aA + mt * 16384 + ks * 2048, 8192, 1024)
+                                                                        : ptx::smem_desc(aA + mt * 16384 + ks * 32, 16, 1024);
+                            ptx::mma_f16(tmem + buf * ACC_COLS + mt * (NB * 64), adesc, bdesc, idesc, (kb > 0 || ks > 0) ? 1u : 0u);
+                        }
+                    }
+                    ptx::mma_commit(&empty[s]);
+                }
+                if (!dead) ptx::mma_commit(&acc_full[buf]);
+                ++jt;
+            }
+        }
+        __syncwarp();
+    } else {                                          // ---- epilogue warps ----
+        const int mt = warp >> 2, wq = warp & 3;
+        uint8_t* stg = stg_all + warp * STG;
+        if (p.zero_fill) {
+            // blocks wholly in padding: sample b's blocks [off[b+1]-off[b], nbT); CTAs share them round-robin
+            const int inv_per_m = p.B * p.nbT - nblk;
+            const long long total_inv = (long long)p.tiles_m * inv_per_m;
+            for (long long q = blockIdx.x; q < total_inv; q += gridDim.x) {
+                const int m = (int)(q / inv_per_m), jj = (int)(q - (long long)m * inv_per_m);
+                int lo = 0, hi = p.B - 1;              // largest b with b * nbT - off[b] <= jj
+                while (lo < hi) {
+                    const int mid = (lo + hi + 1) >> 1;
+                    if (mid * p.nbT - s_off[mid] <= jj) lo = mid; else hi = mid - 1;
+                }
+                const int b = lo;
+                const int t0 = ((s_off[b + 1] - s_off[b]) + (jj - (b * p.nbT - s_off[b]))) * 64;
+                for (int i = tid; i < 128 * MT * 8; i += 128 * MT) {
+                    const int r = m * (128 * MT) + (i >> 3), cb = (i & 7) * 8;
+                    if (r < p.M && t0 + cb < p.Tp) {
+                        const size_t e = ((size_t)b * p.M + r) * p.Tp + t0 + cb;
+                        if (MT == 1 && p.out_f32) {
+                            *reinterpret_cast<uint4*>(reinterpret_cast<float*>(p.out) + e) = make_uint4(0, 0, 0, 0);
+                            *reinterpret_cast<uint4*>(reinterpret_cast<float*>(p.out) + e + 4) = make_uint4(0, 0, 0, 0);
+                        } else {
+                            *reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(p.out) + e) = make_uint4(0, 0, 0, 0);
+                        }
+                    }
+                }
+            }
+        }
+        int jt = 0, m, j, nb, cur_m = -1;
+        long long pos = u_begin;
+        float sn = 0.f, sd = 0.f, sq = 0.f, pivot = 0.f;     // statistics of this thread's channel over the CTA's range of one M tile
+        auto flush_stats = [&]() {
+            if (MODE != MODE_FWD || !p.stats || cur_m < 0) return;
+            const int row = cur_m * (128 * MT) + mt * 128 + wq * 32 + lane;
+            if (row < p.M) p.stats[(size_t)blockIdx.x * p.M + row] = make_float4(sn, fmaf(pivot, sn, sd), sn > 0.f ? sq - sd * sd / sn : 0.f, 0.f);
+        };
+        while (flat_next_tile<NB>(pos, u_end, nblk, m, j, nb)) {
+            if (m != cur_m) { flush_stats(); cur_m = m; sn = sd = sq = 0.f; }
+            const int buf = jt % NBUF;
+            if (!ptx::mbar_wait_warp(&acc_full[buf], (jt / NBUF) & 1)) { if (lane == 0) raise_status(p.status, kErrTimeout); break; }
+            ptx::tc_fence_after();
+            const int row_w = m * (128 * MT) + mt * 128 + wq * 32;
+            const int row = row_w + lane;
+            const float bias = (MODE == MODE_FWD && p.bias && row < p.M) ? p.bias[row] : 0.f;
+            int b = flat_find_sample(s_off, p.B, j);
+            for (int i = 0; i < nb; ++i) {
+                while (j + i >= s_off[b + 1]) ++b;
+                const int t0 = (j + i - s_off[b]) * 64;
+                const int len = min(p.len_out[b], p.Tp);
+#pragma unroll 1
+                for (int h = 0; h < 2; ++h) {
+                    const int c0 = t0 + 32 * h;
+                    if (c0 >= p.Tp) break;
+                    float f[32];
+                    {
+                        uint32_t r[32];
+                        ptx::tmem_ld32(tmem + ((uint32_t)(wq * 32) << 16) + buf * ACC_COLS + mt * (NB * 64) + i * 64 + h * 32, r);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int q = 0; q < 32; ++q) f[q] = __uint_as_float(r[q]);
+                    }
+                    if (MODE == MODE_FWD) {
+                        if (p.bias) {
+#pragma unroll
+                            for (int q = 0; q < 32; ++q) f[q] += bias;
+                        }
+                        const int nv = max(0, min(32, len - c0));
+                        if (p.stats && nv > 0) {
+                            if (sn == 0.f) pivot = f[0];
+                            if (nv == 32) {
+                                // packed pairs: d = f - pivot, sum d, sum d^2 in three two-wide instructions per pair
+                                const uint64_t np2 = ptx::pack2(-pivot, -pivot);
+                                uint64_t sd2 = ptx::pack2(0.f, 0.f), sq2 = ptx::pack2(0.f, 0.f);
+#pragma unroll
+                                for (int q = 0; q < 16; ++q) {
+                                    const uint64_t d2 = ptx::add2(ptx::pack2(f[2 * q], f[2 * q + 1]), np2);
+                                    sd2 = ptx::add2(sd2, d2);
+                                    sq2 = ptx::fma2(d2, d2, sq2);
+                                }
+                                float a0, a1, b0, b1;
+                                ptx::unpack2(sd2, a0, a1); ptx::unpack2(sq2, b0, b1);
+                                sd += a0 + a1; sq += b0 + b1;
+                            } else {
+#pragma unroll
+                                for (int q = 0; q < 32; ++q) if (q < nv) { const float d = f[q] - pivot; sd += d; sq = fmaf(d, d, sq); }
+                            }
+                            sn += (float)nv;
+                        }
+                        if (nv < 32) {
+#pragma unroll
+                            for (int q = 0; q < 32; ++q) if (q >= nv) f[q] = 0.f;
+                        }
+                        if (!p.out_f32 && (p.out_half || Fmt<T>::v == 0)) clamp_half32(f, p.status);
+                    }
+                    const size_t base = ((size_t)b * p.M + row_w) * p.Tp + c0;
+                    const int rl = p.M - row_w, cl = p.Tp - c0;
+                    if (MT == 1 && MODE == MODE_FWD && p.out_f32)
+                        store_block_staged<float>(reinterpret_cast<float*>(stg), f, reinterpret_cast<float*>(p.out) + base, p.Tp, rl, cl, lane);
+                    else if (MODE == MODE_FWD && p.out_half)
+                        store_block16<__half>(stg, f, reinterpret_cast<__half*>(p.out) + base, p.Tp, rl, cl, lane);
+                    else
+                        store_block16<T>(stg, f, reinterpret_cast<T*>(p.out) + base, p.Tp, rl, cl, lane);
+                }
+            }
+            ptx::tc_fence_before();
+            ptx::mbar_arrive(&acc_empty[buf]);        // this thread is done reading the accumulator
+            ++jt;
+        }
+        flush_stats();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 0) ptx::tmem_dealloc(tmem, TMEM_COLS);
+}
+
+// Self-test of the bounded-wait exit: one thread waits on an mbarrier on which nothing ever arrives, with a
+// short poll limit; the wait gives up, raises the timeout status and the kernel returns normally.  No copy is
+// in flight and no tensor memory is held, so there is nothing to drain.
+__global__ void bounded_wait_selftest_kernel(int* status) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&bar, 1);
+        ptx::fence_barrier_init();
+        bool ok = false;
+        for (uint32_t i = 0; i < (1u << 12) && !ok; ++i) ok = ptx::mbar_try_wait(&bar, 0);
+        if (!ok) raise_status(status, kErrTimeout);
+    }
 }
 
 // ---- host side -------------------------------------------------------------------------------
@@ -518,12 +863,8 @@ bool make_map(const TcState* st, CUtensorMap* m, int dtype, const void* base, in
 template <typename T, int MODE, int MT, int BN, int STAGES>
 void launch(const Launch& L, dim3 grid, const CUtensorMap& a, const CUtensorMap& b, const TcParams& p) {
     constexpr int smem = STAGES * (MT * 16384 + BN * 128) + 1024 + 256 + 4 * kStgFloatsPerWarp * 4;
-    static bool configured = false;
     auto kern = tc_gemm_kernel<T, MODE, MT, BN, STAGES>;
-    if (!configured) {
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        configured = true;
-    }
+    set_max_smem_once<tc_gemm_kernel<T, MODE, MT, BN, STAGES>>(smem);
     kern<<<grid, kThreads, smem, L.stream>>>(a, b, p);
     L.count();
 }
@@ -538,12 +879,8 @@ template <typename T, int MODE, int MT, int BN, int STAGES>
 void launch_persistent(const Launch& L, int sm_count, const CUtensorMap& a, const CUtensorMap& b, const TcParams& p,
                        int tiles_n, int tiles_m, int batch) {
     constexpr int smem = STAGES * (MT * 16384 + BN * 128) + 1024 + 256 + 4 * MT * kStgFloatsPerWarp * 4;
-    static bool configured = false;
     auto kern = tc_gemm_persistent_kernel<T, MODE, MT, BN, STAGES>;
-    if (!configured) {
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        configured = true;
-    }
+    set_max_smem_once<tc_gemm_persistent_kernel<T, MODE, MT, BN, STAGES>>(smem);
     const int total = tiles_n * tiles_m * batch;
     kern<<<std::min(sm_count, total), 32 * (4 * MT + 2), smem, L.stream>>>(a, b, p, tiles_n, tiles_m, total);
     L.count();
@@ -578,6 +915,11 @@ WgradPlan plan_wgrad(int B, int Cin, int Cout, int Tp) {
 
 }  // namespace
 
+void selftest_bounded_wait(const Launch& L) {
+    bounded_wait_selftest_kernel<<<1, 32, 0, L.stream>>>(L.status);
+    L.count();
+}
+
 int tc_init(TcState* st, int device, int sm_count) {
     (void)device;
     st->sm_count = sm_count;
@@ -586,8 +928,7 @@ int tc_init(TcState* st, int device, int sm_count) {
     cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
     st->encode_fn = (e == cudaSuccess && q == cudaDriverEntryPointSuccess) ? fn : nullptr;
     st->ready = st->encode_fn != nullptr;
-    const char* e_p = getenv("SEPCONV_GEMM_PERSISTENT");
-    st->persistent = !(e_p && e_p[0] == '0');
+    st->persistent = true;
     if (!st->ready) { fprintf(stderr, "sepconv: cuTensorMapEncodeTiled not available\n"); return -11; }
     return 0;
 }
@@ -604,51 +945,104 @@ size_t tc_wgrad_scratch_bytes(const TcState*, int Cin, int Cout) {
     return (size_t)w.nsplit * Cin * Cout * sizeof(float);
 }
 
-bool tc_gemm_fwd(const TcState* st, const Launch& L, int dtype, const void* w, const void* u, const float* bias,
-                 void* v, int out_dtype, const int* len_out, int B, int Cin, int Cout, int Tp, float2* partials,
-                 int* parts_per_b, int* tile_w) {
-    KScope ks_(L, KC_PW_FWD, (double)B * Tp * (2.0 * Cin + dtype_size(out_dtype) * Cout), 2.0 * B * Tp * Cin * Cout);
+namespace {
+template <typename T, int MODE, int MT, int NB, int NBUF>
+void launch_flat(const Launch& L, int sm_count, const CUtensorMap& a, const CUtensorMap& b, const FlatParams& p, int* grid_out) {
+    const int smem = FlatCfg<MT, NB>::smem_bytes(p.B);
+    auto kern = tc_gemm_flat_kernel<T, MODE, MT, NB, NBUF>;
+    set_max_smem_once<tc_gemm_flat_kernel<T, MODE, MT, NB, NBUF>>(FlatCfg<MT, NB>::smem_bytes(kFlatMaxB));
+    const long long units = (long long)p.tiles_m * p.B * p.nbT;
+    const int grid = (int)std::max(1ll, std::min<long long>(std::min(sm_count, kFlatMaxGrid), units));
+    kern<<<grid, 32 * (4 * MT + 2), smem, L.stream>>>(a, b, p);
+    L.count();
+    if (grid_out) *grid_out = grid;
+}
+// shape 0: 256 x 256 tiles, one accumulator; 1: 256 x 128 tiles, two accumulators; 2: 128 x 256 tiles, two accumulators
+template <typename T, int MODE>
+void launch_flat_shape(int shape, int mt, const Launch& L, int sm_count, const CUtensorMap& a, const CUtensorMap& b,
+                       const FlatParams& p, int* grid_out) {
+    if (mt == 1) { launch_flat<T, MODE, 1, 4, 2>(L, sm_count, a, b, p, grid_out); return; }
+    if (shape == 0) launch_flat<T, MODE, 2, 4, 1>(L, sm_count, a, b, p, grid_out);
+    else launch_flat<T, MODE, 2, 2, 2>(L, sm_count, a, b, p, grid_out);
+}
+template <int MODE>
+void launch_flat_dt(int dtype, int shape, int mt, const Launch& L, int sm_count, const CUtensorMap& a, const CUtensorMap& b,
+                    const FlatParams& p, int* grid_out) {
+    if (dtype == F16) launch_flat_shape<__half, MODE>(shape, mt, L, sm_count, a, b, p, grid_out);
+    else launch_flat_shape<__nv_bfloat16, MODE>(shape, mt, L, sm_count, a, b, p, grid_out);
+}
+// M sub-tiles per CTA for a given tile shape and row count
+inline int flat_mt(int shape, int rows) { return (shape == 2 || rows <= 128) ? 1 : 2; }
+}  // namespace
+
+size_t tc_stats_bytes(int B, int Cout, int Tp) {
+    return std::max((size_t)B * tc_max_parts_per_sample(Tp) * Cout * sizeof(float2), (size_t)kFlatMaxGrid * Cout * sizeof(float4));
+}
+
+void tc_gemm_fwd(const TcState* st, const Launch& L, int dtype, const void* w, const void* u, const float* bias,
+                 void* v, int out_dtype, const int* len_out, const int* blk_off, int B, int Cin, int Cout, int Tp,
+                 void* partials, StatsLayout* layout) {
+    // algorithmic bytes: operand and result once each (16-bit), weights once
+    KScope ks_(L, KC_PW_FWD, (double)B * Tp * (2.0 * Cin + dtype_size(out_dtype) * Cout) + 2.0 * Cin * Cout, 2.0 * B * Tp * Cin * Cout);
     CUtensorMap ma, mb;
     const uint64_t da[2] = {(uint64_t)Cin, (uint64_t)Cout};
     const uint32_t ba[2] = {64, 128};
     const uint64_t db[3] = {(uint64_t)Tp, (uint64_t)Cin, (uint64_t)B};
     const uint32_t bb[3] = {64, 64, 1};
-    if (!make_map(st, &ma, dtype, w, 2, da, ba) || !make_map(st, &mb, dtype, u, 3, db, bb)) return false;
+    if (layout) *layout = StatsLayout{};
+    if (!make_map(st, &ma, dtype, w, 2, da, ba) || !make_map(st, &mb, dtype, u, 3, db, bb)) return;
+    int mt = Cout > 128 ? 2 : 1;
+    if (st->flat && blk_off && B <= kFlatMaxB && (out_dtype != F32 || Cout <= 128)) {
+        mt = flat_mt(st->flat_shape, Cout);
+        FlatParams p{};
+        p.out = v; p.bias = bias; p.len_out = len_out; p.blk_off = blk_off; p.stats = (float4*)partials; p.status = L.status;
+        p.M = Cout; p.Kdim = Cin; p.B = B; p.Tp = Tp; p.nbT = (Tp + 63) / 64;
+        p.tiles_m = (Cout + 128 * mt - 1) / (128 * mt);
+        p.zero_fill = partials ? 0 : 1;     // a linear layer's result is the block output: padding must read as zero
+        p.out_half = (out_dtype == F16 && dtype != F16) ? 1 : 0;
+        p.out_f32 = out_dtype == F32 ? 1 : 0;
+        int grid = 0;
+        launch_flat_dt<MODE_FWD>(dtype, st->flat_shape, mt, L, st->sm_count, ma, mb, p, &grid);
+        if (layout && partials) { layout->kind = 2; layout->grid = grid; layout->tiles_m = p.tiles_m; layout->rows_per_tile = 128 * mt; }
+        return;
+    }
     TcParams p{};
-    p.out = v; p.bias = bias; p.len_out = len_out; p.stats = partials; p.status = L.status;
+    p.out = v; p.bias = bias; p.len_out = len_out; p.stats = (float2*)partials; p.status = L.status;
     p.M = Cout; p.Ncols = Tp; p.Kdim = Cin; p.B = B; p.Tp = Tp;
-    p.zero_fill = partials ? 0 : 1;     // a linear layer's result is the block output: padding must read as zero
-    p.out_f32 = (out_dtype == F32);
-    const int mt = Cout > 128 ? 2 : 1;
+    p.zero_fill = partials ? 0 : 1;
+    p.out_kind = out_dtype == F32 ? 1 : (out_dtype == dtype ? 0 : 2);
     dim3 grid((Tp + FWD_BN - 1) / FWD_BN, (Cout + 128 * mt - 1) / (128 * mt), B);
-    if (st->persistent) {
-        if (mt == 2) launch_persistent_dt<MODE_FWD, 2, FWD_BN, 3>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
-        else launch_persistent_dt<MODE_FWD, 1, FWD_BN, 6>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
-    } else if (mt == 2) launch_dt<MODE_FWD, 2, FWD_BN, 2>(dtype, L, grid, ma, mb, p);
-    else launch_dt<MODE_FWD, 1, FWD_BN, 3>(dtype, L, grid, ma, mb, p);
-    *parts_per_b = grid.x; *tile_w = FWD_BN;
-    return partials != nullptr;
+    if (mt == 2) launch_persistent_dt<MODE_FWD, 2, FWD_BN, 3>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
+    else launch_persistent_dt<MODE_FWD, 1, FWD_BN, 6>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
+    if (layout && partials) { layout->kind = 1; layout->parts_per_b = grid.x; layout->tile_w = FWD_BN; }
 }
 
 void tc_gemm_dgrad(const TcState* st, const Launch& L, int dtype, const void* w, const void* gv, void* gu, int B,
-                   int Cin, int Cout, int Tp, const int* len_out) {
-    KScope ks_(L, KC_PW_DGRAD, 2.0 * B * Tp * (Cin + Cout), 2.0 * B * Tp * Cin * Cout);
+                   int Cin, int Cout, int Tp, const int* len_out, const int* blk_off) {
+    KScope ks_(L, KC_PW_DGRAD, 2.0 * B * Tp * (Cin + Cout) + 2.0 * Cin * Cout, 2.0 * B * Tp * Cin * Cout);
     CUtensorMap ma, mb;
     const uint64_t da[2] = {(uint64_t)Cin, (uint64_t)Cout};
     const uint32_t ba[2] = {64, 64};
     const uint64_t db[3] = {(uint64_t)Tp, (uint64_t)Cout, (uint64_t)B};
     const uint32_t bb[3] = {64, 64, 1};
     if (!make_map(st, &ma, dtype, w, 2, da, ba) || !make_map(st, &mb, dtype, gv, 3, db, bb)) return;
+    int mt = Cin > 128 ? 2 : 1;
+    if (st->flat && blk_off && B <= kFlatMaxB) {
+        mt = flat_mt(st->flat_shape, Cin);
+        FlatParams p{};
+        p.out = gu; p.len_out = len_out; p.blk_off = blk_off; p.status = L.status;
+        p.M = Cin; p.Kdim = Cout; p.B = B; p.Tp = Tp; p.nbT = (Tp + 63) / 64;
+        p.tiles_m = (Cin + 128 * mt - 1) / (128 * mt);
+        p.zero_fill = 1;
+        launch_flat_dt<MODE_DGRAD>(dtype, st->flat_shape, mt, L, st->sm_count, ma, mb, p, nullptr);
+        return;
+    }
     TcParams p{};
     p.out = gu; p.len_out = len_out; p.status = L.status;
     p.M = Cin; p.Ncols = Tp; p.Kdim = Cout; p.B = B; p.Tp = Tp; p.zero_fill = 1;
-    const int mt = Cin > 128 ? 2 : 1;
     dim3 grid((Tp + FWD_BN - 1) / FWD_BN, (Cin + 128 * mt - 1) / (128 * mt), B);
-    if (st->persistent) {
-        if (mt == 2) launch_persistent_dt<MODE_DGRAD, 2, FWD_BN, 3>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
-        else launch_persistent_dt<MODE_DGRAD, 1, FWD_BN, 6>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
-    } else if (mt == 2) launch_dt<MODE_DGRAD, 2, FWD_BN, 2>(dtype, L, grid, ma, mb, p);
-    else launch_dt<MODE_DGRAD, 1, FWD_BN, 3>(dtype, L, grid, ma, mb, p);
+    if (mt == 2) launch_persistent_dt<MODE_DGRAD, 2, FWD_BN, 3>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
+    else launch_persistent_dt<MODE_DGRAD, 1, FWD_BN, 6>(dtype, L, st->sm_count, ma, mb, p, grid.x, grid.y, B);
 }
 
 void tc_gemm_wgrad(const TcState* st, const Launch& L, int dtype, const void* gv, const void* u, float* dw,

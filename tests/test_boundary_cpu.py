@@ -44,7 +44,9 @@ def test_strerror_and_workspace_sizes(api):
     d = api.block_desc(si.config(2).layers[0], 32, 400, "f16")
     f, b = api.sepconv_workspace_bytes(d)
     assert f > 0 and b > 32 * 256 * 400 * 2
-    d.K = 4
+    d.K = 4                                     # even K is a supported variant
+    assert api.sepconv_workspace_bytes(d)[0] > 0
+    d.K = 0
     with pytest.raises(api.SepconvError) as e:
         api.sepconv_workspace_bytes(d)
     assert e.value.code == -6
@@ -65,6 +67,21 @@ def test_encoder_spec_layout(api):
     bad = [si.LayerCfg(8, 16, K=3, residual="identity")]
     with pytest.raises(api.SepconvError):
         api.encoder_workspace_bytes(api.EncoderSpec(bad, 2, 32, "f32"))
+
+
+def test_overlapping_residual_spans_are_rejected(api):
+    """One pending residual gradient at a time: nested spans or a shared source cannot be represented."""
+    import synth_inputs as si
+    plain = si.LayerCfg(8, 8, K=3)
+    def res(j):
+        return si.LayerCfg(8, 8, K=3, residual="identity", res_from=j)
+    ok = [plain, plain, res(1), plain, res(3)]
+    assert api.encoder_workspace_bytes(api.EncoderSpec(ok, 2, 32, "f32")) > 0
+    for bad in ([plain, plain, plain, res(2), plain, res(1)],       # nested: [2,3] inside [1,5]
+                [plain, plain, res(1), res(1)]):                     # two layers share source 1
+        with pytest.raises(api.SepconvError) as e:
+            api.encoder_workspace_bytes(api.EncoderSpec(bad, 2, 32, "f32"))
+        assert e.value.code == -6
 
 
 def test_missing_library_fails_loudly(api, tmp_path):
