@@ -227,13 +227,21 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--gemm-mode", type=int, default=0)
     ap.add_argument("--tile-shape", type=int, default=None, help="tile shape of the pointwise contractions (0, 1, 2)")
+    ap.add_argument("--dp", action="store_true",
+                    help="with N > 1 ranks: data-parallel step -- every rank its own batch, per-replica batch statistics, "
+                         "and an NCCL all-reduce of the gradient blob inside the step (default: independent replicas)")
+    ap.add_argument("--no-pdl", action="store_true", help="launch kernels without programmatic stream serialization")
     ap.add_argument("--no-overlap", action="store_true",
                     help="every kernel on one stream in program order (default: weight gradients and the residual "
                          "projection overlap the critical path on the library's second stream)")
-    ap.add_argument("--no-graph", action="store_true",
-                    help="launch every kernel from the host each step instead of replaying a captured CUDA graph")
+    ap.add_argument("--graph", action="store_true",
+                    help="replay the step as a captured CUDA graph (default: every kernel launched from the host each step "
+                         "with programmatic dependent launch, which measured faster: a kernel's set-up then overlaps the "
+                         "previous kernel's tail, and stream capture drops that overlap)")
+    ap.add_argument("--no-graph", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    args.no_graph = not args.graph
     if args.impl == "reference":
         run_reference(args)
         return
@@ -258,7 +266,7 @@ def main():
     d = si.draw(w)
     ctx = api.Context(local)
     ctx.set_gemm_mode(args.gemm_mode)
-    ctx.set_overlap(not args.no_overlap)
+    ctx.set_overlap(not args.no_overlap, not args.no_pdl)
     if args.tile_shape is not None:
         ctx.set_tile_shape(args.tile_shape)
     spec = api.EncoderSpec(w.layers, w.B, w.T, w.dtype)
@@ -276,8 +284,15 @@ def main():
     grads_h = torch.empty(spec.grad_bytes, dtype=torch.uint8).pin_memory()
     stream = torch.cuda.current_stream()
 
+    dp_exchange = args.dp and world > 1
+    if dp_exchange:
+        from paper_1909_09577_b200 import data_parallel as dp
+        args.no_graph = True          # the collective is launched from the host every step
+
     def step():
         api.encoder_fwd_bwd(ctx, spec, x_d, len_d, blob, g_d, grads_blob=grads, workspace=ws, logits=logits)
+        if dp_exchange:
+            dp.all_reduce_gradients(grads)
 
     def step_e2e():
         x_d.copy_(x_h, non_blocking=True)
@@ -334,17 +349,34 @@ def main():
     ms, t0, t1 = timed(step, args.steps)
     launches = (ctx.launch_count() - l0) if args.no_graph else launches_per_step * args.steps
     clocks = sampler.stop(t0, t1) if sampler else None
+    other_ms = None
+    if args.no_graph and not dp_exchange:
+        # for context: the same K steps replayed as one captured CUDA graph (no per-launch host cost, but stream
+        # capture turns the programmatic launch dependencies into full ones)
+        try:
+            graph = torch.cuda.CUDAGraph()
+            cap_stream = torch.cuda.Stream()
+            cap_stream.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.graph(graph, stream=cap_stream):
+                api.encoder_fwd_bwd(ctx, spec, x_d, len_d, blob, g_d, grads_blob=grads, workspace=ws, logits=logits,
+                                    stream=cap_stream)
+            for _ in range(3):
+                graph.replay()
+            other_ms, _, _ = timed(graph.replay, args.steps)
+            other_ms /= args.steps
+        except Exception as e:      # the comparison figure is optional
+            other_ms = None
     # Per-kernel-class CUDA-event brackets cannot sit inside a replayed graph: every class is timed right
     # after the timed region, same buffers and kernels, launched one by one from the host.
     # The profiled steps run every kernel alone, in program order (overlap off): a class's time is its kernels'
     # own duration, not that of whatever shared the GPU with them.
     nprof = max(3, args.steps // 4)
-    ctx.set_overlap(False)
+    ctx.set_overlap(False, False)
     ctx.profile_begin("all", max_launches=600 * nprof)
     for _ in range(nprof):
         (step if args.no_graph else eager_step)()
     prof = ctx.profile_end()
-    ctx.set_overlap(not args.no_overlap)
+    ctx.set_overlap(not args.no_overlap, not args.no_pdl)
 
     # ---- end to end: pinned host inputs in, logits + gradients out, every step --------------------
     if args.no_e2e:
@@ -369,8 +401,10 @@ def main():
             "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
             "config": {"workload": w.name, "B": w.B, "T_in": w.T, "layers": len(w.layers),
                        "valid_frames": int(d.lengths.sum()), "l2": "per-step working set (GBs) exceeds L2",
-                       "parallelism": "replicas" if world > 1 else "single",
-                       "launch": "host launches" if args.no_graph else "CUDA graph replay",
+                       "parallelism": ("dp%d: per-replica batch statistics, gradient all-reduce (NCCL)" % world) if dp_exchange
+                       else ("replicas" if world > 1 else "single"),
+                       "launch": "host launches, programmatic dependent launch" if args.no_graph else "CUDA graph replay",
+                       "graph_replay_ms_per_step": other_ms,
                        "overlap": "off" if args.no_overlap else "weight gradients and residual projection on a second stream"},
             "clocks": clocks, "gpu_launches": int(launches),
             "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),

@@ -306,12 +306,14 @@ int  sepconv_set_gemm_mode(sc_ctx* ctx, int mode);
  * depend on it except for the summation order of the batch-norm statistics. */
 int  sepconv_set_tile_shape(sc_ctx* ctx, int shape);
 
-/* Overlap of independent kernels (on by default).  The weight-gradient contractions of a layer and the residual
- * projection's forward contraction do not feed the next kernel of the pass; with overlap on they run on a second
- * stream that the context owns, forked from and joined back into `cuda_stream` with events before the call
- * returns, so to the caller every call still behaves as work enqueued on `cuda_stream` alone (stream capture
- * included).  0 turns it off: every kernel on `cuda_stream`, in program order.  Results are bit-identical either
- * way.  (The paper has no counterpart.) */
+/* Overlap between kernels (both forms on by default; `on` is a bit mask, 3 = both, 0 = neither).
+ * Bit 0: the weight-gradient contractions of a layer and the residual projection's forward contraction do not
+ * feed the next kernel of the pass; they run on a second stream that the context owns, forked from and joined
+ * back into `cuda_stream` with events before the call returns.  Bit 1: every kernel is launched with
+ * programmatic stream serialization: it may start (set up its barriers, allocate tensor memory) while the
+ * kernel before it drains, and waits for that kernel's completion before it touches global memory.  To the
+ * caller every call still behaves as work enqueued on `cuda_stream` alone (stream capture included), and the
+ * results are bit-identical for every setting.  (The paper has no counterpart.) */
 int  sepconv_set_overlap(sc_ctx* ctx, int on);
 
 /* Number of kernel launches this context has enqueued so far (for reporting; the paper has no

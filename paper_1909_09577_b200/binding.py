@@ -202,9 +202,11 @@ class Context:
         """Enqueues the kernel whose bounded wait must run out (see sepconv.h)."""
         _check(self.lib.sepconv_selftest_bounded_wait(self.h, _stream_ptr(stream)), "sepconv_selftest_bounded_wait")
 
-    def set_overlap(self, on: bool):
-        """Run independent kernels on the context's second stream (default) or everything in program order."""
-        _check(self.lib.sepconv_set_overlap(self.h, int(bool(on))), "sepconv_set_overlap")
+    def set_overlap(self, second_stream: bool = True, dependent_launch: bool = True):
+        """second_stream: independent kernels on the context's second stream; dependent_launch: every kernel
+        launched so that its set-up overlaps the previous kernel's tail.  Both default to on."""
+        _check(self.lib.sepconv_set_overlap(self.h, int(bool(second_stream)) | (int(bool(dependent_launch)) << 1)),
+               "sepconv_set_overlap")
 
     def set_tile_shape(self, shape: int):
         _check(self.lib.sepconv_set_tile_shape(self.h, shape), "sepconv_set_tile_shape")

@@ -26,6 +26,7 @@ struct sc_ctx {
     cudaStream_t side = nullptr;
     cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};   // fork A, fork B, done[2], fwd fork, fwd join
     int overlap = 1;
+    int pdl = 1;          // launch kernels with programmatic stream serialization
 };
 
 namespace sc {
@@ -510,21 +511,23 @@ const char* sepconv_strerror(int s) {
 
 int sepconv_selftest_bounded_wait(sc_ctx* ctx, void* cuda_stream) {
     if (!ctx) return SC_ERR_NULL;
-    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode};
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode, ctx->pdl};
     selftest_bounded_wait(L);
     return finish(ctx);
 }
 
 int sepconv_set_tile_shape(sc_ctx* ctx, int shape) {
     if (!ctx) return SC_ERR_NULL;
-    if (shape < 0 || shape > 2) return SC_ERR_UNSUPPORTED;
+    if (shape < 0 || shape > 3) return SC_ERR_UNSUPPORTED;
     ctx->tc.flat_shape = shape;
     return SC_OK;
 }
 
 int sepconv_set_overlap(sc_ctx* ctx, int on) {
     if (!ctx) return SC_ERR_NULL;
-    ctx->overlap = on ? 1 : 0;
+    if (on < 0 || on > 3) return SC_ERR_UNSUPPORTED;
+    ctx->overlap = on & 1;
+    ctx->pdl = (on >> 1) & 1;
     return SC_OK;
 }
 
@@ -598,7 +601,7 @@ int sepconv_fwd(sc_ctx* ctx, const sc_block_desc* desc, const sc_tensor* x, cons
     FwdScratch f;
     plan_fwd(desc, m, ws, &f, &ctx->tc);
     if (!ws.ok()) return SC_ERR_WORKSPACE;
-    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode};
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode, ctx->pdl};
     BlockIO io{};
     io.x = x->ptr; io.xres = desc->residual != SC_RES_NONE ? (x_res ? x_res->ptr : x->ptr) : nullptr;
     io.y = y->ptr; io.len_in = lengths_dev; io.len_out = f.len_out; io.nvalid = f.nvalid; io.blk_off = f.blk_off;
@@ -653,7 +656,7 @@ int sepconv_infer(sc_ctx* ctx, const sc_block_desc* desc, const sc_tensor* x, co
     InferScratch q;
     plan_infer(desc, m, ws, &q, &ctx->tc);
     if (!ws.ok()) return SC_ERR_WORKSPACE;
-    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode};
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode, ctx->pdl};
     BlockIO io{};
     io.x = x->ptr; io.xres = desc->residual != SC_RES_NONE ? (x_res ? x_res->ptr : x->ptr) : nullptr;
     io.y = y->ptr; io.len_in = lengths_dev; io.len_out = q.f.len_out; io.nvalid = q.f.nvalid; io.blk_off = q.f.blk_off;
@@ -694,7 +697,7 @@ int sepconv_bwd(sc_ctx* ctx, const sc_block_desc* desc, const sc_tensor* dy, con
     BwdScratch s;
     plan_bwd(desc, m, ws, &s, &ctx->tc);
     if (!ws.ok()) return SC_ERR_WORKSPACE;
-    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode};
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode, ctx->pdl};
     lengths(L, lengths_dev, m.B, m.T, m.s, s.len_out, s.nvalid, s.blk_off);
     BwdIO io{};
     io.dy = dy->ptr; io.x = x->ptr; io.y = y->ptr;
@@ -842,7 +845,7 @@ int encoder_infer(sc_ctx* ctx, const sc_encoder_desc* e, const sc_tensor* x, con
     const int dt = P.L[0].d.io_dtype;
     SC_TRY(check_tensor(x, dt, m0.B, m0.Cin, m0.T));
     SC_TRY(check_tensor(out, dt, ml.B, ml.Cout, ml.Tp));
-    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode};
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode, ctx->pdl};
     auto input_of = [&](int i) -> const void* { return i == 0 ? x->ptr : P.L[i - 1].y; };
     auto res_src = [&](int i) -> int { return (e->res_from && e->res_from[i] >= 0) ? e->res_from[i] : i; };
     auto stat = [&](int i, int j) -> const float* {
@@ -898,7 +901,7 @@ int encoder_fwd_bwd(sc_ctx* ctx, const sc_encoder_desc* e, const sc_tensor* x, c
         SC_TRY(check_params(&P.L[i].d, &prm[i]));
         SC_TRY(check_grads(&P.L[i].d, &grd[i]));
     }
-    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode};
+    Launch L{(cudaStream_t)cuda_stream, ctx->status_dev, &ctx->launches, &ctx->prof, ctx->gemm_mode, ctx->pdl};
     auto input_of = [&](int i) -> const void* { return i == 0 ? x->ptr : P.L[i - 1].y; };
     auto len_in_of = [&](int i) -> const int* { return i == 0 ? lengths_dev : P.L[i - 1].len_out; };
     auto res_src = [&](int i) -> int { return (e->res_from && e->res_from[i] >= 0) ? e->res_from[i] : i; };

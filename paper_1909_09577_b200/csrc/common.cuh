@@ -57,6 +57,26 @@ template <> __device__ __forceinline__ float round_io<__nv_bfloat16>(float v) { 
 // must be the same bit on every path.
 __device__ __forceinline__ float bn_norm(float v, float mu, float is) { return __fmul_rn(__fsub_rn(v, mu), is); }
 
+// Two-wide fp32 arithmetic (one instruction for a pair of floats; each lane rounds like the scalar
+// instruction, so a value computed here equals the one computed by the scalar helper above).
+namespace pk {
+__device__ __forceinline__ uint64_t pack(float a, float b) { uint64_t r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b)); return r; }
+__device__ __forceinline__ void unpack(uint64_t r, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(r)); }
+__device__ __forceinline__ uint64_t add(uint64_t a, uint64_t b) { uint64_t r; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ uint64_t mul(uint64_t a, uint64_t b) { uint64_t r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ uint64_t fma(uint64_t a, uint64_t b, uint64_t c) { uint64_t r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
+// (v - mu) * is for a pair: nmu = pack(-mu, -mu), is2 = pack(is, is); same bits as bn_norm on each lane
+__device__ __forceinline__ uint64_t bn_norm2(uint64_t v, uint64_t nmu, uint64_t is2) { return mul(add(v, nmu), is2); }
+}  // namespace pk
+
+// Is the value, once rounded to the storage type T, greater than zero?  Rounding to nearest even sends
+// everything up to half the smallest subnormal to zero, so the test is a comparison with that constant:
+// the same decision as round_io<T>(a) > 0 without the two conversions.
+template <typename T> __device__ __forceinline__ bool rounds_positive(float a);
+template <> __device__ __forceinline__ bool rounds_positive<float>(float a) { return a > 0.f; }
+template <> __device__ __forceinline__ bool rounds_positive<__half>(float a) { return a > 0x1p-25f; }
+template <> __device__ __forceinline__ bool rounds_positive<__nv_bfloat16>(float a) { return a > 0x1p-134f; }
+
 // Rounds the first n of 8 consecutive values to the storage type with error diffusion: the rounding
 // residual of one element is added to the next before it is rounded, so the residuals of a vector do
 // not add up.  Plain rounding is biased whenever the values sit on a lattice that the storage grid
@@ -152,6 +172,17 @@ __device__ __forceinline__ void chan_merge(float& n, float& mean, float& m2, flo
     m2 += m2b + d * d * (n * nb / nt);
     n = nt;
 }
+
+// Programmatic dependent launch.  Every kernel of the library is launched so that it may start while the
+// kernel before it on the stream is still draining; it therefore (1) tells the runtime right away that its own
+// dependents may be launched -- the trigger fires once every CTA has said so, i.e. when the last wave is on
+// the SMs -- and (2) waits for the kernels before it to complete, with their writes visible, before it reads
+// or writes global memory.  Work placed before pdl_wait() (barrier set-up, tensor-memory allocation,
+// descriptor prefetch) overlaps the previous kernel's tail.  Both are no-ops in a kernel launched without
+// the attribute.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_sync() { pdl_launch_dependents(); pdl_wait(); }
 
 __device__ __forceinline__ void raise_status(int* status, int code) {
     if (status) atomicCAS(status, 0, code);

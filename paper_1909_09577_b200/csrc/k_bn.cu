@@ -43,6 +43,7 @@ __device__ __forceinline__ float block_max(float v) { return warp_max(v); }
 __global__ void lengths_kernel(const int* __restrict__ len_in, int B, int T_in, int stride,
                                int* __restrict__ len_out, int* __restrict__ nvalid, int* __restrict__ blk_off,
                                int* status) {
+    pdl_sync();
     // single CTA; B is small (<= a few thousand)
     __shared__ int total;
     if (threadIdx.x == 0) total = 0;
@@ -71,6 +72,7 @@ template <typename T>
 __global__ void __launch_bounds__(kRowThreads)
 bn_stats_kernel(const T* __restrict__ v, const int* __restrict__ len_out, int nrows, int C, int Tp,
                 float2* __restrict__ partials) {
+    pdl_sync();
     SC_ROW_SETUP(nrows)
     const int b = row / C;
     const int len = min(len_out[b], Tp);
@@ -109,6 +111,7 @@ bn_finalize_kernel(const float2* __restrict__ partials, int parts_per_b, int til
                    const int* __restrict__ len_out, const int* __restrict__ nvalid, int B,
                    int C, float eps, float momentum, float* __restrict__ mean_out,
                    float* __restrict__ invstd_out, float* running_mean, float* running_var) {
+    pdl_sync();
     __shared__ float2 s_red[kFinWarps][32];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int o = blockIdx.x * 32 + lane;
@@ -143,21 +146,23 @@ bn_finalize_kernel(const float2* __restrict__ partials, int parts_per_b, int til
     s_red[w][lane] = make_float2(s1, q);
     __syncthreads();
     if (w != 0 || !act) return;
-    const double N = (double)(*nvalid);
-    const double c = (double)(partials[o].x / (float)max(1, count_of(0)));
-    double t = 0.0, m2 = 0.0;
+    // the tail runs in float: a double divide and square root would cost this latency-bound kernel more than the
+    // whole merge, and the pivot keeps the subtraction below free of cancellation
+    const float N = (float)(*nvalid);
+    const float c = partials[o].x / (float)max(1, count_of(0));
+    float t = 0.f, m2 = 0.f;
 #pragma unroll
-    for (int i = 0; i < kFinWarps; ++i) { t += (double)s_red[i][lane].x; m2 += (double)s_red[i][lane].y; }
-    const double mean = N > 0 ? t / N : 0.0;
-    double var = N > 0 ? (m2 - N * (mean - c) * (mean - c)) / N : 0.0;
-    var = var > 0.0 ? var : 0.0;
-    const float invstd = (float)(1.0 / sqrt(var + (double)eps));
-    mean_out[o] = (float)mean;
-    invstd_out[o] = invstd;
-    if (running_mean) running_mean[o] = (1.f - momentum) * running_mean[o] + momentum * (float)mean;
+    for (int i = 0; i < kFinWarps; ++i) { t += s_red[i][lane].x; m2 += s_red[i][lane].y; }
+    const float mean = N > 0.f ? t / N : 0.f;
+    const float dm = mean - c;
+    float var = N > 0.f ? (m2 - N * dm * dm) / N : 0.f;
+    var = fmaxf(var, 0.f);
+    mean_out[o] = mean;
+    invstd_out[o] = 1.f / sqrtf(var + eps);
+    if (running_mean) running_mean[o] = (1.f - momentum) * running_mean[o] + momentum * mean;
     if (running_var) {
-        double unb = N > 1 ? var * (N / (N - 1.0)) : var;
-        running_var[o] = (1.f - momentum) * running_var[o] + momentum * (float)unb;
+        const float unb = N > 1.f ? var * (N / (N - 1.f)) : var;
+        running_var[o] = (1.f - momentum) * running_var[o] + momentum * unb;
     }
 }
 
@@ -169,6 +174,7 @@ bn_finalize_flat_kernel(const float4* __restrict__ partials, int G, int tiles_m,
                         const int* __restrict__ blk_off, const int* __restrict__ nvalid, int B, int C, float eps,
                         float momentum, float* __restrict__ mean_out, float* __restrict__ invstd_out,
                         float* running_mean, float* running_var) {
+    pdl_sync();
     __shared__ float2 s_red[kFinWarps][32];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int o = blockIdx.x * 32 + lane;
@@ -177,11 +183,14 @@ bn_finalize_flat_kernel(const float4* __restrict__ partials, int G, int tiles_m,
     const long long U = (long long)tiles_m * nblk;
     const int m = min(o, C - 1) / rows_per_tile;
     const long long lo = m * nblk, hi = lo + nblk;
+    const bool small = U * (G + 1) < (1ll << 31);      // the same quotients in 32-bit arithmetic (no 64-bit divisions)
     auto takes_part = [&](int c) -> bool {
-        const long long b0 = U * c / G, b1 = U * (c + 1) / G;
+        long long b0, b1;
+        if (small) { b0 = (uint32_t)U * (uint32_t)c / (uint32_t)G; b1 = (uint32_t)U * (uint32_t)(c + 1) / (uint32_t)G; }
+        else { b0 = U * c / G; b1 = U * (c + 1) / G; }
         return max(b0, lo) < min(b1, hi);
     };
-    int c_first = U > 0 ? (int)(lo * G / U) : 0;
+    int c_first = U > 0 ? (small ? (int)((uint32_t)lo * (uint32_t)G / (uint32_t)U) : (int)(lo * G / U)) : 0;
     while (c_first < G - 1 && !takes_part(c_first)) ++c_first;
     float pivot = 0.f;
     if (act && U > 0) { const float4 pv = partials[(size_t)c_first * C + o]; pivot = pv.x > 0.f ? pv.y / pv.x : 0.f; }
@@ -207,24 +216,26 @@ bn_finalize_flat_kernel(const float4* __restrict__ partials, int G, int tiles_m,
     s_red[w][lane] = make_float2(s1, q);
     __syncthreads();
     if (w != 0 || !act) return;
-    const double N = (double)(*nvalid);
-    double t = 0.0, m2 = 0.0;
+    const float N = (float)(*nvalid);
+    float t = 0.f, m2 = 0.f;
 #pragma unroll
-    for (int i = 0; i < kFinWarps; ++i) { t += (double)s_red[i][lane].x; m2 += (double)s_red[i][lane].y; }
-    const double mean = N > 0 ? t / N : 0.0;
-    double var = N > 0 ? (m2 - N * (mean - (double)pivot) * (mean - (double)pivot)) / N : 0.0;
-    var = var > 0.0 ? var : 0.0;
-    mean_out[o] = (float)mean;
-    invstd_out[o] = (float)(1.0 / sqrt(var + (double)eps));
-    if (running_mean) running_mean[o] = (1.f - momentum) * running_mean[o] + momentum * (float)mean;
+    for (int i = 0; i < kFinWarps; ++i) { t += s_red[i][lane].x; m2 += s_red[i][lane].y; }
+    const float mean = N > 0.f ? t / N : 0.f;
+    const float dm = mean - pivot;
+    float var = N > 0.f ? (m2 - N * dm * dm) / N : 0.f;
+    var = fmaxf(var, 0.f);
+    mean_out[o] = mean;
+    invstd_out[o] = 1.f / sqrtf(var + eps);
+    if (running_mean) running_mean[o] = (1.f - momentum) * running_mean[o] + momentum * mean;
     if (running_var) {
-        double unb = N > 1 ? var * (N / (N - 1.0)) : var;
-        running_var[o] = (1.f - momentum) * running_var[o] + momentum * (float)unb;
+        const float unb = N > 1.f ? var * (N / (N - 1.f)) : var;
+        running_var[o] = (1.f - momentum) * running_var[o] + momentum * unb;
     }
 }
 
 template <typename T, typename NT>
 __global__ void __launch_bounds__(kRowThreads) bn_apply_kernel(ApplyArgs a) {
+    pdl_sync();
     SC_ROW_SETUP(a.B * a.C)
     const int b = row / a.C, o = row % a.C;
     const int Tp = a.Tp, len = min(a.len_out[b], Tp);
@@ -329,6 +340,7 @@ __device__ __forceinline__ size_t bwd_part_index(const BnBwdArgs& a, int b, int 
 
 template <typename T, typename NT>
 __global__ void __launch_bounds__(kRowThreads) bn_bwd_reduce_kernel(BnBwdArgs a) {
+    pdl_sync();
     SC_ROW_SETUP(a.B * a.C)
     const int b = row / a.C, o = row % a.C;
     BwdRow<T, NT> R(a, row, b, o);
@@ -358,6 +370,7 @@ constexpr int kBwdMaxSlotsUnrolled = 8;
 __global__ void __launch_bounds__(32 * kFinWarps)
 bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const float* gamma_r, float* dgamma, float* dbeta,
                        float* dgamma_r, float* dbeta_r, float* dbias, int accumulate) {
+    pdl_sync();
     __shared__ float4 s_sum[kFinWarps][32];
     __shared__ float s_max[kFinWarps][32];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -392,7 +405,7 @@ bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const float* gamma_r, fl
     s_max[w][lane] = amax;
     __syncthreads();
     if (w != 0 || !act) return;
-    double d0 = 0, d1 = 0, d2 = 0, d3 = 0;
+    float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
     amax = 0.f;
 #pragma unroll
     for (int i = 0; i < kFinWarps; ++i) {
@@ -412,8 +425,8 @@ bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const float* gamma_r, fl
                                      (amax + fabsf((float)d2) / N + sqrtf(N) * fabsf((float)d3) / N));
         if (bound < 3.0e38f) atomicMax(reinterpret_cast<unsigned int*>(a.gmax), __float_as_uint(bound));
     }
-    auto put = [&](float* dst, double val) {
-        if (dst) dst[o] = accumulate ? dst[o] + (float)val : (float)val;
+    auto put = [&](float* dst, float val) {
+        if (dst) dst[o] = accumulate ? dst[o] + val : val;
     };
     if (a.has_bn) {
         put(dbeta, d0); put(dgamma, d1);
@@ -430,6 +443,7 @@ bn_bwd_finalize_kernel(BnBwdArgs a, const float* gamma, const float* gamma_r, fl
 
 template <typename T, typename NT, typename GT>
 __global__ void __launch_bounds__(kRowThreads) bn_bwd_apply_kernel(BnBwdArgs a) {
+    pdl_sync();
     SC_ROW_SETUP(a.B * a.C)
     const int b = row / a.C, o = row % a.C;
     BwdRow<T, NT> R(a, row, b, o);
@@ -486,11 +500,186 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_apply_kernel(BnBwdArgs a) 
     }
 }
 
+// One 8-frame vector of the forward apply step: y = [t < len] * relu(gamma * vhat + beta (+ r)); n = frames of the
+// vector inside the sample (0: wholly padding), rv / rr = the raw 16 bytes of v and of the residual operand.
+template <typename T, typename NT, int RES>
+__device__ __forceinline__ void apply_vec(const ApplyArgs& a, int o, int n, size_t off, const uint4& rv, const uint4& rr) {
+    float out[8];
+    if (n > 0) {
+        float f[8], r[8];
+        cvt8<NT>(rv, f);
+        if (RES == 1) cvt8<T>(rr, r);
+        if (RES == 2) cvt8<NT>(rr, r);
+        const float mu = a.mean[o], is = a.invstd[o], ga = a.gamma[o], be = a.beta[o];
+        float mur = 0.f, isr = 0.f, gar = 0.f, ber = 0.f;
+        if (RES == 2) { mur = a.mean_r[o]; isr = a.invstd_r[o]; gar = a.gamma_r[o]; ber = a.beta_r[o]; }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float rres = 0.f;
+            if (RES == 1) rres = r[i];
+            if (RES == 2) rres = fmaf(gar, bn_norm(r[i], mur, isr), ber);
+            const float q = fmaxf(fmaf(ga, bn_norm(f[i], mu, is), be) + rres, 0.f);
+            out[i] = i < n ? q : 0.f;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) out[i] = 0.f;
+    }
+    st8<T>((T*)a.y + off, out);
+}
+
+// One 8-frame vector of the backward apply step (gv and the residual branch's gradient), computed and stored.
+template <typename T, typename NT, typename GT, int RES>
+__device__ __forceinline__ void bwd_apply_vec(const BnBwdArgs& a, int o, int n, size_t off, float sc, bool fold,
+                                              const uint4& rg, const uint4& rv, const uint4& rr, const uint4& ry) {
+    float o1[8], o2[8];
+    if (n > 0) {
+        float g[8], y[8], vn[8], vnr[8];
+        cvt8<T>(rg, g);
+        cvt8<NT>(rv, vn);
+        const float mu = a.mean[o], is = a.invstd[o];
+        const uint64_t nmu2 = pk::pack(-mu, -mu), is2 = pk::pack(is, is);
+        uint64_t vn2[4], vr2[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) vn2[q] = pk::bn_norm2(pk::pack(vn[2 * q], vn[2 * q + 1]), nmu2, is2);
+        if (RES == 2) {
+            cvt8<NT>(rr, vnr);
+            const float mur = a.mean_r[o], isr = a.invstd_r[o];
+            const uint64_t nmur2 = pk::pack(-mur, -mur), isr2 = pk::pack(isr, isr);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) vr2[q] = pk::bn_norm2(pk::pack(vnr[2 * q], vnr[2 * q + 1]), nmur2, isr2);
+        }
+        bool gate[8];
+        if (RES == 0) {
+            // without a residual the forward output is relu(gamma * vhat + beta), rounded to the
+            // activation type: the gate is recomputed from v and the output need not be read
+            const float ga_ = a.gamma[o], be_ = a.beta[o];
+            const uint64_t ga2 = pk::pack(ga_, ga_), be2 = pk::pack(be_, be_);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                float a0, a1;
+                pk::unpack(pk::fma(ga2, vn2[q], be2), a0, a1);
+                gate[2 * q] = rounds_positive<T>(a0); gate[2 * q + 1] = rounds_positive<T>(a1);
+            }
+        } else {
+            cvt8<T>(ry, y);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) gate[i] = y[i] > 0.f;
+        }
+        // gv = k (ga - c1 - c2 vhat) as two fused multiply-adds; when gv itself is the scaled half tensor the
+        // power-of-two scale is folded into k (exact)
+        const float4 cf = a.coef[o];
+        const float kx = (fold ? sc : 1.f) * cf.x;
+        const uint64_t kx2 = pk::pack(kx, kx), k02 = pk::pack(-kx * cf.y, -kx * cf.y), k22 = pk::pack(-kx * cf.z, -kx * cf.z);
+        uint64_t kr2 = 0, r02 = 0, r22 = 0;
+        if (RES == 2) {
+            const float4 cr = a.coef_r[o];
+            kr2 = pk::pack(cr.x, cr.x); r02 = pk::pack(-cr.x * cr.y, -cr.x * cr.y); r22 = pk::pack(-cr.x * cr.z, -cr.x * cr.z);
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const bool in0 = 2 * q < n, in1 = 2 * q + 1 < n;
+            const float g0 = (in0 && gate[2 * q]) ? g[2 * q] : 0.f;
+            const float g1 = (in1 && gate[2 * q + 1]) ? g[2 * q + 1] : 0.f;
+            const uint64_t ga2 = pk::pack(g0, g1);
+            float x0, x1;
+            pk::unpack(pk::fma(k22, vn2[q], pk::fma(kx2, ga2, k02)), x0, x1);
+            o1[2 * q] = in0 ? x0 : 0.f; o1[2 * q + 1] = in1 ? x1 : 0.f;
+            if (RES == 2) {
+                pk::unpack(pk::fma(r22, vr2[q], pk::fma(kr2, ga2, r02)), x0, x1);
+                o2[2 * q] = in0 ? x0 : 0.f; o2[2 * q + 1] = in1 ? x1 : 0.f;
+            }
+            if (RES == 1) { o2[2 * q] = g0; o2[2 * q + 1] = g1; }
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { o1[i] = 0.f; o2[i] = 0.f; }
+    }
+    if (a.gv16) {            // half copy for the weight gradient; gv itself keeps plain rounding
+        float h[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) h[i] = o1[i] * sc;
+        diffuse8<__half>(h, n);
+        st8<__half>((__half*)a.gv16 + off, h);
+    } else {
+        diffuse8<GT>(o1, n);
+    }
+    if (RES == 2) {
+        if (a.gvr16) {
+            float h[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) h[i] = o2[i] * sc;
+            diffuse8<__half>(h, n);
+            st8<__half>((__half*)a.gvr16 + off, h);
+        } else {
+            diffuse8<T>(o2, n);
+        }
+    }
+    st8<GT>((GT*)a.gv + off, o1);
+    if (RES == 2) st8<T>((T*)a.gvr + off, o2);
+    if (RES == 1) st8<T>((T*)a.gres + off, o2);
+}
+
+// One 8-frame vector of the backward reduction: s0 = sum ga, s1 = sum ga * vhat, s3 = sum ga * vhat_r, m = max |ga|
+// over its n (> 0) frames inside the sample.
+template <typename T, typename NT, int RES>
+__device__ __forceinline__ void reduce_vec(const BnBwdArgs& a, int o, int n, const uint4& rg, const uint4& rv, const uint4& rr,
+                                           const uint4& ry, float& s0, float& s1, float& s3, float& m_out) {
+    float g[8], y[8], vn[8], vnr[8];
+    cvt8<T>(rg, g);
+    cvt8<NT>(rv, vn);
+    const float mu = a.mean[o], is = a.invstd[o];
+    const uint64_t nmu2 = pk::pack(-mu, -mu), is2 = pk::pack(is, is);
+    uint64_t vn2[4], vr2[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) vn2[q] = pk::bn_norm2(pk::pack(vn[2 * q], vn[2 * q + 1]), nmu2, is2);
+    if (RES == 2) {
+        cvt8<NT>(rr, vnr);
+        const float mur = a.mean_r[o], isr = a.invstd_r[o];
+        const uint64_t nmur2 = pk::pack(-mur, -mur), isr2 = pk::pack(isr, isr);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) vr2[q] = pk::bn_norm2(pk::pack(vnr[2 * q], vnr[2 * q + 1]), nmur2, isr2);
+    }
+    bool gate[8];
+    if (RES == 0) {          // gate from v (see bn_bwd_apply_fast_kernel)
+        const float ga_ = a.gamma[o], be_ = a.beta[o];
+        const uint64_t ga2 = pk::pack(ga_, ga_), be2 = pk::pack(be_, be_);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            float a0, a1;
+            pk::unpack(pk::fma(ga2, vn2[q], be2), a0, a1);
+            gate[2 * q] = rounds_positive<T>(a0); gate[2 * q + 1] = rounds_positive<T>(a1);
+        }
+    } else {
+        cvt8<T>(ry, y);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) gate[i] = y[i] > 0.f;
+    }
+    uint64_t s0_2 = pk::pack(0.f, 0.f), s1_2 = pk::pack(0.f, 0.f), s3_2 = pk::pack(0.f, 0.f);
+    float m = 0.f;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const float g0 = (2 * q < n && gate[2 * q]) ? g[2 * q] : 0.f;
+        const float g1 = (2 * q + 1 < n && gate[2 * q + 1]) ? g[2 * q + 1] : 0.f;
+        const uint64_t ga2 = pk::pack(g0, g1);
+        s0_2 = pk::add(s0_2, ga2);
+        s1_2 = pk::fma(ga2, vn2[q], s1_2);
+        if (RES == 2) s3_2 = pk::fma(ga2, vr2[q], s3_2);
+        m = fmaxf(m, fmaxf(fabsf(g0), fabsf(g1)));
+    }
+    float t0_, t1_;
+    pk::unpack(s0_2, t0_, t1_); s0 = t0_ + t1_;
+    pk::unpack(s1_2, t0_, t1_); s1 = t0_ + t1_;
+    pk::unpack(s3_2, t0_, t1_); s3 = t0_ + t1_;
+    m_out = m;
+}
+
 // ---- flattened fast paths (the encoder's configuration: BN + ReLU, residual joined before the ReLU,
 // rows a multiple of 8 frames).  A warp takes 32 * V consecutive 8-frame vectors, lane l the vectors
 // l, l + 32, ...: no row tails, and V independent 16-byte loads per tensor in flight per thread.
 template <typename T, typename NT, int RES, int V>
 __global__ void __launch_bounds__(256) bn_apply_fast_kernel(ApplyArgs a, int vpr, long long total) {
+    pdl_sync();
     const uint32_t tid = blockIdx.x * 256u + threadIdx.x;        // the launcher guarantees total < 2^31
     const uint32_t base = (tid >> 5) * (32u * V) + (threadIdx.x & 31), tot = (uint32_t)total;
     size_t off[V]; int nin[V], ch[V];
@@ -516,34 +705,13 @@ __global__ void __launch_bounds__(256) bn_apply_fast_kernel(ApplyArgs a, int vpr
 #pragma unroll
     for (int j = 0; j < V; ++j) {
         if (nin[j] < 0) continue;
-        float out[8];
-        if (nin[j] > 0) {
-            const int o = ch[j];
-            float f[8], r[8];
-            cvt8<NT>(rv[j], f);
-            if (RES == 1) cvt8<T>(rr[j], r);
-            if (RES == 2) cvt8<NT>(rr[j], r);
-            const float mu = a.mean[o], is = a.invstd[o], ga = a.gamma[o], be = a.beta[o];
-            float mur = 0.f, isr = 0.f, gar = 0.f, ber = 0.f;
-            if (RES == 2) { mur = a.mean_r[o]; isr = a.invstd_r[o]; gar = a.gamma_r[o]; ber = a.beta_r[o]; }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                float rres = 0.f;
-                if (RES == 1) rres = r[i];
-                if (RES == 2) rres = fmaf(gar, bn_norm(r[i], mur, isr), ber);
-                const float q = fmaxf(fmaf(ga, bn_norm(f[i], mu, is), be) + rres, 0.f);
-                out[i] = i < nin[j] ? q : 0.f;
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) out[i] = 0.f;
-        }
-        st8<T>((T*)a.y + off[j], out);
+        apply_vec<T, NT, RES>(a, ch[j], nin[j], off[j], rv[j], rr[j]);
     }
 }
 
 template <typename T, typename NT, typename GT, int RES, int V>
 __global__ void __launch_bounds__(256) bn_bwd_apply_fast_kernel(BnBwdArgs a, int vpr, long long total) {
+    pdl_sync();
     const uint32_t tid = blockIdx.x * 256u + threadIdx.x;        // the launcher guarantees total < 2^31
     const uint32_t base = (tid >> 5) * (32u * V) + (threadIdx.x & 31), tot = (uint32_t)total;
     const float sc = a.gmax ? pow2_scale(*a.gmax) : 1.f;          // multiplying by it is exact: a power of two
@@ -572,73 +740,7 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_fast_kernel(BnBwdArgs a, int
 #pragma unroll
     for (int j = 0; j < V; ++j) {
         if (nin[j] < 0) continue;
-        float o1[8], o2[8];
-        const int n = nin[j];
-        if (n > 0) {
-            const int o = ch[j];
-            float g[8], y[8], vn[8], vnr[8];
-            cvt8<T>(rg[j], g);
-            cvt8<NT>(rv[j], vn);
-            const float mu = a.mean[o], is = a.invstd[o];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) vn[i] = bn_norm(vn[i], mu, is);
-            if (RES == 2) {
-                cvt8<NT>(rr[j], vnr);
-                const float mur = a.mean_r[o], isr = a.invstd_r[o];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) vnr[i] = bn_norm(vnr[i], mur, isr);
-            }
-            if (RES == 0) {
-                // without a residual the forward output is relu(gamma * vhat + beta), rounded to the
-                // activation type: the gate is recomputed from v and the output need not be read
-                const float ga_ = a.gamma[o], be_ = a.beta[o];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) y[i] = round_io<T>(fmaf(ga_, vn[i], be_));
-            } else {
-                cvt8<T>(ry[j], y);
-            }
-            // gv = k (ga - c1 - c2 vhat) as two fused multiply-adds; when gv itself is the scaled half tensor the
-            // power-of-two scale is folded into k (exact)
-            const float4 cf = a.coef[o];
-            const float kx = (fold ? sc : 1.f) * cf.x;
-            const float k0 = -kx * cf.y, k2 = -kx * cf.z;
-            float kr = 0.f, r0 = 0.f, r2 = 0.f;
-            if (RES == 2) { const float4 cr = a.coef_r[o]; kr = cr.x; r0 = -kr * cr.y; r2 = -kr * cr.z; }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const bool in = i < n;
-                const float ga = (in && y[i] > 0.f) ? g[i] : 0.f;
-                o1[i] = in ? fmaf(k2, vn[i], fmaf(kx, ga, k0)) : 0.f;
-                if (RES == 2) o2[i] = in ? fmaf(r2, vnr[i], fmaf(kr, ga, r0)) : 0.f;
-                if (RES == 1) o2[i] = ga;
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) { o1[i] = 0.f; o2[i] = 0.f; }
-        }
-        if (a.gv16) {            // half copy for the weight gradient; gv itself keeps plain rounding
-            float h[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) h[i] = o1[i] * sc;
-            diffuse8<__half>(h, n);
-            st8<__half>((__half*)a.gv16 + off[j], h);
-        } else {
-            diffuse8<GT>(o1, n);
-        }
-        if (RES == 2) {
-            if (a.gvr16) {
-                float h[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) h[i] = o2[i] * sc;
-                diffuse8<__half>(h, n);
-                st8<__half>((__half*)a.gvr16 + off[j], h);
-            } else {
-                diffuse8<T>(o2, n);
-            }
-        }
-        st8<GT>((GT*)a.gv + off[j], o1);
-        if (RES == 2) st8<T>((T*)a.gvr + off[j], o2);
-        if (RES == 1) st8<T>((T*)a.gres + off[j], o2);
+        bwd_apply_vec<T, NT, GT, RES>(a, ch[j], nin[j], off[j], sc, fold, rg[j], rv[j], rr[j], ry[j]);
     }
 }
 
@@ -648,6 +750,7 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_fast_kernel(BnBwdArgs a, int
 // summed later in slot order.
 template <typename T, typename NT, int RES, int V>
 __global__ void __launch_bounds__(256) bn_bwd_reduce_fast_kernel(BnBwdArgs a, int vpr, long long total) {
+    pdl_sync();
     const uint32_t tid = blockIdx.x * 256u + threadIdx.x;        // the launcher guarantees total < 2^31
     const int lane = threadIdx.x & 31;
     const uint32_t wg = tid >> 5;                                // global warp index
@@ -681,34 +784,8 @@ __global__ void __launch_bounds__(256) bn_bwd_reduce_fast_kernel(BnBwdArgs a, in
     for (int j = 0; j < V; ++j) {
         const int n = nin[j];
         if (n <= 0) continue;
-        const int o = ch[j];
-        float g[8], y[8], vn[8], vnr[8];
-        cvt8<T>(rg[j], g);
-        cvt8<NT>(rv[j], vn);
-        const float mu = a.mean[o], is = a.invstd[o];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) vn[i] = bn_norm(vn[i], mu, is);
-        if (RES == 2) {
-            cvt8<NT>(rr[j], vnr);
-            const float mur = a.mean_r[o], isr = a.invstd_r[o];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) vnr[i] = bn_norm(vnr[i], mur, isr);
-        }
-        if (RES == 0) {          // gate from v (see bn_bwd_apply_fast_kernel)
-            const float ga_ = a.gamma[o], be_ = a.beta[o];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) y[i] = round_io<T>(fmaf(ga_, vn[i], be_));
-        } else {
-            cvt8<T>(ry[j], y);
-        }
-        float s0 = 0.f, s1 = 0.f, s3 = 0.f, m = 0.f;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float ga = (i < n && y[i] > 0.f) ? g[i] : 0.f;
-            s0 += ga; s1 = fmaf(ga, vn[i], s1);
-            if (RES == 2) s3 = fmaf(ga, vnr[i], s3);
-            m = fmaxf(m, fabsf(ga));
-        }
+        float s0, s1, s3, m;
+        reduce_vec<T, NT, RES>(a, ch[j], n, rg[j], rv[j], rr[j], ry[j], s0, s1, s3, m);
         const int seg = rw[j] != row0 ? 1 : 0;
         acc[seg][0] += s0; acc[seg][1] += s1; acc[seg][2] += s0; acc[seg][3] += s3;
         amx[seg] = fmaxf(amx[seg], m);
@@ -734,6 +811,7 @@ __global__ void __launch_bounds__(256) bn_bwd_reduce_fast_kernel(BnBwdArgs a, in
 template <typename T>
 __global__ void __launch_bounds__(kRowThreads)
 ew_add_masked_kernel(T* out, const T* a, const T* b, const T* c, const int* len, int nrows, int C, int Tt) {
+    pdl_sync();
     SC_ROW_SETUP(nrows)
     const int bb = row / C;
     const int l = min(len[bb], Tt);
@@ -780,15 +858,15 @@ ew_add_masked_kernel(T* out, const T* a, const T* b, const T* c, const int* len,
 
 void lengths(const Launch& L, const int* len_in, int B, int T_in, int stride, int* len_out, int* nvalid, int* blk_off) {
     KScope ks_(L, KC_LENGTHS, 8.0 * B, 0.0);
-    lengths_kernel<<<1, 256, 0, L.stream>>>(len_in, B, T_in, stride, len_out, nvalid, blk_off, L.status);
+    launch_k(L, lengths_kernel, 1, 256, 0, len_in, B, T_in, stride, len_out, nvalid, blk_off, L.status);
     L.count();
 }
 
 void bn_stats(const Launch& L, int vdtype, const void* v, const int* len_out, int B, int C, int Tp,
               float2* partials) {
     KScope ks_(L, KC_BN_STATS, (double)dtype_size(vdtype) * B * C * Tp, 0.0);
-    if (vdtype == F32) bn_stats_kernel<float><<<(B * C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>((const float*)v, len_out, B * C, C, Tp, partials);
-    else bn_stats_kernel<__half><<<(B * C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>((const __half*)v, len_out, B * C, C, Tp, partials);
+    if (vdtype == F32) launch_k(L, bn_stats_kernel<float>, (B * C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, (const float*)v, len_out, B * C, C, Tp, partials);
+    else launch_k(L, bn_stats_kernel<__half>, (B * C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, (const __half*)v, len_out, B * C, C, Tp, partials);
     L.count();
 }
 
@@ -796,7 +874,7 @@ void bn_finalize(const Launch& L, const float2* partials, int parts_per_b, int t
                  const int* nvalid, int B, int C, float eps, float momentum, float* mean, float* invstd,
                  float* running_mean, float* running_var) {
     KScope ks_(L, KC_BN_FINALIZE, 8.0 * B * parts_per_b * C, 0.0);
-    bn_finalize_kernel<<<(C + 31) / 32, 32 * kFinWarps, 0, L.stream>>>(partials, parts_per_b, tile_w, len_out, nvalid, B, C,
+    launch_k(L, bn_finalize_kernel, (C + 31) / 32, 32 * kFinWarps, 0, partials, parts_per_b, tile_w, len_out, nvalid, B, C,
                                                                      eps, momentum, mean, invstd, running_mean, running_var);
     L.count();
 }
@@ -805,7 +883,7 @@ void bn_finalize_flat(const Launch& L, const float4* partials, int grid, int til
                       const int* blk_off, const int* nvalid, int B, int C, float eps, float momentum, float* mean,
                       float* invstd, float* running_mean, float* running_var) {
     KScope ks_(L, KC_BN_FINALIZE, 16.0 * grid * C / std::max(1, tiles_m), 0.0);
-    bn_finalize_flat_kernel<<<(C + 31) / 32, 32 * kFinWarps, 0, L.stream>>>(partials, grid, tiles_m, rows_per_tile, blk_off, nvalid, B,
+    launch_k(L, bn_finalize_flat_kernel, (C + 31) / 32, 32 * kFinWarps, 0, partials, grid, tiles_m, rows_per_tile, blk_off, nvalid, B,
                                                                           C, eps, momentum, mean, invstd, running_mean, running_var);
     L.count();
 }
@@ -824,13 +902,13 @@ void bn_apply(const Launch& L, int dtype, const ApplyArgs& a_in) {
         a.dvpr = FastDiv((uint32_t)vpr); a.dC = FastDiv((uint32_t)a.C);
         const long long total = (long long)a.B * a.C * vpr;
         const unsigned grid = fast_grid(total, 2);
-#define SC_APPLY_FAST(RES) SC_DISPATCH16(dtype, (bn_apply_fast_kernel<T, NT, RES, 2><<<grid, 256, 0, L.stream>>>(a, vpr, total)))
+#define SC_APPLY_FAST(RES) SC_DISPATCH16(dtype, (launch_k(L, bn_apply_fast_kernel<T, NT, RES, 2>, grid, 256, 0, a, vpr, total)))
         if (a.residual == 0) { SC_APPLY_FAST(0); } else if (a.residual == 1) { SC_APPLY_FAST(1); } else { SC_APPLY_FAST(2); }
 #undef SC_APPLY_FAST
         L.count();
         return;
     }
-    SC_DISPATCH3(dtype, (bn_apply_kernel<T, NT><<<(a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>(a)));
+    SC_DISPATCH3(dtype, (launch_k(L, bn_apply_kernel<T, NT>, (a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, a)));
     L.count();
 }
 
@@ -841,21 +919,21 @@ void bn_bwd_reduce(const Launch& L, int dtype, BnBwdArgs& a) {
         a.dvpr = FastDiv((uint32_t)(a.Tp / 8)); a.dC = FastDiv((uint32_t)a.C);
         KScope ks2_(L, KC_BN_BWD_REDUCE, (double)a.B * a.C * a.Tp * (e * (a.residual == 0 ? 1 : 2) + en * (a.residual == 2 ? 2 : 1)), 0.0);
         const int vpr = a.Tp / 8;
-        const int V = vpr >= 64 ? 2 : 1;
-        a.vpw = 32 * V; a.vpw_shift = V == 2 ? 6 : 5;
         a.nslots = bn_bwd_max_slots(a.Tp);
         const long long total = (long long)a.B * a.C * vpr;
+        const int V = vpr >= 64 ? 2 : 1;
+        a.vpw = 32 * V; a.vpw_shift = V == 2 ? 6 : 5;
         const unsigned grid = fast_grid(total, V);
 #define SC_RED_FAST(RES)                                                                                                   \
-        if (V == 2) { SC_DISPATCH16(dtype, (bn_bwd_reduce_fast_kernel<T, NT, RES, 2><<<grid, 256, 0, L.stream>>>(a, vpr, total))); } \
-        else { SC_DISPATCH16(dtype, (bn_bwd_reduce_fast_kernel<T, NT, RES, 1><<<grid, 256, 0, L.stream>>>(a, vpr, total))); }
+        if (V == 2) { SC_DISPATCH16(dtype, (launch_k(L, bn_bwd_reduce_fast_kernel<T, NT, RES, 2>, grid, 256, 0, a, vpr, total))); } \
+        else { SC_DISPATCH16(dtype, (launch_k(L, bn_bwd_reduce_fast_kernel<T, NT, RES, 1>, grid, 256, 0, a, vpr, total))); }
         if (a.residual == 2) { SC_RED_FAST(2); } else if (a.residual == 1) { SC_RED_FAST(1); } else { SC_RED_FAST(0); }
 #undef SC_RED_FAST
         L.count();
         return;
     }
     KScope ks_(L, KC_BN_BWD_REDUCE, (double)a.B * a.C * a.Tp * (e * (a.has_relu && a.res_before_relu ? 2 : 1) + (a.has_bn ? en : 0) + (a.residual == 2 ? en : 0)), 0.0);
-    SC_DISPATCH3(dtype, (bn_bwd_reduce_kernel<T, NT><<<(a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>(a)));
+    SC_DISPATCH3(dtype, (launch_k(L, bn_bwd_reduce_kernel<T, NT>, (a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, a)));
     L.count();
 }
 
@@ -863,7 +941,7 @@ void bn_bwd_finalize(const Launch& L, const BnBwdArgs& a, const float* gamma, co
                      float* dgamma, float* dbeta, float* dgamma_r, float* dbeta_r, float* dbias,
                      int accumulate) {
     KScope ks_(L, KC_BN_BWD_FINALIZE, 16.0 * a.B * a.C * a.nslots, 0.0);
-    bn_bwd_finalize_kernel<<<(a.C + 31) / 32, 32 * kFinWarps, 0, L.stream>>>(a, gamma, gamma_r, dgamma, dbeta, dgamma_r,
+    launch_k(L, bn_bwd_finalize_kernel, (a.C + 31) / 32, 32 * kFinWarps, 0, a, gamma, gamma_r, dgamma, dbeta, dgamma_r,
                                                                           dbeta_r, dbias, accumulate);
     L.count();
 }
@@ -880,39 +958,41 @@ void bn_bwd_apply(const Launch& L, int dtype, const BnBwdArgs& a_in) {
         const unsigned grid = fast_grid(total, 2);
 #define SC_BWD_FAST(RES)                                                                                             \
         if (dtype == BF16 && a.gv_dtype == F16)                                                                      \
-            bn_bwd_apply_fast_kernel<__nv_bfloat16, __half, __half, RES, 2><<<grid, 256, 0, L.stream>>>(a, vpr, total); \
-        else { SC_DISPATCH16(dtype, (bn_bwd_apply_fast_kernel<T, NT, T, RES, 2><<<grid, 256, 0, L.stream>>>(a, vpr, total))); }
+            launch_k(L, bn_bwd_apply_fast_kernel<__nv_bfloat16, __half, __half, RES, 2>, grid, 256, 0, a, vpr, total); \
+        else { SC_DISPATCH16(dtype, (launch_k(L, bn_bwd_apply_fast_kernel<T, NT, T, RES, 2>, grid, 256, 0, a, vpr, total))); }
         if (a.residual == 0) { SC_BWD_FAST(0); } else if (a.residual == 1) { SC_BWD_FAST(1); } else { SC_BWD_FAST(2); }
 #undef SC_BWD_FAST
         L.count();
         return;
     }
     if (dtype == BF16 && a.gv_dtype == F16)
-        bn_bwd_apply_kernel<__nv_bfloat16, __half, __half><<<(a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>(a);
+        launch_k(L, bn_bwd_apply_kernel<__nv_bfloat16, __half, __half>, (a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, a);
     else
-        SC_DISPATCH3(dtype, (bn_bwd_apply_kernel<T, NT, T><<<(a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>(a)));
+        SC_DISPATCH3(dtype, (launch_k(L, bn_bwd_apply_kernel<T, NT, T>, (a.B * a.C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, a)));
     L.count();
 }
 
 void ew_add_masked(const Launch& L, int dtype, void* out, const void* a, const void* b, const void* c,
                    const int* len, int B, int C, int Tt) {
     KScope ks_(L, KC_EW, (double)dtype_size(dtype) * B * C * Tt * (2 + (b ? 1 : 0) + (c ? 1 : 0)), 0.0);
-    SC_DISPATCH(dtype, (ew_add_masked_kernel<T><<<(B * C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, L.stream>>>((T*)out, (const T*)a, (const T*)b,
+    SC_DISPATCH(dtype, (launch_k(L, ew_add_masked_kernel<T>, (B * C + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, (T*)out, (const T*)a, (const T*)b,
                                                                                       (const T*)c, len, B * C, C, Tt)));
     L.count();
 }
 
 __global__ void convert_bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ src, __half* __restrict__ dst, long long n) {
+    pdl_sync();
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) dst[i] = __float2half_rn(__bfloat162float(src[i]));
 }
 void convert_bf16_to_f16(const Launch& L, const void* src, void* dst, int64_t n) {
     KScope ks_(L, KC_EW, 4.0 * n, 0.0);
-    convert_bf16_to_f16_kernel<<<(unsigned)((n + 255) / 256), 256, 0, L.stream>>>((const __nv_bfloat16*)src, (__half*)dst, n);
+    launch_k(L, convert_bf16_to_f16_kernel, (unsigned)((n + 255) / 256), 256, 0, (const __nv_bfloat16*)src, (__half*)dst, n);
     L.count();
 }
 
 __global__ void convert_many_kernel(ConvertList list) {
+    pdl_sync();
     const int item = blockIdx.y;
     const __nv_bfloat16* src = (const __nv_bfloat16*)list.src[item];
     __half* dst = (__half*)list.dst[item];
@@ -925,7 +1005,7 @@ void convert_bf16_to_f16_many(const Launch& L, const ConvertList& list) {
     double total = 0;
     for (int i = 0; i < list.count; ++i) total += list.n[i];
     KScope ks_(L, KC_EW, 4.0 * total, 0.0);
-    convert_many_kernel<<<dim3(64, list.count), 256, 0, L.stream>>>(list);
+    launch_k(L, convert_many_kernel, dim3(64, list.count), 256, 0, list);
     L.count();
 }
 
@@ -934,6 +1014,7 @@ namespace {
 __global__ void __launch_bounds__(256)
 mask_convert_f16_kernel(__half* __restrict__ out, const __nv_bfloat16* __restrict__ in, const int* __restrict__ len,
                         int C, int Tt, long long total, int vec, int* status) {
+    pdl_sync();
     const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
     if (idx >= total) return;
     const int per_row = vec ? Tt / 8 : Tt;
@@ -969,7 +1050,7 @@ void mask_convert_f16(const Launch& L, void* out, const void* in, const int* len
     KScope ks_(L, KC_EW, 4.0 * B * C * Tt, 0.0);
     const int vec = (Tt % 8 == 0) ? 1 : 0;
     const long long total = (long long)B * C * (vec ? Tt / 8 : Tt);
-    mask_convert_f16_kernel<<<(unsigned)((total + 255) / 256), 256, 0, L.stream>>>((__half*)out, (const __nv_bfloat16*)in, len,
+    launch_k(L, mask_convert_f16_kernel, (unsigned)((total + 255) / 256), 256, 0, (__half*)out, (const __nv_bfloat16*)in, len,
                                                                                 C, Tt, total, vec, L.status);
     L.count();
 }

@@ -13,6 +13,7 @@ namespace {
 template <typename T>
 __global__ void __launch_bounds__(256)
 log_softmax_fwd_kernel(const float* __restrict__ z, T* __restrict__ y, const int* __restrict__ len_out, int B, int C, int Tp) {
+    pdl_sync();
     const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
     if (idx >= (long long)B * Tp) return;
     const int b = (int)(idx / Tp), t = (int)(idx - (long long)b * Tp);
@@ -35,6 +36,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 log_softmax_bwd_kernel(T* __restrict__ dz, const T* __restrict__ g, const T* __restrict__ logp,
                        const int* __restrict__ len_out, int B, int C, int Tp) {
+    pdl_sync();
     const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
     if (idx >= (long long)B * Tp) return;
     const int b = (int)(idx / Tp), t = (int)(idx - (long long)b * Tp);
@@ -52,6 +54,7 @@ log_softmax_bwd_kernel(T* __restrict__ dz, const T* __restrict__ g, const T* __r
 }
 
 __global__ void invstd_from_var_kernel(const float* __restrict__ var, float eps, float* __restrict__ invstd, int C) {
+    pdl_sync();
     const int o = blockIdx.x * blockDim.x + threadIdx.x;
     if (o < C) invstd[o] = 1.f / sqrtf(var[o] + eps);
 }
@@ -68,7 +71,7 @@ __global__ void invstd_from_var_kernel(const float* __restrict__ var, float eps,
 void log_softmax_fwd(const Launch& L, int dtype, const float* z, void* y, const int* len_out, int B, int C, int Tp) {
     KScope ks_(L, KC_EW, (4.0 + dtype_size(dtype)) * B * C * Tp, 0.0);
     const unsigned grid = (unsigned)(((long long)B * Tp + 255) / 256);
-    SC_DISPATCH(dtype, (log_softmax_fwd_kernel<T><<<grid, 256, 0, L.stream>>>(z, (T*)y, len_out, B, C, Tp)));
+    SC_DISPATCH(dtype, (launch_k(L, log_softmax_fwd_kernel<T>, grid, 256, 0, z, (T*)y, len_out, B, C, Tp)));
     L.count();
 }
 
@@ -76,13 +79,13 @@ void log_softmax_bwd(const Launch& L, int dtype, void* dz, const void* g, const 
                      int C, int Tp) {
     KScope ks_(L, KC_EW, 3.0 * dtype_size(dtype) * B * C * Tp, 0.0);
     const unsigned grid = (unsigned)(((long long)B * Tp + 255) / 256);
-    SC_DISPATCH(dtype, (log_softmax_bwd_kernel<T><<<grid, 256, 0, L.stream>>>((T*)dz, (const T*)g, (const T*)logp, len_out, B, C, Tp)));
+    SC_DISPATCH(dtype, (launch_k(L, log_softmax_bwd_kernel<T>, grid, 256, 0, (T*)dz, (const T*)g, (const T*)logp, len_out, B, C, Tp)));
     L.count();
 }
 
 void invstd_from_var(const Launch& L, const float* var, float eps, float* invstd, int C) {
     KScope ks_(L, KC_EW, 8.0 * C, 0.0);
-    invstd_from_var_kernel<<<(C + 255) / 256, 256, 0, L.stream>>>(var, eps, invstd, C);
+    launch_k(L, invstd_from_var_kernel, (C + 255) / 256, 256, 0, var, eps, invstd, C);
     L.count();
 }
 

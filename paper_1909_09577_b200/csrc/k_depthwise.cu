@@ -39,6 +39,7 @@ dw_corr_s1_kernel(const TI* __restrict__ in, const TW* __restrict__ w, TO* __res
                   const TO* __restrict__ add1, const TO* __restrict__ add2, const float* __restrict__ gmax,
                   const int* __restrict__ len_src, const int* __restrict__ len_dst,
                   int C, int Tt, int K, int Kpad, int flip, int* status) {
+    pdl_sync();
     using T = TO;
     extern __shared__ float smem[];
     const int lane = threadIdx.x, wrp = threadIdx.y;
@@ -155,6 +156,7 @@ __global__ void __launch_bounds__(GT)
 dw_fwd_generic_kernel(const T* __restrict__ x, const T* __restrict__ w, TO* __restrict__ u,
                       const int* __restrict__ len_in, const int* __restrict__ len_out,
                       int C, int Tt, int Tp, int K, int s, int dil, int* status) {
+    pdl_sync();
     extern __shared__ float smem[];
     const int b = blockIdx.z, c = blockIdx.y, t0 = blockIdx.x * GT;
     const int P = (dil * (K - 1)) / 2, XW = (GT - 1) * s + (K - 1) * dil + 1;
@@ -183,6 +185,7 @@ dw_dgrad_generic_kernel(const TG* __restrict__ gu, const T* __restrict__ w, T* _
                         const T* __restrict__ add1, const T* __restrict__ add2, const float* __restrict__ gmax,
                         const int* __restrict__ len_in, const int* __restrict__ len_out,
                         int C, int Tt, int Tp, int K, int s, int dil) {
+    pdl_sync();
     extern __shared__ float smem[];
     const int b = blockIdx.z, c = blockIdx.y, tau0 = blockIdx.x * GT;
     const int P = (dil * (K - 1)) / 2;
@@ -221,6 +224,7 @@ __global__ void __launch_bounds__(128)
 dw_wgrad_generic_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float* __restrict__ partials,
                         const int* __restrict__ len_in, const int* __restrict__ len_out,
                         int B, int C, int Tt, int Tp, int K, int s, int dil) {
+    pdl_sync();
     const int c = blockIdx.x, lane = threadIdx.x & 31, wrp = threadIdx.x >> 5;
     const int P = (dil * (K - 1)) / 2;
     // partials[b][c][k]; warps stride over samples
@@ -248,6 +252,7 @@ __global__ void __launch_bounds__(128)
 dw_wgrad_strided_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float* __restrict__ partials,
                         const int* __restrict__ len_in, const int* __restrict__ len_out,
                         int C, int Tt, int Tp, int K, int s) {
+    pdl_sync();
     extern __shared__ float smem[];
     const int c = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
     const int P = (K - 1) / 2, XW = (WS_TT - 1) * s + K;
@@ -294,6 +299,7 @@ __global__ void __launch_bounds__(WG_THREADS)
 dw_wgrad_s1_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float* __restrict__ partials,
                    const int* __restrict__ len_in, const int* __restrict__ len_out,
                    int B, int C, int Tt, int K, int Kpad) {
+    pdl_sync();
     extern __shared__ float smem[];
     const int c = blockIdx.x, bg = blockIdx.y;
     const int P = (K - 1) / 2;
@@ -376,6 +382,7 @@ __global__ void __launch_bounds__(WR_THREADS, 3)
 dw_wgrad_reg_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float* __restrict__ partials,
                     const int* __restrict__ len_in, const int* __restrict__ len_out,
                     int B, int C, int Tt, int K, int Ppad, int NR, int NST, int RSP) {
+    pdl_sync();
     extern __shared__ float smem[];
     const int tid = threadIdx.x, lane = tid & 31, wrp = tid >> 5;
     const int c = blockIdx.x;
@@ -496,6 +503,7 @@ __global__ void __launch_bounds__(WR_THREADS, (NCH <= 8 ? 4 : 3))
 dw_wgrad_reg16_kernel(const TG* __restrict__ gu, const T* __restrict__ x, float* __restrict__ partials,
                       const int* __restrict__ len_in, const int* __restrict__ len_out,
                       int B, int C, int Tt, int K, int Ppad, int NR, int NST, int RS) {
+    pdl_sync();
     static_assert(sizeof(TG) == 2 && sizeof(T) == 2, "16-bit tensors only");
     extern __shared__ __align__(16) unsigned short smem16[];
     const int tid = threadIdx.x, lane = tid & 31, wrp = tid >> 5;
@@ -656,13 +664,13 @@ void dw_fwd(const Launch& L, int dtype, int odt, const void* x, const void* wd, 
         const int Kp = kpad(K);
         const size_t smem = (size_t)CH * (host_phys(TT + Kp) + 4 + Kp) * sizeof(float);
         dim3 grid((Tt + TT - 1) / TT, (C + CH - 1) / CH, B), block(32, CH);
-        SC_DISPATCH_IO(dtype, odt, (dw_corr_s1_kernel<T, T, OT><<<grid, block, smem, L.stream>>>(
+        SC_DISPATCH_IO(dtype, odt, (launch_k(L, dw_corr_s1_kernel<T, T, OT>, grid, block, smem, 
                                        (const T*)x, (const T*)wd, (OT*)u, nullptr, nullptr, nullptr, len_in, len_out, C, Tt,
                                        K, Kp, 0, L.status)));
     } else {
         const size_t smem = (size_t)((GT - 1) * s + (K - 1) * dil + 1 + K) * sizeof(float);
         dim3 grid((Tp + GT - 1) / GT, C, B);
-        SC_DISPATCH_IO(dtype, odt, (dw_fwd_generic_kernel<T, OT><<<grid, GT, smem, L.stream>>>(
+        SC_DISPATCH_IO(dtype, odt, (launch_k(L, dw_fwd_generic_kernel<T, OT>, grid, GT, smem, 
                                        (const T*)x, (const T*)wd, (OT*)u, len_in, len_out, C, Tt, Tp, K, s, dil, L.status)));
     }
     L.count();
@@ -682,13 +690,13 @@ void dw_dgrad(const Launch& L, int dtype, int odt, const void* gu, const void* w
         const int Kp = kpad(K);
         const size_t smem = (size_t)CH * (host_phys(TT + Kp) + 4 + Kp) * sizeof(float);
         dim3 grid((Tt + TT - 1) / TT, (C + CH - 1) / CH, B), block(32, CH);
-        SC_DISPATCH_IO(dtype, odt, (dw_corr_s1_kernel<OT, T, T><<<grid, block, smem, L.stream>>>(
+        SC_DISPATCH_IO(dtype, odt, (launch_k(L, dw_corr_s1_kernel<OT, T, T>, grid, block, smem, 
                                        (const OT*)gu, (const T*)wd, (T*)dx, (const T*)add1, (const T*)add2, gmax, len_out,
                                        len_in, C, Tt, K, Kp, 1, L.status)));
     } else {
         const size_t smem = (size_t)((GT + (K - 1) * dil + 1) / s + 4 + K) * sizeof(float);
         dim3 grid((Tt + GT - 1) / GT, C, B);
-        SC_DISPATCH_IO(dtype, odt, (dw_dgrad_generic_kernel<OT, T><<<grid, GT, smem, L.stream>>>(
+        SC_DISPATCH_IO(dtype, odt, (launch_k(L, dw_dgrad_generic_kernel<OT, T>, grid, GT, smem, 
                                        (const OT*)gu, (const T*)wd, (T*)dx, (const T*)add1, (const T*)add2, gmax, len_in,
                                        len_out, C, Tt, Tp, K, s, dil)));
     }
@@ -729,7 +737,7 @@ void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x
             case N: {                                                                                          \
                 auto kern = dw_wgrad_reg_kernel<float, float, N>;                                              \
                 set_max_smem_once<dw_wgrad_reg_kernel<float, float, N>>(64 * 1024);                            \
-                kern<<<grid, WR_THREADS, smem, L.stream>>>((const float*)gu, (const float*)x, partials, len_in, len_out, \
+                launch_k(L, kern, grid, WR_THREADS, smem, (const float*)gu, (const float*)x, partials, len_in, len_out, \
                                                            B, C, Tt, K, Ppad, NR, NST, rsp);                   \
             } break;
             switch (nch) {
@@ -754,17 +762,17 @@ void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x
                 if (dtype == F16) {                                                                            \
                     auto kern = dw_wgrad_reg16_kernel<__half, __half, N>;                                      \
                     set_max_smem_once<dw_wgrad_reg16_kernel<__half, __half, N>>(96 * 1024);   \
-                    kern<<<grid, WR_THREADS, smem, L.stream>>>((const __half*)gu, (const __half*)x, partials, len_in, len_out, \
+                    launch_k(L, kern, grid, WR_THREADS, smem, (const __half*)gu, (const __half*)x, partials, len_in, len_out, \
                                                                B, C, Tt, K, Ppad, NR, NST, RS);               \
                 } else if (odt == F16) {                                                                       \
                     auto kern = dw_wgrad_reg16_kernel<__half, __nv_bfloat16, N>;                               \
                     set_max_smem_once<dw_wgrad_reg16_kernel<__half, __nv_bfloat16, N>>(96 * 1024);   \
-                    kern<<<grid, WR_THREADS, smem, L.stream>>>((const __half*)gu, (const __nv_bfloat16*)x, partials, len_in, len_out, \
+                    launch_k(L, kern, grid, WR_THREADS, smem, (const __half*)gu, (const __nv_bfloat16*)x, partials, len_in, len_out, \
                                                                B, C, Tt, K, Ppad, NR, NST, RS);               \
                 } else {                                                                                       \
                     auto kern = dw_wgrad_reg16_kernel<__nv_bfloat16, __nv_bfloat16, N>;                        \
                     set_max_smem_once<dw_wgrad_reg16_kernel<__nv_bfloat16, __nv_bfloat16, N>>(96 * 1024);   \
-                    kern<<<grid, WR_THREADS, smem, L.stream>>>((const __nv_bfloat16*)gu, (const __nv_bfloat16*)x, partials, len_in, len_out, \
+                    launch_k(L, kern, grid, WR_THREADS, smem, (const __nv_bfloat16*)gu, (const __nv_bfloat16*)x, partials, len_in, len_out, \
                                                                B, C, Tt, K, Ppad, NR, NST, RS);               \
                 }                                                                                              \
             } break;
@@ -781,17 +789,17 @@ void dw_wgrad(const Launch& L, int dtype, int odt, const void* gu, const void* x
         const size_t smem = (size_t)(GW + GW + Kp + nseg * Kp) * sizeof(float);
         nsplit = (B + WG_BG - 1) / WG_BG;
         dim3 grid(C, nsplit);
-        SC_DISPATCH_IO(dtype, odt, (dw_wgrad_s1_kernel<OT, T><<<grid, WG_THREADS, smem, L.stream>>>(
+        SC_DISPATCH_IO(dtype, odt, (launch_k(L, dw_wgrad_s1_kernel<OT, T>, grid, WG_THREADS, smem, 
                                        (const OT*)gu, (const T*)x, partials, len_in, len_out, B, C, Tt, K, Kp)));
     } else if (plain && K <= 128) {
         nsplit = B;
         const size_t smem = (size_t)(WS_TT + (WS_TT - 1) * s + K + 128) * sizeof(float);
         dim3 grid(C, B);
-        SC_DISPATCH_IO(dtype, odt, (dw_wgrad_strided_kernel<OT, T><<<grid, 128, smem, L.stream>>>(
+        SC_DISPATCH_IO(dtype, odt, (launch_k(L, dw_wgrad_strided_kernel<OT, T>, grid, 128, smem, 
                                        (const OT*)gu, (const T*)x, partials, len_in, len_out, C, Tt, Tp, K, s)));
     } else {
         nsplit = B;
-        SC_DISPATCH_IO(dtype, odt, (dw_wgrad_generic_kernel<OT, T><<<C, 128, 0, L.stream>>>(
+        SC_DISPATCH_IO(dtype, odt, (launch_k(L, dw_wgrad_generic_kernel<OT, T>, C, 128, 0, 
                                        (const OT*)gu, (const T*)x, partials, len_in, len_out, B, C, Tt, Tp, K, s, dil)));
     }
     L.count();

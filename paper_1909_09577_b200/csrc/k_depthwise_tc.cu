@@ -47,6 +47,7 @@ dw_tc_kernel(const TI* __restrict__ in, const TW* __restrict__ w, TO* __restrict
              const TO* __restrict__ add1, const TO* __restrict__ add2, const float* __restrict__ gmax,
              const int* __restrict__ len_src, const int* __restrict__ len_dst,
              int B, int C, int Tt, int K, int nb, int* status) {
+    pdl_sync();
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
     uint4* A16 = reinterpret_cast<uint4*>(smem);                        // [8 chunks][ROWS_ALLOC] 16-byte units
@@ -227,7 +228,7 @@ void launch_tc(const Launch& L, const void* in, const void* w, void* out, const 
     const int S = (Tt + NB - 1) / NB + 2;
     const int nb = std::max(1, std::min(B, MAXROWS / S));
     dim3 grid(C, (B + nb - 1) / nb);
-    kern<<<grid, kThreads, kSmemBytes, L.stream>>>((const TI*)in, (const TW*)w, (TO*)out, (const TO*)add1, (const TO*)add2,
+    launch_k(L, kern, grid, kThreads, kSmemBytes, (const TI*)in, (const TW*)w, (TO*)out, (const TO*)add1, (const TO*)add2,
                                                    gmax, len_src, len_dst, B, C, Tt, K, nb, L.status);
     L.count();
 }

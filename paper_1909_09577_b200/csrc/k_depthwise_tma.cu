@@ -86,6 +86,7 @@ __device__ __forceinline__ void named_bar(int id, int nthreads) {
 template <typename TI, typename TW, typename TO>
 __global__ void __launch_bounds__(DT_THREADS, 1)
 dw_tma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapO, DtParams p) {
+    pdl_launch_dependents();
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint8_t* sB = smem + p.nstages * p.stage_bytes;                         // [2][b_stride], 1024-byte aligned
@@ -111,6 +112,7 @@ dw_tma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ 
         ptx::prefetch_tensormap(&mapO);
     }
     if (warp == 0) { ptx::tmem_alloc(tmem_slot, DT_NACC * DT_ACC_COLS); ptx::tmem_relinquish(); }
+    pdl_wait();                                        // everything above overlaps the previous kernel's tail
     ptx::tc_fence_before();
     __syncthreads();
     ptx::tc_fence_after();
@@ -424,7 +426,7 @@ template <typename TI, typename TW, typename TO>
 void launch_dt(const Launch& L, int grid, const CUtensorMap& mx, const CUtensorMap& mo, const DtParams& p) {
     auto kern = dw_tma_kernel<TI, TW, TO>;
     set_max_smem_once<dw_tma_kernel<TI, TW, TO>>(kDtSmem);
-    kern<<<grid, DT_THREADS, kDtSmem, L.stream>>>(mx, mo, p);
+    launch_k(L, kern, grid, DT_THREADS, kDtSmem, mx, mo, p);
     L.count();
 }
 

@@ -116,6 +116,7 @@ struct Ring {
 template <typename TG, typename TX>
 __global__ void __launch_bounds__(WT_THREADS, 1)
 dw_wgrad_tc_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_constant__ CUtensorMap mapX, WtParams p) {
+    pdl_launch_dependents();
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + WT_RING_BYTES);
@@ -143,6 +144,7 @@ dw_wgrad_tc_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_consta
         ptx::prefetch_tensormap(&mapG);
         ptx::prefetch_tensormap(&mapX);
     }
+    pdl_wait();                                        // the barrier set-up above overlaps the previous kernel's tail
     // longest output length in every sample chunk: time blocks past it hold only zeros of gu
     for (int ch = tid; ch < p.nchunks && ch < WT_MAX_CHUNKS; ch += WT_THREADS) {
         int m = 0;
@@ -361,7 +363,7 @@ template <typename TG, typename TX>
 void launch_wt(const Launch& L, int grid, const CUtensorMap& mg, const CUtensorMap& mx, const WtParams& p) {
     auto kern = dw_wgrad_tc_kernel<TG, TX>;
     set_max_smem_once<dw_wgrad_tc_kernel<TG, TX>>(kWtSmem);
-    kern<<<grid, WT_THREADS, kWtSmem, L.stream>>>(mg, mx, p);
+    launch_k(L, kern, grid, WT_THREADS, kWtSmem, mg, mx, p);
     L.count();
 }
 

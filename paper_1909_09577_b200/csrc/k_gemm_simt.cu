@@ -27,6 +27,7 @@ template <typename T, typename OT, int MODE>   // MODE 0: fwd (bias+mask, T out)
 __global__ void __launch_bounds__(NT)
 gemm_simt_kernel(GemmDesc d, const T* __restrict__ a, const T* __restrict__ b, void* __restrict__ out,
                  const float* __restrict__ bias, const int* __restrict__ len_out, int* status) {
+    pdl_sync();
     __shared__ float As[BK][BM + 4];
     __shared__ float Bs[BK][BN + 4];
     const int z = blockIdx.z;
@@ -117,6 +118,7 @@ gemm_simt_kernel(GemmDesc d, const T* __restrict__ a, const T* __restrict__ b, v
 
 __global__ void reduce_partials_kernel(const float* __restrict__ p, int nsplit, long long n,
                                        float* __restrict__ out, int accumulate, const float* __restrict__ gmax) {
+    pdl_sync();
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     float s = 0.f;
@@ -130,6 +132,7 @@ __global__ void reduce_partials_kernel(const float* __restrict__ p, int nsplit, 
 __global__ void __launch_bounds__(256)
 reduce_partials_vec4_kernel(const float4* __restrict__ p, int nsplit, long long n4, float4* __restrict__ out,
                             int accumulate, const float* __restrict__ gmax) {
+    pdl_sync();
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n4) return;
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -163,10 +166,10 @@ void reduce_partials(const Launch& L, const float* partials, int nsplit, int64_t
                      const float* gmax) {
     KScope ks_(L, KC_REDUCE, 4.0 * (nsplit + 1) * n, 0.0);
     if (n % 4 == 0 && (reinterpret_cast<uintptr_t>(partials) & 15) == 0 && (reinterpret_cast<uintptr_t>(out) & 15) == 0)
-        reduce_partials_vec4_kernel<<<(unsigned)((n / 4 + 255) / 256), 256, 0, L.stream>>>(
+        launch_k(L, reduce_partials_vec4_kernel, (unsigned)((n / 4 + 255) / 256), 256, 0, 
             reinterpret_cast<const float4*>(partials), nsplit, n / 4, reinterpret_cast<float4*>(out), accumulate, gmax);
     else
-        reduce_partials_kernel<<<(unsigned)((n + 255) / 256), 256, 0, L.stream>>>(partials, nsplit, n, out, accumulate, gmax);
+        launch_k(L, reduce_partials_kernel, (unsigned)((n + 255) / 256), 256, 0, partials, nsplit, n, out, accumulate, gmax);
     L.count();
 }
 
@@ -179,13 +182,13 @@ void gemm_fwd_simt(const Launch& L, int dtype, const void* w, const void* u, con
     d.b_z = (long long)Cin * Tp; d.b_k = Tp; d.b_n = 1;
     dim3 grid((Tp + BN - 1) / BN, (Cout + BM - 1) / BM, B);
     if (out_dtype == dtype) {
-        SC_DISPATCH(dtype, (gemm_simt_kernel<T, T, 0><<<grid, NT, 0, L.stream>>>(d, (const T*)w, (const T*)u, v, bias, len_out, L.status)));
+        SC_DISPATCH(dtype, (launch_k(L, gemm_simt_kernel<T, T, 0>, grid, NT, 0, d, (const T*)w, (const T*)u, v, bias, len_out, L.status)));
     } else if (dtype == BF16 && out_dtype == F16) {   // bfloat16 operands, float16 result
-        gemm_simt_kernel<__nv_bfloat16, __half, 0><<<grid, NT, 0, L.stream>>>(d, (const __nv_bfloat16*)w, (const __nv_bfloat16*)u, v, bias, len_out, L.status);
+        launch_k(L, gemm_simt_kernel<__nv_bfloat16, __half, 0>, grid, NT, 0, d, (const __nv_bfloat16*)w, (const __nv_bfloat16*)u, v, bias, len_out, L.status);
     } else if (dtype == BF16) {   // 16-bit operands, float result
-        gemm_simt_kernel<__nv_bfloat16, float, 0><<<grid, NT, 0, L.stream>>>(d, (const __nv_bfloat16*)w, (const __nv_bfloat16*)u, v, bias, len_out, L.status);
+        launch_k(L, gemm_simt_kernel<__nv_bfloat16, float, 0>, grid, NT, 0, d, (const __nv_bfloat16*)w, (const __nv_bfloat16*)u, v, bias, len_out, L.status);
     } else {
-        gemm_simt_kernel<__half, float, 0><<<grid, NT, 0, L.stream>>>(d, (const __half*)w, (const __half*)u, v, bias, len_out, L.status);
+        launch_k(L, gemm_simt_kernel<__half, float, 0>, grid, NT, 0, d, (const __half*)w, (const __half*)u, v, bias, len_out, L.status);
     }
     L.count();
 }
@@ -198,7 +201,7 @@ void gemm_dgrad_simt(const Launch& L, int dtype, const void* w, const void* gv, 
     d.a_z = 0; d.a_m = 1; d.a_k = Cin;            // A(m=c, k=o) = w[o*Cin + c]
     d.b_z = (long long)Cout * Tp; d.b_k = Tp; d.b_n = 1;
     dim3 grid((Tp + BN - 1) / BN, (Cin + BM - 1) / BM, B);
-    SC_DISPATCH(dtype, (gemm_simt_kernel<T, T, 1><<<grid, NT, 0, L.stream>>>(d, (const T*)w, (const T*)gv, gu, nullptr, nullptr, nullptr)));
+    SC_DISPATCH(dtype, (launch_k(L, gemm_simt_kernel<T, T, 1>, grid, NT, 0, d, (const T*)w, (const T*)gv, gu, nullptr, nullptr, nullptr)));
     L.count();
 }
 
@@ -220,7 +223,7 @@ void gemm_wgrad_simt(const Launch& L, int dtype, const void* gv, const void* u, 
     d.b_n = Tp; d.b_kz = (long long)Cin * Tp;     // B(k=(b,t), n=c) = u[b,c,t]
     d.k_len_per_z = Tp;
     dim3 grid((Cin + BN - 1) / BN, (Cout + BM - 1) / BM, ns);
-    SC_DISPATCH(dtype, (gemm_simt_kernel<T, T, 2><<<grid, NT, 0, L.stream>>>(d, (const T*)gv, (const T*)u, partials, nullptr, nullptr, nullptr)));
+    SC_DISPATCH(dtype, (launch_k(L, gemm_simt_kernel<T, T, 2>, grid, NT, 0, d, (const T*)gv, (const T*)u, partials, nullptr, nullptr, nullptr)));
     L.count();
     }
     reduce_partials(L, partials, ns, (int64_t)Cin * Cout, dw, accumulate, gmax);

@@ -3,6 +3,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <utility>
 #include <vector>
 
 namespace sc {
@@ -31,8 +32,22 @@ struct Launch {
     int64_t* counter;     // host launch counter
     Prof* prof = nullptr;
     int simt_only = 0;    // 1: never take a tensor-core kernel (used by tests)
+    int pdl = 1;          // 1: launch with programmatic stream serialization (see pdl_sync in common.cuh)
     void count(int n = 1) const { if (counter) *counter += n; }
 };
+
+// Launches `kern` on L.stream; with L.pdl the launch carries the programmatic-stream-serialization attribute, so
+// the kernel may begin (up to its pdl_wait()) before the previous kernel on the stream has completed.
+template <typename K, typename... Args>
+inline void launch_k(const Launch& L, K kern, dim3 grid, dim3 block, size_t smem, Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = L.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = L.pdl ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
 
 // Brackets the launches of one launcher call.  bytes/flops are the algorithmic figures of the call.
 struct KScope {

@@ -99,6 +99,7 @@ __device__ __forceinline__ void store_block_staged(float* stg, const float (&f)[
 template <typename T, int MODE, int MT, int BN, int STAGES>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, TcParams p) {
+    pdl_sync();
     constexpr int A_BYTES = MT * 128 * 128;        // MT sub-tiles of 128 rows x 128 bytes
     constexpr int B_BYTES = BN * 128;
     constexpr int STAGE = A_BYTES + B_BYTES;
@@ -311,6 +312,7 @@ template <typename T, int MODE, int MT, int BN, int STAGES>
 __global__ void __launch_bounds__(32 * (4 * MT + 2), 1)
 tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                           TcParams p, int tiles_n, int tiles_m, int tiles_total) {
+    pdl_sync();
     static_assert(MODE == MODE_FWD || MODE == MODE_DGRAD, "forward / input gradient only");
     constexpr int A_BYTES = MT * 128 * 128;
     constexpr int B_BYTES = BN * 128;
@@ -516,7 +518,7 @@ tc_gemm_persistent_kernel(const __grid_constant__ CUtensorMap mapA, const __grid
 // from the row's first valid frame, and writes one (count, sum, M2) partial per (CTA, channel).
 constexpr int kFlatMaxNB = 4;          // blocks per tile (N up to 256)
 constexpr int kFlatMaxB = 2048;        // samples whose block offsets fit the shared-memory copy
-constexpr int kFlatMaxGrid = 256;
+constexpr int kFlatMaxGrid = 320;
 constexpr int kOutPitch = 80;          // bytes per row of a warp's 32 x 32 staging block of 16-bit values
 constexpr int kOutStageBytes = 32 * kOutPitch;
 
@@ -576,22 +578,26 @@ __device__ __forceinline__ bool flat_next_tile(long long& pos, long long end, in
 
 // Shapes: MT M sub-tiles of 128 rows, NB blocks per tile, NBUF accumulator buffers (MT * NB * 64 * NBUF <= 512
 // tensor-memory columns).  With NBUF = 2 the epilogue of a tile overlaps the MMAs of the next one.
-template <int MT, int NB> struct FlatCfg {
+// OCC = CTAs per SM: with 2, each CTA has a two-stage ring and half of tensor memory, and the two CTAs of an SM
+// cover each other's set-up, pipeline fill and epilogue.
+template <int MT, int NB, int OCC> struct FlatCfg {
     static constexpr int A_BYTES = MT * 128 * 128;
     static constexpr int STAGE = A_BYTES + NB * 8192;
-    static constexpr int STAGES = STAGE <= 49152 ? 4 : 3;
-    // per-warp staging: 32 x 32 16-bit values, or (one M sub-tile only) 32 x 32 floats for a float32 result
-    static constexpr int STG = MT == 1 ? kStgFloatsPerWarp * 4 : kOutStageBytes;
+    static constexpr int STAGES = OCC == 2 ? 2 : (STAGE <= 49152 ? 4 : 3);
+    // per-warp staging: 32 x 32 16-bit values, or (one M sub-tile, one CTA per SM only) 32 x 32 floats for a float32 result
+    static constexpr int STG = (MT == 1 && OCC == 1) ? kStgFloatsPerWarp * 4 : kOutStageBytes;
+    static constexpr int MAXB = OCC == 2 ? 256 : kFlatMaxB;
     static constexpr int smem_bytes(int B) { return STAGES * STAGE + 256 + 4 * MT * STG + (B + 1) * 4 + 1024; }
 };
 
-template <typename T, int MODE, int MT, int NB, int NBUF>
-__global__ void __launch_bounds__(32 * (4 * MT + 2), 1)
+template <typename T, int MODE, int MT, int NB, int NBUF, int OCC>
+__global__ void __launch_bounds__(32 * (4 * MT + 2), OCC)
 tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, FlatParams p) {
+    pdl_launch_dependents();
     static_assert(MODE == MODE_FWD || MODE == MODE_DGRAD, "forward / input gradient only");
-    constexpr int A_BYTES = FlatCfg<MT, NB>::A_BYTES;
-    constexpr int STAGE = FlatCfg<MT, NB>::STAGE;
-    constexpr int STAGES = FlatCfg<MT, NB>::STAGES;
+    constexpr int A_BYTES = FlatCfg<MT, NB, OCC>::A_BYTES;
+    constexpr int STAGE = FlatCfg<MT, NB, OCC>::STAGE;
+    constexpr int STAGES = FlatCfg<MT, NB, OCC>::STAGES;
     constexpr uint32_t ACC_COLS = MT * NB * 64;
     constexpr uint32_t TMEM_COLS = ACC_COLS * NBUF;
     static_assert(TMEM_COLS == 128 || TMEM_COLS == 256 || TMEM_COLS == 512, "tensor-memory columns");
@@ -604,7 +610,7 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
     uint64_t* acc_empty = acc_full + NBUF;     // [NBUF]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + NBUF);
     uint8_t* stg_all = smem + STAGES * STAGE + 256;
-    constexpr int STG = FlatCfg<MT, NB>::STG;
+    constexpr int STG = FlatCfg<MT, NB, OCC>::STG;
     int* s_off = reinterpret_cast<int*>(stg_all + 4 * MT * STG);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -616,6 +622,7 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
         ptx::prefetch_tensormap(&mapB);
     }
     if (warp == 0) { ptx::tmem_alloc(tmem_slot, TMEM_COLS); ptx::tmem_relinquish(); }
+    pdl_wait();                                   // everything above overlaps the previous kernel's tail
     for (int i = tid; i <= p.B; i += blockDim.x) s_off[i] = p.blk_off[i];
     ptx::tc_fence_before();
     __syncthreads();
@@ -718,7 +725,7 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                     const int r = m * (128 * MT) + (i >> 3), cb = (i & 7) * 8;
                     if (r < p.M && t0 + cb < p.Tp) {
                         const size_t e = ((size_t)b * p.M + r) * p.Tp + t0 + cb;
-                        if (MT == 1 && p.out_f32) {
+                        if (MT == 1 && OCC == 1 && p.out_f32) {
                             *reinterpret_cast<uint4*>(reinterpret_cast<float*>(p.out) + e) = make_uint4(0, 0, 0, 0);
                             *reinterpret_cast<uint4*>(reinterpret_cast<float*>(p.out) + e + 4) = make_uint4(0, 0, 0, 0);
                         } else {
@@ -796,7 +803,7 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                     }
                     const size_t base = ((size_t)b * p.M + row_w) * p.Tp + c0;
                     const int rl = p.M - row_w, cl = p.Tp - c0;
-                    if (MT == 1 && MODE == MODE_FWD && p.out_f32)
+                    if (MT == 1 && OCC == 1 && MODE == MODE_FWD && p.out_f32)
                         store_block_staged<float>(reinterpret_cast<float*>(stg), f, reinterpret_cast<float*>(p.out) + base, p.Tp, rl, cl, lane);
                     else if (MODE == MODE_FWD && p.out_half)
                         store_block16<__half>(stg, f, reinterpret_cast<__half*>(p.out) + base, p.Tp, rl, cl, lane);
@@ -819,6 +826,7 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
 // short poll limit; the wait gives up, raises the timeout status and the kernel returns normally.  No copy is
 // in flight and no tensor memory is held, so there is nothing to drain.
 __global__ void bounded_wait_selftest_kernel(int* status) {
+    pdl_sync();
     __shared__ uint64_t bar;
     if (threadIdx.x == 0) {
         ptx::mbar_init(&bar, 1);
@@ -865,7 +873,7 @@ void launch(const Launch& L, dim3 grid, const CUtensorMap& a, const CUtensorMap&
     constexpr int smem = STAGES * (MT * 16384 + BN * 128) + 1024 + 256 + 4 * kStgFloatsPerWarp * 4;
     auto kern = tc_gemm_kernel<T, MODE, MT, BN, STAGES>;
     set_max_smem_once<tc_gemm_kernel<T, MODE, MT, BN, STAGES>>(smem);
-    kern<<<grid, kThreads, smem, L.stream>>>(a, b, p);
+    launch_k(L, kern, grid, kThreads, smem, a, b, p);
     L.count();
 }
 
@@ -882,7 +890,7 @@ void launch_persistent(const Launch& L, int sm_count, const CUtensorMap& a, cons
     auto kern = tc_gemm_persistent_kernel<T, MODE, MT, BN, STAGES>;
     set_max_smem_once<tc_gemm_persistent_kernel<T, MODE, MT, BN, STAGES>>(smem);
     const int total = tiles_n * tiles_m * batch;
-    kern<<<std::min(sm_count, total), 32 * (4 * MT + 2), smem, L.stream>>>(a, b, p, tiles_n, tiles_m, total);
+    launch_k(L, kern, std::min(sm_count, total), 32 * (4 * MT + 2), smem, a, b, p, tiles_n, tiles_m, total);
     L.count();
 }
 template <int MODE, int MT, int BN, int STAGES>
@@ -901,7 +909,9 @@ constexpr int FWD_BN = 128;
 struct WgradPlan { int mt, bn, tiles, nsplit, kb_per_split, nkb_total, nkb_t; };
 WgradPlan plan_wgrad(int B, int Cin, int Cout, int Tp) {
     WgradPlan w;
-    w.mt = Cout >= 512 ? 2 : 1;
+    // one 128-row M sub-tile per CTA: twice the output tiles of the two-sub-tile form, so half the k-slices are
+    // needed to fill the SMs and the fp32 partials (written once, read once by the reduction) halve
+    w.mt = 1;
     w.bn = Cin >= 512 ? 256 : (Cin > 64 ? 128 : 64);
     w.tiles = ((Cout + 128 * w.mt - 1) / (128 * w.mt)) * ((Cin + w.bn - 1) / w.bn);
     w.nkb_t = (Tp + BK - 1) / BK;
@@ -916,7 +926,7 @@ WgradPlan plan_wgrad(int B, int Cin, int Cout, int Tp) {
 }  // namespace
 
 void selftest_bounded_wait(const Launch& L) {
-    bounded_wait_selftest_kernel<<<1, 32, 0, L.stream>>>(L.status);
+    launch_k(L, bounded_wait_selftest_kernel, 1, 32, 0, L.status);
     L.count();
 }
 
@@ -946,21 +956,23 @@ size_t tc_wgrad_scratch_bytes(const TcState*, int Cin, int Cout) {
 }
 
 namespace {
-template <typename T, int MODE, int MT, int NB, int NBUF>
+template <typename T, int MODE, int MT, int NB, int NBUF, int OCC = 1>
 void launch_flat(const Launch& L, int sm_count, const CUtensorMap& a, const CUtensorMap& b, const FlatParams& p, int* grid_out) {
-    const int smem = FlatCfg<MT, NB>::smem_bytes(p.B);
-    auto kern = tc_gemm_flat_kernel<T, MODE, MT, NB, NBUF>;
-    set_max_smem_once<tc_gemm_flat_kernel<T, MODE, MT, NB, NBUF>>(FlatCfg<MT, NB>::smem_bytes(kFlatMaxB));
+    const int smem = FlatCfg<MT, NB, OCC>::smem_bytes(p.B);
+    auto kern = tc_gemm_flat_kernel<T, MODE, MT, NB, NBUF, OCC>;
+    set_max_smem_once<tc_gemm_flat_kernel<T, MODE, MT, NB, NBUF, OCC>>(FlatCfg<MT, NB, OCC>::smem_bytes(FlatCfg<MT, NB, OCC>::MAXB));
     const long long units = (long long)p.tiles_m * p.B * p.nbT;
-    const int grid = (int)std::max(1ll, std::min<long long>(std::min(sm_count, kFlatMaxGrid), units));
-    kern<<<grid, 32 * (4 * MT + 2), smem, L.stream>>>(a, b, p);
+    const int grid = (int)std::max(1ll, std::min<long long>(std::min(sm_count * OCC, kFlatMaxGrid), units));
+    launch_k(L, kern, grid, 32 * (4 * MT + 2), smem, a, b, p);
     L.count();
     if (grid_out) *grid_out = grid;
 }
-// shape 0: 256 x 256 tiles, one accumulator; 1: 256 x 128 tiles, two accumulators; 2: 128 x 256 tiles, two accumulators
+// shape 0: 256 x 256 tiles, one accumulator; 1: 256 x 128 tiles, two accumulators; 2: 128 x 256 tiles, two accumulators;
+// 3: 128 x 256 tiles, one accumulator, two CTAs per SM
 template <typename T, int MODE>
 void launch_flat_shape(int shape, int mt, const Launch& L, int sm_count, const CUtensorMap& a, const CUtensorMap& b,
                        const FlatParams& p, int* grid_out) {
+    if (shape == 3 && !p.out_f32 && p.B <= FlatCfg<1, 4, 2>::MAXB) { launch_flat<T, MODE, 1, 4, 1, 2>(L, sm_count, a, b, p, grid_out); return; }
     if (mt == 1) { launch_flat<T, MODE, 1, 4, 2>(L, sm_count, a, b, p, grid_out); return; }
     if (shape == 0) launch_flat<T, MODE, 2, 4, 1>(L, sm_count, a, b, p, grid_out);
     else launch_flat<T, MODE, 2, 2, 2>(L, sm_count, a, b, p, grid_out);
@@ -972,7 +984,7 @@ void launch_flat_dt(int dtype, int shape, int mt, const Launch& L, int sm_count,
     else launch_flat_shape<__nv_bfloat16, MODE>(shape, mt, L, sm_count, a, b, p, grid_out);
 }
 // M sub-tiles per CTA for a given tile shape and row count
-inline int flat_mt(int shape, int rows) { return (shape == 2 || rows <= 128) ? 1 : 2; }
+inline int flat_mt(int shape, int rows) { return (shape >= 2 || rows <= 128) ? 1 : 2; }
 }  // namespace
 
 size_t tc_stats_bytes(int B, int Cout, int Tp) {
