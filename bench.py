@@ -431,7 +431,7 @@ def main():
     if args.breakdown:
         with open(args.breakdown, "w") as f:
             f.write(f"# per-kernel-class CUDA-event time, {w.name}, {nprof} host-launched steps; "
-                    f"graph-replayed step {ms / args.steps:.3f} ms\n")
+                    f"timed step ({'graph replay' if args.graph else 'host launches'}) {ms / args.steps:.3f} ms\n")
             f.write("class launches/step ms/step share GB/s TFLOP/s bound frac\n")
             for k, v in sorted(per_class.items(), key=lambda kv: -kv[1]["share"]):
                 f.write(f"{k} {v['launches_per_step']:.0f} {v['ms_per_step']:.4f} {v['share']:.3f} {v['GB/s']:.0f} "

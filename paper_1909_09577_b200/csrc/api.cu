@@ -341,9 +341,8 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
     a.gv = s.gv; a.gvr = s.gvr;
     // identity residual: its gradient is the gated upstream gradient itself
     a.gres = (d->residual == SC_RES_IDENTITY) ? (io.dx_res ? io.dx_res : s.gres) : nullptr;
-    bn_bwd_reduce(L, dt, a);
-    bn_bwd_finalize(L, a, p->gamma, p->gamma_r, g->dgamma, g->dbeta, g->dgamma_r, g->dbeta_r,
-                    d->has_bias ? g->dbias : nullptr, acc);
+    bn_bwd_reduce_finalize(L, dt, a, p->gamma, p->gamma_r, g->dgamma, g->dbeta, g->dgamma_r, g->dbeta_r,
+                           d->has_bias ? g->dbias : nullptr, acc);
     bn_bwd_apply(L, dt, a);
 
     // The weight gradients are off the critical path (nothing later in the backward pass reads them): they run on

@@ -500,52 +500,61 @@ __global__ void __launch_bounds__(kRowThreads) bn_bwd_apply_kernel(BnBwdArgs a) 
     }
 }
 
+// Per-channel constants of the forward apply step and of the backward kernels, loaded (or, in the
+// channel-per-CTA kernels, computed) once and passed by value.
+struct FwdChan { float mu, is, ga, be, mur, isr, gar, ber; };
+struct BwdChan { float mu, is, ga, be, mur, isr; float4 cf, cr; };
+
 // One 8-frame vector of the forward apply step: y = [t < len] * relu(gamma * vhat + beta (+ r)); n = frames of the
 // vector inside the sample (0: wholly padding), rv / rr = the raw 16 bytes of v and of the residual operand.
 template <typename T, typename NT, int RES>
-__device__ __forceinline__ void apply_vec(const ApplyArgs& a, int o, int n, size_t off, const uint4& rv, const uint4& rr) {
+__device__ __forceinline__ void apply_core(T* yp, int n, const uint4& rv, const uint4& rr, const FwdChan& c) {
     float out[8];
     if (n > 0) {
         float f[8], r[8];
         cvt8<NT>(rv, f);
         if (RES == 1) cvt8<T>(rr, r);
         if (RES == 2) cvt8<NT>(rr, r);
-        const float mu = a.mean[o], is = a.invstd[o], ga = a.gamma[o], be = a.beta[o];
-        float mur = 0.f, isr = 0.f, gar = 0.f, ber = 0.f;
-        if (RES == 2) { mur = a.mean_r[o]; isr = a.invstd_r[o]; gar = a.gamma_r[o]; ber = a.beta_r[o]; }
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             float rres = 0.f;
             if (RES == 1) rres = r[i];
-            if (RES == 2) rres = fmaf(gar, bn_norm(r[i], mur, isr), ber);
-            const float q = fmaxf(fmaf(ga, bn_norm(f[i], mu, is), be) + rres, 0.f);
+            if (RES == 2) rres = fmaf(c.gar, bn_norm(r[i], c.mur, c.isr), c.ber);
+            const float q = fmaxf(fmaf(c.ga, bn_norm(f[i], c.mu, c.is), c.be) + rres, 0.f);
             out[i] = i < n ? q : 0.f;
         }
     } else {
 #pragma unroll
         for (int i = 0; i < 8; ++i) out[i] = 0.f;
     }
-    st8<T>((T*)a.y + off, out);
+    st8<T>(yp, out);
+}
+template <typename T, typename NT, int RES>
+__device__ __forceinline__ void apply_vec(const ApplyArgs& a, int o, int n, size_t off, const uint4& rv, const uint4& rr) {
+    FwdChan c{};
+    if (n > 0) {
+        c.mu = a.mean[o]; c.is = a.invstd[o]; c.ga = a.gamma[o]; c.be = a.beta[o];
+        if (RES == 2) { c.mur = a.mean_r[o]; c.isr = a.invstd_r[o]; c.gar = a.gamma_r[o]; c.ber = a.beta_r[o]; }
+    }
+    apply_core<T, NT, RES>((T*)a.y + off, n, rv, rr, c);
 }
 
 // One 8-frame vector of the backward apply step (gv and the residual branch's gradient), computed and stored.
 template <typename T, typename NT, typename GT, int RES>
-__device__ __forceinline__ void bwd_apply_vec(const BnBwdArgs& a, int o, int n, size_t off, float sc, bool fold,
-                                              const uint4& rg, const uint4& rv, const uint4& rr, const uint4& ry) {
+__device__ __forceinline__ void bwd_apply_core(const BnBwdArgs& a, int n, size_t off, float sc, bool fold, const uint4& rg,
+                                               const uint4& rv, const uint4& rr, const uint4& ry, const BwdChan& c) {
     float o1[8], o2[8];
     if (n > 0) {
         float g[8], y[8], vn[8], vnr[8];
         cvt8<T>(rg, g);
         cvt8<NT>(rv, vn);
-        const float mu = a.mean[o], is = a.invstd[o];
-        const uint64_t nmu2 = pk::pack(-mu, -mu), is2 = pk::pack(is, is);
+        const uint64_t nmu2 = pk::pack(-c.mu, -c.mu), is2 = pk::pack(c.is, c.is);
         uint64_t vn2[4], vr2[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) vn2[q] = pk::bn_norm2(pk::pack(vn[2 * q], vn[2 * q + 1]), nmu2, is2);
         if (RES == 2) {
             cvt8<NT>(rr, vnr);
-            const float mur = a.mean_r[o], isr = a.invstd_r[o];
-            const uint64_t nmur2 = pk::pack(-mur, -mur), isr2 = pk::pack(isr, isr);
+            const uint64_t nmur2 = pk::pack(-c.mur, -c.mur), isr2 = pk::pack(c.isr, c.isr);
 #pragma unroll
             for (int q = 0; q < 4; ++q) vr2[q] = pk::bn_norm2(pk::pack(vnr[2 * q], vnr[2 * q + 1]), nmur2, isr2);
         }
@@ -553,8 +562,7 @@ __device__ __forceinline__ void bwd_apply_vec(const BnBwdArgs& a, int o, int n, 
         if (RES == 0) {
             // without a residual the forward output is relu(gamma * vhat + beta), rounded to the
             // activation type: the gate is recomputed from v and the output need not be read
-            const float ga_ = a.gamma[o], be_ = a.beta[o];
-            const uint64_t ga2 = pk::pack(ga_, ga_), be2 = pk::pack(be_, be_);
+            const uint64_t ga2 = pk::pack(c.ga, c.ga), be2 = pk::pack(c.be, c.be);
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 float a0, a1;
@@ -568,12 +576,12 @@ __device__ __forceinline__ void bwd_apply_vec(const BnBwdArgs& a, int o, int n, 
         }
         // gv = k (ga - c1 - c2 vhat) as two fused multiply-adds; when gv itself is the scaled half tensor the
         // power-of-two scale is folded into k (exact)
-        const float4 cf = a.coef[o];
+        const float4 cf = c.cf;
         const float kx = (fold ? sc : 1.f) * cf.x;
         const uint64_t kx2 = pk::pack(kx, kx), k02 = pk::pack(-kx * cf.y, -kx * cf.y), k22 = pk::pack(-kx * cf.z, -kx * cf.z);
         uint64_t kr2 = 0, r02 = 0, r22 = 0;
         if (RES == 2) {
-            const float4 cr = a.coef_r[o];
+            const float4 cr = c.cr;
             kr2 = pk::pack(cr.x, cr.x); r02 = pk::pack(-cr.x * cr.y, -cr.x * cr.y); r22 = pk::pack(-cr.x * cr.z, -cr.x * cr.z);
         }
 #pragma unroll
@@ -620,30 +628,39 @@ __device__ __forceinline__ void bwd_apply_vec(const BnBwdArgs& a, int o, int n, 
     if (RES == 1) st8<T>((T*)a.gres + off, o2);
 }
 
+template <typename T, typename NT, typename GT, int RES>
+__device__ __forceinline__ void bwd_apply_vec(const BnBwdArgs& a, int o, int n, size_t off, float sc, bool fold,
+                                              const uint4& rg, const uint4& rv, const uint4& rr, const uint4& ry) {
+    BwdChan c{};
+    if (n > 0) {
+        c.mu = a.mean[o]; c.is = a.invstd[o]; c.cf = a.coef[o];
+        if (RES == 0) { c.ga = a.gamma[o]; c.be = a.beta[o]; }
+        if (RES == 2) { c.mur = a.mean_r[o]; c.isr = a.invstd_r[o]; c.cr = a.coef_r[o]; }
+    }
+    bwd_apply_core<T, NT, GT, RES>(a, n, off, sc, fold, rg, rv, rr, ry, c);
+}
+
 // One 8-frame vector of the backward reduction: s0 = sum ga, s1 = sum ga * vhat, s3 = sum ga * vhat_r, m = max |ga|
 // over its n (> 0) frames inside the sample.
 template <typename T, typename NT, int RES>
-__device__ __forceinline__ void reduce_vec(const BnBwdArgs& a, int o, int n, const uint4& rg, const uint4& rv, const uint4& rr,
-                                           const uint4& ry, float& s0, float& s1, float& s3, float& m_out) {
+__device__ __forceinline__ void reduce_core(int n, const uint4& rg, const uint4& rv, const uint4& rr, const uint4& ry,
+                                            const BwdChan& c, float& s0, float& s1, float& s3, float& m_out) {
     float g[8], y[8], vn[8], vnr[8];
     cvt8<T>(rg, g);
     cvt8<NT>(rv, vn);
-    const float mu = a.mean[o], is = a.invstd[o];
-    const uint64_t nmu2 = pk::pack(-mu, -mu), is2 = pk::pack(is, is);
+    const uint64_t nmu2 = pk::pack(-c.mu, -c.mu), is2 = pk::pack(c.is, c.is);
     uint64_t vn2[4], vr2[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) vn2[q] = pk::bn_norm2(pk::pack(vn[2 * q], vn[2 * q + 1]), nmu2, is2);
     if (RES == 2) {
         cvt8<NT>(rr, vnr);
-        const float mur = a.mean_r[o], isr = a.invstd_r[o];
-        const uint64_t nmur2 = pk::pack(-mur, -mur), isr2 = pk::pack(isr, isr);
+        const uint64_t nmur2 = pk::pack(-c.mur, -c.mur), isr2 = pk::pack(c.isr, c.isr);
 #pragma unroll
         for (int q = 0; q < 4; ++q) vr2[q] = pk::bn_norm2(pk::pack(vnr[2 * q], vnr[2 * q + 1]), nmur2, isr2);
     }
     bool gate[8];
     if (RES == 0) {          // gate from v (see bn_bwd_apply_fast_kernel)
-        const float ga_ = a.gamma[o], be_ = a.beta[o];
-        const uint64_t ga2 = pk::pack(ga_, ga_), be2 = pk::pack(be_, be_);
+        const uint64_t ga2 = pk::pack(c.ga, c.ga), be2 = pk::pack(c.be, c.be);
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             float a0, a1;
@@ -672,6 +689,16 @@ __device__ __forceinline__ void reduce_vec(const BnBwdArgs& a, int o, int n, con
     pk::unpack(s1_2, t0_, t1_); s1 = t0_ + t1_;
     pk::unpack(s3_2, t0_, t1_); s3 = t0_ + t1_;
     m_out = m;
+}
+
+template <typename T, typename NT, int RES>
+__device__ __forceinline__ void reduce_vec(const BnBwdArgs& a, int o, int n, const uint4& rg, const uint4& rv, const uint4& rr,
+                                           const uint4& ry, float& s0, float& s1, float& s3, float& m_out) {
+    BwdChan c{};
+    c.mu = a.mean[o]; c.is = a.invstd[o];
+    if (RES == 0) { c.ga = a.gamma[o]; c.be = a.beta[o]; }
+    if (RES == 2) { c.mur = a.mean_r[o]; c.isr = a.invstd_r[o]; }
+    reduce_core<T, NT, RES>(n, rg, rv, rr, ry, c, s0, s1, s3, m_out);
 }
 
 // ---- flattened fast paths (the encoder's configuration: BN + ReLU, residual joined before the ReLU,
@@ -808,6 +835,92 @@ __global__ void __launch_bounds__(256) bn_bwd_reduce_fast_kernel(BnBwdArgs a, in
     }
 }
 
+// ---- channel-per-CTA backward reduction ----------------------------------------------------------------
+// One CTA streams channel o of every sample: B * vpr 8-frame vectors, numbered sample-major, thread t the vectors
+// t, t + blockDim, ... in batches of U independent 16-byte loads per tensor, sums in registers.  Because the CTA sees
+// the whole channel it needs no per-row partials and no finalize launch: it ends with the channel's coefficients.
+// (The same mapping was measured for the two apply kernels and lost to the flattened one: a CTA that hops between
+// the 32 rows of a channel streams about 10 % slower than one that walks the tensor in address order, and a forward
+// apply that merges the contraction's statistics partials in its prologue pays that merge once per CTA.)
+constexpr int kChThreads = 256;
+
+// Backward reduction of channel o over every sample, then the channel's coefficients, parameter gradients and its
+// term of the bound on |gv| (what bn_bwd_finalize_kernel does for the row-mapped reduction).
+template <typename T, typename NT, int RES>
+__global__ void __launch_bounds__(kChThreads, 4)
+bn_bwd_reduce_ch_kernel(BnBwdArgs a, int vpr, const float* gamma_r, float* dgamma, float* dbeta, float* dgamma_r,
+                        float* dbeta_r, int accumulate) {
+    pdl_sync();
+    constexpr int NT_ = kChThreads;
+    constexpr int U = RES == 2 ? 2 : 4;            // 16-byte loads in flight per thread: U * (2 or 4 tensors)
+    __shared__ float4 s_sum[NT_ / 32];
+    const int o = blockIdx.x, tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    BwdChan c{};
+    c.mu = a.mean[o]; c.is = a.invstd[o];
+    if (RES == 0) { c.ga = a.gamma[o]; c.be = a.beta[o]; }
+    if (RES == 2) { c.mur = a.mean_r[o]; c.isr = a.invstd_r[o]; }
+    const int nvec = a.B * vpr;
+    float s0 = 0.f, s1 = 0.f, s3 = 0.f, amax = 0.f;
+    for (int jb = tid; jb < nvec; jb += U * NT_) {
+        int nin[U];
+        uint4 rg[U], rv[U], rr[U], ry[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int j = jb + u * NT_;
+            nin[u] = 0;
+            rg[u] = rv[u] = rr[u] = ry[u] = make_uint4(0, 0, 0, 0);
+            if (j < nvec) {
+                const int b = (int)a.dvpr.div((uint32_t)j), t0 = (j - b * vpr) * 8;
+                nin[u] = max(0, min(a.len_out[b], a.Tp) - t0);
+                if (nin[u] > 0) {
+                    const size_t off = ((size_t)b * a.C + o) * a.Tp + t0;
+                    rg[u] = *reinterpret_cast<const uint4*>((const T*)a.g + off);
+                    rv[u] = *reinterpret_cast<const uint4*>((const NT*)a.v + off);
+                    if (RES == 2) rr[u] = *reinterpret_cast<const uint4*>((const NT*)a.vr + off);
+                    if (RES != 0) ry[u] = *reinterpret_cast<const uint4*>((const T*)a.y + off);
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (nin[u] <= 0) continue;
+            float q0, q1, q3, m;
+            reduce_core<T, NT, RES>(nin[u], rg[u], rv[u], rr[u], ry[u], c, q0, q1, q3, m);
+            s0 += q0; s1 += q1; s3 += q3; amax = fmaxf(amax, m);
+        }
+    }
+    s0 = warp_sum(s0); s1 = warp_sum(s1);
+    if (RES == 2) s3 = warp_sum(s3);
+    if (a.gmax) amax = warp_max(amax);
+    if (lane == 0) s_sum[w] = make_float4(s0, s1, s3, amax);
+    __syncthreads();
+    if (tid != 0) return;
+    float d0 = 0.f, d1 = 0.f, d3 = 0.f;
+    amax = 0.f;
+#pragma unroll
+    for (int i = 0; i < NT_ / 32; ++i) {                // warp order: bit-repeatable
+        const float4 q = s_sum[i];
+        d0 += q.x; d1 += q.y; d3 += q.z; amax = fmaxf(amax, q.w);
+    }
+    const float N = (float)(*a.nvalid);
+    const float k = a.gamma[o] * c.is;
+    const float kr = RES == 2 ? gamma_r[o] * c.isr : 0.f;
+    if (a.gmax) {            // see bn_bwd_finalize_kernel
+        float bound = fabsf(k) * (amax + fabsf(d0) / N + sqrtf(N) * fabsf(d1) / N);
+        if (RES == 2) bound = fmaxf(bound, fabsf(kr) * (amax + fabsf(d0) / N + sqrtf(N) * fabsf(d3) / N));
+        if (bound < 3.0e38f) atomicMax(reinterpret_cast<unsigned int*>(a.gmax), __float_as_uint(bound));
+    }
+    auto put = [&](float* dst, float val) {
+        if (dst) dst[o] = accumulate ? dst[o] + val : val;
+    };
+    put(dbeta, d0); put(dgamma, d1);
+    a.coef[o] = make_float4(k, d0 / N, d1 / N, 0.f);
+    if (RES == 2) {
+        put(dbeta_r, d0); put(dgamma_r, d3);            // the residual sum receives the same gated gradient
+        a.coef_r[o] = make_float4(kr, d0 / N, d3 / N, 0.f);
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kRowThreads)
 ew_add_masked_kernel(T* out, const T* a, const T* b, const T* c, const int* len, int nrows, int C, int Tt) {
@@ -893,6 +1006,10 @@ static bool fits32(int B, int C, int Tp) { return (long long)B * C * (Tp / 8) < 
 static unsigned fast_grid(long long total, int V) { return (unsigned)((total + 256ll * V - 1) / (256ll * V)); }
 
 // Algorithmic bytes per element of the batch-norm kernels: every tensor they must read or write, once.
+// The channel-per-CTA reduction pays off once a channel holds a few vectors per thread; below that (or with few
+// channels) the row-mapped kernel and its separate finalize step are used.
+static bool channel_mapped(int B, int C, int Tp) { return C >= 32 && (long long)B * (Tp / 8) >= 4 * kChThreads; }
+
 void bn_apply(const Launch& L, int dtype, const ApplyArgs& a_in) {
     ApplyArgs a = a_in;
     const double e = (double)dtype_size(dtype), en = (double)dtype_size(ntype_of(dtype));
@@ -944,6 +1061,26 @@ void bn_bwd_finalize(const Launch& L, const BnBwdArgs& a, const float* gamma, co
     launch_k(L, bn_bwd_finalize_kernel, (a.C + 31) / 32, 32 * kFinWarps, 0, a, gamma, gamma_r, dgamma, dbeta, dgamma_r,
                                                                           dbeta_r, dbias, accumulate);
     L.count();
+}
+
+void bn_bwd_reduce_finalize(const Launch& L, int dtype, BnBwdArgs& a, const float* gamma, const float* gamma_r,
+                            float* dgamma, float* dbeta, float* dgamma_r, float* dbeta_r, float* dbias, int accumulate) {
+    const bool fast = dtype != F32 && a.Tp % 8 == 0 && a.has_bn && a.has_relu && a.res_before_relu && fits32(a.B, a.C, a.Tp);
+    if (fast && channel_mapped(a.B, a.C, a.Tp)) {
+        a.nslots = 1; a.vpw = 32; a.vpw_shift = 5;
+        const double e = (double)dtype_size(dtype), en = (double)dtype_size(ntype_of(dtype));
+        KScope ks_(L, KC_BN_BWD_REDUCE, (double)a.B * a.C * a.Tp * (e * (a.residual == 0 ? 1 : 2) + en * (a.residual == 2 ? 2 : 1)), 0.0);
+        const int vpr = a.Tp / 8;
+        a.dvpr = FastDiv((uint32_t)vpr);
+#define SC_RED_CH(RES) SC_DISPATCH16(dtype, (launch_k(L, bn_bwd_reduce_ch_kernel<T, NT, RES>, (unsigned)a.C, kChThreads, 0, a, vpr, \
+                                                       gamma_r, dgamma, dbeta, dgamma_r, dbeta_r, accumulate)))
+        if (a.residual == 2) { SC_RED_CH(2); } else if (a.residual == 1) { SC_RED_CH(1); } else { SC_RED_CH(0); }
+#undef SC_RED_CH
+        L.count();
+        return;
+    }
+    bn_bwd_reduce(L, dtype, a);
+    bn_bwd_finalize(L, a, gamma, gamma_r, dgamma, dbeta, dgamma_r, dbeta_r, dbias, accumulate);
 }
 
 void bn_bwd_apply(const Launch& L, int dtype, const BnBwdArgs& a_in) {

@@ -246,6 +246,10 @@ inline int bn_bwd_max_slots(int Tp) { return Tp / 256 + 2; }
 void bn_bwd_finalize(const Launch& L, const BnBwdArgs& a, const float* gamma, const float* gamma_r,
                      float* dgamma, float* dbeta, float* dgamma_r, float* dbeta_r, float* dbias,
                      int accumulate);
+// bn_bwd_reduce followed by bn_bwd_finalize, or -- for the encoder's block shape -- one kernel with a CTA per
+// channel that does both.
+void bn_bwd_reduce_finalize(const Launch& L, int dtype, BnBwdArgs& a, const float* gamma, const float* gamma_r,
+                            float* dgamma, float* dbeta, float* dgamma_r, float* dbeta_r, float* dbias, int accumulate);
 void bn_bwd_apply(const Launch& L, int dtype, const BnBwdArgs& a);
 
 // ---- decoder tail / evaluation mode ---------------------------------------------------------------
