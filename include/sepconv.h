@@ -301,9 +301,11 @@ int  encoder_infer(sc_ctx* ctx, const sc_encoder_desc* desc,
 int  sepconv_set_gemm_mode(sc_ctx* ctx, int mode);
 
 /* Tile shape of the forward / input-gradient pointwise contractions (tuning aid; the paper has no counterpart):
- * 0 = 256 output channels x 256 frames per tile with one accumulator in tensor memory, 1 = 256 x 128 and
- * 2 = 128 x 256 with two accumulators, so that a tile's epilogue overlaps the next tile's MMAs.  Results do not
- * depend on it except for the summation order of the batch-norm statistics. */
+ * 0 = 256 output channels x 256 frames per tile with one accumulator in tensor memory, drained by sixteen epilogue
+ * warps when the batch has at most 256 samples (else as 4); 1 = 256 x 128 and 2 = 128 x 256 with two accumulators,
+ * so that a tile's epilogue overlaps the next tile's MMAs; 3 = 128 x 256, one accumulator, two CTAs per SM;
+ * 4 = as 0 with eight epilogue warps.  Other values: SC_ERR_UNSUPPORTED.  Results do not depend on the shape except
+ * for the summation order of the batch-norm statistics. */
 int  sepconv_set_tile_shape(sc_ctx* ctx, int shape);
 
 /* Overlap between kernels (both forms on by default; `on` is a bit mask, 3 = both, 0 = neither).

@@ -54,9 +54,10 @@ template <> struct Fmt<__nv_bfloat16> { static constexpr uint32_t v = 1; };
 // (16-bit) row segments.  `rows_left` / `cols_left` bound the valid part; cols are a multiple of 8.
 // A float16 result beyond the half range is clamped to the largest finite value and flagged.
 __device__ __forceinline__ void clamp_half32(float (&f)[32], int* status) {
-    float m = 0.f;
+    float m4[4] = {0.f, 0.f, 0.f, 0.f};          // four independent chains: the maximum is latency-bound otherwise
 #pragma unroll
-    for (int i = 0; i < 32; ++i) m = fmaxf(m, fabsf(f[i]));
+    for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], fabsf(f[i]));
+    const float m = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
     if (m > 65504.f) {
 #pragma unroll
         for (int i = 0; i < 32; ++i) f[i] = fminf(fmaxf(f[i], -65504.f), 65504.f);
@@ -531,6 +532,10 @@ struct FlatParams {
     int zero_fill;  // blocks wholly in padding must be written as zeros
     int out_half;   // the result is float16 although the operands are bfloat16
     int out_f32;    // the result is float32 (one M sub-tile per CTA only: narrow heads such as the class scores)
+    int tma_out;    // 16-bit result leaves through TMA stores (third tensor map: 32 frames x 32 rows, 64-byte swizzle)
+    int stg_stride; // bytes of staging per epilogue warp (a multiple of 512)
+    int stg_nbuf;   // 2: a warp alternates between two 2 KiB staging buffers, so that it need not wait for the store
+                    // before last to have read its source
 };
 
 // Coalesced store of a warp's 32 x 32 block as 16-bit values: lane l holds 32 consecutive columns of row l;
@@ -553,6 +558,19 @@ __device__ __forceinline__ void store_block16(uint8_t* stg, const float (&f)[32]
             const uint4 v = *reinterpret_cast<const uint4*>(stg + r * kOutPitch + (lane & 3) * 16);
             *reinterpret_cast<uint4*>(out + (size_t)r * ld + c) = v;
         }
+    }
+}
+
+// Staging for a TMA store of the same block: dense 64-byte rows, the 16-byte chunk c of row r in slot
+// c ^ ((r >> 1) & 3) -- the 64-byte swizzle of the tensor map, which also keeps the row-wise writes free of bank
+// conflicts.  The warp's registers then cross the load/store path once (to shared memory); the copy engine does the
+// rest, clipping rows and frames beyond the tensor.
+template <typename OT>
+__device__ __forceinline__ void stage_block16_swz(uint8_t* stg, const float (&f)[32], int lane) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float g[8] = {f[8 * i], f[8 * i + 1], f[8 * i + 2], f[8 * i + 3], f[8 * i + 4], f[8 * i + 5], f[8 * i + 6], f[8 * i + 7]};
+        st8<OT>(reinterpret_cast<OT*>(stg + lane * 64 + ((i ^ ((lane >> 1) & 3)) << 4)), g);
     }
 }
 
@@ -580,46 +598,53 @@ __device__ __forceinline__ bool flat_next_tile(long long& pos, long long end, in
 // tensor-memory columns).  With NBUF = 2 the epilogue of a tile overlaps the MMAs of the next one.
 // OCC = CTAs per SM: with 2, each CTA has a two-stage ring and half of tensor memory, and the two CTAs of an SM
 // cover each other's set-up, pipeline fill and epilogue.
-template <int MT, int NB, int OCC> struct FlatCfg {
+// EPI = epilogue warps per 32 accumulator rows: with 2, the two warps that may read the same quarter of tensor
+// memory's lanes take one 32-column half of every block each.  A warp's work on a 32 x 32 block is a chain of short
+// latencies (tensor-memory load, statistics, staging, fence, store issue); twice the warps overlap twice as many of
+// these chains, and the accumulator -- the only one, so the next tile's MMAs wait for it -- is free in half the time.
+template <int MT, int NB, int OCC, int EPI = 1> struct FlatCfg {
     static constexpr int A_BYTES = MT * 128 * 128;
     static constexpr int STAGE = A_BYTES + NB * 8192;
     static constexpr int STAGES = OCC == 2 ? 2 : (STAGE <= 49152 ? 4 : 3);
     // per-warp staging: 32 x 32 16-bit values, or (one M sub-tile, one CTA per SM only) 32 x 32 floats for a float32 result
-    static constexpr int STG = (MT == 1 && OCC == 1) ? kStgFloatsPerWarp * 4 : kOutStageBytes;
-    static constexpr int MAXB = OCC == 2 ? 256 : kFlatMaxB;
-    static constexpr int smem_bytes(int B) { return STAGES * STAGE + 256 + 4 * MT * STG + (B + 1) * 4 + 1024; }
+    static constexpr int STG = EPI == 2 ? 2048 : ((MT == 1 && OCC == 1) ? kStgFloatsPerWarp * 4 : kOutStageBytes);
+    static constexpr int MAXB = (OCC == 2 || EPI == 2) ? 256 : kFlatMaxB;
+    static constexpr int smem_bytes(int B) { return STAGES * STAGE + 256 + 4 * MT * EPI * STG + (B + 1) * 4 + 1024; }
 };
 
-template <typename T, int MODE, int MT, int NB, int NBUF, int OCC>
-__global__ void __launch_bounds__(32 * (4 * MT + 2), OCC)
-tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, FlatParams p) {
+template <typename T, int MODE, int MT, int NB, int NBUF, int OCC, int EPI>
+__global__ void __launch_bounds__(32 * (4 * MT * EPI + 2), OCC)
+tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                    const __grid_constant__ CUtensorMap mapO, FlatParams p) {
     pdl_launch_dependents();
     static_assert(MODE == MODE_FWD || MODE == MODE_DGRAD, "forward / input gradient only");
-    constexpr int A_BYTES = FlatCfg<MT, NB, OCC>::A_BYTES;
-    constexpr int STAGE = FlatCfg<MT, NB, OCC>::STAGE;
-    constexpr int STAGES = FlatCfg<MT, NB, OCC>::STAGES;
+    constexpr int A_BYTES = FlatCfg<MT, NB, OCC, EPI>::A_BYTES;
+    constexpr int STAGE = FlatCfg<MT, NB, OCC, EPI>::STAGE;
+    constexpr int STAGES = FlatCfg<MT, NB, OCC, EPI>::STAGES;
     constexpr uint32_t ACC_COLS = MT * NB * 64;
     constexpr uint32_t TMEM_COLS = ACC_COLS * NBUF;
     static_assert(TMEM_COLS == 128 || TMEM_COLS == 256 || TMEM_COLS == 512, "tensor-memory columns");
+    static_assert(EPI == 1 || (EPI == 2 && OCC == 1), "epilogue warps per lane quarter");
+    constexpr int EW = 4 * MT * EPI;               // epilogue warps; then the producer warp and the MMA warp
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE);
+    uint8_t* stg_all = smem + STAGES * STAGE;      // per-warp staging: 512-byte aligned (the swizzle of the output map)
+    uint64_t* full = reinterpret_cast<uint64_t*>(stg_all + EW * p.stg_stride);
     uint64_t* empty = full + STAGES;
     uint64_t* acc_full = empty + STAGES;       // [NBUF]
     uint64_t* acc_empty = acc_full + NBUF;     // [NBUF]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + NBUF);
-    uint8_t* stg_all = smem + STAGES * STAGE + 256;
-    constexpr int STG = FlatCfg<MT, NB, OCC>::STG;
-    int* s_off = reinterpret_cast<int*>(stg_all + 4 * MT * STG);
+    int* s_off = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(full) + 256);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
-        for (int i = 0; i < NBUF; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 128 * MT); }
+        for (int i = 0; i < NBUF; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 32 * EW); }
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&mapA);
         ptx::prefetch_tensormap(&mapB);
+        if (p.tma_out) ptx::prefetch_tensormap(&mapO);
     }
     if (warp == 0) { ptx::tmem_alloc(tmem_slot, TMEM_COLS); ptx::tmem_relinquish(); }
     pdl_wait();                                   // everything above overlaps the previous kernel's tail
@@ -633,7 +658,7 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
     const long long U = (long long)p.tiles_m * nblk;
     const long long u_begin = U * blockIdx.x / gridDim.x, u_end = U * (blockIdx.x + 1) / gridDim.x;
 
-    if (warp == 4 * MT) {
+    if (warp == EW) {
         if (lane == 0) {                              // ---- TMA producer ----
             int it = 0, m, j, nb;
             bool dead = false;
@@ -673,7 +698,7 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             }
         }
         __syncwarp();
-    } else if (warp == 4 * MT + 1) {
+    } else if (warp == EW + 1) {
         if (lane == 0) {                              // ---- MMA issuer ----
             int it = 0, jt = 0, m, j, nb;
             bool dead = false;
@@ -706,8 +731,10 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
         }
         __syncwarp();
     } else {                                          // ---- epilogue warps ----
-        const int mt = warp >> 2, wq = warp & 3;
-        uint8_t* stg = stg_all + warp * STG;
+        const int mt = (warp >> 2) % MT, wq = warp & 3;
+        const int hsel = (warp >> 2) / MT;            // EPI == 2: the 32-column half of every block this warp takes
+        uint8_t* stg = stg_all + warp * p.stg_stride;
+        uint32_t nstore = 0;                          // TMA stores issued by this warp
         if (p.zero_fill) {
             // blocks wholly in padding: sample b's blocks [off[b+1]-off[b], nbT); CTAs share them round-robin
             const int inv_per_m = p.B * p.nbT - nblk;
@@ -721,7 +748,7 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                 }
                 const int b = lo;
                 const int t0 = ((s_off[b + 1] - s_off[b]) + (jj - (b * p.nbT - s_off[b]))) * 64;
-                for (int i = tid; i < 128 * MT * 8; i += 128 * MT) {
+                for (int i = tid; i < 128 * MT * 8; i += 32 * EW) {
                     const int r = m * (128 * MT) + (i >> 3), cb = (i & 7) * 8;
                     if (r < p.M && t0 + cb < p.Tp) {
                         const size_t e = ((size_t)b * p.M + r) * p.Tp + t0 + cb;
@@ -738,15 +765,41 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
         int jt = 0, m, j, nb, cur_m = -1;
         long long pos = u_begin;
         float sn = 0.f, sd = 0.f, sq = 0.f, pivot = 0.f;     // statistics of this thread's channel over the CTA's range of one M tile
+        bool dead = false;            // a wait ran out: no further accumulator is touched, but every pair barrier below is still met
         auto flush_stats = [&]() {
             if (MODE != MODE_FWD || !p.stats || cur_m < 0) return;
+            float n = sn, sum = fmaf(pivot, sn, sd), m2 = sn > 0.f ? sq - sd * sd / sn : 0.f;
+            if (EPI == 2) {
+                // the two warps of a row hold the statistics of its two column halves: the second hands its triple
+                // over through its staging buffer (its stores have read it by then), the first merges (Chan) and writes
+                const uint32_t bar_id = 1 + mt * 4 + wq;
+                if (hsel == 1) {
+                    if (p.tma_out && lane == 0) ptx::bulk_wait_read();
+                    __syncwarp();
+                    reinterpret_cast<float4*>(stg)[lane] = make_float4(n, sum, m2, 0.f);
+                }
+                asm volatile("bar.sync %0, 64;" ::"r"(bar_id) : "memory");
+                if (hsel == 0) {
+                    const float4 o = reinterpret_cast<const float4*>(stg + 4 * MT * p.stg_stride)[lane];
+                    if (o.x > 0.f) {
+                        if (n > 0.f) {
+                            const float nt = n + o.x, dlt = o.y / o.x - sum / n;
+                            m2 += o.z + dlt * dlt * (n * o.x / nt);
+                            sum += o.y; n = nt;
+                        } else { n = o.x; sum = o.y; m2 = o.z; }
+                    }
+                }
+                asm volatile("bar.sync %0, 64;" ::"r"(bar_id) : "memory");
+                if (hsel == 1) return;
+            }
             const int row = cur_m * (128 * MT) + mt * 128 + wq * 32 + lane;
-            if (row < p.M) p.stats[(size_t)blockIdx.x * p.M + row] = make_float4(sn, fmaf(pivot, sn, sd), sn > 0.f ? sq - sd * sd / sn : 0.f, 0.f);
+            if (row < p.M) p.stats[(size_t)blockIdx.x * p.M + row] = make_float4(n, sum, m2, 0.f);
         };
         while (flat_next_tile<NB>(pos, u_end, nblk, m, j, nb)) {
             if (m != cur_m) { flush_stats(); cur_m = m; sn = sd = sq = 0.f; }
             const int buf = jt % NBUF;
-            if (!ptx::mbar_wait_warp(&acc_full[buf], (jt / NBUF) & 1)) { if (lane == 0) raise_status(p.status, kErrTimeout); break; }
+            if (dead) { ++jt; continue; }
+            if (!ptx::mbar_wait_warp(&acc_full[buf], (jt / NBUF) & 1)) { if (lane == 0) raise_status(p.status, kErrTimeout); dead = true; ++jt; continue; }
             ptx::tc_fence_after();
             const int row_w = m * (128 * MT) + mt * 128 + wq * 32;
             const int row = row_w + lane;
@@ -757,7 +810,7 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                 const int t0 = (j + i - s_off[b]) * 64;
                 const int len = min(p.len_out[b], p.Tp);
 #pragma unroll 1
-                for (int h = 0; h < 2; ++h) {
+                for (int h = (EPI == 2 ? hsel : 0); h < (EPI == 2 ? hsel + 1 : 2); ++h) {
                     const int c0 = t0 + 32 * h;
                     if (c0 >= p.Tp) break;
                     float f[32];
@@ -777,18 +830,18 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                         if (p.stats && nv > 0) {
                             if (sn == 0.f) pivot = f[0];
                             if (nv == 32) {
-                                // packed pairs: d = f - pivot, sum d, sum d^2 in three two-wide instructions per pair
-                                const uint64_t np2 = ptx::pack2(-pivot, -pivot);
-                                uint64_t sd2 = ptx::pack2(0.f, 0.f), sq2 = ptx::pack2(0.f, 0.f);
+                                // d = f - pivot, sum d, sum d^2 in four independent chains (a warp has one other warp to
+                                // share its scheduler with, so dependent adds would leave the issue slots empty; the
+                                // two-wide fp32 instructions were measured slower per element than the scalar ones)
+                                float d4[4] = {0.f, 0.f, 0.f, 0.f}, q4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                                for (int q = 0; q < 16; ++q) {
-                                    const uint64_t d2 = ptx::add2(ptx::pack2(f[2 * q], f[2 * q + 1]), np2);
-                                    sd2 = ptx::add2(sd2, d2);
-                                    sq2 = ptx::fma2(d2, d2, sq2);
+                                for (int q = 0; q < 32; ++q) {
+                                    const float d = f[q] - pivot;
+                                    d4[q & 3] += d;
+                                    q4[q & 3] = fmaf(d, d, q4[q & 3]);
                                 }
-                                float a0, a1, b0, b1;
-                                ptx::unpack2(sd2, a0, a1); ptx::unpack2(sq2, b0, b1);
-                                sd += a0 + a1; sq += b0 + b1;
+                                sd += (d4[0] + d4[1]) + (d4[2] + d4[3]);
+                                sq += (q4[0] + q4[1]) + (q4[2] + q4[3]);
                             } else {
 #pragma unroll
                                 for (int q = 0; q < 32; ++q) if (q < nv) { const float d = f[q] - pivot; sd += d; sq = fmaf(d, d, sq); }
@@ -803,7 +856,20 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                     }
                     const size_t base = ((size_t)b * p.M + row_w) * p.Tp + c0;
                     const int rl = p.M - row_w, cl = p.Tp - c0;
-                    if (MT == 1 && OCC == 1 && MODE == MODE_FWD && p.out_f32)
+                    if (p.tma_out) {
+                        // the previous store from this buffer has read its source; write, publish to the copy engine, store
+                        uint8_t* sb = stg + ((p.stg_nbuf == 2 && (nstore & 1)) ? 2048 : 0);
+                        if (lane == 0) { if (p.stg_nbuf == 2) ptx::bulk_wait_read1(); else ptx::bulk_wait_read(); }
+                        __syncwarp();
+                        if (MODE == MODE_FWD && p.out_half) stage_block16_swz<__half>(sb, f, lane);
+                        else stage_block16_swz<T>(sb, f, lane);
+                        ptx::fence_proxy_async();
+                        __syncwarp();
+                        if (row_w < p.M) {                                  // no box starts outside the tensor
+                            if (lane == 0) { ptx::tma_store_3d(&mapO, sb, c0, row_w, b); ptx::bulk_commit(); }
+                            ++nstore;
+                        }
+                    } else if (MT == 1 && OCC == 1 && MODE == MODE_FWD && p.out_f32)
                         store_block_staged<float>(reinterpret_cast<float*>(stg), f, reinterpret_cast<float*>(p.out) + base, p.Tp, rl, cl, lane);
                     else if (MODE == MODE_FWD && p.out_half)
                         store_block16<__half>(stg, f, reinterpret_cast<__half*>(p.out) + base, p.Tp, rl, cl, lane);
@@ -816,6 +882,7 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             ++jt;
         }
         flush_stats();
+        if (p.tma_out && lane == 0) ptx::bulk_wait_all();     // this thread's stores have completed
     }
     ptx::tc_fence_before();
     __syncthreads();
@@ -845,7 +912,7 @@ using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, voi
 }  // namespace
 
 bool tc_make_map(const TcState* st, void* map_out, int dtype, const void* base, int rank, const uint64_t* dims,
-                 const uint32_t* box) {
+                 const uint32_t* box, int swizzle_bytes) {
     CUtensorMap* m = static_cast<CUtensorMap*>(map_out);
     cuuint64_t gdim[3]; cuuint64_t gstride[2]; cuuint32_t bdim[3]; cuuint32_t estr[3] = {1, 1, 1};
     uint64_t stride = 2;
@@ -856,7 +923,8 @@ bool tc_make_map(const TcState* st, void* map_out, int dtype, const void* base, 
     }
     CUresult r = reinterpret_cast<EncodeFn>(st->encode_fn)(
         m, dtype == F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank,
-        const_cast<void*>(base), gdim, gstride, bdim, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+        const_cast<void*>(base), gdim, gstride, bdim, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+        swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { fprintf(stderr, "sepconv: cuTensorMapEncodeTiled failed (%d)\n", (int)r); return false; }
     return true;
@@ -864,8 +932,14 @@ bool tc_make_map(const TcState* st, void* map_out, int dtype, const void* base, 
 
 namespace {
 bool make_map(const TcState* st, CUtensorMap* m, int dtype, const void* base, int rank, const uint64_t* dims,
-              const uint32_t* box) {
-    return tc_make_map(st, m, dtype, base, rank, dims, box);
+              const uint32_t* box, int swizzle_bytes = 128) {
+    return tc_make_map(st, m, dtype, base, rank, dims, box, swizzle_bytes);
+}
+// map of a [B, M, Tp] 16-bit result for the epilogue's stores: boxes of 32 frames x 32 rows, 64-byte swizzle
+bool make_out_map(const TcState* st, CUtensorMap* m, const void* out, int B, int M, int Tp) {
+    const uint64_t d[3] = {(uint64_t)Tp, (uint64_t)M, (uint64_t)B};
+    const uint32_t b[3] = {32, 32, 1};
+    return make_map(st, m, F16, out, 3, d, b, 64);
 }
 
 template <typename T, int MODE, int MT, int BN, int STAGES>
@@ -956,35 +1030,48 @@ size_t tc_wgrad_scratch_bytes(const TcState*, int Cin, int Cout) {
 }
 
 namespace {
-template <typename T, int MODE, int MT, int NB, int NBUF, int OCC = 1>
-void launch_flat(const Launch& L, int sm_count, const CUtensorMap& a, const CUtensorMap& b, const FlatParams& p, int* grid_out) {
-    const int smem = FlatCfg<MT, NB, OCC>::smem_bytes(p.B);
-    auto kern = tc_gemm_flat_kernel<T, MODE, MT, NB, NBUF, OCC>;
-    set_max_smem_once<tc_gemm_flat_kernel<T, MODE, MT, NB, NBUF, OCC>>(FlatCfg<MT, NB, OCC>::smem_bytes(FlatCfg<MT, NB, OCC>::MAXB));
+template <typename T, int MODE, int MT, int NB, int NBUF, int OCC = 1, int EPI = 1>
+void launch_flat(const Launch& L, int sm_count, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& o, const FlatParams& p_in,
+                 int* grid_out) {
+    using Cfg = FlatCfg<MT, NB, OCC, EPI>;
+    FlatParams p = p_in;
+    // per-warp staging: the shape's own size, or (TMA stores, one CTA per SM, room left) two 2 KiB buffers
+    constexpr int kSmemMax = 232448;
+    p.stg_stride = Cfg::STG; p.stg_nbuf = Cfg::STG >= 4096 ? 2 : 1;
+    if (p.tma_out && OCC == 1 && Cfg::STG < 4096 && Cfg::smem_bytes(p.B) + 4 * MT * EPI * (4096 - Cfg::STG) <= kSmemMax) {
+        p.stg_stride = 4096; p.stg_nbuf = 2;
+    }
+    const int smem = Cfg::smem_bytes(p.B) + 4 * MT * EPI * (p.stg_stride - Cfg::STG);
+    auto kern = tc_gemm_flat_kernel<T, MODE, MT, NB, NBUF, OCC, EPI>;
+    set_max_smem_once<tc_gemm_flat_kernel<T, MODE, MT, NB, NBUF, OCC, EPI>>(OCC == 1 ? kSmemMax : Cfg::smem_bytes(Cfg::MAXB));
     const long long units = (long long)p.tiles_m * p.B * p.nbT;
     const int grid = (int)std::max(1ll, std::min<long long>(std::min(sm_count * OCC, kFlatMaxGrid), units));
-    launch_k(L, kern, grid, 32 * (4 * MT + 2), smem, a, b, p);
+    launch_k(L, kern, grid, 32 * (4 * MT * EPI + 2), smem, a, b, o, p);
     L.count();
     if (grid_out) *grid_out = grid;
 }
 // shape 0: 256 x 256 tiles, one accumulator; 1: 256 x 128 tiles, two accumulators; 2: 128 x 256 tiles, two accumulators;
-// 3: 128 x 256 tiles, one accumulator, two CTAs per SM
+// 3: 128 x 256 tiles, one accumulator, two CTAs per SM; 0 takes sixteen epilogue warps (two per 32 accumulator rows) when
+// the batch's block offsets fit beside their staging buffers, 4 is 0 with eight epilogue warps always
 template <typename T, int MODE>
 void launch_flat_shape(int shape, int mt, const Launch& L, int sm_count, const CUtensorMap& a, const CUtensorMap& b,
-                       const FlatParams& p, int* grid_out) {
-    if (shape == 3 && !p.out_f32 && p.B <= FlatCfg<1, 4, 2>::MAXB) { launch_flat<T, MODE, 1, 4, 1, 2>(L, sm_count, a, b, p, grid_out); return; }
-    if (mt == 1) { launch_flat<T, MODE, 1, 4, 2>(L, sm_count, a, b, p, grid_out); return; }
-    if (shape == 0) launch_flat<T, MODE, 2, 4, 1>(L, sm_count, a, b, p, grid_out);
-    else launch_flat<T, MODE, 2, 2, 2>(L, sm_count, a, b, p, grid_out);
+                       const CUtensorMap& o, const FlatParams& p, int* grid_out) {
+    if (shape == 3 && !p.out_f32 && p.B <= FlatCfg<1, 4, 2>::MAXB) { launch_flat<T, MODE, 1, 4, 1, 2>(L, sm_count, a, b, o, p, grid_out); return; }
+    if (mt == 1) { launch_flat<T, MODE, 1, 4, 2>(L, sm_count, a, b, o, p, grid_out); return; }
+    // sixteen epilogue warps need TMA stores (their 2 KiB staging buffers have the store's layout) and a batch
+    // whose block offsets fit beside those buffers
+    if (shape == 0 && p.tma_out && p.B <= FlatCfg<2, 4, 1, 2>::MAXB) launch_flat<T, MODE, 2, 4, 1, 1, 2>(L, sm_count, a, b, o, p, grid_out);
+    else if (shape == 0 || shape == 4) launch_flat<T, MODE, 2, 4, 1>(L, sm_count, a, b, o, p, grid_out);
+    else launch_flat<T, MODE, 2, 2, 2>(L, sm_count, a, b, o, p, grid_out);
 }
 template <int MODE>
 void launch_flat_dt(int dtype, int shape, int mt, const Launch& L, int sm_count, const CUtensorMap& a, const CUtensorMap& b,
-                    const FlatParams& p, int* grid_out) {
-    if (dtype == F16) launch_flat_shape<__half, MODE>(shape, mt, L, sm_count, a, b, p, grid_out);
-    else launch_flat_shape<__nv_bfloat16, MODE>(shape, mt, L, sm_count, a, b, p, grid_out);
+                    const CUtensorMap& o, const FlatParams& p, int* grid_out) {
+    if (dtype == F16) launch_flat_shape<__half, MODE>(shape, mt, L, sm_count, a, b, o, p, grid_out);
+    else launch_flat_shape<__nv_bfloat16, MODE>(shape, mt, L, sm_count, a, b, o, p, grid_out);
 }
 // M sub-tiles per CTA for a given tile shape and row count
-inline int flat_mt(int shape, int rows) { return (shape >= 2 || rows <= 128) ? 1 : 2; }
+inline int flat_mt(int shape, int rows) { return (shape == 2 || shape == 3 || rows <= 128) ? 1 : 2; }
 }  // namespace
 
 size_t tc_stats_bytes(int B, int Cout, int Tp) {
@@ -1013,8 +1100,10 @@ void tc_gemm_fwd(const TcState* st, const Launch& L, int dtype, const void* w, c
         p.zero_fill = partials ? 0 : 1;     // a linear layer's result is the block output: padding must read as zero
         p.out_half = (out_dtype == F16 && dtype != F16) ? 1 : 0;
         p.out_f32 = out_dtype == F32 ? 1 : 0;
+        CUtensorMap mo = ma;
+        p.tma_out = (!p.out_f32 && make_out_map(st, &mo, v, B, Cout, Tp)) ? 1 : 0;
         int grid = 0;
-        launch_flat_dt<MODE_FWD>(dtype, st->flat_shape, mt, L, st->sm_count, ma, mb, p, &grid);
+        launch_flat_dt<MODE_FWD>(dtype, st->flat_shape, mt, L, st->sm_count, ma, mb, mo, p, &grid);
         if (layout && partials) { layout->kind = 2; layout->grid = grid; layout->tiles_m = p.tiles_m; layout->rows_per_tile = 128 * mt; }
         return;
     }
@@ -1046,7 +1135,9 @@ void tc_gemm_dgrad(const TcState* st, const Launch& L, int dtype, const void* w,
         p.M = Cin; p.Kdim = Cout; p.B = B; p.Tp = Tp; p.nbT = (Tp + 63) / 64;
         p.tiles_m = (Cin + 128 * mt - 1) / (128 * mt);
         p.zero_fill = 1;
-        launch_flat_dt<MODE_DGRAD>(dtype, st->flat_shape, mt, L, st->sm_count, ma, mb, p, nullptr);
+        CUtensorMap mo = ma;
+        p.tma_out = make_out_map(st, &mo, gu, B, Cin, Tp) ? 1 : 0;
+        launch_flat_dt<MODE_DGRAD>(dtype, st->flat_shape, mt, L, st->sm_count, ma, mb, mo, p, nullptr);
         return;
     }
     TcParams p{};

@@ -18,10 +18,11 @@ struct TcState {
 
 int tc_init(TcState* st, int device, int sm_count);
 
-// Encodes a tiled tensor map (128-byte swizzle, zero fill outside the tensor) for a dense 16-bit tensor
-// whose dimensions, innermost first, are dims[0..rank-1]; map_out points to a CUtensorMap.
+// Encodes a tiled tensor map (128-byte swizzle by default, 64-byte with swizzle_bytes = 64; zero fill outside the
+// tensor) for a dense 16-bit tensor whose dimensions, innermost first, are dims[0..rank-1]; map_out points to a
+// CUtensorMap.
 bool tc_make_map(const TcState* st, void* map_out, int dtype, const void* base, int rank, const uint64_t* dims,
-                 const uint32_t* box);
+                 const uint32_t* box, int swizzle_bytes = 128);
 
 // Upper bound on statistics partials per sample that the fused epilogue may emit.
 int tc_max_parts_per_sample(int Tp);

@@ -105,6 +105,23 @@ def test_tensorcore_shapes(api, ctx, dtype, case):
     rep.check()
 
 
+@pytest.mark.parametrize("shape", [0, 1, 2, 3, 4])
+@pytest.mark.parametrize("case", [2, 4])
+def test_tile_shapes(api, ctx, shape, case):
+    """Every tile shape of the flattened-block contraction (forward with statistics, input gradient): a projection
+    block with channel tails on both sides, and a 512 -> 1024 pointwise layer (several M tiles per CTA range)."""
+    kw, B, T, ragged = TC_SHAPES[case]
+    L = si.LayerCfg(**kw)
+    d = _draw_block(L, 8 * B, T, "bf16", seed=300 + case, ragged=ragged, lo_frac=0.1)
+    ctx.set_tile_shape(shape)
+    try:
+        rep = U.run_block(ctx, api, L, "bf16", d.x, d.lengths, d.params[0], d.g)
+    finally:
+        ctx.set_tile_shape(0)
+    print(f"\ntile shape {shape} case {case}: {rep}")
+    rep.check()
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_len_one_and_full(api, ctx, dtype):
     L = si.LayerCfg(16, 16, K=9, residual="identity")
