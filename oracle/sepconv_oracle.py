@@ -107,6 +107,45 @@ def depthwise_bwd(gu, xm, wd, stride: int, dilation: int = 1):
     return gxp[:, :, P:P + T], dwd
 
 
+def conv_fwd(xm, w, stride: int, dilation: int = 1):
+    """Non-separable 1-D convolution over time (the convolution of the original Jasper block, which the
+    separable block factorises; paper section 4.1.1):
+        v[b,o,t] = sum_{c,k} w[o,c,k] * xm[b,c,t*stride + k*dilation - P],
+    zero outside [0,T), P = left padding.  Same conventions as depthwise_fwd (cross-correlation, "same"
+    padding, stride on the convolution)."""
+    B, C, T = xm.shape
+    K = w.shape[2]
+    P, Pr = same_padding(K, dilation)
+    Tp = out_time(T, K, stride, dilation)
+    xp = np.zeros((B, C, T + P + Pr), F64)
+    xp[:, :, P:P + T] = xm
+    v = np.zeros((B, w.shape[0], Tp), F64)
+    span = (Tp - 1) * stride + 1
+    for k in range(K):
+        v += np.einsum("oc,bct->bot", w[:, :, k], xp[:, :, k * dilation:k * dilation + span:stride], optimize=True)
+    return v
+
+
+def conv_bwd(gv, xm, w, stride: int, dilation: int = 1):
+    """Adjoint of conv_fwd: returns (gx, dw).
+    gx[b,c,tau] = sum over (o,k,t) with t*stride+k*dilation-P = tau of w[o,c,k]*gv[b,o,t];
+    dw[o,c,k]   = sum_{b,t} gv[b,o,t] * xm[b,c,t*stride+k*dilation-P]."""
+    B, C, T = xm.shape
+    K = w.shape[2]
+    P, Pr = same_padding(K, dilation)
+    Tp = gv.shape[2]
+    xp = np.zeros((B, C, T + P + Pr), F64)
+    xp[:, :, P:P + T] = xm
+    gxp = np.zeros_like(xp)
+    dw = np.zeros(w.shape, F64)
+    span = (Tp - 1) * stride + 1
+    for k in range(K):
+        o = k * dilation
+        gxp[:, :, o:o + span:stride] += np.einsum("oc,bot->bct", w[:, :, k], gv, optimize=True)
+        dw[:, :, k] = np.einsum("bot,bct->oc", gv, xp[:, :, o:o + span:stride], optimize=True)
+    return gxp[:, :, P:P + T], dw
+
+
 def pointwise_fwd(u, wp):
     """v[b,o,t] = sum_c wp[o,c] * u[b,c,t]."""
     return np.einsum("oc,bct->bot", wp, u, optimize=True)
@@ -190,9 +229,11 @@ def block_fwd(L, x, lengths, params, res_src=None):
     """
     x = np.asarray(x, dtype=F64)
     B, C_in, T = x.shape
-    s = L.stride if L.has_dw else 1
-    K = L.K if L.has_dw else 1
-    dil = getattr(L, "dilation", 1) if L.has_dw else 1
+    full = bool(getattr(L, "full_conv", False))         # block variant: one non-separable K-tap convolution
+    taps = L.has_dw or full
+    s = L.stride if taps else 1
+    K = L.K if taps else 1
+    dil = getattr(L, "dilation", 1) if taps else 1
     Tp = out_time(T, K, s, dil)
     lengths = np.asarray(lengths, dtype=np.int64)
     out_len = out_lengths(lengths, s)
@@ -202,10 +243,13 @@ def block_fwd(L, x, lengths, params, res_src=None):
     # mask on the conv input
     xm = np.where(time_mask(lengths, T), x, 0.0)
     S["xm"] = xm
-    u = depthwise_fwd(xm, _p(params, "wd"), s, dil) if L.has_dw else xm
-    u = np.where(valid, u, 0.0)                         # frames beyond len' are never used
-    S["u"] = u
-    v = pointwise_fwd(u, _p(params, "wp"))
+    if full:
+        v = conv_fwd(xm, _p(params, "wp"), s, dil)      # wp is [C_out, C_in, K] here
+    else:
+        u = depthwise_fwd(xm, _p(params, "wd"), s, dil) if L.has_dw else xm
+        u = np.where(valid, u, 0.0)                     # frames beyond len' are never used
+        S["u"] = u
+        v = pointwise_fwd(u, _p(params, "wp"))
     if L.has_bias:
         v = v + _p(params, "bias")[None, :, None]
     S["v"] = v
@@ -262,17 +306,22 @@ def block_infer(L, x, lengths, params, running, res_src=None):
     (plus out_len, valid)."""
     x = np.asarray(x, dtype=F64)
     B, C_in, T = x.shape
-    s = L.stride if L.has_dw else 1
-    K = L.K if L.has_dw else 1
-    dil = getattr(L, "dilation", 1) if L.has_dw else 1
+    full = bool(getattr(L, "full_conv", False))
+    taps = L.has_dw or full
+    s = L.stride if taps else 1
+    K = L.K if taps else 1
+    dil = getattr(L, "dilation", 1) if taps else 1
     Tp = out_time(T, K, s, dil)
     lengths = np.asarray(lengths, dtype=np.int64)
     out_len = out_lengths(lengths, s)
     valid = time_mask(out_len, Tp)
     xm = np.where(time_mask(lengths, T), x, 0.0)
-    u = depthwise_fwd(xm, _p(params, "wd"), s, dil) if L.has_dw else xm
-    u = np.where(valid, u, 0.0)
-    v = pointwise_fwd(u, _p(params, "wp"))
+    if full:
+        v = conv_fwd(xm, _p(params, "wp"), s, dil)
+    else:
+        u = depthwise_fwd(xm, _p(params, "wd"), s, dil) if L.has_dw else xm
+        u = np.where(valid, u, 0.0)
+        v = pointwise_fwd(u, _p(params, "wp"))
     if L.has_bias:
         v = v + _p(params, "bias")[None, :, None]
 
@@ -320,7 +369,8 @@ def block_bwd(L, g, lengths, params, S, gate=None):
     adds dx and dx_res."""
     g = np.asarray(g, dtype=F64)
     valid = S["valid"]
-    s = L.stride if L.has_dw else 1
+    full = bool(getattr(L, "full_conv", False))
+    s = L.stride if (L.has_dw or full) else 1
     T = S["xm"].shape[2]
     G = {}
     gm = np.where(valid, g, 0.0)                        # output mask
@@ -345,11 +395,14 @@ def block_bwd(L, g, lengths, params, S, gate=None):
         gv = ga
     if L.has_bias:
         G["dbias"] = np.sum(gv, axis=(0, 2))
-    gu, G["dwp"] = pointwise_bwd(gv, S["u"], _p(params, "wp"))
-    if L.has_dw:
-        gx, G["dwd"] = depthwise_bwd(gu, S["xm"], _p(params, "wd"), s, getattr(L, "dilation", 1))
+    if full:
+        gx, G["dwp"] = conv_bwd(np.where(valid, gv, 0.0), S["xm"], _p(params, "wp"), s, getattr(L, "dilation", 1))
     else:
-        gx = gu
+        gu, G["dwp"] = pointwise_bwd(gv, S["u"], _p(params, "wp"))
+        if L.has_dw:
+            gx, G["dwd"] = depthwise_bwd(gu, S["xm"], _p(params, "wd"), s, getattr(L, "dilation", 1))
+        else:
+            gx = gu
     G["dx"] = np.where(time_mask(lengths, T), gx, 0.0)
 
     if gr is not None:

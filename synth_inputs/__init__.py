@@ -75,12 +75,13 @@ class LayerCfg:
     eps: float = 1e-3
     log_softmax: bool = False       # decoder tail on a linear layer: log-softmax over the channels
     dilation: int = 1               # frames between neighbouring taps of the depthwise step
+    full_conv: bool = False         # block variant: one non-separable K-tap convolution [C_out, C_in, K] (needs has_dw=False)
 
     def param_shapes(self) -> Dict[str, tuple]:
         s: Dict[str, tuple] = {}
         if self.has_dw:
             s["wd"] = (self.C_in, self.K)
-        s["wp"] = (self.C_out, self.C_in)
+        s["wp"] = (self.C_out, self.C_in, self.K) if self.full_conv else (self.C_out, self.C_in)
         if self.has_bn:
             s["gamma"] = (self.C_out,)
             s["beta"] = (self.C_out,)
@@ -125,7 +126,7 @@ class Workload:
     def out_T(self) -> int:
         T = self.T
         for L in self.layers:
-            if L.has_dw:
+            if L.has_dw or L.full_conv:
                 T = (T - 1) // L.stride + 1      # "same" padding: dilation * (K - 1) zeros in total
         return T
 
@@ -220,7 +221,7 @@ def draw_layer_params(rng, L: LayerCfg, dtype: str, affine: str) -> Dict[str, np
         if name == "wd":
             a = quantise(_kaiming_uniform(rng, shp, L.K), dtype)
         elif name == "wp":
-            a = quantise(_kaiming_uniform(rng, shp, L.C_in), dtype)
+            a = quantise(_kaiming_uniform(rng, shp, L.C_in * (L.K if L.full_conv else 1)), dtype)
         elif name == "wr":
             a = quantise(_kaiming_uniform(rng, shp, L.C_res), dtype)
         elif name in ("gamma", "gamma_r"):

@@ -31,9 +31,10 @@ def rand_params(rng, L):
 # ----------------------------------------------------------------------------------------------
 def brute_block(L, x, lengths, p, res_src=None):
     B, Ci, T = x.shape
-    s = L.stride if L.has_dw else 1
-    K = L.K if L.has_dw else 1
-    dil = L.dilation if L.has_dw else 1
+    taps = L.has_dw or L.full_conv
+    s = L.stride if taps else 1
+    K = L.K if taps else 1
+    dil = L.dilation if taps else 1
     P = (dil * (K - 1)) // 2                 # zeros on the left; the right side gets the rest
     Tp = (T - 1) // s + 1
     Co = L.C_out
@@ -65,8 +66,14 @@ def brute_block(L, x, lengths, p, res_src=None):
                     out[b][o][t] = gamma[o] * (v[b][o][t] - mu) / math.sqrt(var + L.eps) + beta[o]
         return out
 
-    bn = pw_bn(u, p["wp"], p.get("gamma"), p.get("beta"), p.get("bias") if L.has_bias else None,
-               Ci, L.has_bn)
+    if L.full_conv:
+        # the non-separable convolution written as a pointwise contraction over the C_in * K shifted copies of x
+        cols = [[[xt(b, c, t * s + k * dil - P) for t in range(Tp)] for c in range(Ci) for k in range(K)] for b in range(B)]
+        wflat = [[p["wp"][o][c][k] for c in range(Ci) for k in range(K)] for o in range(Co)]
+        bn = pw_bn(cols, wflat, p.get("gamma"), p.get("beta"), p.get("bias") if L.has_bias else None, Ci * K, L.has_bn)
+    else:
+        bn = pw_bn(u, p["wp"], p.get("gamma"), p.get("beta"), p.get("bias") if L.has_bias else None,
+                   Ci, L.has_bn)
     r = None
     if L.residual != "none":
         rs = x if res_src is None else res_src
@@ -97,6 +104,10 @@ TINY = [
     dict(C_in=3, C_out=3, K=4, stride=1, residual="identity"),            # even K: one more zero on the right
     dict(C_in=2, C_out=3, K=3, stride=1, dilation=2, residual="proj"),
     dict(C_in=2, C_out=2, K=2, stride=2, dilation=3, residual="none"),
+    # non-separable convolution (the original Jasper block's)
+    dict(C_in=3, C_out=3, K=3, has_dw=False, full_conv=True, residual="identity"),
+    dict(C_in=2, C_out=3, K=4, stride=2, dilation=2, has_dw=False, full_conv=True, residual="none"),
+    dict(C_in=2, C_out=2, K=3, has_dw=False, full_conv=True, has_bn=False, has_relu=False, has_bias=True),
 ]
 
 
@@ -560,6 +571,63 @@ def test_same_padding_convention_matches_torch(K, dil):
     np.testing.assert_allclose(gx, xt.grad.numpy(), atol=1e-12)
     np.testing.assert_allclose(dwd, wt.grad.numpy(), atol=1e-12)
     assert O.out_time(11, K, 1, dil) == 11 and O.out_time(11, K, 2, dil) == 6
+
+
+@pytest.mark.parametrize("K,stride,dil", [(3, 1, 1), (4, 1, 1), (5, 2, 1), (3, 1, 2), (4, 2, 3)])
+def test_full_conv_matches_torch(K, stride, dil):
+    """The non-separable convolution against torch's dense conv1d (explicit zero padding: dilation*(K-1) in total,
+    the odd one on the right), forward and both gradients."""
+    rng = np.random.default_rng(60 + K + stride + dil)
+    x = rng.standard_normal((2, 3, 11))
+    w = rng.standard_normal((4, 3, K))
+    Tp = O.out_time(11, K, stride, dil)
+    g = rng.standard_normal((2, 4, Tp))
+    v = O.conv_fwd(x, w, stride, dil)
+    xt, wt = torch.tensor(x, requires_grad=True), torch.tensor(w, requires_grad=True)
+    pl, pr = O.same_padding(K, dil)
+    ref = F.conv1d(F.pad(xt, (pl, pr)), wt, stride=stride, dilation=dil)
+    assert ref.shape[2] == Tp
+    np.testing.assert_allclose(v, ref.detach().numpy(), atol=1e-12)
+    ref.backward(torch.tensor(g))
+    gx, dw = O.conv_bwd(g, x, w, stride, dil)
+    np.testing.assert_allclose(gx, xt.grad.numpy(), atol=1e-12)
+    np.testing.assert_allclose(dw, wt.grad.numpy(), atol=1e-12)
+    if stride == 1:
+        np.testing.assert_allclose(v, F.conv1d(xt, wt, padding="same", dilation=dil).detach().numpy(), atol=1e-12)
+
+
+def test_full_conv_with_factorised_weights_is_the_separable_block():
+    """w[o,c,k] = wp[o,c] * wd[c,k] makes the non-separable convolution the depthwise step followed by the pointwise
+    step: the two variants of the block then agree on every output and input gradient, and the full weight gradient
+    contracts to the two separable ones.  K = 1 is the pointwise layer itself."""
+    rng = np.random.default_rng(71)
+    B, T = 3, 12
+    for kw in (dict(K=5, stride=1), dict(K=3, stride=2), dict(K=4, stride=1, dilation=2)):
+        Ls = si.LayerCfg(4, 5, residual="proj", **kw)
+        Lf = si.LayerCfg(4, 5, residual="proj", has_dw=False, full_conv=True, **kw)
+        x = rng.standard_normal((B, 4, T))
+        lengths = np.array([T, T, T])          # the separable path zeroes u beyond len'; with full lengths nothing is beyond
+        ps = rand_params(rng, Ls)
+        pf = {k: v for k, v in ps.items() if k != "wd"}
+        pf["wp"] = ps["wp"][:, :, None] * ps["wd"][None, :, :]
+        res = rng.standard_normal((B, 4, O.out_time(T, kw["K"], kw["stride"], kw.get("dilation", 1))))
+        g = rng.standard_normal((B, 5, res.shape[2]))
+        Ss, Sf = O.block_fwd(Ls, x, lengths, ps, res_src=res), O.block_fwd(Lf, x, lengths, pf, res_src=res)
+        np.testing.assert_allclose(Sf["v"], Ss["v"], atol=1e-11)
+        np.testing.assert_allclose(Sf["y"], Ss["y"], atol=1e-11)
+        Gs, Gf = O.block_bwd(Ls, g, lengths, ps, Ss), O.block_bwd(Lf, g, lengths, pf, Sf)
+        np.testing.assert_allclose(Gf["dx"], Gs["dx"], atol=1e-10)
+        np.testing.assert_allclose(Gf["dx_res"], Gs["dx_res"], atol=1e-10)
+        np.testing.assert_allclose(np.einsum("ock,ck->oc", Gf["dwp"], ps["wd"]), Gs["dwp"], atol=1e-10)
+        np.testing.assert_allclose(np.einsum("ock,oc->ck", Gf["dwp"], ps["wp"]), Gs["dwd"], atol=1e-10)
+        for n in ("dgamma", "dbeta", "dwr", "dgamma_r", "dbeta_r"):
+            np.testing.assert_allclose(Gf[n], Gs[n], atol=1e-10, err_msg=n)
+    Lp = si.LayerCfg(4, 5, K=1, has_dw=False)
+    Lq = si.LayerCfg(4, 5, K=1, has_dw=False, full_conv=True)
+    x = rng.standard_normal((B, 4, T)); lengths = np.array([T, 5, 9])
+    pp = rand_params(rng, Lp)
+    pq = dict(pp); pq["wp"] = pp["wp"][:, :, None]
+    np.testing.assert_allclose(O.block_fwd(Lq, x, lengths, pq)["y"], O.block_fwd(Lp, x, lengths, pp)["y"], atol=1e-12)
 
 
 def test_running_stats():
