@@ -103,6 +103,11 @@ typedef struct {
                                 /* module's log_probs (section 4.1.1); only on a layer with has_bn = 0,  */
                                 /* has_relu = 0 and no residual.  Backward then takes dL/dlog_probs      */
     int32_t dilation;           /* frames between neighbouring depthwise taps (0 or 1: adjacent)          */
+    int32_t full_conv;          /* 1: block variant with ONE non-separable K-tap convolution in place of  */
+                                /* depthwise + pointwise (the convolution of the original Jasper block,   */
+                                /* section 4.1.1): params.wp is [C_out, C_in, K]; K, stride and dilation   */
+                                /* apply to it with the depthwise step's conventions; has_dw must be 0 and */
+                                /* log_softmax 0; saved.u is not used.  Plain (non-tensor-core) kernels    */
 } sc_block_desc;
 
 typedef struct {          /* device pointers; absent parts may be null                             */

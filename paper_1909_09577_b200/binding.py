@@ -41,11 +41,12 @@ class sc_block_desc(C.Structure):
                 ("residual", C.c_int32), ("C_res", C.c_int32),
                 ("has_dw", C.c_int32), ("has_bn", C.c_int32), ("has_relu", C.c_int32),
                 ("has_bias", C.c_int32), ("res_before_relu", C.c_int32),
-                ("bn_eps", C.c_float), ("bn_momentum", C.c_float), ("log_softmax", C.c_int32), ("dilation", C.c_int32)]
+                ("bn_eps", C.c_float), ("bn_momentum", C.c_float), ("log_softmax", C.c_int32), ("dilation", C.c_int32),
+                ("full_conv", C.c_int32)]
 
     @property
     def T_out(self) -> int:
-        s = self.stride if self.has_dw else 1
+        s = self.stride if (self.has_dw or self.full_conv) else 1
         return (self.T_in - 1) // s + 1
 
 
@@ -175,6 +176,7 @@ def block_desc(L, B: int, T: int, dtype: str) -> sc_block_desc:
     d.bn_momentum = 0.1
     d.log_softmax = int(getattr(L, "log_softmax", False))
     d.dilation = int(getattr(L, "dilation", 1))
+    d.full_conv = int(getattr(L, "full_conv", False))
     return d
 
 

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libsepconv_b200.so")
-SOURCES = ["api.cu", "k_bn.cu", "k_depthwise.cu", "k_depthwise_tc.cu", "k_dw_wgrad_tc.cu", "k_depthwise_tma.cu", "k_gemm_simt.cu", "tc_gemm.cu", "static_scratch.cu", "k_decoder.cu"]
+SOURCES = ["api.cu", "k_bn.cu", "k_depthwise.cu", "k_depthwise_tc.cu", "k_dw_wgrad_tc.cu", "k_depthwise_tma.cu", "k_gemm_simt.cu", "tc_gemm.cu", "static_scratch.cu", "k_decoder.cu", "k_conv_simt.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 NVCC_FLAGS = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")]

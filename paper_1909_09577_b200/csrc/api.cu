@@ -55,15 +55,18 @@ struct Bump {
     bool ok() const { return base == nullptr || off <= cap; }
 };
 
-struct Dims { int B, Cin, Cout, Cres, T, Tp, K, s, dil; bool plain; };   // plain: odd K, adjacent taps
+struct Dims { int B, Cin, Cout, Cres, T, Tp, K, s, dil; bool plain, full; };   // plain: odd K, adjacent taps; full: non-separable convolution
 
 int desc_dims(const sc_block_desc* d, Dims* o) {
     if (!d) return SC_ERR_NULL;
     if (d->io_dtype < 0 || d->io_dtype > 2) return SC_ERR_INCOMPATIBLE;
     if (d->B < 1 || d->C_in < 1 || d->C_out < 1 || d->T_in < 1) return SC_ERR_DIM_INCOMPATIBLE;
     o->B = d->B; o->Cin = d->C_in; o->Cout = d->C_out; o->T = d->T_in;
-    o->K = d->has_dw ? d->K : 1; o->s = d->has_dw ? d->stride : 1;
-    o->dil = (d->has_dw && d->dilation > 1) ? d->dilation : 1;
+    o->full = d->full_conv != 0;
+    if (o->full && (d->has_dw || d->log_softmax)) return SC_ERR_UNSUPPORTED;
+    const bool taps = d->has_dw || o->full;       // the K-tap step: depthwise, or the non-separable convolution
+    o->K = taps ? d->K : 1; o->s = taps ? d->stride : 1;
+    o->dil = (taps && d->dilation > 1) ? d->dilation : 1;
     if (d->dilation < 0 || o->K < 1) return SC_ERR_UNSUPPORTED;
     if (o->s != 1 && o->s != 2) return SC_ERR_UNSUPPORTED;
     o->plain = o->dil == 1 && (o->K & 1);
@@ -191,8 +194,26 @@ int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
                           sv->invstd_r, f.partials_r, nullptr, nullptr);
         record_side(ctx, ctx->ev[5]);
     }
-    const void* u;
-    if (d->has_dw) {
+    if (m.full) {
+        // block variant: one K-tap convolution over all input channels (it masks its input by len_in itself)
+        if (!d->has_bn) {
+            conv_fwd_simt(L, dt, p->wp, io.x, d->has_bias ? p->bias : nullptr, io.y, dt, io.len_in, io.len_out, m.B, m.Cin, m.Cout,
+                          m.T, m.Tp, m.K, m.s, m.dil);
+            return SC_OK;
+        }
+        const int vdt = ntype_of(dt);
+        conv_fwd_simt(L, dt, p->wp, io.x, nullptr, sv->v, vdt, io.len_in, io.len_out, m.B, m.Cin, m.Cout, m.T, m.Tp, m.K, m.s, m.dil);
+        if (inf) {
+            invstd_from_var(L, inf->var, d->bn_eps, sv->invstd, m.Cout);
+        } else {
+            bn_stats(L, vdt, sv->v, io.len_out, m.B, m.Cout, m.Tp, (float2*)f.partials);
+            bn_finalize(L, (const float2*)f.partials, 1, m.Tp, io.len_out, io.nvalid, m.B, m.Cout, d->bn_eps, d->bn_momentum, sv->mean,
+                        sv->invstd, rmean, rvar);
+        }
+    }
+    const void* u = nullptr;
+    if (m.full) {
+    } else if (d->has_dw) {
         if (ctx->gemm_mode == 0 && m.plain && dw_tma_supported(&ctx->tc, dt, m.B, m.T, m.K, m.s))
             dw_tma_fwd(&ctx->tc, L, dt, odt, io.x, p->wd, sv->u, io.len_in, io.len_out, m.B, m.Cin, m.T, m.K,
                        io.x_clean ? 1 : 0);
@@ -219,12 +240,13 @@ int block_fwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
         return SC_OK;
     }
     const void* wp_op = p->wp;
-    if (odt != dt) {
+    if (odt != dt && !m.full) {
         void* dst = io.w16_keep ? io.w16_keep : f.w16;
         if (!(io.w16_keep && io.w16_ready)) convert_bf16_to_f16(L, p->wp, dst, (int64_t)m.Cout * m.Cin);
         wp_op = dst;
     }
-    if (inf) pointwise_fixed(ctx, L, d, m, m.Cin, odt, wp_op, u, sv->v, io.len_out, io.blk_off, inf->var, sv->invstd);
+    if (m.full) {}
+    else if (inf) pointwise_fixed(ctx, L, d, m, m.Cin, odt, wp_op, u, sv->v, io.len_out, io.blk_off, inf->var, sv->invstd);
     else pointwise_bn(ctx, L, d, m, m.Cin, odt, wp_op, u, sv->v, io.len_out, io.nvalid, io.blk_off, sv->mean, sv->invstd,
                       f.partials, rmean, rvar);
     ApplyArgs a{};
@@ -252,7 +274,9 @@ struct BwdScratch {
 
 void plan_bwd(const sc_block_desc* d, const Dims& m, Bump& ws, BwdScratch* s, const TcState* tc) {
     const size_t e = esize(d->io_dtype);
-    const size_t act_out = e * m.B * m.Cout * m.Tp, act_in = e * m.B * m.Cin * m.Tp;
+    // gu holds the gradient w.r.t. the pointwise operand [B, C_in, T']; with the non-separable convolution it is the
+    // staging tensor of the input gradient [B, C_in, T]
+    const size_t act_out = e * m.B * m.Cout * m.Tp, act_in = e * m.B * m.Cin * (m.full ? m.T : m.Tp);
     s->len_out = (int*)ws.take(sizeof(int) * m.B);
     s->nvalid = (int*)ws.take(sizeof(int));
     s->blk_off = (int*)ws.take(sizeof(int) * (m.B + 1));
@@ -269,7 +293,7 @@ void plan_bwd(const sc_block_desc* d, const Dims& m, Bump& ws, BwdScratch* s, co
     s->gu = ws.take(act_in);
     s->gxr = d->residual == SC_RES_PROJ ? ws.take(e * m.B * m.Cres * m.Tp) : nullptr;
     s->xr = d->residual == SC_RES_PROJ ? ws.take(e * m.B * m.Cres * m.Tp) : nullptr;
-    const bool bf = d->io_dtype == SC_BF16 && d->has_bn;
+    const bool bf = d->io_dtype == SC_BF16 && d->has_bn && !m.full;
     s->gv16 = (bf && !d->has_dw) ? ws.take(act_out) : nullptr;
     s->x16 = (bf && !d->has_dw) ? ws.take(act_in) : nullptr;
     s->gvr16 = (bf && d->residual == SC_RES_PROJ) ? ws.take(act_out) : nullptr;
@@ -277,6 +301,7 @@ void plan_bwd(const sc_block_desc* d, const Dims& m, Bump& ws, BwdScratch* s, co
     size_t wb = gemm_wgrad_simt_scratch_bytes(m.B, std::max(m.Cin, m.Cres), m.Cout);
     wb = std::max(wb, tc_wgrad_scratch_bytes(tc, std::max(m.Cin, m.Cres), m.Cout));
     wb = std::max(wb, dw_wgrad_scratch_bytes(m.B, m.Cin, m.K));
+    if (m.full) wb = std::max(wb, conv_wgrad_scratch_bytes(m.B, m.Cin, m.Cout, m.K));
     s->wpart = (float*)ws.take(wb);
     s->wpart_bytes = wb;
 }
@@ -317,7 +342,7 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
     // half copy of that gradient, and of the other operand, for their weight-gradient contraction: with
     // 8 significand bits the rounding of the gradient alone uses most of the error budget of dwp / dwr
     const bool tc_ok = ctx->gemm_mode == 0;
-    const bool half_gv = dt == SC_BF16 && d->has_bn && !d->has_dw && s.gv16 && tc_ok &&
+    const bool half_gv = dt == SC_BF16 && d->has_bn && !d->has_dw && !m.full && s.gv16 && tc_ok &&
                          tc_wgrad_supported(&ctx->tc, SC_F16, m.Cin, m.Cout, m.Tp);
     const bool half_gvr = dt == SC_BF16 && d->has_bn && d->residual == SC_RES_PROJ && s.gvr16 && tc_ok &&
                           tc_wgrad_supported(&ctx->tc, SC_F16, m.Cres, m.Cout, m.Tp);
@@ -350,7 +375,9 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
     const Launch Ls = side_launch(ctx, L);
     fork_to_side(ctx, L, ctx->ev[0]);                   // gv, gvr and their half copies are complete
     const void* u = d->has_dw ? sv->u : (io.x_clean ? io.x : sv->u);
-    if (half_gv) {
+    if (m.full) {
+        conv_wgrad_simt(Ls, dt, s.gv, io.x, g->dwp, s.wpart, acc, io.len_in, io.len_out, m.B, m.Cin, m.Cout, m.T, m.Tp, m.K, m.s, m.dil);
+    } else if (half_gv) {
         mask_convert_f16(Ls, s.x16, io.x, io.len_in, m.B, m.Cin, m.T);
         pointwise_wgrad(ctx, Ls, SC_F16, s.gv16, s.x16, g->dwp, s.wpart, acc, m.B, m.Cin, m.Cout, m.Tp, io.len_out, gmax);
     } else {
@@ -369,7 +396,7 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
     }
 
     const void* wp_op = p->wp;
-    if (odt != dt) {
+    if (odt != dt && !m.full) {
         if (io.w16_kept) wp_op = io.w16_kept;
         else { convert_bf16_to_f16(L, p->wp, s.w16, (int64_t)m.Cout * m.Cin); wp_op = s.w16; }
     }
@@ -382,7 +409,13 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
         extra = s.gres;
     }
 
-    if (d->has_dw) {
+    if (m.full) {
+        if (io.dx) {
+            void* tgt = (!io.dx_add && !extra) ? io.dx : s.gu;
+            conv_dgrad_simt(L, dt, p->wp, s.gv, tgt, io.len_in, io.len_out, m.B, m.Cin, m.Cout, m.T, m.Tp, m.K, m.s, m.dil);
+            if (tgt != io.dx) ew_add_masked(L, dt, io.dx, s.gu, io.dx_add, extra, io.len_in, m.B, m.Cin, m.T);
+        }
+    } else if (d->has_dw) {
         pointwise_dgrad(ctx, L, odt, wp_op, s.gv, s.gu, m.B, m.Cin, m.Cout, m.Tp, io.len_out, io.blk_off);
         fork_to_side(ctx, L, ctx->ev[1]);               // gu is complete
         if (ctx->gemm_mode == 0 && m.plain && dw_wgrad_tc_supported(&ctx->tc, dt, m.B, m.T, m.K, m.s))
@@ -421,7 +454,7 @@ int check_params(const sc_block_desc* d, const sc_block_params* p) {
 }
 int check_saved(const sc_block_desc* d, const sc_block_saved* s, bool x_clean) {
     if (!s) return SC_ERR_NULL;
-    if ((d->has_dw || !x_clean) && !s->u) return SC_ERR_NULL;
+    if (!d->full_conv && (d->has_dw || !x_clean) && !s->u) return SC_ERR_NULL;
     if (d->has_bn && (!s->v || !s->mean || !s->invstd)) return SC_ERR_NULL;
     if (d->residual == SC_RES_PROJ && (!s->vr || !s->mean_r || !s->invstd_r)) return SC_ERR_NULL;
     return SC_OK;

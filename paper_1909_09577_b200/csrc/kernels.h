@@ -156,6 +156,18 @@ void convert_bf16_to_f16(const Launch& L, const void* src, void* dst, int64_t n)
 struct ConvertList { const void* src[48]; void* dst[48]; int n[48]; int count; };
 void convert_bf16_to_f16_many(const Launch& L, const ConvertList& list);
 
+// ---- non-separable convolution (block variant; k_conv_simt.cu) ---------------------------------
+// w [Cout, Cin, K] and x [B, Cin, T] in `dtype`; v [B, Cout, Tp] in out_dtype (dtype, or F16 for BF16 operands).
+// "Same" padding with (dil * (K - 1)) / 2 zeros on the left; the input is read as zero from len_in[b] on, the
+// result is zero from len_out[b] on.  gv zero in padding is not assumed.
+void conv_fwd_simt(const Launch& L, int dtype, const void* w, const void* x, const float* bias, void* v, int out_dtype,
+                   const int* len_in, const int* len_out, int B, int Cin, int Cout, int T, int Tp, int K, int stride, int dil);
+void conv_dgrad_simt(const Launch& L, int dtype, const void* w, const void* gv, void* dx, const int* len_in, const int* len_out,
+                     int B, int Cin, int Cout, int T, int Tp, int K, int stride, int dil);
+size_t conv_wgrad_scratch_bytes(int B, int Cin, int Cout, int K);
+void conv_wgrad_simt(const Launch& L, int dtype, const void* gv, const void* x, float* dw, float* partials, int accumulate,
+                     const int* len_in, const int* len_out, int B, int Cin, int Cout, int T, int Tp, int K, int stride, int dil);
+
 // ---- batch norm -----------------------------------------------------------------------------
 // Per-(b,channel) row moments over t < len_out[b]: partials[(b*C+o)] = (sum, M2 about the row mean).
 void bn_stats(const Launch& L, int vdtype, const void* v, const int* len_out, int B, int C, int Tp,

@@ -45,6 +45,12 @@ SMALL = [
     (dict(C_in=16, C_out=24, K=4, residual="proj"), 3, 72, True),
     (dict(C_in=16, C_out=16, K=11, dilation=3, residual="identity"), 3, 120, True),
     (dict(C_in=8, C_out=16, K=6, dilation=2, stride=2, residual="none"), 2, 131, True),
+    # block variant: one non-separable K-tap convolution (tiles with channel and frame tails, stride 2, dilation,
+    # even K, a linear layer with bias)
+    (dict(C_in=24, C_out=40, K=5, has_dw=False, full_conv=True, residual="proj"), 3, 77, True),
+    (dict(C_in=70, C_out=70, K=11, has_dw=False, full_conv=True, residual="identity"), 5, 150, True),
+    (dict(C_in=16, C_out=24, K=4, stride=2, dilation=2, has_dw=False, full_conv=True, residual="none"), 6, 131, True),
+    (dict(C_in=16, C_out=8, K=3, has_dw=False, full_conv=True, has_bn=False, has_relu=False, has_bias=True), 2, 40, True),
 ]
 
 

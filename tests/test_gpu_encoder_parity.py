@@ -118,6 +118,23 @@ def test_tiny_encoder(api, ctx, dtype, ragged):
         assert rep.worst()[1] <= E2E_GRAD_LIMIT, rep.worst()
 
 
+def test_encoder_with_non_separable_prologue(api, ctx):
+    """The encoder driver with the original Jasper block's convolution in two places: a strided non-separable prologue
+    and a non-separable layer that closes a residual span."""
+    base = si.tiny_encoder(dtype="bf16", B=6, T=256, ragged=True, width=32)
+    layers = list(base.layers)
+    L0, L3 = layers[0], layers[3]
+    layers[0] = si.LayerCfg(L0.C_in, L0.C_out, K=L0.K, stride=L0.stride, has_dw=False, full_conv=True)
+    layers[3] = si.LayerCfg(L3.C_in, L3.C_out, K=L3.K, has_dw=False, full_conv=True, residual="proj", res_from=L3.res_from,
+                            C_res_override=L3.C_res_override)
+    w = si.Workload("tiny_encoder_jasper_prologue", base.dtype, base.B, base.T, layers, 21, len_lo=base.len_lo, len_hi=base.len_hi,
+                    affine=base.affine)
+    d = si.draw(w)
+    reports, chain = U.run_chain(ctx, api, w, d)          # every layer against the oracle, teacher-forced
+    spec, logits, out_len, gblob, dx = run_encoder(ctx, api, w, d)
+    assert_encoder_equals_chain(w, d, spec, logits, out_len, gblob, dx, chain)
+
+
 def test_encoder_without_dx_and_accumulate(api, ctx):
     w = si.tiny_encoder(dtype="bf16", B=2, T=64, ragged=True, width=32)
     d = si.draw(w)
