@@ -415,7 +415,7 @@ def main():
     line["roofline_per_class"] = per_class
     line["roofline_note"] = ("class times: CUDA events around every launch of %d host-launched steps run right after the "
                              "timed region, one stream, no overlap (they sum to %.3f ms/step against %.3f ms for the "
-                             "replayed graph, in which independent kernels overlap); bytes and "
+                             "timed step, in which independent kernels overlap); bytes and "
                              "flops are algorithmic, valid frames only; peaks: %s HBM %.0f GB/s, bf16 %.0f TFLOP/s sustained"
                              % (nprof, sum(v["ms_per_step"] for v in per_class.values()), ms / args.steps,
                                 peaks["source"], peaks["hbm_gbs"], peaks["bf16_tflops_sustained"]))

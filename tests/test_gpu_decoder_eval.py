@@ -78,6 +78,7 @@ INFER_CASES = [
     (dict(C_in=64, C_out=256, K=33, stride=2), 4, 400),
     (dict(C_in=512, C_out=1024, K=1, has_dw=False), 2, 264),
     (dict(C_in=1024, C_out=29, K=1, has_dw=False, has_bn=False, has_relu=False, has_bias=True, log_softmax=True), 3, 200),
+    (dict(C_in=24, C_out=40, K=5, stride=2, has_dw=False, full_conv=True), 3, 78),        # non-separable convolution
 ]
 
 
