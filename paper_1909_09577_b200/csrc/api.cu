@@ -24,7 +24,7 @@ struct sc_ctx {
     // residual projection's contraction) run there, forked from and joined back into the caller's stream with
     // events, so that they fill the SMs a latency-bound kernel of the critical path leaves idle.
     cudaStream_t side = nullptr;
-    cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};   // fork A, fork B, done[2], fwd fork, fwd join
+    cudaEvent_t ev[8] = {};     // backward fork, (unused), done[0], done[1], forward fork, forward join, done[2], (unused)
     int overlap = 1;
     int pdl = 1;          // launch kernels with programmatic stream serialization
 };
@@ -329,6 +329,8 @@ struct BwdIO {
     bool x_clean, res_clean;
     const void* w16_kept;        // float16 copy of wp left by the forward pass (optional)
     cudaEvent_t done;            // recorded on the side stream after this layer's last side-stream kernel
+    float* gmax_zeroed;          // optional: a float the caller has already set to zero, used for the |gv| bound
+                                 // (a memset between two kernels would end the programmatic overlap of that pair)
 };
 
 int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const Dims& m, BwdIO io,
@@ -346,8 +348,8 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
                          tc_wgrad_supported(&ctx->tc, SC_F16, m.Cin, m.Cout, m.Tp);
     const bool half_gvr = dt == SC_BF16 && d->has_bn && d->residual == SC_RES_PROJ && s.gvr16 && tc_ok &&
                           tc_wgrad_supported(&ctx->tc, SC_F16, m.Cres, m.Cout, m.Tp);
-    float* gmax = (dt != SC_F32 && d->has_bn && (d->has_dw || half_gv || half_gvr)) ? s.gmax : nullptr;
-    if (gmax) cudaMemsetAsync(gmax, 0, sizeof(float), L.stream);
+    float* gmax = (dt != SC_F32 && d->has_bn && (d->has_dw || half_gv || half_gvr)) ? (io.gmax_zeroed ? io.gmax_zeroed : s.gmax) : nullptr;
+    if (gmax && !io.gmax_zeroed) cudaMemsetAsync(gmax, 0, sizeof(float), L.stream);
     const void* dy = io.dy;
     if (d->log_softmax) {      // upstream gradient is w.r.t. the log-probabilities: back through the log-softmax first
         log_softmax_bwd(L, dt, s.dz, io.dy, io.y, io.len_out, m.B, m.Cout, m.Tp);
@@ -370,30 +372,43 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
                            d->has_bias ? g->dbias : nullptr, acc);
     bn_bwd_apply(L, dt, a);
 
-    // The weight gradients are off the critical path (nothing later in the backward pass reads them): they run on
-    // the side stream while this stream goes on with the input gradients.
+    // The weight gradients are off the critical path (nothing later in the backward pass reads them): they run on the
+    // side stream.  They are enqueued after the input-gradient kernels of this stream: the host issues launches in
+    // program order, and kernels of the critical path that sit behind side-stream launches in that order start late
+    // whenever the GPU is ahead of the host.  One event, recorded behind this layer's last main-stream kernel, releases
+    // them (an event between two kernels ends the programmatic overlap of that pair, so there is only one per layer);
+    // they then overlap the next layer's main-stream kernels.
     const Launch Ls = side_launch(ctx, L);
-    fork_to_side(ctx, L, ctx->ev[0]);                   // gv, gvr and their half copies are complete
-    const void* u = d->has_dw ? sv->u : (io.x_clean ? io.x : sv->u);
-    if (m.full) {
-        conv_wgrad_simt(Ls, dt, s.gv, io.x, g->dwp, s.wpart, acc, io.len_in, io.len_out, m.B, m.Cin, m.Cout, m.T, m.Tp, m.K, m.s, m.dil);
-    } else if (half_gv) {
-        mask_convert_f16(Ls, s.x16, io.x, io.len_in, m.B, m.Cin, m.T);
-        pointwise_wgrad(ctx, Ls, SC_F16, s.gv16, s.x16, g->dwp, s.wpart, acc, m.B, m.Cin, m.Cout, m.Tp, io.len_out, gmax);
-    } else {
-        pointwise_wgrad(ctx, Ls, odt, s.gv, u, g->dwp, s.wpart, acc, m.B, m.Cin, m.Cout, m.Tp, io.len_out,
-                        a.gv_scaled ? gmax : nullptr);
-    }
-    if (d->residual == SC_RES_PROJ) {
-        if (half_gvr) {
-            mask_convert_f16(Ls, s.xr16, io.xres, io.len_out, m.B, m.Cres, m.Tp);
-            pointwise_wgrad(ctx, Ls, SC_F16, s.gvr16, s.xr16, g->dwr, s.wpart, acc, m.B, m.Cres, m.Cout, m.Tp, io.len_out, gmax);
+    auto weight_gradients = [&]() {
+        fork_to_side(ctx, L, ctx->ev[0]);               // gv, gvr, gu and the half copies are complete
+        const void* u = d->has_dw ? sv->u : (io.x_clean ? io.x : sv->u);
+        if (m.full) {
+            conv_wgrad_simt(Ls, dt, s.gv, io.x, g->dwp, s.wpart, acc, io.len_in, io.len_out, m.B, m.Cin, m.Cout, m.T, m.Tp, m.K, m.s, m.dil);
+        } else if (half_gv) {
+            mask_convert_f16(Ls, s.x16, io.x, io.len_in, m.B, m.Cin, m.T);
+            pointwise_wgrad(ctx, Ls, SC_F16, s.gv16, s.x16, g->dwp, s.wpart, acc, m.B, m.Cin, m.Cout, m.Tp, io.len_out, gmax);
         } else {
-            const void* xr = io.xres;
-            if (!io.res_clean) { mask_copy(Ls, dt, s.xr, io.xres, io.len_out, m.B, m.Cres, m.Tp); xr = s.xr; }
-            pointwise_wgrad(ctx, Ls, dt, s.gvr, xr, g->dwr, s.wpart, acc, m.B, m.Cres, m.Cout, m.Tp, io.len_out, nullptr);
+            pointwise_wgrad(ctx, Ls, odt, s.gv, u, g->dwp, s.wpart, acc, m.B, m.Cin, m.Cout, m.Tp, io.len_out,
+                            a.gv_scaled ? gmax : nullptr);
         }
-    }
+        if (d->residual == SC_RES_PROJ) {
+            if (half_gvr) {
+                mask_convert_f16(Ls, s.xr16, io.xres, io.len_out, m.B, m.Cres, m.Tp);
+                pointwise_wgrad(ctx, Ls, SC_F16, s.gvr16, s.xr16, g->dwr, s.wpart, acc, m.B, m.Cres, m.Cout, m.Tp, io.len_out, gmax);
+            } else {
+                const void* xr = io.xres;
+                if (!io.res_clean) { mask_copy(Ls, dt, s.xr, io.xres, io.len_out, m.B, m.Cres, m.Tp); xr = s.xr; }
+                pointwise_wgrad(ctx, Ls, dt, s.gvr, xr, g->dwr, s.wpart, acc, m.B, m.Cres, m.Cout, m.Tp, io.len_out, nullptr);
+            }
+        }
+        if (d->has_dw && !m.full) {
+            if (ctx->gemm_mode == 0 && m.plain && dw_wgrad_tc_supported(&ctx->tc, dt, m.B, m.T, m.K, m.s))
+                dw_wgrad_tc(&ctx->tc, Ls, dt, odt, s.gu, io.x, g->dwd, s.wpart, acc, gmax, io.len_in, io.len_out, m.B, m.Cin,
+                            m.T, m.K, io.x_clean ? 1 : 0);
+            else
+                dw_wgrad(Ls, dt, odt, s.gu, io.x, g->dwd, s.wpart, acc, gmax, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s, m.dil);
+        }
+    };
 
     const void* wp_op = p->wp;
     if (odt != dt && !m.full) {
@@ -417,12 +432,6 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
         }
     } else if (d->has_dw) {
         pointwise_dgrad(ctx, L, odt, wp_op, s.gv, s.gu, m.B, m.Cin, m.Cout, m.Tp, io.len_out, io.blk_off);
-        fork_to_side(ctx, L, ctx->ev[1]);               // gu is complete
-        if (ctx->gemm_mode == 0 && m.plain && dw_wgrad_tc_supported(&ctx->tc, dt, m.B, m.T, m.K, m.s))
-            dw_wgrad_tc(&ctx->tc, Ls, dt, odt, s.gu, io.x, g->dwd, s.wpart, acc, gmax, io.len_in, io.len_out, m.B, m.Cin,
-                        m.T, m.K, io.x_clean ? 1 : 0);
-        else
-            dw_wgrad(Ls, dt, odt, s.gu, io.x, g->dwd, s.wpart, acc, gmax, io.len_in, io.len_out, m.B, m.Cin, m.T, m.Tp, m.K, m.s, m.dil);
         if (io.dx) {
             if (ctx->gemm_mode == 0 && m.plain && dw_tma_supported(&ctx->tc, dt, m.B, m.T, m.K, m.s))
                 dw_tma_dgrad(&ctx->tc, L, dt, odt, s.gu, p->wd, io.dx, io.dx_add, extra, gmax, io.len_in, io.len_out, m.B,
@@ -439,6 +448,7 @@ int block_bwd_impl(sc_ctx* ctx, const Launch& L, const sc_block_desc* d, const D
             ew_add_masked(L, dt, io.dx, s.gu, io.dx_add, extra, io.len_in, m.B, m.Cin, m.T);
         }
     }
+    weight_gradients();
     // the caller joins: it waits for io.done on its stream before it reuses this scratch or returns
     if (io.done) record_side(ctx, io.done);
     return SC_OK;
@@ -497,7 +507,7 @@ int sepconv_ctx_create(sc_ctx** out, int device) {
     int r = tc_init(&c->tc, device, c->sm_count);
     if (r != SC_OK) { cudaFree(c->status_dev); delete c; return r; }
     bool ok = cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess;
-    for (int i = 0; i < 6 && ok; ++i) ok = cudaEventCreateWithFlags(&c->ev[i], cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < 8 && ok; ++i) ok = cudaEventCreateWithFlags(&c->ev[i], cudaEventDisableTiming) == cudaSuccess;
     if (!ok) { sepconv_ctx_destroy(c); return SC_ERR_CUDA; }
     *out = c;
     return SC_OK;
@@ -509,6 +519,7 @@ void sepconv_ctx_destroy(sc_ctx* ctx) {
     for (cudaEvent_t e : ctx->ev) if (e) cudaEventDestroy(e);
     if (ctx->side) cudaStreamDestroy(ctx->side);
     cudaFree(ctx->status_dev);
+    tc_destroy(&ctx->tc);
     delete ctx;
 }
 
@@ -751,12 +762,18 @@ struct LayerPlan {
     sc_block_saved sv; void* y; int* len_out; int* nvalid; int* blk_off; void* w16;
     bool own_lengths;
 };
+// Backward layer i works in scratch region i % kScratchRegions: its weight-gradient kernels (side stream) may still
+// read their operands while the next layers already write their own, and the main stream waits for them only when it
+// comes back to the region, kScratchRegions layers later.  (Three regions measured slower than two: weight gradients
+// that may lag two layers behind take SMs from the critical path more often than the wait costs.)
+constexpr int kScratchRegions = 2;
 struct EncPlan {
     std::vector<LayerPlan> L;
     void* gbuf[2]; void* pending;
+    float* gmax_all;               // one |gv| bound per layer, zeroed by one memset at the start of the call
     size_t bytes;
     size_t scratch_mark;           // offset where the shared per-layer scratch starts
-    size_t scratch_size;           // its size; a second region of the same size follows (backward layers alternate)
+    size_t scratch_size;           // its size; kScratchRegions regions of that size in all (backward layers rotate)
 };
 
 int plan_encoder(const sc_encoder_desc* e, void* base, size_t cap, EncPlan* P, const TcState* tc) {
@@ -823,13 +840,12 @@ int plan_encoder(const sc_encoder_desc* e, void* base, size_t cap, EncPlan* P, c
         Bump b(base, cap); b.off = mark; FwdScratch f; plan_fwd(&P->L[i].d, P->L[i].m, b, &f, tc); hi = std::max(hi, b.off);
         Bump c(base, cap); c.off = mark; BwdScratch s; plan_bwd(&P->L[i].d, P->L[i].m, c, &s, tc); hi = std::max(hi, c.off);
     }
-    // two scratch regions: backward layer i works in region i & 1, so that the weight-gradient kernels of layer i
-    // (side stream) may still read their operands while layer i - 1 already writes its own
     hi = (hi + 255) & ~(size_t)255;
-    ws.off = hi + (hi - mark);
+    ws.off = hi + (size_t)(kScratchRegions - 1) * (hi - mark);
     P->scratch_size = hi - mark;
     P->gbuf[0] = ws.take(max_act); P->gbuf[1] = ws.take(max_act);
     P->pending = max_res ? ws.take(max_res) : nullptr;
+    P->gmax_all = (float*)ws.take(sizeof(float) * e->n_layers);
     P->bytes = ws.off + 256;
     if (!ws.ok()) return SC_ERR_WORKSPACE;
     P->scratch_mark = mark;
@@ -938,6 +954,7 @@ int encoder_fwd_bwd(sc_ctx* ctx, const sc_encoder_desc* e, const sc_tensor* x, c
     auto len_in_of = [&](int i) -> const int* { return i == 0 ? lengths_dev : P.L[i - 1].len_out; };
     auto res_src = [&](int i) -> int { return (e->res_from && e->res_from[i] >= 0) ? e->res_from[i] : i; };
 
+    cudaMemsetAsync(P.gmax_all, 0, sizeof(float) * n, L.stream);
     // float16 copies of the pointwise weights of every layer that needs one: one launch
     {
         ConvertList cl; cl.count = 0;
@@ -970,15 +987,17 @@ int encoder_fwd_bwd(sc_ctx* ctx, const sc_encoder_desc* e, const sc_tensor* x, c
     // backward
     const void* g = dlogits->ptr;
     std::vector<char> has_pending(n, 0);
-    bool side_busy[2] = {false, false};
+    bool side_busy[kScratchRegions] = {};
+    cudaEvent_t done_ev[3] = {ctx->ev[2], ctx->ev[3], ctx->ev[6]};
     for (int i = n - 1; i >= 0; --i) {
         LayerPlan& lp = P.L[i];
-        // this layer reuses the scratch region of layer i + 2: that layer's side-stream kernels must be done
-        if (side_busy[i & 1]) wait_side(ctx, L, ctx->ev[2 + (i & 1)]);
-        Bump b(workspace, workspace_bytes); b.off = mark + (size_t)(i & 1) * P.scratch_size;
+        // this layer reuses the scratch region of layer i + kScratchRegions: that layer's side-stream kernels must be done
+        const int region = i % kScratchRegions;
+        if (side_busy[region]) wait_side(ctx, L, done_ev[region]);
+        Bump b(workspace, workspace_bytes); b.off = mark + (size_t)region * P.scratch_size;
         BwdScratch s; plan_bwd(&lp.d, lp.m, b, &s, &ctx->tc);
         BwdIO io{};
-        io.done = ctx->ev[2 + (i & 1)]; side_busy[i & 1] = true;
+        io.done = done_ev[region]; side_busy[region] = true;
         io.dy = g; io.x = input_of(i); io.y = (i + 1 < n) ? lp.y : logits->ptr;
         io.xres = lp.d.residual != SC_RES_NONE ? input_of(res_src(i)) : nullptr;
         io.dx = (i == 0) ? (dx ? dx->ptr : nullptr) : P.gbuf[i & 1];
@@ -988,10 +1007,11 @@ int encoder_fwd_bwd(sc_ctx* ctx, const sc_encoder_desc* e, const sc_tensor* x, c
         io.len_in = len_in_of(i); io.len_out = lp.len_out; io.nvalid = lp.nvalid; io.blk_off = lp.blk_off;
         io.x_clean = i > 0; io.res_clean = lp.d.residual != SC_RES_NONE && res_src(i) > 0;
         io.w16_kept = lp.w16;
+        io.gmax_zeroed = P.gmax_all + i;
         SC_TRY(block_bwd_impl(ctx, L, &lp.d, lp.m, io, &prm[i], &lp.sv, &grd[i], accumulate, s));
         g = io.dx;
     }
-    for (int q = 0; q < 2; ++q) if (side_busy[q]) wait_side(ctx, L, ctx->ev[2 + q]);     // join before returning
+    for (int q = 0; q < kScratchRegions; ++q) if (side_busy[q]) wait_side(ctx, L, done_ev[q]);     // join before returning
     return finish(ctx);
 }
 

@@ -911,9 +911,41 @@ using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, voi
 
 }  // namespace
 
+// Encoded tensor maps, kept per context: a training loop presents the same tensors every step, and encoding a map
+// costs the host a few microseconds, of which a step with several hundred launches has few to spare.  Direct-mapped
+// by a hash of everything the encoding depends on; a collision just re-encodes.
+struct TcMapCache {
+    static constexpr int kSlots = 1024;
+    struct Key {
+        const void* base; uint64_t dims[3]; uint32_t box[3]; int32_t dtype, rank, swizzle;
+        bool operator==(const Key& o) const {
+            return base == o.base && dtype == o.dtype && rank == o.rank && swizzle == o.swizzle && dims[0] == o.dims[0] &&
+                   dims[1] == o.dims[1] && dims[2] == o.dims[2] && box[0] == o.box[0] && box[1] == o.box[1] && box[2] == o.box[2];
+        }
+    };
+    struct alignas(64) Slot { CUtensorMap map; Key key; bool used; };
+    Slot slots[kSlots];
+};
+
+void tc_destroy(TcState* st) {
+    delete st->map_cache;
+    st->map_cache = nullptr;
+}
+
 bool tc_make_map(const TcState* st, void* map_out, int dtype, const void* base, int rank, const uint64_t* dims,
                  const uint32_t* box, int swizzle_bytes) {
     CUtensorMap* m = static_cast<CUtensorMap*>(map_out);
+    TcMapCache::Slot* slot = nullptr;
+    TcMapCache::Key key{};
+    if (st->map_cache) {
+        key.base = base; key.dtype = dtype; key.rank = rank; key.swizzle = swizzle_bytes;
+        for (int i = 0; i < rank; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; }
+        uint64_t h = reinterpret_cast<uintptr_t>(base) * 0x9E3779B97F4A7C15ull;
+        for (int i = 0; i < 3; ++i) h = (h ^ key.dims[i] ^ ((uint64_t)key.box[i] << 40)) * 0xC2B2AE3D27D4EB4Full;
+        h ^= (uint64_t)(dtype * 131 + rank * 17 + swizzle_bytes);
+        slot = &st->map_cache->slots[(h >> 32) % TcMapCache::kSlots];
+        if (slot->used && slot->key == key) { *m = slot->map; return true; }
+    }
     cuuint64_t gdim[3]; cuuint64_t gstride[2]; cuuint32_t bdim[3]; cuuint32_t estr[3] = {1, 1, 1};
     uint64_t stride = 2;
     for (int i = 0; i < rank; ++i) {
@@ -927,6 +959,7 @@ bool tc_make_map(const TcState* st, void* map_out, int dtype, const void* base, 
         swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { fprintf(stderr, "sepconv: cuTensorMapEncodeTiled failed (%d)\n", (int)r); return false; }
+    if (slot) { slot->map = *m; slot->key = key; slot->used = true; }
     return true;
 }
 
@@ -1013,6 +1046,7 @@ int tc_init(TcState* st, int device, int sm_count) {
     st->encode_fn = (e == cudaSuccess && q == cudaDriverEntryPointSuccess) ? fn : nullptr;
     st->ready = st->encode_fn != nullptr;
     st->persistent = true;
+    if (st->ready && !st->map_cache) st->map_cache = new TcMapCache();      // value-initialised: every slot unused
     if (!st->ready) { fprintf(stderr, "sepconv: cuTensorMapEncodeTiled not available\n"); return -11; }
     return 0;
 }

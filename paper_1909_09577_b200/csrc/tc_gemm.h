@@ -6,8 +6,10 @@
 
 namespace sc {
 
+struct TcMapCache;
 struct TcState {
     void* encode_fn = nullptr;   // cuTensorMapEncodeTiled, resolved through the runtime
+    TcMapCache* map_cache = nullptr;   // encoded tensor maps of this context (tc_make_map); calls on one context are not concurrent
     int sm_count = 0;
     bool ready = false;
     bool persistent = true;      // forward / input gradient: persistent warp-specialised kernel
@@ -17,6 +19,7 @@ struct TcState {
 };
 
 int tc_init(TcState* st, int device, int sm_count);
+void tc_destroy(TcState* st);
 
 // Encodes a tiled tensor map (128-byte swizzle by default, 64-byte with swizzle_bytes = 64; zero fill outside the
 // tensor) for a dense 16-bit tensor whose dimensions, innermost first, are dims[0..rank-1]; map_out points to a
