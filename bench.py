@@ -351,8 +351,7 @@ def main():
     clocks = sampler.stop(t0, t1) if sampler else None
     other_ms = None
     if args.no_graph and not dp_exchange:
-        # for context: the same K steps replayed as one captured CUDA graph (no per-launch host cost, but stream
-        # capture turns the programmatic launch dependencies into full ones)
+        # for context: the same K steps replayed as one captured CUDA graph (no per-launch host cost)
         try:
             graph = torch.cuda.CUDAGraph()
             cap_stream = torch.cuda.Stream()
