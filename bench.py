@@ -6,7 +6,10 @@ Default workload: the bf16 QuartzNet-5x5-style encoder, B=32, T=1600 input frame
 (config 4); `--config 5` runs the ragged B=64, T=3200 encoder.  Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config 4|5] [--impl reference]
-                  [--no-cpu-baseline] [--no-e2e] [--no-graph] [--block C_in,C_out,K,B,T]
+                  [--no-cpu-baseline] [--no-e2e] [--host-launches] [--block C_in,C_out,K,B,T]
+
+The timed steps replay one captured CUDA graph of the step (`--host-launches`: every kernel launched from the host
+instead; the line reports the other mode's time beside the timed one).
 
 Besides the step throughput the line carries `roofline_per_class`: for every kernel class of the step
 its CUDA-event time, launches, algorithmic bytes and flops (every tensor the class must read or write
