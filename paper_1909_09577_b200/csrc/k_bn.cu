@@ -842,12 +842,12 @@ __global__ void __launch_bounds__(256) bn_bwd_reduce_fast_kernel(BnBwdArgs a, in
 // (The same mapping was measured for the two apply kernels and lost to the flattened one: a CTA that hops between
 // the 32 rows of a channel streams about 10 % slower than one that walks the tensor in address order, and a forward
 // apply that merges the contraction's statistics partials in its prologue pays that merge once per CTA.)
-constexpr int kChThreads = 256;
+constexpr int kChThreads = 512;
 
 // Backward reduction of channel o over every sample, then the channel's coefficients, parameter gradients and its
 // term of the bound on |gv| (what bn_bwd_finalize_kernel does for the row-mapped reduction).
 template <typename T, typename NT, int RES>
-__global__ void __launch_bounds__(kChThreads, 4)
+__global__ void __launch_bounds__(kChThreads, 2)
 bn_bwd_reduce_ch_kernel(BnBwdArgs a, int vpr, const float* gamma_r, float* dgamma, float* dbeta, float* dgamma_r,
                         float* dbeta_r, int accumulate) {
     pdl_sync();
@@ -1008,7 +1008,7 @@ static unsigned fast_grid(long long total, int V) { return (unsigned)((total + 2
 // Algorithmic bytes per element of the batch-norm kernels: every tensor they must read or write, once.
 // The channel-per-CTA reduction pays off once a channel holds a few vectors per thread; below that (or with few
 // channels) the row-mapped kernel and its separate finalize step are used.
-static bool channel_mapped(int B, int C, int Tp) { return C >= 32 && (long long)B * (Tp / 8) >= 4 * kChThreads; }
+static bool channel_mapped(int B, int C, int Tp) { return C >= 32 && (long long)B * (Tp / 8) >= 1024; }
 
 void bn_apply(const Launch& L, int dtype, const ApplyArgs& a_in) {
     ApplyArgs a = a_in;
