@@ -229,7 +229,7 @@ def main():
     ap.add_argument("--breakdown", default=None, help="also write the per-kernel-class table to this text file")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--gemm-mode", type=int, default=0)
-    ap.add_argument("--tile-shape", type=int, default=None, help="tile shape of the pointwise contractions (0..4, see sepconv_set_tile_shape)")
+    ap.add_argument("--tile-shape", type=int, default=None, help="tile shape of the pointwise contractions (0..5, see sepconv_set_tile_shape)")
     ap.add_argument("--dp", action="store_true",
                     help="with N > 1 ranks: data-parallel step -- every rank its own batch, per-replica batch statistics, "
                          "and an NCCL all-reduce of the gradient blob inside the step (default: independent replicas)")

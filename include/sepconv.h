@@ -309,7 +309,8 @@ int  sepconv_set_gemm_mode(sc_ctx* ctx, int mode);
  * 0 = 256 output channels x 256 frames per tile with one accumulator in tensor memory, drained by sixteen epilogue
  * warps when the batch has at most 256 samples (else as 4); 1 = 256 x 128 and 2 = 128 x 256 with two accumulators,
  * so that a tile's epilogue overlaps the next tile's MMAs; 3 = 128 x 256, one accumulator, two CTAs per SM;
- * 4 = as 0 with eight epilogue warps.  Other values: SC_ERR_UNSUPPORTED.  Results do not depend on the shape except
+ * 4 = as 0 with eight epilogue warps; 5 = as 2 with sixteen epilogue warps (four per 32 accumulator rows; batches of
+ * more than 256 samples take 2).  Other values: SC_ERR_UNSUPPORTED.  Results do not depend on the shape except
  * for the summation order of the batch-norm statistics. */
 int  sepconv_set_tile_shape(sc_ctx* ctx, int shape);
 

@@ -561,7 +561,7 @@ int sepconv_selftest_bounded_wait(sc_ctx* ctx, void* cuda_stream) {
 
 int sepconv_set_tile_shape(sc_ctx* ctx, int shape) {
     if (!ctx) return SC_ERR_NULL;
-    if (shape < 0 || shape > 4) return SC_ERR_UNSUPPORTED;
+    if (shape < 0 || shape > 5) return SC_ERR_UNSUPPORTED;
     ctx->tc.flat_shape = shape;
     return SC_OK;
 }

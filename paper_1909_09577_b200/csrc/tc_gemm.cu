@@ -607,8 +607,8 @@ template <int MT, int NB, int OCC, int EPI = 1> struct FlatCfg {
     static constexpr int STAGE = A_BYTES + NB * 8192;
     static constexpr int STAGES = OCC == 2 ? 2 : (STAGE <= 49152 ? 4 : 3);
     // per-warp staging: 32 x 32 16-bit values, or (one M sub-tile, one CTA per SM only) 32 x 32 floats for a float32 result
-    static constexpr int STG = EPI == 2 ? 2048 : ((MT == 1 && OCC == 1) ? kStgFloatsPerWarp * 4 : kOutStageBytes);
-    static constexpr int MAXB = (OCC == 2 || EPI == 2) ? 256 : kFlatMaxB;
+    static constexpr int STG = EPI >= 2 ? 2048 : ((MT == 1 && OCC == 1) ? kStgFloatsPerWarp * 4 : kOutStageBytes);
+    static constexpr int MAXB = (OCC == 2 || EPI >= 2) ? 256 : kFlatMaxB;
     static constexpr int smem_bytes(int B) { return STAGES * STAGE + 256 + 4 * MT * EPI * STG + (B + 1) * 4 + 1024; }
 };
 
@@ -624,7 +624,7 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
     constexpr uint32_t ACC_COLS = MT * NB * 64;
     constexpr uint32_t TMEM_COLS = ACC_COLS * NBUF;
     static_assert(TMEM_COLS == 128 || TMEM_COLS == 256 || TMEM_COLS == 512, "tensor-memory columns");
-    static_assert(EPI == 1 || (EPI == 2 && OCC == 1), "epilogue warps per lane quarter");
+    static_assert(EPI == 1 || ((EPI == 2 || EPI == 4) && OCC == 1), "epilogue warps per lane quarter");
     constexpr int EW = 4 * MT * EPI;               // epilogue warps; then the producer warp and the MMA warp
 
     extern __shared__ uint8_t smem_raw[];
@@ -732,7 +732,8 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
         __syncwarp();
     } else {                                          // ---- epilogue warps ----
         const int mt = (warp >> 2) % MT, wq = warp & 3;
-        const int hsel = (warp >> 2) / MT;            // EPI == 2: the 32-column half of every block this warp takes
+        const int hsel = (warp >> 2) / MT;            // EPI > 1: which of a tile's 32-column chunks this warp takes: chunk
+                                                      // 2 * block + half belongs to the warp with hsel == chunk % EPI
         uint8_t* stg = stg_all + warp * p.stg_stride;
         uint32_t nstore = 0;                          // TMA stores issued by this warp
         if (p.zero_fill) {
@@ -769,28 +770,32 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
         auto flush_stats = [&]() {
             if (MODE != MODE_FWD || !p.stats || cur_m < 0) return;
             float n = sn, sum = fmaf(pivot, sn, sd), m2 = sn > 0.f ? sq - sd * sd / sn : 0.f;
-            if (EPI == 2) {
-                // the two warps of a row hold the statistics of its two column halves: the second hands its triple
-                // over through its staging buffer (its stores have read it by then), the first merges (Chan) and writes
+            if (EPI > 1) {
+                // the EPI warps of a row hold the statistics of its column chunks: the others hand their triples
+                // over through their staging buffers (their stores have read them by then), the first merges them
+                // in warp order (Chan) and writes
                 const uint32_t bar_id = 1 + mt * 4 + wq;
-                if (hsel == 1) {
+                if (hsel > 0) {
                     if (p.tma_out && lane == 0) ptx::bulk_wait_read();
                     __syncwarp();
                     reinterpret_cast<float4*>(stg)[lane] = make_float4(n, sum, m2, 0.f);
                 }
-                asm volatile("bar.sync %0, 64;" ::"r"(bar_id) : "memory");
+                asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(32 * EPI) : "memory");
                 if (hsel == 0) {
-                    const float4 o = reinterpret_cast<const float4*>(stg + 4 * MT * p.stg_stride)[lane];
-                    if (o.x > 0.f) {
-                        if (n > 0.f) {
-                            const float nt = n + o.x, dlt = o.y / o.x - sum / n;
-                            m2 += o.z + dlt * dlt * (n * o.x / nt);
-                            sum += o.y; n = nt;
-                        } else { n = o.x; sum = o.y; m2 = o.z; }
+#pragma unroll
+                    for (int e = 1; e < EPI; ++e) {
+                        const float4 o = reinterpret_cast<const float4*>(stg + e * 4 * MT * p.stg_stride)[lane];
+                        if (o.x > 0.f) {
+                            if (n > 0.f) {
+                                const float nt = n + o.x, dlt = o.y / o.x - sum / n;
+                                m2 += o.z + dlt * dlt * (n * o.x / nt);
+                                sum += o.y; n = nt;
+                            } else { n = o.x; sum = o.y; m2 = o.z; }
+                        }
                     }
                 }
-                asm volatile("bar.sync %0, 64;" ::"r"(bar_id) : "memory");
-                if (hsel == 1) return;
+                asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(32 * EPI) : "memory");
+                if (hsel > 0) return;
             }
             const int row = cur_m * (128 * MT) + mt * 128 + wq * 32 + lane;
             if (row < p.M) p.stats[(size_t)blockIdx.x * p.M + row] = make_float4(n, sum, m2, 0.f);
@@ -810,7 +815,8 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                 const int t0 = (j + i - s_off[b]) * 64;
                 const int len = min(p.len_out[b], p.Tp);
 #pragma unroll 1
-                for (int h = (EPI == 2 ? hsel : 0); h < (EPI == 2 ? hsel + 1 : 2); ++h) {
+                for (int h = 0; h < 2; ++h) {
+                    if (EPI > 1 && ((2 * i + h) % EPI) != hsel) continue;
                     const int c0 = t0 + 32 * h;
                     if (c0 >= p.Tp) break;
                     float f[32];
@@ -1091,6 +1097,8 @@ template <typename T, int MODE>
 void launch_flat_shape(int shape, int mt, const Launch& L, int sm_count, const CUtensorMap& a, const CUtensorMap& b,
                        const CUtensorMap& o, const FlatParams& p, int* grid_out) {
     if (shape == 3 && !p.out_f32 && p.B <= FlatCfg<1, 4, 2>::MAXB) { launch_flat<T, MODE, 1, 4, 1, 2>(L, sm_count, a, b, o, p, grid_out); return; }
+    // 5: 128 x 256 tiles, two accumulators, sixteen epilogue warps (four per 32 accumulator rows)
+    if (shape == 5 && mt == 1 && p.tma_out && p.B <= FlatCfg<1, 4, 1, 4>::MAXB) { launch_flat<T, MODE, 1, 4, 2, 1, 4>(L, sm_count, a, b, o, p, grid_out); return; }
     if (mt == 1) { launch_flat<T, MODE, 1, 4, 2>(L, sm_count, a, b, o, p, grid_out); return; }
     // sixteen epilogue warps need TMA stores (their 2 KiB staging buffers have the store's layout) and a batch
     // whose block offsets fit beside those buffers
@@ -1105,7 +1113,7 @@ void launch_flat_dt(int dtype, int shape, int mt, const Launch& L, int sm_count,
     else launch_flat_shape<__nv_bfloat16, MODE>(shape, mt, L, sm_count, a, b, o, p, grid_out);
 }
 // M sub-tiles per CTA for a given tile shape and row count
-inline int flat_mt(int shape, int rows) { return (shape == 2 || shape == 3 || rows <= 128) ? 1 : 2; }
+inline int flat_mt(int shape, int rows) { return (shape == 2 || shape == 3 || shape == 5 || rows <= 128) ? 1 : 2; }
 }  // namespace
 
 size_t tc_stats_bytes(int B, int Cout, int Tp) {

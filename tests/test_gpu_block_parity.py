@@ -111,7 +111,7 @@ def test_tensorcore_shapes(api, ctx, dtype, case):
     rep.check()
 
 
-@pytest.mark.parametrize("shape", [0, 1, 2, 3, 4])
+@pytest.mark.parametrize("shape", [0, 1, 2, 3, 4, 5])
 @pytest.mark.parametrize("case", [2, 4])
 def test_tile_shapes(api, ctx, shape, case):
     """Every tile shape of the flattened-block contraction (forward with statistics, input gradient): a projection
