@@ -586,10 +586,11 @@ __device__ __forceinline__ int flat_find_sample(const int* off, int B, int j) {
 
 // next tile of a CTA's unit range: M tile m, first block j, nb blocks
 template <int NB>
-__device__ __forceinline__ bool flat_next_tile(long long& pos, long long end, int nblk, int& m, int& j, int& nb) {
+__device__ __forceinline__ bool flat_next_tile(uint32_t& pos, uint32_t end, uint32_t nblk, int& m, int& j, int& nb) {
     if (pos >= end) return false;
-    m = (int)(pos / nblk); j = (int)(pos - (long long)m * nblk);
-    nb = (int)min((long long)NB, min(end - pos, (long long)(nblk - j)));
+    const uint32_t mm = pos / nblk, jj = pos - mm * nblk;
+    m = (int)mm; j = (int)jj;
+    nb = (int)min((uint32_t)NB, min(end - pos, nblk - jj));
     pos += nb;
     return true;
 }
@@ -655,14 +656,18 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
     const uint32_t tmem = *tmem_slot;
     const int nkb = (p.Kdim + BK - 1) / BK;
     const int nblk = s_off[p.B];
-    const long long U = (long long)p.tiles_m * nblk;
-    const long long u_begin = U * blockIdx.x / gridDim.x, u_end = U * (blockIdx.x + 1) / gridDim.x;
+    // 32-bit arithmetic throughout (the launcher bounds the unit count): 64-bit divisions in front of the first copy
+    // cost every CTA about a microsecond.  floor(U * c / G) = (U / G) * c + ((U % G) * c) / G, every product below 2^32
+    const uint32_t U = (uint32_t)p.tiles_m * (uint32_t)nblk;
+    const uint32_t Uq = U / gridDim.x, Ur = U - Uq * gridDim.x;
+    const uint32_t u_begin = Uq * blockIdx.x + (Ur * blockIdx.x) / gridDim.x;
+    const uint32_t u_end = Uq * (blockIdx.x + 1) + (Ur * (blockIdx.x + 1)) / gridDim.x;
 
     if (warp == EW) {
         if (lane == 0) {                              // ---- TMA producer ----
             int it = 0, m, j, nb;
             bool dead = false;
-            long long pos = u_begin;
+            uint32_t pos = u_begin;
             while (!dead && flat_next_tile<NB>(pos, u_end, nblk, m, j, nb)) {
                 int bb[NB], tt[NB];
                 int b = flat_find_sample(s_off, p.B, j);
@@ -702,7 +707,7 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
         if (lane == 0) {                              // ---- MMA issuer ----
             int it = 0, jt = 0, m, j, nb;
             bool dead = false;
-            long long pos = u_begin;
+            uint32_t pos = u_begin;
             while (!dead && flat_next_tile<NB>(pos, u_end, nblk, m, j, nb)) {
                 const int buf = jt % NBUF;
                 if (!ptx::mbar_wait(&acc_empty[buf], ((jt / NBUF) & 1) ^ 1)) { raise_status(p.status, kErrTimeout); break; }
@@ -739,9 +744,9 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
         if (p.zero_fill) {
             // blocks wholly in padding: sample b's blocks [off[b+1]-off[b], nbT); CTAs share them round-robin
             const int inv_per_m = p.B * p.nbT - nblk;
-            const long long total_inv = (long long)p.tiles_m * inv_per_m;
-            for (long long q = blockIdx.x; q < total_inv; q += gridDim.x) {
-                const int m = (int)(q / inv_per_m), jj = (int)(q - (long long)m * inv_per_m);
+            const uint32_t total_inv = (uint32_t)p.tiles_m * (uint32_t)inv_per_m;
+            for (uint32_t q = blockIdx.x; q < total_inv; q += gridDim.x) {
+                const int m = (int)(q / (uint32_t)inv_per_m), jj = (int)(q - (uint32_t)m * (uint32_t)inv_per_m);
                 int lo = 0, hi = p.B - 1;              // largest b with b * nbT - off[b] <= jj
                 while (lo < hi) {
                     const int mid = (lo + hi + 1) >> 1;
@@ -764,7 +769,7 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             }
         }
         int jt = 0, m, j, nb, cur_m = -1;
-        long long pos = u_begin;
+        uint32_t pos = u_begin;
         float sn = 0.f, sd = 0.f, sq = 0.f, pivot = 0.f;     // statistics of this thread's channel over the CTA's range of one M tile
         bool dead = false;            // a wait ran out: no further accumulator is touched, but every pair barrier below is still met
         auto flush_stats = [&]() {
@@ -1112,6 +1117,8 @@ void launch_flat_dt(int dtype, int shape, int mt, const Launch& L, int sm_count,
     if (dtype == F16) launch_flat_shape<__half, MODE>(shape, mt, L, sm_count, a, b, o, p, grid_out);
     else launch_flat_shape<__nv_bfloat16, MODE>(shape, mt, L, sm_count, a, b, o, p, grid_out);
 }
+// the flattened-block kernel counts its work units (M tiles x 64-frame blocks) in 32 bits
+inline bool flat_units_fit(int B, int Tp, int rows) { return (long long)((rows + 127) / 128) * B * ((Tp + 63) / 64) < (1ll << 31); }
 // M sub-tiles per CTA for a given tile shape and row count
 inline int flat_mt(int shape, int rows) { return (shape == 2 || shape == 3 || shape == 5 || rows <= 128) ? 1 : 2; }
 }  // namespace
@@ -1133,7 +1140,7 @@ void tc_gemm_fwd(const TcState* st, const Launch& L, int dtype, const void* w, c
     if (layout) *layout = StatsLayout{};
     if (!make_map(st, &ma, dtype, w, 2, da, ba) || !make_map(st, &mb, dtype, u, 3, db, bb)) return;
     int mt = Cout > 128 ? 2 : 1;
-    if (st->flat && blk_off && B <= kFlatMaxB && (out_dtype != F32 || Cout <= 128)) {
+    if (st->flat && blk_off && B <= kFlatMaxB && flat_units_fit(B, Tp, Cout) && (out_dtype != F32 || Cout <= 128)) {
         mt = flat_mt(st->flat_shape, Cout);
         FlatParams p{};
         p.out = v; p.bias = bias; p.len_out = len_out; p.blk_off = blk_off; p.stats = (float4*)partials; p.status = L.status;
@@ -1170,7 +1177,7 @@ void tc_gemm_dgrad(const TcState* st, const Launch& L, int dtype, const void* w,
     const uint32_t bb[3] = {64, 64, 1};
     if (!make_map(st, &ma, dtype, w, 2, da, ba) || !make_map(st, &mb, dtype, gv, 3, db, bb)) return;
     int mt = Cin > 128 ? 2 : 1;
-    if (st->flat && blk_off && B <= kFlatMaxB) {
+    if (st->flat && blk_off && B <= kFlatMaxB && flat_units_fit(B, Tp, Cin)) {
         mt = flat_mt(st->flat_shape, Cin);
         FlatParams p{};
         p.out = gu; p.len_out = len_out; p.blk_off = blk_off; p.status = L.status;
