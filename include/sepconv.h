@@ -266,10 +266,14 @@ int  sepconv_fwd_static(sc_ctx* ctx, const sc_block_desc* desc,
 
 /* ---- whole encoder -------------------------------------------------------------------------- */
 
-/* Bytes of workspace encoder_fwd_bwd needs for this layer list (host-only computation).  Returns
- * SC_ERR_UNSUPPORTED when the block-level residual spans [res_from[i], i] overlap or share a source:
- * the encoder keeps one pending residual gradient at a time, which is all the Jasper-style encoders
- * of section 4.1.1 need (each block's residual comes from that block's input only). */
+/* Bytes of workspace encoder_fwd_bwd needs for this layer list (host-only computation).  A layer's residual
+ * may come from the input of any earlier layer (res_from[i] <= i; a later one: SC_ERR_UNSUPPORTED); the spans
+ * [res_from[i], i] may nest or overlap and several layers may name the same source.  The residual path's gradient
+ * for a source waits in a pending buffer until the backward pass reaches that source; spans that do not overlap
+ * share one buffer (the Jasper-style encoders of section 4.1.1, where each block's residual comes from that block's
+ * input, need a single one), each overlapping span adds a buffer of the source's size to the workspace.  One
+ * residual source per layer: the sum of several projected sources at one layer (the dense-residual variant of the
+ * Jasper family) is not expressible. */
 int  encoder_workspace_bytes(const sc_encoder_desc* desc, size_t* bytes);
 
 /* The whole encoder module of section 4.1.1 plus the 1x1 decoder convolution that ends in the logits

@@ -769,7 +769,9 @@ struct LayerPlan {
 constexpr int kScratchRegions = 2;
 struct EncPlan {
     std::vector<LayerPlan> L;
-    void* gbuf[2]; void* pending;
+    void* gbuf[2];
+    std::vector<void*> pend;       // per layer: where the residual gradients for that layer's input collect (or null)
+    void* pend_tmp;                // a second residual gradient for a source that already holds one lands here first
     float* gmax_all;               // one |gv| bound per layer, zeroed by one memset at the start of the call
     size_t bytes;
     size_t scratch_mark;           // offset where the shared per-layer scratch starts
@@ -782,14 +784,17 @@ int plan_encoder(const sc_encoder_desc* e, void* base, size_t cap, EncPlan* P, c
     P->L.resize(e->n_layers);
     int B = e->layers[0].B, T = e->layers[0].T_in, C = e->layers[0].C_in;
     size_t max_act = 0, max_res = 0;
-    // One pending residual-gradient buffer serves the whole backward pass, so the spans [source, layer]
-    // of the block-level residuals must not overlap (which also rules out two layers sharing a source).
-    int span_end = -1;
-    for (int i = 0; i < e->n_layers; ++i) {
+    // Residual spans [source, layer]: the residual path's gradient waits in a pending buffer from the backward step of
+    // `layer` down to that of `source`.  Spans that do not overlap share a buffer (the five blocks of the QuartzNet
+    // encoder use one); spans that overlap or nest get buffers of their own; several layers may share a source (their
+    // gradients are summed in the source's buffer).
+    const int nl = e->n_layers;
+    std::vector<int> last_user(nl, -1), users(nl, 0);
+    std::vector<size_t> res_bytes(nl, 0);
+    for (int i = 0; i < nl; ++i) {
         if (e->layers[i].residual == SC_RES_NONE || !e->res_from || e->res_from[i] < 0 || e->res_from[i] == i) continue;
         if (e->res_from[i] > i) return SC_ERR_UNSUPPORTED;
-        if (e->res_from[i] <= span_end) return SC_ERR_UNSUPPORTED;
-        span_end = i;
+        last_user[e->res_from[i]] = i; ++users[e->res_from[i]];
     }
     for (int i = 0; i < e->n_layers; ++i) {
         LayerPlan& lp = P->L[i];
@@ -810,6 +815,7 @@ int plan_encoder(const sc_encoder_desc* e, void* base, size_t cap, EncPlan* P, c
             int j = (e->res_from && e->res_from[i] >= 0) ? e->res_from[i] : i;
             if (P->L[j].m.T != m.Tp) return SC_ERR_UNSUPPORTED;
             max_res = std::max(max_res, es * m.B * m.Cres * m.Tp);
+            if (j != i) res_bytes[j] = es * m.B * m.Cres * m.Tp;
         }
         lp.own_lengths = (i == 0) || (m.s != 1);
         if (lp.own_lengths) {
@@ -844,7 +850,27 @@ int plan_encoder(const sc_encoder_desc* e, void* base, size_t cap, EncPlan* P, c
     ws.off = hi + (size_t)(kScratchRegions - 1) * (hi - mark);
     P->scratch_size = hi - mark;
     P->gbuf[0] = ws.take(max_act); P->gbuf[1] = ws.take(max_act);
-    P->pending = max_res ? ws.take(max_res) : nullptr;
+    {
+        // interval colouring in source order: a buffer whose span ended strictly before this source is free again
+        struct Buf { int end; size_t bytes; };
+        std::vector<Buf> bufs;
+        std::vector<int> colour(nl, -1);
+        bool need_tmp = false;
+        for (int j = 0; j < nl; ++j) {
+            if (last_user[j] < 0) continue;
+            if (users[j] > 1) need_tmp = true;
+            int c = -1;
+            for (size_t q = 0; q < bufs.size(); ++q) if (bufs[q].end < j) { c = (int)q; break; }
+            if (c < 0) { bufs.push_back(Buf{0, 0}); c = (int)bufs.size() - 1; }
+            bufs[c].end = last_user[j]; bufs[c].bytes = std::max(bufs[c].bytes, res_bytes[j]);
+            colour[j] = c;
+        }
+        std::vector<void*> addr(bufs.size(), nullptr);
+        for (size_t q = 0; q < bufs.size(); ++q) addr[q] = ws.take(bufs[q].bytes);
+        P->pend.assign(nl, nullptr);
+        for (int j = 0; j < nl; ++j) if (colour[j] >= 0) P->pend[j] = addr[colour[j]];
+        P->pend_tmp = need_tmp ? ws.take(max_res) : nullptr;
+    }
     P->gmax_all = (float*)ws.take(sizeof(float) * e->n_layers);
     P->bytes = ws.off + 256;
     if (!ws.ok()) return SC_ERR_WORKSPACE;
@@ -1002,13 +1028,18 @@ int encoder_fwd_bwd(sc_ctx* ctx, const sc_encoder_desc* e, const sc_tensor* x, c
         io.xres = lp.d.residual != SC_RES_NONE ? input_of(res_src(i)) : nullptr;
         io.dx = (i == 0) ? (dx ? dx->ptr : nullptr) : P.gbuf[i & 1];
         io.dx_res = nullptr;
-        if (lp.d.residual != SC_RES_NONE && res_src(i) != i) { io.dx_res = P.pending; has_pending[res_src(i)] = 1; }
-        io.dx_add = has_pending[i] ? P.pending : nullptr;
+        const int src = res_src(i);
+        const bool to_pending = lp.d.residual != SC_RES_NONE && src != i;
+        const bool second = to_pending && has_pending[src];       // the source's buffer already holds a gradient
+        if (to_pending) { io.dx_res = second ? P.pend_tmp : P.pend[src]; has_pending[src] = 1; }
+        io.dx_add = has_pending[i] ? P.pend[i] : nullptr;
         io.len_in = len_in_of(i); io.len_out = lp.len_out; io.nvalid = lp.nvalid; io.blk_off = lp.blk_off;
         io.x_clean = i > 0; io.res_clean = lp.d.residual != SC_RES_NONE && res_src(i) > 0;
         io.w16_kept = lp.w16;
         io.gmax_zeroed = P.gmax_all + i;
         SC_TRY(block_bwd_impl(ctx, L, &lp.d, lp.m, io, &prm[i], &lp.sv, &grd[i], accumulate, s));
+        if (second)
+            ew_add_masked(L, dt, P.pend[src], P.pend[src], P.pend_tmp, nullptr, len_in_of(src), P.L[src].m.B, P.L[src].m.Cin, P.L[src].m.T);
         g = io.dx;
     }
     for (int q = 0; q < kScratchRegions; ++q) if (side_busy[q]) wait_side(ctx, L, done_ev[q]);     // join before returning

@@ -312,8 +312,8 @@ def run_chain(ctx, api, w, d, check=True, oracle_layers=None, pool=None):
         dx_add = pending.pop(i, None)
         dx, dx_res, grads = api.sepconv_bwd(ctx, f["desc"], g, f["xd"], f["y"], f["ld"], f["pd"], f["saved"],
                                             x_res=f["xr"], dx_add=dx_add, want_dx_res=want_res)
-        if want_res:
-            pending[f["j"]] = dx_res
+        if want_res:          # several layers may feed one source: their residual gradients are summed as stored tensors
+            pending[f["j"]] = dx_res if f["j"] not in pending else pending[f["j"]] + dx_res
         grads_all[i] = grads
         if oracle_layers is None or i in oracle_layers:
             tasks[i] = dict(index=i, L=L, dtype=w.dtype, x=_cpu(f["xd"]), lengths=lens[i], params=d.params[i],

@@ -135,6 +135,36 @@ def test_encoder_with_non_separable_prologue(api, ctx):
     assert_encoder_equals_chain(w, d, spec, logits, out_len, gblob, dx, chain)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_encoder_with_overlapping_residual_spans(api, ctx, dtype):
+    """Residuals beyond the one-per-block pattern: a span nested inside another, two layers that share a source
+    (their residual gradients are summed in the source's pending buffer) and an identity residual taken from another
+    layer's input.  Every layer against the oracle teacher-forced, the one-call encoder bit-equal to the chain of block
+    calls, and the whole thing end to end against the oracle on its own activations."""
+    w_ = 32
+    layers = [si.LayerCfg(16, w_, K=5, stride=2),
+              si.LayerCfg(w_, w_, K=7),
+              si.LayerCfg(w_, w_, K=7),
+              si.LayerCfg(w_, w_, K=7, residual="proj", res_from=2, C_res_override=w_),            # span [2, 3]
+              si.LayerCfg(w_, 2 * w_, K=9),
+              si.LayerCfg(2 * w_, 2 * w_, K=9, residual="proj", res_from=1, C_res_override=w_),    # span [1, 5] around it
+              si.LayerCfg(2 * w_, 2 * w_, K=9, residual="proj", res_from=1, C_res_override=w_),    # the same source again
+              si.LayerCfg(2 * w_, 2 * w_, K=11, residual="identity", res_from=6),                  # span [6, 7]
+              si.LayerCfg(2 * w_, 4 * w_, K=1, has_dw=False),
+              si.LayerCfg(4 * w_, 29, K=1, has_dw=False, has_bn=False, has_relu=False, has_bias=True)]
+    w = si.Workload("tiny_encoder_overlapping_residuals", dtype, 8, 512, layers, 23, len_lo=128, len_hi=512, affine="random")
+    d = si.draw(w)
+    reports, chain = U.run_chain(ctx, api, w, d)
+    spec, logits, out_len, gblob, dx = run_encoder(ctx, api, w, d)
+    assert_encoder_equals_chain(w, d, spec, logits, out_len, gblob, dx, chain)
+    rep, adopted, hard = end_to_end(w, d, spec, logits, gblob, dx, chain)
+    print(f"\noverlapping residual spans {dtype}: teacher-forced worst {max((r.worst() for r in reports), key=lambda t: t[1])}, "
+          f"end-to-end logits {rep.rows[0][1]:.3f} worst {rep.worst()} adopted gates {adopted} hard mismatches {hard}")
+    assert rep.rows[0][1] <= E2E_LOGITS_LIMIT, rep.rows[0]
+    if hard == 0:
+        assert rep.worst()[1] <= E2E_GRAD_LIMIT, rep.worst()
+
+
 def test_encoder_without_dx_and_accumulate(api, ctx):
     w = si.tiny_encoder(dtype="bf16", B=2, T=64, ragged=True, width=32)
     d = si.draw(w)
