@@ -636,6 +636,24 @@ def test_running_stats():
     np.testing.assert_allclose(rv, [0.9 + 0.1 * 4 * 10 / 9, 0.9 + 0.1 * 9 * 10 / 9])
 
 
+def test_running_stats_match_torch_batch_norm():
+    """The running-statistics reading (momentum 0.1, unbiased variance into the running buffer) against torch's own
+    update: batch_norm in training mode on the valid frames of a ragged batch packed into one [1, C, N] tensor
+    (masked statistics reduce to plain statistics there), starting from non-trivial running buffers."""
+    rng = np.random.default_rng(77)
+    B, C, T = 3, 5, 11
+    lengths = np.array([11, 4, 7])
+    v = rng.normal(size=(B, C, T)) * rng.uniform(0.5, 2.0, size=(1, C, 1)) + rng.normal(size=(1, C, 1))
+    mean, var, N = O.bn_stats(v, O.time_mask(lengths, T))
+    rm0, rv0 = rng.normal(size=C), rng.uniform(0.5, 1.5, size=C)
+    rm, rv = O.running_stats_update(rm0, rv0, mean, var, N)
+    packed = torch.from_numpy(np.concatenate([v[b, :, :lengths[b]] for b in range(B)], axis=1)[None])
+    trm, trv = torch.from_numpy(rm0.copy()), torch.from_numpy(rv0.copy())
+    F.batch_norm(packed, trm, trv, training=True, momentum=0.1, eps=1e-3)
+    np.testing.assert_allclose(rm, trm.numpy(), rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(rv, trv.numpy(), rtol=1e-12, atol=1e-12)
+
+
 def test_inputs_are_seeded_and_representable():
     a, b = si.draw(si.config(2)), si.draw(si.config(2))
     np.testing.assert_array_equal(a.x, b.x)
