@@ -128,6 +128,31 @@ def test_tile_shapes(api, ctx, shape, case):
     rep.check()
 
 
+@pytest.mark.parametrize("shape", [0, 1, 2, 3, 5])
+def test_tile_shapes_large_batch(api, ctx, shape):
+    """More than 256 samples: the block offsets no longer fit beside the sixteen epilogue warps' staging buffers (nor
+    beside two CTAs per SM), so shapes 0, 3 and 5 take their eight-warp / one-CTA forms."""
+    L = si.LayerCfg(C_in=136, C_out=144, K=9, residual="proj")
+    d = _draw_block(L, 272, 72, "bf16", seed=411, ragged=True, lo_frac=0.1)
+    ctx.set_tile_shape(shape)
+    try:
+        rep = U.run_block(ctx, api, L, "bf16", d.x, d.lengths, d.params[0], d.g)
+    finally:
+        ctx.set_tile_shape(0)
+    print(f"\nlarge batch, tile shape {shape}: {rep}")
+    rep.check()
+
+
+def test_batch_beyond_the_flattened_block_list(api, ctx):
+    """More than 2048 samples: the contraction leaves the flattened-block kernel (its shared-memory copy of the block
+    offsets is bounded) for the per-sample tiled one."""
+    L = si.LayerCfg(C_in=8, C_out=16, K=5, residual="none")
+    d = _draw_block(L, 2100, 16, "f16", seed=412, ragged=True, lo_frac=0.1)
+    rep = U.run_block(ctx, api, L, "f16", d.x, d.lengths, d.params[0], d.g)
+    print(f"\n2100 samples: {rep}")
+    rep.check()
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_len_one_and_full(api, ctx, dtype):
     L = si.LayerCfg(16, 16, K=9, residual="identity")
