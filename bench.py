@@ -233,6 +233,8 @@ def main():
     ap.add_argument("--dp", action="store_true",
                     help="with N > 1 ranks: data-parallel step -- every rank its own batch, per-replica batch statistics, "
                          "and an NCCL all-reduce of the gradient blob inside the step (default: independent replicas)")
+    ap.add_argument("--stream-priority", type=int, default=0,
+                    help="priority of the stream the step is captured on (0 = default, -1 = above the library's second stream)")
     ap.add_argument("--no-pdl", action="store_true", help="launch kernels without programmatic stream serialization")
     ap.add_argument("--no-overlap", action="store_true",
                     help="every kernel on one stream in program order (default: weight gradients and the residual "
@@ -326,7 +328,7 @@ def main():
         # replay it, which removes the per-launch host cost and most of the inter-kernel gaps.
         l0 = ctx.launch_count()
         graph = torch.cuda.CUDAGraph()
-        cap_stream = torch.cuda.Stream()
+        cap_stream = torch.cuda.Stream(priority=args.stream_priority)
         cap_stream.wait_stream(torch.cuda.current_stream())
         with torch.cuda.graph(graph, stream=cap_stream):
             api.encoder_fwd_bwd(ctx, spec, x_d, len_d, blob, g_d, grads_blob=grads, workspace=ws, logits=logits,
@@ -351,7 +353,7 @@ def main():
         # for context: the same K steps replayed as one captured CUDA graph (no per-launch host cost)
         try:
             graph = torch.cuda.CUDAGraph()
-            cap_stream = torch.cuda.Stream()
+            cap_stream = torch.cuda.Stream(priority=args.stream_priority)
             cap_stream.wait_stream(torch.cuda.current_stream())
             with torch.cuda.graph(graph, stream=cap_stream):
                 api.encoder_fwd_bwd(ctx, spec, x_d, len_d, blob, g_d, grads_blob=grads, workspace=ws, logits=logits,
@@ -402,7 +404,7 @@ def main():
                 q["run"] = run
             else:
                 gq = torch.cuda.CUDAGraph()
-                cs = torch.cuda.Stream()
+                cs = torch.cuda.Stream(priority=args.stream_priority)
                 cs.wait_stream(torch.cuda.current_stream())
                 with torch.cuda.graph(gq, stream=cs):
                     run(strm=cs)
