@@ -635,13 +635,17 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
     uint64_t* empty = full + STAGES;
     uint64_t* acc_full = empty + STAGES;       // [NBUF]
     uint64_t* acc_empty = acc_full + NBUF;     // [NBUF]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + NBUF);
+    // One accumulator: a tile's epilogue first reports the columns of its blocks 0 and 1 drained, then the whole
+    // accumulator.  A following tile of at most two blocks (the ragged end of a CTA's range) lives in those columns
+    // alone, so its MMAs are issued under the second half of the epilogue.
+    uint64_t* acc_half = acc_empty + NBUF;     // [NBUF], used when NBUF == 1
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_half + NBUF);
     int* s_off = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(full) + 256);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
-        for (int i = 0; i < NBUF; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 32 * EW); }
+        for (int i = 0; i < NBUF; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 32 * EW); ptx::mbar_init(&acc_half[i], 32 * EW); }
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&mapA);
         ptx::prefetch_tensormap(&mapB);
@@ -710,7 +714,15 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             uint32_t pos = u_begin;
             while (!dead && flat_next_tile<NB>(pos, u_end, nblk, m, j, nb)) {
                 const int buf = jt % NBUF;
-                if (!ptx::mbar_wait(&acc_empty[buf], ((jt / NBUF) & 1) ^ 1)) { raise_status(p.status, kErrTimeout); break; }
+                const uint32_t par_prev = ((jt / NBUF) & 1) ^ 1;      // completion of the phase the previous user of `buf` arrives on
+                bool whole_later = false;
+                if (NBUF == 1) {
+                    // every phase of both barriers is waited for, in order (a parity wait cannot tell phases two apart):
+                    // the half always here, the whole accumulator here or, for a tile of at most two blocks, after its MMAs
+                    if (!ptx::mbar_wait(&acc_half[0], par_prev)) { raise_status(p.status, kErrTimeout); break; }
+                    whole_later = nb <= 2;
+                }
+                if (!whole_later && !ptx::mbar_wait(&acc_empty[buf], par_prev)) { raise_status(p.status, kErrTimeout); break; }
                 ptx::tc_fence_after();
                 const uint32_t idesc = ptx::instr_desc(Fmt<T>::v, MODE == MODE_DGRAD ? 1u : 0u, 1u, 128, 64u * nb);
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
@@ -731,6 +743,7 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                     ptx::mma_commit(&empty[s]);
                 }
                 if (!dead) ptx::mma_commit(&acc_full[buf]);
+                if (!dead && whole_later && !ptx::mbar_wait(&acc_empty[buf], par_prev)) { raise_status(p.status, kErrTimeout); break; }
                 ++jt;
             }
         }
@@ -887,8 +900,13 @@ tc_gemm_flat_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                     else
                         store_block16<T>(stg, f, reinterpret_cast<T*>(p.out) + base, p.Tp, rl, cl, lane);
                 }
+                if (NBUF == 1 && i == 1 && nb > 2) {  // this thread is done with the columns of blocks 0 and 1
+                    ptx::tc_fence_before();
+                    ptx::mbar_arrive(&acc_half[0]);
+                }
             }
             ptx::tc_fence_before();
+            if (NBUF == 1 && nb <= 2) ptx::mbar_arrive(&acc_half[0]);
             ptx::mbar_arrive(&acc_empty[buf]);        // this thread is done reading the accumulator
             ++jt;
         }
